@@ -1,0 +1,204 @@
+/*
+ * bsr.h -- C ABI of the Block Selective Reprogramming (BSR) fine-tuning step for Vision
+ * Transformers on NVIDIA B200 (sm_100a).
+ *
+ * The calls follow the paper's statement of the method (arXiv 2405.10951, Section 4.1 and
+ * Fig. 2): a pre-trained ViT of which only chosen blocks and the classification head train,
+ * with tokens dropped at designated blocks by the classification token's attention (Eq. 6).
+ *
+ * Conventions for every function
+ *   - returns a bsr_status (0 = BSR_OK, negative = error); never throws, aborts or traps;
+ *   - "dev" pointers are device (global-memory) addresses valid on the current CUDA device,
+ *     "host" pointers are ordinary host addresses; nothing here takes a framework type;
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream);
+ *   - the library allocates no device memory: weights, optimiser state, saved activations and
+ *     scratch are carved from the single workspace block the caller hands to bsr_create, and
+ *     the caller keeps ownership of that block and of every input and output buffer;
+ *   - bsr_train_step / bsr_eval_forward only enqueue work on `stream` and do not synchronise;
+ *     results are in device memory once the stream reaches that point;
+ *   - tensors are dense row-major; linear weights are [out_features, in_features].
+ *
+ * Parameter names (bsr_set_param / bsr_get_tensor), L = dim, F = mlp_hidden:
+ *   patch_embed.weight [L, C*P*P] (input flattened as channel, row, column), patch_embed.bias [L],
+ *   cls_token [L], pos_embed [N+1, L],
+ *   blocks.<l>.norm1.weight|bias [L], blocks.<l>.attn.qkv.weight [3L, L] (rows: all Q heads, all K
+ *   heads, all V heads), blocks.<l>.attn.qkv.bias [3L], blocks.<l>.attn.proj.weight [L, L], .bias [L],
+ *   blocks.<l>.norm2.weight|bias [L], blocks.<l>.mlp.fc1.weight [F, L], .bias [F],
+ *   blocks.<l>.mlp.fc2.weight [L, F], .bias [L],
+ *   MoE blocks instead of mlp.*: blocks.<l>.moe.gate.weight [tasks, E, L], moe.fc1.weight [E, F, L],
+ *   moe.fc1.bias [E, F], moe.fc2.weight [E, L, F], moe.fc2.bias [E, L],
+ *   norm.weight|bias [L], head.<t>.weight [classes_t, L], head.<t>.bias [classes_t].
+ */
+#ifndef BSR_H_
+#define BSR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  BSR_OK = 0,
+  BSR_ERR_INVALID_ARG = -1,         /* null pointer, bad dimension, unknown name, batch > max_batch */
+  BSR_ERR_UNSUPPORTED = -2,         /* valid request this build does not implement */
+  BSR_ERR_WORKSPACE_TOO_SMALL = -3,
+  BSR_ERR_CUDA = -4,                /* a CUDA runtime/driver call failed; see bsr_last_error */
+  BSR_ERR_DEVICE_TIMEOUT = -5,      /* a bounded device-side wait gave up (reported by bsr_sync_status) */
+  BSR_ERR_NONFINITE = -6            /* loss was not finite (reported by bsr_sync_status) */
+} bsr_status;
+
+enum { BSR_DTYPE_FP32 = 0, BSR_DTYPE_BF16 = 1 };
+enum { BSR_FUSE_NONE = 0, BSR_FUSE_WEIGHTED_SUM = 1 };
+enum { BSR_MAX_DROPS = 8, BSR_MAX_TASKS = 4, BSR_MAX_DEPTH = 32 };
+
+/* Model dimensions (Section 3.1: N patches + 1 classification token, embedding length L, H heads). */
+typedef struct {
+  int32_t image_size, patch_size, in_chans;
+  int32_t dim, heads, depth, mlp_hidden;
+  int32_t num_tasks, num_classes[BSR_MAX_TASKS];
+  int32_t moe_experts, moe_top_k;   /* 0 = dense FFN everywhere */
+  uint32_t moe_block_mask;          /* bit l set: block l's FFN is an MoE layer (Section 5.2) */
+  int32_t dtype;                    /* BSR_DTYPE_*: storage type of weights and activations */
+  float ln_eps;
+} bsr_dims;
+
+/* The BSR configuration (Section 4.1, Fig. 2): which blocks train, where and how many tokens drop. */
+typedef struct {
+  bsr_dims dims;
+  uint32_t trainable_mask;          /* bit l set: block l trains; head and final LayerNorm always train */
+  int32_t n_drop;                   /* number of token drop locations */
+  int32_t drop_block[BSR_MAX_DROPS];/* 0-based block index of each location, strictly ascending */
+  int32_t keep_num[BSR_MAX_DROPS];  /* keep rate of the location = keep_num / keep_den (1 - drop rate) */
+  int32_t keep_den[BSR_MAX_DROPS];
+  int32_t fuse_mode;                /* BSR_FUSE_* */
+  float lr, beta1, beta2, eps, weight_decay;   /* AdamW (Section 5, training hyper-parameters) */
+  int32_t max_batch;
+} bsr_config;
+
+/* HBM footprint of a created handle, in bytes. */
+typedef struct {
+  uint64_t workspace_bytes;         /* whole workspace */
+  uint64_t weight_bytes;            /* weights in the storage dtype (all blocks) */
+  uint64_t master_bytes;            /* fp32 master copy of trainable parameters */
+  uint64_t optimizer_bytes;         /* AdamW first and second moments */
+  uint64_t grad_bytes;              /* fp32 gradients of trainable parameters */
+  uint64_t saved_activation_bytes;  /* activations kept for backward: trainable blocks only, at max_batch */
+  uint64_t scratch_bytes;           /* forward/backward scratch shared by all blocks */
+  uint64_t paper_activation_bytes;  /* the same blocks in the paper's fp32 accounting (Table 1), at max_batch */
+  uint64_t trainable_params;
+} bsr_footprint;
+
+typedef struct bsr_handle bsr_handle;
+
+/* Token schedule implied by a configuration (Section 4.1: K from the drop rate; Section 4.3,
+ * Discussion 3: the MHSA of a drop location sees all incoming tokens, its FFN the reduced set).
+ * Host-only.  Writes, for each block l < depth, the tokens entering its MHSA (tokens_attn[l]), the
+ * tokens entering its FFN (tokens_ffn[l]) and K (keep[l], or -1 if l is not a drop location), with
+ * K = ceil(keep_num * M / keep_den) clamped to [1, M], M = incoming tokens minus the classification
+ * token.  Arrays are host memory of `depth` int32 each, owned by the caller. */
+int32_t bsr_token_schedule(const bsr_config* cfg_host, int32_t* tokens_attn_host, int32_t* tokens_ffn_host,
+                           int32_t* keep_host);
+
+/* Size of the workspace bsr_create needs for this configuration.  Host-only. */
+int32_t bsr_workspace_bytes(const bsr_config* cfg_host, size_t* bytes_host);
+
+/* Creates the step engine (Fig. 2).  `workspace_dev` must be 256-byte aligned device memory of at
+ * least bsr_workspace_bytes() bytes and must outlive the handle.  Validates the configuration
+ * (BSR_ERR_INVALID_ARG), rejects what is not built (BSR_ERR_UNSUPPORTED: a trainable set that is not
+ * "the last k blocks"), zeroes optimiser state and sets the step counter to 0.  Parameters are
+ * undefined until set with bsr_set_param.  On failure *out_host is NULL. */
+int32_t bsr_create(const bsr_config* cfg_host, void* workspace_dev, size_t bytes, bsr_handle** out_host);
+
+int32_t bsr_destroy(bsr_handle* h);
+
+/* Static, human-readable description of the last error on this handle (or of the last failed
+ * handle-less call when h is NULL).  Never NULL; valid until the next call on the same handle. */
+const char* bsr_last_error(const bsr_handle* h);
+
+/* Loads one parameter ("pre-trained weights", Section 5).  `src_dev` holds `count` float32 values
+ * in device memory; they are converted to the storage dtype (and copied to the fp32 master for
+ * trainable tensors) on `stream`.  `count` must equal the tensor's element count. */
+int32_t bsr_set_param(bsr_handle* h, const char* name, const float* src_dev, size_t count, void* stream);
+
+/* Reads a tensor as float32 into device memory `dst_dev` (capacity `count` elements, which must
+ * equal the tensor's size) on `stream`.  Names: a parameter name (the fp32 master if it trains,
+ * else the stored weight widened), "grad/<param>", "adam_m/<param>", "adam_v/<param>" (trainable
+ * parameters only), "logits" ([max_batch, max classes], rows of the last step; classes a task does
+ * not have hold -inf), "loss" (1 element). */
+int32_t bsr_get_tensor(bsr_handle* h, const char* name, float* dst_dev, size_t count, void* stream);
+
+/* Learning rate for the next steps (the cosine schedule of Section 5 lives in the caller). */
+int32_t bsr_set_lr(bsr_handle* h, float lr);
+/* Number of optimiser steps already taken (for bias correction when resuming). */
+int32_t bsr_set_step(bsr_handle* h, int64_t steps_done);
+
+/* One BSR fine-tuning step (Fig. 2; Section 4.1; Eq. 2-5 and Eq. 8 for the backward pass): forward
+ * through the frozen blocks without saving activations, token selection and fusion at the drop
+ * locations, forward + backward of the trainable blocks and head, AdamW on their parameters.
+ *   images_dev   [batch, in_chans, image_size, image_size] in the storage dtype (fp32 or bf16 bits)
+ *   labels_dev   [batch] int32, each in [0, num_classes[task])
+ *   task_ids_dev [batch] int32, or NULL when num_tasks == 1
+ *   loss_dev_out 1 float32: mean cross-entropy of the batch before the update
+ *   kept_idx_dev_out  optional (may be NULL): int32, concatenated over drop locations i, each
+ *                [batch, K_i]: positions (0-based, among the M non-classification tokens entering
+ *                that location, ascending) of the tokens kept for each image.
+ * batch must be in [1, max_batch]. */
+int32_t bsr_train_step(bsr_handle* h, const void* images_dev, const int32_t* labels_dev,
+                       const int32_t* task_ids_dev, int32_t batch, void* stream,
+                       float* loss_dev_out, int32_t* kept_idx_dev_out);
+
+/* Inference with the same token dropping (Section 2: unlike other on-device methods the dropping
+ * also speeds up inference).  logits_dev_out: [batch, max classes] float32. */
+int32_t bsr_eval_forward(bsr_handle* h, const void* images_dev, const int32_t* task_ids_dev, int32_t batch,
+                         void* stream, float* logits_dev_out, int32_t* kept_idx_dev_out);
+
+/* Memory report (Section 3.2, Table 1: activations dominate training memory). Host-only. */
+int32_t bsr_get_footprint(const bsr_handle* h, bsr_footprint* out_host);
+
+/* Synchronises `stream` and reads the device status word: BSR_OK, BSR_ERR_DEVICE_TIMEOUT if a
+ * bounded wait in a kernel expired, BSR_ERR_NONFINITE if the last loss was not finite.  Clears it. */
+int32_t bsr_sync_status(bsr_handle* h, void* stream);
+
+/* ---- stand-alone forms of the paper-specific token kernels (no handle) ---------------------- */
+
+/* Token importance and top-K (Eq. 6; Section 4.1).  p_dev [batch, heads, m] float32: for every
+ * head the classification token's attention probabilities to the m other tokens.  Computes
+ * s[b, j] = (p[b,0,j] + ... + p[b,heads-1,j]) / heads in float32, summed in head order, and keeps
+ * the k largest per image (equal scores: lower index first).
+ *   scores_dev_out  [batch, m] float32
+ *   kept_dev_out    [batch, k] int32 ascending;  dropped_dev_out [batch, m-k] int32 ascending
+ * 1 <= k <= m <= 4096. */
+int32_t bsr_token_select(const float* p_dev, int32_t batch, int32_t heads, int32_t m, int32_t k,
+                         float* scores_dev_out, int32_t* kept_dev_out, int32_t* dropped_dev_out, void* stream);
+
+/* Compaction between MHSA and FFN (Section 4.1: kept tokens preserved, the others fused).
+ * x_dev [batch, 1+m, dim] in `dtype`; out_dev [batch, 1+k+f, dim] with f = 1 when
+ * fuse_mode == BSR_FUSE_WEIGHTED_SUM and k < m, else 0.  Row 0 is copied, rows 1..k are the kept
+ * rows in the order of kept_dev, the last row is sum_j scores[b, j] * x[b, 1+j] over dropped j
+ * (float32 accumulation in a fixed order).  dim * sizeof(dtype) must be a multiple of 16. */
+int32_t bsr_gather_fuse(const void* x_dev, int32_t dtype, int32_t batch, int32_t m, int32_t dim, int32_t k,
+                        const int32_t* kept_dev, const int32_t* dropped_dev, const float* scores_dev,
+                        int32_t fuse_mode, void* out_dev, void* stream);
+
+/* ---- stand-alone forms of the dense kernels, for unit checks against the oracle ------------- */
+
+/* y = act(x W^T + bias) + residual (FFN / projection layers of Section 3.1).  x [m, k], w [n, k],
+ * y [m, n], residual [m, n] or NULL, bias [n] float32 or NULL; x, w, y, residual in `dtype`;
+ * act_gelu != 0 applies the exact GELU.  use_tensor_cores != 0 selects the tcgen05 kernel (bf16 only). */
+int32_t bsr_linear_forward(const void* x_dev, const void* w_dev, const float* bias_dev, const void* residual_dev,
+                           void* y_dev, int32_t m, int32_t n, int32_t k, int32_t dtype, int32_t act_gelu,
+                           int32_t use_tensor_cores, void* stream);
+
+/* Multi-head self-attention, Eq. 1, on packed projections.  qkv_dev [batch, t, 3, heads, d] in
+ * `dtype`; out_dev [batch, t, heads*d]; cls_prob_dev_out optional [batch, heads, t-1] float32: the
+ * classification token's row of the attention map without its own column. d must be 64 or less
+ * and a multiple of 8. */
+int32_t bsr_attention_forward(const void* qkv_dev, int32_t dtype, int32_t batch, int32_t t, int32_t heads,
+                              int32_t d, void* out_dev, float* cls_prob_dev_out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BSR_H_ */

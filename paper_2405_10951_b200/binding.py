@@ -1,0 +1,292 @@
+"""ctypes binding of libbsr.so: the same entry points as include/bsr.h, argument marshalling only.
+
+PyTorch supplies device memory and streams; every step of the path runs in the library's
+kernels.  There is no fallback: if the library is missing, loading raises.
+"""
+
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbsr.so")
+
+BSR_OK = 0
+DTYPE_FP32, DTYPE_BF16 = 0, 1
+MAX_DROPS, MAX_TASKS, MAX_DEPTH = 8, 4, 32
+
+STATUS_NAMES = {0: "BSR_OK", -1: "BSR_ERR_INVALID_ARG", -2: "BSR_ERR_UNSUPPORTED", -3: "BSR_ERR_WORKSPACE_TOO_SMALL",
+                -4: "BSR_ERR_CUDA", -5: "BSR_ERR_DEVICE_TIMEOUT", -6: "BSR_ERR_NONFINITE"}
+
+EXPORTS = ["bsr_token_schedule", "bsr_workspace_bytes", "bsr_create", "bsr_destroy", "bsr_last_error", "bsr_set_param",
+           "bsr_get_tensor", "bsr_set_lr", "bsr_set_step", "bsr_train_step", "bsr_eval_forward", "bsr_get_footprint",
+           "bsr_sync_status", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_attention_forward"]
+
+
+class bsr_dims(C.Structure):
+    _fields_ = [("image_size", C.c_int32), ("patch_size", C.c_int32), ("in_chans", C.c_int32),
+                ("dim", C.c_int32), ("heads", C.c_int32), ("depth", C.c_int32), ("mlp_hidden", C.c_int32),
+                ("num_tasks", C.c_int32), ("num_classes", C.c_int32 * MAX_TASKS),
+                ("moe_experts", C.c_int32), ("moe_top_k", C.c_int32), ("moe_block_mask", C.c_uint32),
+                ("dtype", C.c_int32), ("ln_eps", C.c_float)]
+
+
+class bsr_config(C.Structure):
+    _fields_ = [("dims", bsr_dims), ("trainable_mask", C.c_uint32), ("n_drop", C.c_int32),
+                ("drop_block", C.c_int32 * MAX_DROPS), ("keep_num", C.c_int32 * MAX_DROPS),
+                ("keep_den", C.c_int32 * MAX_DROPS), ("fuse_mode", C.c_int32),
+                ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("weight_decay", C.c_float), ("max_batch", C.c_int32)]
+
+
+class bsr_footprint(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in ("workspace_bytes", "weight_bytes", "master_bytes", "optimizer_bytes",
+                                           "grad_bytes", "saved_activation_bytes", "scratch_bytes",
+                                           "paper_activation_bytes", "trainable_params")]
+
+
+class BsrError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libbsr.so (once).  Raises if it has not been built: there is no other path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2405_10951_b200.build` "
+                               "(nvcc, sm_100a); there is no CPU or PyTorch fallback")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, f32p, i32p = C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p
+        L.bsr_token_schedule.argtypes = [C.POINTER(bsr_config), C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        L.bsr_workspace_bytes.argtypes = [C.POINTER(bsr_config), C.POINTER(C.c_size_t)]
+        L.bsr_create.argtypes = [C.POINTER(bsr_config), vp, C.c_size_t, C.POINTER(vp)]
+        L.bsr_destroy.argtypes = [vp]
+        L.bsr_last_error.argtypes = [vp]
+        L.bsr_last_error.restype = C.c_char_p
+        L.bsr_set_param.argtypes = [vp, C.c_char_p, f32p, C.c_size_t, vp]
+        L.bsr_get_tensor.argtypes = [vp, C.c_char_p, f32p, C.c_size_t, vp]
+        L.bsr_set_lr.argtypes = [vp, C.c_float]
+        L.bsr_set_step.argtypes = [vp, C.c_int64]
+        L.bsr_train_step.argtypes = [vp, vp, i32p, i32p, i32, vp, f32p, i32p]
+        L.bsr_eval_forward.argtypes = [vp, vp, i32p, i32, vp, f32p, i32p]
+        L.bsr_get_footprint.argtypes = [vp, C.POINTER(bsr_footprint)]
+        L.bsr_sync_status.argtypes = [vp, vp]
+        L.bsr_token_select.argtypes = [f32p, i32, i32, i32, i32, f32p, i32p, i32p, vp]
+        L.bsr_gather_fuse.argtypes = [vp, i32, i32, i32, i32, i32, i32p, i32p, f32p, i32, vp, vp]
+        L.bsr_linear_forward.argtypes = [vp, vp, f32p, vp, vp, i32, i32, i32, i32, i32, i32, vp]
+        L.bsr_attention_forward.argtypes = [vp, i32, i32, i32, i32, i32, vp, f32p, vp]
+        for name in EXPORTS:
+            if name != "bsr_last_error":
+                getattr(L, name).restype = C.c_int32
+        _lib = L
+    return _lib
+
+
+def _check(status: int, handle=None):
+    if status != BSR_OK:
+        msg = lib().bsr_last_error(handle)
+        raise BsrError(status, msg.decode() if msg else "")
+
+
+def make_config(cfg, max_batch: Optional[int] = None) -> bsr_config:
+    """Translates a synth.Config-like object (attributes only) into the C struct."""
+    c = bsr_config()
+    d = c.dims
+    d.image_size, d.patch_size, d.in_chans = cfg.image_size, cfg.patch_size, cfg.in_chans
+    d.dim, d.heads, d.depth, d.mlp_hidden = cfg.dim, cfg.heads, cfg.depth, cfg.mlp_hidden
+    d.num_tasks = len(cfg.num_classes)
+    for i, n in enumerate(cfg.num_classes):
+        d.num_classes[i] = n
+    d.moe_experts, d.moe_top_k = cfg.moe_experts, cfg.moe_top_k
+    d.moe_block_mask = sum(1 << l for l in cfg.moe_blocks)
+    d.dtype = DTYPE_FP32 if cfg.dtype == "fp32" else DTYPE_BF16
+    d.ln_eps = cfg.ln_eps
+    c.trainable_mask = sum(1 << l for l in cfg.trainable)
+    c.n_drop = len(cfg.drop_blocks)
+    for i, l in enumerate(cfg.drop_blocks):
+        c.drop_block[i], c.keep_num[i], c.keep_den[i] = l, cfg.keep_num, cfg.keep_den
+    c.fuse_mode = cfg.fuse_mode
+    c.lr, c.beta1, c.beta2, c.eps, c.weight_decay = cfg.lr, cfg.beta1, cfg.beta2, cfg.eps, cfg.weight_decay
+    c.max_batch = cfg.batch if max_batch is None else max_batch
+    return c
+
+
+# ---- host-only calls ---------------------------------------------------------------------------
+def bsr_token_schedule(c: bsr_config):
+    n = c.dims.depth
+    ta, tf, k = (C.c_int32 * MAX_DEPTH)(), (C.c_int32 * MAX_DEPTH)(), (C.c_int32 * MAX_DEPTH)()
+    _check(lib().bsr_token_schedule(C.byref(c), ta, tf, k))
+    return list(ta[:max(n, 0)]), list(tf[:max(n, 0)]), list(k[:max(n, 0)])
+
+
+def bsr_workspace_bytes(c: bsr_config) -> int:
+    out = C.c_size_t(0)
+    _check(lib().bsr_workspace_bytes(C.byref(c), C.byref(out)))
+    return out.value
+
+
+# ---- device calls (torch tensors give pointers and the current stream) --------------------------
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def bsr_token_select(p, k: int):
+    """p: float32 CUDA tensor [B, H, M].  Returns (scores [B, M], kept [B, k], dropped [B, M-k])."""
+    import torch
+    B, H, M = p.shape
+    scores = torch.empty((B, M), dtype=torch.float32, device=p.device)
+    kept = torch.empty((B, k), dtype=torch.int32, device=p.device)
+    dropped = torch.empty((B, M - k), dtype=torch.int32, device=p.device)
+    _check(lib().bsr_token_select(_ptr(p), B, H, M, k, _ptr(scores), _ptr(kept), _ptr(dropped), _stream()))
+    return scores, kept, dropped
+
+
+def bsr_gather_fuse(x, kept, dropped, scores, fuse_mode: int = 1, out=None):
+    import torch
+    B, T, D = x.shape
+    M, k = T - 1, kept.shape[1]
+    f = 1 if (fuse_mode == 1 and k < M) else 0
+    if out is None:
+        out = torch.empty((B, 1 + k + f, D), dtype=x.dtype, device=x.device)
+    dt = DTYPE_FP32 if x.dtype == torch.float32 else DTYPE_BF16
+    _check(lib().bsr_gather_fuse(_ptr(x), dt, B, M, D, k, _ptr(kept), _ptr(dropped), _ptr(scores), fuse_mode, _ptr(out), _stream()))
+    return out
+
+
+def bsr_linear_forward(x, w, bias=None, residual=None, act_gelu: bool = False, use_tensor_cores: bool = False):
+    import torch
+    m, k = x.shape
+    n = w.shape[0]
+    y = torch.empty((m, n), dtype=x.dtype, device=x.device)
+    dt = DTYPE_FP32 if x.dtype == torch.float32 else DTYPE_BF16
+    _check(lib().bsr_linear_forward(_ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(y), m, n, k, dt, int(act_gelu),
+                                    int(use_tensor_cores), _stream()))
+    return y
+
+
+def bsr_attention_forward(qkv, heads: int, want_cls_prob: bool = True):
+    """qkv: CUDA tensor [B, T, 3, H, d].  Returns (out [B, T, H*d], cls_prob [B, H, T-1] or None)."""
+    import torch
+    B, T, three, H, d = qkv.shape
+    assert three == 3 and H == heads
+    out = torch.empty((B, T, H * d), dtype=qkv.dtype, device=qkv.device)
+    cp = torch.empty((B, H, T - 1), dtype=torch.float32, device=qkv.device) if want_cls_prob else None
+    dt = DTYPE_FP32 if qkv.dtype == torch.float32 else DTYPE_BF16
+    _check(lib().bsr_attention_forward(_ptr(qkv), dt, B, T, H, d, _ptr(out), _ptr(cp), _stream()))
+    return out, cp
+
+
+class Engine:
+    """Owns a handle and its workspace tensor; thin convenience over the bsr_* calls."""
+
+    def __init__(self, cfg, max_batch: Optional[int] = None, device: str = "cuda:0"):
+        import torch
+        self.torch = torch
+        self.cfg = cfg
+        self.device = torch.device(device)
+        self.c = make_config(cfg, max_batch)
+        self.ta, self.tf, self.k = bsr_token_schedule(self.c)
+        nbytes = bsr_workspace_bytes(self.c)
+        torch.cuda.set_device(self.device)
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        base = self.workspace.data_ptr()
+        self._ws_ptr = (base + 255) & ~255
+        h = C.c_void_p()
+        _check(lib().bsr_create(C.byref(self.c), C.c_void_p(self._ws_ptr), nbytes, C.byref(h)))
+        self.h = h
+        self.cmax = max(cfg.num_classes)
+        self.storage_dtype = torch.float32 if cfg.dtype == "fp32" else torch.bfloat16
+        self.kept_counts = [k for k in self.k if k >= 0]
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib().bsr_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- parameters --
+    def set_param(self, name: str, value):
+        t = self.torch.as_tensor(np.ascontiguousarray(value, dtype=np.float32)).to(self.device) \
+            if not self.torch.is_tensor(value) else value.to(self.device, self.torch.float32).contiguous()
+        _check(lib().bsr_set_param(self.h, name.encode(), _ptr(t), t.numel(), _stream()), self.h)
+        self.torch.cuda.current_stream().synchronize()
+
+    def set_params(self, params: Dict[str, np.ndarray]):
+        for name, v in params.items():
+            self.set_param(name, v)
+
+    def get_tensor(self, name: str, shape: Sequence[int]):
+        n = int(np.prod(shape))
+        out = self.torch.empty(n, dtype=self.torch.float32, device=self.device)
+        _check(lib().bsr_get_tensor(self.h, name.encode(), _ptr(out), n, _stream()), self.h)
+        return out.reshape(tuple(shape))
+
+    def set_lr(self, lr: float):
+        _check(lib().bsr_set_lr(self.h, lr), self.h)
+
+    def set_step(self, n: int):
+        _check(lib().bsr_set_step(self.h, n), self.h)
+
+    # -- the step --
+    def images_to_device(self, images: np.ndarray):
+        t = self.torch.as_tensor(np.ascontiguousarray(images, dtype=np.float32))
+        return t.to(self.device).to(self.storage_dtype).contiguous()
+
+    def train_step(self, images, labels, task_ids=None, want_kept: bool = True):
+        """images: CUDA tensor [B, C, S, S] in the storage dtype; labels/task_ids: int32 CUDA tensors.
+        Returns (loss tensor [1], list of kept-index tensors [B, K_i] or None).  Does not synchronise."""
+        torch = self.torch
+        B = images.shape[0]
+        loss = torch.empty(1, dtype=torch.float32, device=self.device)
+        kept = None
+        if want_kept and self.kept_counts:
+            kept = torch.empty(B * sum(self.kept_counts), dtype=torch.int32, device=self.device)
+        _check(lib().bsr_train_step(self.h, _ptr(images), _ptr(labels), _ptr(task_ids), B, _stream(), _ptr(loss), _ptr(kept)), self.h)
+        return loss, self._split_kept(kept, B)
+
+    def eval_forward(self, images, task_ids=None, want_kept: bool = True):
+        torch = self.torch
+        B = images.shape[0]
+        logits = torch.empty((B, self.cmax), dtype=torch.float32, device=self.device)
+        kept = None
+        if want_kept and self.kept_counts:
+            kept = torch.empty(B * sum(self.kept_counts), dtype=torch.int32, device=self.device)
+        _check(lib().bsr_eval_forward(self.h, _ptr(images), _ptr(task_ids), B, _stream(), _ptr(logits), _ptr(kept)), self.h)
+        return logits, self._split_kept(kept, B)
+
+    def _split_kept(self, kept, B):
+        if kept is None:
+            return None
+        out, off = [], 0
+        for k in self.kept_counts:
+            out.append(kept[off: off + B * k].view(B, k))
+            off += B * k
+        return out
+
+    def sync_status(self):
+        _check(lib().bsr_sync_status(self.h, _stream()), self.h)
+
+    def footprint(self) -> Dict[str, int]:
+        fp = bsr_footprint()
+        _check(lib().bsr_get_footprint(self.h, C.byref(fp)), self.h)
+        return {n: int(getattr(fp, n)) for n, _ in bsr_footprint._fields_}

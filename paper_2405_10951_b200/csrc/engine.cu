@@ -1,0 +1,875 @@
+// Step engine and C ABI of the BSR fine-tuning step (see include/bsr.h for the contract).
+//
+// The engine carves one caller-owned workspace into: parameters in the storage dtype, fp32 master /
+// gradient / AdamW moments of the trainable parameters (flat arrays), the activations the trainable
+// blocks keep for their backward pass, and scratch shared by all blocks.  Frozen blocks write nothing
+// that outlives them (paper Fig. 2: gradient propagation stops at the earliest trainable block).
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <vector>
+
+#include "../../include/bsr.h"
+#include "common.cuh"
+#include "kernels.h"
+
+using namespace bsr;
+
+namespace {
+
+thread_local char g_error[256] = "no error";
+
+struct Schedule {
+  int ta[BSR_MAX_DEPTH], tf[BSR_MAX_DEPTH], k[BSR_MAX_DEPTH];
+};
+
+struct Tensor {
+  std::string name;
+  size_t numel = 0;
+  bool matrix = false;      // stored in the storage dtype; vectors (biases, LayerNorm, cls, pos) stay float
+  bool trainable = false;
+  bool decay = false;
+  size_t w_off = 0;         // byte offset of the stored copy (for trainable float tensors: inside master)
+  size_t flat = 0;          // element offset in the flat trainable arrays
+};
+
+struct BlockBufs {          // byte offsets into the workspace; filled for frozen (scratch) and trainable (arena) blocks
+  size_t x_in, y1, qkv, o, xp_full, xp, y2, z, hh, x_out;
+  size_t mean1, rstd1, lse, mean2, rstd2, p, s, kept, dropped;
+};
+
+struct Bump {
+  size_t off = 0;
+  size_t take(size_t bytes) {
+    size_t o = off;
+    off += (bytes + 255) & ~(size_t)255;
+    return o;
+  }
+};
+
+int set_err(char* buf, int code, const char* fmt, ...) __attribute__((format(printf, 3, 4)));
+int set_err(char* buf, int code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, 256, fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+int compute_schedule(const bsr_config* cfg, Schedule* s, char* err) {
+  const bsr_dims& d = cfg->dims;
+  if (d.patch_size <= 0 || d.image_size <= 0 || d.image_size % d.patch_size != 0)
+    return set_err(err, BSR_ERR_INVALID_ARG, "image_size must be a positive multiple of patch_size");
+  if (d.depth < 1 || d.depth > BSR_MAX_DEPTH) return set_err(err, BSR_ERR_INVALID_ARG, "depth must be in [1, %d]", BSR_MAX_DEPTH);
+  if (cfg->n_drop < 0 || cfg->n_drop > BSR_MAX_DROPS) return set_err(err, BSR_ERR_INVALID_ARG, "n_drop must be in [0, %d]", BSR_MAX_DROPS);
+  int g = d.image_size / d.patch_size;
+  int t = g * g + 1;
+  int di = 0;
+  for (int i = 0; i < cfg->n_drop; ++i) {
+    if (cfg->drop_block[i] < 0 || cfg->drop_block[i] >= d.depth || (i > 0 && cfg->drop_block[i] <= cfg->drop_block[i - 1]))
+      return set_err(err, BSR_ERR_INVALID_ARG, "drop_block must be strictly ascending block indices");
+    if (cfg->keep_den[i] <= 0 || cfg->keep_num[i] <= 0 || cfg->keep_num[i] > cfg->keep_den[i])
+      return set_err(err, BSR_ERR_INVALID_ARG, "keep rate must satisfy 0 < keep_num <= keep_den");
+  }
+  for (int l = 0; l < d.depth; ++l) {
+    s->ta[l] = t;
+    s->k[l] = -1;
+    if (di < cfg->n_drop && cfg->drop_block[di] == l) {
+      long m = t - 1;
+      long k = ((long)cfg->keep_num[di] * m + cfg->keep_den[di] - 1) / cfg->keep_den[di];   // ceil(keep * M)
+      if (k < 1) k = 1;
+      if (k > m) k = m;
+      s->k[l] = (int)k;
+      if (k < m) t = 1 + (int)k + (cfg->fuse_mode == BSR_FUSE_WEIGHTED_SUM ? 1 : 0);
+      ++di;
+    }
+    s->tf[l] = t;
+  }
+  return BSR_OK;
+}
+
+int validate(const bsr_config* cfg, char* err) {
+  if (cfg == nullptr) return set_err(err, BSR_ERR_INVALID_ARG, "config is null");
+  const bsr_dims& d = cfg->dims;
+  if (d.dtype != BSR_DTYPE_FP32 && d.dtype != BSR_DTYPE_BF16) return set_err(err, BSR_ERR_INVALID_ARG, "dtype must be fp32 (0) or bf16 (1)");
+  if (d.in_chans < 1 || d.dim < 8 || d.heads < 1 || d.mlp_hidden < 8) return set_err(err, BSR_ERR_INVALID_ARG, "bad model dimension");
+  if (d.dim % d.heads != 0) return set_err(err, BSR_ERR_INVALID_ARG, "dim must be a multiple of heads");
+  if (d.dim % 8 != 0 || d.mlp_hidden % 8 != 0 || d.dim > 1024) return set_err(err, BSR_ERR_INVALID_ARG, "dim and mlp_hidden must be multiples of 8, dim <= 1024");
+  int hd = d.dim / d.heads;
+  if (hd > 64 || hd % 8 != 0) return set_err(err, BSR_ERR_INVALID_ARG, "head dimension must be a multiple of 8, at most 64");
+  if (d.num_tasks < 1 || d.num_tasks > BSR_MAX_TASKS) return set_err(err, BSR_ERR_INVALID_ARG, "num_tasks must be in [1, %d]", BSR_MAX_TASKS);
+  for (int t = 0; t < d.num_tasks; ++t)
+    if (d.num_classes[t] < 1) return set_err(err, BSR_ERR_INVALID_ARG, "num_classes must be positive");
+  if (cfg->max_batch < 1) return set_err(err, BSR_ERR_INVALID_ARG, "max_batch must be positive");
+  if (cfg->fuse_mode != BSR_FUSE_NONE && cfg->fuse_mode != BSR_FUSE_WEIGHTED_SUM) return set_err(err, BSR_ERR_INVALID_ARG, "unknown fuse_mode");
+  if (!(d.ln_eps > 0.f)) return set_err(err, BSR_ERR_INVALID_ARG, "ln_eps must be positive");
+  Schedule s;
+  int rc = compute_schedule(cfg, &s, err);
+  if (rc != BSR_OK) return rc;
+  if (d.depth < 32 && (cfg->trainable_mask >> d.depth) != 0) return set_err(err, BSR_ERR_INVALID_ARG, "trainable_mask names a block beyond depth");
+  if (d.moe_experts != 0 || d.moe_block_mask != 0) return set_err(err, BSR_ERR_UNSUPPORTED, "MoE layers are not built yet");
+  // trainable set must be "the last k blocks"
+  uint32_t m = cfg->trainable_mask;
+  if (m != 0) {
+    int t0 = __builtin_ctz(m);
+    uint32_t suffix = (d.depth >= 32 ? 0xffffffffu : ((1u << d.depth) - 1u)) & ~((1u << t0) - 1u);
+    if (m != suffix) return set_err(err, BSR_ERR_UNSUPPORTED, "trainable blocks must be the last k blocks (frozen blocks inside the gradient path are not built yet)");
+  }
+  return BSR_OK;
+}
+
+}  // namespace
+
+struct bsr_handle {
+  bsr_config cfg;
+  Schedule sched;
+  char* base = nullptr;
+  size_t bytes = 0;
+  char err[256];
+  int sm_count = 148;
+  int use_tc = 1;
+  int64_t step = 0;
+  float lr = 0.f;
+  int t0 = 0;                        // earliest trainable block (depth if none)
+  std::vector<Tensor> tensors;
+  std::map<std::string, int> index;
+  size_t n_flat = 0;                 // elements in the flat trainable arrays
+  size_t off_status = 0, off_loss = 0;
+  size_t off_weights = 0, weights_bytes = 0;
+  size_t off_frozen_vec = 0;
+  size_t off_master = 0, off_grad = 0, off_m = 0, off_v = 0;
+  size_t off_chunks = 0;
+  int n_chunks = 0;
+  std::vector<BlockBufs> bufs_train;  // per block (valid for l >= t0)
+  BlockBufs bufs_frozen[2];           // ping-pong by block parity
+  size_t off_x_last = 0;
+  size_t arena_bytes = 0, scratch_bytes = 0;
+  // scratch
+  size_t off_patches = 0, off_emb = 0;
+  size_t off_xn = 0, off_meanf = 0, off_rstdf = 0, off_logits = 0, off_per_image = 0, off_dlogits = 0, off_dxn = 0;
+  size_t off_dxa = 0, off_dxb = 0, off_dz = 0, off_dy = 0, off_dxg = 0, off_dxp = 0, off_do = 0, off_dqkv = 0;
+  size_t off_escore = 0, off_delta = 0, off_ln_partials = 0, off_cs_partials = 0;
+  size_t off_kept_all = 0;
+  size_t off_stage = 0;
+
+  template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(base + off); }
+  void* w(const char* name) const {
+    auto it = index.find(name);
+    return it == index.end() ? nullptr : base + tensors[it->second].w_off;
+  }
+  void* wb(int l, const char* suffix) const { return w(("blocks." + std::to_string(l) + "." + suffix).c_str()); }
+  float* gradp(const std::string& name) const {
+    auto it = index.find(name);
+    return at<float>(off_grad) + tensors[it->second].flat;
+  }
+  float* gb(int l, const char* suffix) const { return gradp("blocks." + std::to_string(l) + "." + suffix); }
+};
+
+namespace {
+
+void build_tensors(bsr_handle* h) {
+  const bsr_dims& d = h->cfg.dims;
+  int D = d.dim, F = d.mlp_hidden;
+  int g = d.image_size / d.patch_size;
+  auto add = [&](const std::string& name, size_t numel, bool matrix, bool trainable) {
+    Tensor t;
+    t.name = name; t.numel = numel; t.matrix = matrix; t.trainable = trainable;
+    t.decay = name.size() >= 6 && name.compare(name.size() - 6, 6, "weight") == 0 && name.find("norm") == std::string::npos;
+    h->index[name] = (int)h->tensors.size();
+    h->tensors.push_back(t);
+  };
+  add("patch_embed.weight", (size_t)D * d.in_chans * d.patch_size * d.patch_size, true, false);
+  add("patch_embed.bias", D, false, false);
+  add("cls_token", D, false, false);
+  add("pos_embed", (size_t)(g * g + 1) * D, false, false);
+  for (int l = 0; l < d.depth; ++l) {
+    bool tr = (h->cfg.trainable_mask >> l) & 1u;
+    std::string p = "blocks." + std::to_string(l) + ".";
+    add(p + "norm1.weight", D, false, tr);
+    add(p + "norm1.bias", D, false, tr);
+    add(p + "attn.qkv.weight", (size_t)3 * D * D, true, tr);
+    add(p + "attn.qkv.bias", 3 * D, false, tr);
+    add(p + "attn.proj.weight", (size_t)D * D, true, tr);
+    add(p + "attn.proj.bias", D, false, tr);
+    add(p + "norm2.weight", D, false, tr);
+    add(p + "norm2.bias", D, false, tr);
+    add(p + "mlp.fc1.weight", (size_t)F * D, true, tr);
+    add(p + "mlp.fc1.bias", F, false, tr);
+    add(p + "mlp.fc2.weight", (size_t)D * F, true, tr);
+    add(p + "mlp.fc2.bias", D, false, tr);
+  }
+  add("norm.weight", D, false, true);
+  add("norm.bias", D, false, true);
+  for (int t = 0; t < d.num_tasks; ++t) {
+    add("head." + std::to_string(t) + ".weight", (size_t)d.num_classes[t] * D, true, true);
+    add("head." + std::to_string(t) + ".bias", d.num_classes[t], false, true);
+  }
+}
+
+constexpr uint32_t ADAM_CHUNK = 4096;
+
+// Lays the workspace out; identical for sizing (base == nullptr) and for creation.
+size_t plan(bsr_handle* h) {
+  const bsr_config& cfg = h->cfg;
+  const bsr_dims& d = cfg.dims;
+  const Schedule& s = h->sched;
+  size_t es = dtype_size(d.dtype);
+  int D = d.dim, F = d.mlp_hidden, H = d.heads, Bm = cfg.max_batch;
+  int g = d.image_size / d.patch_size, N = g * g, T0 = N + 1;
+  int cmax = 0;
+  for (int t = 0; t < d.num_tasks; ++t) cmax = d.num_classes[t] > cmax ? d.num_classes[t] : cmax;
+  Bump b;
+  h->off_status = b.take(256);
+  h->off_loss = h->off_status + 64;
+  // flat trainable arrays
+  size_t flat = 0;
+  for (auto& t : h->tensors)
+    if (t.trainable) { t.flat = flat; flat += (t.numel + 63) & ~(size_t)63; }
+  h->n_flat = flat;
+  h->off_master = b.take(flat * 4);
+  h->off_grad = b.take(flat * 4);
+  h->off_m = b.take(flat * 4);
+  h->off_v = b.take(flat * 4);
+  // stored copies
+  size_t w0 = b.off;
+  for (auto& t : h->tensors) {
+    bool alias_master = t.trainable && (!t.matrix || d.dtype == BSR_DTYPE_FP32);
+    if (alias_master) t.w_off = h->off_master + t.flat * 4;
+    else t.w_off = b.take(t.numel * (t.matrix ? es : 4));
+  }
+  h->off_weights = w0;
+  h->weights_bytes = b.off - w0;
+  // AdamW chunk table
+  int nch = 0;
+  for (auto& t : h->tensors)
+    if (t.trainable) nch += (int)((t.numel + ADAM_CHUNK - 1) / ADAM_CHUNK);
+  h->n_chunks = nch;
+  h->off_chunks = b.take((size_t)nch * sizeof(AdamChunk));
+  // activations kept by the trainable blocks
+  size_t a0 = b.off;
+  h->bufs_train.assign(d.depth, BlockBufs());
+  h->t0 = cfg.trainable_mask ? __builtin_ctz(cfg.trainable_mask) : d.depth;
+  size_t next_in = 0;
+  for (int l = h->t0; l < d.depth; ++l) {
+    BlockBufs& bb = h->bufs_train[l];
+    size_t Ma = (size_t)Bm * s.ta[l], Mf = (size_t)Bm * s.tf[l];
+    bool drop = s.k[l] >= 0 && s.tf[l] != s.ta[l];
+    bb.x_in = (l == h->t0) ? b.take(Ma * D * es) : next_in;
+    bb.mean1 = b.take(Ma * 4); bb.rstd1 = b.take(Ma * 4);
+    bb.y1 = b.take(Ma * D * es);
+    bb.qkv = b.take(Ma * 3 * D * es);
+    bb.lse = b.take((size_t)Bm * H * s.ta[l] * 4);
+    bb.o = b.take(Ma * D * es);
+    bb.xp = b.take(Mf * D * es);
+    bb.xp_full = drop ? b.take(Ma * D * es) : bb.xp;
+    if (s.k[l] >= 0) {
+      bb.p = b.take((size_t)Bm * H * (s.ta[l] - 1) * 4);
+      bb.s = b.take((size_t)Bm * (s.ta[l] - 1) * 4);
+      bb.kept = b.take((size_t)Bm * (s.ta[l] - 1) * 4);
+      bb.dropped = b.take((size_t)Bm * (s.ta[l] - 1) * 4);
+    }
+    bb.mean2 = b.take(Mf * 4); bb.rstd2 = b.take(Mf * 4);
+    bb.y2 = b.take(Mf * D * es);
+    bb.z = b.take(Mf * F * es);
+    bb.hh = b.take(Mf * F * es);
+    bb.x_out = b.take(Mf * D * es);
+    next_in = bb.x_out;
+  }
+  h->arena_bytes = b.off - a0;
+  // scratch
+  size_t s0 = b.off;
+  size_t M0 = (size_t)Bm * T0;
+  h->off_patches = b.take((size_t)Bm * N * d.in_chans * d.patch_size * d.patch_size * es);
+  h->off_emb = b.take((size_t)Bm * N * D * es);
+  size_t xa = b.take(M0 * D * es), xb = b.take(M0 * D * es);
+  for (int i = 0; i < 2; ++i) {
+    BlockBufs& bb = h->bufs_frozen[i];
+    bb.x_in = i == 0 ? xa : xb;
+    bb.x_out = i == 0 ? xb : xa;
+  }
+  {
+    BlockBufs& bb = h->bufs_frozen[0];
+    bb.mean1 = bb.rstd1 = bb.mean2 = bb.rstd2 = bb.lse = 0;
+    bb.y1 = b.take(M0 * D * es);
+    bb.qkv = b.take(M0 * 3 * D * es);
+    bb.o = b.take(M0 * D * es);
+    bb.xp_full = b.take(M0 * D * es);
+    bb.xp = b.take(M0 * D * es);
+    bb.y2 = bb.y1;
+    bb.z = 0;
+    bb.hh = b.take(M0 * F * es);
+    bb.p = b.take((size_t)Bm * H * (T0 - 1) * 4);
+    bb.s = b.take((size_t)Bm * (T0 - 1) * 4);
+    bb.kept = b.take((size_t)Bm * (T0 - 1) * 4);
+    bb.dropped = b.take((size_t)Bm * (T0 - 1) * 4);
+    size_t in1 = h->bufs_frozen[1].x_in, out1 = h->bufs_frozen[1].x_out;
+    h->bufs_frozen[1] = bb;
+    h->bufs_frozen[1].x_in = in1;
+    h->bufs_frozen[1].x_out = out1;
+  }
+  h->off_xn = b.take((size_t)Bm * D * 4);
+  h->off_meanf = b.take((size_t)Bm * 4);
+  h->off_rstdf = b.take((size_t)Bm * 4);
+  h->off_logits = b.take((size_t)Bm * cmax * 4);
+  h->off_per_image = b.take((size_t)Bm * 4);
+  h->off_dlogits = b.take((size_t)Bm * cmax * 4);
+  h->off_dxn = b.take((size_t)Bm * D * 4);
+  size_t kept_total = 0;
+  for (int l = 0; l < d.depth; ++l)
+    if (s.k[l] >= 0) kept_total += (size_t)Bm * s.k[l];
+  h->off_kept_all = b.take((kept_total + 1) * 4);
+  if (h->t0 < d.depth) {
+    size_t Mt = (size_t)Bm * s.ta[h->t0];
+    h->off_dxa = b.take(Mt * D * es);
+    h->off_dxb = b.take(Mt * D * es);
+    h->off_dz = b.take(Mt * F * es);
+    h->off_dy = b.take(Mt * D * es);
+    h->off_dxg = b.take(Mt * D * es);
+    h->off_dxp = b.take(Mt * D * es);
+    h->off_do = b.take(Mt * D * es);
+    h->off_dqkv = b.take(Mt * 3 * D * es);
+    h->off_escore = b.take((size_t)Bm * s.ta[h->t0] * 4);
+    h->off_delta = b.take((size_t)Bm * H * s.ta[h->t0] * 4);
+  }
+  int maxn = 3 * D > F ? 3 * D : F;
+  h->off_ln_partials = b.take((size_t)2 * 512 * D * 4);
+  h->off_cs_partials = b.take((size_t)64 * maxn * 4);
+  size_t biggest = 0;
+  for (auto& t : h->tensors) biggest = t.numel > biggest ? t.numel : biggest;
+  h->off_stage = b.take(biggest * 4);
+  h->scratch_bytes = b.off - s0;
+  return b.off;
+}
+
+Ctx make_ctx(const bsr_handle* h, void* stream) {
+  Ctx c;
+  c.stream = (cudaStream_t)stream;
+  c.dtype = h->cfg.dims.dtype;
+  c.status = h->at<int>(h->off_status);
+  c.sm_count = h->sm_count;
+  c.use_tc = h->use_tc;
+  return c;
+}
+
+int check_cuda(bsr_handle* h, const char* what) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return set_err(h ? h->err : g_error, BSR_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+  return BSR_OK;
+}
+
+// One encoder block forward.  `save` keeps the statistics and pre-activations the backward pass needs.
+int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb, bool save, int* kept_out) {
+  const bsr_dims& d = h->cfg.dims;
+  const Schedule& s = h->sched;
+  int D = d.dim, F = d.mlp_hidden, H = d.heads, hd = D / H;
+  int Ta = s.ta[l], Tf = s.tf[l], k = s.k[l];
+  int Ma = B * Ta, Mf = B * Tf;
+  bool is_drop = k >= 0;
+  bool shrinks = is_drop && Tf != Ta;
+  layernorm_fwd(c, h->base + bb.x_in, D, (const float*)h->wb(l, "norm1.weight"), (const float*)h->wb(l, "norm1.bias"),
+                h->base + bb.y1, 0, save ? h->at<float>(bb.mean1) : nullptr, save ? h->at<float>(bb.rstd1) : nullptr, Ma, D, d.ln_eps);
+  GemmEpilogue e1;
+  e1.bias = (const float*)h->wb(l, "attn.qkv.bias");
+  gemm(c, h->base + bb.y1, D, 1, h->wb(l, "attn.qkv.weight"), D, 1, h->base + bb.qkv, 0, Ma, 3 * D, D, e1);
+  int rc = attention_fwd(c, h->base + bb.qkv, h->base + bb.o, save ? h->at<float>(bb.lse) : nullptr,
+                         is_drop ? h->at<float>(bb.p) : nullptr, B, Ta, H, hd);
+  if (rc != 0) return set_err(h->err, BSR_ERR_UNSUPPORTED, "attention: %d tokens of head dimension %d do not fit this kernel", Ta, hd);
+  GemmEpilogue e2;
+  e2.bias = (const float*)h->wb(l, "attn.proj.bias");
+  e2.residual = h->base + bb.x_in;
+  void* xp_dst = h->base + (shrinks ? bb.xp_full : bb.xp);
+  gemm(c, h->base + bb.o, D, 1, h->wb(l, "attn.proj.weight"), D, 1, xp_dst, 0, Ma, D, D, e2);
+  if (is_drop) {
+    int M = Ta - 1;
+    token_select(c.stream, h->at<float>(bb.p), B, H, M, k, h->at<float>(bb.s), h->at<int>(bb.kept), h->at<int>(bb.dropped));
+    if (kept_out != nullptr)
+      cudaMemcpyAsync(kept_out, h->base + bb.kept, (size_t)B * k * sizeof(int), cudaMemcpyDeviceToDevice, c.stream);
+    if (shrinks)
+      gather_fuse(c, h->base + bb.xp_full, B, M, D, k, h->at<int>(bb.kept), h->at<int>(bb.dropped), h->at<float>(bb.s),
+                  h->cfg.fuse_mode, h->base + bb.xp);
+  }
+  layernorm_fwd(c, h->base + bb.xp, D, (const float*)h->wb(l, "norm2.weight"), (const float*)h->wb(l, "norm2.bias"),
+                h->base + bb.y2, 0, save ? h->at<float>(bb.mean2) : nullptr, save ? h->at<float>(bb.rstd2) : nullptr, Mf, D, d.ln_eps);
+  GemmEpilogue e3;
+  e3.bias = (const float*)h->wb(l, "mlp.fc1.bias");
+  e3.act = 1;
+  e3.aux_out = save ? h->base + bb.z : nullptr;
+  gemm(c, h->base + bb.y2, D, 1, h->wb(l, "mlp.fc1.weight"), D, 1, h->base + bb.hh, 0, Mf, F, D, e3);
+  GemmEpilogue e4;
+  e4.bias = (const float*)h->wb(l, "mlp.fc2.bias");
+  e4.residual = h->base + bb.xp;
+  gemm(c, h->base + bb.hh, F, 1, h->wb(l, "mlp.fc2.weight"), F, 1, h->base + bb.x_out, 0, Mf, D, F, e4);
+  return BSR_OK;
+}
+
+// Backward of one trainable block (Eq. 2-5).  dxo: gradient at the block output [B*Tf, D]; dxi receives the
+// gradient at the block input unless it is null (earliest trainable block: Eq. 8, nothing flows further).
+int block_backward(bsr_handle* h, const Ctx& c, int l, int B, void* dxo, void* dxi) {
+  const bsr_dims& d = h->cfg.dims;
+  const Schedule& s = h->sched;
+  const BlockBufs& bb = h->bufs_train[l];
+  int D = d.dim, F = d.mlp_hidden, H = d.heads, hd = D / H;
+  int Ta = s.ta[l], Tf = s.tf[l], k = s.k[l];
+  int Ma = B * Ta, Mf = B * Tf;
+  bool shrinks = k >= 0 && Tf != Ta;
+  float* csp = h->at<float>(h->off_cs_partials);
+  float* lnp = h->at<float>(h->off_ln_partials);
+  void* dz = h->base + h->off_dz;
+  void* dy = h->base + h->off_dy;
+  void* dxg = h->base + h->off_dxg;
+  void* dxp = shrinks ? (void*)(h->base + h->off_dxp) : dxg;
+  void* d_o = h->base + h->off_do;
+  void* dqkv = h->base + h->off_dqkv;
+  GemmEpilogue none;
+  // FFN second layer: dz = (dxo W2) * GELU'(z); dW2 = dxo^T h; db2 = column sums of dxo
+  GemmEpilogue eg;
+  eg.act = 2;
+  eg.aux_in = h->base + bb.z;
+  gemm(c, dxo, D, 1, h->wb(l, "mlp.fc2.weight"), 1, F, dz, 0, Mf, F, D, eg);
+  gemm(c, dxo, 1, D, h->base + bb.hh, 1, F, h->gb(l, "mlp.fc2.weight"), 1, D, F, Mf, none);
+  colsum(c, dxo, Mf, D, csp, h->gb(l, "mlp.fc2.bias"));
+  // FFN first layer
+  gemm(c, dz, F, 1, h->wb(l, "mlp.fc1.weight"), 1, D, dy, 0, Mf, D, F, none);
+  gemm(c, dz, 1, F, h->base + bb.y2, 1, D, h->gb(l, "mlp.fc1.weight"), 1, F, D, Mf, none);
+  colsum(c, dz, Mf, F, csp, h->gb(l, "mlp.fc1.bias"));
+  layernorm_bwd(c, dy, 0, h->base + bb.xp, D, h->at<float>(bb.mean2), h->at<float>(bb.rstd2),
+                (const float*)h->wb(l, "norm2.weight"), dxo, dxg, D, lnp, h->gb(l, "norm2.weight"), h->gb(l, "norm2.bias"), Mf, D);
+  const float* cls_extra = nullptr;
+  if (shrinks) {
+    gather_fuse_bwd(c, dxg, h->base + bb.xp_full, B, Ta - 1, D, k, h->at<int>(bb.kept), h->at<int>(bb.dropped),
+                    h->at<float>(bb.s), h->cfg.fuse_mode, dxp, h->at<float>(h->off_escore));
+    if (h->cfg.fuse_mode == BSR_FUSE_WEIGHTED_SUM) cls_extra = h->at<float>(h->off_escore);
+  }
+  // attention output projection
+  gemm(c, dxp, D, 1, h->wb(l, "attn.proj.weight"), 1, D, d_o, 0, Ma, D, D, none);
+  gemm(c, dxp, 1, D, h->base + bb.o, 1, D, h->gb(l, "attn.proj.weight"), 1, D, D, Ma, none);
+  colsum(c, dxp, Ma, D, csp, h->gb(l, "attn.proj.bias"));
+  int rc = attention_bwd(c, h->base + bb.qkv, h->base + bb.o, d_o, h->at<float>(bb.lse), h->at<float>(h->off_delta),
+                         cls_extra, dqkv, B, Ta, H, hd);
+  if (rc != 0) return set_err(h->err, BSR_ERR_UNSUPPORTED, "attention backward: %d tokens do not fit this kernel", Ta);
+  // QKV projection
+  gemm(c, dqkv, 3 * D, 1, h->wb(l, "attn.qkv.weight"), 1, D, dy, 0, Ma, D, 3 * D, none);
+  gemm(c, dqkv, 1, 3 * D, h->base + bb.y1, 1, D, h->gb(l, "attn.qkv.weight"), 1, 3 * D, D, Ma, none);
+  colsum(c, dqkv, Ma, 3 * D, csp, h->gb(l, "attn.qkv.bias"));
+  layernorm_bwd(c, dy, 0, h->base + bb.x_in, D, h->at<float>(bb.mean1), h->at<float>(bb.rstd1),
+                (const float*)h->wb(l, "norm1.weight"), dxp, dxi, D, lnp, h->gb(l, "norm1.weight"), h->gb(l, "norm1.bias"), Ma, D);
+  return BSR_OK;
+}
+
+HeadDesc head_desc(bsr_handle* h) {
+  const bsr_dims& d = h->cfg.dims;
+  HeadDesc hd;
+  memset(&hd, 0, sizeof(hd));
+  hd.num_tasks = d.num_tasks;
+  hd.D = d.dim;
+  for (int t = 0; t < d.num_tasks; ++t) {
+    std::string n = "head." + std::to_string(t);
+    hd.ncls[t] = d.num_classes[t];
+    hd.cmax = d.num_classes[t] > hd.cmax ? d.num_classes[t] : hd.cmax;
+    hd.w[t] = h->w((n + ".weight").c_str());
+    hd.bias[t] = (const float*)h->w((n + ".bias").c_str());
+    hd.dw[t] = h->gradp(n + ".weight");
+    hd.db[t] = h->gradp(n + ".bias");
+  }
+  return hd;
+}
+
+// Forward through all blocks.  train: blocks >= t0 write the activation arena.  Returns the offset of the last output.
+int forward_all(bsr_handle* h, const Ctx& c, const void* images, int B, bool train, size_t* x_last_off) {
+  const bsr_dims& d = h->cfg.dims;
+  int D = d.dim;
+  int g = d.image_size / d.patch_size, N = g * g;
+  int pin = d.in_chans * d.patch_size * d.patch_size;
+  patchify(c, images, h->base + h->off_patches, B, d.in_chans, d.image_size, d.patch_size);
+  GemmEpilogue ep;
+  ep.bias = (const float*)h->w("patch_embed.bias");
+  gemm(c, h->base + h->off_patches, pin, 1, h->w("patch_embed.weight"), pin, 1, h->base + h->off_emb, 0, B * N, D, pin, ep);
+  int first_train = train ? h->t0 : d.depth;
+  size_t x0 = (first_train == 0) ? h->bufs_train[0].x_in : h->bufs_frozen[0].x_in;
+  assemble_tokens(c, h->base + h->off_emb, (const float*)h->w("cls_token"), (const float*)h->w("pos_embed"), h->base + x0, B, N, D);
+  int* kept_all = h->at<int>(h->off_kept_all);
+  size_t kept_off = 0;
+  size_t cur = x0;
+  for (int l = 0; l < d.depth; ++l) {
+    BlockBufs bb;
+    bool save = l >= first_train;
+    if (save) {
+      bb = h->bufs_train[l];
+    } else {
+      bb = h->bufs_frozen[l & 1];
+      if (l + 1 == first_train) bb.x_out = h->bufs_train[l + 1].x_in;   // hand over to the first trainable block
+    }
+    bb.x_in = cur;
+    int* kept_dst = nullptr;
+    if (h->sched.k[l] >= 0) { kept_dst = kept_all + kept_off; kept_off += (size_t)B * h->sched.k[l]; }
+    int rc = block_forward(h, c, l, B, bb, save, kept_dst);
+    if (rc != BSR_OK) return rc;
+    cur = bb.x_out;
+  }
+  *x_last_off = cur;
+  return BSR_OK;
+}
+
+size_t kept_total(const bsr_handle* h, int B) {
+  size_t n = 0;
+  for (int l = 0; l < h->cfg.dims.depth; ++l)
+    if (h->sched.k[l] >= 0) n += (size_t)B * h->sched.k[l];
+  return n;
+}
+
+int check_batch(bsr_handle* h, const void* images, int batch) {
+  if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
+  if (images == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "images_dev is null");
+  if (batch < 1 || batch > h->cfg.max_batch) return set_err(h->err, BSR_ERR_INVALID_ARG, "batch %d outside [1, %d]", batch, h->cfg.max_batch);
+  return BSR_OK;
+}
+
+}  // namespace
+
+// =================================================================================================
+// C ABI
+// =================================================================================================
+extern "C" {
+
+int32_t bsr_token_schedule(const bsr_config* cfg, int32_t* ta, int32_t* tf, int32_t* keep) {
+  if (cfg == nullptr || ta == nullptr || tf == nullptr || keep == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "null argument");
+  Schedule s;
+  int rc = compute_schedule(cfg, &s, g_error);
+  if (rc != BSR_OK) return rc;
+  for (int l = 0; l < cfg->dims.depth; ++l) { ta[l] = s.ta[l]; tf[l] = s.tf[l]; keep[l] = s.k[l]; }
+  return BSR_OK;
+}
+
+int32_t bsr_workspace_bytes(const bsr_config* cfg, size_t* bytes) {
+  if (bytes == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "bytes is null");
+  int rc = validate(cfg, g_error);
+  if (rc != BSR_OK) return rc;
+  bsr_handle tmp;
+  tmp.cfg = *cfg;
+  compute_schedule(cfg, &tmp.sched, g_error);
+  build_tensors(&tmp);
+  *bytes = plan(&tmp);
+  return BSR_OK;
+}
+
+int32_t bsr_create(const bsr_config* cfg, void* workspace, size_t bytes, bsr_handle** out) {
+  if (out == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "out is null");
+  *out = nullptr;
+  int rc = validate(cfg, g_error);
+  if (rc != BSR_OK) return rc;
+  if (workspace == nullptr || ((uintptr_t)workspace & 255) != 0) return set_err(g_error, BSR_ERR_INVALID_ARG, "workspace must be non-null and 256-byte aligned");
+  bsr_handle* h = new bsr_handle();
+  h->cfg = *cfg;
+  snprintf(h->err, sizeof(h->err), "no error");
+  compute_schedule(cfg, &h->sched, h->err);
+  build_tensors(h);
+  size_t need = plan(h);
+  if (bytes < need) {
+    delete h;
+    return set_err(g_error, BSR_ERR_WORKSPACE_TOO_SMALL, "workspace of %zu bytes given, %zu needed", bytes, need);
+  }
+  h->base = (char*)workspace;
+  h->bytes = bytes;
+  h->lr = cfg->lr;
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    delete h;
+    return set_err(g_error, BSR_ERR_CUDA, "no usable CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
+  }
+  h->sm_count = prop.multiProcessorCount;
+  if (prop.major != 10) {
+    delete h;
+    return set_err(g_error, BSR_ERR_UNSUPPORTED, "this library is built for sm_100a only (device is sm_%d%d)", prop.major, prop.minor);
+  }
+  // optimiser state and status start at zero; the chunk table is uploaded once
+  cudaMemsetAsync(h->base + h->off_status, 0, 256, 0);
+  cudaMemsetAsync(h->base + h->off_m, 0, h->n_flat * 4, 0);
+  cudaMemsetAsync(h->base + h->off_v, 0, h->n_flat * 4, 0);
+  cudaMemsetAsync(h->base + h->off_grad, 0, h->n_flat * 4, 0);
+  cudaMemsetAsync(h->base + h->off_master, 0, h->n_flat * 4, 0);
+  std::vector<AdamChunk> chunks;
+  for (auto& t : h->tensors) {
+    if (!t.trainable) continue;
+    bool has_shadow = t.matrix && cfg->dims.dtype == BSR_DTYPE_BF16;
+    for (size_t o = 0; o < t.numel; o += ADAM_CHUNK) {
+      AdamChunk ch;
+      ch.offset = (uint32_t)(t.flat + o);
+      ch.count = (uint32_t)((t.numel - o) < ADAM_CHUNK ? (t.numel - o) : ADAM_CHUNK);
+      ch.shadow = has_shadow ? (int64_t)((t.w_off - h->off_weights) / 2 + o) : -1;
+      ch.decay = t.decay ? 1u : 0u;
+      ch.pad = 0;
+      chunks.push_back(ch);
+    }
+  }
+  if (!chunks.empty())
+    cudaMemcpy(h->base + h->off_chunks, chunks.data(), chunks.size() * sizeof(AdamChunk), cudaMemcpyHostToDevice);
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    delete h;
+    return set_err(g_error, BSR_ERR_CUDA, "workspace initialisation failed: %s", cudaGetErrorString(e));
+  }
+  *out = h;
+  return BSR_OK;
+}
+
+int32_t bsr_destroy(bsr_handle* h) {
+  delete h;
+  return BSR_OK;
+}
+
+const char* bsr_last_error(const bsr_handle* h) { return h ? h->err : g_error; }
+
+int32_t bsr_set_param(bsr_handle* h, const char* name, const float* src, size_t count, void* stream) {
+  if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
+  if (name == nullptr || src == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "null argument");
+  auto it = h->index.find(name);
+  if (it == h->index.end()) return set_err(h->err, BSR_ERR_INVALID_ARG, "unknown parameter '%s'", name);
+  const Tensor& t = h->tensors[it->second];
+  if (count != t.numel) return set_err(h->err, BSR_ERR_INVALID_ARG, "'%s' has %zu elements, %zu given", name, t.numel, count);
+  Ctx c = make_ctx(h, stream);
+  if (t.trainable)
+    cudaMemcpyAsync(h->at<float>(h->off_master) + t.flat, src, count * 4, cudaMemcpyDeviceToDevice, c.stream);
+  bool alias_master = t.trainable && (!t.matrix || c.dtype == BSR_DTYPE_FP32);
+  if (!alias_master) {
+    if (t.matrix) convert_from_float(c, src, h->base + t.w_off, count);
+    else cudaMemcpyAsync(h->base + t.w_off, src, count * 4, cudaMemcpyDeviceToDevice, c.stream);
+  }
+  return check_cuda(h, "bsr_set_param");
+}
+
+int32_t bsr_get_tensor(bsr_handle* h, const char* name, float* dst, size_t count, void* stream) {
+  if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
+  if (name == nullptr || dst == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "null argument");
+  Ctx c = make_ctx(h, stream);
+  std::string n(name);
+  const float* src = nullptr;
+  size_t numel = 0;
+  if (n == "loss") { src = h->at<float>(h->off_loss); numel = 1; }
+  else if (n == "logits") {
+    int cmax = 0;
+    for (int t = 0; t < h->cfg.dims.num_tasks; ++t) cmax = h->cfg.dims.num_classes[t] > cmax ? h->cfg.dims.num_classes[t] : cmax;
+    src = h->at<float>(h->off_logits); numel = (size_t)h->cfg.max_batch * cmax;
+  } else {
+    size_t base_off = 0;
+    std::string pn = n;
+    bool state = false;
+    if (n.rfind("grad/", 0) == 0) { base_off = h->off_grad; pn = n.substr(5); state = true; }
+    else if (n.rfind("adam_m/", 0) == 0) { base_off = h->off_m; pn = n.substr(7); state = true; }
+    else if (n.rfind("adam_v/", 0) == 0) { base_off = h->off_v; pn = n.substr(7); state = true; }
+    auto it = h->index.find(pn);
+    if (it == h->index.end()) return set_err(h->err, BSR_ERR_INVALID_ARG, "unknown tensor '%s'", name);
+    const Tensor& t = h->tensors[it->second];
+    numel = t.numel;
+    if (state) {
+      if (!t.trainable) return set_err(h->err, BSR_ERR_INVALID_ARG, "'%s' is frozen: it has no gradient or optimiser state", pn.c_str());
+      src = h->at<float>(base_off) + t.flat;
+    } else if (t.trainable) {
+      src = h->at<float>(h->off_master) + t.flat;
+    } else if (!t.matrix) {
+      src = h->at<float>(t.w_off);
+    } else {
+      if (count != numel) return set_err(h->err, BSR_ERR_INVALID_ARG, "'%s' has %zu elements, %zu given", name, numel, count);
+      convert_to_float(c, h->base + t.w_off, dst, numel);
+      return check_cuda(h, "bsr_get_tensor");
+    }
+  }
+  if (count != numel) return set_err(h->err, BSR_ERR_INVALID_ARG, "'%s' has %zu elements, %zu given", name, numel, count);
+  cudaMemcpyAsync(dst, src, numel * 4, cudaMemcpyDeviceToDevice, c.stream);
+  return check_cuda(h, "bsr_get_tensor");
+}
+
+int32_t bsr_set_lr(bsr_handle* h, float lr) {
+  if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
+  h->lr = lr;
+  return BSR_OK;
+}
+
+int32_t bsr_set_step(bsr_handle* h, int64_t steps_done) {
+  if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
+  if (steps_done < 0) return set_err(h->err, BSR_ERR_INVALID_ARG, "steps_done must not be negative");
+  h->step = steps_done;
+  return BSR_OK;
+}
+
+int32_t bsr_train_step(bsr_handle* h, const void* images, const int32_t* labels, const int32_t* task_ids, int32_t batch,
+                       void* stream, float* loss_out, int32_t* kept_out) {
+  int rc = check_batch(h, images, batch);
+  if (rc != BSR_OK) return rc;
+  if (labels == nullptr || loss_out == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "labels_dev and loss_dev_out must not be null");
+  if (h->cfg.dims.num_tasks > 1 && task_ids == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "task_ids_dev is required with several tasks");
+  const bsr_dims& d = h->cfg.dims;
+  Ctx c = make_ctx(h, stream);
+  int D = d.dim, B = batch;
+  size_t es = dtype_size(d.dtype);
+  size_t x_last = 0;
+  rc = forward_all(h, c, images, B, true, &x_last);
+  if (rc != BSR_OK) return rc;
+  int Tl = h->sched.tf[d.depth - 1];
+  HeadDesc hd = head_desc(h);
+  float* xn = h->at<float>(h->off_xn);
+  layernorm_fwd(c, h->base + x_last, (long)Tl * D, (const float*)h->w("norm.weight"), (const float*)h->w("norm.bias"), xn, 1,
+                h->at<float>(h->off_meanf), h->at<float>(h->off_rstdf), B, D, d.ln_eps);
+  head_fwd(c, hd, xn, task_ids, h->at<float>(h->off_logits), B);
+  cross_entropy(c, hd, h->at<float>(h->off_logits), labels, task_ids, h->at<float>(h->off_per_image), h->at<float>(h->off_dlogits),
+                h->at<float>(h->off_loss), B);
+  cudaMemcpyAsync(loss_out, h->at<float>(h->off_loss), 4, cudaMemcpyDeviceToDevice, c.stream);
+  if (kept_out != nullptr && kept_total(h, B) > 0)
+    cudaMemcpyAsync(kept_out, h->base + h->off_kept_all, kept_total(h, B) * 4, cudaMemcpyDeviceToDevice, c.stream);
+  // backward: head, final LayerNorm, trainable blocks in reverse, nothing before the earliest one
+  head_bwd(c, hd, xn, h->at<float>(h->off_dlogits), task_ids, h->at<float>(h->off_dxn), B);
+  float* lnp = h->at<float>(h->off_ln_partials);
+  if (h->t0 < d.depth) {
+    void* dxo = h->base + h->off_dxa;
+    void* dxi = h->base + h->off_dxb;
+    cudaMemsetAsync(dxo, 0, (size_t)B * Tl * D * es, c.stream);
+    layernorm_bwd(c, h->at<float>(h->off_dxn), 1, h->base + x_last, (long)Tl * D, h->at<float>(h->off_meanf), h->at<float>(h->off_rstdf),
+                  (const float*)h->w("norm.weight"), nullptr, dxo, (long)Tl * D, lnp, h->gradp("norm.weight"), h->gradp("norm.bias"), B, D);
+    for (int l = d.depth - 1; l >= h->t0; --l) {
+      rc = block_backward(h, c, l, B, dxo, l > h->t0 ? dxi : nullptr);
+      if (rc != BSR_OK) return rc;
+      void* t = dxo; dxo = dxi; dxi = t;
+    }
+  } else {
+    layernorm_bwd(c, h->at<float>(h->off_dxn), 1, h->base + x_last, (long)Tl * D, h->at<float>(h->off_meanf), h->at<float>(h->off_rstdf),
+                  (const float*)h->w("norm.weight"), nullptr, nullptr, 0, lnp, h->gradp("norm.weight"), h->gradp("norm.bias"), B, D);
+  }
+  h->step += 1;
+  double bc1 = 1.0 - std::pow((double)h->cfg.beta1, (double)h->step);
+  double bc2 = 1.0 - std::pow((double)h->cfg.beta2, (double)h->step);
+  adamw(c, h->at<AdamChunk>(h->off_chunks), h->n_chunks, h->at<float>(h->off_master), h->at<float>(h->off_grad), h->at<float>(h->off_m),
+        h->at<float>(h->off_v), h->base + h->off_weights, h->lr, h->cfg.beta1, h->cfg.beta2, h->cfg.eps, h->cfg.weight_decay,
+        (float)bc1, (float)bc2);
+  return check_cuda(h, "bsr_train_step");
+}
+
+int32_t bsr_eval_forward(bsr_handle* h, const void* images, const int32_t* task_ids, int32_t batch, void* stream,
+                         float* logits_out, int32_t* kept_out) {
+  int rc = check_batch(h, images, batch);
+  if (rc != BSR_OK) return rc;
+  if (logits_out == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "logits_dev_out is null");
+  if (h->cfg.dims.num_tasks > 1 && task_ids == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "task_ids_dev is required with several tasks");
+  const bsr_dims& d = h->cfg.dims;
+  Ctx c = make_ctx(h, stream);
+  size_t x_last = 0;
+  rc = forward_all(h, c, images, batch, false, &x_last);
+  if (rc != BSR_OK) return rc;
+  int Tl = h->sched.tf[d.depth - 1];
+  HeadDesc hd = head_desc(h);
+  float* xn = h->at<float>(h->off_xn);
+  layernorm_fwd(c, h->base + x_last, (long)Tl * d.dim, (const float*)h->w("norm.weight"), (const float*)h->w("norm.bias"), xn, 1,
+                nullptr, nullptr, batch, d.dim, d.ln_eps);
+  head_fwd(c, hd, xn, task_ids, h->at<float>(h->off_logits), batch);
+  cudaMemcpyAsync(logits_out, h->at<float>(h->off_logits), (size_t)batch * hd.cmax * 4, cudaMemcpyDeviceToDevice, c.stream);
+  if (kept_out != nullptr && kept_total(h, batch) > 0)
+    cudaMemcpyAsync(kept_out, h->base + h->off_kept_all, kept_total(h, batch) * 4, cudaMemcpyDeviceToDevice, c.stream);
+  return check_cuda(h, "bsr_eval_forward");
+}
+
+int32_t bsr_get_footprint(const bsr_handle* h, bsr_footprint* out) {
+  if (h == nullptr || out == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "null argument");
+  const bsr_dims& d = h->cfg.dims;
+  memset(out, 0, sizeof(*out));
+  out->workspace_bytes = h->bytes;
+  out->weight_bytes = h->weights_bytes;
+  out->master_bytes = h->n_flat * 4;
+  out->optimizer_bytes = h->n_flat * 8;
+  out->grad_bytes = h->n_flat * 4;
+  out->saved_activation_bytes = h->arena_bytes;
+  out->scratch_bytes = h->scratch_bytes;
+  uint64_t paper = 0, params = 0;
+  for (int l = h->t0; l < d.depth; ++l) {
+    // Table 1 accounting in fp32: Q,K,V + softmax input + GELU input, plus the inputs of the six linear layers
+    uint64_t ta = h->sched.ta[l], tf = h->sched.tf[l];
+    uint64_t el = 3 * ta * d.dim + (uint64_t)d.heads * ta * ta + tf * d.mlp_hidden;
+    el += 3 * ta * d.dim + 2 * tf * d.dim + tf * d.mlp_hidden;
+    paper += el * 4 * (uint64_t)h->cfg.max_batch;
+  }
+  for (auto& t : h->tensors)
+    if (t.trainable) params += t.numel;
+  out->paper_activation_bytes = paper;
+  out->trainable_params = params;
+  return BSR_OK;
+}
+
+int32_t bsr_sync_status(bsr_handle* h, void* stream) {
+  if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
+  int st = 0;
+  cudaError_t e = cudaMemcpyAsync(&st, h->base + h->off_status, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->base + h->off_status, 0, 4, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) return set_err(h->err, BSR_ERR_CUDA, "bsr_sync_status: %s", cudaGetErrorString(e));
+  if (st & STATUS_TIMEOUT) return set_err(h->err, BSR_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired");
+  if (st & STATUS_NONFINITE) return set_err(h->err, BSR_ERR_NONFINITE, "the loss was not finite");
+  return BSR_OK;
+}
+
+// ---- stand-alone kernels ------------------------------------------------------------------------
+
+static Ctx bare_ctx(int dtype, void* stream) {
+  Ctx c;
+  c.stream = (cudaStream_t)stream;
+  c.dtype = dtype;
+  c.status = nullptr;
+  c.sm_count = 0;
+  c.use_tc = 0;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess) c.sm_count = sms;
+  return c;
+}
+
+int32_t bsr_token_select(const float* p, int32_t batch, int32_t heads, int32_t m, int32_t k, float* scores, int32_t* kept,
+                         int32_t* dropped, void* stream) {
+  if (p == nullptr || scores == nullptr || kept == nullptr || (dropped == nullptr && k < m)) return set_err(g_error, BSR_ERR_INVALID_ARG, "null argument");
+  if (batch < 1 || heads < 1 || m < 1 || m > 4096 || k < 1 || k > m) return set_err(g_error, BSR_ERR_INVALID_ARG, "need batch, heads >= 1 and 1 <= k <= m <= 4096");
+  token_select((cudaStream_t)stream, p, batch, heads, m, k, scores, kept, dropped);
+  return check_cuda(nullptr, "bsr_token_select");
+}
+
+int32_t bsr_gather_fuse(const void* x, int32_t dtype, int32_t batch, int32_t m, int32_t dim, int32_t k, const int32_t* kept,
+                        const int32_t* dropped, const float* scores, int32_t fuse_mode, void* out, void* stream) {
+  if (x == nullptr || kept == nullptr || out == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "null argument");
+  if (dtype != BSR_DTYPE_FP32 && dtype != BSR_DTYPE_BF16) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad dtype");
+  if (batch < 1 || m < 1 || k < 1 || k > m || dim < 1 || (dim * dtype_size(dtype)) % 16 != 0) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad shape: rows must be a multiple of 16 bytes, 1 <= k <= m");
+  bool fuse = fuse_mode == BSR_FUSE_WEIGHTED_SUM && k < m;
+  if (fuse && (dropped == nullptr || scores == nullptr)) return set_err(g_error, BSR_ERR_INVALID_ARG, "fusion needs dropped_dev and scores_dev");
+  Ctx c = bare_ctx(dtype, stream);
+  gather_fuse(c, x, batch, m, dim, k, kept, dropped, scores, fuse_mode, out);
+  return check_cuda(nullptr, "bsr_gather_fuse");
+}
+
+int32_t bsr_linear_forward(const void* x, const void* w, const float* bias, const void* residual, void* y, int32_t m, int32_t n,
+                           int32_t k, int32_t dtype, int32_t act_gelu, int32_t use_tensor_cores, void* stream) {
+  if (x == nullptr || w == nullptr || y == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "null argument");
+  if (dtype != BSR_DTYPE_FP32 && dtype != BSR_DTYPE_BF16) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad dtype");
+  if (m < 1 || n < 1 || k < 1) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad shape");
+  Ctx c = bare_ctx(dtype, stream);
+  GemmEpilogue e;
+  e.bias = bias;
+  e.residual = residual;
+  e.act = act_gelu ? 1 : 0;
+  if (use_tensor_cores) {
+    if (dtype != BSR_DTYPE_BF16 || !gemm_tc_supported(m, n, k)) return set_err(g_error, BSR_ERR_UNSUPPORTED, "the tcgen05 kernel needs bf16 and k, n multiples of 8");
+    int rc = gemm_tc(c, x, w, y, 0, m, n, k, e);
+    if (rc != 0) return set_err(g_error, BSR_ERR_CUDA, "tcgen05 GEMM set-up failed (%d)", rc);
+  } else {
+    gemm(c, x, k, 1, w, k, 1, y, 0, m, n, k, e);
+  }
+  return check_cuda(nullptr, "bsr_linear_forward");
+}
+
+int32_t bsr_attention_forward(const void* qkv, int32_t dtype, int32_t batch, int32_t t, int32_t heads, int32_t d, void* out,
+                              float* cls_prob, void* stream) {
+  if (qkv == nullptr || out == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "null argument");
+  if (dtype != BSR_DTYPE_FP32 && dtype != BSR_DTYPE_BF16) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad dtype");
+  if (batch < 1 || t < 1 || heads < 1 || d < 8 || d > 64 || d % 8 != 0) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad shape: head dimension must be a multiple of 8, at most 64");
+  Ctx c = bare_ctx(dtype, stream);
+  if (attention_fwd(c, qkv, out, nullptr, cls_prob, batch, t, heads, d) != 0)
+    return set_err(g_error, BSR_ERR_UNSUPPORTED, "%d tokens do not fit the attention kernel's shared memory", t);
+  return check_cuda(nullptr, "bsr_attention_forward");
+}
+
+}  // extern "C"

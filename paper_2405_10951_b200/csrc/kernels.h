@@ -1,0 +1,101 @@
+// Host-side launchers of the BSR kernels.  Every launcher enqueues on ctx.stream and returns;
+// pointers are device addresses; `dtype` selects the storage type of activations and matrices
+// (0 = float, 1 = bf16); LayerNorm parameters, biases, statistics, scores and gradients of
+// parameters are always float.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace bsr {
+
+struct Ctx {
+  cudaStream_t stream;
+  int dtype;        // 0 fp32, 1 bf16
+  int* status;      // device status word (may be null for the stand-alone entry points)
+  int sm_count;
+  int use_tc;       // bf16 only: dense contractions on the tcgen05 kernels
+};
+
+inline size_t dtype_size(int dtype) { return dtype == 0 ? 4 : 2; }
+
+// ---- embedding --------------------------------------------------------------------------------
+void patchify(const Ctx& c, const void* images, void* patches, int B, int C, int S, int P);
+void assemble_tokens(const Ctx& c, const void* emb, const float* cls, const float* pos, void* x, int B, int N, int D);
+
+// ---- LayerNorm --------------------------------------------------------------------------------
+// y[r] = LN(x[r]) * g + b for `rows` rows of length D; row r of x starts at x + r * x_stride elements.
+// mean/rstd (optional) receive the row statistics.  y_is_float selects a float output (head path).
+void layernorm_fwd(const Ctx& c, const void* x, long x_stride, const float* g, const float* b, void* y, int y_is_float,
+                   float* mean, float* rstd, int rows, int D, float eps);
+// dx[r] = dres[r] + LN'(dy[r]);  partial sums of dgamma/dbeta go to `partials` ([2][groups][D]) and are
+// reduced in a fixed order into dgamma, dbeta.  dx may be null (only parameter gradients wanted);
+// dres may be null.  dy_is_float: dy is float [rows, D] (head path).  dx rows start at dx + r * dx_stride.
+void layernorm_bwd(const Ctx& c, const void* dy, int dy_is_float, const void* x, long x_stride, const float* mean,
+                   const float* rstd, const float* g, const void* dres, void* dx, long dx_stride, float* partials,
+                   float* dgamma, float* dbeta, int rows, int D);
+int layernorm_bwd_groups(const Ctx& c, int rows);
+
+// ---- column sums (bias gradients) -------------------------------------------------------------
+void colsum(const Ctx& c, const void* x, int rows, int cols, float* partials, float* out);
+int colsum_groups(int rows);
+
+// ---- dense contractions -----------------------------------------------------------------------
+// C[m, n] = epilogue(sum_k A(m, k) * B(n, k)).  A(m,k) = A[m * a_rs + k * a_cs], B alike.
+struct GemmEpilogue {
+  const float* bias = nullptr;      // [n]
+  const void* residual = nullptr;   // [m, n] in the output type, added last
+  int act = 0;                      // 0 none, 1 GELU (pre-activation optionally stored), 2 multiply by GELU'(aux_in)
+  void* aux_out = nullptr;          // act 1: pre-activation [m, n], output type
+  const void* aux_in = nullptr;     // act 2: pre-activation [m, n], storage type
+};
+void gemm(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long b_rs, long b_cs, void* C,
+          int out_is_float, int m, int n, int k, const GemmEpilogue& e);
+// True when the tcgen05 kernel can take this problem (bf16, both operands contiguous along k, aligned).
+bool gemm_tc_supported(int m, int n, int k);
+int gemm_tc(const Ctx& c, const void* A, const void* B, void* C, int out_is_float, int m, int n, int k,
+            const GemmEpilogue& e);
+
+// ---- attention --------------------------------------------------------------------------------
+// qkv [B, T, 3, H, d]; out [B, T, H*d]; lse (optional) [B, H, T] natural-log sum of exponentials of the
+// scaled scores; cls_prob (optional) [B, H, T-1].
+int attention_fwd(const Ctx& c, const void* qkv, void* out, float* lse, float* cls_prob, int B, int T, int H, int d);
+// dqkv from dout; delta scratch [B, H, T]; cls_extra (optional) [B, T-1]: gradient arriving at the head-mean
+// score of each non-classification token (zero for kept tokens); cls_prob needed with it.
+int attention_bwd(const Ctx& c, const void* qkv, const void* out, const void* dout, const float* lse, float* delta,
+                  const float* cls_extra, void* dqkv, int B, int T, int H, int d);
+
+// ---- token selection --------------------------------------------------------------------------
+void token_select(cudaStream_t s, const float* p, int B, int H, int M, int k, float* scores, int* kept, int* dropped);
+void gather_fuse(const Ctx& c, const void* x, int B, int M, int D, int k, const int* kept, const int* dropped,
+                 const float* scores, int fuse, void* out);
+// Backward of the compaction: dx [B, 1+M, D] from dout [B, 1+k+f, D]; escore [B, M] = <g_fused, x_j> for dropped j, else 0.
+void gather_fuse_bwd(const Ctx& c, const void* dout, const void* x, int B, int M, int D, int k, const int* kept,
+                     const int* dropped, const float* scores, int fuse, void* dx, float* escore);
+
+// ---- head, loss, optimiser --------------------------------------------------------------------
+// logits[b, c] = xn[b] . W_task(b)[c] + bias; classes beyond the task's count get -inf.
+struct HeadDesc {
+  int num_tasks, cmax, D;
+  int ncls[4];
+  const void* w[4];       // storage dtype [ncls, D]
+  const float* bias[4];
+  float* dw[4];           // gradients (float)
+  float* db[4];
+};
+void head_fwd(const Ctx& c, const HeadDesc& h, const float* xn, const int* task_ids, float* logits, int B);
+void cross_entropy(const Ctx& c, const HeadDesc& h, const float* logits, const int* labels, const int* task_ids,
+                   float* per_image, float* dlogits, float* loss, int B);
+void head_bwd(const Ctx& c, const HeadDesc& h, const float* xn, const float* dlogits, const int* task_ids, float* dxn, int B);
+
+struct AdamChunk { uint32_t offset; uint32_t count; int64_t shadow; uint32_t decay; uint32_t pad; };
+void adamw(const Ctx& c, const AdamChunk* chunks, int nchunks, float* master, const float* grad, float* m, float* v,
+           void* shadow_base, float lr, float b1, float b2, float eps, float wd, float bc1, float bc2);
+
+// ---- conversions ------------------------------------------------------------------------------
+void convert_from_float(const Ctx& c, const float* src, void* dst, size_t n);   // float -> storage dtype
+void convert_to_float(const Ctx& c, const void* src, float* dst, size_t n);     // storage dtype -> float
+void fill_float(cudaStream_t s, float* dst, float v, size_t n);
+
+}  // namespace bsr

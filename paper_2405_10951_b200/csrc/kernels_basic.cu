@@ -1,0 +1,513 @@
+// Bandwidth-bound kernels of the BSR step: patch extraction, token assembly, LayerNorm forward and
+// backward, column sums, head/loss, AdamW, conversions.  All reductions run in a fixed order.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace bsr {
+
+// ------------------------------------------------------------------------------------------------
+// Patch extraction (Section 3.1: the image is partitioned into N patches).  Output row = one patch
+// flattened as (channel, row in patch, column in patch).
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void patchify_kernel(const T* __restrict__ img, T* __restrict__ out, int B, int C, int S, int P, long total) {
+  long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  int g = S / P;
+  int px = (int)(i % P); long r = i / P;
+  int py = (int)(r % P); r /= P;
+  int ch = (int)(r % C); r /= C;
+  int gx = (int)(r % g); r /= g;
+  int gy = (int)(r % g); r /= g;
+  int b = (int)r;
+  out[i] = img[(((long)b * C + ch) * S + (gy * P + py)) * S + gx * P + px];
+}
+
+void patchify(const Ctx& c, const void* images, void* patches, int B, int C, int S, int P) {
+  int g = S / P;
+  long total = (long)B * g * g * C * P * P;
+  int threads = 256;
+  int blocks = ceil_div(total, threads);
+  if (c.dtype == 0)
+    patchify_kernel<float><<<blocks, threads, 0, c.stream>>>((const float*)images, (float*)patches, B, C, S, P, total);
+  else
+    patchify_kernel<bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)images, (bf16*)patches, B, C, S, P, total);
+}
+
+// x[b, 0] = cls + pos[0];  x[b, 1 + n] = emb[b, n] + pos[1 + n]   (classification token and positional embedding)
+template <typename T>
+__global__ void assemble_kernel(const T* __restrict__ emb, const float* __restrict__ cls, const float* __restrict__ pos,
+                                T* __restrict__ x, int B, int N, int D, long total) {
+  long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  int d = (int)(i % D); long r = i / D;
+  int t = (int)(r % (N + 1));
+  int b = (int)(r / (N + 1));
+  float v = (t == 0) ? cls[d] : to_f(emb[((long)b * N + (t - 1)) * D + d]);
+  x[i] = from_f<T>(v + pos[(long)t * D + d]);
+}
+
+void assemble_tokens(const Ctx& c, const void* emb, const float* cls, const float* pos, void* x, int B, int N, int D) {
+  long total = (long)B * (N + 1) * D;
+  int threads = 256, blocks = ceil_div(total, threads);
+  if (c.dtype == 0)
+    assemble_kernel<float><<<blocks, threads, 0, c.stream>>>((const float*)emb, cls, pos, (float*)x, B, N, D, total);
+  else
+    assemble_kernel<bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)emb, cls, pos, (bf16*)x, B, N, D, total);
+}
+
+// ------------------------------------------------------------------------------------------------
+// LayerNorm.  One warp per row, the row held in registers (D <= 1024, D % Pack::N == 0).
+// ------------------------------------------------------------------------------------------------
+constexpr int LN_MAX_PER_LANE = 32;   // floats per lane: D <= 1024
+
+template <typename TX, typename TY>
+__global__ void layernorm_fwd_kernel(const TX* __restrict__ x, long x_stride, const float* __restrict__ g,
+                                     const float* __restrict__ b, TY* __restrict__ y, float* __restrict__ mean,
+                                     float* __restrict__ rstd, int rows, int D, float eps) {
+  constexpr int N = Pack<TX>::N;
+  constexpr int MAXC = LN_MAX_PER_LANE / N;
+  int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  int lane = threadIdx.x & 31;
+  if (warp >= rows) return;
+  const TX* xr = x + (long)warp * x_stride;
+  int chunks = D / N;
+  float v[LN_MAX_PER_LANE];
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < MAXC; ++i) {
+    int ch = lane + i * 32;
+    if (ch < chunks) {
+      load16(xr + ch * N, v + i * N);
+#pragma unroll
+      for (int j = 0; j < N; ++j) sum += v[i * N + j];
+    }
+  }
+  float mu = warp_sum(sum) / (float)D;
+  float sq = 0.f;
+#pragma unroll
+  for (int i = 0; i < MAXC; ++i) {
+    int ch = lane + i * 32;
+    if (ch < chunks) {
+#pragma unroll
+      for (int j = 0; j < N; ++j) { float t = v[i * N + j] - mu; sq += t * t; }
+    }
+  }
+  float rs = rsqrtf(warp_sum(sq) / (float)D + eps);
+  if (lane == 0) {
+    if (mean) mean[warp] = mu;
+    if (rstd) rstd[warp] = rs;
+  }
+  TY* yr = y + (long)warp * D;
+#pragma unroll
+  for (int i = 0; i < MAXC; ++i) {
+    int ch = lane + i * 32;
+    if (ch < chunks) {
+      float o[N];
+#pragma unroll
+      for (int j = 0; j < N; ++j) {
+        int col = ch * N + j;
+        o[j] = (v[i * N + j] - mu) * rs * g[col] + b[col];
+      }
+      store_n<N>(yr + ch * N, o);
+    }
+  }
+}
+
+void layernorm_fwd(const Ctx& c, const void* x, long x_stride, const float* g, const float* b, void* y, int y_is_float,
+                   float* mean, float* rstd, int rows, int D, float eps) {
+  int threads = 256;
+  int blocks = ceil_div((long)rows * 32, threads);
+  if (c.dtype == 0)
+    layernorm_fwd_kernel<float, float><<<blocks, threads, 0, c.stream>>>((const float*)x, x_stride, g, b, (float*)y, mean, rstd, rows, D, eps);
+  else if (y_is_float)
+    layernorm_fwd_kernel<bf16, float><<<blocks, threads, 0, c.stream>>>((const bf16*)x, x_stride, g, b, (float*)y, mean, rstd, rows, D, eps);
+  else
+    layernorm_fwd_kernel<bf16, bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)x, x_stride, g, b, (bf16*)y, mean, rstd, rows, D, eps);
+}
+
+// Backward.  Each block owns rows blockIdx.x*8 + warp, stepping by gridDim.x*8; every lane accumulates the
+// dgamma/dbeta contributions of its columns, warps are combined through shared memory in warp order, and the
+// block's sums go to partials[0][block][col] (dgamma) and partials[1][block][col] (dbeta).
+constexpr int LNB_WARPS = 8;
+
+template <typename TX, typename TDY>
+__global__ void layernorm_bwd_kernel(const TDY* __restrict__ dy, const TX* __restrict__ x, long x_stride,
+                                     const float* __restrict__ mean, const float* __restrict__ rstd,
+                                     const float* __restrict__ g, const TX* __restrict__ dres, TX* __restrict__ dx,
+                                     long dx_stride, float* __restrict__ partials, int rows, int D) {
+  constexpr int N = Pack<TX>::N;
+  constexpr int MAXC = LN_MAX_PER_LANE / N;
+  extern __shared__ float sm[];   // [LNB_WARPS][2][D]
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int chunks = D / N;
+  float ag[LN_MAX_PER_LANE], ab[LN_MAX_PER_LANE];
+#pragma unroll
+  for (int i = 0; i < LN_MAX_PER_LANE; ++i) { ag[i] = 0.f; ab[i] = 0.f; }
+  for (int r = blockIdx.x * LNB_WARPS + warp; r < rows; r += gridDim.x * LNB_WARPS) {
+    const TX* xr = x + (long)r * x_stride;
+    const TDY* dyr = dy + (long)r * D;
+    float mu = mean[r], rs = rstd[r];
+    float xh[LN_MAX_PER_LANE], dh[LN_MAX_PER_LANE];
+    float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < MAXC; ++i) {
+      int ch = lane + i * 32;
+      if (ch < chunks) {
+        float xv[N], dv[N];
+        load16(xr + ch * N, xv);
+        load_n<N>(dyr + ch * N, dv);
+#pragma unroll
+        for (int j = 0; j < N; ++j) {
+          int col = ch * N + j;
+          float d = dv[j];
+          float h = (xv[j] - mu) * rs;
+          xh[i * N + j] = h;
+          ag[i * N + j] += d * h;
+          ab[i * N + j] += d;
+          float dxh = d * g[col];
+          dh[i * N + j] = dxh;
+          s1 += dxh;
+          s2 += dxh * h;
+        }
+      }
+    }
+    s1 = warp_sum(s1) / (float)D;
+    s2 = warp_sum(s2) / (float)D;
+    if (dx != nullptr) {
+      TX* dxr = dx + (long)r * dx_stride;
+#pragma unroll
+      for (int i = 0; i < MAXC; ++i) {
+        int ch = lane + i * 32;
+        if (ch < chunks) {
+          float o[N];
+          if (dres != nullptr) load16(dres + (long)r * D + ch * N, o);
+          else {
+#pragma unroll
+            for (int j = 0; j < N; ++j) o[j] = 0.f;
+          }
+#pragma unroll
+          for (int j = 0; j < N; ++j) o[j] += rs * (dh[i * N + j] - s1 - xh[i * N + j] * s2);
+          store16(dxr + ch * N, o);
+        }
+      }
+    }
+  }
+  float* mine = sm + (size_t)warp * 2 * D;
+#pragma unroll
+  for (int i = 0; i < MAXC; ++i) {
+    int ch = lane + i * 32;
+    if (ch < chunks) {
+#pragma unroll
+      for (int j = 0; j < N; ++j) {
+        mine[ch * N + j] = ag[i * N + j];
+        mine[D + ch * N + j] = ab[i * N + j];
+      }
+    }
+  }
+  __syncthreads();
+  for (int col = threadIdx.x; col < 2 * D; col += blockDim.x) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < LNB_WARPS; ++w) s += sm[(size_t)w * 2 * D + col];
+    int which = col / D, cc = col % D;
+    partials[((size_t)which * gridDim.x + blockIdx.x) * D + cc] = s;
+  }
+}
+
+// out[col] = sum over groups of partials[group][col], groups in ascending order.
+__global__ void reduce_partials_kernel(const float* __restrict__ partials, int groups, int cols, float* __restrict__ out) {
+  int col = blockIdx.x * blockDim.x + threadIdx.x;
+  if (col >= cols) return;
+  float s = 0.f;
+  for (int gidx = 0; gidx < groups; ++gidx) s += partials[(size_t)gidx * cols + col];
+  out[col] = s;
+}
+
+int layernorm_bwd_groups(const Ctx& c, int rows) {
+  int want = ceil_div(rows, LNB_WARPS);
+  int cap = c.sm_count > 0 ? 2 * c.sm_count : 296;
+  return want < cap ? (want < 1 ? 1 : want) : cap;
+}
+
+void layernorm_bwd(const Ctx& c, const void* dy, int dy_is_float, const void* x, long x_stride, const float* mean,
+                   const float* rstd, const float* g, const void* dres, void* dx, long dx_stride, float* partials,
+                   float* dgamma, float* dbeta, int rows, int D) {
+  int groups = layernorm_bwd_groups(c, rows);
+  size_t smem = (size_t)LNB_WARPS * 2 * D * sizeof(float);
+  int threads = LNB_WARPS * 32;
+  if (c.dtype == 0) {
+    cudaFuncSetAttribute(layernorm_bwd_kernel<float, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    layernorm_bwd_kernel<float, float><<<groups, threads, smem, c.stream>>>(
+        (const float*)dy, (const float*)x, x_stride, mean, rstd, g, (const float*)dres, (float*)dx, dx_stride, partials, rows, D);
+  } else if (dy_is_float) {
+    cudaFuncSetAttribute(layernorm_bwd_kernel<bf16, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    layernorm_bwd_kernel<bf16, float><<<groups, threads, smem, c.stream>>>(
+        (const float*)dy, (const bf16*)x, x_stride, mean, rstd, g, (const bf16*)dres, (bf16*)dx, dx_stride, partials, rows, D);
+  } else {
+    cudaFuncSetAttribute(layernorm_bwd_kernel<bf16, bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    layernorm_bwd_kernel<bf16, bf16><<<groups, threads, smem, c.stream>>>(
+        (const bf16*)dy, (const bf16*)x, x_stride, mean, rstd, g, (const bf16*)dres, (bf16*)dx, dx_stride, partials, rows, D);
+  }
+  int t2 = 256;
+  reduce_partials_kernel<<<ceil_div(D, t2), t2, 0, c.stream>>>(partials, groups, D, dgamma);
+  reduce_partials_kernel<<<ceil_div(D, t2), t2, 0, c.stream>>>(partials + (size_t)groups * D, groups, D, dbeta);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Column sums (bias gradients): two stages, fixed order.
+// ------------------------------------------------------------------------------------------------
+constexpr int CS_ROWLANES = 8;
+constexpr int CS_GROUPS = 64;
+
+template <typename T>
+__global__ void colsum_kernel(const T* __restrict__ x, int rows, int cols, float* __restrict__ partials) {
+  constexpr int N = Pack<T>::N;
+  __shared__ float sm[CS_ROWLANES][32 * N];
+  int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  int col0 = (blockIdx.x * 32 + tx) * N;
+  float acc[N];
+#pragma unroll
+  for (int j = 0; j < N; ++j) acc[j] = 0.f;
+  if (col0 < cols) {
+    for (int r = blockIdx.y * CS_ROWLANES + ty; r < rows; r += gridDim.y * CS_ROWLANES) {
+      float v[N];
+      load16(x + (long)r * cols + col0, v);
+#pragma unroll
+      for (int j = 0; j < N; ++j) acc[j] += v[j];
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < N; ++j) sm[ty][tx * N + j] = acc[j];
+  __syncthreads();
+  for (int cidx = threadIdx.x; cidx < 32 * N; cidx += blockDim.x) {
+    int col = blockIdx.x * 32 * N + cidx;
+    if (col < cols) {
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < CS_ROWLANES; ++w) s += sm[w][cidx];
+      partials[(size_t)blockIdx.y * cols + col] = s;
+    }
+  }
+}
+
+int colsum_groups(int rows) {
+  int want = ceil_div(rows, CS_ROWLANES);
+  return want < CS_GROUPS ? (want < 1 ? 1 : want) : CS_GROUPS;
+}
+
+void colsum(const Ctx& c, const void* x, int rows, int cols, float* partials, float* out) {
+  int groups = colsum_groups(rows);
+  int threads = CS_ROWLANES * 32;
+  if (c.dtype == 0) {
+    dim3 grid(ceil_div(cols, 32 * 4), groups);
+    colsum_kernel<float><<<grid, threads, 0, c.stream>>>((const float*)x, rows, cols, partials);
+  } else {
+    dim3 grid(ceil_div(cols, 32 * 8), groups);
+    colsum_kernel<bf16><<<grid, threads, 0, c.stream>>>((const bf16*)x, rows, cols, partials);
+  }
+  reduce_partials_kernel<<<ceil_div(cols, 256), 256, 0, c.stream>>>(partials, groups, cols, out);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Classification head on the normalised classification token, cross-entropy, head backward.
+// ------------------------------------------------------------------------------------------------
+struct HeadDev {
+  int num_tasks, cmax, D;
+  int ncls[4];
+  const void* w[4];
+  const float* bias[4];
+  float* dw[4];
+  float* db[4];
+};
+
+template <typename T>
+__global__ void head_fwd_kernel(HeadDev h, const float* __restrict__ xn, const int* __restrict__ task_ids,
+                                float* __restrict__ logits, int B) {
+  int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= B * h.cmax) return;
+  int b = warp / h.cmax, cls = warp % h.cmax;
+  int t = task_ids ? task_ids[b] : 0;
+  if (cls >= h.ncls[t]) {
+    if (lane == 0) logits[warp] = -INFINITY;
+    return;
+  }
+  const T* w = (const T*)h.w[t] + (size_t)cls * h.D;
+  const float* xr = xn + (size_t)b * h.D;
+  float s = 0.f;
+  for (int d = lane; d < h.D; d += 32) s += xr[d] * to_f(w[d]);
+  s = warp_sum(s);
+  if (lane == 0) logits[warp] = s + h.bias[t][cls];
+}
+
+static HeadDev to_dev(const HeadDesc& h) {
+  HeadDev d;
+  d.num_tasks = h.num_tasks; d.cmax = h.cmax; d.D = h.D;
+  for (int i = 0; i < 4; ++i) { d.ncls[i] = h.ncls[i]; d.w[i] = h.w[i]; d.bias[i] = h.bias[i]; d.dw[i] = h.dw[i]; d.db[i] = h.db[i]; }
+  return d;
+}
+
+void head_fwd(const Ctx& c, const HeadDesc& h, const float* xn, const int* task_ids, float* logits, int B) {
+  int threads = 256, blocks = ceil_div((long)B * h.cmax * 32, threads);
+  if (c.dtype == 0) head_fwd_kernel<float><<<blocks, threads, 0, c.stream>>>(to_dev(h), xn, task_ids, logits, B);
+  else head_fwd_kernel<bf16><<<blocks, threads, 0, c.stream>>>(to_dev(h), xn, task_ids, logits, B);
+}
+
+// One warp per image: loss_b = logsumexp(logits) - logits[label]; dlogits = (softmax - onehot) / B.
+__global__ void cross_entropy_kernel(HeadDev h, const float* __restrict__ logits, const int* __restrict__ labels,
+                                     const int* __restrict__ task_ids, float* __restrict__ per_image,
+                                     float* __restrict__ dlogits, int B) {
+  int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= B) return;
+  int t = task_ids ? task_ids[warp] : 0;
+  int n = h.ncls[t];
+  const float* lr = logits + (size_t)warp * h.cmax;
+  float mx = -INFINITY;
+  for (int i = lane; i < n; i += 32) mx = fmaxf(mx, lr[i]);
+  mx = warp_max(mx);
+  float se = 0.f;
+  for (int i = lane; i < n; i += 32) se += expf(lr[i] - mx);
+  se = warp_sum(se);
+  int label = labels[warp];
+  float inv = 1.0f / se, invB = 1.0f / (float)B;
+  for (int i = lane; i < h.cmax; i += 32) {
+    float g = 0.f;
+    if (i < n) g = (expf(lr[i] - mx) * inv - (i == label ? 1.f : 0.f)) * invB;
+    dlogits[(size_t)warp * h.cmax + i] = g;
+  }
+  if (lane == 0) per_image[warp] = logf(se) + mx - lr[label];
+}
+
+// Single warp: mean of the per-image losses, lanes stride the images, fixed order.
+__global__ void loss_reduce_kernel(const float* __restrict__ per_image, int B, float* __restrict__ loss, int* status) {
+  int lane = threadIdx.x;
+  float s = 0.f;
+  for (int i = lane; i < B; i += 32) s += per_image[i];
+  s = warp_sum(s);
+  if (lane == 0) {
+    float l = s / (float)B;
+    *loss = l;
+    if (status != nullptr && !isfinite(l)) atomicOr(status, STATUS_NONFINITE);
+  }
+}
+
+void cross_entropy(const Ctx& c, const HeadDesc& h, const float* logits, const int* labels, const int* task_ids,
+                   float* per_image, float* dlogits, float* loss, int B) {
+  int threads = 128, blocks = ceil_div((long)B * 32, threads);
+  cross_entropy_kernel<<<blocks, threads, 0, c.stream>>>(to_dev(h), logits, labels, task_ids, per_image, dlogits, B);
+  loss_reduce_kernel<<<1, 32, 0, c.stream>>>(per_image, B, loss, c.status);
+}
+
+// dW_t[c, d] = sum_b [task(b) = t] dlogits[b, c] xn[b, d];  db_t[c] = sum_b [..] dlogits[b, c]
+__global__ void head_wgrad_kernel(HeadDev h, const float* __restrict__ xn, const float* __restrict__ dlogits,
+                                  const int* __restrict__ task_ids, int B, int t) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  int n = h.ncls[t];
+  if (i >= n * (h.D + 1)) return;
+  int cls = i / (h.D + 1), d = i % (h.D + 1);
+  float s = 0.f;
+  for (int b = 0; b < B; ++b) {
+    int tb = task_ids ? task_ids[b] : 0;
+    if (tb != t) continue;
+    float g = dlogits[(size_t)b * h.cmax + cls];
+    s += (d < h.D) ? g * xn[(size_t)b * h.D + d] : g;
+  }
+  if (d < h.D) h.dw[t][(size_t)cls * h.D + d] = s;
+  else h.db[t][cls] = s;
+}
+
+template <typename T>
+__global__ void head_dgrad_kernel(HeadDev h, const float* __restrict__ dlogits, const int* __restrict__ task_ids,
+                                  float* __restrict__ dxn, int B) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= B * h.D) return;
+  int b = i / h.D, d = i % h.D;
+  int t = task_ids ? task_ids[b] : 0;
+  const T* w = (const T*)h.w[t];
+  float s = 0.f;
+  for (int cidx = 0; cidx < h.ncls[t]; ++cidx) s += dlogits[(size_t)b * h.cmax + cidx] * to_f(w[(size_t)cidx * h.D + d]);
+  dxn[i] = s;
+}
+
+void head_bwd(const Ctx& c, const HeadDesc& h, const float* xn, const float* dlogits, const int* task_ids, float* dxn, int B) {
+  HeadDev hd = to_dev(h);
+  for (int t = 0; t < h.num_tasks; ++t) {
+    int total = h.ncls[t] * (h.D + 1);
+    head_wgrad_kernel<<<ceil_div(total, 128), 128, 0, c.stream>>>(hd, xn, dlogits, task_ids, B, t);
+  }
+  int total = B * h.D;
+  if (c.dtype == 0) head_dgrad_kernel<float><<<ceil_div(total, 128), 128, 0, c.stream>>>(hd, dlogits, task_ids, dxn, B);
+  else head_dgrad_kernel<bf16><<<ceil_div(total, 128), 128, 0, c.stream>>>(hd, dlogits, task_ids, dxn, B);
+}
+
+// ------------------------------------------------------------------------------------------------
+// AdamW over the flat trainable-parameter buffers (Section 5: DeiT-S is trained with AdamW).
+//   m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2;  p <- p - lr * (m/bc1) / (sqrt(v/bc2) + eps) - lr * wd * p
+// One block per chunk; a chunk never straddles two tensors.
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void adamw_kernel(const AdamChunk* __restrict__ chunks, float* __restrict__ master,
+                             const float* __restrict__ grad, float* __restrict__ m, float* __restrict__ v,
+                             T* __restrict__ shadow_base, float lr, float b1, float b2, float eps, float wd,
+                             float bc1, float bc2) {
+  AdamChunk ch = chunks[blockIdx.x];
+  float decay = ch.decay ? lr * wd : 0.f;
+  for (uint32_t i = threadIdx.x; i < ch.count; i += blockDim.x) {
+    size_t idx = (size_t)ch.offset + i;
+    float g = grad[idx];
+    float p = master[idx];
+    float mm = b1 * m[idx] + (1.f - b1) * g;
+    float vv = b2 * v[idx] + (1.f - b2) * g * g;
+    m[idx] = mm;
+    v[idx] = vv;
+    float np = p - lr * (mm / bc1) / (sqrtf(vv / bc2) + eps) - decay * p;
+    master[idx] = np;
+    if (ch.shadow >= 0) shadow_base[ch.shadow + i] = from_f<T>(np);
+  }
+}
+
+void adamw(const Ctx& c, const AdamChunk* chunks, int nchunks, float* master, const float* grad, float* m, float* v,
+           void* shadow_base, float lr, float b1, float b2, float eps, float wd, float bc1, float bc2) {
+  if (nchunks <= 0) return;
+  if (c.dtype == 0)
+    adamw_kernel<float><<<nchunks, 256, 0, c.stream>>>(chunks, master, grad, m, v, (float*)shadow_base, lr, b1, b2, eps, wd, bc1, bc2);
+  else
+    adamw_kernel<bf16><<<nchunks, 256, 0, c.stream>>>(chunks, master, grad, m, v, (bf16*)shadow_base, lr, b1, b2, eps, wd, bc1, bc2);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Conversions
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void from_float_kernel(const float* __restrict__ s, T* __restrict__ d, size_t n) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) d[i] = from_f<T>(s[i]);
+}
+template <typename T>
+__global__ void to_float_kernel(const T* __restrict__ s, float* __restrict__ d, size_t n) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) d[i] = to_f(s[i]);
+}
+__global__ void fill_kernel(float* d, float v, size_t n) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) d[i] = v;
+}
+
+void convert_from_float(const Ctx& c, const float* src, void* dst, size_t n) {
+  if (n == 0) return;
+  int blocks = ceil_div((long)n, 256);
+  if (c.dtype == 0) from_float_kernel<float><<<blocks, 256, 0, c.stream>>>(src, (float*)dst, n);
+  else from_float_kernel<bf16><<<blocks, 256, 0, c.stream>>>(src, (bf16*)dst, n);
+}
+void convert_to_float(const Ctx& c, const void* src, float* dst, size_t n) {
+  if (n == 0) return;
+  int blocks = ceil_div((long)n, 256);
+  if (c.dtype == 0) to_float_kernel<float><<<blocks, 256, 0, c.stream>>>((const float*)src, dst, n);
+  else to_float_kernel<bf16><<<blocks, 256, 0, c.stream>>>((const bf16*)src, dst, n);
+}
+void fill_float(cudaStream_t s, float* dst, float v, size_t n) {
+  if (n == 0) return;
+  fill_kernel<<<ceil_div((long)n, 256), 256, 0, s>>>(dst, v, n);
+}
+
+}  // namespace bsr

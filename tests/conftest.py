@@ -24,3 +24,12 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def native_library():
+    """Builds libbsr.so in-tree when it is missing and nvcc is present (cross-compiles without a GPU)."""
+    from paper_2405_10951_b200 import binding, build
+    if not os.path.exists(binding.LIB_PATH):
+        build.build()
+    yield

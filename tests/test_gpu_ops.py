@@ -1,0 +1,70 @@
+"""Unit parity of the dense kernels (linear layers, attention) against the oracle's definitions."""
+import numpy as np
+import pytest
+
+from oracle import bsr_oracle as O
+from paper_2405_10951_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def rel(a, b):
+    return float(np.linalg.norm(a - b) / np.linalg.norm(b))
+
+
+def linear_case(m, n, k, dtype, gelu, use_tc, with_res=True):
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    rng = np.random.default_rng(m + 3 * n + 7 * k)
+    x, w = rng.standard_normal((m, k)), rng.standard_normal((n, k)) / np.sqrt(k)
+    bias, res = rng.standard_normal(n), rng.standard_normal((m, n))
+    if dtype == "bf16":
+        x, w, res = synth.round_to_bf16(x), synth.round_to_bf16(w), synth.round_to_bf16(res)
+    y = O.linear(x, w, bias)
+    if gelu:
+        y = O.gelu(y)
+    if with_res:
+        y = y + res
+    tdt = torch.float32 if dtype == "fp32" else torch.bfloat16
+    g = lambda a: torch.as_tensor(a.astype(np.float32)).cuda().to(tdt)
+    out = Bd.bsr_linear_forward(g(x), g(w), torch.as_tensor(bias.astype(np.float32)).cuda(), g(res) if with_res else None,
+                                act_gelu=gelu, use_tensor_cores=use_tc)
+    torch.cuda.synchronize()
+    return rel(out.float().cpu().numpy().astype(np.float64), y)
+
+
+@pytest.mark.parametrize("m,n,k", [(65, 192, 192), (130, 100, 72), (520, 768, 192), (8, 10, 192), (333, 72, 40)])
+@pytest.mark.parametrize("gelu", [False, True])
+def test_linear_fp32(m, n, k, gelu):
+    assert linear_case(m, n, k, "fp32", gelu, False) < 2e-6
+
+
+@pytest.mark.parametrize("m,n,k", [(65, 192, 192), (520, 768, 192), (197, 384, 1536)])
+def test_linear_bf16_simt(m, n, k):
+    assert linear_case(m, n, k, "bf16", True, False) < 4e-3
+
+
+@pytest.mark.parametrize("dtype,tol", [("fp32", 2e-6), ("bf16", 4e-3)])
+@pytest.mark.parametrize("B,T,H,d", [(2, 65, 3, 64), (3, 47, 2, 32), (2, 197, 6, 64), (1, 5, 1, 16), (1, 290, 2, 64)])
+def test_attention_forward(dtype, tol, B, T, H, d):
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    if dtype == "fp32" and T > 200:
+        pytest.skip("fp32 rows of this length exceed the kernel's shared memory by design")
+    rng = np.random.default_rng(T * 31 + d)
+    qkv = rng.standard_normal((B, T, 3, H, d))
+    if dtype == "bf16":
+        qkv = synth.round_to_bf16(qkv)
+    q, k, v = (qkv[:, :, i].transpose(0, 2, 1, 3) for i in range(3))
+
+    class Cfg:
+        heads = H
+        dim = H * d
+    o, A = O.attention_fwd(Cfg, q, k, v)
+    want = O.merge_heads(o)
+    tdt = torch.float32 if dtype == "fp32" else torch.bfloat16
+    out, cp = Bd.bsr_attention_forward(torch.as_tensor(qkv.astype(np.float32)).cuda().to(tdt), H)
+    torch.cuda.synchronize()
+    assert rel(out.float().cpu().numpy().astype(np.float64), want) < tol
+    if T > 1:
+        assert rel(cp.cpu().numpy().astype(np.float64), A[:, :, 0, 1:]) < (2e-6 if dtype == "fp32" else 1e-5)

@@ -1,0 +1,110 @@
+"""The whole BSR step on the GPU (through the C ABI) against the float64 oracle."""
+import numpy as np
+import pytest
+
+from oracle import bsr_oracle as O
+from paper_2405_10951_b200 import synth
+from paper_2405_10951_b200.synth import CONFIGS, Config
+
+import parity as P
+
+pytestmark = pytest.mark.gpu
+
+TINY = CONFIGS["tiny_fp32"]
+MINI_BF16 = Config("mini_bf16", 64, 8, 128, 2, 6, 256, (10,), 6, (3, 4, 5), (1, 3, 4), 7, 10, dtype="bf16", seed=1)
+
+FP32_CASES = {
+    "tiny_config": TINY,
+    "trainable_drop_location": TINY.with_(trainable=(2, 3, 4, 5)),
+    "two_locations_no_fusion": TINY.with_(drop_blocks=(1, 4), fuse_mode=0, trainable=(3, 4, 5)),
+    "keep_one_all_trainable": TINY.with_(keep_num=1, keep_den=1, trainable=(0, 1, 2, 3, 4, 5)),
+    "head_only": TINY.with_(trainable=()),
+    "half_rate_three_locations": TINY.with_(drop_blocks=(1, 3, 5), keep_num=1, keep_den=2, trainable=(2, 3, 4, 5), batch=5),
+    "odd_shapes": Config("odd", 20, 4, 96, 3, 3, 136, (7,), 3, (1, 2), (0, 1), 2, 3, dtype="fp32", seed=4),
+}
+
+
+@pytest.mark.parametrize("peaked", [True, False])
+@pytest.mark.parametrize("case", list(FP32_CASES))
+def test_fp32_step_matches_oracle(case, peaked):
+    cfg = FP32_CASES[case]
+    images, labels, task_ids, params = synth.make_workload(cfg, peaked=peaked)
+    gpu = P.run_gpu_step(cfg, images, labels, task_ids, params)
+    rep = P.compare_step(cfg, images, labels, task_ids, params, gpu, P.FP32_TOL, P.EXACT_MARGIN, 1e-4)
+    if peaked and rep["sets"]:
+        assert rep["sets_identical"] == rep["sets"], rep
+
+
+BF16_CASES = {
+    "mini": MINI_BF16,
+    "mini_no_fusion": MINI_BF16.with_(fuse_mode=0),
+    "deit_s_batch4": CONFIGS["deit_s"].with_(batch=4),
+}
+
+
+@pytest.mark.parametrize("case", list(BF16_CASES))
+def test_bf16_step_matches_oracle(case):
+    cfg = BF16_CASES[case]
+    images, labels, task_ids, params = synth.make_workload(cfg, peaked=True)
+    gpu = P.run_gpu_step(cfg, images, labels, task_ids, params)
+    rep = P.compare_step(cfg, images, labels, task_ids, params, gpu, P.BF16_TOL, 10 * P.BF16_SCORE_TOL, P.BF16_SCORE_TOL)
+    assert rep["sets_identical"] >= 0.8 * rep["sets"], rep
+
+
+def test_eval_forward_matches_oracle_and_train_forward():
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    cfg = TINY.with_(trainable=(2, 3, 4, 5))
+    images, labels, task_ids, params = synth.make_workload(cfg, peaked=True)
+    eng = Bd.Engine(cfg)
+    eng.set_params(params)
+    logits, kept = eng.eval_forward(eng.images_to_device(images))
+    torch.cuda.synchronize()
+    ref = O.forward(cfg, params, images)
+    assert P.rel_err(logits.cpu().numpy(), ref["logits"]) < P.FP32_TOL
+    for a, b in zip(kept, ref["kept"]):
+        assert np.array_equal(a.cpu().numpy(), b)
+    # a smaller batch than max_batch
+    logits3, kept3 = eng.eval_forward(eng.images_to_device(images[:3]))
+    assert torch.equal(logits3, logits[:3])
+
+
+def test_two_steps_follow_the_oracle_and_are_deterministic():
+    cfg = TINY.with_(trainable=(2, 3, 4, 5), lr=1e-3)
+    images, labels, task_ids, params = synth.make_workload(cfg, peaked=True)
+    a = P.run_gpu_step(cfg, images, labels, task_ids, params, steps=2)
+    b = P.run_gpu_step(cfg, images, labels, task_ids, params, steps=2)
+    assert a["loss"] == b["loss"]
+    for n in a["grads"]:
+        assert np.array_equal(a["grads"][n], b["grads"][n]), n
+        assert np.array_equal(a["params"][n], b["params"][n]), n
+    o1 = O.train_step(cfg, params, images, labels, task_ids)
+    o2 = O.train_step(cfg, o1["params"], images, labels, task_ids, opt_state=o1["opt_state"], step=2)
+    assert abs(a["loss"] - o2["loss"]) < 2e-3 * abs(o2["loss"])      # second-step loss: after one (sign-like) update
+    assert o2["loss"] < o1["loss"]
+
+
+def test_error_paths_leave_the_context_usable():
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    cfg = TINY
+    eng = Bd.Engine(cfg, max_batch=4)
+    images, labels, task_ids, params = synth.make_workload(cfg)
+    eng.set_params(params)
+    img = eng.images_to_device(images)            # batch 8 > max_batch 4
+    lab = torch.as_tensor(labels).cuda()
+    with pytest.raises(Bd.BsrError) as e:
+        eng.train_step(img, lab)
+    assert e.value.status == -1
+    with pytest.raises(Bd.BsrError):
+        eng.set_param("blocks.0.nope", np.zeros(3))
+    with pytest.raises(Bd.BsrError):
+        eng.set_param("norm.weight", np.zeros(3))
+    with pytest.raises(Bd.BsrError):
+        eng.get_tensor("grad/blocks.0.norm1.weight", (cfg.dim,))     # frozen: no gradient exists
+    loss, _ = eng.train_step(img[:4], lab[:4])
+    eng.sync_status()
+    assert np.isfinite(float(loss.cpu()[0]))
+    fp = eng.footprint()
+    assert fp["saved_activation_bytes"] > 0 and fp["trainable_params"] == sum(
+        int(np.prod(synth.param_shapes(cfg)[n])) for n in O.trainable_names(cfg, params))
