@@ -191,6 +191,15 @@ int32_t bsr_linear_forward(const void* x_dev, const void* w_dev, const float* bi
                            void* y_dev, int32_t m, int32_t n, int32_t k, int32_t dtype, int32_t act_gelu,
                            int32_t use_tensor_cores, void* stream);
 
+/* Backward of y = x W^T: dx = dy W (Eq. 2: needs only the weights) and dw = dy^T x (Eq. 4: needs the stored
+ * input).  x [m, k], w [n, k], dy [m, n], dx [m, k] in `dtype`; dw [n, k] float32.  With
+ * use_tensor_cores != 0 (bf16, m, n, k multiples of 8) the operands are read in place through
+ * transposing shared-memory descriptors; workspace_dev (float32, may be NULL) lets a long
+ * reduction over m be split and summed in a fixed order. */
+int32_t bsr_linear_backward(const void* x_dev, const void* w_dev, const void* dy_dev, void* dx_dev, float* dw_dev,
+                            int32_t m, int32_t n, int32_t k, int32_t dtype, int32_t use_tensor_cores,
+                            float* workspace_dev, size_t workspace_floats, void* stream);
+
 /* Multi-head self-attention, Eq. 1, on packed projections.  qkv_dev [batch, t, 3, heads, d] in
  * `dtype`; out_dev [batch, t, heads*d]; cls_prob_dev_out optional [batch, heads, t-1] float32: the
  * classification token's row of the attention map without its own column. d must be 64 or less

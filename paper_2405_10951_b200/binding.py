@@ -24,7 +24,8 @@ STATUS_NAMES = {0: "BSR_OK", -1: "BSR_ERR_INVALID_ARG", -2: "BSR_ERR_UNSUPPORTED
 
 EXPORTS = ["bsr_token_schedule", "bsr_workspace_bytes", "bsr_create", "bsr_destroy", "bsr_last_error", "bsr_set_param",
            "bsr_get_tensor", "bsr_set_lr", "bsr_set_step", "bsr_train_step", "bsr_eval_forward", "bsr_get_footprint",
-           "bsr_sync_status", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_attention_forward"]
+           "bsr_sync_status", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_backward",
+           "bsr_attention_forward"]
 
 
 class bsr_dims(C.Structure):
@@ -84,6 +85,7 @@ def lib() -> C.CDLL:
         L.bsr_token_select.argtypes = [f32p, i32, i32, i32, i32, f32p, i32p, i32p, vp]
         L.bsr_gather_fuse.argtypes = [vp, i32, i32, i32, i32, i32, i32p, i32p, f32p, i32, vp, vp]
         L.bsr_linear_forward.argtypes = [vp, vp, f32p, vp, vp, i32, i32, i32, i32, i32, i32, vp]
+        L.bsr_linear_backward.argtypes = [vp, vp, vp, vp, f32p, i32, i32, i32, i32, i32, f32p, C.c_size_t, vp]
         L.bsr_attention_forward.argtypes = [vp, i32, i32, i32, i32, i32, vp, f32p, vp]
         for name in EXPORTS:
             if name != "bsr_last_error":
@@ -177,6 +179,19 @@ def bsr_linear_forward(x, w, bias=None, residual=None, act_gelu: bool = False, u
     _check(lib().bsr_linear_forward(_ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(y), m, n, k, dt, int(act_gelu),
                                     int(use_tensor_cores), _stream()))
     return y
+
+
+def bsr_linear_backward(x, w, dy, use_tensor_cores: bool = False, workspace=None):
+    """Returns (dx [m, k] in x's dtype, dw [n, k] float32)."""
+    import torch
+    m, k = x.shape
+    n = w.shape[0]
+    dx = torch.empty((m, k), dtype=x.dtype, device=x.device)
+    dw = torch.empty((n, k), dtype=torch.float32, device=x.device)
+    dt = DTYPE_FP32 if x.dtype == torch.float32 else DTYPE_BF16
+    _check(lib().bsr_linear_backward(_ptr(x), _ptr(w), _ptr(dy), _ptr(dx), _ptr(dw), m, n, k, dt, int(use_tensor_cores),
+                                     _ptr(workspace), 0 if workspace is None else workspace.numel(), _stream()))
+    return dx, dw
 
 
 def bsr_attention_forward(qkv, heads: int, want_cls_prob: bool = True):

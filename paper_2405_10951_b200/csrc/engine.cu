@@ -154,6 +154,7 @@ struct bsr_handle {
   size_t off_escore = 0, off_delta = 0, off_ln_partials = 0, off_cs_partials = 0;
   size_t off_kept_all = 0;
   size_t off_stage = 0;
+  size_t off_split = 0, split_floats = 0;
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(base + off); }
   void* w(const char* name) const {
@@ -340,6 +341,8 @@ size_t plan(bsr_handle* h) {
   size_t biggest = 0;
   for (auto& t : h->tensors) biggest = t.numel > biggest ? t.numel : biggest;
   h->off_stage = b.take(biggest * 4);
+  h->split_floats = (d.dtype == BSR_DTYPE_BF16) ? (size_t)160 * 128 * 256 : 0;   // one 128x256 fp32 tile per SM
+  h->off_split = b.take(h->split_floats * 4);
   h->scratch_bytes = b.off - s0;
   return b.off;
 }
@@ -351,6 +354,8 @@ Ctx make_ctx(const bsr_handle* h, void* stream) {
   c.status = h->at<int>(h->off_status);
   c.sm_count = h->sm_count;
   c.use_tc = h->use_tc;
+  c.split_ws = h->split_floats ? h->at<float>(h->off_split) : nullptr;
+  c.split_ws_floats = h->split_floats;
   return c;
 }
 
@@ -500,7 +505,7 @@ int forward_all(bsr_handle* h, const Ctx& c, const void* images, int B, bool tra
       bb = h->bufs_train[l];
     } else {
       bb = h->bufs_frozen[l & 1];
-      if (l + 1 == first_train) bb.x_out = h->bufs_train[l + 1].x_in;   // hand over to the first trainable block
+      if (l + 1 == first_train && first_train < d.depth) bb.x_out = h->bufs_train[l + 1].x_in;   // hand over to the first trainable block
     }
     bb.x_in = cur;
     int* kept_dst = nullptr;
@@ -859,6 +864,25 @@ int32_t bsr_linear_forward(const void* x, const void* w, const float* bias, cons
     gemm(c, x, k, 1, w, k, 1, y, 0, m, n, k, e);
   }
   return check_cuda(nullptr, "bsr_linear_forward");
+}
+
+int32_t bsr_linear_backward(const void* x, const void* w, const void* dy, void* dx, float* dw, int32_t m, int32_t n, int32_t k,
+                            int32_t dtype, int32_t use_tensor_cores, float* workspace, size_t workspace_floats, void* stream) {
+  if (x == nullptr || w == nullptr || dy == nullptr || dx == nullptr || dw == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "null argument");
+  if (dtype != BSR_DTYPE_FP32 && dtype != BSR_DTYPE_BF16) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad dtype");
+  if (m < 1 || n < 1 || k < 1) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad shape");
+  Ctx c = bare_ctx(dtype, stream);
+  GemmEpilogue none;
+  if (use_tensor_cores) {
+    if (dtype != BSR_DTYPE_BF16 || (m % 8) || (n % 8) || (k % 8)) return set_err(g_error, BSR_ERR_UNSUPPORTED, "the tcgen05 kernels need bf16 and m, n, k multiples of 8");
+    int rc = gemm_tc_strided(c, dy, n, 1, w, 1, k, dx, 0, m, k, n, none, nullptr, 0);                       // dX = dY W
+    if (rc == 0) rc = gemm_tc_strided(c, dy, 1, n, x, 1, k, dw, 1, n, k, m, none, workspace, workspace_floats);   // dW = dY^T X
+    if (rc != 0) return set_err(g_error, BSR_ERR_CUDA, "tcgen05 GEMM set-up failed (%d)", rc);
+  } else {
+    gemm(c, dy, n, 1, w, 1, k, dx, 0, m, k, n, none);
+    gemm(c, dy, 1, n, x, 1, k, dw, 1, n, k, m, none);
+  }
+  return check_cuda(nullptr, "bsr_linear_backward");
 }
 
 int32_t bsr_attention_forward(const void* qkv, int32_t dtype, int32_t batch, int32_t t, int32_t heads, int32_t d, void* out,

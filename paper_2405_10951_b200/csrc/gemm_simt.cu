@@ -78,8 +78,8 @@ gemm_simt_kernel(const T* __restrict__ A, long a_rs, long a_cs, const T* __restr
 void gemm(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long b_rs, long b_cs, void* C,
           int out_is_float, int m, int n, int k, const GemmEpilogue& e) {
   if (m <= 0 || n <= 0) return;
-  if (c.dtype == 1 && c.use_tc && !out_is_float && a_cs == 1 && b_cs == 1 && a_rs == k && b_rs == k && gemm_tc_supported(m, n, k)) {
-    if (gemm_tc(c, A, B, C, out_is_float, m, n, k, e) == 0) return;
+  if (c.dtype == 1 && c.use_tc && gemm_tc_supported(m, n, k)) {
+    if (gemm_tc_strided(c, A, a_rs, a_cs, B, b_rs, b_cs, C, out_is_float, m, n, k, e, c.split_ws, c.split_ws_floats) == 0) return;
   }
   dim3 grid(ceil_div(n, SG_BN), ceil_div(m, SG_BM));
   if (c.dtype == 0) {

@@ -1,7 +1,436 @@
-// placeholder until the tcgen05 kernel lands
+// bf16 dense contraction on the 5th-generation tensor cores (sm_100a): TMA -> 128B-swizzled shared
+// memory ring -> tcgen05.mma accumulating fp32 in tensor memory -> tcgen05.ld epilogue.
+//
+//   C[m, n] = epilogue( sum_k A(m, k) * B(n, k) )
+//
+// Each operand may be contiguous along k ("K-major", the forward layers: activations [m, k] and
+// weights [n, k]) or along its own index ("MN-major": the weight in the input-gradient product
+// dX = dY W, and both operands of the weight-gradient product dW = dY^T X, Eq. 2 and Eq. 4 of the
+// paper).  No operand is transposed in memory; the shared-memory descriptors say how to read it.
+//
+// Kernel shape: persistent, one CTA per SM, 128 x 256 output tiles, k in slabs of 64.
+//   warp 0      : TMA producer (one lane)
+//   warp 1      : tensor-memory allocation, MMA issue (one lane)
+//   warps 2..5  : epilogue, one TMEM lane quarter each; two accumulator buffers of 256 columns let
+//                 the epilogue of one tile overlap the main loop of the next.
+// Every wait is bounded: on expiry the CTA raises STATUS_TIMEOUT in the status word, gives the
+// copies it issued time to land, frees its tensor memory and returns.
+#include <cuda.h>
+
 #include "common.cuh"
 #include "kernels.h"
+
 namespace bsr {
-bool gemm_tc_supported(int, int, int) { return false; }
-int gemm_tc(const Ctx&, const void*, const void*, void*, int, int, int, int, const GemmEpilogue&) { return -1; }
+
+namespace tc {
+
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int STAGES = 4;
+constexpr int UMMA_K = 16;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int THREADS = 192;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr unsigned long long WAIT_NS = 2000000000ull;   // 2 s
+
+struct Epi {
+  const float* bias;
+  const void* residual;
+  void* aux_out;
+  const void* aux_in;
+  int act;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false when it gave up (or another role already did).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (int i = 0; i < 4096; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  unsigned long long t0 = global_ns();
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > WAIT_NS) { *abort_flag = 1; return false; }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  K-major operand: rows of 128 bytes (64 bf16 along k),
+// groups of 8 rows 1024 bytes apart (SBO).  MN-major operand: rows of 128 bytes run along m/n, a row per k,
+// groups of 8 k-rows 1024 bytes apart (SBO), successive 64-element m/n chunks LBO bytes apart.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(lbo_bytes >> 4) << 16;
+  d |= (uint64_t)(sbo_bytes >> 4) << 32;
+  d |= (uint64_t)1 << 46;      // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;      // 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: D = f32, A = B = bf16, M = 128, N = 256, operand majors as given.
+__host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+template <typename TOut> __device__ __forceinline__ void store8(TOut* p, const float* v);
+template <> __device__ __forceinline__ void store8<bf16>(bf16* p, const float* v) { store16(p, v); }
+template <> __device__ __forceinline__ void store8<float>(float* p, const float* v) { store16(p, v); store16(p + 4, v + 4); }
+template <typename TOut> __device__ __forceinline__ void load8(const TOut* p, float* v);
+template <> __device__ __forceinline__ void load8<bf16>(const bf16* p, float* v) { load16(p, v); }
+template <> __device__ __forceinline__ void load8<float>(const float* p, float* v) { load16(p, v); load16(p + 4, v + 4); }
+
+template <bool A_MN, bool B_MN, typename TOut>
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TOut* __restrict__ C,
+               int M, int N, int K, Epi ep, int tiles_m, int tiles_n, int splits, int kb_per_split, int* status) {
+  extern __shared__ unsigned char smem_dyn[];
+  uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  uint32_t bars = base + STAGES * STAGE_BYTES;           // full[STAGES], empty[STAGES], tfull[2], tempty[2]
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
+  auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int total_kb = (K + BK - 1) / BK;
+  int work_items = tiles_m * tiles_n * splits;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  uint32_t tmem_base = tmem_base_slot;
+  volatile int* abortp = &abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------- TMA producer -------------------------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int armed = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; w < work_items && ok; w += gridDim.x) {
+        int mt = w % tiles_m, nt = (w / tiles_m) % tiles_n, sp = w / (tiles_m * tiles_n);
+        int kb0 = sp * kb_per_split, kb1 = min(total_kb, kb0 + kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abortp)) { ok = false; break; }
+          mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+          uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
+          if (!A_MN) {
+            tma_load_2d(sa, &map_a, full_bar(stage), kb * BK, mt * BM);
+          } else {
+#pragma unroll
+            for (int j = 0; j < BM / 64; ++j) tma_load_2d(sa + j * (BK * 128), &map_a, full_bar(stage), mt * BM + j * 64, kb * BK);
+          }
+          if (!B_MN) {
+            tma_load_2d(sb, &map_b, full_bar(stage), kb * BK, nt * BN);
+          } else {
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * (BK * 128), &map_b, full_bar(stage), nt * BN + j * 64, kb * BK);
+          }
+          ++armed;
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok && armed > 0) {
+        // copies already issued still land in shared memory: give them a bounded time before the CTA leaves
+        unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 1000000ull) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer ---------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(A_MN, B_MN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; w < work_items && ok; w += gridDim.x, ++local) {
+        int sp = w / (tiles_m * tiles_n);
+        int kb0 = sp * kb_per_split, kb1 = min(total_kb, kb0 + kb_per_split);
+        int buf = local & 1;
+        if (!mbar_wait(tempty_bar(buf), ((local >> 1) & 1) ^ 1u, abortp)) { ok = false; break; }
+        tc_fence_after();
+        uint32_t d_tmem = tmem_base + buf * BN;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abortp)) { ok = false; break; }
+          tc_fence_after();
+          uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            uint64_t da = A_MN ? make_desc(sa + k * (UMMA_K * 128), BK * 128, 1024) : make_desc(sa + k * (UMMA_K * 2), 16, 1024);
+            uint64_t db = B_MN ? make_desc(sb + k * (UMMA_K * 128), BK * 128, 1024) : make_desc(sb + k * (UMMA_K * 2), 16, 1024);
+            umma_bf16(d_tmem, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit(empty_bar(stage));
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit(tfull_bar(buf));
+      }
+    }
+  } else {
+    // ------------------------------- epilogue -----------------------------------
+    int quarter = warp & 3;                 // TMEM lanes 32*quarter .. 32*quarter+31
+    int local = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < work_items && ok; w += gridDim.x, ++local) {
+      int mt = w % tiles_m, nt = (w / tiles_m) % tiles_n, sp = w / (tiles_m * tiles_n);
+      int buf = local & 1;
+      if (!mbar_wait(tfull_bar(buf), (local >> 1) & 1, abortp)) { ok = false; break; }
+      tc_fence_after();
+      int row = mt * BM + quarter * 32 + lane;
+      TOut* crow = C + (size_t)sp * M * N + (size_t)row * N;
+#pragma unroll 1
+      for (int cchunk = 0; cchunk < BN / 32; ++cchunk) {
+        uint32_t r[32];
+        uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cchunk * 32);
+        tmem_ld32(taddr, r);
+        tmem_ld_wait();
+        int col0 = nt * BN + cchunk * 32;
+        if (row < M && col0 < N) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            int col = col0 + g * 8;
+            if (col < N) {
+              float v[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[g * 8 + j]);
+              if (ep.bias != nullptr) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] += __ldg(ep.bias + col + j);
+              }
+              if (ep.act == 1) {
+                if (ep.aux_out != nullptr) store8<TOut>((TOut*)ep.aux_out + (size_t)row * N + col, v);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] = gelu_f(v[j]);
+              } else if (ep.act == 2) {
+                float z[8];
+                load16((const bf16*)ep.aux_in + (size_t)row * N + col, z);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] *= gelu_grad_f(z[j]);
+              }
+              if (ep.residual != nullptr) {
+                float rr[8];
+                load8<TOut>((const TOut*)ep.residual + (size_t)row * N + col, rr);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] += rr[j];
+              }
+              store8<TOut>(crow + col, v);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(buf));
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && abort_flag && status != nullptr) atomicOr(status, STATUS_TIMEOUT);
+}
+
+// out[i] = sum over splits of partial[s][i], ascending s.
+__global__ void splitk_reduce_kernel(const float* __restrict__ partial, float* __restrict__ out, size_t n, int splits) {
+  size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i >= n) return;
+  float4 acc = *reinterpret_cast<const float4*>(partial + i);
+  for (int s = 1; s < splits; ++s) {
+    float4 v = *reinterpret_cast<const float4*>(partial + (size_t)s * n + i);
+    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+  }
+  *reinterpret_cast<float4*>(out + i) = acc;
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeFn encode_fn() {
+  static EncodeFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+      fn = (EncodeFn)p;
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor map: `inner` contiguous elements per row, `outer` rows `ld` elements apart, box {64, box_outer}.
+static bool make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t outer, uint64_t ld, uint32_t box_outer) {
+  EncodeFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {64, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool A_MN, bool B_MN, typename TOut>
+static int launch(const Ctx& c, const CUtensorMap& ma, const CUtensorMap& mb, void* C, int m, int n, int k, const Epi& ep,
+                  int tiles_m, int tiles_n, int splits, int kb_per_split) {
+  auto kern = gemm_tc_kernel<A_MN, B_MN, TOut>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return -3;
+    attr_set = true;
+  }
+  int work = tiles_m * tiles_n * splits;
+  int sms = c.sm_count > 0 ? c.sm_count : 148;
+  int grid = work < sms ? work : sms;
+  kern<<<grid, THREADS, SMEM_BYTES, c.stream>>>(ma, mb, (TOut*)C, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, c.status);
+  return 0;
+}
+
+}  // namespace tc
+
+bool gemm_tc_supported(int m, int n, int k) { return m >= 1 && n >= 8 && k >= 8 && (n % 8) == 0 && (k % 8) == 0; }
+
+// Strides as in gemm(): A(m,k) = A[m*a_rs + k*a_cs].  One of (a_rs, a_cs) must be 1, likewise for B.
+int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long b_rs, long b_cs, void* C,
+                    int out_is_float, int m, int n, int k, const GemmEpilogue& e, float* split_ws, size_t split_ws_floats) {
+  using namespace tc;
+  bool a_mn = (a_cs != 1), b_mn = (b_cs != 1);
+  if (a_mn && a_rs != 1) return -1;
+  if (b_mn && b_rs != 1) return -1;
+  long lda = a_mn ? a_cs : a_rs, ldb = b_mn ? b_cs : b_rs;
+  if ((lda % 8) != 0 || (ldb % 8) != 0 || ((uintptr_t)A & 15) || ((uintptr_t)B & 15) || ((uintptr_t)C & 15)) return -1;
+  if ((n % 8) != 0) return -1;
+  if (a_mn && (m % 8) != 0) return -1;
+  if (a_mn && !b_mn) return -1;                 // combination not instantiated
+  CUtensorMap ma, mb;
+  bool ok = a_mn ? make_map(&ma, A, (uint64_t)m, (uint64_t)k, (uint64_t)lda, BK) : make_map(&ma, A, (uint64_t)k, (uint64_t)m, (uint64_t)lda, BM);
+  ok = ok && (b_mn ? make_map(&mb, B, (uint64_t)n, (uint64_t)k, (uint64_t)ldb, BK) : make_map(&mb, B, (uint64_t)k, (uint64_t)n, (uint64_t)ldb, BN));
+  if (!ok) return -2;
+  int tiles_m = ceil_div(m, BM), tiles_n = ceil_div(n, BN);
+  int total_kb = ceil_div(k, BK);
+  int splits = 1;
+  bool plain = e.bias == nullptr && e.residual == nullptr && e.act == 0;
+  int sms = c.sm_count > 0 ? c.sm_count : 148;
+  if (out_is_float && plain && split_ws != nullptr && tiles_m * tiles_n * 2 <= sms && total_kb >= 8) {
+    splits = sms / (tiles_m * tiles_n);
+    if (splits > total_kb / 4) splits = total_kb / 4;
+    if (splits > 16) splits = 16;
+    while (splits > 1 && (size_t)splits * m * n > split_ws_floats) --splits;
+    if (splits < 1) splits = 1;
+  }
+  int kb_per_split = ceil_div(total_kb, splits);
+  splits = ceil_div(total_kb, kb_per_split);
+  Epi ep;
+  ep.bias = e.bias; ep.residual = e.residual; ep.aux_out = e.aux_out; ep.aux_in = e.aux_in; ep.act = e.act;
+  void* dst = (splits > 1) ? (void*)split_ws : C;
+  int rc;
+  if (out_is_float) {
+    if (a_mn) rc = launch<true, true, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split);
+    else if (b_mn) rc = launch<false, true, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split);
+    else rc = launch<false, false, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split);
+  } else {
+    if (a_mn) rc = launch<true, true, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split);
+    else if (b_mn) rc = launch<false, true, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split);
+    else rc = launch<false, false, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split);
+  }
+  if (rc != 0) return rc;
+  if (splits > 1) {
+    size_t total = (size_t)m * n;
+    splitk_reduce_kernel<<<ceil_div((long)(total / 4), 256), 256, 0, c.stream>>>(split_ws, (float*)C, total, splits);
+  }
+  return 0;
+}
+
+int gemm_tc(const Ctx& c, const void* A, const void* B, void* C, int out_is_float, int m, int n, int k, const GemmEpilogue& e) {
+  return gemm_tc_strided(c, A, k, 1, B, k, 1, C, out_is_float, m, n, k, e, nullptr, 0);
+}
+
+}  // namespace bsr

@@ -16,6 +16,8 @@ struct Ctx {
   int* status;      // device status word (may be null for the stand-alone entry points)
   int sm_count;
   int use_tc;       // bf16 only: dense contractions on the tcgen05 kernels
+  float* split_ws = nullptr;       // scratch for split-k partial sums (optional)
+  size_t split_ws_floats = 0;
 };
 
 inline size_t dtype_size(int dtype) { return dtype == 0 ? 4 : 2; }
@@ -56,6 +58,10 @@ void gemm(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long
 bool gemm_tc_supported(int m, int n, int k);
 int gemm_tc(const Ctx& c, const void* A, const void* B, void* C, int out_is_float, int m, int n, int k,
             const GemmEpilogue& e);
+// Same with operand strides as in gemm(); each operand contiguous along k or along its own index.  A problem
+// with few output tiles and a long k (weight gradients) is split along k into split_ws and reduced in order.
+int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long b_rs, long b_cs, void* C,
+                    int out_is_float, int m, int n, int k, const GemmEpilogue& e, float* split_ws, size_t split_ws_floats);
 
 // ---- attention --------------------------------------------------------------------------------
 // qkv [B, T, 3, H, d]; out [B, T, H*d]; lse (optional) [B, H, T] natural-log sum of exponentials of the

@@ -68,3 +68,48 @@ def test_attention_forward(dtype, tol, B, T, H, d):
     assert rel(out.float().cpu().numpy().astype(np.float64), want) < tol
     if T > 1:
         assert rel(cp.cpu().numpy().astype(np.float64), A[:, :, 0, 1:]) < (2e-6 if dtype == "fp32" else 1e-5)
+
+
+TC_SHAPES = [(128, 256, 64), (197, 384, 192), (1000, 3072, 768), (2600, 768, 3072), (100, 72, 40), (9216, 2304, 768)]
+
+
+@pytest.mark.parametrize("m,n,k", TC_SHAPES)
+@pytest.mark.parametrize("gelu", [False, True])
+def test_linear_bf16_tensor_cores(m, n, k, gelu):
+    """tcgen05 kernel, operands contiguous along k; tiles spanning several CTAs and ragged edges in m, n and k."""
+    assert linear_case(m, n, k, "bf16", gelu, True) < 4e-3
+    assert linear_case(m, n, k, "bf16", gelu, True, with_res=False) < 4e-3
+
+
+@pytest.mark.parametrize("m,n,k,ws", [(128, 256, 64, False), (200, 384, 192, False), (1024, 768, 384, True),
+                                      (12800, 768, 768, True), (9216, 3072, 768, True), (72, 40, 104, False)])
+@pytest.mark.parametrize("tc", [False, True])
+def test_linear_backward_bf16(m, n, k, ws, tc):
+    """Input and weight gradients of a linear layer (Eq. 2 and Eq. 4), operands read in place (no transposes)."""
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    rng = np.random.default_rng(m + n + k)
+    x = synth.round_to_bf16(rng.standard_normal((m, k)))
+    w = synth.round_to_bf16(rng.standard_normal((n, k)) / np.sqrt(k))
+    dy = synth.round_to_bf16(rng.standard_normal((m, n)))
+    dx_ref, dw_ref, _ = O.linear_bwd(dy, x, w)
+    g = lambda a: torch.as_tensor(a.astype(np.float32)).cuda().to(torch.bfloat16)
+    wsb = torch.empty(160 * 128 * 256, dtype=torch.float32, device="cuda") if ws else None
+    dx, dw = Bd.bsr_linear_backward(g(x), g(w), g(dy), use_tensor_cores=tc, workspace=wsb)
+    torch.cuda.synchronize()
+    assert rel(dx.float().cpu().numpy().astype(np.float64), dx_ref) < 4e-3
+    assert rel(dw.cpu().numpy().astype(np.float64), dw_ref) < 1e-4
+
+
+def test_linear_backward_fp32():
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    rng = np.random.default_rng(3)
+    m, n, k = 130, 72, 100
+    x, w, dy = rng.standard_normal((m, k)), rng.standard_normal((n, k)), rng.standard_normal((m, n))
+    dx_ref, dw_ref, _ = O.linear_bwd(dy, x, w)
+    g = lambda a: torch.as_tensor(a.astype(np.float32)).cuda()
+    dx, dw = Bd.bsr_linear_backward(g(x), g(w), g(dy))
+    torch.cuda.synchronize()
+    assert rel(dx.cpu().numpy().astype(np.float64), dx_ref) < 2e-6
+    assert rel(dw.cpu().numpy().astype(np.float64), dw_ref) < 2e-6

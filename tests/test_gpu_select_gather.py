@@ -40,8 +40,7 @@ def test_gather_fuse_matches_oracle(dtype, B, M, D, k, fuse):
         pytest.skip("row not a multiple of 16 bytes")
     rng = np.random.default_rng(M * 7 + D)
     x = rng.standard_normal((B, M + 1, D))
-    if dtype == "bf16":
-        x = synth.round_to_bf16(x)
+    x = synth.round_to_bf16(x) if dtype == "bf16" else x.astype(np.float32).astype(np.float64)
     p = synth.make_scores(rng, B, 2, M)
     s = O.head_mean_scores(p, np.float32)
     kept = np.stack([O.select_tokens(s[b], k)[0] for b in range(B)])
