@@ -47,6 +47,23 @@ __device__ __forceinline__ void store16(bf16* p, const float* f) {
   *reinterpret_cast<uint4*>(p) = v;
 }
 
+// four consecutive elements (16 bytes of float, 8 bytes of bf16)
+__device__ __forceinline__ void load4(const float* p, float* f) { load16(p, f); }
+__device__ __forceinline__ void load4(const bf16* p, float* f) {
+  uint2 v = *reinterpret_cast<const uint2*>(p);
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+  float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
+  f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y;
+}
+__device__ __forceinline__ void store4(float* p, const float* f) { store16(p, f); }
+__device__ __forceinline__ void store4(bf16* p, const float* f) {
+  uint2 v;
+  __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&v);
+  h[0] = __floats2bfloat162_rn(f[0], f[1]);
+  h[1] = __floats2bfloat162_rn(f[2], f[3]);
+  *reinterpret_cast<uint2*>(p) = v;
+}
+
 // N consecutive elements (N = 4 or 8) through 16-byte accesses, whatever the element type.
 template <int N> __device__ __forceinline__ void load_n(const float* p, float* f) {
 #pragma unroll

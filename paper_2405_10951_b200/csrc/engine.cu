@@ -151,6 +151,7 @@ struct bsr_handle {
   size_t off_patches = 0, off_emb = 0;
   size_t off_xn = 0, off_meanf = 0, off_rstdf = 0, off_logits = 0, off_per_image = 0, off_dlogits = 0, off_dxn = 0;
   size_t off_dxa = 0, off_dxb = 0, off_dz = 0, off_dy = 0, off_dxg = 0, off_dxp = 0, off_do = 0, off_dqkv = 0;
+  size_t off_dxa_c = 0, off_dxb_c = 0, off_dxg_c = 0, off_dxp_c = 0;
   size_t off_escore = 0, off_delta = 0, off_ln_partials = 0, off_cs_partials = 0;
   size_t off_kept_all = 0;
   size_t off_stage = 0;
@@ -258,14 +259,14 @@ size_t plan(bsr_handle* h) {
     BlockBufs& bb = h->bufs_train[l];
     size_t Ma = (size_t)Bm * s.ta[l], Mf = (size_t)Bm * s.tf[l];
     bool drop = s.k[l] >= 0 && s.tf[l] != s.ta[l];
-    bb.x_in = (l == h->t0) ? b.take(Ma * D * es) : next_in;
+    bb.x_in = (l == h->t0) ? b.take(Ma * D * 4) : next_in;       // residual stream: float
     bb.mean1 = b.take(Ma * 4); bb.rstd1 = b.take(Ma * 4);
     bb.y1 = b.take(Ma * D * es);
     bb.qkv = b.take(Ma * 3 * D * es);
     bb.lse = b.take((size_t)Bm * H * s.ta[l] * 4);
     bb.o = b.take(Ma * D * es);
-    bb.xp = b.take(Mf * D * es);
-    bb.xp_full = drop ? b.take(Ma * D * es) : bb.xp;
+    bb.xp = b.take(Mf * D * 4);
+    bb.xp_full = drop ? b.take(Ma * D * 4) : bb.xp;
     if (s.k[l] >= 0) {
       bb.p = b.take((size_t)Bm * H * (s.ta[l] - 1) * 4);
       bb.s = b.take((size_t)Bm * (s.ta[l] - 1) * 4);
@@ -276,7 +277,7 @@ size_t plan(bsr_handle* h) {
     bb.y2 = b.take(Mf * D * es);
     bb.z = b.take(Mf * F * es);
     bb.hh = b.take(Mf * F * es);
-    bb.x_out = b.take(Mf * D * es);
+    bb.x_out = b.take(Mf * D * 4);
     next_in = bb.x_out;
   }
   h->arena_bytes = b.off - a0;
@@ -285,7 +286,7 @@ size_t plan(bsr_handle* h) {
   size_t M0 = (size_t)Bm * T0;
   h->off_patches = b.take((size_t)Bm * N * d.in_chans * d.patch_size * d.patch_size * es);
   h->off_emb = b.take((size_t)Bm * N * D * es);
-  size_t xa = b.take(M0 * D * es), xb = b.take(M0 * D * es);
+  size_t xa = b.take(M0 * D * 4), xb = b.take(M0 * D * 4);
   for (int i = 0; i < 2; ++i) {
     BlockBufs& bb = h->bufs_frozen[i];
     bb.x_in = i == 0 ? xa : xb;
@@ -297,8 +298,8 @@ size_t plan(bsr_handle* h) {
     bb.y1 = b.take(M0 * D * es);
     bb.qkv = b.take(M0 * 3 * D * es);
     bb.o = b.take(M0 * D * es);
-    bb.xp_full = b.take(M0 * D * es);
-    bb.xp = b.take(M0 * D * es);
+    bb.xp_full = b.take(M0 * D * 4);
+    bb.xp = b.take(M0 * D * 4);
     bb.y2 = bb.y1;
     bb.z = 0;
     bb.hh = b.take(M0 * F * es);
@@ -324,12 +325,18 @@ size_t plan(bsr_handle* h) {
   h->off_kept_all = b.take((kept_total + 1) * 4);
   if (h->t0 < d.depth) {
     size_t Mt = (size_t)Bm * s.ta[h->t0];
-    h->off_dxa = b.take(Mt * D * es);
-    h->off_dxb = b.take(Mt * D * es);
+    h->off_dxa = b.take(Mt * D * 4);            // gradient of the residual stream: float ...
+    h->off_dxb = b.take(Mt * D * 4);
+    h->off_dxg = b.take(Mt * D * 4);
+    h->off_dxp = b.take(Mt * D * 4);
+    if (d.dtype == BSR_DTYPE_BF16) {            // ... with a bf16 copy as GEMM operand
+      h->off_dxa_c = b.take(Mt * D * es);
+      h->off_dxb_c = b.take(Mt * D * es);
+      h->off_dxg_c = b.take(Mt * D * es);
+      h->off_dxp_c = b.take(Mt * D * es);
+    }
     h->off_dz = b.take(Mt * F * es);
     h->off_dy = b.take(Mt * D * es);
-    h->off_dxg = b.take(Mt * D * es);
-    h->off_dxp = b.take(Mt * D * es);
     h->off_do = b.take(Mt * D * es);
     h->off_dqkv = b.take(Mt * 3 * D * es);
     h->off_escore = b.take((size_t)Bm * s.ta[h->t0] * 4);
@@ -374,7 +381,9 @@ int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb
   int Ma = B * Ta, Mf = B * Tf;
   bool is_drop = k >= 0;
   bool shrinks = is_drop && Tf != Ta;
-  layernorm_fwd(c, h->base + bb.x_in, D, (const float*)h->wb(l, "norm1.weight"), (const float*)h->wb(l, "norm1.bias"),
+  Ctx cf = c;                // the residual stream is float whatever the storage dtype
+  cf.dtype = 0;
+  layernorm_fwd(c, h->at<float>(bb.x_in), D, (const float*)h->wb(l, "norm1.weight"), (const float*)h->wb(l, "norm1.bias"),
                 h->base + bb.y1, 0, save ? h->at<float>(bb.mean1) : nullptr, save ? h->at<float>(bb.rstd1) : nullptr, Ma, D, d.ln_eps);
   GemmEpilogue e1;
   e1.bias = (const float*)h->wb(l, "attn.qkv.bias");
@@ -386,17 +395,17 @@ int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb
   e2.bias = (const float*)h->wb(l, "attn.proj.bias");
   e2.residual = h->base + bb.x_in;
   void* xp_dst = h->base + (shrinks ? bb.xp_full : bb.xp);
-  gemm(c, h->base + bb.o, D, 1, h->wb(l, "attn.proj.weight"), D, 1, xp_dst, 0, Ma, D, D, e2);
+  gemm(c, h->base + bb.o, D, 1, h->wb(l, "attn.proj.weight"), D, 1, xp_dst, 1, Ma, D, D, e2);
   if (is_drop) {
     int M = Ta - 1;
     token_select(c.stream, h->at<float>(bb.p), B, H, M, k, h->at<float>(bb.s), h->at<int>(bb.kept), h->at<int>(bb.dropped));
     if (kept_out != nullptr)
       cudaMemcpyAsync(kept_out, h->base + bb.kept, (size_t)B * k * sizeof(int), cudaMemcpyDeviceToDevice, c.stream);
     if (shrinks)
-      gather_fuse(c, h->base + bb.xp_full, B, M, D, k, h->at<int>(bb.kept), h->at<int>(bb.dropped), h->at<float>(bb.s),
+      gather_fuse(cf, h->base + bb.xp_full, B, M, D, k, h->at<int>(bb.kept), h->at<int>(bb.dropped), h->at<float>(bb.s),
                   h->cfg.fuse_mode, h->base + bb.xp);
   }
-  layernorm_fwd(c, h->base + bb.xp, D, (const float*)h->wb(l, "norm2.weight"), (const float*)h->wb(l, "norm2.bias"),
+  layernorm_fwd(c, h->at<float>(bb.xp), D, (const float*)h->wb(l, "norm2.weight"), (const float*)h->wb(l, "norm2.bias"),
                 h->base + bb.y2, 0, save ? h->at<float>(bb.mean2) : nullptr, save ? h->at<float>(bb.rstd2) : nullptr, Mf, D, d.ln_eps);
   GemmEpilogue e3;
   e3.bias = (const float*)h->wb(l, "mlp.fc1.bias");
@@ -406,13 +415,18 @@ int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb
   GemmEpilogue e4;
   e4.bias = (const float*)h->wb(l, "mlp.fc2.bias");
   e4.residual = h->base + bb.xp;
-  gemm(c, h->base + bb.hh, F, 1, h->wb(l, "mlp.fc2.weight"), F, 1, h->base + bb.x_out, 0, Mf, D, F, e4);
+  gemm(c, h->base + bb.hh, F, 1, h->wb(l, "mlp.fc2.weight"), F, 1, h->base + bb.x_out, 1, Mf, D, F, e4);
   return BSR_OK;
 }
 
 // Backward of one trainable block (Eq. 2-5).  dxo: gradient at the block output [B*Tf, D]; dxi receives the
 // gradient at the block input unless it is null (earliest trainable block: Eq. 8, nothing flows further).
-int block_backward(bsr_handle* h, const Ctx& c, int l, int B, void* dxo, void* dxi) {
+struct GradStream {      // gradient of the residual stream: float rows, plus the bf16 copy the GEMMs read (bf16 only)
+  float* f;
+  void* c;
+};
+
+int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, GradStream dxi, bool need_dxi) {
   const bsr_dims& d = h->cfg.dims;
   const Schedule& s = h->sched;
   const BlockBufs& bb = h->bufs_train[l];
@@ -420,38 +434,43 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, void* dxo, void* d
   int Ta = s.ta[l], Tf = s.tf[l], k = s.k[l];
   int Ma = B * Ta, Mf = B * Tf;
   bool shrinks = k >= 0 && Tf != Ta;
+  bool bf = d.dtype == BSR_DTYPE_BF16;
+  Ctx cf = c;
+  cf.dtype = 0;
   float* csp = h->at<float>(h->off_cs_partials);
   float* lnp = h->at<float>(h->off_ln_partials);
   void* dz = h->base + h->off_dz;
   void* dy = h->base + h->off_dy;
-  void* dxg = h->base + h->off_dxg;
-  void* dxp = shrinks ? (void*)(h->base + h->off_dxp) : dxg;
+  GradStream dxg = {h->at<float>(h->off_dxg), bf ? (void*)(h->base + h->off_dxg_c) : nullptr};
+  GradStream dxp = shrinks ? GradStream{h->at<float>(h->off_dxp), bf ? (void*)(h->base + h->off_dxp_c) : nullptr} : dxg;
   void* d_o = h->base + h->off_do;
   void* dqkv = h->base + h->off_dqkv;
+  auto op = [&](const GradStream& g) -> const void* { return bf ? g.c : (const void*)g.f; };   // GEMM operand view
   GemmEpilogue none;
   // FFN second layer: dz = (dxo W2) * GELU'(z); dW2 = dxo^T h; db2 = column sums of dxo
   GemmEpilogue eg;
   eg.act = 2;
   eg.aux_in = h->base + bb.z;
-  gemm(c, dxo, D, 1, h->wb(l, "mlp.fc2.weight"), 1, F, dz, 0, Mf, F, D, eg);
-  gemm(c, dxo, 1, D, h->base + bb.hh, 1, F, h->gb(l, "mlp.fc2.weight"), 1, D, F, Mf, none);
-  colsum(c, dxo, Mf, D, csp, h->gb(l, "mlp.fc2.bias"));
+  gemm(c, op(dxo), D, 1, h->wb(l, "mlp.fc2.weight"), 1, F, dz, 0, Mf, F, D, eg);
+  gemm(c, op(dxo), 1, D, h->base + bb.hh, 1, F, h->gb(l, "mlp.fc2.weight"), 1, D, F, Mf, none);
+  colsum(cf, dxo.f, Mf, D, csp, h->gb(l, "mlp.fc2.bias"));
   // FFN first layer
   gemm(c, dz, F, 1, h->wb(l, "mlp.fc1.weight"), 1, D, dy, 0, Mf, D, F, none);
   gemm(c, dz, 1, F, h->base + bb.y2, 1, D, h->gb(l, "mlp.fc1.weight"), 1, F, D, Mf, none);
   colsum(c, dz, Mf, F, csp, h->gb(l, "mlp.fc1.bias"));
-  layernorm_bwd(c, dy, 0, h->base + bb.xp, D, h->at<float>(bb.mean2), h->at<float>(bb.rstd2),
-                (const float*)h->wb(l, "norm2.weight"), dxo, dxg, D, lnp, h->gb(l, "norm2.weight"), h->gb(l, "norm2.bias"), Mf, D);
+  layernorm_bwd(c, dy, 0, h->at<float>(bb.xp), D, h->at<float>(bb.mean2), h->at<float>(bb.rstd2),
+                (const float*)h->wb(l, "norm2.weight"), dxo.f, dxg.f, D, shrinks ? nullptr : dxg.c, lnp,
+                h->gb(l, "norm2.weight"), h->gb(l, "norm2.bias"), Mf, D);
   const float* cls_extra = nullptr;
   if (shrinks) {
-    gather_fuse_bwd(c, dxg, h->base + bb.xp_full, B, Ta - 1, D, k, h->at<int>(bb.kept), h->at<int>(bb.dropped),
-                    h->at<float>(bb.s), h->cfg.fuse_mode, dxp, h->at<float>(h->off_escore));
+    gather_fuse_bwd(c, dxg.f, h->base + bb.xp_full, B, Ta - 1, D, k, h->at<int>(bb.kept), h->at<int>(bb.dropped),
+                    h->at<float>(bb.s), h->cfg.fuse_mode, dxp.f, dxp.c, h->at<float>(h->off_escore));
     if (h->cfg.fuse_mode == BSR_FUSE_WEIGHTED_SUM) cls_extra = h->at<float>(h->off_escore);
   }
   // attention output projection
-  gemm(c, dxp, D, 1, h->wb(l, "attn.proj.weight"), 1, D, d_o, 0, Ma, D, D, none);
-  gemm(c, dxp, 1, D, h->base + bb.o, 1, D, h->gb(l, "attn.proj.weight"), 1, D, D, Ma, none);
-  colsum(c, dxp, Ma, D, csp, h->gb(l, "attn.proj.bias"));
+  gemm(c, op(dxp), D, 1, h->wb(l, "attn.proj.weight"), 1, D, d_o, 0, Ma, D, D, none);
+  gemm(c, op(dxp), 1, D, h->base + bb.o, 1, D, h->gb(l, "attn.proj.weight"), 1, D, D, Ma, none);
+  colsum(cf, dxp.f, Ma, D, csp, h->gb(l, "attn.proj.bias"));
   int rc = attention_bwd(c, h->base + bb.qkv, h->base + bb.o, d_o, h->at<float>(bb.lse), h->at<float>(h->off_delta),
                          cls_extra, dqkv, B, Ta, H, hd);
   if (rc != 0) return set_err(h->err, BSR_ERR_UNSUPPORTED, "attention backward: %d tokens do not fit this kernel", Ta);
@@ -459,8 +478,9 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, void* dxo, void* d
   gemm(c, dqkv, 3 * D, 1, h->wb(l, "attn.qkv.weight"), 1, D, dy, 0, Ma, D, 3 * D, none);
   gemm(c, dqkv, 1, 3 * D, h->base + bb.y1, 1, D, h->gb(l, "attn.qkv.weight"), 1, 3 * D, D, Ma, none);
   colsum(c, dqkv, Ma, 3 * D, csp, h->gb(l, "attn.qkv.bias"));
-  layernorm_bwd(c, dy, 0, h->base + bb.x_in, D, h->at<float>(bb.mean1), h->at<float>(bb.rstd1),
-                (const float*)h->wb(l, "norm1.weight"), dxp, dxi, D, lnp, h->gb(l, "norm1.weight"), h->gb(l, "norm1.bias"), Ma, D);
+  layernorm_bwd(c, dy, 0, h->at<float>(bb.x_in), D, h->at<float>(bb.mean1), h->at<float>(bb.rstd1),
+                (const float*)h->wb(l, "norm1.weight"), dxp.f, need_dxi ? dxi.f : nullptr, D, need_dxi ? dxi.c : nullptr, lnp,
+                h->gb(l, "norm1.weight"), h->gb(l, "norm1.bias"), Ma, D);
   return BSR_OK;
 }
 
@@ -494,7 +514,7 @@ int forward_all(bsr_handle* h, const Ctx& c, const void* images, int B, bool tra
   gemm(c, h->base + h->off_patches, pin, 1, h->w("patch_embed.weight"), pin, 1, h->base + h->off_emb, 0, B * N, D, pin, ep);
   int first_train = train ? h->t0 : d.depth;
   size_t x0 = (first_train == 0) ? h->bufs_train[0].x_in : h->bufs_frozen[0].x_in;
-  assemble_tokens(c, h->base + h->off_emb, (const float*)h->w("cls_token"), (const float*)h->w("pos_embed"), h->base + x0, B, N, D);
+  assemble_tokens(c, h->base + h->off_emb, (const float*)h->w("cls_token"), (const float*)h->w("pos_embed"), h->at<float>(x0), B, N, D);
   int* kept_all = h->at<int>(h->off_kept_all);
   size_t kept_off = 0;
   size_t cur = x0;
@@ -716,7 +736,7 @@ int32_t bsr_train_step(bsr_handle* h, const void* images, const int32_t* labels,
   int Tl = h->sched.tf[d.depth - 1];
   HeadDesc hd = head_desc(h);
   float* xn = h->at<float>(h->off_xn);
-  layernorm_fwd(c, h->base + x_last, (long)Tl * D, (const float*)h->w("norm.weight"), (const float*)h->w("norm.bias"), xn, 1,
+  layernorm_fwd(c, h->at<float>(x_last), (long)Tl * D, (const float*)h->w("norm.weight"), (const float*)h->w("norm.bias"), xn, 1,
                 h->at<float>(h->off_meanf), h->at<float>(h->off_rstdf), B, D, d.ln_eps);
   head_fwd(c, hd, xn, task_ids, h->at<float>(h->off_logits), B);
   cross_entropy(c, hd, h->at<float>(h->off_logits), labels, task_ids, h->at<float>(h->off_per_image), h->at<float>(h->off_dlogits),
@@ -727,20 +747,23 @@ int32_t bsr_train_step(bsr_handle* h, const void* images, const int32_t* labels,
   // backward: head, final LayerNorm, trainable blocks in reverse, nothing before the earliest one
   head_bwd(c, hd, xn, h->at<float>(h->off_dlogits), task_ids, h->at<float>(h->off_dxn), B);
   float* lnp = h->at<float>(h->off_ln_partials);
+  bool bf = d.dtype == BSR_DTYPE_BF16;
   if (h->t0 < d.depth) {
-    void* dxo = h->base + h->off_dxa;
-    void* dxi = h->base + h->off_dxb;
-    cudaMemsetAsync(dxo, 0, (size_t)B * Tl * D * es, c.stream);
-    layernorm_bwd(c, h->at<float>(h->off_dxn), 1, h->base + x_last, (long)Tl * D, h->at<float>(h->off_meanf), h->at<float>(h->off_rstdf),
-                  (const float*)h->w("norm.weight"), nullptr, dxo, (long)Tl * D, lnp, h->gradp("norm.weight"), h->gradp("norm.bias"), B, D);
+    GradStream dxo = {h->at<float>(h->off_dxa), bf ? (void*)(h->base + h->off_dxa_c) : nullptr};
+    GradStream dxi = {h->at<float>(h->off_dxb), bf ? (void*)(h->base + h->off_dxb_c) : nullptr};
+    // only the classification rows of the last block's output receive a gradient
+    cudaMemsetAsync(dxo.f, 0, (size_t)B * Tl * D * 4, c.stream);
+    if (bf) cudaMemsetAsync(dxo.c, 0, (size_t)B * Tl * D * es, c.stream);
+    layernorm_bwd(c, h->at<float>(h->off_dxn), 1, h->at<float>(x_last), (long)Tl * D, h->at<float>(h->off_meanf), h->at<float>(h->off_rstdf),
+                  (const float*)h->w("norm.weight"), nullptr, dxo.f, (long)Tl * D, dxo.c, lnp, h->gradp("norm.weight"), h->gradp("norm.bias"), B, D);
     for (int l = d.depth - 1; l >= h->t0; --l) {
-      rc = block_backward(h, c, l, B, dxo, l > h->t0 ? dxi : nullptr);
+      rc = block_backward(h, c, l, B, dxo, dxi, l > h->t0);
       if (rc != BSR_OK) return rc;
-      void* t = dxo; dxo = dxi; dxi = t;
+      GradStream t = dxo; dxo = dxi; dxi = t;
     }
   } else {
-    layernorm_bwd(c, h->at<float>(h->off_dxn), 1, h->base + x_last, (long)Tl * D, h->at<float>(h->off_meanf), h->at<float>(h->off_rstdf),
-                  (const float*)h->w("norm.weight"), nullptr, nullptr, 0, lnp, h->gradp("norm.weight"), h->gradp("norm.bias"), B, D);
+    layernorm_bwd(c, h->at<float>(h->off_dxn), 1, h->at<float>(x_last), (long)Tl * D, h->at<float>(h->off_meanf), h->at<float>(h->off_rstdf),
+                  (const float*)h->w("norm.weight"), nullptr, nullptr, 0, nullptr, lnp, h->gradp("norm.weight"), h->gradp("norm.bias"), B, D);
   }
   h->step += 1;
   double bc1 = 1.0 - std::pow((double)h->cfg.beta1, (double)h->step);
@@ -765,7 +788,7 @@ int32_t bsr_eval_forward(bsr_handle* h, const void* images, const int32_t* task_
   int Tl = h->sched.tf[d.depth - 1];
   HeadDesc hd = head_desc(h);
   float* xn = h->at<float>(h->off_xn);
-  layernorm_fwd(c, h->base + x_last, (long)Tl * d.dim, (const float*)h->w("norm.weight"), (const float*)h->w("norm.bias"), xn, 1,
+  layernorm_fwd(c, h->at<float>(x_last), (long)Tl * d.dim, (const float*)h->w("norm.weight"), (const float*)h->w("norm.bias"), xn, 1,
                 nullptr, nullptr, batch, d.dim, d.ln_eps);
   head_fwd(c, hd, xn, task_ids, h->at<float>(h->off_logits), batch);
   cudaMemcpyAsync(logits_out, h->at<float>(h->off_logits), (size_t)batch * hd.cmax * 4, cudaMemcpyDeviceToDevice, c.stream);

@@ -24,19 +24,20 @@ inline size_t dtype_size(int dtype) { return dtype == 0 ? 4 : 2; }
 
 // ---- embedding --------------------------------------------------------------------------------
 void patchify(const Ctx& c, const void* images, void* patches, int B, int C, int S, int P);
-void assemble_tokens(const Ctx& c, const void* emb, const float* cls, const float* pos, void* x, int B, int N, int D);
+void assemble_tokens(const Ctx& c, const void* emb, const float* cls, const float* pos, float* x, int B, int N, int D);
 
-// ---- LayerNorm --------------------------------------------------------------------------------
+// ---- LayerNorm (the residual stream is float in every configuration) ----------------------------
 // y[r] = LN(x[r]) * g + b for `rows` rows of length D; row r of x starts at x + r * x_stride elements.
-// mean/rstd (optional) receive the row statistics.  y_is_float selects a float output (head path).
-void layernorm_fwd(const Ctx& c, const void* x, long x_stride, const float* g, const float* b, void* y, int y_is_float,
+// y takes the storage dtype unless y_is_float.  mean/rstd (optional) receive the row statistics.
+void layernorm_fwd(const Ctx& c, const float* x, long x_stride, const float* g, const float* b, void* y, int y_is_float,
                    float* mean, float* rstd, int rows, int D, float eps);
-// dx[r] = dres[r] + LN'(dy[r]);  partial sums of dgamma/dbeta go to `partials` ([2][groups][D]) and are
-// reduced in a fixed order into dgamma, dbeta.  dx may be null (only parameter gradients wanted);
-// dres may be null.  dy_is_float: dy is float [rows, D] (head path).  dx rows start at dx + r * dx_stride.
-void layernorm_bwd(const Ctx& c, const void* dy, int dy_is_float, const void* x, long x_stride, const float* mean,
-                   const float* rstd, const float* g, const void* dres, void* dx, long dx_stride, float* partials,
-                   float* dgamma, float* dbeta, int rows, int D);
+// dx[r] = dres[r] + LN'(dy[r]) (float; rows dx_stride apart); dx_copy (optional, bf16 configurations) receives
+// the same rows in the storage dtype.  Partial sums of dgamma/dbeta go to `partials` ([2][groups][D]) and are
+// reduced in a fixed order.  dx may be null (only parameter gradients wanted); dres may be null.
+// dy is in the storage dtype, or float [rows, D] when dy_is_float (head path).
+void layernorm_bwd(const Ctx& c, const void* dy, int dy_is_float, const float* x, long x_stride, const float* mean,
+                   const float* rstd, const float* g, const float* dres, float* dx, long dx_stride, void* dx_copy,
+                   float* partials, float* dgamma, float* dbeta, int rows, int D);
 int layernorm_bwd_groups(const Ctx& c, int rows);
 
 // ---- column sums (bias gradients) -------------------------------------------------------------
@@ -77,8 +78,9 @@ void token_select(cudaStream_t s, const float* p, int B, int H, int M, int k, fl
 void gather_fuse(const Ctx& c, const void* x, int B, int M, int D, int k, const int* kept, const int* dropped,
                  const float* scores, int fuse, void* out);
 // Backward of the compaction: dx [B, 1+M, D] from dout [B, 1+k+f, D]; escore [B, M] = <g_fused, x_j> for dropped j, else 0.
+// dx_copy (optional): the same rows in bf16 for the GEMMs that consume them (float streams only).
 void gather_fuse_bwd(const Ctx& c, const void* dout, const void* x, int B, int M, int D, int k, const int* kept,
-                     const int* dropped, const float* scores, int fuse, void* dx, float* escore);
+                     const int* dropped, const float* scores, int fuse, void* dx, void* dx_copy, float* escore);
 
 // ---- head, loss, optimiser --------------------------------------------------------------------
 // logits[b, c] = xn[b] . W_task(b)[c] + bias; classes beyond the task's count get -inf.

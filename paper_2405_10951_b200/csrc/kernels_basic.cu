@@ -37,60 +37,61 @@ void patchify(const Ctx& c, const void* images, void* patches, int B, int C, int
 // x[b, 0] = cls + pos[0];  x[b, 1 + n] = emb[b, n] + pos[1 + n]   (classification token and positional embedding)
 template <typename T>
 __global__ void assemble_kernel(const T* __restrict__ emb, const float* __restrict__ cls, const float* __restrict__ pos,
-                                T* __restrict__ x, int B, int N, int D, long total) {
+                                float* __restrict__ x, int B, int N, int D, long total) {
   long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
   int d = (int)(i % D); long r = i / D;
   int t = (int)(r % (N + 1));
   int b = (int)(r / (N + 1));
   float v = (t == 0) ? cls[d] : to_f(emb[((long)b * N + (t - 1)) * D + d]);
-  x[i] = from_f<T>(v + pos[(long)t * D + d]);
+  x[i] = v + pos[(long)t * D + d];
 }
 
-void assemble_tokens(const Ctx& c, const void* emb, const float* cls, const float* pos, void* x, int B, int N, int D) {
+void assemble_tokens(const Ctx& c, const void* emb, const float* cls, const float* pos, float* x, int B, int N, int D) {
   long total = (long)B * (N + 1) * D;
   int threads = 256, blocks = ceil_div(total, threads);
   if (c.dtype == 0)
-    assemble_kernel<float><<<blocks, threads, 0, c.stream>>>((const float*)emb, cls, pos, (float*)x, B, N, D, total);
+    assemble_kernel<float><<<blocks, threads, 0, c.stream>>>((const float*)emb, cls, pos, x, B, N, D, total);
   else
-    assemble_kernel<bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)emb, cls, pos, (bf16*)x, B, N, D, total);
+    assemble_kernel<bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)emb, cls, pos, x, B, N, D, total);
 }
 
 // ------------------------------------------------------------------------------------------------
-// LayerNorm.  One warp per row, the row held in registers (D <= 1024, D % Pack::N == 0).
+// LayerNorm.  The residual stream x is float in every configuration (only the small block updates
+// would survive bf16 rounding of the stream poorly); the normalised output feeds a GEMM and takes
+// the storage dtype.  One warp per row, the row held in registers (D <= 1024, D % 4 == 0).
 // ------------------------------------------------------------------------------------------------
 constexpr int LN_MAX_PER_LANE = 32;   // floats per lane: D <= 1024
+constexpr int LN_MAXC = LN_MAX_PER_LANE / 4;
 
-template <typename TX, typename TY>
-__global__ void layernorm_fwd_kernel(const TX* __restrict__ x, long x_stride, const float* __restrict__ g,
+template <typename TY>
+__global__ void layernorm_fwd_kernel(const float* __restrict__ x, long x_stride, const float* __restrict__ g,
                                      const float* __restrict__ b, TY* __restrict__ y, float* __restrict__ mean,
                                      float* __restrict__ rstd, int rows, int D, float eps) {
-  constexpr int N = Pack<TX>::N;
-  constexpr int MAXC = LN_MAX_PER_LANE / N;
   int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   int lane = threadIdx.x & 31;
   if (warp >= rows) return;
-  const TX* xr = x + (long)warp * x_stride;
-  int chunks = D / N;
+  const float* xr = x + (long)warp * x_stride;
+  int chunks = D / 4;
   float v[LN_MAX_PER_LANE];
   float sum = 0.f;
 #pragma unroll
-  for (int i = 0; i < MAXC; ++i) {
+  for (int i = 0; i < LN_MAXC; ++i) {
     int ch = lane + i * 32;
     if (ch < chunks) {
-      load16(xr + ch * N, v + i * N);
+      load16(xr + ch * 4, v + i * 4);
 #pragma unroll
-      for (int j = 0; j < N; ++j) sum += v[i * N + j];
+      for (int j = 0; j < 4; ++j) sum += v[i * 4 + j];
     }
   }
   float mu = warp_sum(sum) / (float)D;
   float sq = 0.f;
 #pragma unroll
-  for (int i = 0; i < MAXC; ++i) {
+  for (int i = 0; i < LN_MAXC; ++i) {
     int ch = lane + i * 32;
     if (ch < chunks) {
 #pragma unroll
-      for (int j = 0; j < N; ++j) { float t = v[i * N + j] - mu; sq += t * t; }
+      for (int j = 0; j < 4; ++j) { float t = v[i * 4 + j] - mu; sq += t * t; }
     }
   }
   float rs = rsqrtf(warp_sum(sq) / (float)D + eps);
@@ -100,73 +101,72 @@ __global__ void layernorm_fwd_kernel(const TX* __restrict__ x, long x_stride, co
   }
   TY* yr = y + (long)warp * D;
 #pragma unroll
-  for (int i = 0; i < MAXC; ++i) {
+  for (int i = 0; i < LN_MAXC; ++i) {
     int ch = lane + i * 32;
     if (ch < chunks) {
-      float o[N];
-#pragma unroll
-      for (int j = 0; j < N; ++j) {
-        int col = ch * N + j;
-        o[j] = (v[i * N + j] - mu) * rs * g[col] + b[col];
-      }
-      store_n<N>(yr + ch * N, o);
+      float4 gg = *reinterpret_cast<const float4*>(g + ch * 4), bb = *reinterpret_cast<const float4*>(b + ch * 4);
+      float o[4];
+      o[0] = (v[i * 4 + 0] - mu) * rs * gg.x + bb.x;
+      o[1] = (v[i * 4 + 1] - mu) * rs * gg.y + bb.y;
+      o[2] = (v[i * 4 + 2] - mu) * rs * gg.z + bb.z;
+      o[3] = (v[i * 4 + 3] - mu) * rs * gg.w + bb.w;
+      store4(yr + ch * 4, o);
     }
   }
 }
 
-void layernorm_fwd(const Ctx& c, const void* x, long x_stride, const float* g, const float* b, void* y, int y_is_float,
+void layernorm_fwd(const Ctx& c, const float* x, long x_stride, const float* g, const float* b, void* y, int y_is_float,
                    float* mean, float* rstd, int rows, int D, float eps) {
   int threads = 256;
   int blocks = ceil_div((long)rows * 32, threads);
-  if (c.dtype == 0)
-    layernorm_fwd_kernel<float, float><<<blocks, threads, 0, c.stream>>>((const float*)x, x_stride, g, b, (float*)y, mean, rstd, rows, D, eps);
-  else if (y_is_float)
-    layernorm_fwd_kernel<bf16, float><<<blocks, threads, 0, c.stream>>>((const bf16*)x, x_stride, g, b, (float*)y, mean, rstd, rows, D, eps);
+  if (c.dtype == 0 || y_is_float)
+    layernorm_fwd_kernel<float><<<blocks, threads, 0, c.stream>>>(x, x_stride, g, b, (float*)y, mean, rstd, rows, D, eps);
   else
-    layernorm_fwd_kernel<bf16, bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)x, x_stride, g, b, (bf16*)y, mean, rstd, rows, D, eps);
+    layernorm_fwd_kernel<bf16><<<blocks, threads, 0, c.stream>>>(x, x_stride, g, b, (bf16*)y, mean, rstd, rows, D, eps);
 }
 
 // Backward.  Each block owns rows blockIdx.x*8 + warp, stepping by gridDim.x*8; every lane accumulates the
 // dgamma/dbeta contributions of its columns, warps are combined through shared memory in warp order, and the
 // block's sums go to partials[0][block][col] (dgamma) and partials[1][block][col] (dbeta).
+// dx (float, the gradient of the residual stream) = dres + LN'(dy); dx_copy receives the same values in the
+// storage dtype for the GEMMs that consume them.
 constexpr int LNB_WARPS = 8;
 
-template <typename TX, typename TDY>
-__global__ void layernorm_bwd_kernel(const TDY* __restrict__ dy, const TX* __restrict__ x, long x_stride,
+template <typename TDY, typename TC>
+__global__ void layernorm_bwd_kernel(const TDY* __restrict__ dy, const float* __restrict__ x, long x_stride,
                                      const float* __restrict__ mean, const float* __restrict__ rstd,
-                                     const float* __restrict__ g, const TX* __restrict__ dres, TX* __restrict__ dx,
-                                     long dx_stride, float* __restrict__ partials, int rows, int D) {
-  constexpr int N = Pack<TX>::N;
-  constexpr int MAXC = LN_MAX_PER_LANE / N;
+                                     const float* __restrict__ g, const float* __restrict__ dres, float* __restrict__ dx,
+                                     long dx_stride, TC* __restrict__ dx_copy, float* __restrict__ partials, int rows, int D) {
   extern __shared__ float sm[];   // [LNB_WARPS][2][D]
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  int chunks = D / N;
+  int chunks = D / 4;
   float ag[LN_MAX_PER_LANE], ab[LN_MAX_PER_LANE];
 #pragma unroll
   for (int i = 0; i < LN_MAX_PER_LANE; ++i) { ag[i] = 0.f; ab[i] = 0.f; }
   for (int r = blockIdx.x * LNB_WARPS + warp; r < rows; r += gridDim.x * LNB_WARPS) {
-    const TX* xr = x + (long)r * x_stride;
+    const float* xr = x + (long)r * x_stride;
     const TDY* dyr = dy + (long)r * D;
     float mu = mean[r], rs = rstd[r];
     float xh[LN_MAX_PER_LANE], dh[LN_MAX_PER_LANE];
     float s1 = 0.f, s2 = 0.f;
 #pragma unroll
-    for (int i = 0; i < MAXC; ++i) {
+    for (int i = 0; i < LN_MAXC; ++i) {
       int ch = lane + i * 32;
       if (ch < chunks) {
-        float xv[N], dv[N];
-        load16(xr + ch * N, xv);
-        load_n<N>(dyr + ch * N, dv);
+        float xv[4], dv[4];
+        load16(xr + ch * 4, xv);
+        load4(dyr + ch * 4, dv);
+        float4 gg = *reinterpret_cast<const float4*>(g + ch * 4);
+        float gv[4] = {gg.x, gg.y, gg.z, gg.w};
 #pragma unroll
-        for (int j = 0; j < N; ++j) {
-          int col = ch * N + j;
+        for (int j = 0; j < 4; ++j) {
           float d = dv[j];
           float h = (xv[j] - mu) * rs;
-          xh[i * N + j] = h;
-          ag[i * N + j] += d * h;
-          ab[i * N + j] += d;
-          float dxh = d * g[col];
-          dh[i * N + j] = dxh;
+          xh[i * 4 + j] = h;
+          ag[i * 4 + j] += d * h;
+          ab[i * 4 + j] += d;
+          float dxh = d * gv[j];
+          dh[i * 4 + j] = dxh;
           s1 += dxh;
           s2 += dxh * h;
         }
@@ -175,33 +175,34 @@ __global__ void layernorm_bwd_kernel(const TDY* __restrict__ dy, const TX* __res
     s1 = warp_sum(s1) / (float)D;
     s2 = warp_sum(s2) / (float)D;
     if (dx != nullptr) {
-      TX* dxr = dx + (long)r * dx_stride;
+      float* dxr = dx + (long)r * dx_stride;
 #pragma unroll
-      for (int i = 0; i < MAXC; ++i) {
+      for (int i = 0; i < LN_MAXC; ++i) {
         int ch = lane + i * 32;
         if (ch < chunks) {
-          float o[N];
-          if (dres != nullptr) load16(dres + (long)r * D + ch * N, o);
+          float o[4];
+          if (dres != nullptr) load16(dres + (long)r * D + ch * 4, o);
           else {
 #pragma unroll
-            for (int j = 0; j < N; ++j) o[j] = 0.f;
+            for (int j = 0; j < 4; ++j) o[j] = 0.f;
           }
 #pragma unroll
-          for (int j = 0; j < N; ++j) o[j] += rs * (dh[i * N + j] - s1 - xh[i * N + j] * s2);
-          store16(dxr + ch * N, o);
+          for (int j = 0; j < 4; ++j) o[j] += rs * (dh[i * 4 + j] - s1 - xh[i * 4 + j] * s2);
+          store16(dxr + ch * 4, o);
+          if (dx_copy != nullptr) store4(dx_copy + (long)r * dx_stride + ch * 4, o);
         }
       }
     }
   }
   float* mine = sm + (size_t)warp * 2 * D;
 #pragma unroll
-  for (int i = 0; i < MAXC; ++i) {
+  for (int i = 0; i < LN_MAXC; ++i) {
     int ch = lane + i * 32;
     if (ch < chunks) {
 #pragma unroll
-      for (int j = 0; j < N; ++j) {
-        mine[ch * N + j] = ag[i * N + j];
-        mine[D + ch * N + j] = ab[i * N + j];
+      for (int j = 0; j < 4; ++j) {
+        mine[ch * 4 + j] = ag[i * 4 + j];
+        mine[D + ch * 4 + j] = ab[i * 4 + j];
       }
     }
   }
@@ -230,25 +231,26 @@ int layernorm_bwd_groups(const Ctx& c, int rows) {
   return want < cap ? (want < 1 ? 1 : want) : cap;
 }
 
-void layernorm_bwd(const Ctx& c, const void* dy, int dy_is_float, const void* x, long x_stride, const float* mean,
-                   const float* rstd, const float* g, const void* dres, void* dx, long dx_stride, float* partials,
-                   float* dgamma, float* dbeta, int rows, int D) {
+template <typename TDY, typename TC>
+static void launch_ln_bwd(const Ctx& c, int groups, size_t smem, const void* dy, const float* x, long x_stride, const float* mean,
+                          const float* rstd, const float* g, const float* dres, float* dx, long dx_stride, void* dx_copy,
+                          float* partials, int rows, int D) {
+  cudaFuncSetAttribute(layernorm_bwd_kernel<TDY, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  layernorm_bwd_kernel<TDY, TC><<<groups, LNB_WARPS * 32, smem, c.stream>>>((const TDY*)dy, x, x_stride, mean, rstd, g, dres, dx,
+                                                                           dx_stride, (TC*)dx_copy, partials, rows, D);
+}
+
+void layernorm_bwd(const Ctx& c, const void* dy, int dy_is_float, const float* x, long x_stride, const float* mean,
+                   const float* rstd, const float* g, const float* dres, float* dx, long dx_stride, void* dx_copy,
+                   float* partials, float* dgamma, float* dbeta, int rows, int D) {
   int groups = layernorm_bwd_groups(c, rows);
   size_t smem = (size_t)LNB_WARPS * 2 * D * sizeof(float);
-  int threads = LNB_WARPS * 32;
-  if (c.dtype == 0) {
-    cudaFuncSetAttribute(layernorm_bwd_kernel<float, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    layernorm_bwd_kernel<float, float><<<groups, threads, smem, c.stream>>>(
-        (const float*)dy, (const float*)x, x_stride, mean, rstd, g, (const float*)dres, (float*)dx, dx_stride, partials, rows, D);
-  } else if (dy_is_float) {
-    cudaFuncSetAttribute(layernorm_bwd_kernel<bf16, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    layernorm_bwd_kernel<bf16, float><<<groups, threads, smem, c.stream>>>(
-        (const float*)dy, (const bf16*)x, x_stride, mean, rstd, g, (const bf16*)dres, (bf16*)dx, dx_stride, partials, rows, D);
-  } else {
-    cudaFuncSetAttribute(layernorm_bwd_kernel<bf16, bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    layernorm_bwd_kernel<bf16, bf16><<<groups, threads, smem, c.stream>>>(
-        (const bf16*)dy, (const bf16*)x, x_stride, mean, rstd, g, (const bf16*)dres, (bf16*)dx, dx_stride, partials, rows, D);
-  }
+  if (c.dtype == 0)
+    launch_ln_bwd<float, float>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, nullptr, partials, rows, D);
+  else if (dy_is_float)
+    launch_ln_bwd<float, bf16>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, dx_copy, partials, rows, D);
+  else
+    launch_ln_bwd<bf16, bf16>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, dx_copy, partials, rows, D);
   int t2 = 256;
   reduce_partials_kernel<<<ceil_div(D, t2), t2, 0, c.stream>>>(partials, groups, D, dgamma);
   reduce_partials_kernel<<<ceil_div(D, t2), t2, 0, c.stream>>>(partials + (size_t)groups * D, groups, D, dbeta);

@@ -155,57 +155,59 @@ void gather_fuse(const Ctx& c, const void* x, int B, int M, int D, int k, const 
 
 // Backward of the compaction, one warp per input row (the index sets are constants, the fusion weights are
 // differentiated):  dx_0 = g_0;  dx_{kept_i} = g_{1+i};  dx_j = s_j g_f and e_j = <g_f, x_j> for dropped j.
-template <typename T>
-__global__ void gather_fuse_bwd_kernel(const T* __restrict__ dout, const T* __restrict__ x, int B, int M, int D, int k,
+// Rows are float (residual stream); dx_copy optionally receives the same rows in bf16.
+__global__ void gather_fuse_bwd_kernel(const float* __restrict__ dout, const float* __restrict__ x, int B, int M, int D, int k,
                                        const int* __restrict__ kept, const int* __restrict__ dropped,
-                                       const float* __restrict__ scores, int fuse, T* __restrict__ dx,
-                                       float* __restrict__ escore) {
-  constexpr int N = Pack<T>::N;
+                                       const float* __restrict__ scores, int fuse, float* __restrict__ dx,
+                                       bf16* __restrict__ dx_copy, float* __restrict__ escore) {
   int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= B * (1 + M)) return;
   int b = warp / (1 + M), e = warp % (1 + M);
-  int chunks = D / N;
+  int chunks = D / 4;
   int t_out = 1 + k + (fuse ? 1 : 0);
-  const T* gb = dout + (size_t)b * t_out * D;
-  T* dxb = dx + (size_t)b * (1 + M) * D;
+  const float* gb = dout + (size_t)b * t_out * D;
+  size_t ob = (size_t)b * (1 + M) * D;
   if (e <= k) {                         // classification row or a kept row: plain copy
     int dst = (e == 0) ? 0 : 1 + kept[(size_t)b * k + (e - 1)];
-    for (int ch = lane; ch < chunks; ch += 32)
-      *reinterpret_cast<uint4*>(dxb + (size_t)dst * D + ch * N) = *reinterpret_cast<const uint4*>(gb + (size_t)e * D + ch * N);
+    for (int ch = lane; ch < chunks; ch += 32) {
+      float v[4];
+      load16(gb + (size_t)e * D + ch * 4, v);
+      store16(dx + ob + (size_t)dst * D + ch * 4, v);
+      if (dx_copy != nullptr) store4(dx_copy + ob + (size_t)dst * D + ch * 4, v);
+    }
     if (e > 0 && lane == 0) escore[(size_t)b * M + (dst - 1)] = 0.f;
     return;
   }
   int j = dropped[(size_t)b * (M - k) + (e - 1 - k)];
   float w = fuse ? scores[(size_t)b * M + j] : 0.f;
-  const T* gf = gb + (size_t)(1 + k) * D;
-  const T* xr = x + ((size_t)b * (1 + M) + 1 + j) * D;
+  const float* gf = gb + (size_t)(1 + k) * D;
+  const float* xr = x + ob + (size_t)(1 + j) * D;
   float dot = 0.f;
   for (int ch = lane; ch < chunks; ch += 32) {
-    float g[N], o[N];
+    float g[4], o[4];
     if (fuse) {
-      float xv[N];
-      load16(gf + ch * N, g);
-      load16(xr + ch * N, xv);
+      float xv[4];
+      load16(gf + ch * 4, g);
+      load16(xr + ch * 4, xv);
 #pragma unroll
-      for (int i = 0; i < N; ++i) { dot += g[i] * xv[i]; o[i] = w * g[i]; }
+      for (int i = 0; i < 4; ++i) { dot += g[i] * xv[i]; o[i] = w * g[i]; }
     } else {
 #pragma unroll
-      for (int i = 0; i < N; ++i) o[i] = 0.f;
+      for (int i = 0; i < 4; ++i) o[i] = 0.f;
     }
-    store16(dxb + (size_t)(1 + j) * D + ch * N, o);
+    store16(dx + ob + (size_t)(1 + j) * D + ch * 4, o);
+    if (dx_copy != nullptr) store4(dx_copy + ob + (size_t)(1 + j) * D + ch * 4, o);
   }
   dot = warp_sum(dot);
   if (lane == 0) escore[(size_t)b * M + j] = dot;
 }
 
 void gather_fuse_bwd(const Ctx& c, const void* dout, const void* x, int B, int M, int D, int k, const int* kept,
-                     const int* dropped, const float* scores, int fuse, void* dx, float* escore) {
+                     const int* dropped, const float* scores, int fuse, void* dx, void* dx_copy, float* escore) {
   int do_fuse = (fuse == 1 && k < M) ? 1 : 0;
   int threads = 256, blocks = ceil_div((long)B * (1 + M) * 32, threads);
-  if (c.dtype == 0)
-    gather_fuse_bwd_kernel<float><<<blocks, threads, 0, c.stream>>>((const float*)dout, (const float*)x, B, M, D, k, kept, dropped, scores, do_fuse, (float*)dx, escore);
-  else
-    gather_fuse_bwd_kernel<bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)dout, (const bf16*)x, B, M, D, k, kept, dropped, scores, do_fuse, (bf16*)dx, escore);
+  gather_fuse_bwd_kernel<<<blocks, threads, 0, c.stream>>>((const float*)dout, (const float*)x, B, M, D, k, kept, dropped, scores,
+                                                           do_fuse, (float*)dx, (bf16*)dx_copy, escore);
 }
 
 }  // namespace bsr
