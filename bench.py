@@ -1,0 +1,289 @@
+"""Throughput of one BSR fine-tuning step (ViT-B/16, bf16, batch 128) on B200, with the CPU oracle beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload vit_b]
+
+Prints ONE JSON line (rank 0).  A step is one pass of the whole path (frozen-prefix forward, token
+selection and fusion, forward + backward of the trainable blocks and head, AdamW) over one synthetic
+batch.  `value` is images/s with inputs resident in HBM; `e2e` includes the pinned-host -> device copy of
+the images and the device -> host read of the loss in every step.  With N > 1 every rank runs an
+independent replica on its own batch (no data-path collective); the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2405_10951_b200 import synth  # noqa: E402
+
+METRIC = "BSR fine-tune images/s"
+UNIT = "images/s"
+
+
+def step_flops(cfg, batch):
+    """Algorithmic FLOPs of one step: forward of every block at its token counts, plus twice the forward
+    FLOPs of the trainable blocks for their backward pass, head x3.  Token counts from the library."""
+    from paper_2405_10951_b200 import binding as Bd
+    ta, tf, _ = Bd.bsr_token_schedule(Bd.make_config(cfg))
+    D, F = cfg.dim, cfg.mlp_hidden
+    fwd = 2 * cfg.num_patches * (cfg.in_chans * cfg.patch_size ** 2) * D
+    bwd = 0
+    for l in range(cfg.depth):
+        blk = 2 * (ta[l] * 4 * D * D + 2 * ta[l] * ta[l] * D + 2 * tf[l] * D * F)
+        fwd += blk
+        if l in cfg.trainable:
+            bwd += 2 * blk
+    head = 2 * D * max(cfg.num_classes)
+    return float(batch) * (fwd + bwd + 3 * head)
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"tflops": float(p["bf16_tflops_sustained"]), "tflops_burst": float(p["bf16_tflops"]),
+                "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    return {"tflops": 1400.0, "tflops_burst": 1590.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons while the timed regions run."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(self.index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 8:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, f[4:8]):
+                    if v == "Active":
+                        reasons.add(n)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def oracle_sample_step(cfg, images, labels, task_ids, params):
+    from oracle import bsr_oracle as O
+    t0 = time.perf_counter()
+    O.train_step(cfg, params, images, labels, task_ids)
+    return time.perf_counter() - t0
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def run_reference(args, cfg):
+    """The CPU oracle, as it stands, on the host cores: each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_ref = max(1, min(cfg.batch, args.ref_batch))
+    images, labels, task_ids, params = synth.make_workload(cfg, batch=n_ref)
+    t1 = oracle_sample_step(cfg, images[:1], labels[:1], task_ids[:1], params)       # calibration, untimed
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    n_ref = int(max(1, min(n_ref, budget / max(t1, 1e-3))))
+    for _ in range(args.warmup):
+        oracle_sample_step(cfg, images[:n_ref], labels[:n_ref], task_ids[:n_ref], params)
+    t = [oracle_sample_step(cfg, images[:n_ref], labels[:n_ref], task_ids[:n_ref], params) for _ in range(args.steps)]
+    ms = 1e3 * sum(t) / len(t)
+    v = n_ref / (ms / 1e3)
+    cores = blas_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "sample": f"{n_ref} of {cfg.batch} images per step, full model dimensions"},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"{n_ref} images per step, {args.steps} steps"},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="vit_b", choices=list(synth.CONFIGS))
+    ap.add_argument("--ref-batch", type=int, default=8)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    cfg = synth.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the BSR step has no CPU path")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    warm = max(args.warmup, 3)
+
+    images, labels, task_ids, params = synth.make_workload(cfg, seed=cfg.seed + rank)
+    eng = Bd.Engine(cfg, device=f"cuda:{local}")
+    eng.set_params(params)
+    del params
+    storage = eng.storage_dtype
+    host_img = torch.as_tensor(np.ascontiguousarray(images, dtype=np.float32)).to(storage).pin_memory()
+    dev_img = host_img.cuda(non_blocking=True)
+    lab = torch.as_tensor(labels).cuda()
+    tid = torch.as_tensor(task_ids).cuda() if cfg.num_tasks > 1 else None
+    host_loss = torch.empty(1, dtype=torch.float32).pin_memory()
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warm):
+        eng.train_step(dev_img, lab, tid, want_kept=False)
+    eng.sync_status()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+
+    # ---- device-resident throughput -------------------------------------------------------------
+    eng.profile_enable(False)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        loss, _ = eng.train_step(dev_img, lab, tid, want_kept=False)
+    e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    launches = eng.profile_read()["kernel_launches"]
+
+    # ---- end to end: pinned host images in, loss out, every step ----------------------------------
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    stage = torch.empty_like(dev_img)
+    f0.record(stream)
+    for _ in range(args.steps):
+        stage.copy_(host_img, non_blocking=True)
+        loss, _ = eng.train_step(stage, lab, tid, want_kept=False)
+        host_loss.copy_(loss, non_blocking=True)
+        stream.synchronize()
+    f1.record(stream)
+    barrier()
+    ms_e2e = f0.elapsed_time(f1)
+
+    # ---- dominant kernel (tcgen05 GEMM): every launch bracketed by CUDA events ---------------------
+    eng.profile_enable(True)
+    for _ in range(min(args.steps, 5)):
+        eng.train_step(dev_img, lab, tid, want_kept=False)
+    prof = eng.profile_read()
+    eng.profile_enable(False)
+    eng.sync_status()
+    clocks = sampler.stop() if rank == 0 else {}
+
+    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_step = ms_total / args.steps
+    value = world * cfg.batch / (ms_step / 1e3)
+    e2e_value = world * cfg.batch / (ms_e2e / args.steps / 1e3)
+
+    if rank == 0:
+        pk = peaks()
+        flops = step_flops(cfg, cfg.batch)
+        gemm_tflops = prof["gemm_flops"] / (prof["gemm_ms"] * 1e-3) / 1e12 if prof["gemm_ms"] > 0 else 0.0
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": cfg.name, "global_batch": world * cfg.batch, "tokens": cfg.num_patches + 1,
+                       "trainable_blocks": list(cfg.trainable), "drop_blocks": list(cfg.drop_blocks),
+                       "keep_rate": cfg.keep_num / cfg.keep_den, "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                       "l2": "no flush: weights (172 MB) plus per-step activations (> 1 GB) exceed the 126 MB L2"},
+            "clocks": {k: clocks.get(k) for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples")},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(host_img.numel() * host_img.element_size()),
+                    "d2h_bytes_per_step": 4},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel (tcgen05 bf16 GEMM, all launches of a step)",
+                         "achieved": gemm_tflops, "peak": pk["tflops"], "unit": "TFLOP/s",
+                         "frac": gemm_tflops / pk["tflops"], "traffic": None, "peak_source": pk["source"] + " (sustained)",
+                         "gemm_ms_per_step": prof["gemm_ms"] / max(1, min(args.steps, 5)),
+                         "gemm_launches_per_step": prof["gemm_launches"] / max(1, min(args.steps, 5))},
+            "step_flops": flops,
+            "step_tflops": flops / (ms_step * 1e-3) / 1e12,
+            "step_roofline_frac": flops / (ms_step * 1e-3) / 1e12 / pk["tflops_burst"],
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            n_ref = min(cfg.batch, args.ref_batch)
+            im, lb, tk, pr = synth.make_workload(cfg, batch=n_ref)
+            sec = oracle_sample_step(cfg, im, lb, tk, pr)
+            line["cpu_baseline"] = {"value": n_ref / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                    "sample": f"one step on {n_ref} of {cfg.batch} images, full model dimensions, {sec:.1f} s"}
+        else:
+            line["cpu_baseline"] = None
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

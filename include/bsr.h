@@ -161,6 +161,21 @@ int32_t bsr_get_footprint(const bsr_handle* h, bsr_footprint* out_host);
  * bounded wait in a kernel expired, BSR_ERR_NONFINITE if the last loss was not finite.  Clears it. */
 int32_t bsr_sync_status(bsr_handle* h, void* stream);
 
+/* Measurement support (no counterpart in the paper).  bsr_profile_enable resets the counters; with
+ * time_gemms != 0 every tensor-core GEMM launch of the following steps is bracketed by a pair of CUDA
+ * events on the launching stream (host objects; this slows the step slightly, so timed throughput is
+ * taken with it off).  bsr_profile_read synchronises `stream` and reports, since the last enable: kernels
+ * launched by the library (host count, whole process), and for the timed GEMMs their number, their
+ * algorithmic FLOPs (2 m n k each) and the sum of their durations in milliseconds. */
+typedef struct {
+  uint64_t kernel_launches;
+  uint64_t gemm_launches;
+  double gemm_flops;
+  double gemm_ms;
+} bsr_profile;
+int32_t bsr_profile_enable(bsr_handle* h, int32_t time_gemms);
+int32_t bsr_profile_read(bsr_handle* h, void* stream, bsr_profile* out_host);
+
 /* ---- stand-alone forms of the paper-specific token kernels (no handle) ---------------------- */
 
 /* Token importance and top-K (Eq. 6; Section 4.1).  p_dev [batch, heads, m] float32: for every

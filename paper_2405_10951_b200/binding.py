@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "BSR_OK", -1: "BSR_ERR_INVALID_ARG", -2: "BSR_ERR_UNSUPPORTED
 
 EXPORTS = ["bsr_token_schedule", "bsr_workspace_bytes", "bsr_create", "bsr_destroy", "bsr_last_error", "bsr_set_param",
            "bsr_get_tensor", "bsr_set_lr", "bsr_set_step", "bsr_train_step", "bsr_eval_forward", "bsr_get_footprint",
-           "bsr_sync_status", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_backward",
+           "bsr_sync_status", "bsr_profile_enable", "bsr_profile_read", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_backward",
            "bsr_attention_forward"]
 
 
@@ -48,6 +48,10 @@ class bsr_footprint(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in ("workspace_bytes", "weight_bytes", "master_bytes", "optimizer_bytes",
                                            "grad_bytes", "saved_activation_bytes", "scratch_bytes",
                                            "paper_activation_bytes", "trainable_params")]
+
+
+class bsr_profile(C.Structure):
+    _fields_ = [("kernel_launches", C.c_uint64), ("gemm_launches", C.c_uint64), ("gemm_flops", C.c_double), ("gemm_ms", C.c_double)]
 
 
 class BsrError(RuntimeError):
@@ -82,6 +86,8 @@ def lib() -> C.CDLL:
         L.bsr_eval_forward.argtypes = [vp, vp, i32p, i32, vp, f32p, i32p]
         L.bsr_get_footprint.argtypes = [vp, C.POINTER(bsr_footprint)]
         L.bsr_sync_status.argtypes = [vp, vp]
+        L.bsr_profile_enable.argtypes = [vp, i32]
+        L.bsr_profile_read.argtypes = [vp, vp, C.POINTER(bsr_profile)]
         L.bsr_token_select.argtypes = [f32p, i32, i32, i32, i32, f32p, i32p, i32p, vp]
         L.bsr_gather_fuse.argtypes = [vp, i32, i32, i32, i32, i32, i32p, i32p, f32p, i32, vp, vp]
         L.bsr_linear_forward.argtypes = [vp, vp, f32p, vp, vp, i32, i32, i32, i32, i32, i32, vp]
@@ -300,6 +306,15 @@ class Engine:
 
     def sync_status(self):
         _check(lib().bsr_sync_status(self.h, _stream()), self.h)
+
+    def profile_enable(self, time_gemms: bool):
+        _check(lib().bsr_profile_enable(self.h, int(time_gemms)), self.h)
+
+    def profile_read(self) -> Dict[str, float]:
+        p = bsr_profile()
+        _check(lib().bsr_profile_read(self.h, _stream(), C.byref(p)), self.h)
+        return {"kernel_launches": int(p.kernel_launches), "gemm_launches": int(p.gemm_launches),
+                "gemm_flops": float(p.gemm_flops), "gemm_ms": float(p.gemm_ms)}
 
     def footprint(self) -> Dict[str, int]:
         fp = bsr_footprint()

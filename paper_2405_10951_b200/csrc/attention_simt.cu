@@ -278,6 +278,7 @@ static int launch_fwd(const Ctx& c, const void* qkv, void* out, float* lse, floa
   cudaFuncSetAttribute(attn_fwd_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   int qs = split_for(c, B * H, T_);
   dim3 grid(B * H, qs);
+  note_launch(1);
   attn_fwd_kernel<T><<<grid, AT_WARPS * 32, smem, c.stream>>>((const T*)qkv, (T*)out, lse, cls_prob, B, T_, H, d, qs);
   return 0;
 }
@@ -299,6 +300,7 @@ static int launch_bwd(const Ctx& c, const void* qkv, const void* dout, const flo
   cudaFuncSetAttribute(attn_bwd_dkv_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
   int qs = split_for(c, B * H, T_);
   dim3 grid(B * H, qs);
+  note_launch(2);
   attn_bwd_dq_kernel<T><<<grid, AT_WARPS * 32, smem1, c.stream>>>((const T*)qkv, (const T*)dout, lse, delta, cls_extra, (T*)dqkv, B, T_, H, d, qs);
   attn_bwd_dkv_kernel<T><<<grid, AT_WARPS * 32, smem2, c.stream>>>((const T*)qkv, (const T*)dout, lse, delta, cls_extra, (T*)dqkv, B, T_, H, d, qs);
   return 0;

@@ -104,6 +104,10 @@ __device__ __forceinline__ float gelu_grad_f(float x) {
   return 0.5f * (1.0f + erff(x * 0.70710678118654752f)) + x * 0.39894228040143268f * expf(-0.5f * x * x);
 }
 
+// Host-side count of kernel launches made by this library (read through bsr_profile_read).
+extern long g_kernel_launches;
+static inline void note_launch(int n = 1) { g_kernel_launches += n; }
+
 static inline int ceil_div(long a, long b) { return (int)((a + b - 1) / b); }
 
 }  // namespace bsr

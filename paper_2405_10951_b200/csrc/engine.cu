@@ -156,6 +156,8 @@ struct bsr_handle {
   size_t off_kept_all = 0;
   size_t off_stage = 0;
   size_t off_split = 0, split_floats = 0;
+  GemmProfile prof;
+  long launches_at_enable = 0;
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(base + off); }
   void* w(const char* name) const {
@@ -363,6 +365,7 @@ Ctx make_ctx(const bsr_handle* h, void* stream) {
   c.use_tc = h->use_tc;
   c.split_ws = h->split_floats ? h->at<float>(h->off_split) : nullptr;
   c.split_ws_floats = h->split_floats;
+  c.prof = const_cast<GemmProfile*>(&h->prof);
   return c;
 }
 
@@ -642,6 +645,8 @@ int32_t bsr_create(const bsr_config* cfg, void* workspace, size_t bytes, bsr_han
 }
 
 int32_t bsr_destroy(bsr_handle* h) {
+  if (h != nullptr)
+    for (cudaEvent_t ev : h->prof.events) cudaEventDestroy(ev);
   delete h;
   return BSR_OK;
 }
@@ -832,6 +837,31 @@ int32_t bsr_sync_status(bsr_handle* h, void* stream) {
   if (e != cudaSuccess) return set_err(h->err, BSR_ERR_CUDA, "bsr_sync_status: %s", cudaGetErrorString(e));
   if (st & STATUS_TIMEOUT) return set_err(h->err, BSR_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired");
   if (st & STATUS_NONFINITE) return set_err(h->err, BSR_ERR_NONFINITE, "the loss was not finite");
+  return BSR_OK;
+}
+
+int32_t bsr_profile_enable(bsr_handle* h, int32_t time_gemms) {
+  if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
+  h->prof.on = time_gemms != 0;
+  h->prof.used = 0;
+  h->prof.flops = 0.0;
+  h->launches_at_enable = g_kernel_launches;
+  return BSR_OK;
+}
+
+int32_t bsr_profile_read(bsr_handle* h, void* stream, bsr_profile* out) {
+  if (h == nullptr || out == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "null argument");
+  cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) return set_err(h->err, BSR_ERR_CUDA, "bsr_profile_read: %s", cudaGetErrorString(e));
+  double ms = 0.0;
+  for (size_t i = 0; i + 1 < h->prof.used; i += 2) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, h->prof.events[i], h->prof.events[i + 1]) == cudaSuccess) ms += t;
+  }
+  out->kernel_launches = (uint64_t)(g_kernel_launches - h->launches_at_enable);
+  out->gemm_launches = h->prof.used / 2;
+  out->gemm_flops = h->prof.flops;
+  out->gemm_ms = ms;
   return BSR_OK;
 }
 

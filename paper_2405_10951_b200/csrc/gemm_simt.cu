@@ -82,6 +82,7 @@ void gemm(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long
     if (gemm_tc_strided(c, A, a_rs, a_cs, B, b_rs, b_cs, C, out_is_float, m, n, k, e, c.split_ws, c.split_ws_floats) == 0) return;
   }
   dim3 grid(ceil_div(n, SG_BN), ceil_div(m, SG_BM));
+  note_launch(1);
   if (c.dtype == 0) {
     gemm_simt_kernel<float, float><<<grid, SG_THREADS, 0, c.stream>>>(
         (const float*)A, a_rs, a_cs, (const float*)B, b_rs, b_cs, (float*)C, m, n, k, e.bias, (const float*)e.residual,

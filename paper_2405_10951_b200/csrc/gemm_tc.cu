@@ -370,6 +370,7 @@ static int launch(const Ctx& c, const CUtensorMap& ma, const CUtensorMap& mb, vo
   int work = tiles_m * tiles_n * splits;
   int sms = c.sm_count > 0 ? c.sm_count : 148;
   int grid = work < sms ? work : sms;
+  note_launch(1);
   kern<<<grid, THREADS, SMEM_BYTES, c.stream>>>(ma, mb, (TOut*)C, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, c.status);
   return 0;
 }
@@ -411,6 +412,7 @@ int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const voi
   Epi ep;
   ep.bias = e.bias; ep.residual = e.residual; ep.aux_out = e.aux_out; ep.aux_in = e.aux_in; ep.act = e.act;
   void* dst = (splits > 1) ? (void*)split_ws : C;
+  if (c.prof != nullptr && c.prof->on) c.prof->begin(c.stream, 2.0 * m * n * (double)k);
   int rc;
   if (out_is_float) {
     if (a_mn) rc = launch<true, true, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split);
@@ -424,8 +426,10 @@ int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const voi
   if (rc != 0) return rc;
   if (splits > 1) {
     size_t total = (size_t)m * n;
+    note_launch(1);
     splitk_reduce_kernel<<<ceil_div((long)(total / 4), 256), 256, 0, c.stream>>>(split_ws, (float*)C, total, splits);
   }
+  if (c.prof != nullptr && c.prof->on) c.prof->end(c.stream);
   return 0;
 }
 

@@ -8,7 +8,31 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <vector>
+
 namespace bsr {
+
+// Optional timing of the tensor-core GEMM launches: each launch is bracketed by a pair of CUDA events on the
+// launching stream (events are host objects; no device memory is involved).
+struct GemmProfile {
+  bool on = false;
+  std::vector<cudaEvent_t> events;   // pairs
+  size_t used = 0;
+  double flops = 0.0;
+  void begin(cudaStream_t s, double f) {
+    if (used + 2 > events.size()) {
+      size_t old = events.size();
+      events.resize(old + 512);
+      for (size_t i = old; i < events.size(); ++i) cudaEventCreate(&events[i]);
+    }
+    cudaEventRecord(events[used], s);
+    flops += f;
+  }
+  void end(cudaStream_t s) {
+    cudaEventRecord(events[used + 1], s);
+    used += 2;
+  }
+};
 
 struct Ctx {
   cudaStream_t stream;
@@ -18,6 +42,7 @@ struct Ctx {
   int use_tc;       // bf16 only: dense contractions on the tcgen05 kernels
   float* split_ws = nullptr;       // scratch for split-k partial sums (optional)
   size_t split_ws_floats = 0;
+  GemmProfile* prof = nullptr;
 };
 
 inline size_t dtype_size(int dtype) { return dtype == 0 ? 4 : 2; }

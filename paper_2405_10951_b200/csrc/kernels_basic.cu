@@ -5,6 +5,8 @@
 
 namespace bsr {
 
+long g_kernel_launches = 0;
+
 // ------------------------------------------------------------------------------------------------
 // Patch extraction (Section 3.1: the image is partitioned into N patches).  Output row = one patch
 // flattened as (channel, row in patch, column in patch).
@@ -24,6 +26,7 @@ __global__ void patchify_kernel(const T* __restrict__ img, T* __restrict__ out, 
 }
 
 void patchify(const Ctx& c, const void* images, void* patches, int B, int C, int S, int P) {
+  note_launch(1);
   int g = S / P;
   long total = (long)B * g * g * C * P * P;
   int threads = 256;
@@ -48,6 +51,7 @@ __global__ void assemble_kernel(const T* __restrict__ emb, const float* __restri
 }
 
 void assemble_tokens(const Ctx& c, const void* emb, const float* cls, const float* pos, float* x, int B, int N, int D) {
+  note_launch(1);
   long total = (long)B * (N + 1) * D;
   int threads = 256, blocks = ceil_div(total, threads);
   if (c.dtype == 0)
@@ -117,6 +121,7 @@ __global__ void layernorm_fwd_kernel(const float* __restrict__ x, long x_stride,
 
 void layernorm_fwd(const Ctx& c, const float* x, long x_stride, const float* g, const float* b, void* y, int y_is_float,
                    float* mean, float* rstd, int rows, int D, float eps) {
+  note_launch(1);
   int threads = 256;
   int blocks = ceil_div((long)rows * 32, threads);
   if (c.dtype == 0 || y_is_float)
@@ -243,6 +248,7 @@ static void launch_ln_bwd(const Ctx& c, int groups, size_t smem, const void* dy,
 void layernorm_bwd(const Ctx& c, const void* dy, int dy_is_float, const float* x, long x_stride, const float* mean,
                    const float* rstd, const float* g, const float* dres, float* dx, long dx_stride, void* dx_copy,
                    float* partials, float* dgamma, float* dbeta, int rows, int D) {
+  note_launch(3);
   int groups = layernorm_bwd_groups(c, rows);
   size_t smem = (size_t)LNB_WARPS * 2 * D * sizeof(float);
   if (c.dtype == 0)
@@ -299,6 +305,7 @@ int colsum_groups(int rows) {
 }
 
 void colsum(const Ctx& c, const void* x, int rows, int cols, float* partials, float* out) {
+  note_launch(2);
   int groups = colsum_groups(rows);
   int threads = CS_ROWLANES * 32;
   if (c.dtype == 0) {
@@ -350,6 +357,7 @@ static HeadDev to_dev(const HeadDesc& h) {
 }
 
 void head_fwd(const Ctx& c, const HeadDesc& h, const float* xn, const int* task_ids, float* logits, int B) {
+  note_launch(1);
   int threads = 256, blocks = ceil_div((long)B * h.cmax * 32, threads);
   if (c.dtype == 0) head_fwd_kernel<float><<<blocks, threads, 0, c.stream>>>(to_dev(h), xn, task_ids, logits, B);
   else head_fwd_kernel<bf16><<<blocks, threads, 0, c.stream>>>(to_dev(h), xn, task_ids, logits, B);
@@ -395,6 +403,7 @@ __global__ void loss_reduce_kernel(const float* __restrict__ per_image, int B, f
 
 void cross_entropy(const Ctx& c, const HeadDesc& h, const float* logits, const int* labels, const int* task_ids,
                    float* per_image, float* dlogits, float* loss, int B) {
+  note_launch(2);
   int threads = 128, blocks = ceil_div((long)B * 32, threads);
   cross_entropy_kernel<<<blocks, threads, 0, c.stream>>>(to_dev(h), logits, labels, task_ids, per_image, dlogits, B);
   loss_reduce_kernel<<<1, 32, 0, c.stream>>>(per_image, B, loss, c.status);
@@ -432,6 +441,7 @@ __global__ void head_dgrad_kernel(HeadDev h, const float* __restrict__ dlogits, 
 }
 
 void head_bwd(const Ctx& c, const HeadDesc& h, const float* xn, const float* dlogits, const int* task_ids, float* dxn, int B) {
+  note_launch(h.num_tasks + 1);
   HeadDev hd = to_dev(h);
   for (int t = 0; t < h.num_tasks; ++t) {
     int total = h.ncls[t] * (h.D + 1);
@@ -471,6 +481,7 @@ __global__ void adamw_kernel(const AdamChunk* __restrict__ chunks, float* __rest
 void adamw(const Ctx& c, const AdamChunk* chunks, int nchunks, float* master, const float* grad, float* m, float* v,
            void* shadow_base, float lr, float b1, float b2, float eps, float wd, float bc1, float bc2) {
   if (nchunks <= 0) return;
+  note_launch(1);
   if (c.dtype == 0)
     adamw_kernel<float><<<nchunks, 256, 0, c.stream>>>(chunks, master, grad, m, v, (float*)shadow_base, lr, b1, b2, eps, wd, bc1, bc2);
   else
@@ -496,18 +507,21 @@ __global__ void fill_kernel(float* d, float v, size_t n) {
 }
 
 void convert_from_float(const Ctx& c, const float* src, void* dst, size_t n) {
+  note_launch(1);
   if (n == 0) return;
   int blocks = ceil_div((long)n, 256);
   if (c.dtype == 0) from_float_kernel<float><<<blocks, 256, 0, c.stream>>>(src, (float*)dst, n);
   else from_float_kernel<bf16><<<blocks, 256, 0, c.stream>>>(src, (bf16*)dst, n);
 }
 void convert_to_float(const Ctx& c, const void* src, float* dst, size_t n) {
+  note_launch(1);
   if (n == 0) return;
   int blocks = ceil_div((long)n, 256);
   if (c.dtype == 0) to_float_kernel<float><<<blocks, 256, 0, c.stream>>>((const float*)src, dst, n);
   else to_float_kernel<bf16><<<blocks, 256, 0, c.stream>>>((const bf16*)src, dst, n);
 }
 void fill_float(cudaStream_t s, float* dst, float v, size_t n) {
+  note_launch(1);
   if (n == 0) return;
   fill_kernel<<<ceil_div((long)n, 256), 256, 0, s>>>(dst, v, n);
 }

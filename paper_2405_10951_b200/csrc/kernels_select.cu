@@ -64,6 +64,7 @@ __global__ void token_select_kernel(const float* __restrict__ p, int B, int H, i
 }
 
 void token_select(cudaStream_t s, const float* p, int B, int H, int M, int k, float* scores, int* kept, int* dropped) {
+  note_launch(1);
   size_t smem = (size_t)SEL_WARPS * M * sizeof(uint32_t);
   if (smem > 48 * 1024) cudaFuncSetAttribute(token_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   token_select_kernel<<<ceil_div(B, SEL_WARPS), SEL_WARPS * 32, smem, s>>>(p, B, H, M, k, scores, kept, dropped);
@@ -138,6 +139,7 @@ __global__ void gather_fuse_kernel(const T* __restrict__ x, int M, int D, int k,
 
 void gather_fuse(const Ctx& c, const void* x, int B, int M, int D, int k, const int* kept, const int* dropped,
                  const float* scores, int fuse, void* out) {
+  note_launch(1);
   int n = (c.dtype == 0) ? 4 : 8;
   int chunks = D / n;
   int do_fuse = (fuse == 1 && k < M) ? 1 : 0;
@@ -204,6 +206,7 @@ __global__ void gather_fuse_bwd_kernel(const float* __restrict__ dout, const flo
 
 void gather_fuse_bwd(const Ctx& c, const void* dout, const void* x, int B, int M, int D, int k, const int* kept,
                      const int* dropped, const float* scores, int fuse, void* dx, void* dx_copy, float* escore) {
+  note_launch(1);
   int do_fuse = (fuse == 1 && k < M) ? 1 : 0;
   int threads = 256, blocks = ceil_div((long)B * (1 + M) * 32, threads);
   gather_fuse_bwd_kernel<<<blocks, threads, 0, c.stream>>>((const float*)dout, (const float*)x, B, M, D, k, kept, dropped, scores,

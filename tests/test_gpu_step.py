@@ -47,8 +47,8 @@ def test_bf16_step_matches_oracle(case):
     cfg = BF16_CASES[case]
     images, labels, task_ids, params = synth.make_workload(cfg, peaked=True)
     gpu = P.run_gpu_step(cfg, images, labels, task_ids, params)
-    rep = P.compare_step(cfg, images, labels, task_ids, params, gpu, P.BF16_TOL, 10 * P.BF16_SCORE_TOL, P.BF16_SCORE_TOL)
-    assert rep["sets_identical"] >= 0.8 * rep["sets"], rep
+    rep = P.compare_step(cfg, images, labels, task_ids, params, gpu, P.BF16_TOL, 2 * P.BF16_SCORE_TOL, P.BF16_SCORE_TOL)
+    assert rep["sets_identical"] >= 0.6 * rep["sets"], rep
 
 
 def test_eval_forward_matches_oracle_and_train_forward():
