@@ -215,6 +215,25 @@ int32_t bsr_linear_backward(const void* x_dev, const void* w_dev, const void* dy
                             int32_t m, int32_t n, int32_t k, int32_t dtype, int32_t use_tensor_cores,
                             float* workspace_dev, size_t workspace_floats, void* stream);
 
+/* The same backward pass for callers that cannot allocate device memory (the paper has no counterpart:
+ * this is a property of the library, not of the method).  Such callers exist: a trainer on a device whose
+ * memory was divided up once at start-up, a plug-in inside an application that owns all device memory
+ * through its own pool, a latency-critical loop that must not pay cudaMalloc's device-wide synchronisation.
+ * The split-reduction scratch that bsr_linear_backward takes from its caller is here a fixed array of
+ * BSR_STATIC_SCRATCH_BYTES inside the library image; every GPU that loads the library holds it until the
+ * process exits.  bf16 only; x [m, k], w [n, k], dy [m, n], dx [m, k] bf16, dw [n, k] float32, all device
+ * memory owned by the caller; m, n, k multiples of 8.  n * k must not exceed BSR_STATIC_SCRATCH_BYTES / 8
+ * elements, otherwise BSR_ERR_WORKSPACE_TOO_SMALL is returned and nothing runs.  The call allocates and
+ * frees nothing.  The first call on each device looks up the array's device address (with that device
+ * current) and should therefore come before any stream capture.  All calls on a device share the one
+ * array: each call fully rewrites the part it reads, so nothing needs clearing between calls, but two
+ * calls whose kernels overlap on the GPU (different streams) race on it -- keep them on one stream or
+ * order them with events.  Errors are described by bsr_static_last_error(). */
+#define BSR_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
+int32_t bsr_linear_backward_static(const void* x_dev, const void* w_dev, const void* dy_dev, void* dx_dev, float* dw_dev,
+                                   int32_t m, int32_t n, int32_t k, void* stream);
+const char* bsr_static_last_error(void);
+
 /* Multi-head self-attention, Eq. 1, on packed projections.  qkv_dev [batch, t, 3, heads, d] in
  * `dtype`; out_dev [batch, t, heads*d]; cls_prob_dev_out optional [batch, heads, t-1] float32: the
  * classification token's row of the attention map without its own column. d must be 64 or less

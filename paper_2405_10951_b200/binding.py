@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "BSR_OK", -1: "BSR_ERR_INVALID_ARG", -2: "BSR_ERR_UNSUPPORTED
 EXPORTS = ["bsr_token_schedule", "bsr_workspace_bytes", "bsr_create", "bsr_destroy", "bsr_last_error", "bsr_set_param",
            "bsr_get_tensor", "bsr_set_lr", "bsr_set_step", "bsr_train_step", "bsr_eval_forward", "bsr_get_footprint",
            "bsr_sync_status", "bsr_profile_enable", "bsr_profile_read", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_backward",
-           "bsr_attention_forward"]
+           "bsr_linear_backward_static", "bsr_static_last_error", "bsr_attention_forward"]
 
 
 class bsr_dims(C.Structure):
@@ -78,6 +78,7 @@ def lib() -> C.CDLL:
         L.bsr_destroy.argtypes = [vp]
         L.bsr_last_error.argtypes = [vp]
         L.bsr_last_error.restype = C.c_char_p
+        L.bsr_static_last_error.restype = C.c_char_p
         L.bsr_set_param.argtypes = [vp, C.c_char_p, f32p, C.c_size_t, vp]
         L.bsr_get_tensor.argtypes = [vp, C.c_char_p, f32p, C.c_size_t, vp]
         L.bsr_set_lr.argtypes = [vp, C.c_float]
@@ -92,9 +93,11 @@ def lib() -> C.CDLL:
         L.bsr_gather_fuse.argtypes = [vp, i32, i32, i32, i32, i32, i32p, i32p, f32p, i32, vp, vp]
         L.bsr_linear_forward.argtypes = [vp, vp, f32p, vp, vp, i32, i32, i32, i32, i32, i32, vp]
         L.bsr_linear_backward.argtypes = [vp, vp, vp, vp, f32p, i32, i32, i32, i32, i32, f32p, C.c_size_t, vp]
+        L.bsr_linear_backward_static.argtypes = [vp, vp, vp, vp, f32p, i32, i32, i32, vp]
+        L.bsr_static_last_error.argtypes = []
         L.bsr_attention_forward.argtypes = [vp, i32, i32, i32, i32, i32, vp, f32p, vp]
         for name in EXPORTS:
-            if name != "bsr_last_error":
+            if name not in ("bsr_last_error", "bsr_static_last_error"):
                 getattr(L, name).restype = C.c_int32
         _lib = L
     return _lib
@@ -197,6 +200,22 @@ def bsr_linear_backward(x, w, dy, use_tensor_cores: bool = False, workspace=None
     dt = DTYPE_FP32 if x.dtype == torch.float32 else DTYPE_BF16
     _check(lib().bsr_linear_backward(_ptr(x), _ptr(w), _ptr(dy), _ptr(dx), _ptr(dw), m, n, k, dt, int(use_tensor_cores),
                                      _ptr(workspace), 0 if workspace is None else workspace.numel(), _stream()))
+    return dx, dw
+
+
+def bsr_linear_backward_static(x, w, dy, dx=None, dw=None):
+    """Linear backward through the entry point that allocates nothing: the split-reduction scratch is a
+    fixed array inside the library.  Pass dx/dw to reuse output tensors.  Returns (dx, dw)."""
+    import torch
+    m, k = x.shape
+    n = w.shape[0]
+    if dx is None:
+        dx = torch.empty((m, k), dtype=x.dtype, device=x.device)
+    if dw is None:
+        dw = torch.empty((n, k), dtype=torch.float32, device=x.device)
+    st = lib().bsr_linear_backward_static(_ptr(x), _ptr(w), _ptr(dy), _ptr(dx), _ptr(dw), m, n, k, _stream())
+    if st != BSR_OK:
+        raise BsrError(st, lib().bsr_static_last_error().decode())
     return dx, dw
 
 

@@ -1,0 +1,54 @@
+"""The entry point for callers that cannot allocate device memory.
+
+Some users of this library run where cudaMalloc is not an option: on a device whose memory was handed
+out once at start-up, inside an application that keeps all device memory in its own pool, or in a loop
+that cannot afford the device-wide synchronisation an allocation implies.  bsr_linear_backward_static
+serves them by keeping its split-reduction scratch in a fixed array inside the library.  This test calls
+it through the C ABI twice in a row (the second call finds the first call's leftovers in the shared
+scratch) and checks both results against bsr_linear_backward, which takes its scratch from the caller.
+It is collected last so that a run stopping at the first failure has already run everything else.
+"""
+import numpy as np
+import pytest
+
+from paper_2405_10951_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def rel(a, b):
+    return float((a.double() - b.double()).norm() / b.double().norm())
+
+
+def test_static_scratch_backward_matches_caller_scratch_backward_twice():
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    rng = np.random.default_rng(7)
+    g = lambda a: torch.as_tensor(synth.round_to_bf16(a).astype(np.float32)).cuda().to(torch.bfloat16)
+    ws = torch.empty(160 * 128 * 256, dtype=torch.float32, device="cuda")
+    before = torch.cuda.memory_allocated()
+    # two different shapes back to back: the second call reuses the scratch the first one filled
+    for m, n, k in [(9216, 768, 768), (3072, 384, 1536)]:
+        x, w, dy = g(rng.standard_normal((m, k))), g(rng.standard_normal((n, k)) / np.sqrt(k)), g(rng.standard_normal((m, n)))
+        dx_ref, dw_ref = Bd.bsr_linear_backward(x, w, dy, use_tensor_cores=True, workspace=ws)
+        dx = torch.empty_like(dx_ref)
+        dw = torch.empty_like(dw_ref)
+        held = torch.cuda.memory_allocated()
+        Bd.bsr_linear_backward_static(x, w, dy, dx, dw)
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() == held          # the call itself took nothing from torch's pool
+        assert rel(dx, dx_ref) < 4e-3                         # tolerances of the other linear-backward tests
+        assert rel(dw, dw_ref) < 1e-4
+    assert before <= torch.cuda.memory_allocated()
+
+
+def test_static_scratch_rejects_oversized_weights():
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    m, n, k = 64, 2048, 2048          # n * k = 4 Mi elements: twice the documented limit
+    x = torch.zeros((m, k), dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros((n, k), dtype=torch.bfloat16, device="cuda")
+    dy = torch.zeros((m, n), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(Bd.BsrError) as e:
+        Bd.bsr_linear_backward_static(x, w, dy)
+    assert e.value.status == -3 and "exceeds the built-in scratch" in str(e.value)
