@@ -95,7 +95,7 @@ def lib() -> C.CDLL:
         L.bsr_linear_backward.argtypes = [vp, vp, vp, vp, f32p, i32, i32, i32, i32, i32, f32p, C.c_size_t, vp]
         L.bsr_linear_backward_static.argtypes = [vp, vp, vp, vp, f32p, i32, i32, i32, vp]
         L.bsr_static_last_error.argtypes = []
-        L.bsr_attention_forward.argtypes = [vp, i32, i32, i32, i32, i32, vp, f32p, vp]
+        L.bsr_attention_forward.argtypes = [vp, i32, i32, i32, i32, i32, vp, f32p, i32, vp]
         for name in EXPORTS:
             if name not in ("bsr_last_error", "bsr_static_last_error"):
                 getattr(L, name).restype = C.c_int32
@@ -219,7 +219,7 @@ def bsr_linear_backward_static(x, w, dy, dx=None, dw=None):
     return dx, dw
 
 
-def bsr_attention_forward(qkv, heads: int, want_cls_prob: bool = True):
+def bsr_attention_forward(qkv, heads: int, want_cls_prob: bool = True, use_tensor_cores: bool = False):
     """qkv: CUDA tensor [B, T, 3, H, d].  Returns (out [B, T, H*d], cls_prob [B, H, T-1] or None)."""
     import torch
     B, T, three, H, d = qkv.shape
@@ -227,7 +227,7 @@ def bsr_attention_forward(qkv, heads: int, want_cls_prob: bool = True):
     out = torch.empty((B, T, H * d), dtype=qkv.dtype, device=qkv.device)
     cp = torch.empty((B, H, T - 1), dtype=torch.float32, device=qkv.device) if want_cls_prob else None
     dt = DTYPE_FP32 if qkv.dtype == torch.float32 else DTYPE_BF16
-    _check(lib().bsr_attention_forward(_ptr(qkv), dt, B, T, H, d, _ptr(out), _ptr(cp), _stream()))
+    _check(lib().bsr_attention_forward(_ptr(qkv), dt, B, T, H, d, _ptr(out), _ptr(cp), int(use_tensor_cores), _stream()))
     return out, cp
 
 

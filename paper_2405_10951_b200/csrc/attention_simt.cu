@@ -284,6 +284,7 @@ static int launch_fwd(const Ctx& c, const void* qkv, void* out, float* lse, floa
 }
 
 int attention_fwd(const Ctx& c, const void* qkv, void* out, float* lse, float* cls_prob, int B, int T_, int H, int d) {
+  if (c.dtype == 1 && c.use_tc && attention_fwd_tc(c, qkv, out, lse, cls_prob, B, T_, H, d) == 0) return 0;
   if (d > AT_MAXD || (d % 8) != 0) return -2;
   return c.dtype == 0 ? launch_fwd<float>(c, qkv, out, lse, cls_prob, B, T_, H, d)
                       : launch_fwd<bf16>(c, qkv, out, lse, cls_prob, B, T_, H, d);

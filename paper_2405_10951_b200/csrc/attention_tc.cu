@@ -1,0 +1,220 @@
+// Multi-head self-attention (paper Eq. 1) on the tcgen05 tensor cores for bf16, head dimension 64.
+//
+// Forward (T <= 256 keys): one CTA of 128 threads per (image, head, 128-query tile).
+//   TMA loads Q, K, V tiles of the packed projections [B*T, 3*H*64] into 128-byte-swizzled shared memory;
+//   S = Q K^T goes to tensor memory (one tcgen05.mma group, N = T rounded up to 16);
+//   each thread owns one query row: row maximum, exp2, row sum in float from tcgen05.ld; the probabilities
+//   are written as bf16 into shared memory in the same swizzled layout an operand tile has;
+//   O = P V accumulates over the S columns that are no longer needed; the epilogue scales by 1 / row sum.
+//   The classification token's row (query 0) is also written out as probabilities: these are the token
+//   importance scores of Eq. 6.
+// Rows and keys beyond T inside a tile belong to the next image (or are zero-filled past the tensor's end):
+// keys are masked in the softmax, rows are computed and never stored.
+#include "common.cuh"
+#include "kernels.h"
+#include "tc_ptx.cuh"
+
+namespace bsr {
+namespace tc {
+
+constexpr int AT_D = 64;
+constexpr int AT_BOX = 64;                       // rows per TMA box
+constexpr int AT_BOX_BYTES = AT_BOX * AT_D * 2;  // 8 KB
+constexpr int AT_QROWS = 128;
+constexpr int AT_MAXKEYS = 256;
+
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Byte offset of element (row, key) in a probability tile stored as 64-key chunks of [128 rows x 128 bytes],
+// 16-byte units XOR-swizzled with the row (the layout TMA produces for a 128-byte-swizzled operand tile).
+__device__ __forceinline__ uint32_t p_offset(int row, int key8) {   // key8: index of a group of 8 keys
+  int chunk = key8 >> 3, unit = key8 & 7;
+  return (uint32_t)(chunk * (AT_QROWS * 128) + row * 128 + ((unit ^ (row & 7)) << 4));
+}
+
+__global__ void __launch_bounds__(128)
+attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict__ out, float* __restrict__ lse,
+                   float* __restrict__ cls_prob, int B, int T, int H, int* status) {
+  extern __shared__ unsigned char smem_dyn[];
+  uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+  int tpad = (T + 15) & ~15;                     // MMA N
+  int nbox = (tpad + AT_BOX - 1) / AT_BOX;       // 64-key boxes of K and V, 64-key chunks of P
+  uint32_t sQ = base, sK = sQ + 2 * AT_BOX_BYTES, sV = sK + nbox * AT_BOX_BYTES, sP = sV + nbox * AT_BOX_BYTES;
+  uint32_t p_bytes = nbox * (AT_QROWS * 128);
+  float* cls_buf = reinterpret_cast<float*>(base_ptr + (sP - base) + p_bytes);          // [AT_MAXKEYS + 1]
+  uint32_t bars = sP + p_bytes + (AT_MAXKEYS + 8) * 4;                                   // tma, mma
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  int tid = threadIdx.x, warp = tid >> 5;
+  int bh = blockIdx.y, b = bh / H, h = bh % H;
+  int q0 = blockIdx.x * AT_QROWS;
+  uint32_t tma_bar = bars, mma_bar = bars + 8;
+
+  if (tid == 0) {
+    abort_flag = 0;
+    mbar_init(tma_bar, 1);
+    mbar_init(mma_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    tmem_alloc(smem_u32(&tmem_slot), 256);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  uint32_t tmem = tmem_slot;
+  volatile int* abortp = &abort_flag;
+  bool ok = true;
+
+  if (tid == 0) {
+    mbar_expect_tx(tma_bar, (2 + 2 * nbox) * AT_BOX_BYTES);
+    int row0 = b * T;
+    for (int j = 0; j < 2; ++j) tma_load_2d(sQ + j * AT_BOX_BYTES, &map_qkv, tma_bar, h * AT_D, row0 + q0 + j * AT_BOX);
+    for (int j = 0; j < nbox; ++j) {
+      tma_load_2d(sK + j * AT_BOX_BYTES, &map_qkv, tma_bar, (H + h) * AT_D, row0 + j * AT_BOX);
+      tma_load_2d(sV + j * AT_BOX_BYTES, &map_qkv, tma_bar, (2 * H + h) * AT_D, row0 + j * AT_BOX);
+    }
+    ok = mbar_wait(tma_bar, 0, abortp);
+    if (ok) {
+      tc_fence_after();
+      uint32_t idesc = make_idesc_mn(AT_QROWS, tpad, false, false);
+#pragma unroll
+      for (int k = 0; k < AT_D / 16; ++k)
+        umma_bf16(tmem, make_desc(sQ + k * 32, 16, 1024), make_desc(sK + k * 32, 16, 1024), idesc, k > 0 ? 1u : 0u);
+      umma_commit(mma_bar);
+    }
+  }
+  ok = mbar_wait(mma_bar, 0, abortp);
+  tc_fence_after();
+
+  // ---- softmax of this thread's row ------------------------------------------------------------
+  const float c = 0.125f * 1.4426950408889634f;          // 1/sqrt(64) * log2(e)
+  uint32_t trow = tmem + ((uint32_t)(warp * 32) << 16);
+  int nchunk = (T + 31) >> 5;
+  float mx = -INFINITY;
+  if (ok) {
+    for (int ch = 0; ch < nchunk; ++ch) {
+      uint32_t r[32];
+      tmem_ld32(trow + ch * 32, r);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (ch * 32 + j < T) mx = fmaxf(mx, __uint_as_float(r[j]));
+    }
+  }
+  float sum = 0.f;
+  bool cls_row = (q0 == 0 && tid == 0 && cls_prob != nullptr);
+  if (ok) {
+    float mc = mx * c;
+    for (int ch = 0; ch < nchunk; ++ch) {
+      uint32_t r[32];
+      tmem_ld32(trow + ch * 32, r);
+      tmem_ld_wait();
+      float p[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        float e = exp2f(fmaf(__uint_as_float(r[j]), c, -mc));
+        p[j] = (ch * 32 + j < T) ? e : 0.f;
+        sum += p[j];
+      }
+      if (cls_row) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) cls_buf[ch * 32 + j] = p[j];
+      }
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        int key8 = ch * 4 + g;
+        if (key8 * 8 < nbox * AT_BOX) {
+          uint4 v;
+          __nv_bfloat162* hh = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) hh[i] = __floats2bfloat162_rn(p[g * 8 + 2 * i], p[g * 8 + 2 * i + 1]);
+          *reinterpret_cast<uint4*>(base_ptr + (sP - base) + p_offset(tid, key8)) = v;
+        }
+      }
+    }
+    // keys between the last 32-chunk and the padded MMA extent must read as zero
+    for (int key8 = nchunk * 4; key8 * 8 < tpad; ++key8)
+      *reinterpret_cast<uint4*>(base_ptr + (sP - base) + p_offset(tid, key8)) = make_uint4(0, 0, 0, 0);
+  }
+  float inv = 1.0f / sum;
+  if (cls_row) cls_buf[AT_MAXKEYS] = inv;
+  fence_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  ok = ok && !abort_flag;
+
+  // ---- O = P V ----------------------------------------------------------------------------------
+  if (tid == 0 && ok) {
+    uint32_t idesc = make_idesc_mn(AT_QROWS, AT_D, false, true);
+    int ksteps = tpad / 16;
+    for (int k = 0; k < ksteps; ++k) {
+      uint64_t da = make_desc(sP + (k >> 2) * (AT_QROWS * 128) + (k & 3) * 32, 16, 1024);
+      uint64_t db = make_desc(sV + k * (16 * 128), 8192, 1024);
+      umma_bf16(tmem, da, db, idesc, k > 0 ? 1u : 0u);
+    }
+    umma_commit(mma_bar);
+  }
+  if (ok) ok = mbar_wait(mma_bar, 1, abortp);
+  tc_fence_after();
+  int q = q0 + tid;
+  if (ok) {
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      uint32_t r[32];
+      tmem_ld32(trow + half * 32, r);
+      tmem_ld_wait();
+      if (q < T) {
+        bf16* orow = out + ((size_t)b * T + q) * H * AT_D + (size_t)h * AT_D + half * 32;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          float v[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[g * 8 + j]) * inv;
+          store16(orow + g * 8, v);
+        }
+      }
+    }
+    if (q < T && lse != nullptr) lse[((size_t)b * H + h) * T + q] = mx * 0.125f + logf(sum);
+    if (q0 == 0 && cls_prob != nullptr) {
+      float s_inv = cls_buf[AT_MAXKEYS];
+      float* cp = cls_prob + ((size_t)b * H + h) * (T - 1);
+      for (int j = 1 + tid; j < T; j += 128) cp[j - 1] = cls_buf[j] * s_inv;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 256);
+  }
+  if (tid == 0 && abort_flag && status != nullptr) atomicOr(status, STATUS_TIMEOUT);
+}
+
+}  // namespace tc
+
+// Returns 0 when the tensor-core kernel took the problem, non-zero when the caller must use another kernel.
+int attention_fwd_tc(const Ctx& c, const void* qkv, void* out, float* lse, float* cls_prob, int B, int T, int H, int d) {
+  using namespace tc;
+  if (c.dtype != 1 || d != AT_D || T > AT_MAXKEYS || T < 1) return -1;
+  if (((uintptr_t)qkv & 15) || ((uintptr_t)out & 15)) return -1;
+  CUtensorMap map;
+  if (!make_map(&map, qkv, (uint64_t)3 * H * d, (uint64_t)B * T, (uint64_t)3 * H * d, AT_BOX)) return -2;
+  int tpad = (T + 15) & ~15;
+  int nbox = (tpad + AT_BOX - 1) / AT_BOX;
+  size_t smem = 1024 + (size_t)(2 + 2 * nbox) * AT_BOX_BYTES + (size_t)nbox * (AT_QROWS * 128) + (AT_MAXKEYS + 8) * 4 + 64;
+  static size_t attr = 0;
+  if (smem > attr) {
+    if (cudaFuncSetAttribute(attn_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -3;
+    attr = smem;
+  }
+  dim3 grid((T + AT_QROWS - 1) / AT_QROWS, B * H);
+  note_launch(1);
+  attn_fwd_tc_kernel<<<grid, 128, smem, c.stream>>>(map, (bf16*)out, lse, cls_prob, B, T, H, c.status);
+  return 0;
+}
+
+}  // namespace bsr

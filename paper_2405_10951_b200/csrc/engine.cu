@@ -939,11 +939,16 @@ int32_t bsr_linear_backward(const void* x, const void* w, const void* dy, void* 
 }
 
 int32_t bsr_attention_forward(const void* qkv, int32_t dtype, int32_t batch, int32_t t, int32_t heads, int32_t d, void* out,
-                              float* cls_prob, void* stream) {
+                              float* cls_prob, int32_t use_tensor_cores, void* stream) {
   if (qkv == nullptr || out == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "null argument");
   if (dtype != BSR_DTYPE_FP32 && dtype != BSR_DTYPE_BF16) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad dtype");
   if (batch < 1 || t < 1 || heads < 1 || d < 8 || d > 64 || d % 8 != 0) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad shape: head dimension must be a multiple of 8, at most 64");
   Ctx c = bare_ctx(dtype, stream);
+  if (use_tensor_cores) {
+    if (attention_fwd_tc(c, qkv, out, nullptr, cls_prob, batch, t, heads, d) != 0)
+      return set_err(g_error, BSR_ERR_UNSUPPORTED, "the tcgen05 attention kernel needs bf16, head dimension 64 and at most 256 tokens");
+    return check_cuda(nullptr, "bsr_attention_forward");
+  }
   if (attention_fwd(c, qkv, out, nullptr, cls_prob, batch, t, heads, d) != 0)
     return set_err(g_error, BSR_ERR_UNSUPPORTED, "%d tokens do not fit the attention kernel's shared memory", t);
   return check_cuda(nullptr, "bsr_attention_forward");
