@@ -310,6 +310,7 @@ static int launch_bwd(const Ctx& c, const void* qkv, const void* dout, const flo
 int attention_bwd(const Ctx& c, const void* qkv, const void* out, const void* dout, const float* lse, float* delta,
                   const float* cls_extra, void* dqkv, int B, int T_, int H, int d) {
   (void)out;
+  if (c.dtype == 1 && c.use_tc && attention_bwd_tc(c, qkv, dout, lse, cls_extra, dqkv, B, T_, H, d) == 0) return 0;
   if (d > AT_MAXD || (d % 8) != 0) return -2;
   return c.dtype == 0 ? launch_bwd<float>(c, qkv, dout, lse, delta, cls_extra, dqkv, B, T_, H, d)
                       : launch_bwd<bf16>(c, qkv, dout, lse, delta, cls_extra, dqkv, B, T_, H, d);

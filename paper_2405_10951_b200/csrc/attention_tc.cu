@@ -87,6 +87,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict
     }
   }
   ok = mbar_wait(mma_bar, 0, abortp);
+  ok = __all_sync(0xffffffffu, ok);               // tcgen05.ld below is warp-collective
   tc_fence_after();
 
   // ---- softmax of this thread's row ------------------------------------------------------------
@@ -159,6 +160,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict
     umma_commit(mma_bar);
   }
   if (ok) ok = mbar_wait(mma_bar, 1, abortp);
+  ok = __all_sync(0xffffffffu, ok);
   tc_fence_after();
   int q = q0 + tid;
   if (ok) {
@@ -194,6 +196,197 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict
   if (tid == 0 && abort_flag && status != nullptr) atomicOr(status, STATUS_TIMEOUT);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Backward (T <= 128): one CTA of 128 threads per (image, head).  With P = exp(S - lse):
+//   dP = dO V^T;  delta_i = sum_j P_ij dP_ij;  dS = P * (dP - delta) / sqrt(d)
+//   dQ = dS K;  dK = dS^T Q;  dV = P^T dO                      (chain rule through Eq. 1, cf. Eq. 3)
+// S and dP are two MMA groups into tensor memory; each thread owns one query row and writes P and dS as
+// bf16 operand tiles into shared memory; the three products then read those tiles K-major (dQ) or through
+// transposing descriptors (dK, dV), so nothing is transposed by hand.  A gradient arriving at the head-mean
+// score of token j (cls_extra[b, j-1], from the fused token) is added to dP of the classification row.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_constant__ CUtensorMap map_do,
+                   const float* __restrict__ lse, const float* __restrict__ cls_extra, bf16* __restrict__ dqkv,
+                   int B, int T, int H, int* status) {
+  extern __shared__ unsigned char smem_dyn[];
+  uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+  constexpr uint32_t TILE = 2 * AT_BOX_BYTES;            // 128 rows x 128 bytes
+  uint32_t sQ = base, sK = sQ + TILE, sV = sK + TILE, sG = sV + TILE, sP = sG + TILE, sS = sP + 2 * TILE;
+  uint32_t bars = sS + 2 * TILE;
+  unsigned char* pP = base_ptr + (sP - base);
+  unsigned char* pS = base_ptr + (sS - base);
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  int tid = threadIdx.x, warp = tid >> 5;
+  int bh = blockIdx.x, b = bh / H, h = bh % H;
+  int tpad = (T + 15) & ~15;
+  uint32_t tma_bar = bars, mma_bar = bars + 8;
+  if (tid == 0) {
+    abort_flag = 0;
+    mbar_init(tma_bar, 1);
+    mbar_init(mma_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    tmem_alloc(smem_u32(&tmem_slot), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  uint32_t tmem = tmem_slot;
+  constexpr uint32_t C_S = 0, C_DP = 128, C_DQ = 256, C_DK = 320, C_DV = 384;
+  volatile int* abortp = &abort_flag;
+  bool ok = true;
+  if (tid == 0) {
+    mbar_expect_tx(tma_bar, 4 * TILE);
+    int row0 = b * T;
+    for (int j = 0; j < 2; ++j) {
+      tma_load_2d(sQ + j * AT_BOX_BYTES, &map_qkv, tma_bar, h * AT_D, row0 + j * AT_BOX);
+      tma_load_2d(sK + j * AT_BOX_BYTES, &map_qkv, tma_bar, (H + h) * AT_D, row0 + j * AT_BOX);
+      tma_load_2d(sV + j * AT_BOX_BYTES, &map_qkv, tma_bar, (2 * H + h) * AT_D, row0 + j * AT_BOX);
+      tma_load_2d(sG + j * AT_BOX_BYTES, &map_do, tma_bar, h * AT_D, row0 + j * AT_BOX);
+    }
+    ok = mbar_wait(tma_bar, 0, abortp);
+    if (ok) {
+      tc_fence_after();
+      uint32_t idesc = make_idesc_mn(AT_QROWS, tpad, false, false);
+#pragma unroll
+      for (int k = 0; k < AT_D / 16; ++k)
+        umma_bf16(tmem + C_S, make_desc(sQ + k * 32, 16, 1024), make_desc(sK + k * 32, 16, 1024), idesc, k > 0 ? 1u : 0u);
+#pragma unroll
+      for (int k = 0; k < AT_D / 16; ++k)
+        umma_bf16(tmem + C_DP, make_desc(sG + k * 32, 16, 1024), make_desc(sV + k * 32, 16, 1024), idesc, k > 0 ? 1u : 0u);
+      umma_commit(mma_bar);
+    }
+  }
+  ok = mbar_wait(mma_bar, 0, abortp);
+  ok = __all_sync(0xffffffffu, ok);
+  tc_fence_after();
+
+  const float c = 0.125f * 1.4426950408889634f;
+  uint32_t trow = tmem + ((uint32_t)(warp * 32) << 16);
+  bool valid_row = tid < T;
+  float l2 = valid_row ? lse[((size_t)b * H + h) * T + tid] * 1.4426950408889634f : 0.f;
+  bool extra_row = (tid == 0 && cls_extra != nullptr);
+  const float* ex = extra_row ? cls_extra + (size_t)b * (T - 1) : nullptr;
+  float invH = 1.0f / (float)H;
+  int nchunk = (T + 31) >> 5;
+  float delta = 0.f;
+  // tcgen05.ld is warp-collective: every lane issues it, rows past T only skip the arithmetic
+  if (ok) {
+    for (int ch = 0; ch < nchunk; ++ch) {
+      uint32_t rs[32], rp[32];
+      tmem_ld32(trow + C_S + ch * 32, rs);
+      tmem_ld32(trow + C_DP + ch * 32, rp);
+      tmem_ld_wait();
+      if (valid_row) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          int key = ch * 32 + j;
+          if (key < T) {
+            float p = exp2f(fmaf(__uint_as_float(rs[j]), c, -l2));
+            float dp = __uint_as_float(rp[j]);
+            if (extra_row && key > 0) dp += ex[key - 1] * invH;
+            delta = fmaf(p, dp, delta);
+          }
+        }
+      }
+    }
+    for (int ch = 0; ch < 4; ++ch) {
+      float p[32], ds[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) { p[j] = 0.f; ds[j] = 0.f; }
+      if (ch < nchunk) {
+        uint32_t rs[32], rp[32];
+        tmem_ld32(trow + C_S + ch * 32, rs);
+        tmem_ld32(trow + C_DP + ch * 32, rp);
+        tmem_ld_wait();
+        if (valid_row) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            int key = ch * 32 + j;
+            if (key < T) {
+              float pv = exp2f(fmaf(__uint_as_float(rs[j]), c, -l2));
+              float dp = __uint_as_float(rp[j]);
+              if (extra_row && key > 0) dp += ex[key - 1] * invH;
+              p[j] = pv;
+              ds[j] = pv * (dp - delta) * 0.125f;
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        uint4 vp, vs;
+        __nv_bfloat162* hp = reinterpret_cast<__nv_bfloat162*>(&vp);
+        __nv_bfloat162* hs = reinterpret_cast<__nv_bfloat162*>(&vs);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          hp[i] = __floats2bfloat162_rn(p[g * 8 + 2 * i], p[g * 8 + 2 * i + 1]);
+          hs[i] = __floats2bfloat162_rn(ds[g * 8 + 2 * i], ds[g * 8 + 2 * i + 1]);
+        }
+        uint32_t off = p_offset(tid, ch * 4 + g);
+        *reinterpret_cast<uint4*>(pP + off) = vp;
+        *reinterpret_cast<uint4*>(pS + off) = vs;
+      }
+    }
+  }
+  fence_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  ok = ok && !abort_flag;
+  if (tid == 0 && ok) {
+    // dQ = dS K: A = dS (contiguous along keys), B = K read with keys as the reduction index
+    uint32_t id_q = make_idesc_mn(AT_QROWS, AT_D, false, true);
+    for (int k = 0; k < tpad / 16; ++k)
+      umma_bf16(tmem + C_DQ, make_desc(sS + (k >> 2) * TILE + (k & 3) * 32, 16, 1024), make_desc(sK + k * 2048, 8192, 1024), id_q,
+                k > 0 ? 1u : 0u);
+    // dK = dS^T Q and dV = P^T dO: both operands read with queries as the reduction index
+    uint32_t id_t = make_idesc_mn(AT_QROWS, AT_D, true, true);
+    for (int k = 0; k < AT_QROWS / 16; ++k)
+      umma_bf16(tmem + C_DK, make_desc(sS + k * 2048, TILE, 1024), make_desc(sQ + k * 2048, 8192, 1024), id_t, k > 0 ? 1u : 0u);
+    for (int k = 0; k < AT_QROWS / 16; ++k)
+      umma_bf16(tmem + C_DV, make_desc(sP + k * 2048, TILE, 1024), make_desc(sG + k * 2048, 8192, 1024), id_t, k > 0 ? 1u : 0u);
+    umma_commit(mma_bar);
+  }
+  if (ok) ok = mbar_wait(mma_bar, 1, abortp);
+  ok = __all_sync(0xffffffffu, ok);
+  tc_fence_after();
+  if (ok) {
+    const uint32_t cols[3] = {C_DQ, C_DK, C_DV};
+#pragma unroll
+    for (int which = 0; which < 3; ++which) {
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        uint32_t r[32];
+        tmem_ld32(trow + cols[which] + half * 32, r);
+        tmem_ld_wait();
+        if (valid_row) {
+          bf16* drow = dqkv + (((size_t)b * T + tid) * 3 + which) * H * AT_D + (size_t)h * AT_D + half * 32;
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[g * 8 + j]);
+            store16(drow + g * 8, v);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+  if (tid == 0 && abort_flag && status != nullptr) atomicOr(status, STATUS_TIMEOUT);
+}
+
 }  // namespace tc
 
 // Returns 0 when the tensor-core kernel took the problem, non-zero when the caller must use another kernel.
@@ -214,6 +407,29 @@ int attention_fwd_tc(const Ctx& c, const void* qkv, void* out, float* lse, float
   dim3 grid((T + AT_QROWS - 1) / AT_QROWS, B * H);
   note_launch(1);
   attn_fwd_tc_kernel<<<grid, 128, smem, c.stream>>>(map, (bf16*)out, lse, cls_prob, B, T, H, c.status);
+  return 0;
+}
+
+}  // namespace bsr
+
+namespace bsr {
+
+int attention_bwd_tc(const Ctx& c, const void* qkv, const void* dout, const float* lse, const float* cls_extra, void* dqkv,
+                     int B, int T, int H, int d) {
+  using namespace tc;
+  if (c.dtype != 1 || d != AT_D || T > AT_QROWS || T < 1) return -1;
+  if (((uintptr_t)qkv & 15) || ((uintptr_t)dout & 15) || ((uintptr_t)dqkv & 15)) return -1;
+  CUtensorMap mq, mg;
+  if (!make_map(&mq, qkv, (uint64_t)3 * H * d, (uint64_t)B * T, (uint64_t)3 * H * d, AT_BOX)) return -2;
+  if (!make_map(&mg, dout, (uint64_t)H * d, (uint64_t)B * T, (uint64_t)H * d, AT_BOX)) return -2;
+  size_t smem = 1024 + 8 * (size_t)(2 * AT_BOX_BYTES) + 64;
+  static bool attr = false;
+  if (!attr) {
+    if (cudaFuncSetAttribute(attn_bwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -3;
+    attr = true;
+  }
+  note_launch(1);
+  attn_bwd_tc_kernel<<<B * H, 128, smem, c.stream>>>(mq, mg, lse, cls_extra, (bf16*)dqkv, B, T, H, c.status);
   return 0;
 }
 

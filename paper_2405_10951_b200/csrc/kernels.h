@@ -94,6 +94,8 @@ int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const voi
 // scaled scores; cls_prob (optional) [B, H, T-1].
 // tcgen05 kernels (bf16, head dimension 64); return non-zero when they do not take the problem.
 int attention_fwd_tc(const Ctx& c, const void* qkv, void* out, float* lse, float* cls_prob, int B, int T, int H, int d);
+int attention_bwd_tc(const Ctx& c, const void* qkv, const void* dout, const float* lse, const float* cls_extra, void* dqkv,
+                     int B, int T, int H, int d);
 int attention_fwd(const Ctx& c, const void* qkv, void* out, float* lse, float* cls_prob, int B, int T, int H, int d);
 // dqkv from dout; delta scratch [B, H, T]; cls_extra (optional) [B, T-1]: gradient arriving at the head-mean
 // score of each non-classification token (zero for kept tokens); cls_prob needed with it.
