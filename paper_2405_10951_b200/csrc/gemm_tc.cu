@@ -11,8 +11,9 @@
 // Kernel shape: persistent, one CTA per SM, 128 x 256 output tiles, k in slabs of 64.
 //   warp 0      : TMA producer (one lane)
 //   warp 1      : tensor-memory allocation, MMA issue (one lane)
-//   warps 2..5  : epilogue, one TMEM lane quarter each; two accumulator buffers of 256 columns let
-//                 the epilogue of one tile overlap the main loop of the next.
+//   warps 2..9  : epilogue, two warps per TMEM lane quarter; chunks of 32 x 32 outputs go through a staging
+//                 buffer so that global loads and stores are row-contiguous; two accumulator buffers of 256
+//                 columns let the epilogue of one tile overlap the main loop of the next.
 // Every wait is bounded: on expiry the CTA raises STATUS_TIMEOUT in the status word, gives the
 // copies it issued time to land, frees its tensor memory and returns.
 #include <cuda.h>
@@ -30,8 +31,10 @@ constexpr int STAGES = 4;
 constexpr int UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr int THREADS = 192;
+constexpr int EPI_WARPS = 8;                     // two warps per TMEM lane quarter, each takes half of the columns
+constexpr int STAGING_BYTES = 32 * 128;          // per epilogue warp: 32 rows x 128 bytes, 16-byte units XOR-swizzled
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * STAGING_BYTES + 1024 /*alignment slack*/ + 128 /*barriers*/;
+constexpr int THREADS = 64 + EPI_WARPS * 32;
 constexpr uint32_t TMEM_COLS = 512;
 
 struct Epi {
@@ -48,12 +51,87 @@ __host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn) {
          ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
 
-template <typename TOut> __device__ __forceinline__ void store8(TOut* p, const float* v);
-template <> __device__ __forceinline__ void store8<bf16>(bf16* p, const float* v) { store16(p, v); }
-template <> __device__ __forceinline__ void store8<float>(float* p, const float* v) { store16(p, v); store16(p + 4, v + 4); }
-template <typename TOut> __device__ __forceinline__ void load8(const TOut* p, float* v);
-template <> __device__ __forceinline__ void load8<bf16>(const bf16* p, float* v) { load16(p, v); }
-template <> __device__ __forceinline__ void load8<float>(const float* p, float* v) { load16(p, v); load16(p + 4, v + 4); }
+// erf by the rational approximation 7.1.26 of Abramowitz and Stegun (|error| < 1.5e-7, about 1e-6 with the fast
+// reciprocal and exponential used here): far below the bf16 resolution of the values this epilogue produces.
+// Also returns e = exp(-x^2), which the derivative of GELU needs.
+__device__ __forceinline__ float erf_fast(float x, float& e) {
+  float ax = fabsf(x);
+  float t = __fdividef(1.0f, fmaf(0.3275911f, ax, 1.0f));
+  e = __expf(-ax * ax);
+  float poly = t * (0.254829592f + t * (-0.284496736f + t * (1.421413741f + t * (-1.453152027f + t * 1.061405429f))));
+  return copysignf(1.0f - poly * e, x);
+}
+__device__ __forceinline__ float gelu_fast(float z) {
+  float e;
+  return 0.5f * z * (1.0f + erf_fast(z * 0.70710678118654752f, e));
+}
+__device__ __forceinline__ float gelu_grad_fast(float z) {
+  float e;
+  float er = erf_fast(z * 0.70710678118654752f, e);
+  return 0.5f * (1.0f + er) + z * 0.39894228040143268f * e;
+}
+
+// A warp moves a 32-row x 32-column chunk between registers (lane = row, v[32] = the row's columns) and global
+// memory through its staging buffer, so that the global accesses are row-contiguous: each instruction touches a
+// few full rows instead of one 16-byte piece of 32 different rows.
+template <typename T>
+struct ChunkIO {
+  static constexpr int E = 16 / sizeof(T);          // elements per 16-byte unit
+  static constexpr int UNITS = 32 / E;               // units per chunk row: 4 (bf16) or 8 (float)
+  static constexpr int ROWS_PER_PASS = 32 / UNITS;
+  __device__ static uint32_t slot(int r, int u) { return (uint32_t)(r * 128 + ((u ^ (r & 7)) << 4)); }
+
+  __device__ static void load(const T* g, int ld, int row0, int col0, int M, int N, unsigned char* st, int lane, float* v) {
+#pragma unroll
+    for (int i = 0; i < UNITS; ++i) {
+      int r = i * ROWS_PER_PASS + lane / UNITS, u = lane % UNITS;
+      int col = col0 + u * E;
+      uint4 x = make_uint4(0, 0, 0, 0);
+      if (row0 + r < M && col < N) x = *reinterpret_cast<const uint4*>(g + (size_t)(row0 + r) * ld + col);
+      *reinterpret_cast<uint4*>(st + slot(r, u)) = x;
+    }
+    __syncwarp();
+#pragma unroll
+    for (int u = 0; u < UNITS; ++u) {
+      uint4 x = *reinterpret_cast<const uint4*>(st + slot(lane, u));
+      unpack(x, v + u * E);
+    }
+    __syncwarp();
+  }
+  __device__ static void store(T* g, int ld, int row0, int col0, int M, int N, unsigned char* st, int lane, const float* v) {
+#pragma unroll
+    for (int u = 0; u < UNITS; ++u) *reinterpret_cast<uint4*>(st + slot(lane, u)) = pack(v + u * E);
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < UNITS; ++i) {
+      int r = i * ROWS_PER_PASS + lane / UNITS, u = lane % UNITS;
+      int col = col0 + u * E;
+      if (row0 + r < M && col < N)
+        *reinterpret_cast<uint4*>(g + (size_t)(row0 + r) * ld + col) = *reinterpret_cast<const uint4*>(st + slot(r, u));
+    }
+    __syncwarp();
+  }
+  __device__ static void unpack(const uint4& x, float* f);
+  __device__ static uint4 pack(const float* f);
+};
+template <> __device__ __forceinline__ void ChunkIO<float>::unpack(const uint4& x, float* f) {
+  f[0] = __uint_as_float(x.x); f[1] = __uint_as_float(x.y); f[2] = __uint_as_float(x.z); f[3] = __uint_as_float(x.w);
+}
+template <> __device__ __forceinline__ uint4 ChunkIO<float>::pack(const float* f) {
+  return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+}
+template <> __device__ __forceinline__ void ChunkIO<bf16>::unpack(const uint4& x, float* f) {
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&x);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { float2 t = __bfloat1622float2(h[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
+}
+template <> __device__ __forceinline__ uint4 ChunkIO<bf16>::pack(const float* f) {
+  uint4 x;
+  __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&x);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+  return x;
+}
 
 template <bool A_MN, bool B_MN, typename TOut>
 __global__ void __launch_bounds__(THREADS, 1)
@@ -61,7 +139,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                int M, int N, int K, Epi ep, int tiles_m, int tiles_n, int splits, int kb_per_split, int* status) {
   extern __shared__ unsigned char smem_dyn[];
   uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
-  uint32_t bars = base + STAGES * STAGE_BYTES;           // full[STAGES], empty[STAGES], tfull[2], tempty[2]
+  uint32_t staging0 = base + STAGES * STAGE_BYTES;
+  uint32_t bars = staging0 + EPI_WARPS * STAGING_BYTES;   // full[STAGES], empty[STAGES], tfull[2], tempty[2]
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
   auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
@@ -75,7 +154,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), EPI_WARPS); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -157,54 +236,59 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   } else {
     // ------------------------------- epilogue -----------------------------------
-    int quarter = warp & 3;                 // TMEM lanes 32*quarter .. 32*quarter+31
+    int ew = warp - 2;                      // 0..7
+    int quarter = warp & 3;                 // TMEM lanes 32*quarter .. 32*quarter+31 (fixed by the warp's rank)
+    int chalf = ew >> 2;                    // which 128 of the tile's 256 columns
+    unsigned char* st = smem_dyn + (staging0 - smem_u32(smem_dyn)) + ew * STAGING_BYTES;
     int local = 0;
     bool ok = true;
     for (int w = blockIdx.x; w < work_items && ok; w += gridDim.x, ++local) {
       int mt = w % tiles_m, nt = (w / tiles_m) % tiles_n, sp = w / (tiles_m * tiles_n);
       int buf = local & 1;
-      if (!mbar_wait(tfull_bar(buf), (local >> 1) & 1, abortp)) { ok = false; break; }
+      ok = mbar_wait(tfull_bar(buf), (local >> 1) & 1, abortp);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
       tc_fence_after();
-      int row = mt * BM + quarter * 32 + lane;
-      TOut* crow = C + (size_t)sp * M * N + (size_t)row * N;
+      int row0 = mt * BM + quarter * 32;
+      TOut* Cs = C + (size_t)sp * M * N;
 #pragma unroll 1
-      for (int cchunk = 0; cchunk < BN / 32; ++cchunk) {
+      for (int cc = 0; cc < 4; ++cc) {
+        int cchunk = chalf * 4 + cc;
         uint32_t r[32];
         uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cchunk * 32);
         tmem_ld32(taddr, r);
         tmem_ld_wait();
         int col0 = nt * BN + cchunk * 32;
-        if (row < M && col0 < N) {
+        if (row0 < M && col0 < N) {           // warp-uniform
+          float v[32];
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            int col = col0 + g * 8;
-            if (col < N) {
-              float v[8];
+          for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+          if (ep.bias != nullptr) {
 #pragma unroll
-              for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[g * 8 + j]);
-              if (ep.bias != nullptr) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] += __ldg(ep.bias + col + j);
+            for (int g = 0; g < 8; ++g) {
+              if (col0 + g * 4 < N) {
+                float4 bb = __ldg(reinterpret_cast<const float4*>(ep.bias + col0 + g * 4));
+                v[g * 4 + 0] += bb.x; v[g * 4 + 1] += bb.y; v[g * 4 + 2] += bb.z; v[g * 4 + 3] += bb.w;
               }
-              if (ep.act == 1) {
-                if (ep.aux_out != nullptr) store8<TOut>((TOut*)ep.aux_out + (size_t)row * N + col, v);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = gelu_f(v[j]);
-              } else if (ep.act == 2) {
-                float z[8];
-                load16((const bf16*)ep.aux_in + (size_t)row * N + col, z);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] *= gelu_grad_f(z[j]);
-              }
-              if (ep.residual != nullptr) {
-                float rr[8];
-                load8<TOut>((const TOut*)ep.residual + (size_t)row * N + col, rr);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] += rr[j];
-              }
-              store8<TOut>(crow + col, v);
             }
           }
+          if (ep.act == 1) {
+            if (ep.aux_out != nullptr) ChunkIO<TOut>::store((TOut*)ep.aux_out, N, row0, col0, M, N, st, lane, v);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = gelu_fast(v[j]);
+          } else if (ep.act == 2) {
+            float z[32];
+            ChunkIO<bf16>::load((const bf16*)ep.aux_in, N, row0, col0, M, N, st, lane, z);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] *= gelu_grad_fast(z[j]);
+          }
+          if (ep.residual != nullptr) {
+            float rr[32];
+            ChunkIO<TOut>::load((const TOut*)ep.residual, N, row0, col0, M, N, st, lane, rr);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] += rr[j];
+          }
+          ChunkIO<TOut>::store(Cs, N, row0, col0, M, N, st, lane, v);
         }
       }
       tc_fence_before();
