@@ -25,11 +25,37 @@ __global__ void patchify_kernel(const T* __restrict__ img, T* __restrict__ out, 
   out[i] = img[(((long)b * C + ch) * S + (gy * P + py)) * S + gx * P + px];
 }
 
+// Same copy in 16-byte units (P * sizeof(T) a multiple of 16): a patch row is P/E units.
+template <typename T>
+__global__ void patchify_vec_kernel(const T* __restrict__ img, T* __restrict__ out, int B, int C, int S, int P, long units) {
+  constexpr int E = 16 / sizeof(T);
+  long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= units) return;
+  int g = S / P, upr = P / E;
+  int ux = (int)(i % upr); long r = i / upr;
+  int py = (int)(r % P); r /= P;
+  int ch = (int)(r % C); r /= C;
+  int gx = (int)(r % g); r /= g;
+  int gy = (int)(r % g); r /= g;
+  int b = (int)r;
+  const T* src = img + (((long)b * C + ch) * S + (gy * P + py)) * S + gx * P + ux * E;
+  *reinterpret_cast<uint4*>(out + i * E) = *reinterpret_cast<const uint4*>(src);
+}
+
 void patchify(const Ctx& c, const void* images, void* patches, int B, int C, int S, int P) {
   note_launch(1);
   int g = S / P;
   long total = (long)B * g * g * C * P * P;
   int threads = 256;
+  size_t es = dtype_size(c.dtype);
+  bool vec = (P * es) % 16 == 0 && (((uintptr_t)images | (uintptr_t)patches) & 15) == 0;
+  if (vec) {
+    long units = total * (long)es / 16;
+    int blocks = ceil_div(units, threads);
+    if (c.dtype == 0) patchify_vec_kernel<float><<<blocks, threads, 0, c.stream>>>((const float*)images, (float*)patches, B, C, S, P, units);
+    else patchify_vec_kernel<bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)images, (bf16*)patches, B, C, S, P, units);
+    return;
+  }
   int blocks = ceil_div(total, threads);
   if (c.dtype == 0)
     patchify_kernel<float><<<blocks, threads, 0, c.stream>>>((const float*)images, (float*)patches, B, C, S, P, total);
@@ -37,27 +63,34 @@ void patchify(const Ctx& c, const void* images, void* patches, int B, int C, int
     patchify_kernel<bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)images, (bf16*)patches, B, C, S, P, total);
 }
 
-// x[b, 0] = cls + pos[0];  x[b, 1 + n] = emb[b, n] + pos[1 + n]   (classification token and positional embedding)
+// x[b, 0] = cls + pos[0];  x[b, 1 + n] = emb[b, n] + pos[1 + n]   (classification token and positional embedding);
+// four columns per thread (D % 4 == 0).
 template <typename T>
 __global__ void assemble_kernel(const T* __restrict__ emb, const float* __restrict__ cls, const float* __restrict__ pos,
-                                float* __restrict__ x, int B, int N, int D, long total) {
+                                float* __restrict__ x, int B, int N, int D, long total4) {
   long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= total) return;
-  int d = (int)(i % D); long r = i / D;
+  if (i >= total4) return;
+  int d4 = D / 4;
+  int d = (int)(i % d4) * 4; long r = i / d4;
   int t = (int)(r % (N + 1));
   int b = (int)(r / (N + 1));
-  float v = (t == 0) ? cls[d] : to_f(emb[((long)b * N + (t - 1)) * D + d]);
-  x[i] = v + pos[(long)t * D + d];
+  float v[4], p[4];
+  if (t == 0) load16(cls + d, v);
+  else load4(emb + ((long)b * N + (t - 1)) * D + d, v);
+  load16(pos + (long)t * D + d, p);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) v[j] += p[j];
+  store16(x + i * 4, v);
 }
 
 void assemble_tokens(const Ctx& c, const void* emb, const float* cls, const float* pos, float* x, int B, int N, int D) {
   note_launch(1);
-  long total = (long)B * (N + 1) * D;
-  int threads = 256, blocks = ceil_div(total, threads);
+  long total4 = (long)B * (N + 1) * D / 4;
+  int threads = 256, blocks = ceil_div(total4, threads);
   if (c.dtype == 0)
-    assemble_kernel<float><<<blocks, threads, 0, c.stream>>>((const float*)emb, cls, pos, x, B, N, D, total);
+    assemble_kernel<float><<<blocks, threads, 0, c.stream>>>((const float*)emb, cls, pos, x, B, N, D, total4);
   else
-    assemble_kernel<bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)emb, cls, pos, x, B, N, D, total);
+    assemble_kernel<bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)emb, cls, pos, x, B, N, D, total4);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -65,10 +98,9 @@ void assemble_tokens(const Ctx& c, const void* emb, const float* cls, const floa
 // would survive bf16 rounding of the stream poorly); the normalised output feeds a GEMM and takes
 // the storage dtype.  One warp per row, the row held in registers (D <= 1024, D % 4 == 0).
 // ------------------------------------------------------------------------------------------------
-constexpr int LN_MAX_PER_LANE = 32;   // floats per lane: D <= 1024
-constexpr int LN_MAXC = LN_MAX_PER_LANE / 4;
+// NCH = 16-byte chunks of the row each lane holds (D <= 128 * NCH); instantiated for 2, 3, 4, 6 and 8.
 
-template <typename TY>
+template <typename TY, int NCH>
 __global__ void layernorm_fwd_kernel(const float* __restrict__ x, long x_stride, const float* __restrict__ g,
                                      const float* __restrict__ b, TY* __restrict__ y, float* __restrict__ mean,
                                      float* __restrict__ rstd, int rows, int D, float eps) {
@@ -77,10 +109,10 @@ __global__ void layernorm_fwd_kernel(const float* __restrict__ x, long x_stride,
   if (warp >= rows) return;
   const float* xr = x + (long)warp * x_stride;
   int chunks = D / 4;
-  float v[LN_MAX_PER_LANE];
+  float v[(NCH * 4)];
   float sum = 0.f;
 #pragma unroll
-  for (int i = 0; i < LN_MAXC; ++i) {
+  for (int i = 0; i < NCH; ++i) {
     int ch = lane + i * 32;
     if (ch < chunks) {
       load16(xr + ch * 4, v + i * 4);
@@ -91,7 +123,7 @@ __global__ void layernorm_fwd_kernel(const float* __restrict__ x, long x_stride,
   float mu = warp_sum(sum) / (float)D;
   float sq = 0.f;
 #pragma unroll
-  for (int i = 0; i < LN_MAXC; ++i) {
+  for (int i = 0; i < NCH; ++i) {
     int ch = lane + i * 32;
     if (ch < chunks) {
 #pragma unroll
@@ -105,7 +137,7 @@ __global__ void layernorm_fwd_kernel(const float* __restrict__ x, long x_stride,
   }
   TY* yr = y + (long)warp * D;
 #pragma unroll
-  for (int i = 0; i < LN_MAXC; ++i) {
+  for (int i = 0; i < NCH; ++i) {
     int ch = lane + i * 32;
     if (ch < chunks) {
       float4 gg = *reinterpret_cast<const float4*>(g + ch * 4), bb = *reinterpret_cast<const float4*>(b + ch * 4);
@@ -119,15 +151,22 @@ __global__ void layernorm_fwd_kernel(const float* __restrict__ x, long x_stride,
   }
 }
 
+template <typename TY>
+static void launch_ln_fwd(const Ctx& c, const float* x, long x_stride, const float* g, const float* b, TY* y, float* mean,
+                          float* rstd, int rows, int D, float eps) {
+  int threads = 256;
+  int blocks = ceil_div((long)rows * 32, threads);
+  int nch = ceil_div(D, 128);
+#define BSR_LN_FWD(N) layernorm_fwd_kernel<TY, N><<<blocks, threads, 0, c.stream>>>(x, x_stride, g, b, y, mean, rstd, rows, D, eps)
+  if (nch <= 2) BSR_LN_FWD(2); else if (nch == 3) BSR_LN_FWD(3); else if (nch == 4) BSR_LN_FWD(4); else if (nch <= 6) BSR_LN_FWD(6); else BSR_LN_FWD(8);
+#undef BSR_LN_FWD
+}
+
 void layernorm_fwd(const Ctx& c, const float* x, long x_stride, const float* g, const float* b, void* y, int y_is_float,
                    float* mean, float* rstd, int rows, int D, float eps) {
   note_launch(1);
-  int threads = 256;
-  int blocks = ceil_div((long)rows * 32, threads);
-  if (c.dtype == 0 || y_is_float)
-    layernorm_fwd_kernel<float><<<blocks, threads, 0, c.stream>>>(x, x_stride, g, b, (float*)y, mean, rstd, rows, D, eps);
-  else
-    layernorm_fwd_kernel<bf16><<<blocks, threads, 0, c.stream>>>(x, x_stride, g, b, (bf16*)y, mean, rstd, rows, D, eps);
+  if (c.dtype == 0 || y_is_float) launch_ln_fwd<float>(c, x, x_stride, g, b, (float*)y, mean, rstd, rows, D, eps);
+  else launch_ln_fwd<bf16>(c, x, x_stride, g, b, (bf16*)y, mean, rstd, rows, D, eps);
 }
 
 // Backward.  Each block owns rows blockIdx.x*8 + warp, stepping by gridDim.x*8; every lane accumulates the
@@ -137,25 +176,25 @@ void layernorm_fwd(const Ctx& c, const float* x, long x_stride, const float* g, 
 // storage dtype for the GEMMs that consume them.
 constexpr int LNB_WARPS = 8;
 
-template <typename TDY, typename TC>
-__global__ void layernorm_bwd_kernel(const TDY* __restrict__ dy, const float* __restrict__ x, long x_stride,
+template <typename TDY, typename TC, int NCH>
+__global__ void __launch_bounds__(256, 2) layernorm_bwd_kernel(const TDY* __restrict__ dy, const float* __restrict__ x, long x_stride,
                                      const float* __restrict__ mean, const float* __restrict__ rstd,
                                      const float* __restrict__ g, const float* __restrict__ dres, float* __restrict__ dx,
                                      long dx_stride, TC* __restrict__ dx_copy, float* __restrict__ partials, int rows, int D) {
   extern __shared__ float sm[];   // [LNB_WARPS][2][D]
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int chunks = D / 4;
-  float ag[LN_MAX_PER_LANE], ab[LN_MAX_PER_LANE];
+  float ag[(NCH * 4)], ab[(NCH * 4)];
 #pragma unroll
-  for (int i = 0; i < LN_MAX_PER_LANE; ++i) { ag[i] = 0.f; ab[i] = 0.f; }
+  for (int i = 0; i < (NCH * 4); ++i) { ag[i] = 0.f; ab[i] = 0.f; }
   for (int r = blockIdx.x * LNB_WARPS + warp; r < rows; r += gridDim.x * LNB_WARPS) {
     const float* xr = x + (long)r * x_stride;
     const TDY* dyr = dy + (long)r * D;
     float mu = mean[r], rs = rstd[r];
-    float xh[LN_MAX_PER_LANE], dh[LN_MAX_PER_LANE];
+    float xh[(NCH * 4)], dh[(NCH * 4)];
     float s1 = 0.f, s2 = 0.f;
 #pragma unroll
-    for (int i = 0; i < LN_MAXC; ++i) {
+    for (int i = 0; i < NCH; ++i) {
       int ch = lane + i * 32;
       if (ch < chunks) {
         float xv[4], dv[4];
@@ -182,7 +221,7 @@ __global__ void layernorm_bwd_kernel(const TDY* __restrict__ dy, const float* __
     if (dx != nullptr) {
       float* dxr = dx + (long)r * dx_stride;
 #pragma unroll
-      for (int i = 0; i < LN_MAXC; ++i) {
+      for (int i = 0; i < NCH; ++i) {
         int ch = lane + i * 32;
         if (ch < chunks) {
           float o[4];
@@ -201,7 +240,7 @@ __global__ void layernorm_bwd_kernel(const TDY* __restrict__ dy, const float* __
   }
   float* mine = sm + (size_t)warp * 2 * D;
 #pragma unroll
-  for (int i = 0; i < LN_MAXC; ++i) {
+  for (int i = 0; i < NCH; ++i) {
     int ch = lane + i * 32;
     if (ch < chunks) {
 #pragma unroll
@@ -221,13 +260,25 @@ __global__ void layernorm_bwd_kernel(const TDY* __restrict__ dy, const float* __
   }
 }
 
-// out[col] = sum over groups of partials[group][col], groups in ascending order.
-__global__ void reduce_partials_kernel(const float* __restrict__ partials, int groups, int cols, float* __restrict__ out) {
-  int col = blockIdx.x * blockDim.x + threadIdx.x;
-  if (col >= cols) return;
+// out_y[col] = sum over groups of partials[y][group][col] for y = blockIdx.y (one or two outputs per launch).
+// 16 lanes stride the groups and are combined through shared memory in lane order: the result is deterministic.
+__global__ void reduce_partials_kernel(const float* __restrict__ partials, int groups, int cols, float* __restrict__ out0,
+                                       float* __restrict__ out1) {
+  __shared__ float sm[16][17];
+  int cx = threadIdx.x & 15, gy = threadIdx.x >> 4;
+  int col = blockIdx.x * 16 + cx;
+  const float* p = partials + (size_t)blockIdx.y * groups * cols;
   float s = 0.f;
-  for (int gidx = 0; gidx < groups; ++gidx) s += partials[(size_t)gidx * cols + col];
-  out[col] = s;
+  if (col < cols)
+    for (int g = gy; g < groups; g += 16) s += p[(size_t)g * cols + col];
+  sm[gy][cx] = s;
+  __syncthreads();
+  if (gy == 0 && col < cols) {
+    float t = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) t += sm[i][cx];
+    (blockIdx.y ? out1 : out0)[col] = t;
+  }
 }
 
 int layernorm_bwd_groups(const Ctx& c, int rows) {
@@ -240,15 +291,21 @@ template <typename TDY, typename TC>
 static void launch_ln_bwd(const Ctx& c, int groups, size_t smem, const void* dy, const float* x, long x_stride, const float* mean,
                           const float* rstd, const float* g, const float* dres, float* dx, long dx_stride, void* dx_copy,
                           float* partials, int rows, int D) {
-  cudaFuncSetAttribute(layernorm_bwd_kernel<TDY, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  layernorm_bwd_kernel<TDY, TC><<<groups, LNB_WARPS * 32, smem, c.stream>>>((const TDY*)dy, x, x_stride, mean, rstd, g, dres, dx,
-                                                                           dx_stride, (TC*)dx_copy, partials, rows, D);
+  int nch = ceil_div(D, 128);
+#define BSR_LN_BWD(N)                                                                                                   \
+  do {                                                                                                                  \
+    cudaFuncSetAttribute(layernorm_bwd_kernel<TDY, TC, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);       \
+    layernorm_bwd_kernel<TDY, TC, N><<<groups, LNB_WARPS * 32, smem, c.stream>>>((const TDY*)dy, x, x_stride, mean, rstd, g, dres, \
+                                                                                 dx, dx_stride, (TC*)dx_copy, partials, rows, D); \
+  } while (0)
+  if (nch <= 2) BSR_LN_BWD(2); else if (nch == 3) BSR_LN_BWD(3); else if (nch == 4) BSR_LN_BWD(4); else if (nch <= 6) BSR_LN_BWD(6); else BSR_LN_BWD(8);
+#undef BSR_LN_BWD
 }
 
 void layernorm_bwd(const Ctx& c, const void* dy, int dy_is_float, const float* x, long x_stride, const float* mean,
                    const float* rstd, const float* g, const float* dres, float* dx, long dx_stride, void* dx_copy,
                    float* partials, float* dgamma, float* dbeta, int rows, int D) {
-  note_launch(3);
+  note_launch(2);
   int groups = layernorm_bwd_groups(c, rows);
   size_t smem = (size_t)LNB_WARPS * 2 * D * sizeof(float);
   if (c.dtype == 0)
@@ -257,9 +314,8 @@ void layernorm_bwd(const Ctx& c, const void* dy, int dy_is_float, const float* x
     launch_ln_bwd<float, bf16>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, dx_copy, partials, rows, D);
   else
     launch_ln_bwd<bf16, bf16>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, dx_copy, partials, rows, D);
-  int t2 = 256;
-  reduce_partials_kernel<<<ceil_div(D, t2), t2, 0, c.stream>>>(partials, groups, D, dgamma);
-  reduce_partials_kernel<<<ceil_div(D, t2), t2, 0, c.stream>>>(partials + (size_t)groups * D, groups, D, dbeta);
+  dim3 grid(ceil_div(D, 16), 2);
+  reduce_partials_kernel<<<grid, 256, 0, c.stream>>>(partials, groups, D, dgamma, dbeta);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -315,7 +371,7 @@ void colsum(const Ctx& c, const void* x, int rows, int cols, float* partials, fl
     dim3 grid(ceil_div(cols, 32 * 8), groups);
     colsum_kernel<bf16><<<grid, threads, 0, c.stream>>>((const bf16*)x, rows, cols, partials);
   }
-  reduce_partials_kernel<<<ceil_div(cols, 256), 256, 0, c.stream>>>(partials, groups, cols, out);
+  reduce_partials_kernel<<<dim3(ceil_div(cols, 16), 1), 256, 0, c.stream>>>(partials, groups, cols, out, out);
 }
 
 // ------------------------------------------------------------------------------------------------
