@@ -911,7 +911,7 @@ int32_t bsr_linear_forward(const void* x, const void* w, const float* bias, cons
   e.act = act_gelu ? 1 : 0;
   if (use_tensor_cores) {
     if (dtype != BSR_DTYPE_BF16 || !gemm_tc_supported(m, n, k)) return set_err(g_error, BSR_ERR_UNSUPPORTED, "the tcgen05 kernel needs bf16 and k, n multiples of 8");
-    int rc = gemm_tc(c, x, w, y, 0, m, n, k, e);
+    int rc = use_tensor_cores >= 2 ? gemm_tc2_strided(c, x, k, 1, w, k, 1, y, 0, m, n, k, e, nullptr, 0) : gemm_tc(c, x, w, y, 0, m, n, k, e);
     if (rc != 0) return set_err(g_error, BSR_ERR_CUDA, "tcgen05 GEMM set-up failed (%d)", rc);
   } else {
     gemm(c, x, k, 1, w, k, 1, y, 0, m, n, k, e);
@@ -928,8 +928,14 @@ int32_t bsr_linear_backward(const void* x, const void* w, const void* dy, void* 
   GemmEpilogue none;
   if (use_tensor_cores) {
     if (dtype != BSR_DTYPE_BF16 || (m % 8) || (n % 8) || (k % 8)) return set_err(g_error, BSR_ERR_UNSUPPORTED, "the tcgen05 kernels need bf16 and m, n, k multiples of 8");
-    int rc = gemm_tc_strided(c, dy, n, 1, w, 1, k, dx, 0, m, k, n, none, nullptr, 0);                       // dX = dY W
-    if (rc == 0) rc = gemm_tc_strided(c, dy, 1, n, x, 1, k, dw, 1, n, k, m, none, workspace, workspace_floats);   // dW = dY^T X
+    int rc;
+    if (use_tensor_cores >= 2) {
+      rc = gemm_tc2_strided(c, dy, n, 1, w, 1, k, dx, 0, m, k, n, none, nullptr, 0);
+      if (rc == 0) rc = gemm_tc2_strided(c, dy, 1, n, x, 1, k, dw, 1, n, k, m, none, workspace, workspace_floats);
+    } else {
+      rc = gemm_tc_strided(c, dy, n, 1, w, 1, k, dx, 0, m, k, n, none, nullptr, 0);                       // dX = dY W
+      if (rc == 0) rc = gemm_tc_strided(c, dy, 1, n, x, 1, k, dw, 1, n, k, m, none, workspace, workspace_floats);   // dW = dY^T X
+    }
     if (rc != 0) return set_err(g_error, BSR_ERR_CUDA, "tcgen05 GEMM set-up failed (%d)", rc);
   } else {
     gemm(c, dy, n, 1, w, 1, k, dx, 0, m, k, n, none);

@@ -79,6 +79,8 @@ void gemm(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long
           int out_is_float, int m, int n, int k, const GemmEpilogue& e) {
   if (m <= 0 || n <= 0) return;
   if (c.dtype == 1 && c.use_tc && gemm_tc_supported(m, n, k)) {
+    if (c.use_tc >= 2 && m > 128 &&
+        gemm_tc2_strided(c, A, a_rs, a_cs, B, b_rs, b_cs, C, out_is_float, m, n, k, e, c.split_ws, c.split_ws_floats) == 0) return;
     if (gemm_tc_strided(c, A, a_rs, a_cs, B, b_rs, b_cs, C, out_is_float, m, n, k, e, c.split_ws, c.split_ws_floats) == 0) return;
   }
   dim3 grid(ceil_div(n, SG_BN), ceil_div(m, SG_BM));

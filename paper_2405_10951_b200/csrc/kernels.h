@@ -89,6 +89,11 @@ int gemm_tc(const Ctx& c, const void* A, const void* B, void* C, int out_is_floa
 int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long b_rs, long b_cs, void* C,
                     int out_is_float, int m, int n, int k, const GemmEpilogue& e, float* split_ws, size_t split_ws_floats);
 
+// The same on CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles); preferred when m > 128.
+int gemm_tc2_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long b_rs, long b_cs, void* C,
+                     int out_is_float, int m, int n, int k, const GemmEpilogue& e, float* split_ws, size_t split_ws_floats);
+void splitk_reduce(cudaStream_t s, const float* partial, float* out, size_t n, int splits);
+
 // ---- attention --------------------------------------------------------------------------------
 // qkv [B, T, 3, H, d]; out [B, T, H*d]; lse (optional) [B, H, T] natural-log sum of exponentials of the
 // scaled scores; cls_prob (optional) [B, H, T-1].

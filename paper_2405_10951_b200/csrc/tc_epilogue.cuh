@@ -1,0 +1,139 @@
+// Epilogue of the tcgen05 GEMM kernels: a warp turns 32 rows x 32 columns of fp32 accumulators (lane = row) into
+// outputs with bias, GELU, GELU-derivative and residual options, moving data to and from global memory through a
+// swizzled staging buffer so that every global access is row-contiguous.
+#pragma once
+
+#include "common.cuh"
+
+namespace bsr {
+namespace tc {
+
+struct Epi {
+  const float* bias;
+  const void* residual;
+  void* aux_out;
+  const void* aux_in;
+  int act;
+};
+
+// erf by the rational approximation 7.1.26 of Abramowitz and Stegun (|error| < 1.5e-7, about 1e-6 with the fast
+// reciprocal and exponential used here): far below the bf16 resolution of the values this epilogue produces.
+// Also returns e = exp(-x^2), which the derivative of GELU needs.
+__device__ __forceinline__ float erf_fast(float x, float& e) {
+  float ax = fabsf(x);
+  float t = __fdividef(1.0f, fmaf(0.3275911f, ax, 1.0f));
+  e = __expf(-ax * ax);
+  float poly = t * (0.254829592f + t * (-0.284496736f + t * (1.421413741f + t * (-1.453152027f + t * 1.061405429f))));
+  return copysignf(1.0f - poly * e, x);
+}
+__device__ __forceinline__ float gelu_fast(float z) {
+  float e;
+  return 0.5f * z * (1.0f + erf_fast(z * 0.70710678118654752f, e));
+}
+__device__ __forceinline__ float gelu_grad_fast(float z) {
+  float e;
+  float er = erf_fast(z * 0.70710678118654752f, e);
+  return 0.5f * (1.0f + er) + z * 0.39894228040143268f * e;
+}
+
+// A warp moves a 32-row x 32-column chunk between registers (lane = row, v[32] = the row's columns) and global
+// memory through its staging buffer, so that the global accesses are row-contiguous: each instruction touches a
+// few full rows instead of one 16-byte piece of 32 different rows.
+template <typename T>
+struct ChunkIO {
+  static constexpr int E = 16 / sizeof(T);          // elements per 16-byte unit
+  static constexpr int UNITS = 32 / E;               // units per chunk row: 4 (bf16) or 8 (float)
+  static constexpr int ROWS_PER_PASS = 32 / UNITS;
+  __device__ static uint32_t slot(int r, int u) { return (uint32_t)(r * 128 + ((u ^ (r & 7)) << 4)); }
+
+  __device__ static void load(const T* g, int ld, int row0, int col0, int M, int N, unsigned char* st, int lane, float* v) {
+#pragma unroll
+    for (int i = 0; i < UNITS; ++i) {
+      int r = i * ROWS_PER_PASS + lane / UNITS, u = lane % UNITS;
+      int col = col0 + u * E;
+      uint4 x = make_uint4(0, 0, 0, 0);
+      if (row0 + r < M && col < N) x = *reinterpret_cast<const uint4*>(g + (size_t)(row0 + r) * ld + col);
+      *reinterpret_cast<uint4*>(st + slot(r, u)) = x;
+    }
+    __syncwarp();
+#pragma unroll
+    for (int u = 0; u < UNITS; ++u) {
+      uint4 x = *reinterpret_cast<const uint4*>(st + slot(lane, u));
+      unpack(x, v + u * E);
+    }
+    __syncwarp();
+  }
+  __device__ static void store(T* g, int ld, int row0, int col0, int M, int N, unsigned char* st, int lane, const float* v) {
+#pragma unroll
+    for (int u = 0; u < UNITS; ++u) *reinterpret_cast<uint4*>(st + slot(lane, u)) = pack(v + u * E);
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < UNITS; ++i) {
+      int r = i * ROWS_PER_PASS + lane / UNITS, u = lane % UNITS;
+      int col = col0 + u * E;
+      if (row0 + r < M && col < N)
+        *reinterpret_cast<uint4*>(g + (size_t)(row0 + r) * ld + col) = *reinterpret_cast<const uint4*>(st + slot(r, u));
+    }
+    __syncwarp();
+  }
+  __device__ static void unpack(const uint4& x, float* f);
+  __device__ static uint4 pack(const float* f);
+};
+template <> __device__ __forceinline__ void ChunkIO<float>::unpack(const uint4& x, float* f) {
+  f[0] = __uint_as_float(x.x); f[1] = __uint_as_float(x.y); f[2] = __uint_as_float(x.z); f[3] = __uint_as_float(x.w);
+}
+template <> __device__ __forceinline__ uint4 ChunkIO<float>::pack(const float* f) {
+  return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+}
+template <> __device__ __forceinline__ void ChunkIO<bf16>::unpack(const uint4& x, float* f) {
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&x);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { float2 t = __bfloat1622float2(h[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
+}
+template <> __device__ __forceinline__ uint4 ChunkIO<bf16>::pack(const float* f) {
+  uint4 x;
+  __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&x);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+  return x;
+}
+
+// v[j]: accumulator of (row0 + lane, col0 + j).  All lanes of the warp take part (row0, col0 are warp-uniform).
+template <typename TOut>
+__device__ __forceinline__ void epilogue_chunk(const uint32_t* r, const Epi& ep, TOut* Cs, int M, int N, int row0, int col0,
+                                               unsigned char* st, int lane) {
+  if (row0 < M && col0 < N) {
+    float v[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+    if (ep.bias != nullptr) {
+#pragma unroll
+      for (int g = 0; g < 8; ++g) {
+        if (col0 + g * 4 < N) {
+          float4 bb = __ldg(reinterpret_cast<const float4*>(ep.bias + col0 + g * 4));
+          v[g * 4 + 0] += bb.x; v[g * 4 + 1] += bb.y; v[g * 4 + 2] += bb.z; v[g * 4 + 3] += bb.w;
+        }
+      }
+    }
+    if (ep.act == 1) {
+      if (ep.aux_out != nullptr) ChunkIO<TOut>::store((TOut*)ep.aux_out, N, row0, col0, M, N, st, lane, v);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = gelu_fast(v[j]);
+    } else if (ep.act == 2) {
+      float z[32];
+      ChunkIO<bf16>::load((const bf16*)ep.aux_in, N, row0, col0, M, N, st, lane, z);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] *= gelu_grad_fast(z[j]);
+    }
+    if (ep.residual != nullptr) {
+      float rr[32];
+      ChunkIO<TOut>::load((const TOut*)ep.residual, N, row0, col0, M, N, st, lane, rr);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] += rr[j];
+    }
+    ChunkIO<TOut>::store(Cs, N, row0, col0, M, N, st, lane, v);
+  }
+}
+
+}  // namespace tc
+}  // namespace bsr
