@@ -156,6 +156,7 @@ def main():
     ap.add_argument("--workload", default="vit_b", choices=list(synth.CONFIGS))
     ap.add_argument("--ref-batch", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--gemm-mode", type=int, default=None, help="1: one CTA per tile, 2: CTA pairs (library default if omitted)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     cfg = synth.CONFIGS[args.workload]
@@ -180,6 +181,8 @@ def main():
     images, labels, task_ids, params = synth.make_workload(cfg, seed=cfg.seed + rank)
     eng = Bd.Engine(cfg, device=f"cuda:{local}")
     eng.set_params(params)
+    if args.gemm_mode is not None:
+        eng.set_gemm_mode(args.gemm_mode)
     del params
     storage = eng.storage_dtype
     host_img = torch.as_tensor(np.ascontiguousarray(images, dtype=np.float32)).to(storage).pin_memory()

@@ -161,6 +161,11 @@ int32_t bsr_get_footprint(const bsr_handle* h, bsr_footprint* out_host);
  * bounded wait in a kernel expired, BSR_ERR_NONFINITE if the last loss was not finite.  Clears it. */
 int32_t bsr_sync_status(bsr_handle* h, void* stream);
 
+/* Which kernels run the dense contractions and attention of a bf16 handle (no counterpart in the paper):
+ * 0 = the FP32-FMA kernels of the fp32 configuration (slow; a cross-check), 1 = tcgen05 kernels with one CTA per
+ * tile (the default), 2 = as 1 but GEMMs with more than 128 rows run on CTA pairs (cta_group::2). */
+int32_t bsr_set_gemm_mode(bsr_handle* h, int32_t mode);
+
 /* Measurement support (no counterpart in the paper).  bsr_profile_enable resets the counters; with
  * time_gemms != 0 every tensor-core GEMM launch of the following steps is bracketed by a pair of CUDA
  * events on the launching stream (host objects; this slows the step slightly, so timed throughput is

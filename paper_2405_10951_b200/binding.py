@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "BSR_OK", -1: "BSR_ERR_INVALID_ARG", -2: "BSR_ERR_UNSUPPORTED
 
 EXPORTS = ["bsr_token_schedule", "bsr_workspace_bytes", "bsr_create", "bsr_destroy", "bsr_last_error", "bsr_set_param",
            "bsr_get_tensor", "bsr_set_lr", "bsr_set_step", "bsr_train_step", "bsr_eval_forward", "bsr_get_footprint",
-           "bsr_sync_status", "bsr_profile_enable", "bsr_profile_read", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_backward",
+           "bsr_sync_status", "bsr_set_gemm_mode", "bsr_profile_enable", "bsr_profile_read", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_backward",
            "bsr_linear_backward_static", "bsr_static_last_error", "bsr_attention_forward"]
 
 
@@ -87,6 +87,7 @@ def lib() -> C.CDLL:
         L.bsr_eval_forward.argtypes = [vp, vp, i32p, i32, vp, f32p, i32p]
         L.bsr_get_footprint.argtypes = [vp, C.POINTER(bsr_footprint)]
         L.bsr_sync_status.argtypes = [vp, vp]
+        L.bsr_set_gemm_mode.argtypes = [vp, i32]
         L.bsr_profile_enable.argtypes = [vp, i32]
         L.bsr_profile_read.argtypes = [vp, vp, C.POINTER(bsr_profile)]
         L.bsr_token_select.argtypes = [f32p, i32, i32, i32, i32, f32p, i32p, i32p, vp]
@@ -325,6 +326,9 @@ class Engine:
 
     def sync_status(self):
         _check(lib().bsr_sync_status(self.h, _stream()), self.h)
+
+    def set_gemm_mode(self, mode: int):
+        _check(lib().bsr_set_gemm_mode(self.h, mode), self.h)
 
     def profile_enable(self, time_gemms: bool):
         _check(lib().bsr_profile_enable(self.h, int(time_gemms)), self.h)

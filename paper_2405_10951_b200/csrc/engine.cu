@@ -840,6 +840,13 @@ int32_t bsr_sync_status(bsr_handle* h, void* stream) {
   return BSR_OK;
 }
 
+int32_t bsr_set_gemm_mode(bsr_handle* h, int32_t mode) {
+  if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
+  if (mode < 0 || mode > 2) return set_err(h->err, BSR_ERR_INVALID_ARG, "mode must be 0, 1 or 2");
+  h->use_tc = mode;
+  return BSR_OK;
+}
+
 int32_t bsr_profile_enable(bsr_handle* h, int32_t time_gemms) {
   if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
   h->prof.on = time_gemms != 0;
