@@ -40,10 +40,15 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict
   unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
   int tpad = (T + 15) & ~15;                     // MMA N
   int nbox = (tpad + AT_BOX - 1) / AT_BOX;       // 64-key boxes of K and V, 64-key chunks of P
-  uint32_t sQ = base, sK = sQ + 2 * AT_BOX_BYTES, sV = sK + nbox * AT_BOX_BYTES, sP = sV + nbox * AT_BOX_BYTES;
+  // Q and K are dead once S = Q K^T has completed, so the probability tile P reuses their space (plus a tail).
   uint32_t p_bytes = nbox * (AT_QROWS * 128);
-  float* cls_buf = reinterpret_cast<float*>(base_ptr + (sP - base) + p_bytes);          // [AT_MAXKEYS + 1]
-  uint32_t bars = sP + p_bytes + (AT_MAXKEYS + 8) * 4;                                   // tma, mma
+  uint32_t qk_bytes = (2 + nbox) * AT_BOX_BYTES;
+  uint32_t sQ = base, sK = sQ + 2 * AT_BOX_BYTES, sP = base;
+  uint32_t sV = base + (p_bytes > qk_bytes ? p_bytes : qk_bytes);
+  uint32_t tail = sV + nbox * AT_BOX_BYTES;
+  float* cls_buf = reinterpret_cast<float*>(base_ptr + (tail - base));                   // [AT_MAXKEYS + 1]
+  uint32_t bars = tail + (AT_MAXKEYS + 8) * 4;                                           // tma, mma
+  uint32_t tmem_cols = tpad <= 128 ? 128u : 256u;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   int tid = threadIdx.x, warp = tid >> 5;
@@ -58,7 +63,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
-    tmem_alloc(smem_u32(&tmem_slot), 256);
+    tmem_alloc(smem_u32(&tmem_slot), tmem_cols);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -191,7 +196,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict
   __syncthreads();
   if (warp == 0) {
     tc_fence_after();
-    tmem_dealloc(tmem, 256);
+    tmem_dealloc(tmem, tmem_cols);
   }
   if (tid == 0 && abort_flag && status != nullptr) atomicOr(status, STATUS_TIMEOUT);
 }
@@ -398,7 +403,8 @@ int attention_fwd_tc(const Ctx& c, const void* qkv, void* out, float* lse, float
   if (!make_map(&map, qkv, (uint64_t)3 * H * d, (uint64_t)B * T, (uint64_t)3 * H * d, AT_BOX)) return -2;
   int tpad = (T + 15) & ~15;
   int nbox = (tpad + AT_BOX - 1) / AT_BOX;
-  size_t smem = 1024 + (size_t)(2 + 2 * nbox) * AT_BOX_BYTES + (size_t)nbox * (AT_QROWS * 128) + (AT_MAXKEYS + 8) * 4 + 64;
+  size_t p_bytes = (size_t)nbox * (AT_QROWS * 128), qk_bytes = (size_t)(2 + nbox) * AT_BOX_BYTES;
+  size_t smem = 1024 + (p_bytes > qk_bytes ? p_bytes : qk_bytes) + (size_t)nbox * AT_BOX_BYTES + (AT_MAXKEYS + 8) * 4 + 64;
   static size_t attr = 0;
   if (smem > attr) {
     if (cudaFuncSetAttribute(attn_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -3;
