@@ -180,6 +180,10 @@ typedef struct {
 } bsr_profile;
 int32_t bsr_profile_enable(bsr_handle* h, int32_t time_gemms);
 int32_t bsr_profile_read(bsr_handle* h, void* stream, bsr_profile* out_host);
+/* Per-launch view of the same timed GEMMs, in launch order: writes up to `capacity` entries of FLOPs and
+ * milliseconds into host arrays and the number of timed launches into *count_out_host. */
+int32_t bsr_profile_launches(bsr_handle* h, void* stream, int32_t capacity, double* flops_out_host, float* ms_out_host,
+                             int32_t* count_out_host);
 
 /* ---- stand-alone forms of the paper-specific token kernels (no handle) ---------------------- */
 

@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "BSR_OK", -1: "BSR_ERR_INVALID_ARG", -2: "BSR_ERR_UNSUPPORTED
 
 EXPORTS = ["bsr_token_schedule", "bsr_workspace_bytes", "bsr_create", "bsr_destroy", "bsr_last_error", "bsr_set_param",
            "bsr_get_tensor", "bsr_set_lr", "bsr_set_step", "bsr_train_step", "bsr_eval_forward", "bsr_get_footprint",
-           "bsr_sync_status", "bsr_set_gemm_mode", "bsr_profile_enable", "bsr_profile_read", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_backward",
+           "bsr_sync_status", "bsr_set_gemm_mode", "bsr_profile_enable", "bsr_profile_read", "bsr_profile_launches", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_backward",
            "bsr_linear_backward_static", "bsr_static_last_error", "bsr_attention_forward"]
 
 
@@ -90,6 +90,7 @@ def lib() -> C.CDLL:
         L.bsr_set_gemm_mode.argtypes = [vp, i32]
         L.bsr_profile_enable.argtypes = [vp, i32]
         L.bsr_profile_read.argtypes = [vp, vp, C.POINTER(bsr_profile)]
+        L.bsr_profile_launches.argtypes = [vp, vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_float), C.POINTER(C.c_int32)]
         L.bsr_token_select.argtypes = [f32p, i32, i32, i32, i32, f32p, i32p, i32p, vp]
         L.bsr_gather_fuse.argtypes = [vp, i32, i32, i32, i32, i32, i32p, i32p, f32p, i32, vp, vp]
         L.bsr_linear_forward.argtypes = [vp, vp, f32p, vp, vp, i32, i32, i32, i32, i32, i32, vp]
@@ -338,6 +339,12 @@ class Engine:
         _check(lib().bsr_profile_read(self.h, _stream(), C.byref(p)), self.h)
         return {"kernel_launches": int(p.kernel_launches), "gemm_launches": int(p.gemm_launches),
                 "gemm_flops": float(p.gemm_flops), "gemm_ms": float(p.gemm_ms)}
+
+    def profile_launches(self, capacity: int = 4096):
+        fl, ms, n = (C.c_double * capacity)(), (C.c_float * capacity)(), C.c_int32(0)
+        _check(lib().bsr_profile_launches(self.h, _stream(), capacity, fl, ms, C.byref(n)), self.h)
+        k = min(n.value, capacity)
+        return [(fl[i], ms[i]) for i in range(k)]
 
     def footprint(self) -> Dict[str, int]:
         fp = bsr_footprint()

@@ -852,6 +852,7 @@ int32_t bsr_profile_enable(bsr_handle* h, int32_t time_gemms) {
   h->prof.on = time_gemms != 0;
   h->prof.used = 0;
   h->prof.flops = 0.0;
+  h->prof.launch_flops.clear();
   h->launches_at_enable = g_kernel_launches;
   return BSR_OK;
 }
@@ -869,6 +870,21 @@ int32_t bsr_profile_read(bsr_handle* h, void* stream, bsr_profile* out) {
   out->gemm_launches = h->prof.used / 2;
   out->gemm_flops = h->prof.flops;
   out->gemm_ms = ms;
+  return BSR_OK;
+}
+
+int32_t bsr_profile_launches(bsr_handle* h, void* stream, int32_t capacity, double* flops_out, float* ms_out, int32_t* count_out) {
+  if (h == nullptr || flops_out == nullptr || ms_out == nullptr || count_out == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "null argument");
+  cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) return set_err(h->err, BSR_ERR_CUDA, "bsr_profile_launches: %s", cudaGetErrorString(e));
+  int n = (int)(h->prof.used / 2);
+  *count_out = n;
+  for (int i = 0; i < n && i < capacity; ++i) {
+    float t = 0.f;
+    cudaEventElapsedTime(&t, h->prof.events[2 * i], h->prof.events[2 * i + 1]);
+    ms_out[i] = t;
+    flops_out[i] = h->prof.launch_flops[i];
+  }
   return BSR_OK;
 }
 

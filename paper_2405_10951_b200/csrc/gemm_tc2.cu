@@ -7,7 +7,7 @@
 //   warp 0 (both CTAs) : TMA producer; every copy signals the full barrier of the leader CTA (rank 0)
 //   warp 1 (leader)    : issues the MMAs; its commits arrive on the empty / accumulator-full barriers of both CTAs
 //   warps 2..9 (both)  : epilogue of the CTA's own 128 rows; they release the accumulator on the leader's barrier
-// Six-stage ring of 32 KB per CTA.  Waits are bounded as in the single-CTA kernel.
+// Five-stage ring of 32 KB per CTA; the epilogue prefetches residual / pre-activation chunks with cp.async.  Waits are bounded as in the single-CTA kernel.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -23,13 +23,13 @@ using namespace tc;
 constexpr int BM = 128;                   // rows per CTA (256 per pair)
 constexpr int BN = 256;                   // columns per pair tile; each CTA stages BN/2 of B
 constexpr int BK = 64;
-constexpr int STAGES = 6;
+constexpr int STAGES = 5;
 constexpr int UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = (BN / 2) * BK * 2;
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;      // 32 KB
 constexpr int EPI_WARPS = 8;
 constexpr int STAGING_BYTES = 32 * 128;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * STAGING_BYTES + 1024 + 256;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * EPI_WARPS * STAGING_BYTES + 1024 + 256;
 constexpr int THREADS = 64 + EPI_WARPS * 32;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;         // clears the CTA-rank bit of a shared address: the even CTA of the pair
@@ -86,7 +86,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   extern __shared__ unsigned char smem_dyn[];
   uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   uint32_t staging0 = base + STAGES * STAGE_BYTES;
-  uint32_t bars = staging0 + EPI_WARPS * STAGING_BYTES;   // full[STAGES], empty[STAGES], tfull[2], tempty[2]
+  uint32_t bars = staging0 + 2 * EPI_WARPS * STAGING_BYTES;   // full[STAGES], empty[STAGES], tfull[2], tempty[2]
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
   auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
@@ -190,7 +190,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     int ew = warp - 2;
     int quarter = warp & 3;
     int chalf = ew >> 2;
-    unsigned char* st = smem_dyn + (staging0 - smem_u32(smem_dyn)) + ew * STAGING_BYTES;
+    uint32_t st_in_addr = staging0 + (2 * ew) * STAGING_BYTES;
+    unsigned char* st_in = smem_dyn + (st_in_addr - smem_u32(smem_dyn));
+    unsigned char* st_out = st_in + STAGING_BYTES;
     int local = 0;
     bool ok = true;
     for (int w = cluster_id; w < work_items && ok; w += n_clusters, ++local) {
@@ -202,15 +204,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       tc_fence_after();
       int row0 = pm * (2 * BM) + (int)rank * BM + quarter * 32;
       TOut* Cs = C + (size_t)sp * M * N;
-#pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {
-        int cchunk = chalf * 4 + cc;
-        uint32_t r[32];
-        uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cchunk * 32);
-        tmem_ld32(taddr, r);
+      uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + chalf * 128);
+      auto load_tmem = [&](int cc, uint32_t* r) {
+        tmem_ld32(taddr0 + cc * 32, r);
         tmem_ld_wait();
-        epilogue_chunk<TOut>(r, ep, Cs, M, N, row0, nt * BN + cchunk * 32, st, lane);
-      }
+      };
+      epilogue_warp_tile<TOut>(load_tmem, ep, Cs, M, N, row0, nt * BN + chalf * 128, 4, st_in, st_in_addr, st_out, lane, false);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(tempty_bar(buf));

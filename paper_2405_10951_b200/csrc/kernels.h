@@ -19,6 +19,7 @@ struct GemmProfile {
   std::vector<cudaEvent_t> events;   // pairs
   size_t used = 0;
   double flops = 0.0;
+  std::vector<double> launch_flops;
   void begin(cudaStream_t s, double f) {
     if (used + 2 > events.size()) {
       size_t old = events.size();
@@ -27,6 +28,7 @@ struct GemmProfile {
     }
     cudaEventRecord(events[used], s);
     flops += f;
+    launch_flops.push_back(f);
   }
   void end(cudaStream_t s) {
     cudaEventRecord(events[used + 1], s);

