@@ -8,7 +8,8 @@
 // dX = dY W, and both operands of the weight-gradient product dW = dY^T X, Eq. 2 and Eq. 4 of the
 // paper).  No operand is transposed in memory; the shared-memory descriptors say how to read it.
 //
-// Kernel shape: persistent, one CTA per SM, 128 x 256 output tiles, k in slabs of 64.
+// Kernel shape: persistent, one CTA per SM, 128 x 256 output tiles, k in slabs of 64.  Tiles are walked with the
+// column index fastest, so that the CTAs running at one time share rows of A and find them in L2.
 //   warp 0      : TMA producer (one lane)
 //   warp 1      : tensor-memory allocation, MMA issue (one lane)
 //   warps 2..9  : epilogue, two warps per TMEM lane quarter; chunks of 32 x 32 outputs go through a staging
@@ -86,7 +87,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int armed = 0;
       bool ok = true;
       for (int w = blockIdx.x; w < work_items && ok; w += gridDim.x) {
-        int mt = w % tiles_m, nt = (w / tiles_m) % tiles_n, sp = w / (tiles_m * tiles_n);
+        int nt = w % tiles_n, mt = (w / tiles_n) % tiles_m, sp = w / (tiles_m * tiles_n);
         int kb0 = sp * kb_per_split, kb1 = min(total_kb, kb0 + kb_per_split);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abortp)) { ok = false; break; }
@@ -154,7 +155,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     int local = 0;
     bool ok = true;
     for (int w = blockIdx.x; w < work_items && ok; w += gridDim.x, ++local) {
-      int mt = w % tiles_m, nt = (w / tiles_m) % tiles_n, sp = w / (tiles_m * tiles_n);
+      int nt = w % tiles_n, mt = (w / tiles_n) % tiles_m, sp = w / (tiles_m * tiles_n);
       int buf = local & 1;
       ok = mbar_wait(tfull_bar(buf), (local >> 1) & 1, abortp);
       ok = __all_sync(0xffffffffu, ok);

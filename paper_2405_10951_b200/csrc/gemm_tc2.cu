@@ -124,7 +124,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       int armed = 0;
       bool ok = true;
       for (int w = cluster_id; w < work_items && ok; w += n_clusters) {
-        int pm = w % pairs_m, nt = (w / pairs_m) % tiles_n, sp = w / (pairs_m * tiles_n);
+        int nt = w % tiles_n, pm = (w / tiles_n) % pairs_m, sp = w / (pairs_m * tiles_n);
         int kb0 = sp * kb_per_split, kb1 = min(total_kb, kb0 + kb_per_split);
         int m0 = pm * (2 * BM) + (int)rank * BM;          // this CTA's rows of A
         int n0 = nt * BN + (int)rank * (BN / 2);          // this CTA's share of B
@@ -196,7 +196,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     int local = 0;
     bool ok = true;
     for (int w = cluster_id; w < work_items && ok; w += n_clusters, ++local) {
-      int pm = w % pairs_m, nt = (w / pairs_m) % tiles_n, sp = w / (pairs_m * tiles_n);
+      int nt = w % tiles_n, pm = (w / tiles_n) % pairs_m, sp = w / (pairs_m * tiles_n);
       int buf = local & 1;
       ok = mbar_wait(tfull_bar(buf), (local >> 1) & 1, abortp);
       ok = __all_sync(0xffffffffu, ok);
