@@ -39,6 +39,7 @@ struct Tensor {
 struct BlockBufs {          // byte offsets into the workspace; filled for frozen (scratch) and trainable (arena) blocks
   size_t x_in, y1, qkv, o, xp_full, xp, y2, z, hh, x_out;
   size_t mean1, rstd1, lse, mean2, rstd2, p, s, kept, dropped;
+  size_t o_cls, xin_cls;    // classification rows of o and of the block input (last block only)
 };
 
 struct Bump {
@@ -280,6 +281,8 @@ size_t plan(bsr_handle* h) {
     bb.z = b.take(Mf * F * es);
     bb.hh = b.take(Mf * F * es);
     bb.x_out = b.take(Mf * D * 4);
+    bb.o_cls = b.take((size_t)Bm * D * es);
+    bb.xin_cls = b.take((size_t)Bm * D * 4);
     next_in = bb.x_out;
   }
   h->arena_bytes = b.off - a0;
@@ -309,6 +312,8 @@ size_t plan(bsr_handle* h) {
     bb.s = b.take((size_t)Bm * (T0 - 1) * 4);
     bb.kept = b.take((size_t)Bm * (T0 - 1) * 4);
     bb.dropped = b.take((size_t)Bm * (T0 - 1) * 4);
+    bb.o_cls = b.take((size_t)Bm * D * es);
+    bb.xin_cls = b.take((size_t)Bm * D * 4);
     size_t in1 = h->bufs_frozen[1].x_in, out1 = h->bufs_frozen[1].x_out;
     h->bufs_frozen[1] = bb;
     h->bufs_frozen[1].x_in = in1;
@@ -375,6 +380,11 @@ int check_cuda(bsr_handle* h, const char* what) {
   return BSR_OK;
 }
 
+// In the last block only the classification token's output is ever used (the head reads row 0), so everything
+// after the attention product -- projection, LayerNorm 2, FFN and their backward -- runs on the B classification
+// rows alone.  The results are identical: the other rows' outputs feed nothing and their gradients are zero.
+bool cls_tail(const bsr_handle* h, int l) { return l == h->cfg.dims.depth - 1 && h->sched.k[l] < 0; }
+
 // One encoder block forward.  `save` keeps the statistics and pre-activations the backward pass needs.
 int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb, bool save, int* kept_out) {
   const bsr_dims& d = h->cfg.dims;
@@ -394,11 +404,23 @@ int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb
   int rc = attention_fwd(c, h->base + bb.qkv, h->base + bb.o, save ? h->at<float>(bb.lse) : nullptr,
                          is_drop ? h->at<float>(bb.p) : nullptr, B, Ta, H, hd);
   if (rc != 0) return set_err(h->err, BSR_ERR_UNSUPPORTED, "attention: %d tokens of head dimension %d do not fit this kernel", Ta, hd);
+  size_t es = dtype_size(d.dtype);
+  bool tail = cls_tail(h, l);
+  const void* proj_in = h->base + bb.o;
+  const void* proj_res = h->base + bb.x_in;
+  if (tail) {                  // from here on: B rows
+    copy_rows(c.stream, h->base + bb.o, (long)Ta * D * es, h->base + bb.o_cls, (long)D * es, B, (int)(D * es));
+    copy_rows(c.stream, h->base + bb.x_in, (long)Ta * D * 4, h->base + bb.xin_cls, (long)D * 4, B, D * 4);
+    proj_in = h->base + bb.o_cls;
+    proj_res = h->base + bb.xin_cls;
+    Ma = B;
+    Mf = B;
+  }
   GemmEpilogue e2;
   e2.bias = (const float*)h->wb(l, "attn.proj.bias");
-  e2.residual = h->base + bb.x_in;
+  e2.residual = proj_res;
   void* xp_dst = h->base + (shrinks ? bb.xp_full : bb.xp);
-  gemm(c, h->base + bb.o, D, 1, h->wb(l, "attn.proj.weight"), D, 1, xp_dst, 1, Ma, D, D, e2);
+  gemm(c, proj_in, D, 1, h->wb(l, "attn.proj.weight"), D, 1, xp_dst, 1, Ma, D, D, e2);
   if (is_drop) {
     int M = Ta - 1;
     token_select(c.stream, h->at<float>(bb.p), B, H, M, k, h->at<float>(bb.s), h->at<int>(bb.kept), h->at<int>(bb.dropped));
@@ -438,6 +460,10 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
   int Ma = B * Ta, Mf = B * Tf;
   bool shrinks = k >= 0 && Tf != Ta;
   bool bf = d.dtype == BSR_DTYPE_BF16;
+  bool tail = cls_tail(h, l);
+  size_t es = dtype_size(d.dtype);
+  int Mdense = Ma;
+  if (tail) { Ma = B; Mf = B; }          // FFN and projection gradients live on the classification rows only
   Ctx cf = c;
   cf.dtype = 0;
   float* csp = h->at<float>(h->off_cs_partials);
@@ -471,9 +497,25 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
     if (h->cfg.fuse_mode == BSR_FUSE_WEIGHTED_SUM) cls_extra = h->at<float>(h->off_escore);
   }
   // attention output projection
-  gemm(c, op(dxp), D, 1, h->wb(l, "attn.proj.weight"), 1, D, d_o, 0, Ma, D, D, none);
-  gemm(c, op(dxp), 1, D, h->base + bb.o, 1, D, h->gb(l, "attn.proj.weight"), 1, D, D, Ma, none);
-  colsum(cf, dxp.f, Ma, D, csp, h->gb(l, "attn.proj.bias"));
+  const float* ln1_res = dxp.f;
+  if (!tail) {
+    gemm(c, op(dxp), D, 1, h->wb(l, "attn.proj.weight"), 1, D, d_o, 0, Ma, D, D, none);
+    gemm(c, op(dxp), 1, D, h->base + bb.o, 1, D, h->gb(l, "attn.proj.weight"), 1, D, D, Ma, none);
+    colsum(cf, dxp.f, Ma, D, csp, h->gb(l, "attn.proj.bias"));
+  } else {
+    // B rows: dO_cls = dx'_cls Wo, dWo = dx'_cls^T o_cls; then both gradients go back into zeroed dense tensors
+    void* do_cls = h->base + h->off_dy;                      // free at this point
+    gemm(c, op(dxp), D, 1, h->wb(l, "attn.proj.weight"), 1, D, do_cls, 0, B, D, D, none);
+    gemm(c, op(dxp), 1, D, h->base + bb.o_cls, 1, D, h->gb(l, "attn.proj.weight"), 1, D, D, B, none);
+    colsum(cf, dxp.f, B, D, csp, h->gb(l, "attn.proj.bias"));
+    cudaMemsetAsync(d_o, 0, (size_t)Mdense * D * es, c.stream);
+    copy_rows(c.stream, do_cls, (long)D * es, d_o, (long)Ta * D * es, B, (int)(D * es));
+    float* dense_res = h->at<float>(h->off_dxp);
+    cudaMemsetAsync(dense_res, 0, (size_t)Mdense * D * 4, c.stream);
+    copy_rows(c.stream, dxp.f, (long)D * 4, dense_res, (long)Ta * D * 4, B, D * 4);
+    ln1_res = dense_res;
+    Ma = Mdense;
+  }
   int rc = attention_bwd(c, h->base + bb.qkv, h->base + bb.o, d_o, h->at<float>(bb.lse), h->at<float>(h->off_delta),
                          cls_extra, dqkv, B, Ta, H, hd);
   if (rc != 0) return set_err(h->err, BSR_ERR_UNSUPPORTED, "attention backward: %d tokens do not fit this kernel", Ta);
@@ -482,7 +524,7 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
   gemm(c, dqkv, 1, 3 * D, h->base + bb.y1, 1, D, h->gb(l, "attn.qkv.weight"), 1, 3 * D, D, Ma, none);
   colsum(c, dqkv, Ma, 3 * D, csp, h->gb(l, "attn.qkv.bias"));
   layernorm_bwd(c, dy, 0, h->at<float>(bb.x_in), D, h->at<float>(bb.mean1), h->at<float>(bb.rstd1),
-                (const float*)h->wb(l, "norm1.weight"), dxp.f, need_dxi ? dxi.f : nullptr, D, need_dxi ? dxi.c : nullptr, lnp,
+                (const float*)h->wb(l, "norm1.weight"), ln1_res, need_dxi ? dxi.f : nullptr, D, need_dxi ? dxi.c : nullptr, lnp,
                 h->gb(l, "norm1.weight"), h->gb(l, "norm1.bias"), Ma, D);
   return BSR_OK;
 }
@@ -738,7 +780,7 @@ int32_t bsr_train_step(bsr_handle* h, const void* images, const int32_t* labels,
   size_t x_last = 0;
   rc = forward_all(h, c, images, B, true, &x_last);
   if (rc != BSR_OK) return rc;
-  int Tl = h->sched.tf[d.depth - 1];
+  int Tl = cls_tail(h, d.depth - 1) ? 1 : h->sched.tf[d.depth - 1];   // rows per image in the last block's output
   HeadDesc hd = head_desc(h);
   float* xn = h->at<float>(h->off_xn);
   layernorm_fwd(c, h->at<float>(x_last), (long)Tl * D, (const float*)h->w("norm.weight"), (const float*)h->w("norm.bias"), xn, 1,
@@ -790,7 +832,7 @@ int32_t bsr_eval_forward(bsr_handle* h, const void* images, const int32_t* task_
   size_t x_last = 0;
   rc = forward_all(h, c, images, batch, false, &x_last);
   if (rc != BSR_OK) return rc;
-  int Tl = h->sched.tf[d.depth - 1];
+  int Tl = cls_tail(h, d.depth - 1) ? 1 : h->sched.tf[d.depth - 1];   // rows per image in the last block's output
   HeadDesc hd = head_desc(h);
   float* xn = h->at<float>(h->off_xn);
   layernorm_fwd(c, h->at<float>(x_last), (long)Tl * d.dim, (const float*)h->w("norm.weight"), (const float*)h->w("norm.bias"), xn, 1,

@@ -137,6 +137,9 @@ struct AdamChunk { uint32_t offset; uint32_t count; int64_t shadow; uint32_t dec
 void adamw(const Ctx& c, const AdamChunk* chunks, int nchunks, float* master, const float* grad, float* m, float* v,
            void* shadow_base, float lr, float b1, float b2, float eps, float wd, float bc1, float bc2);
 
+// dst row r = src row r (row_bytes a multiple of 16), independent pitches: gathers / scatters token rows.
+void copy_rows(cudaStream_t s, const void* src, long src_pitch_bytes, void* dst, long dst_pitch_bytes, int rows, int row_bytes);
+
 // ---- conversions ------------------------------------------------------------------------------
 void convert_from_float(const Ctx& c, const float* src, void* dst, size_t n);   // float -> storage dtype
 void convert_to_float(const Ctx& c, const void* src, float* dst, size_t n);     // storage dtype -> float

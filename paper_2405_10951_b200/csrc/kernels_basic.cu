@@ -545,6 +545,25 @@ void adamw(const Ctx& c, const AdamChunk* chunks, int nchunks, float* master, co
 }
 
 // ------------------------------------------------------------------------------------------------
+// Strided row copy in 16-byte units: dst[r] = src[r] for rows of row_bytes, each side with its own row pitch.
+// Gathers the classification rows of a [B, T, D] tensor into [B, D] and scatters them back.
+// ------------------------------------------------------------------------------------------------
+__global__ void copy_rows_kernel(const char* __restrict__ src, long src_pitch, char* __restrict__ dst, long dst_pitch, int rows,
+                                 int units) {
+  long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (long)rows * units) return;
+  int r = (int)(i / units), u = (int)(i % units);
+  *reinterpret_cast<uint4*>(dst + (long)r * dst_pitch + u * 16L) = *reinterpret_cast<const uint4*>(src + (long)r * src_pitch + u * 16L);
+}
+
+void copy_rows(cudaStream_t st, const void* src, long src_pitch_bytes, void* dst, long dst_pitch_bytes, int rows, int row_bytes) {
+  note_launch(1);
+  int units = row_bytes / 16;
+  long total = (long)rows * units;
+  copy_rows_kernel<<<ceil_div(total, 256), 256, 0, st>>>((const char*)src, src_pitch_bytes, (char*)dst, dst_pitch_bytes, rows, units);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Conversions
 // ------------------------------------------------------------------------------------------------
 template <typename T>
