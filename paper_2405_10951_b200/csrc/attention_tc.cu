@@ -218,15 +218,18 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
   uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
   constexpr uint32_t TILE = 2 * AT_BOX_BYTES;            // 128 rows x 128 bytes
-  uint32_t sQ = base, sK = sQ + TILE, sV = sK + TILE, sG = sV + TILE, sP = sG + TILE, sS = sP + 2 * TILE;
-  uint32_t bars = sS + 2 * TILE;
+  int tpad = (T + 15) & ~15;
+  // P and dS hold tpad query rows per 64-key chunk; dS starts in V's space (V is dead once dP = dO V^T is done).
+  uint32_t CH = (uint32_t)tpad * 128u;
+  uint32_t sQ = base, sK = sQ + TILE, sG = sK + TILE, sV = sG + TILE, sS = sV;
+  uint32_t sP = sV + (2 * CH > TILE ? 2 * CH : TILE);
+  uint32_t bars = sP + 2 * CH + (3 * CH < 16384u ? 16384u - 3 * CH : 0u);   // slack: MMA row extent past tpad stays in bounds
   unsigned char* pP = base_ptr + (sP - base);
   unsigned char* pS = base_ptr + (sS - base);
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   int tid = threadIdx.x, warp = tid >> 5;
   int bh = blockIdx.x, b = bh / H, h = bh % H;
-  int tpad = (T + 15) & ~15;
   uint32_t tma_bar = bars, mma_bar = bars + 8;
   if (tid == 0) {
     abort_flag = 0;
@@ -235,14 +238,15 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
-    tmem_alloc(smem_u32(&tmem_slot), 512);
+    tmem_alloc(smem_u32(&tmem_slot), 256);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   uint32_t tmem = tmem_slot;
-  constexpr uint32_t C_S = 0, C_DP = 128, C_DQ = 256, C_DK = 320, C_DV = 384;
+  // dQ, dK, dV reuse the columns of S and dP, which are dead once P and dS sit in shared memory
+  constexpr uint32_t C_S = 0, C_DP = 128, C_DQ = 0, C_DK = 64, C_DV = 128;
   volatile int* abortp = &abort_flag;
   bool ok = true;
   if (tid == 0) {
@@ -333,9 +337,12 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
           hp[i] = __floats2bfloat162_rn(p[g * 8 + 2 * i], p[g * 8 + 2 * i + 1]);
           hs[i] = __floats2bfloat162_rn(ds[g * 8 + 2 * i], ds[g * 8 + 2 * i + 1]);
         }
-        uint32_t off = p_offset(tid, ch * 4 + g);
-        *reinterpret_cast<uint4*>(pP + off) = vp;
-        *reinterpret_cast<uint4*>(pS + off) = vs;
+        if (tid < tpad) {
+          int key8 = ch * 4 + g;
+          uint32_t off = (uint32_t)(key8 >> 3) * CH + (uint32_t)tid * 128u + (uint32_t)(((key8 & 7) ^ (tid & 7)) << 4);
+          *reinterpret_cast<uint4*>(pP + off) = vp;
+          *reinterpret_cast<uint4*>(pS + off) = vs;
+        }
       }
     }
   }
@@ -348,14 +355,14 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
     // dQ = dS K: A = dS (contiguous along keys), B = K read with keys as the reduction index
     uint32_t id_q = make_idesc_mn(AT_QROWS, AT_D, false, true);
     for (int k = 0; k < tpad / 16; ++k)
-      umma_bf16(tmem + C_DQ, make_desc(sS + (k >> 2) * TILE + (k & 3) * 32, 16, 1024), make_desc(sK + k * 2048, 8192, 1024), id_q,
+      umma_bf16(tmem + C_DQ, make_desc(sS + (k >> 2) * CH + (k & 3) * 32, 16, 1024), make_desc(sK + k * 2048, 8192, 1024), id_q,
                 k > 0 ? 1u : 0u);
     // dK = dS^T Q and dV = P^T dO: both operands read with queries as the reduction index
     uint32_t id_t = make_idesc_mn(AT_QROWS, AT_D, true, true);
-    for (int k = 0; k < AT_QROWS / 16; ++k)
-      umma_bf16(tmem + C_DK, make_desc(sS + k * 2048, TILE, 1024), make_desc(sQ + k * 2048, 8192, 1024), id_t, k > 0 ? 1u : 0u);
-    for (int k = 0; k < AT_QROWS / 16; ++k)
-      umma_bf16(tmem + C_DV, make_desc(sP + k * 2048, TILE, 1024), make_desc(sG + k * 2048, 8192, 1024), id_t, k > 0 ? 1u : 0u);
+    for (int k = 0; k < tpad / 16; ++k)
+      umma_bf16(tmem + C_DK, make_desc(sS + k * 2048, CH, 1024), make_desc(sQ + k * 2048, 8192, 1024), id_t, k > 0 ? 1u : 0u);
+    for (int k = 0; k < tpad / 16; ++k)
+      umma_bf16(tmem + C_DV, make_desc(sP + k * 2048, CH, 1024), make_desc(sG + k * 2048, 8192, 1024), id_t, k > 0 ? 1u : 0u);
     umma_commit(mma_bar);
   }
   if (ok) ok = mbar_wait(mma_bar, 1, abortp);
@@ -387,7 +394,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
   __syncthreads();
   if (warp == 0) {
     tc_fence_after();
-    tmem_dealloc(tmem, 512);
+    tmem_dealloc(tmem, 256);
   }
   if (tid == 0 && abort_flag && status != nullptr) atomicOr(status, STATUS_TIMEOUT);
 }
@@ -428,11 +435,12 @@ int attention_bwd_tc(const Ctx& c, const void* qkv, const void* dout, const floa
   CUtensorMap mq, mg;
   if (!make_map(&mq, qkv, (uint64_t)3 * H * d, (uint64_t)B * T, (uint64_t)3 * H * d, AT_BOX)) return -2;
   if (!make_map(&mg, dout, (uint64_t)H * d, (uint64_t)B * T, (uint64_t)H * d, AT_BOX)) return -2;
-  size_t smem = 1024 + 8 * (size_t)(2 * AT_BOX_BYTES) + 64;
-  static bool attr = false;
-  if (!attr) {
+  size_t tile = 2 * (size_t)AT_BOX_BYTES, ch = (size_t)((T + 15) & ~15) * 128;
+  size_t smem = 1024 + 3 * tile + (2 * ch > tile ? 2 * ch : tile) + 2 * ch + (3 * ch < 16384 ? 16384 - 3 * ch : 0) + 64;
+  static size_t attr = 0;
+  if (smem > attr) {
     if (cudaFuncSetAttribute(attn_bwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -3;
-    attr = true;
+    attr = smem;
   }
   note_launch(1);
   attn_bwd_tc_kernel<<<B * H, 128, smem, c.stream>>>(mq, mg, lse, cls_extra, (bf16*)dqkv, B, T, H, c.status);
