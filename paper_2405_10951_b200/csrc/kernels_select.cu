@@ -63,11 +63,84 @@ __global__ void token_select_kernel(const float* __restrict__ p, int B, int H, i
   }
 }
 
+// Same selection with the keys of one image held in registers (IPL per lane, M <= 32 * IPL): the 32 threshold
+// steps are register compares and one warp reduction each.  Element j lives in lane j % 32, slot j / 32, so a
+// slot is a run of 32 consecutive tokens and ballots give positions in token order.
+template <int IPL>
+__global__ void __launch_bounds__(SEL_WARPS * 32)
+token_select_reg_kernel(const float* __restrict__ p, int B, int H, int M, int k, float* __restrict__ scores,
+                        int* __restrict__ kept, int* __restrict__ dropped) {
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int b = blockIdx.x * SEL_WARPS + warp;
+  if (b >= B) return;
+  const float* pb = p + (size_t)b * H * M;
+  uint32_t key[IPL];
+  float acc[IPL];
+  // head sum in head order per token; the IPL loads of one head are independent, so many are in flight
+#pragma unroll
+  for (int i = 0; i < IPL; ++i) acc[i] = (i * 32 + lane < M) ? pb[i * 32 + lane] : 0.f;
+#pragma unroll 2
+  for (int h = 1; h < H; ++h) {
+    const float* ph = pb + (size_t)h * M;
+#pragma unroll
+    for (int i = 0; i < IPL; ++i)
+      if (i * 32 + lane < M) acc[i] = acc[i] + ph[i * 32 + lane];
+  }
+#pragma unroll
+  for (int i = 0; i < IPL; ++i) {
+    int j = i * 32 + lane;
+    key[i] = 0u;
+    if (j < M) {
+      float s = acc[i] / (float)H;
+      scores[(size_t)b * M + j] = s;
+      key[i] = ordered_key(s);
+    }
+  }
+  // keys of absent elements are 0, below every real key (a real key has its top bit set unless the score is negative;
+  // scores are probabilities), and they are excluded by index below anyway
+  uint32_t t = 0;
+  for (int bit = 31; bit >= 0; --bit) {
+    uint32_t cand = t | (1u << bit);
+    int cnt = 0;
+#pragma unroll
+    for (int i = 0; i < IPL; ++i) cnt += (i * 32 + lane < M && key[i] >= cand) ? 1 : 0;
+    cnt = __reduce_add_sync(0xffffffffu, cnt);
+    if (cnt >= k) t = cand;
+  }
+  int gt = 0;
+#pragma unroll
+  for (int i = 0; i < IPL; ++i) gt += (i * 32 + lane < M && key[i] > t) ? 1 : 0;
+  gt = __reduce_add_sync(0xffffffffu, gt);
+  int need_eq = k - gt;
+  int n_kept = 0, n_drop = 0, eq_seen = 0;
+  uint32_t lt_mask = (1u << lane) - 1u;
+#pragma unroll
+  for (int i = 0; i < IPL; ++i) {
+    int j = i * 32 + lane;
+    if (i * 32 >= M) break;
+    bool valid = j < M;
+    bool is_eq = valid && key[i] == t;
+    uint32_t eq_mask = __ballot_sync(0xffffffffu, is_eq);
+    int eq_rank = eq_seen + __popc(eq_mask & lt_mask);
+    bool keep = valid && (key[i] > t || (is_eq && eq_rank < need_eq));
+    uint32_t keep_mask = __ballot_sync(0xffffffffu, keep);
+    uint32_t drop_mask = __ballot_sync(0xffffffffu, valid && !keep);
+    if (keep) kept[(size_t)b * k + n_kept + __popc(keep_mask & lt_mask)] = j;
+    else if (valid) dropped[(size_t)b * (M - k) + n_drop + __popc(drop_mask & lt_mask)] = j;
+    n_kept += __popc(keep_mask);
+    n_drop += __popc(drop_mask);
+    eq_seen += __popc(eq_mask);
+  }
+}
+
 void token_select(cudaStream_t s, const float* p, int B, int H, int M, int k, float* scores, int* kept, int* dropped) {
   note_launch(1);
+  int blocks = ceil_div(B, SEL_WARPS), threads = SEL_WARPS * 32;
+  if (M <= 256) { token_select_reg_kernel<8><<<blocks, threads, 0, s>>>(p, B, H, M, k, scores, kept, dropped); return; }
+  if (M <= 640) { token_select_reg_kernel<20><<<blocks, threads, 0, s>>>(p, B, H, M, k, scores, kept, dropped); return; }
   size_t smem = (size_t)SEL_WARPS * M * sizeof(uint32_t);
   if (smem > 48 * 1024) cudaFuncSetAttribute(token_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  token_select_kernel<<<ceil_div(B, SEL_WARPS), SEL_WARPS * 32, smem, s>>>(p, B, H, M, k, scores, kept, dropped);
+  token_select_kernel<<<blocks, threads, smem, s>>>(p, B, H, M, k, scores, kept, dropped);
 }
 
 // ------------------------------------------------------------------------------------------------

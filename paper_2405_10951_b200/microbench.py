@@ -1,0 +1,105 @@
+"""Stand-alone timing of single kernels of the BSR step through the C ABI.
+
+    python -m paper_2405_10951_b200.microbench gemm --m 25216 --n 2304 --k 768 [--gelu] [--mode 1|2] [--iters 20]
+    python -m paper_2405_10951_b200.microbench backward --m 12800 --n 2304 --k 768
+    python -m paper_2405_10951_b200.microbench select_gather --batch 4096 --heads 12 --tokens 197 --dim 768 --keep 0.7
+    python -m paper_2405_10951_b200.microbench attention --batch 128 --heads 12 --tokens 197
+
+Each prints one JSON line with the time per launch (CUDA events on the current stream, after warm-up) and the
+achieved TFLOP/s or GB/s on the kernel's algorithmic work.  Inputs are seeded and synthetic.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+
+import torch
+
+from . import binding as Bd
+
+
+def timed(fn, iters, flush=None):
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    total = 0.0
+    for _ in range(iters):
+        if flush is not None:
+            flush.zero_()                       # evict the previous iteration's data from L2
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        total += e0.elapsed_time(e1)
+    return total / iters
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("what", choices=["gemm", "backward", "select_gather", "attention"])
+    ap.add_argument("--m", type=int, default=25216)
+    ap.add_argument("--n", type=int, default=2304)
+    ap.add_argument("--k", type=int, default=768)
+    ap.add_argument("--gelu", action="store_true")
+    ap.add_argument("--residual", action="store_true")
+    ap.add_argument("--mode", type=int, default=1)
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--batch", type=int, default=4096)
+    ap.add_argument("--heads", type=int, default=12)
+    ap.add_argument("--tokens", type=int, default=197)
+    ap.add_argument("--dim", type=int, default=768)
+    ap.add_argument("--keep", type=float, default=0.7)
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
+    ap.add_argument("--flush-l2", action="store_true")
+    a = ap.parse_args()
+    torch.manual_seed(0)
+    dev = "cuda"
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev) if a.flush_l2 else None
+    out = {"kernel": a.what}
+    if a.what == "gemm":
+        x = torch.randn(a.m, a.k, device=dev).bfloat16()
+        w = (torch.randn(a.n, a.k, device=dev) / math.sqrt(a.k)).bfloat16()
+        b = torch.randn(a.n, device=dev)
+        r = torch.randn(a.m, a.n, device=dev).bfloat16() if a.residual else None
+        ms = timed(lambda: Bd.bsr_linear_forward(x, w, b, r, act_gelu=a.gelu, use_tensor_cores=a.mode), a.iters, flush)
+        out.update(m=a.m, n=a.n, k=a.k, gelu=a.gelu, mode=a.mode, us=ms * 1e3, tflops=2.0 * a.m * a.n * a.k / ms / 1e9)
+    elif a.what == "backward":
+        x = torch.randn(a.m, a.k, device=dev).bfloat16()
+        w = (torch.randn(a.n, a.k, device=dev) / math.sqrt(a.k)).bfloat16()
+        dy = torch.randn(a.m, a.n, device=dev).bfloat16()
+        ws = torch.empty(160 * 128 * 256, dtype=torch.float32, device=dev)
+        ms = timed(lambda: Bd.bsr_linear_backward(x, w, dy, use_tensor_cores=a.mode, workspace=ws), a.iters, flush)
+        out.update(m=a.m, n=a.n, k=a.k, mode=a.mode, us=ms * 1e3, tflops=4.0 * a.m * a.n * a.k / ms / 1e9)
+    elif a.what == "select_gather":
+        B, H, T, D = a.batch, a.heads, a.tokens, a.dim
+        M = T - 1
+        k = max(1, min(M, math.ceil(a.keep * M - 1e-9)))
+        tdt = torch.bfloat16 if a.dtype == "bf16" else torch.float32
+        z = torch.randn(B, H, M + 1, device=dev) * 2.5
+        p = torch.softmax(z, dim=-1)[..., 1:].contiguous()
+        x = torch.randn(B, T, D, device=dev).to(tdt)
+        s, kept, dropped = Bd.bsr_token_select(p, k)
+        o = Bd.bsr_gather_fuse(x, kept, dropped, s, 1)
+        import ctypes as C
+        L, st = Bd.lib(), C.c_void_p(torch.cuda.current_stream().cuda_stream)
+        ptr = lambda t: C.c_void_p(t.data_ptr())
+        # outputs pre-allocated so that the timed region holds the launch only
+        ms_sel = timed(lambda: L.bsr_token_select(ptr(p), B, H, M, k, ptr(s), ptr(kept), ptr(dropped), st), a.iters, flush)
+        ms_gat = timed(lambda: Bd.bsr_gather_fuse(x, kept, dropped, s, 1, out=o), a.iters, flush)
+        es = x.element_size()
+        sel_bytes = B * (H * M * 4 + M * 4 + M * 4)
+        gat_bytes = B * ((1 + M) * D * es + (1 + k + 1) * D * es + M * 8)
+        out.update(batch=B, heads=H, tokens=T, dim=D, k=k, dtype=a.dtype, select_us=ms_sel * 1e3, select_gbs=sel_bytes / ms_sel / 1e6,
+                   gather_us=ms_gat * 1e3, gather_gbs=gat_bytes / ms_gat / 1e6, select_bytes=sel_bytes, gather_bytes=gat_bytes)
+    else:
+        B, H, T = a.batch, a.heads, a.tokens
+        qkv = torch.randn(B, T, 3, H, 64, device=dev).bfloat16()
+        ms = timed(lambda: Bd.bsr_attention_forward(qkv, H, use_tensor_cores=True), a.iters, flush)
+        out.update(batch=B, heads=H, tokens=T, us=ms * 1e3, tflops=4.0 * B * H * T * T * 64 / ms / 1e9)
+    print(json.dumps(out), flush=True)
+
+
+if __name__ == "__main__":
+    main()
