@@ -196,15 +196,26 @@ def moe_route(cfg, glogits):
     return order, e / e.sum(axis=-1, keepdims=True)
 
 
-def moe_fwd(cfg, params, l, y, task_ids):
-    """y: [B, T, D] (LayerNorm output).  Returns output and cache."""
+def moe_fwd(cfg, params, l, y, task_ids, forced_experts=None):
+    """y: [B, T, D] (LayerNorm output).  Returns output and cache.
+
+    forced_experts [B, T, k] replaces the router's top-k choice (the weights are still the softmax of this
+    oracle's own gate logits at those experts): used when a lower-precision run made a different choice
+    between near-equal logits, exactly as forced_keep does for the kept tokens."""
     p = f"blocks.{l}.moe."
     B, T, D = y.shape
     wg = params[p + "gate.weight"][task_ids]                 # [B, E, D]: task-dependent router
     glogits = np.einsum("btd,bed->bte", y, wg)
     experts, w = moe_route(cfg, glogits)                     # [B, T, k]
+    own_experts = experts
+    if forced_experts is not None:
+        forced = np.asarray(forced_experts, dtype=np.int64).reshape(B, T, cfg.moe_top_k)
+        experts = np.where(forced < 0, own_experts, forced)          # negative entries: keep this oracle's choice
+        sel = np.take_along_axis(glogits, experts, axis=-1)
+        ee = np.exp(sel - sel.max(axis=-1, keepdims=True))
+        w = ee / ee.sum(axis=-1, keepdims=True)
     out = np.zeros_like(y)
-    cache = {"y": y, "experts": experts, "w": w, "z": {}, "h": {}, "yo": {}}
+    cache = {"y": y, "experts": experts, "w": w, "z": {}, "h": {}, "yo": {}, "own_experts": own_experts, "glogits": glogits}
     for e in range(cfg.moe_experts):
         for slot in range(cfg.moe_top_k):
             mask = experts[..., slot] == e                   # [B, T]
@@ -264,7 +275,7 @@ def moe_bwd(cfg, params, l, dout, cache, task_ids, grads, want_param_grads):
     return dy
 
 
-def block_fwd(cfg, params, l, x, task_ids, k, forced_keep):
+def block_fwd(cfg, params, l, x, task_ids, k, forced_keep, forced_experts=None):
     """One encoder block; at a token drop location the compaction sits between MHSA and FFN."""
     p = f"blocks.{l}."
     c = {"x": x}
@@ -306,7 +317,7 @@ def block_fwd(cfg, params, l, x, task_ids, k, forced_keep):
     y2, c["ln2"] = layer_norm(xp, params[p + "norm2.weight"], params[p + "norm2.bias"], cfg.ln_eps)
     c["y2"] = y2
     if l in cfg.moe_blocks:
-        f, c["moe"] = moe_fwd(cfg, params, l, y2, task_ids)
+        f, c["moe"] = moe_fwd(cfg, params, l, y2, task_ids, forced_experts)
     else:
         z = linear(y2, params[p + "mlp.fc1.weight"], params[p + "mlp.fc1.bias"])
         h = gelu(z)
@@ -364,7 +375,7 @@ def block_bwd(cfg, params, l, dout, c, task_ids, grads, want_param_grads, need_d
     return (dxp + dln1) if need_dx else None
 
 
-def forward(cfg, params, images, task_ids=None, forced_keep=None, keep_cache=False):
+def forward(cfg, params, images, task_ids=None, forced_keep=None, keep_cache=False, forced_experts=None):
     """Forward with token dropping.  Returns a dict with logits (list per image), kept sets, caches."""
     B = images.shape[0]
     if task_ids is None:
@@ -372,13 +383,17 @@ def forward(cfg, params, images, task_ids=None, forced_keep=None, keep_cache=Fal
     sched = token_schedule(cfg)
     x = embed(cfg, params, np.asarray(images, dtype=np.float64))
     caches, kept, margins, scores, tokens = [], [], [], [], []
+    routing = {}
     di = 0
     for l in range(cfg.depth):
         ta, tf, k = sched[l]
         fk = None
         if k is not None and forced_keep is not None and forced_keep[di] is not None:
             fk = forced_keep[di]
-        x, c, info = block_fwd(cfg, params, l, x, task_ids, k, fk)
+        fe = forced_experts.get(l) if forced_experts else None
+        x, c, info = block_fwd(cfg, params, l, x, task_ids, k, fk, fe)
+        if l in cfg.moe_blocks:
+            routing[l] = {"experts": c["moe"]["experts"], "own_experts": c["moe"]["own_experts"], "glogits": c["moe"]["glogits"]}
         if k is not None:
             kept.append(info["kept"])
             margins.append(info["margins"])
@@ -394,7 +409,7 @@ def forward(cfg, params, images, task_ids=None, forced_keep=None, keep_cache=Fal
         if sel.any():
             logits[sel, :ncls] = linear(xn[sel], params[f"head.{t}.weight"], params[f"head.{t}.bias"])
     return {"logits": logits, "kept": kept, "margins": margins, "scores": scores, "tokens": tokens,
-            "caches": caches, "xn": xn, "lnf": lnf, "x_last": x, "task_ids": task_ids}
+            "caches": caches, "xn": xn, "lnf": lnf, "x_last": x, "task_ids": task_ids, "routing": routing}
 
 
 def cross_entropy(logits, labels):
@@ -436,9 +451,9 @@ def adamw(cfg, p, g, m, v, step, decay):
     return new, m, v
 
 
-def train_step(cfg, params, images, labels, task_ids=None, forced_keep=None, opt_state=None, step=1):
+def train_step(cfg, params, images, labels, task_ids=None, forced_keep=None, opt_state=None, step=1, forced_experts=None):
     """One BSR fine-tuning step.  Returns loss, logits, gradients, updated parameters and moments."""
-    fw = forward(cfg, params, images, task_ids, forced_keep, keep_cache=True)
+    fw = forward(cfg, params, images, task_ids, forced_keep, keep_cache=True, forced_experts=forced_experts)
     task_ids = fw["task_ids"]
     loss, dlogits = cross_entropy(fw["logits"], np.asarray(labels))
     grads = {}
@@ -467,7 +482,7 @@ def train_step(cfg, params, images, labels, task_ids=None, forced_keep=None, opt
     fw.pop("caches")
     return {"loss": loss, "logits": fw["logits"], "grads": grads, "params": new_params,
             "opt_state": {"m": new_m, "v": new_v}, "kept": fw["kept"], "margins": fw["margins"],
-            "scores": fw["scores"], "tokens": fw["tokens"]}
+            "scores": fw["scores"], "tokens": fw["tokens"], "routing": fw["routing"]}
 
 
 def gather_fuse(xp, kept, dropped, s, fuse_mode=1):

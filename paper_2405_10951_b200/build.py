@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbsr.so")
-SOURCES = ["engine.cu", "kernels_basic.cu", "kernels_select.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_tc2.cu", "attention_simt.cu", "attention_tc.cu", "noalloc.cu"]
+SOURCES = ["engine.cu", "kernels_basic.cu", "kernels_select.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_tc2.cu", "attention_simt.cu", "attention_tc.cu", "moe.cu", "noalloc.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC",
          "--expt-relaxed-constexpr"]
 

@@ -40,6 +40,8 @@ struct BlockBufs {          // byte offsets into the workspace; filled for froze
   size_t x_in, y1, qkv, o, xp_full, xp, y2, z, hh, x_out;
   size_t mean1, rstd1, lse, mean2, rstd2, p, s, kept, dropped;
   size_t o_cls, xin_cls;    // classification rows of o and of the block input (last block only)
+  // MoE blocks: routing tables and expert-ordered buffers
+  size_t m_eidx, m_ew, m_pos, m_row_token, m_row_w, m_seg, m_tile, m_cnt, m_off, m_xg, m_zg, m_hg, m_og;
 };
 
 struct Bump {
@@ -111,7 +113,13 @@ int validate(const bsr_config* cfg, char* err) {
   int rc = compute_schedule(cfg, &s, err);
   if (rc != BSR_OK) return rc;
   if (d.depth < 32 && (cfg->trainable_mask >> d.depth) != 0) return set_err(err, BSR_ERR_INVALID_ARG, "trainable_mask names a block beyond depth");
-  if (d.moe_experts != 0 || d.moe_block_mask != 0) return set_err(err, BSR_ERR_UNSUPPORTED, "MoE layers are not built yet");
+  if (d.moe_block_mask != 0) {
+    if (d.depth < 32 && (d.moe_block_mask >> d.depth) != 0) return set_err(err, BSR_ERR_INVALID_ARG, "moe_block_mask names a block beyond depth");
+    if (d.moe_experts < 1 || d.moe_experts > 32 || d.moe_top_k < 1 || d.moe_top_k > 4 || d.moe_top_k > d.moe_experts)
+      return set_err(err, BSR_ERR_INVALID_ARG, "MoE needs 1 <= experts <= 32 and 1 <= top_k <= min(4, experts)");
+    if (d.dtype != BSR_DTYPE_BF16) return set_err(err, BSR_ERR_UNSUPPORTED, "MoE layers run on the bf16 tensor-core kernels only");
+    if (d.dim % 64 != 0 || d.mlp_hidden % 64 != 0) return set_err(err, BSR_ERR_UNSUPPORTED, "MoE layers need dim and mlp_hidden to be multiples of 64");
+  }
   // trainable set must be "the last k blocks"
   uint32_t m = cfg->trainable_mask;
   if (m != 0) {
@@ -157,6 +165,8 @@ struct bsr_handle {
   size_t off_kept_all = 0;
   size_t off_stage = 0;
   size_t off_split = 0, split_floats = 0;
+  std::vector<size_t> moe_rec_eidx, moe_rec_ew;
+  size_t off_m_dog = 0, off_m_dzg = 0, off_m_dxg = 0, off_m_dw = 0, off_m_dsel = 0;
   GemmProfile prof;
   long launches_at_enable = 0;
 
@@ -201,10 +211,19 @@ void build_tensors(bsr_handle* h) {
     add(p + "attn.proj.bias", D, false, tr);
     add(p + "norm2.weight", D, false, tr);
     add(p + "norm2.bias", D, false, tr);
-    add(p + "mlp.fc1.weight", (size_t)F * D, true, tr);
-    add(p + "mlp.fc1.bias", F, false, tr);
-    add(p + "mlp.fc2.weight", (size_t)D * F, true, tr);
-    add(p + "mlp.fc2.bias", D, false, tr);
+    if ((d.moe_block_mask >> l) & 1u) {
+      size_t E = d.moe_experts;
+      add(p + "moe.gate.weight", (size_t)d.num_tasks * E * D, true, tr);
+      add(p + "moe.fc1.weight", E * F * D, true, tr);
+      add(p + "moe.fc1.bias", E * F, false, tr);
+      add(p + "moe.fc2.weight", E * D * F, true, tr);
+      add(p + "moe.fc2.bias", E * D, false, tr);
+    } else {
+      add(p + "mlp.fc1.weight", (size_t)F * D, true, tr);
+      add(p + "mlp.fc1.bias", F, false, tr);
+      add(p + "mlp.fc2.weight", (size_t)D * F, true, tr);
+      add(p + "mlp.fc2.bias", D, false, tr);
+    }
   }
   add("norm.weight", D, false, true);
   add("norm.bias", D, false, true);
@@ -253,6 +272,33 @@ size_t plan(bsr_handle* h) {
     if (t.trainable) nch += (int)((t.numel + ADAM_CHUNK - 1) / ADAM_CHUNK);
   h->n_chunks = nch;
   h->off_chunks = b.take((size_t)nch * sizeof(AdamChunk));
+  // routing record of every MoE block (kept for inspection), then the activations kept by the trainable blocks
+  int E = d.moe_experts, Kx = d.moe_top_k;
+  std::vector<size_t> rec_eidx(d.depth, 0), rec_ew(d.depth, 0);
+  for (int l = 0; l < d.depth; ++l)
+    if ((d.moe_block_mask >> l) & 1u) {
+      rec_eidx[l] = b.take((size_t)Bm * s.tf[l] * Kx * 4);
+      rec_ew[l] = b.take((size_t)Bm * s.tf[l] * Kx * 4);
+    }
+  auto take_moe = [&](BlockBufs& bb, int l, size_t tokens_ffn) {
+    size_t M = (size_t)Bm * tokens_ffn;
+    size_t cap = (size_t)moe_rows_cap((int)M, E, Kx);
+    bb.m_eidx = rec_eidx[l];
+    bb.m_ew = rec_ew[l];
+    bb.m_pos = b.take(M * Kx * 4);
+    bb.m_row_token = b.take(cap * 4);
+    bb.m_row_w = b.take(cap * 4);
+    bb.m_seg = b.take((size_t)(E + 1) * 4);
+    bb.m_tile = b.take((cap / 128) * 4);
+    bb.m_cnt = b.take((size_t)moe_blocks((int)M) * E * 4);
+    bb.m_off = b.take((size_t)moe_blocks((int)M) * E * 4);
+    bb.m_xg = b.take(cap * D * es);
+    bb.m_zg = b.take(cap * F * es);
+    bb.m_hg = b.take(cap * F * es);
+    bb.m_og = b.take(cap * D * es);
+  };
+  h->moe_rec_eidx = rec_eidx;
+  h->moe_rec_ew = rec_ew;
   // activations kept by the trainable blocks
   size_t a0 = b.off;
   h->bufs_train.assign(d.depth, BlockBufs());
@@ -283,6 +329,7 @@ size_t plan(bsr_handle* h) {
     bb.x_out = b.take(Mf * D * 4);
     bb.o_cls = b.take((size_t)Bm * D * es);
     bb.xin_cls = b.take((size_t)Bm * D * 4);
+    if ((d.moe_block_mask >> l) & 1u) take_moe(bb, l, s.tf[l]);
     next_in = bb.x_out;
   }
   h->arena_bytes = b.off - a0;
@@ -314,6 +361,7 @@ size_t plan(bsr_handle* h) {
     bb.dropped = b.take((size_t)Bm * (T0 - 1) * 4);
     bb.o_cls = b.take((size_t)Bm * D * es);
     bb.xin_cls = b.take((size_t)Bm * D * 4);
+    if (d.moe_block_mask != 0) take_moe(bb, 0, T0);          // frozen MoE blocks share one set sized for the longest sequence
     size_t in1 = h->bufs_frozen[1].x_in, out1 = h->bufs_frozen[1].x_out;
     h->bufs_frozen[1] = bb;
     h->bufs_frozen[1].x_in = in1;
@@ -348,6 +396,14 @@ size_t plan(bsr_handle* h) {
     h->off_dqkv = b.take(Mt * 3 * D * es);
     h->off_escore = b.take((size_t)Bm * s.ta[h->t0] * 4);
     h->off_delta = b.take((size_t)Bm * H * s.ta[h->t0] * 4);
+  }
+  if (d.moe_block_mask != 0 && h->t0 < d.depth) {
+    size_t cap = (size_t)moe_rows_cap(Bm * s.tf[h->t0], E, Kx);
+    h->off_m_dog = b.take(cap * D * es);
+    h->off_m_dzg = b.take(cap * F * es);
+    h->off_m_dxg = b.take(cap * D * es);
+    h->off_m_dw = b.take(cap * 4);
+    h->off_m_dsel = b.take(cap * 4);
   }
   int maxn = 3 * D > F ? 3 * D : F;
   h->off_ln_partials = b.take((size_t)2 * 512 * D * 4);
@@ -386,7 +442,19 @@ int check_cuda(bsr_handle* h, const char* what) {
 bool cls_tail(const bsr_handle* h, int l) { return l == h->cfg.dims.depth - 1 && h->sched.k[l] < 0; }
 
 // One encoder block forward.  `save` keeps the statistics and pre-activations the backward pass needs.
-int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb, bool save, int* kept_out) {
+bool is_moe(const bsr_handle* h, int l) { return (h->cfg.dims.moe_block_mask >> l) & 1u; }
+
+MoeBufs moe_bufs(const bsr_handle* h, const BlockBufs& bb) {
+  MoeBufs m;
+  m.eidx = h->at<int>(bb.m_eidx); m.ew = h->at<float>(bb.m_ew); m.pos = h->at<int>(bb.m_pos);
+  m.row_token = h->at<int>(bb.m_row_token); m.row_w = h->at<float>(bb.m_row_w);
+  m.seg_start = h->at<int>(bb.m_seg); m.tile_expert = h->at<int>(bb.m_tile);
+  m.blk_counts = h->at<int>(bb.m_cnt); m.blk_off = h->at<int>(bb.m_off);
+  m.xg = h->base + bb.m_xg; m.zg = h->base + bb.m_zg; m.hg = h->base + bb.m_hg; m.og = h->base + bb.m_og;
+  return m;
+}
+
+int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb, bool save, int* kept_out, const int* task_ids) {
   const bsr_dims& d = h->cfg.dims;
   const Schedule& s = h->sched;
   int D = d.dim, F = d.mlp_hidden, H = d.heads, hd = D / H;
@@ -432,6 +500,24 @@ int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb
   }
   layernorm_fwd(c, h->at<float>(bb.xp), D, (const float*)h->wb(l, "norm2.weight"), (const float*)h->wb(l, "norm2.bias"),
                 h->base + bb.y2, 0, save ? h->at<float>(bb.mean2) : nullptr, save ? h->at<float>(bb.rstd2) : nullptr, Mf, D, d.ln_eps);
+  if (is_moe(h, l)) {
+    // MoE layer in place of the FFN (Section 5.2): route, run the chosen experts as grouped GEMMs, combine
+    int E = d.moe_experts, K = d.moe_top_k;
+    MoeBufs mb = moe_bufs(h, bb);
+    moe_route(c, mb, h->base + bb.y2, h->wb(l, "moe.gate.weight"), task_ids, tail ? 1 : Tf, Mf, D, E, K);
+    int cap = moe_rows_cap(Mf, E, K);
+    GemmEpilogue m1;
+    m1.bias = (const float*)h->wb(l, "moe.fc1.bias");
+    m1.act = 1;
+    m1.aux_out = save ? mb.zg : nullptr;
+    int rc1 = gemm_tc_grouped_rows(c, mb.xg, h->wb(l, "moe.fc1.weight"), 0, mb.hg, cap, F, D, E, mb.tile_expert, m1);
+    GemmEpilogue m2;
+    m2.bias = (const float*)h->wb(l, "moe.fc2.bias");
+    int rc2 = gemm_tc_grouped_rows(c, mb.hg, h->wb(l, "moe.fc2.weight"), 0, mb.og, cap, D, F, E, mb.tile_expert, m2);
+    if (rc1 != 0 || rc2 != 0) return set_err(h->err, BSR_ERR_CUDA, "grouped GEMM set-up failed (%d, %d)", rc1, rc2);
+    moe_combine(c, mb, h->at<float>(bb.xp), h->at<float>(bb.x_out), Mf, D, K);
+    return BSR_OK;
+  }
   GemmEpilogue e3;
   e3.bias = (const float*)h->wb(l, "mlp.fc1.bias");
   e3.act = 1;
@@ -451,7 +537,7 @@ struct GradStream {      // gradient of the residual stream: float rows, plus th
   void* c;
 };
 
-int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, GradStream dxi, bool need_dxi) {
+int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, GradStream dxi, bool need_dxi, const int* task_ids) {
   const bsr_dims& d = h->cfg.dims;
   const Schedule& s = h->sched;
   const BlockBufs& bb = h->bufs_train[l];
@@ -476,6 +562,28 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
   void* dqkv = h->base + h->off_dqkv;
   auto op = [&](const GradStream& g) -> const void* { return bf ? g.c : (const void*)g.f; };   // GEMM operand view
   GemmEpilogue none;
+  if (is_moe(h, l)) {
+    int E = d.moe_experts, K = d.moe_top_k;
+    MoeBufs mb = moe_bufs(h, bb);
+    int cap = moe_rows_cap(Mf, E, K);
+    void* dog = h->base + h->off_m_dog;
+    void* dzg = h->base + h->off_m_dzg;
+    void* dxg = h->base + h->off_m_dxg;
+    float* dwsel = h->at<float>(h->off_m_dw);
+    moe_combine_bwd(c, mb, dxo.f, dog, dwsel, Mf, D, E, K);
+    GemmEpilogue eg;
+    eg.act = 2;
+    eg.aux_in = mb.zg;
+    int r1 = gemm_tc_grouped_rows(c, dog, h->wb(l, "moe.fc2.weight"), 1, dzg, cap, F, D, E, mb.tile_expert, eg);
+    int r2 = gemm_tc_grouped_wgrad(c, dog, mb.hg, h->gb(l, "moe.fc2.weight"), cap, D, F, E, mb.seg_start);
+    moe_seg_colsum(c, mb, dog, D, E, h->gb(l, "moe.fc2.bias"));
+    int r3 = gemm_tc_grouped_rows(c, dzg, h->wb(l, "moe.fc1.weight"), 1, dxg, cap, D, F, E, mb.tile_expert, none);
+    int r4 = gemm_tc_grouped_wgrad(c, dzg, mb.xg, h->gb(l, "moe.fc1.weight"), cap, F, D, E, mb.seg_start);
+    moe_seg_colsum(c, mb, dzg, F, E, h->gb(l, "moe.fc1.bias"));
+    if (r1 || r2 || r3 || r4) return set_err(h->err, BSR_ERR_CUDA, "grouped GEMM set-up failed (%d, %d, %d, %d)", r1, r2, r3, r4);
+    moe_gate_bwd(c, mb, dxg, dwsel, h->wb(l, "moe.gate.weight"), task_ids, tail ? 1 : Tf, d.num_tasks, Mf, D, E, K, dy,
+                 h->at<float>(h->off_m_dsel), h->gb(l, "moe.gate.weight"));
+  } else {
   // FFN second layer: dz = (dxo W2) * GELU'(z); dW2 = dxo^T h; db2 = column sums of dxo
   GemmEpilogue eg;
   eg.act = 2;
@@ -487,6 +595,7 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
   gemm(c, dz, F, 1, h->wb(l, "mlp.fc1.weight"), 1, D, dy, 0, Mf, D, F, none);
   gemm(c, dz, 1, F, h->base + bb.y2, 1, D, h->gb(l, "mlp.fc1.weight"), 1, F, D, Mf, none);
   colsum(c, dz, Mf, F, csp, h->gb(l, "mlp.fc1.bias"));
+  }
   layernorm_bwd(c, dy, 0, h->at<float>(bb.xp), D, h->at<float>(bb.mean2), h->at<float>(bb.rstd2),
                 (const float*)h->wb(l, "norm2.weight"), dxo.f, dxg.f, D, shrinks ? nullptr : dxg.c, lnp,
                 h->gb(l, "norm2.weight"), h->gb(l, "norm2.bias"), Mf, D);
@@ -548,7 +657,7 @@ HeadDesc head_desc(bsr_handle* h) {
 }
 
 // Forward through all blocks.  train: blocks >= t0 write the activation arena.  Returns the offset of the last output.
-int forward_all(bsr_handle* h, const Ctx& c, const void* images, int B, bool train, size_t* x_last_off) {
+int forward_all(bsr_handle* h, const Ctx& c, const void* images, int B, bool train, size_t* x_last_off, const int* task_ids) {
   const bsr_dims& d = h->cfg.dims;
   int D = d.dim;
   int g = d.image_size / d.patch_size, N = g * g;
@@ -573,9 +682,10 @@ int forward_all(bsr_handle* h, const Ctx& c, const void* images, int B, bool tra
       if (l + 1 == first_train && first_train < d.depth) bb.x_out = h->bufs_train[l + 1].x_in;   // hand over to the first trainable block
     }
     bb.x_in = cur;
+    if (is_moe(h, l)) { bb.m_eidx = h->moe_rec_eidx[l]; bb.m_ew = h->moe_rec_ew[l]; }
     int* kept_dst = nullptr;
     if (h->sched.k[l] >= 0) { kept_dst = kept_all + kept_off; kept_off += (size_t)B * h->sched.k[l]; }
-    int rc = block_forward(h, c, l, B, bb, save, kept_dst);
+    int rc = block_forward(h, c, l, B, bb, save, kept_dst, task_ids);
     if (rc != BSR_OK) return rc;
     cur = bb.x_out;
   }
@@ -725,6 +835,11 @@ int32_t bsr_get_tensor(bsr_handle* h, const char* name, float* dst, size_t count
     int cmax = 0;
     for (int t = 0; t < h->cfg.dims.num_tasks; ++t) cmax = h->cfg.dims.num_classes[t] > cmax ? h->cfg.dims.num_classes[t] : cmax;
     src = h->at<float>(h->off_logits); numel = (size_t)h->cfg.max_batch * cmax;
+  } else if (n.rfind("moe_experts/", 0) == 0) {
+    int l = atoi(n.c_str() + 12);
+    if (l < 0 || l >= h->cfg.dims.depth || !is_moe(h, l)) return set_err(h->err, BSR_ERR_INVALID_ARG, "'%s': not an MoE block", name);
+    convert_int_to_float(c.stream, h->at<int>(h->moe_rec_eidx[l]), dst, count);
+    return check_cuda(h, "bsr_get_tensor");
   } else {
     size_t base_off = 0;
     std::string pn = n;
@@ -778,7 +893,7 @@ int32_t bsr_train_step(bsr_handle* h, const void* images, const int32_t* labels,
   int D = d.dim, B = batch;
   size_t es = dtype_size(d.dtype);
   size_t x_last = 0;
-  rc = forward_all(h, c, images, B, true, &x_last);
+  rc = forward_all(h, c, images, B, true, &x_last, task_ids);
   if (rc != BSR_OK) return rc;
   int Tl = cls_tail(h, d.depth - 1) ? 1 : h->sched.tf[d.depth - 1];   // rows per image in the last block's output
   HeadDesc hd = head_desc(h);
@@ -804,7 +919,7 @@ int32_t bsr_train_step(bsr_handle* h, const void* images, const int32_t* labels,
     layernorm_bwd(c, h->at<float>(h->off_dxn), 1, h->at<float>(x_last), (long)Tl * D, h->at<float>(h->off_meanf), h->at<float>(h->off_rstdf),
                   (const float*)h->w("norm.weight"), nullptr, dxo.f, (long)Tl * D, dxo.c, lnp, h->gradp("norm.weight"), h->gradp("norm.bias"), B, D);
     for (int l = d.depth - 1; l >= h->t0; --l) {
-      rc = block_backward(h, c, l, B, dxo, dxi, l > h->t0);
+      rc = block_backward(h, c, l, B, dxo, dxi, l > h->t0, task_ids);
       if (rc != BSR_OK) return rc;
       GradStream t = dxo; dxo = dxi; dxi = t;
     }
@@ -830,7 +945,7 @@ int32_t bsr_eval_forward(bsr_handle* h, const void* images, const int32_t* task_
   const bsr_dims& d = h->cfg.dims;
   Ctx c = make_ctx(h, stream);
   size_t x_last = 0;
-  rc = forward_all(h, c, images, batch, false, &x_last);
+  rc = forward_all(h, c, images, batch, false, &x_last, task_ids);
   if (rc != BSR_OK) return rc;
   int Tl = cls_tail(h, d.depth - 1) ? 1 : h->sched.tf[d.depth - 1];   // rows per image in the last block's output
   HeadDesc hd = head_desc(h);

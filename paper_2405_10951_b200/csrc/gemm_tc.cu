@@ -45,10 +45,42 @@ __host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn) {
          ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
 
+// One unit of work of the persistent loop, decoded identically by the three roles.
+struct Work {
+  int mt, nt, kb0, kb1, b_off, bias_off;
+  size_t c_off;
+  bool active;
+};
+__device__ __forceinline__ Work decode_work(int w, int tiles_m, int tiles_n, int total_kb, int kb_per_split, const GemmGroup& g,
+                                            size_t mn) {
+  Work k;
+  k.nt = w % tiles_n;
+  k.mt = (w / tiles_n) % tiles_m;
+  int sp = w / (tiles_m * tiles_n);
+  k.b_off = 0; k.bias_off = 0; k.active = true;
+  if (g.mode == 0) {                       // plain (optionally split along k)
+    k.kb0 = sp * kb_per_split;
+    k.kb1 = min(total_kb, k.kb0 + kb_per_split);
+    k.c_off = (size_t)sp * mn;
+  } else if (g.mode == 1) {                // rows grouped by expert: the tile's expert picks the weight slice
+    int e = g.tile_expert[k.mt];
+    k.active = e >= 0;
+    k.kb0 = 0; k.kb1 = total_kb;
+    k.b_off = e * g.b_stride;
+    k.bias_off = e * g.bias_stride;
+    k.c_off = 0;
+  } else {                                 // weight gradients per expert: reduce over the expert's row segment
+    k.kb0 = g.seg_start[sp] / BK;
+    k.kb1 = g.seg_start[sp + 1] / BK;
+    k.c_off = (size_t)sp * (size_t)g.c_stride;
+  }
+  return k;
+}
+
 template <bool A_MN, bool B_MN, typename TOut>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TOut* __restrict__ C,
-               int M, int N, int K, Epi ep, int tiles_m, int tiles_n, int splits, int kb_per_split, int* status) {
+               int M, int N, int K, Epi ep, int tiles_m, int tiles_n, int splits, int kb_per_split, GemmGroup grp, int* status) {
   extern __shared__ unsigned char smem_dyn[];
   uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   uint32_t staging0 = base + STAGES * STAGE_BYTES;
@@ -87,9 +119,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int armed = 0;
       bool ok = true;
       for (int w = blockIdx.x; w < work_items && ok; w += gridDim.x) {
-        int nt = w % tiles_n, mt = (w / tiles_n) % tiles_m, sp = w / (tiles_m * tiles_n);
-        int kb0 = sp * kb_per_split, kb1 = min(total_kb, kb0 + kb_per_split);
-        for (int kb = kb0; kb < kb1; ++kb) {
+        Work wk = decode_work(w, tiles_m, tiles_n, total_kb, kb_per_split, grp, (size_t)M * N);
+        if (!wk.active) continue;
+        int nt = wk.nt, mt = wk.mt;
+        for (int kb = wk.kb0; kb < wk.kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abortp)) { ok = false; break; }
           mbar_expect_tx(full_bar(stage), STAGE_BYTES);
           uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
@@ -100,10 +133,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int j = 0; j < BM / 64; ++j) tma_load_2d(sa + j * (BK * 128), &map_a, full_bar(stage), mt * BM + j * 64, kb * BK);
           }
           if (!B_MN) {
-            tma_load_2d(sb, &map_b, full_bar(stage), kb * BK, nt * BN);
+            tma_load_2d(sb, &map_b, full_bar(stage), kb * BK, nt * BN + wk.b_off);
           } else {
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * (BK * 128), &map_b, full_bar(stage), nt * BN + j * 64, kb * BK);
+            for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * (BK * 128), &map_b, full_bar(stage), nt * BN + j * 64, kb * BK + wk.b_off);
           }
           ++armed;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -123,9 +156,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       uint32_t phase = 0;
       int local = 0;
       bool ok = true;
-      for (int w = blockIdx.x; w < work_items && ok; w += gridDim.x, ++local) {
-        int sp = w / (tiles_m * tiles_n);
-        int kb0 = sp * kb_per_split, kb1 = min(total_kb, kb0 + kb_per_split);
+      for (int w = blockIdx.x; w < work_items && ok; w += gridDim.x) {
+        Work wk = decode_work(w, tiles_m, tiles_n, total_kb, kb_per_split, grp, (size_t)M * N);
+        if (!wk.active) continue;
+        int kb0 = wk.kb0, kb1 = wk.kb1;
         int buf = local & 1;
         if (!mbar_wait(tempty_bar(buf), ((local >> 1) & 1) ^ 1u, abortp)) { ok = false; break; }
         tc_fence_after();
@@ -144,6 +178,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (ok) umma_commit(tfull_bar(buf));
+        ++local;
       }
     }
   } else {
@@ -154,15 +189,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     unsigned char* st = smem_dyn + (staging0 - smem_u32(smem_dyn)) + ew * STAGING_BYTES;
     int local = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < work_items && ok; w += gridDim.x, ++local) {
-      int nt = w % tiles_n, mt = (w / tiles_n) % tiles_m, sp = w / (tiles_m * tiles_n);
+    for (int w = blockIdx.x; w < work_items && ok; w += gridDim.x) {
+      Work wk = decode_work(w, tiles_m, tiles_n, total_kb, kb_per_split, grp, (size_t)M * N);
+      if (!wk.active) continue;
+      int nt = wk.nt, mt = wk.mt;
       int buf = local & 1;
+      Epi epw = ep;
+      if (epw.bias != nullptr) epw.bias += wk.bias_off;
+      bool empty = wk.kb0 >= wk.kb1;          // an expert without tokens: its gradient tile is zero
       ok = mbar_wait(tfull_bar(buf), (local >> 1) & 1, abortp);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       int row0 = mt * BM + quarter * 32;
-      TOut* Cs = C + (size_t)sp * M * N;
+      TOut* Cs = C + wk.c_off;
 #pragma unroll 1
       for (int cc = 0; cc < 4; ++cc) {
         int cchunk = chalf * 4 + cc;
@@ -170,11 +210,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cchunk * 32);
         tmem_ld32(taddr, r);
         tmem_ld_wait();
-        epilogue_chunk<TOut>(r, ep, Cs, M, N, row0, nt * BN + cchunk * 32, st, lane);
+        if (empty) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) r[j] = 0u;
+        }
+        epilogue_chunk<TOut>(r, epw, Cs, M, N, row0, nt * BN + cchunk * 32, st, lane);
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(buf));
+      ++local;
     }
   }
   tc_fence_before();
@@ -225,7 +270,7 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t outer,
 
 template <bool A_MN, bool B_MN, typename TOut>
 static int launch(const Ctx& c, const CUtensorMap& ma, const CUtensorMap& mb, void* C, int m, int n, int k, const Epi& ep,
-                  int tiles_m, int tiles_n, int splits, int kb_per_split) {
+                  int tiles_m, int tiles_n, int splits, int kb_per_split, const GemmGroup& grp) {
   auto kern = gemm_tc_kernel<A_MN, B_MN, TOut>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -236,7 +281,7 @@ static int launch(const Ctx& c, const CUtensorMap& ma, const CUtensorMap& mb, vo
   int sms = c.sm_count > 0 ? c.sm_count : 148;
   int grid = work < sms ? work : sms;
   note_launch(1);
-  kern<<<grid, THREADS, SMEM_BYTES, c.stream>>>(ma, mb, (TOut*)C, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, c.status);
+  kern<<<grid, THREADS, SMEM_BYTES, c.stream>>>(ma, mb, (TOut*)C, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, grp, c.status);
   return 0;
 }
 
@@ -285,13 +330,13 @@ int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const voi
   if (c.prof != nullptr && c.prof->on) c.prof->begin(c.stream, 2.0 * m * n * (double)k);
   int rc;
   if (out_is_float) {
-    if (a_mn) rc = launch<true, true, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split);
-    else if (b_mn) rc = launch<false, true, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split);
-    else rc = launch<false, false, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split);
+    if (a_mn) rc = launch<true, true, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, GemmGroup());
+    else if (b_mn) rc = launch<false, true, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, GemmGroup());
+    else rc = launch<false, false, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, GemmGroup());
   } else {
-    if (a_mn) rc = launch<true, true, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split);
-    else if (b_mn) rc = launch<false, true, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split);
-    else rc = launch<false, false, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split);
+    if (a_mn) rc = launch<true, true, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, GemmGroup());
+    else if (b_mn) rc = launch<false, true, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, GemmGroup());
+    else rc = launch<false, false, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, GemmGroup());
   }
   if (rc != 0) return rc;
   if (splits > 1) {
@@ -300,6 +345,50 @@ int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const voi
   }
   if (c.prof != nullptr && c.prof->on) c.prof->end(c.stream);
   return 0;
+}
+
+// Expert-grouped contractions of the MoE layer (paper Section 5.2); see kernels.h.
+int gemm_tc_grouped_rows(const Ctx& c, const void* A, const void* Bst, int b_mn, void* C, int rows_cap, int n, int k, int experts,
+                         const int* tile_expert, const GemmEpilogue& e) {
+  using namespace tc;
+  if ((n % 8) || (k % 8) || (rows_cap % BM) || ((uintptr_t)A & 15) || ((uintptr_t)Bst & 15) || ((uintptr_t)C & 15)) return -1;
+  if (b_mn && (k % BK)) return -1;             // a k-slab must not straddle two experts' weights
+  CUtensorMap ma, mb;
+  bool ok = make_map(&ma, A, (uint64_t)k, (uint64_t)rows_cap, (uint64_t)k, BM);
+  ok = ok && (b_mn ? make_map(&mb, Bst, (uint64_t)n, (uint64_t)experts * k, (uint64_t)n, BK)
+                   : make_map(&mb, Bst, (uint64_t)k, (uint64_t)experts * n, (uint64_t)k, BN));
+  if (!ok) return -2;
+  GemmGroup g;
+  g.mode = 1;
+  g.tile_expert = tile_expert;
+  g.b_stride = b_mn ? k : n;
+  g.bias_stride = n;
+  Epi ep;
+  ep.bias = e.bias; ep.residual = e.residual; ep.aux_out = e.aux_out; ep.aux_in = e.aux_in; ep.act = e.act;
+  int tiles_m = rows_cap / BM, tiles_n = ceil_div(n, BN);
+  if (c.prof != nullptr && c.prof->on) c.prof->begin(c.stream, 2.0 * rows_cap * n * (double)k);
+  int rc = b_mn ? launch<false, true, bf16>(c, ma, mb, C, rows_cap, n, k, ep, tiles_m, tiles_n, 1, ceil_div(k, BK), g)
+                : launch<false, false, bf16>(c, ma, mb, C, rows_cap, n, k, ep, tiles_m, tiles_n, 1, ceil_div(k, BK), g);
+  if (c.prof != nullptr && c.prof->on) c.prof->end(c.stream);
+  return rc;
+}
+
+int gemm_tc_grouped_wgrad(const Ctx& c, const void* dY, const void* X, float* dW, int rows_cap, int m, int n, int experts,
+                          const int* seg_start) {
+  using namespace tc;
+  if ((m % 8) || (n % 8) || (rows_cap % BM) || ((uintptr_t)dY & 15) || ((uintptr_t)X & 15) || ((uintptr_t)dW & 15)) return -1;
+  CUtensorMap ma, mb;
+  if (!make_map(&ma, dY, (uint64_t)m, (uint64_t)rows_cap, (uint64_t)m, BK) || !make_map(&mb, X, (uint64_t)n, (uint64_t)rows_cap, (uint64_t)n, BK)) return -2;
+  GemmGroup g;
+  g.mode = 2;
+  g.seg_start = seg_start;
+  g.c_stride = (long)m * n;
+  Epi ep;
+  ep.bias = nullptr; ep.residual = nullptr; ep.aux_out = nullptr; ep.aux_in = nullptr; ep.act = 0;
+  if (c.prof != nullptr && c.prof->on) c.prof->begin(c.stream, 2.0 * rows_cap * n * (double)m);
+  int rc = launch<true, true, float>(c, ma, mb, dW, m, n, rows_cap, ep, ceil_div(m, BM), ceil_div(n, BN), experts, 0, g);
+  if (c.prof != nullptr && c.prof->on) c.prof->end(c.stream);
+  return rc;
 }
 
 int gemm_tc(const Ctx& c, const void* A, const void* B, void* C, int out_is_float, int m, int n, int k, const GemmEpilogue& e) {

@@ -73,6 +73,19 @@ int colsum_groups(int rows);
 
 // ---- dense contractions -----------------------------------------------------------------------
 // C[m, n] = epilogue(sum_k A(m, k) * B(n, k)).  A(m,k) = A[m * a_rs + k * a_cs], B alike.
+// Expert grouping of a contraction (MoE layer).  mode 0: none.  mode 1: every 128-row tile of A / C belongs to one
+// expert (tile_expert[tile], -1 = unused tile) whose slice of the stacked weights and biases is used.  mode 2:
+// weight gradients, one output matrix per expert, reduced over that expert's row segment (seg_start[e] ..
+// seg_start[e+1], multiples of 128).
+struct GemmGroup {
+  const int* tile_expert = nullptr;
+  const int* seg_start = nullptr;
+  int mode = 0;
+  int b_stride = 0;
+  int bias_stride = 0;
+  long c_stride = 0;
+};
+
 struct GemmEpilogue {
   const float* bias = nullptr;      // [n]
   const void* residual = nullptr;   // [m, n] in the output type, added last
@@ -91,6 +104,13 @@ int gemm_tc(const Ctx& c, const void* A, const void* B, void* C, int out_is_floa
 int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long b_rs, long b_cs, void* C,
                     int out_is_float, int m, int n, int k, const GemmEpilogue& e, float* split_ws, size_t split_ws_floats);
 
+// C[rows_cap, n] = epilogue(A[rows_cap, k] . W_e) with W_e the expert's slice of stacked weights: Bst [E*n, k]
+// (b_mn = 0, forward) or [E*k, n] (b_mn = 1, input gradient: C = A W_e).  bf16 in and out; e.bias stacked [E*n].
+int gemm_tc_grouped_rows(const Ctx& c, const void* A, const void* Bst, int b_mn, void* C, int rows_cap, int n, int k, int experts,
+                         const int* tile_expert, const GemmEpilogue& e);
+// dW[e][m, n] = sum over rows r of expert e's segment of dY[r, m] * X[r, n]  (float out).
+int gemm_tc_grouped_wgrad(const Ctx& c, const void* dY, const void* X, float* dW, int rows_cap, int m, int n, int experts,
+                          const int* seg_start);
 // The same on CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles); preferred when m > 128.
 int gemm_tc2_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long b_rs, long b_cs, void* C,
                      int out_is_float, int m, int n, int k, const GemmEpilogue& e, float* split_ws, size_t split_ws_floats);
@@ -140,9 +160,37 @@ void adamw(const Ctx& c, const AdamChunk* chunks, int nchunks, float* master, co
 // dst row r = src row r (row_bytes a multiple of 16), independent pitches: gathers / scatters token rows.
 void copy_rows(cudaStream_t s, const void* src, long src_pitch_bytes, void* dst, long dst_pitch_bytes, int rows, int row_bytes);
 
+// ---- mixture of experts (routing, grouping, combination; the expert MLPs are grouped GEMMs) -----------------------
+struct MoeBufs {
+  int* eidx;          // [M, K] chosen experts per token, best first
+  float* ew;          // [M, K] their weights (softmax over the chosen gate logits)
+  int* pos;           // [M, K] row of each (token, slot) in the expert-ordered buffers
+  int* row_token;     // [rows_cap] token of each row, -1 for padding
+  float* row_w;       // [rows_cap] weight of each row
+  int* seg_start;     // [E + 1] first row of each expert's segment (multiples of 128)
+  int* tile_expert;   // [rows_cap / 128] expert of each 128-row tile, -1 beyond the last segment
+  int* blk_counts;    // [blocks, E]
+  int* blk_off;       // [blocks, E]
+  void* xg;           // [rows_cap, D] gathered expert inputs
+  void* zg;           // [rows_cap, F] FC1 pre-activation (kept by trainable blocks)
+  void* hg;           // [rows_cap, F] GELU output
+  void* og;           // [rows_cap, D] expert outputs
+};
+int moe_rows_cap(int M, int E, int K);
+int moe_blocks(int M);
+// y [M, D]: routes every token, builds the segment tables and gathers the expert inputs into b.xg.
+void moe_route(const Ctx& c, const MoeBufs& b, const void* y, const void* wg, const int* task_ids, int tokens_per_image, int M,
+               int D, int E, int K);
+void moe_combine(const Ctx& c, const MoeBufs& b, const float* res, float* out, int M, int D, int K);
+void moe_combine_bwd(const Ctx& c, const MoeBufs& b, const float* dout, void* dog, float* dw, int M, int D, int E, int K);
+void moe_seg_colsum(const Ctx& c, const MoeBufs& b, const void* x, int cols, int E, float* out);
+void moe_gate_bwd(const Ctx& c, const MoeBufs& b, const void* dxg, const float* dw, const void* wg, const int* task_ids,
+                  int tokens_per_image, int tasks, int M, int D, int E, int K, void* dy, float* dsel_row, float* dwg);
+
 // ---- conversions ------------------------------------------------------------------------------
 void convert_from_float(const Ctx& c, const float* src, void* dst, size_t n);   // float -> storage dtype
 void convert_to_float(const Ctx& c, const void* src, float* dst, size_t n);     // storage dtype -> float
 void fill_float(cudaStream_t s, float* dst, float v, size_t n);
+void convert_int_to_float(cudaStream_t s, const int* src, float* dst, size_t n);
 
 }  // namespace bsr

@@ -595,6 +595,15 @@ void convert_to_float(const Ctx& c, const void* src, float* dst, size_t n) {
   if (c.dtype == 0) to_float_kernel<float><<<blocks, 256, 0, c.stream>>>((const float*)src, dst, n);
   else to_float_kernel<bf16><<<blocks, 256, 0, c.stream>>>((const bf16*)src, dst, n);
 }
+__global__ void int_to_float_kernel(const int* s, float* d, size_t n) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) d[i] = (float)s[i];
+}
+void convert_int_to_float(cudaStream_t st, const int* src, float* dst, size_t n) {
+  if (n == 0) return;
+  note_launch(1);
+  int_to_float_kernel<<<ceil_div((long)n, 256), 256, 0, st>>>(src, dst, n);
+}
 void fill_float(cudaStream_t s, float* dst, float v, size_t n) {
   note_launch(1);
   if (n == 0) return;

@@ -1,0 +1,360 @@
+// Mixture-of-experts FFN (paper Section 5.2): a task-dependent router picks the top-k of E expert MLPs per
+// token and adds their outputs, weighted by a softmax over the selected gate logits.  These are the routing,
+// grouping and combination kernels; the expert MLPs themselves run as expert-grouped tcgen05 GEMMs.
+//
+// Grouping.  Every (token, slot) pair becomes one row of an expert-ordered buffer: expert e owns rows
+// seg_start[e] .. seg_start[e] + count[e], padded with empty rows to a multiple of 128 so that a GEMM tile never
+// mixes experts.  Within an expert rows keep token order, and every reduction runs in row order: results do not
+// depend on scheduling.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace bsr {
+
+constexpr int MOE_BLOCK_TOKENS = 256;
+constexpr int MOE_MAX_E = 32;
+constexpr int MOE_MAX_K = 4;
+
+// ---- routing: gate logits, top-k (ties -> lower expert id), softmax over the selected logits -------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+moe_route_kernel(const T* __restrict__ y, const T* __restrict__ wg, const int* __restrict__ task_ids, int tokens_per_image,
+                 int M, int D, int E, int K, int* __restrict__ eidx, float* __restrict__ ew, int* __restrict__ blk_counts) {
+  __shared__ int counts[MOE_MAX_E];
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x < MOE_MAX_E) counts[threadIdx.x] = 0;
+  __syncthreads();
+  int t0 = blockIdx.x * MOE_BLOCK_TOKENS;
+  for (int tt = warp; tt < MOE_BLOCK_TOKENS; tt += 8) {
+    int tok = t0 + tt;
+    if (tok >= M) break;
+    int task = task_ids ? task_ids[tok / tokens_per_image] : 0;
+    const T* yr = y + (size_t)tok * D;
+    const T* wt = wg + (size_t)task * E * D;
+    float mine = -INFINITY;                       // lane e ends up with the logit of expert e
+    for (int e = 0; e < E; ++e) {
+      const T* we = wt + (size_t)e * D;
+      float s = 0.f;
+      for (int d = lane; d < D; d += 32) s = fmaf(to_f(yr[d]), to_f(we[d]), s);
+      s = warp_sum(s);
+      if (lane == e) mine = s;
+    }
+    float sel[MOE_MAX_K];
+    int sid[MOE_MAX_K];
+    bool taken = false;
+    for (int i = 0; i < K; ++i) {
+      float cand = taken ? -INFINITY : mine;
+      float mx = warp_max(cand);
+      uint32_t m = __ballot_sync(0xffffffffu, !taken && cand == mx && lane < E);
+      int win = __ffs(m) - 1;                     // lowest expert id among equals
+      sel[i] = mx;
+      sid[i] = win;
+      if (lane == win) taken = true;
+    }
+    float den = 0.f;
+    for (int i = 0; i < K; ++i) den += expf(sel[i] - sel[0]);
+    if (lane == 0) {
+      for (int i = 0; i < K; ++i) {
+        eidx[(size_t)tok * K + i] = sid[i];
+        ew[(size_t)tok * K + i] = expf(sel[i] - sel[0]) / den;
+        atomicAdd(&counts[sid[i]], 1);            // integer counts: order-independent
+      }
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < E) blk_counts[(size_t)blockIdx.x * E + threadIdx.x] = counts[threadIdx.x];
+}
+
+// ---- segment table: one warp per expert walks the token blocks in order ------------------------------------------
+__global__ void moe_scan_kernel(const int* __restrict__ blk_counts, int nblk, int E, int tiles_cap, int* __restrict__ blk_off,
+                                int* __restrict__ seg_start, int* __restrict__ tile_expert) {
+  __shared__ int total[MOE_MAX_E];
+  __shared__ int start[MOE_MAX_E + 1];
+  int e = threadIdx.x;
+  if (e < E) {
+    int run = 0;
+    for (int b = 0; b < nblk; ++b) {
+      blk_off[(size_t)b * E + e] = run;
+      run += blk_counts[(size_t)b * E + e];
+    }
+    total[e] = run;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int s = 0;
+    for (int i = 0; i < E; ++i) {
+      start[i] = s;
+      s += (total[i] + 127) & ~127;
+    }
+    start[E] = s;
+    for (int i = 0; i <= E; ++i) seg_start[i] = start[i];
+  }
+  __syncthreads();
+  for (int t = threadIdx.x; t < tiles_cap; t += blockDim.x) {
+    int row = t * 128, ex = -1;
+    for (int i = 0; i < E; ++i)
+      if (row >= start[i] && row < start[i + 1]) ex = i;
+    tile_expert[t] = ex;
+  }
+}
+
+// ---- row assignment: position of every (token, slot) inside its expert's segment, in token order ---------------
+__global__ void __launch_bounds__(256)
+moe_assign_kernel(const int* __restrict__ eidx, const float* __restrict__ ew, const int* __restrict__ blk_off,
+                  const int* __restrict__ seg_start, int M, int E, int K, int* __restrict__ pos, int* __restrict__ row_token,
+                  float* __restrict__ row_w) {
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int t0 = blockIdx.x * MOE_BLOCK_TOKENS;
+  int n_entries = min(MOE_BLOCK_TOKENS, M - t0) * K;
+  uint32_t lt = (1u << lane) - 1u;
+  for (int e = warp; e < E; e += 8) {
+    int base = seg_start[e] + blk_off[(size_t)blockIdx.x * E + e];
+    int run = 0;
+    for (int i0 = 0; i0 < n_entries; i0 += 32) {
+      int i = i0 + lane;
+      bool hit = i < n_entries && eidx[(size_t)t0 * K + i] == e;
+      uint32_t m = __ballot_sync(0xffffffffu, hit);
+      if (hit) {
+        int r = base + run + __popc(m & lt);
+        pos[(size_t)t0 * K + i] = r;
+        row_token[r] = t0 + i / K;
+        row_w[r] = ew[(size_t)t0 * K + i];
+      }
+      run += __popc(m);
+    }
+  }
+}
+
+// ---- gather the expert inputs: xg[r] = y[row_token[r]], empty rows are zero ---------------------------------------
+template <typename T>
+__global__ void moe_gather_kernel(const T* __restrict__ y, const int* __restrict__ row_token, const int* __restrict__ seg_start,
+                                  int E, int D, T* __restrict__ xg, int rows_cap) {
+  constexpr int N = Pack<T>::N;
+  int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= rows_cap || warp >= seg_start[E]) return;
+  int tok = row_token[warp];
+  for (int ch = lane; ch < D / N; ch += 32) {
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (tok >= 0) v = *reinterpret_cast<const uint4*>(y + (size_t)tok * D + ch * N);
+    *reinterpret_cast<uint4*>(xg + (size_t)warp * D + ch * N) = v;
+  }
+}
+
+// ---- combine: out[t] = res[t] + sum_slot w_slot * og[pos(t, slot)]  (float residual stream) ------------------------
+template <typename T>
+__global__ void moe_combine_kernel(const T* __restrict__ og, const int* __restrict__ pos, const float* __restrict__ ew,
+                                   const float* __restrict__ res, float* __restrict__ out, int M, int D, int K) {
+  int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= M) return;
+  for (int ch = lane; ch < D / 4; ch += 32) {
+    float acc[4];
+    load16(res + (size_t)warp * D + ch * 4, acc);
+    for (int s = 0; s < K; ++s) {
+      float w = ew[(size_t)warp * K + s];
+      float v[4];
+      load4(og + (size_t)pos[(size_t)warp * K + s] * D + ch * 4, v);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[j] = fmaf(w, v[j], acc[j]);
+    }
+    store16(out + (size_t)warp * D + ch * 4, acc);
+  }
+}
+
+// ---- backward of the combination: dog[r] = w_r * dout[token_r]; dw[r] = <dout[token_r], og[r]> ------------------
+template <typename T>
+__global__ void moe_combine_bwd_kernel(const float* __restrict__ dout, const T* __restrict__ og, const int* __restrict__ row_token,
+                                       const float* __restrict__ row_w, const int* __restrict__ seg_start, int E, int D,
+                                       T* __restrict__ dog, float* __restrict__ dw, int rows_cap) {
+  int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= rows_cap || warp >= seg_start[E]) return;
+  int tok = row_token[warp];
+  float w = tok >= 0 ? row_w[warp] : 0.f;
+  float dot = 0.f;
+  for (int ch = lane; ch < D / 4; ch += 32) {
+    float g[4] = {0.f, 0.f, 0.f, 0.f}, o[4], r[4];
+    if (tok >= 0) {
+      load16(dout + (size_t)tok * D + ch * 4, g);
+      load4(og + (size_t)warp * D + ch * 4, o);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) dot = fmaf(g[j], o[j], dot);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) r[j] = w * g[j];
+    store4(dog + (size_t)warp * D + ch * 4, r);
+  }
+  dot = warp_sum(dot);
+  if (lane == 0) dw[warp] = dot;
+}
+
+// ---- per-expert column sums (bias gradients): out[e][col] = sum over the expert's rows of x[r][col] -----------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+moe_seg_colsum_kernel(const T* __restrict__ x, const int* __restrict__ seg_start, int cols, float* __restrict__ out) {
+  constexpr int N = Pack<T>::N;
+  __shared__ float sm[8][32 * N];
+  int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  int e = blockIdx.y;
+  int col0 = (blockIdx.x * 32 + tx) * N;
+  float acc[N];
+#pragma unroll
+  for (int j = 0; j < N; ++j) acc[j] = 0.f;
+  if (col0 < cols) {
+    for (int r = seg_start[e] + ty; r < seg_start[e + 1]; r += 8) {
+      float v[N];
+      load16(x + (size_t)r * cols + col0, v);
+#pragma unroll
+      for (int j = 0; j < N; ++j) acc[j] += v[j];
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < N; ++j) sm[ty][tx * N + j] = acc[j];
+  __syncthreads();
+  for (int c = threadIdx.x; c < 32 * N; c += blockDim.x) {
+    int col = blockIdx.x * 32 * N + c;
+    if (col < cols) {
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) s += sm[w][c];
+      out[(size_t)e * cols + col] = s;
+    }
+  }
+}
+
+// ---- gate backward, token side: d(selected logits) and the gradient of the layer input -----------------------------
+//   dsel_s = w_s (dw_s - sum_u w_u dw_u);  dy[t] = sum_s dxg[pos_s] + sum_s dsel_s Wg[task][e_s]
+template <typename T>
+__global__ void moe_gate_bwd_kernel(const T* __restrict__ dxg, const float* __restrict__ dw, const int* __restrict__ pos,
+                                    const int* __restrict__ eidx, const float* __restrict__ ew, const T* __restrict__ wg,
+                                    const int* __restrict__ task_ids, int tokens_per_image, int M, int D, int E, int K,
+                                    T* __restrict__ dy, float* __restrict__ dsel_row) {
+  int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= M) return;
+  int task = task_ids ? task_ids[warp / tokens_per_image] : 0;
+  float w[MOE_MAX_K], d[MOE_MAX_K];
+  int p[MOE_MAX_K], ex[MOE_MAX_K];
+  float mean = 0.f;
+  for (int s = 0; s < K; ++s) {
+    p[s] = pos[(size_t)warp * K + s];
+    ex[s] = eidx[(size_t)warp * K + s];
+    w[s] = ew[(size_t)warp * K + s];
+    d[s] = dw[p[s]];
+    mean = fmaf(w[s], d[s], mean);
+  }
+  for (int s = 0; s < K; ++s) {
+    d[s] = w[s] * (d[s] - mean);
+    if (lane == 0) dsel_row[p[s]] = d[s];
+  }
+  for (int ch = lane; ch < D / 4; ch += 32) {
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int s = 0; s < K; ++s) {
+      float v[4], g[4];
+      load4(dxg + (size_t)p[s] * D + ch * 4, v);
+      load4(wg + ((size_t)task * E + ex[s]) * D + ch * 4, g);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[j] += v[j] + d[s] * g[j];
+    }
+    store4(dy + (size_t)warp * D + ch * 4, acc);
+  }
+}
+
+// ---- gate backward, weight side: dWg[task][e] = sum over expert e's rows of that task of dsel[r] * xg[r] --------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+moe_gate_wgrad_kernel(const T* __restrict__ xg, const float* __restrict__ dsel_row, const int* __restrict__ row_token,
+                      const int* __restrict__ seg_start, const int* __restrict__ task_ids, int tokens_per_image, int D, int E,
+                      float* __restrict__ dwg) {
+  constexpr int N = Pack<T>::N;
+  __shared__ float sm[8][32 * N];
+  int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  int e = blockIdx.y, task = blockIdx.z;
+  int col0 = (blockIdx.x * 32 + tx) * N;
+  float acc[N];
+#pragma unroll
+  for (int j = 0; j < N; ++j) acc[j] = 0.f;
+  if (col0 < D) {
+    for (int r = seg_start[e] + ty; r < seg_start[e + 1]; r += 8) {
+      int tok = row_token[r];
+      if (tok < 0) continue;
+      int tk = task_ids ? task_ids[tok / tokens_per_image] : 0;
+      if (tk != task) continue;
+      float c = dsel_row[r];
+      float v[N];
+      load16(xg + (size_t)r * D + col0, v);
+#pragma unroll
+      for (int j = 0; j < N; ++j) acc[j] = fmaf(c, v[j], acc[j]);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < N; ++j) sm[ty][tx * N + j] = acc[j];
+  __syncthreads();
+  for (int c = threadIdx.x; c < 32 * N; c += blockDim.x) {
+    int col = blockIdx.x * 32 * N + c;
+    if (col < D) {
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) s += sm[w][c];
+      dwg[((size_t)task * E + e) * D + col] = s;
+    }
+  }
+}
+
+// =================================================================================================
+// launchers
+// =================================================================================================
+int moe_rows_cap(int M, int E, int K) { return ((M * K + E * 127) + 127) & ~127; }
+int moe_blocks(int M) { return ceil_div(M, MOE_BLOCK_TOKENS); }
+
+void moe_route(const Ctx& c, const MoeBufs& b, const void* y, const void* wg, const int* task_ids, int tokens_per_image, int M,
+               int D, int E, int K) {
+  int nblk = moe_blocks(M);
+  int rows_cap = moe_rows_cap(M, E, K);
+  note_launch(4);
+  if (c.dtype == 0)
+    moe_route_kernel<float><<<nblk, 256, 0, c.stream>>>((const float*)y, (const float*)wg, task_ids, tokens_per_image, M, D, E, K, b.eidx, b.ew, b.blk_counts);
+  else
+    moe_route_kernel<bf16><<<nblk, 256, 0, c.stream>>>((const bf16*)y, (const bf16*)wg, task_ids, tokens_per_image, M, D, E, K, b.eidx, b.ew, b.blk_counts);
+  moe_scan_kernel<<<1, 128, 0, c.stream>>>(b.blk_counts, nblk, E, rows_cap / 128, b.blk_off, b.seg_start, b.tile_expert);
+  cudaMemsetAsync(b.row_token, 0xFF, (size_t)rows_cap * sizeof(int), c.stream);
+  moe_assign_kernel<<<nblk, 256, 0, c.stream>>>(b.eidx, b.ew, b.blk_off, b.seg_start, M, E, K, b.pos, b.row_token, b.row_w);
+  int blocks = ceil_div((long)rows_cap * 32, 256);
+  if (c.dtype == 0) moe_gather_kernel<float><<<blocks, 256, 0, c.stream>>>((const float*)y, b.row_token, b.seg_start, E, D, (float*)b.xg, rows_cap);
+  else moe_gather_kernel<bf16><<<blocks, 256, 0, c.stream>>>((const bf16*)y, b.row_token, b.seg_start, E, D, (bf16*)b.xg, rows_cap);
+}
+
+void moe_combine(const Ctx& c, const MoeBufs& b, const float* res, float* out, int M, int D, int K) {
+  note_launch(1);
+  int blocks = ceil_div((long)M * 32, 256);
+  if (c.dtype == 0) moe_combine_kernel<float><<<blocks, 256, 0, c.stream>>>((const float*)b.og, b.pos, b.ew, res, out, M, D, K);
+  else moe_combine_kernel<bf16><<<blocks, 256, 0, c.stream>>>((const bf16*)b.og, b.pos, b.ew, res, out, M, D, K);
+}
+
+void moe_combine_bwd(const Ctx& c, const MoeBufs& b, const float* dout, void* dog, float* dw, int M, int D, int E, int K) {
+  note_launch(1);
+  int rows_cap = moe_rows_cap(M, E, K);
+  int blocks = ceil_div((long)rows_cap * 32, 256);
+  if (c.dtype == 0)
+    moe_combine_bwd_kernel<float><<<blocks, 256, 0, c.stream>>>(dout, (const float*)b.og, b.row_token, b.row_w, b.seg_start, E, D, (float*)dog, dw, rows_cap);
+  else
+    moe_combine_bwd_kernel<bf16><<<blocks, 256, 0, c.stream>>>(dout, (const bf16*)b.og, b.row_token, b.row_w, b.seg_start, E, D, (bf16*)dog, dw, rows_cap);
+}
+
+void moe_seg_colsum(const Ctx& c, const MoeBufs& b, const void* x, int cols, int E, float* out) {
+  note_launch(1);
+  if (c.dtype == 0) moe_seg_colsum_kernel<float><<<dim3(ceil_div(cols, 128), E), 256, 0, c.stream>>>((const float*)x, b.seg_start, cols, out);
+  else moe_seg_colsum_kernel<bf16><<<dim3(ceil_div(cols, 256), E), 256, 0, c.stream>>>((const bf16*)x, b.seg_start, cols, out);
+}
+
+void moe_gate_bwd(const Ctx& c, const MoeBufs& b, const void* dxg, const float* dw, const void* wg, const int* task_ids,
+                  int tokens_per_image, int tasks, int M, int D, int E, int K, void* dy, float* dsel_row, float* dwg) {
+  note_launch(2);
+  int blocks = ceil_div((long)M * 32, 256);
+  if (c.dtype == 0) {
+    moe_gate_bwd_kernel<float><<<blocks, 256, 0, c.stream>>>((const float*)dxg, dw, b.pos, b.eidx, b.ew, (const float*)wg, task_ids, tokens_per_image, M, D, E, K, (float*)dy, dsel_row);
+    moe_gate_wgrad_kernel<float><<<dim3(ceil_div(D, 128), E, tasks), 256, 0, c.stream>>>((const float*)b.xg, dsel_row, b.row_token, b.seg_start, task_ids, tokens_per_image, D, E, dwg);
+  } else {
+    moe_gate_bwd_kernel<bf16><<<blocks, 256, 0, c.stream>>>((const bf16*)dxg, dw, b.pos, b.eidx, b.ew, (const bf16*)wg, task_ids, tokens_per_image, M, D, E, K, (bf16*)dy, dsel_row);
+    moe_gate_wgrad_kernel<bf16><<<dim3(ceil_div(D, 256), E, tasks), 256, 0, c.stream>>>((const bf16*)b.xg, dsel_row, b.row_token, b.seg_start, task_ids, tokens_per_image, D, E, dwg);
+  }
+}
+
+}  // namespace bsr

@@ -45,6 +45,11 @@ def run_gpu_step(cfg, images, labels, task_ids, params, batch=None, steps=1):
     out["m"] = {n: eng.get_tensor("adam_m/" + n, shapes[n]).cpu().numpy().astype(np.float64) for n in names}
     out["v"] = {n: eng.get_tensor("adam_v/" + n, shapes[n]).cpu().numpy().astype(np.float64) for n in names}
     out["params"] = {n: eng.get_tensor(n, shapes[n]).cpu().numpy().astype(np.float64) for n in shapes}
+    out["experts"] = {}
+    for l in cfg.moe_blocks:
+        tokens = 1 if (l == cfg.depth - 1 and l not in cfg.drop_blocks) else eng.tf[l]     # last block: classification rows only
+        e = eng.get_tensor(f"moe_experts/{l}", (B * tokens * cfg.moe_top_k,)).cpu().numpy()
+        out["experts"][l] = e.astype(np.int64).reshape(B, tokens, cfg.moe_top_k)
     out["footprint"] = eng.footprint()
     out["engine"] = eng
     return out
@@ -83,10 +88,44 @@ def check_selection(cfg, gpu_kept, forced_run, exact_margin, score_tol):
     return total, same
 
 
+def forced_experts_of(cfg, gpu, token_counts):
+    """The GPU's routing as the oracle's forced_experts input; tokens the GPU never routed (rows of the last
+    block other than the classification row) are left to the oracle (-1)."""
+    out = {}
+    for l, e in gpu.get("experts", {}).items():
+        B, t, k = e.shape
+        full = np.full((B, token_counts[l], k), -1, dtype=np.int64)
+        full[:, :t] = e
+        out[l] = full
+    return out
+
+
+def check_routing(cfg, ref, gpu, logit_tol):
+    """Every expert the GPU chose must be a valid top-k choice of the oracle's gate logits within logit_tol."""
+    flips = total = 0
+    for l, e in gpu.get("experts", {}).items():
+        gl = ref["routing"][l]["glogits"]
+        own = ref["routing"][l]["own_experts"]
+        B, t, k = e.shape
+        for b in range(B):
+            for i in range(t):
+                kth = np.sort(gl[b, i])[-k]
+                assert len(set(e[b, i])) == k
+                assert gl[b, i][e[b, i]].min() >= kth - logit_tol, (l, b, i)
+                total += 1
+                flips += int(set(e[b, i]) != set(own[b, i]))
+    return total, flips
+
+
 def compare_step(cfg, images, labels, task_ids, params, gpu, tol, exact_margin, score_tol):
-    free = O.train_step(cfg, params, images, labels, task_ids)
     forced = gpu["kept"] if gpu["kept"] else None
-    ref = O.train_step(cfg, params, images, labels, task_ids, forced_keep=forced) if forced else free
+    fe = None
+    if gpu.get("experts"):
+        sched = O.token_schedule(cfg)
+        fe = forced_experts_of(cfg, gpu, {l: sched[l][1] for l in cfg.moe_blocks})
+    ref = O.train_step(cfg, params, images, labels, task_ids, forced_keep=forced, forced_experts=fe)
+    if fe:
+        check_routing(cfg, ref, gpu, 2e-2)
     total, same = check_selection(cfg, gpu["kept"], ref, exact_margin, score_tol) if forced else (0, 0)
     report = {"sets": total, "sets_identical": same}
     assert abs(gpu["loss"] - ref["loss"]) <= tol * abs(ref["loss"]), (gpu["loss"], ref["loss"])
