@@ -107,7 +107,7 @@ int32_t bsr_workspace_bytes(const bsr_config* cfg_host, size_t* bytes_host);
 /* Creates the step engine (Fig. 2).  `workspace_dev` must be 256-byte aligned device memory of at
  * least bsr_workspace_bytes() bytes and must outlive the handle.  Validates the configuration
  * (BSR_ERR_INVALID_ARG), rejects what is not built (BSR_ERR_UNSUPPORTED: a trainable set that is not
- * "the last k blocks"), zeroes optimiser state and sets the step counter to 0.  Parameters are
+ * "the last k blocks"; MoE layers outside bf16 or with dim / mlp_hidden not multiples of 64), zeroes optimiser state and sets the step counter to 0.  Parameters are
  * undefined until set with bsr_set_param.  On failure *out_host is NULL. */
 int32_t bsr_create(const bsr_config* cfg_host, void* workspace_dev, size_t bytes, bsr_handle** out_host);
 
@@ -126,7 +126,8 @@ int32_t bsr_set_param(bsr_handle* h, const char* name, const float* src_dev, siz
  * equal the tensor's size) on `stream`.  Names: a parameter name (the fp32 master if it trains,
  * else the stored weight widened), "grad/<param>", "adam_m/<param>", "adam_v/<param>" (trainable
  * parameters only), "logits" ([max_batch, max classes], rows of the last step; classes a task does
- * not have hold -inf), "loss" (1 element). */
+ * not have hold -inf), "loss" (1 element), "moe_experts/<l>" (the experts chosen by block l's router in the last
+ * step, [tokens routed, top_k] as floats, best first; the last block routes only the classification rows). */
 int32_t bsr_get_tensor(bsr_handle* h, const char* name, float* dst_dev, size_t count, void* stream);
 
 /* Learning rate for the next steps (the cosine schedule of Section 5 lives in the caller). */

@@ -295,7 +295,7 @@ size_t plan(bsr_handle* h) {
     bb.m_xg = b.take(cap * D * es);
     bb.m_zg = b.take(cap * F * es);
     bb.m_hg = b.take(cap * F * es);
-    bb.m_og = b.take(cap * D * es);
+    bb.m_og = b.take(cap * D * 4);
   };
   h->moe_rec_eidx = rec_eidx;
   h->moe_rec_ew = rec_ew;
@@ -450,7 +450,7 @@ MoeBufs moe_bufs(const bsr_handle* h, const BlockBufs& bb) {
   m.row_token = h->at<int>(bb.m_row_token); m.row_w = h->at<float>(bb.m_row_w);
   m.seg_start = h->at<int>(bb.m_seg); m.tile_expert = h->at<int>(bb.m_tile);
   m.blk_counts = h->at<int>(bb.m_cnt); m.blk_off = h->at<int>(bb.m_off);
-  m.xg = h->base + bb.m_xg; m.zg = h->base + bb.m_zg; m.hg = h->base + bb.m_hg; m.og = h->base + bb.m_og;
+  m.xg = h->base + bb.m_xg; m.zg = h->base + bb.m_zg; m.hg = h->base + bb.m_hg; m.og = h->at<float>(bb.m_og);
   return m;
 }
 
@@ -510,10 +510,10 @@ int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb
     m1.bias = (const float*)h->wb(l, "moe.fc1.bias");
     m1.act = 1;
     m1.aux_out = save ? mb.zg : nullptr;
-    int rc1 = gemm_tc_grouped_rows(c, mb.xg, h->wb(l, "moe.fc1.weight"), 0, mb.hg, cap, F, D, E, mb.tile_expert, m1);
+    int rc1 = gemm_tc_grouped_rows(c, mb.xg, h->wb(l, "moe.fc1.weight"), 0, mb.hg, 0, cap, F, D, E, mb.tile_expert, m1);
     GemmEpilogue m2;
     m2.bias = (const float*)h->wb(l, "moe.fc2.bias");
-    int rc2 = gemm_tc_grouped_rows(c, mb.hg, h->wb(l, "moe.fc2.weight"), 0, mb.og, cap, D, F, E, mb.tile_expert, m2);
+    int rc2 = gemm_tc_grouped_rows(c, mb.hg, h->wb(l, "moe.fc2.weight"), 0, mb.og, 1, cap, D, F, E, mb.tile_expert, m2);
     if (rc1 != 0 || rc2 != 0) return set_err(h->err, BSR_ERR_CUDA, "grouped GEMM set-up failed (%d, %d)", rc1, rc2);
     moe_combine(c, mb, h->at<float>(bb.xp), h->at<float>(bb.x_out), Mf, D, K);
     return BSR_OK;
@@ -574,10 +574,10 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
     GemmEpilogue eg;
     eg.act = 2;
     eg.aux_in = mb.zg;
-    int r1 = gemm_tc_grouped_rows(c, dog, h->wb(l, "moe.fc2.weight"), 1, dzg, cap, F, D, E, mb.tile_expert, eg);
+    int r1 = gemm_tc_grouped_rows(c, dog, h->wb(l, "moe.fc2.weight"), 1, dzg, 0, cap, F, D, E, mb.tile_expert, eg);
     int r2 = gemm_tc_grouped_wgrad(c, dog, mb.hg, h->gb(l, "moe.fc2.weight"), cap, D, F, E, mb.seg_start);
     moe_seg_colsum(c, mb, dog, D, E, h->gb(l, "moe.fc2.bias"));
-    int r3 = gemm_tc_grouped_rows(c, dzg, h->wb(l, "moe.fc1.weight"), 1, dxg, cap, D, F, E, mb.tile_expert, none);
+    int r3 = gemm_tc_grouped_rows(c, dzg, h->wb(l, "moe.fc1.weight"), 1, dxg, 0, cap, D, F, E, mb.tile_expert, none);
     int r4 = gemm_tc_grouped_wgrad(c, dzg, mb.xg, h->gb(l, "moe.fc1.weight"), cap, F, D, E, mb.seg_start);
     moe_seg_colsum(c, mb, dzg, F, E, h->gb(l, "moe.fc1.bias"));
     if (r1 || r2 || r3 || r4) return set_err(h->err, BSR_ERR_CUDA, "grouped GEMM set-up failed (%d, %d, %d, %d)", r1, r2, r3, r4);

@@ -348,8 +348,8 @@ int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const voi
 }
 
 // Expert-grouped contractions of the MoE layer (paper Section 5.2); see kernels.h.
-int gemm_tc_grouped_rows(const Ctx& c, const void* A, const void* Bst, int b_mn, void* C, int rows_cap, int n, int k, int experts,
-                         const int* tile_expert, const GemmEpilogue& e) {
+int gemm_tc_grouped_rows(const Ctx& c, const void* A, const void* Bst, int b_mn, void* C, int out_is_float, int rows_cap, int n, int k,
+                         int experts, const int* tile_expert, const GemmEpilogue& e) {
   using namespace tc;
   if ((n % 8) || (k % 8) || (rows_cap % BM) || ((uintptr_t)A & 15) || ((uintptr_t)Bst & 15) || ((uintptr_t)C & 15)) return -1;
   if (b_mn && (k % BK)) return -1;             // a k-slab must not straddle two experts' weights
@@ -367,8 +367,13 @@ int gemm_tc_grouped_rows(const Ctx& c, const void* A, const void* Bst, int b_mn,
   ep.bias = e.bias; ep.residual = e.residual; ep.aux_out = e.aux_out; ep.aux_in = e.aux_in; ep.act = e.act;
   int tiles_m = rows_cap / BM, tiles_n = ceil_div(n, BN);
   if (c.prof != nullptr && c.prof->on) c.prof->begin(c.stream, 2.0 * rows_cap * n * (double)k);
-  int rc = b_mn ? launch<false, true, bf16>(c, ma, mb, C, rows_cap, n, k, ep, tiles_m, tiles_n, 1, ceil_div(k, BK), g)
-                : launch<false, false, bf16>(c, ma, mb, C, rows_cap, n, k, ep, tiles_m, tiles_n, 1, ceil_div(k, BK), g);
+  int rc;
+  if (out_is_float)
+    rc = b_mn ? launch<false, true, float>(c, ma, mb, C, rows_cap, n, k, ep, tiles_m, tiles_n, 1, ceil_div(k, BK), g)
+              : launch<false, false, float>(c, ma, mb, C, rows_cap, n, k, ep, tiles_m, tiles_n, 1, ceil_div(k, BK), g);
+  else
+    rc = b_mn ? launch<false, true, bf16>(c, ma, mb, C, rows_cap, n, k, ep, tiles_m, tiles_n, 1, ceil_div(k, BK), g)
+              : launch<false, false, bf16>(c, ma, mb, C, rows_cap, n, k, ep, tiles_m, tiles_n, 1, ceil_div(k, BK), g);
   if (c.prof != nullptr && c.prof->on) c.prof->end(c.stream);
   return rc;
 }

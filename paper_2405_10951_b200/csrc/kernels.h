@@ -105,9 +105,9 @@ int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const voi
                     int out_is_float, int m, int n, int k, const GemmEpilogue& e, float* split_ws, size_t split_ws_floats);
 
 // C[rows_cap, n] = epilogue(A[rows_cap, k] . W_e) with W_e the expert's slice of stacked weights: Bst [E*n, k]
-// (b_mn = 0, forward) or [E*k, n] (b_mn = 1, input gradient: C = A W_e).  bf16 in and out; e.bias stacked [E*n].
-int gemm_tc_grouped_rows(const Ctx& c, const void* A, const void* Bst, int b_mn, void* C, int rows_cap, int n, int k, int experts,
-                         const int* tile_expert, const GemmEpilogue& e);
+// (b_mn = 0, forward) or [E*k, n] (b_mn = 1, input gradient: C = A W_e).  bf16 operands, bf16 or float output; e.bias stacked [E*n].
+int gemm_tc_grouped_rows(const Ctx& c, const void* A, const void* Bst, int b_mn, void* C, int out_is_float, int rows_cap, int n, int k,
+                         int experts, const int* tile_expert, const GemmEpilogue& e);
 // dW[e][m, n] = sum over rows r of expert e's segment of dY[r, m] * X[r, n]  (float out).
 int gemm_tc_grouped_wgrad(const Ctx& c, const void* dY, const void* X, float* dW, int rows_cap, int m, int n, int experts,
                           const int* seg_start);
@@ -174,7 +174,7 @@ struct MoeBufs {
   void* xg;           // [rows_cap, D] gathered expert inputs
   void* zg;           // [rows_cap, F] FC1 pre-activation (kept by trainable blocks)
   void* hg;           // [rows_cap, F] GELU output
-  void* og;           // [rows_cap, D] expert outputs
+  float* og;          // [rows_cap, D] expert outputs (float: they are summed into the residual stream)
 };
 int moe_rows_cap(int M, int E, int K);
 int moe_blocks(int M);

@@ -141,8 +141,7 @@ __global__ void moe_gather_kernel(const T* __restrict__ y, const int* __restrict
 }
 
 // ---- combine: out[t] = res[t] + sum_slot w_slot * og[pos(t, slot)]  (float residual stream) ------------------------
-template <typename T>
-__global__ void moe_combine_kernel(const T* __restrict__ og, const int* __restrict__ pos, const float* __restrict__ ew,
+__global__ void moe_combine_kernel(const float* __restrict__ og, const int* __restrict__ pos, const float* __restrict__ ew,
                                    const float* __restrict__ res, float* __restrict__ out, int M, int D, int K) {
   int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= M) return;
@@ -152,7 +151,7 @@ __global__ void moe_combine_kernel(const T* __restrict__ og, const int* __restri
     for (int s = 0; s < K; ++s) {
       float w = ew[(size_t)warp * K + s];
       float v[4];
-      load4(og + (size_t)pos[(size_t)warp * K + s] * D + ch * 4, v);
+      load16(og + (size_t)pos[(size_t)warp * K + s] * D + ch * 4, v);
 #pragma unroll
       for (int j = 0; j < 4; ++j) acc[j] = fmaf(w, v[j], acc[j]);
     }
@@ -162,7 +161,7 @@ __global__ void moe_combine_kernel(const T* __restrict__ og, const int* __restri
 
 // ---- backward of the combination: dog[r] = w_r * dout[token_r]; dw[r] = <dout[token_r], og[r]> ------------------
 template <typename T>
-__global__ void moe_combine_bwd_kernel(const float* __restrict__ dout, const T* __restrict__ og, const int* __restrict__ row_token,
+__global__ void moe_combine_bwd_kernel(const float* __restrict__ dout, const float* __restrict__ og, const int* __restrict__ row_token,
                                        const float* __restrict__ row_w, const int* __restrict__ seg_start, int E, int D,
                                        T* __restrict__ dog, float* __restrict__ dw, int rows_cap) {
   int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
@@ -174,7 +173,7 @@ __global__ void moe_combine_bwd_kernel(const float* __restrict__ dout, const T* 
     float g[4] = {0.f, 0.f, 0.f, 0.f}, o[4], r[4];
     if (tok >= 0) {
       load16(dout + (size_t)tok * D + ch * 4, g);
-      load4(og + (size_t)warp * D + ch * 4, o);
+      load16(og + (size_t)warp * D + ch * 4, o);
 #pragma unroll
       for (int j = 0; j < 4; ++j) dot = fmaf(g[j], o[j], dot);
     }
@@ -324,8 +323,7 @@ void moe_route(const Ctx& c, const MoeBufs& b, const void* y, const void* wg, co
 void moe_combine(const Ctx& c, const MoeBufs& b, const float* res, float* out, int M, int D, int K) {
   note_launch(1);
   int blocks = ceil_div((long)M * 32, 256);
-  if (c.dtype == 0) moe_combine_kernel<float><<<blocks, 256, 0, c.stream>>>((const float*)b.og, b.pos, b.ew, res, out, M, D, K);
-  else moe_combine_kernel<bf16><<<blocks, 256, 0, c.stream>>>((const bf16*)b.og, b.pos, b.ew, res, out, M, D, K);
+  moe_combine_kernel<<<blocks, 256, 0, c.stream>>>(b.og, b.pos, b.ew, res, out, M, D, K);
 }
 
 void moe_combine_bwd(const Ctx& c, const MoeBufs& b, const float* dout, void* dog, float* dw, int M, int D, int E, int K) {
@@ -333,9 +331,9 @@ void moe_combine_bwd(const Ctx& c, const MoeBufs& b, const float* dout, void* do
   int rows_cap = moe_rows_cap(M, E, K);
   int blocks = ceil_div((long)rows_cap * 32, 256);
   if (c.dtype == 0)
-    moe_combine_bwd_kernel<float><<<blocks, 256, 0, c.stream>>>(dout, (const float*)b.og, b.row_token, b.row_w, b.seg_start, E, D, (float*)dog, dw, rows_cap);
+    moe_combine_bwd_kernel<float><<<blocks, 256, 0, c.stream>>>(dout, b.og, b.row_token, b.row_w, b.seg_start, E, D, (float*)dog, dw, rows_cap);
   else
-    moe_combine_bwd_kernel<bf16><<<blocks, 256, 0, c.stream>>>(dout, (const bf16*)b.og, b.row_token, b.row_w, b.seg_start, E, D, (bf16*)dog, dw, rows_cap);
+    moe_combine_bwd_kernel<bf16><<<blocks, 256, 0, c.stream>>>(dout, b.og, b.row_token, b.row_w, b.seg_start, E, D, (bf16*)dog, dw, rows_cap);
 }
 
 void moe_seg_colsum(const Ctx& c, const MoeBufs& b, const void* x, int cols, int E, float* out) {

@@ -145,6 +145,8 @@ def compare_step(cfg, images, labels, task_ids, params, gpu, tol, exact_margin, 
     # the update itself, from the GPU's own gradient (AdamW's first step is a sign function of g: comparing
     # updated weights across implementations would amplify rounding of near-zero gradients without bound)
     for n in ref["grads"]:
+        if np.abs(gpu["grads"][n]).max() < 1e-6:         # an identically-zero gradient (e.g. the gate of a top-1 router):
+            continue                                     # g / (|g| + eps) is then dominated by float rounding of g itself
         want, _, _ = O.adamw(cfg, params[n], gpu["grads"][n], np.zeros_like(params[n]), np.zeros_like(params[n]), 1, O.is_decayed(n))
         d_gpu = gpu["params"][n] - params[n]
         d_ref = want - params[n]

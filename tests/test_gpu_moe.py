@@ -16,7 +16,7 @@ CASES = {
     "moe_is_last_block": MINI_MOE.with_(depth=4, trainable=(2, 3)),
     "top1_single_task": MINI_MOE.with_(num_classes=(10,), moe_top_k=1, moe_experts=8),
     "moe_drop_block_trainable": MINI_MOE.with_(drop_blocks=(3,), trainable=(3, 4)),
-    "moe_vit_s_batch4": CONFIGS["moe_vit_s"].with_(batch=4),
+    "moe_vit_s_batch16": CONFIGS["moe_vit_s"].with_(batch=16),
 }
 
 
