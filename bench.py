@@ -105,6 +105,19 @@ class ClockSampler:
         return out
 
 
+def aggregate(dist, world, batch, steps, ms_local):
+    """Whole-job throughput from per-rank timings: max over ranks of each elapsed time (a list of milliseconds),
+    then images of all ranks over that time.  `dist` is torch.distributed (any backend) or None."""
+    import torch
+    t = torch.tensor(list(ms_local), dtype=torch.float64)
+    if dist is not None and world > 1:
+        if dist.get_backend() == "nccl":
+            t = t.cuda()
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = [float(x) for x in t.cpu()]
+    return ms, [world * batch * steps / (m / 1e3) for m in ms]
+
+
 def oracle_sample_step(cfg, images, labels, task_ids, params):
     from oracle import bsr_oracle as O
     t0 = time.perf_counter()
@@ -242,13 +255,8 @@ def main():
     eng.sync_status()
     clocks = sampler.stop() if rank == 0 else {}
 
-    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = float(t[0]), float(t[1])
+    (ms_total, ms_e2e), (value, e2e_value) = aggregate(dist, world, cfg.batch, args.steps, [ms_total, ms_e2e])
     ms_step = ms_total / args.steps
-    value = world * cfg.batch / (ms_step / 1e3)
-    e2e_value = world * cfg.batch / (ms_e2e / args.steps / 1e3)
 
     if rank == 0:
         pk = peaks()

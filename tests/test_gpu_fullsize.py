@@ -1,0 +1,62 @@
+"""The headline workload at full size, in the launch configuration bench.py times (ViT-B/16, bf16, batch 128).
+
+The oracle cannot run 128 ViT-B images in a test, but images are independent until the batch-mean loss, so:
+sampled images are recomputed one by one (logits, kept sets), the loss is re-derived from the GPU's logits, and
+the gradients are checked through a property that holds at any size (the gradient of the mean loss over the batch
+is the mean of the gradients over its halves)."""
+import numpy as np
+import pytest
+
+from oracle import bsr_oracle as O
+from paper_2405_10951_b200 import synth
+from paper_2405_10951_b200.synth import CONFIGS
+
+import parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+def test_vit_b_full_batch_sampled_outputs_and_properties():
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    cfg = CONFIGS["vit_b"]
+    images, labels, task_ids, params = synth.make_workload(cfg)
+    eng = Bd.Engine(cfg)
+    eng.set_params(params)
+    img = eng.images_to_device(images)
+    lab = torch.as_tensor(labels).cuda()
+    loss, kept = eng.train_step(img, lab)
+    eng.sync_status()
+    B = cfg.batch
+    logits = eng.get_tensor("logits", (B, eng.cmax)).cpu().numpy().astype(np.float64)
+    kept = [k.cpu().numpy().astype(np.int64) for k in kept]
+    # 1. the loss is the mean cross-entropy of the logits the step produced
+    want_loss, _ = O.cross_entropy(logits, labels)
+    assert abs(float(loss.cpu()[0]) - want_loss) < 1e-5 * want_loss
+    assert abs(want_loss - np.log(100)) < 0.2                     # near ln(classes) at initialisation
+    # 2. sampled images, one by one, through the oracle with the GPU's kept sets
+    for b in (0, 41, 127):
+        forced = [k[b:b + 1] for k in kept]
+        ref = O.forward(cfg, params, images[b:b + 1], forced_keep=forced)
+        assert P.rel_err(logits[b], ref["logits"][0]) < P.BF16_TOL
+        P.check_selection(cfg, forced, ref, 2 * P.BF16_SCORE_TOL, P.BF16_SCORE_TOL)
+    # 3. kept sets are valid index sets for every image
+    ks = [138, 98, 70]
+    for loc, k in enumerate(kept):
+        assert k.shape == (B, ks[loc])
+        assert np.all(np.diff(k, axis=1) > 0) and k.min() >= 0
+    # 4. gradient of the batch mean = mean of the gradients of the two halves (same parameters, two fresh handles)
+    names = ["head.0.weight", "blocks.11.attn.qkv.weight", "blocks.8.mlp.fc1.weight", "blocks.9.norm1.weight", "blocks.8.attn.proj.bias"]
+    shapes = synth.param_shapes(cfg)
+    full = {n: eng.get_tensor("grad/" + n, shapes[n]).cpu().numpy().astype(np.float64) for n in names}
+    eng.close()
+    halves = []
+    for sl in (slice(0, 64), slice(64, 128)):
+        e2 = Bd.Engine(cfg, max_batch=64)
+        e2.set_params(params)
+        e2.train_step(e2.images_to_device(images[sl]), torch.as_tensor(labels[sl]).cuda())
+        e2.sync_status()
+        halves.append({n: e2.get_tensor("grad/" + n, shapes[n]).cpu().numpy().astype(np.float64) for n in names})
+        e2.close()
+    for n in names:
+        assert P.rel_err(full[n], 0.5 * (halves[0][n] + halves[1][n])) < 5e-3, n

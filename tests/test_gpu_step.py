@@ -39,6 +39,8 @@ BF16_CASES = {
     "mini": MINI_BF16,
     "mini_no_fusion": MINI_BF16.with_(fuse_mode=0),
     "deit_s_batch4": CONFIGS["deit_s"].with_(batch=4),
+    "vit_b_batch3": CONFIGS["vit_b"].with_(batch=3),
+    "vit_b_384_batch2": CONFIGS["vit_b_384"].with_(batch=2),
 }
 
 
