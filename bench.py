@@ -203,6 +203,9 @@ def main():
     lab = torch.as_tensor(labels).cuda()
     tid = torch.as_tensor(task_ids).cuda() if cfg.num_tasks > 1 else None
     host_loss = torch.empty(1, dtype=torch.float32).pin_memory()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()          # a capturable stream: the library replays the step as a CUDA graph on it
+    torch.cuda.set_stream(side)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -211,8 +214,10 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    out = None
     for _ in range(warm):
-        eng.train_step(dev_img, lab, tid, want_kept=False)
+        eng.train_step(dev_img, lab, tid, want_kept=False, out=out)
+        out = eng.last_out
     eng.sync_status()
 
     sampler = ClockSampler(local)
@@ -226,7 +231,7 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
-        loss, _ = eng.train_step(dev_img, lab, tid, want_kept=False)
+        loss, _ = eng.train_step(dev_img, lab, tid, want_kept=False, out=out)
     e1.record(stream)
     barrier()
     ms_total = e0.elapsed_time(e1)
@@ -239,7 +244,7 @@ def main():
     f0.record(stream)
     for _ in range(args.steps):
         stage.copy_(host_img, non_blocking=True)
-        loss, _ = eng.train_step(stage, lab, tid, want_kept=False)
+        loss, _ = eng.train_step(stage, lab, tid, want_kept=False, out=out)
         host_loss.copy_(loss, non_blocking=True)
         stream.synchronize()
     f1.record(stream)
@@ -249,7 +254,7 @@ def main():
     # ---- dominant kernel (tcgen05 GEMM): every launch bracketed by CUDA events ---------------------
     eng.profile_enable(True)
     for _ in range(min(args.steps, 5)):
-        eng.train_step(dev_img, lab, tid, want_kept=False)
+        eng.train_step(dev_img, lab, tid, want_kept=False, out=out)
     prof = eng.profile_read()
     eng.profile_enable(False)
     eng.sync_status()

@@ -167,6 +167,12 @@ int32_t bsr_sync_status(bsr_handle* h, void* stream);
  * tile (the default), 2 = as 1 but GEMMs with more than 128 rows run on CTA pairs (cta_group::2). */
 int32_t bsr_set_gemm_mode(bsr_handle* h, int32_t mode);
 
+/* bsr_train_step replays a captured CUDA graph of its ~200 launches when `stream` can be captured (any stream but
+ * the legacy default stream, and not one the caller is capturing) -- the first call with a given set of pointers
+ * and batch captures it, later calls with the same arguments replay it.  on = 0 turns this off (every call
+ * enqueues its kernels one by one); the results are identical.  No counterpart in the paper. */
+int32_t bsr_set_graph_mode(bsr_handle* h, int32_t on);
+
 /* Measurement support (no counterpart in the paper).  bsr_profile_enable resets the counters; with
  * time_gemms != 0 every tensor-core GEMM launch of the following steps is bracketed by a pair of CUDA
  * events on the launching stream (host objects; this slows the step slightly, so timed throughput is

@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "BSR_OK", -1: "BSR_ERR_INVALID_ARG", -2: "BSR_ERR_UNSUPPORTED
 
 EXPORTS = ["bsr_token_schedule", "bsr_workspace_bytes", "bsr_create", "bsr_destroy", "bsr_last_error", "bsr_set_param",
            "bsr_get_tensor", "bsr_set_lr", "bsr_set_step", "bsr_train_step", "bsr_eval_forward", "bsr_get_footprint",
-           "bsr_sync_status", "bsr_set_gemm_mode", "bsr_profile_enable", "bsr_profile_read", "bsr_profile_launches", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_backward",
+           "bsr_sync_status", "bsr_set_gemm_mode", "bsr_set_graph_mode", "bsr_profile_enable", "bsr_profile_read", "bsr_profile_launches", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_backward",
            "bsr_linear_backward_static", "bsr_static_last_error", "bsr_attention_forward"]
 
 
@@ -88,6 +88,7 @@ def lib() -> C.CDLL:
         L.bsr_get_footprint.argtypes = [vp, C.POINTER(bsr_footprint)]
         L.bsr_sync_status.argtypes = [vp, vp]
         L.bsr_set_gemm_mode.argtypes = [vp, i32]
+        L.bsr_set_graph_mode.argtypes = [vp, i32]
         L.bsr_profile_enable.argtypes = [vp, i32]
         L.bsr_profile_read.argtypes = [vp, vp, C.POINTER(bsr_profile)]
         L.bsr_profile_launches.argtypes = [vp, vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_float), C.POINTER(C.c_int32)]
@@ -294,16 +295,22 @@ class Engine:
         t = self.torch.as_tensor(np.ascontiguousarray(images, dtype=np.float32))
         return t.to(self.device).to(self.storage_dtype).contiguous()
 
-    def train_step(self, images, labels, task_ids=None, want_kept: bool = True):
+    def train_step(self, images, labels, task_ids=None, want_kept: bool = True, out=None):
         """images: CUDA tensor [B, C, S, S] in the storage dtype; labels/task_ids: int32 CUDA tensors.
-        Returns (loss tensor [1], list of kept-index tensors [B, K_i] or None).  Does not synchronise."""
+        Returns (loss tensor [1], list of kept-index tensors [B, K_i] or None).  Does not synchronise.
+        `out` = (loss, kept_flat) from an earlier call reuses those output buffers: with identical pointers the
+        library replays its captured graph of the step instead of capturing a new one."""
         torch = self.torch
         B = images.shape[0]
-        loss = torch.empty(1, dtype=torch.float32, device=self.device)
-        kept = None
-        if want_kept and self.kept_counts:
-            kept = torch.empty(B * sum(self.kept_counts), dtype=torch.int32, device=self.device)
+        if out is not None:
+            loss, kept = out
+        else:
+            loss = torch.empty(1, dtype=torch.float32, device=self.device)
+            kept = None
+            if want_kept and self.kept_counts:
+                kept = torch.empty(B * sum(self.kept_counts), dtype=torch.int32, device=self.device)
         _check(lib().bsr_train_step(self.h, _ptr(images), _ptr(labels), _ptr(task_ids), B, _stream(), _ptr(loss), _ptr(kept)), self.h)
+        self.last_out = (loss, kept)
         return loss, self._split_kept(kept, B)
 
     def eval_forward(self, images, task_ids=None, want_kept: bool = True):
@@ -330,6 +337,9 @@ class Engine:
 
     def set_gemm_mode(self, mode: int):
         _check(lib().bsr_set_gemm_mode(self.h, mode), self.h)
+
+    def set_graph_mode(self, on: bool):
+        _check(lib().bsr_set_graph_mode(self.h, int(on)), self.h)
 
     def profile_enable(self, time_gemms: bool):
         _check(lib().bsr_profile_enable(self.h, int(time_gemms)), self.h)

@@ -168,6 +168,11 @@ struct bsr_handle {
   std::vector<size_t> moe_rec_eidx, moe_rec_ew;
   size_t off_m_dog = 0, off_m_dzg = 0, off_m_dxg = 0, off_m_dw = 0, off_m_dsel = 0;
   GemmProfile prof;
+  // captured graphs of the training step, keyed by the caller's pointers
+  struct StepGraph { const void* images; const void* labels; const void* tasks; void* loss; void* kept; int batch; int mode;
+                     cudaGraphExec_t exec; long launches; };
+  std::vector<StepGraph> graphs;
+  int use_graph = 1;
   long launches_at_enable = 0;
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(base + off); }
@@ -797,8 +802,10 @@ int32_t bsr_create(const bsr_config* cfg, void* workspace, size_t bytes, bsr_han
 }
 
 int32_t bsr_destroy(bsr_handle* h) {
-  if (h != nullptr)
+  if (h != nullptr) {
     for (cudaEvent_t ev : h->prof.events) cudaEventDestroy(ev);
+    for (auto& g : h->graphs) cudaGraphExecDestroy(g.exec);
+  }
   delete h;
   return BSR_OK;
 }
@@ -882,12 +889,10 @@ int32_t bsr_set_step(bsr_handle* h, int64_t steps_done) {
   return BSR_OK;
 }
 
-int32_t bsr_train_step(bsr_handle* h, const void* images, const int32_t* labels, const int32_t* task_ids, int32_t batch,
-                       void* stream, float* loss_out, int32_t* kept_out) {
-  int rc = check_batch(h, images, batch);
-  if (rc != BSR_OK) return rc;
-  if (labels == nullptr || loss_out == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "labels_dev and loss_dev_out must not be null");
-  if (h->cfg.dims.num_tasks > 1 && task_ids == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "task_ids_dev is required with several tasks");
+// Enqueues every kernel of one step on `stream` (forward, loss, backward, AdamW reading its scalars from device memory).
+static int enqueue_train_step(bsr_handle* h, const void* images, const int32_t* labels, const int32_t* task_ids, int32_t batch,
+                              void* stream, float* loss_out, int32_t* kept_out) {
+  int rc;
   const bsr_dims& d = h->cfg.dims;
   Ctx c = make_ctx(h, stream);
   int D = d.dim, B = batch;
@@ -927,13 +932,72 @@ int32_t bsr_train_step(bsr_handle* h, const void* images, const int32_t* labels,
     layernorm_bwd(c, h->at<float>(h->off_dxn), 1, h->at<float>(x_last), (long)Tl * D, h->at<float>(h->off_meanf), h->at<float>(h->off_rstdf),
                   (const float*)h->w("norm.weight"), nullptr, nullptr, 0, nullptr, lnp, h->gradp("norm.weight"), h->gradp("norm.bias"), B, D);
   }
+  adamw(c, h->at<AdamChunk>(h->off_chunks), h->n_chunks, h->at<float>(h->off_master), h->at<float>(h->off_grad), h->at<float>(h->off_m),
+        h->at<float>(h->off_v), h->base + h->off_weights, h->at<float>(h->off_status + 128), h->cfg.beta1, h->cfg.beta2, h->cfg.eps,
+        h->cfg.weight_decay);
+  return BSR_OK;
+}
+
+int32_t bsr_train_step(bsr_handle* h, const void* images, const int32_t* labels, const int32_t* task_ids, int32_t batch,
+                       void* stream, float* loss_out, int32_t* kept_out) {
+  int rc = check_batch(h, images, batch);
+  if (rc != BSR_OK) return rc;
+  if (labels == nullptr || loss_out == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "labels_dev and loss_dev_out must not be null");
+  if (h->cfg.dims.num_tasks > 1 && task_ids == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "task_ids_dev is required with several tasks");
+  cudaStream_t st = (cudaStream_t)stream;
   h->step += 1;
   double bc1 = 1.0 - std::pow((double)h->cfg.beta1, (double)h->step);
   double bc2 = 1.0 - std::pow((double)h->cfg.beta2, (double)h->step);
-  adamw(c, h->at<AdamChunk>(h->off_chunks), h->n_chunks, h->at<float>(h->off_master), h->at<float>(h->off_grad), h->at<float>(h->off_m),
-        h->at<float>(h->off_v), h->base + h->off_weights, h->lr, h->cfg.beta1, h->cfg.beta2, h->cfg.eps, h->cfg.weight_decay,
-        (float)bc1, (float)bc2);
-  return check_cuda(h, "bsr_train_step");
+  set_scalars(st, h->at<float>(h->off_status + 128), h->lr, (float)bc1, (float)bc2);
+  // A step is a fixed sequence of ~200 launches: replay it as a CUDA graph when the stream allows capture (not the
+  // legacy default stream, not a stream the caller is capturing) and nothing asks for per-launch events.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  bool can_graph = h->use_graph && st != nullptr && st != cudaStreamLegacy && !h->prof.on &&
+                   cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
+  if (!can_graph) {
+    cudaGetLastError();
+    rc = enqueue_train_step(h, images, labels, task_ids, batch, stream, loss_out, kept_out);
+    if (rc != BSR_OK) return rc;
+    return check_cuda(h, "bsr_train_step");
+  }
+  for (auto& g : h->graphs) {
+    if (g.images == images && g.labels == labels && g.tasks == task_ids && g.loss == loss_out && g.kept == kept_out &&
+        g.batch == batch && g.mode == h->use_tc) {
+      g_kernel_launches += g.launches;
+      if (cudaGraphLaunch(g.exec, st) != cudaSuccess) return set_err(h->err, BSR_ERR_CUDA, "graph launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+      return BSR_OK;
+    }
+  }
+  long before = g_kernel_launches;
+  if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();
+    rc = enqueue_train_step(h, images, labels, task_ids, batch, stream, loss_out, kept_out);
+    return rc != BSR_OK ? rc : check_cuda(h, "bsr_train_step");
+  }
+  rc = enqueue_train_step(h, images, labels, task_ids, batch, stream, loss_out, kept_out);
+  cudaGraph_t graph = nullptr;
+  cudaError_t ce = cudaStreamEndCapture(st, &graph);
+  if (rc != BSR_OK) {
+    if (graph) cudaGraphDestroy(graph);
+    return rc;
+  }
+  bsr_handle::StepGraph sg;
+  sg.images = images; sg.labels = labels; sg.tasks = task_ids; sg.loss = loss_out; sg.kept = kept_out; sg.batch = batch;
+  sg.mode = h->use_tc; sg.exec = nullptr; sg.launches = g_kernel_launches - before;
+  if (ce != cudaSuccess || graph == nullptr || cudaGraphInstantiate(&sg.exec, graph, 0) != cudaSuccess) {
+    if (graph) cudaGraphDestroy(graph);
+    cudaGetLastError();
+    rc = enqueue_train_step(h, images, labels, task_ids, batch, stream, loss_out, kept_out);   // nothing ran during capture
+    return rc != BSR_OK ? rc : check_cuda(h, "bsr_train_step");
+  }
+  cudaGraphDestroy(graph);
+  if (h->graphs.size() >= 4) {
+    cudaGraphExecDestroy(h->graphs.front().exec);
+    h->graphs.erase(h->graphs.begin());
+  }
+  h->graphs.push_back(sg);
+  if (cudaGraphLaunch(sg.exec, st) != cudaSuccess) return set_err(h->err, BSR_ERR_CUDA, "graph launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+  return BSR_OK;
 }
 
 int32_t bsr_eval_forward(bsr_handle* h, const void* images, const int32_t* task_ids, int32_t batch, void* stream,
@@ -1001,6 +1065,12 @@ int32_t bsr_set_gemm_mode(bsr_handle* h, int32_t mode) {
   if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
   if (mode < 0 || mode > 2) return set_err(h->err, BSR_ERR_INVALID_ARG, "mode must be 0, 1 or 2");
   h->use_tc = mode;
+  return BSR_OK;
+}
+
+int32_t bsr_set_graph_mode(bsr_handle* h, int32_t on) {
+  if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
+  h->use_graph = on != 0;
   return BSR_OK;
 }
 

@@ -154,8 +154,10 @@ void cross_entropy(const Ctx& c, const HeadDesc& h, const float* logits, const i
 void head_bwd(const Ctx& c, const HeadDesc& h, const float* xn, const float* dlogits, const int* task_ids, float* dxn, int B);
 
 struct AdamChunk { uint32_t offset; uint32_t count; int64_t shadow; uint32_t decay; uint32_t pad; };
+// scalars (device): learning rate, 1 - beta1^t, 1 - beta2^t of the step being taken.
 void adamw(const Ctx& c, const AdamChunk* chunks, int nchunks, float* master, const float* grad, float* m, float* v,
-           void* shadow_base, float lr, float b1, float b2, float eps, float wd, float bc1, float bc2);
+           void* shadow_base, const float* scalars, float b1, float b2, float eps, float wd);
+void set_scalars(cudaStream_t s, float* dst, float a, float b, float c3);
 
 // dst row r = src row r (row_bytes a multiple of 16), independent pitches: gathers / scatters token rows.
 void copy_rows(cudaStream_t s, const void* src, long src_pitch_bytes, void* dst, long dst_pitch_bytes, int rows, int row_bytes);

@@ -516,8 +516,10 @@ void head_bwd(const Ctx& c, const HeadDesc& h, const float* xn, const float* dlo
 template <typename T>
 __global__ void adamw_kernel(const AdamChunk* __restrict__ chunks, float* __restrict__ master,
                              const float* __restrict__ grad, float* __restrict__ m, float* __restrict__ v,
-                             T* __restrict__ shadow_base, float lr, float b1, float b2, float eps, float wd,
-                             float bc1, float bc2) {
+                             T* __restrict__ shadow_base, const float* __restrict__ scalars, float b1, float b2, float eps,
+                             float wd) {
+  // step-dependent scalars live in device memory so that a captured graph of the step stays valid: lr, 1-b1^t, 1-b2^t
+  float lr = scalars[0], bc1 = scalars[1], bc2 = scalars[2];
   AdamChunk ch = chunks[blockIdx.x];
   float decay = ch.decay ? lr * wd : 0.f;
   for (uint32_t i = threadIdx.x; i < ch.count; i += blockDim.x) {
@@ -534,14 +536,22 @@ __global__ void adamw_kernel(const AdamChunk* __restrict__ chunks, float* __rest
   }
 }
 
+__global__ void set_scalars_kernel(float* dst, float a, float b, float c3) {
+  dst[0] = a; dst[1] = b; dst[2] = c3;
+}
+void set_scalars(cudaStream_t s, float* dst, float a, float b, float c3) {
+  note_launch(1);
+  set_scalars_kernel<<<1, 1, 0, s>>>(dst, a, b, c3);
+}
+
 void adamw(const Ctx& c, const AdamChunk* chunks, int nchunks, float* master, const float* grad, float* m, float* v,
-           void* shadow_base, float lr, float b1, float b2, float eps, float wd, float bc1, float bc2) {
+           void* shadow_base, const float* scalars, float b1, float b2, float eps, float wd) {
   if (nchunks <= 0) return;
   note_launch(1);
   if (c.dtype == 0)
-    adamw_kernel<float><<<nchunks, 256, 0, c.stream>>>(chunks, master, grad, m, v, (float*)shadow_base, lr, b1, b2, eps, wd, bc1, bc2);
+    adamw_kernel<float><<<nchunks, 256, 0, c.stream>>>(chunks, master, grad, m, v, (float*)shadow_base, scalars, b1, b2, eps, wd);
   else
-    adamw_kernel<bf16><<<nchunks, 256, 0, c.stream>>>(chunks, master, grad, m, v, (bf16*)shadow_base, lr, b1, b2, eps, wd, bc1, bc2);
+    adamw_kernel<bf16><<<nchunks, 256, 0, c.stream>>>(chunks, master, grad, m, v, (bf16*)shadow_base, scalars, b1, b2, eps, wd);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -115,3 +115,38 @@ def test_error_paths_leave_the_context_usable():
     fp = eng.footprint()
     assert fp["saved_activation_bytes"] > 0 and fp["trainable_params"] == sum(
         int(np.prod(synth.param_shapes(cfg)[n])) for n in O.trainable_names(cfg, params))
+
+
+def test_graph_replay_equals_launch_by_launch():
+    """On a capturable stream the step is captured once and replayed; three steps give bit-identical results to the
+    same three steps enqueued kernel by kernel (AdamW's step-dependent scalars are read from device memory)."""
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    cfg = MINI_BF16
+    images, labels, task_ids, params = synth.make_workload(cfg, peaked=True)
+    shapes = synth.param_shapes(cfg)
+    names = ("head.0.weight", "blocks.5.mlp.fc1.weight", "blocks.3.attn.qkv.weight")
+    results = []
+    for graph in (False, True):
+        eng = Bd.Engine(cfg)
+        eng.set_params(params)
+        eng.set_graph_mode(graph)
+        img = eng.images_to_device(images)
+        lab = torch.as_tensor(labels).cuda()
+        torch.cuda.synchronize()
+        s = torch.cuda.Stream()
+        losses, out = [], None
+        with torch.cuda.stream(s):
+            for _ in range(3):
+                loss, _ = eng.train_step(img, lab, out=out)      # same output buffers from the second step on
+                out = eng.last_out
+                s.synchronize()
+                losses.append(float(loss.cpu()[0]))
+            eng.sync_status()
+            w = {n: eng.get_tensor(n, shapes[n]).cpu().numpy() for n in names}
+        results.append((losses, w))
+        eng.close()
+    assert results[0][0] == results[1][0]
+    assert results[0][0][2] < results[0][0][0]
+    for n in names:
+        assert np.array_equal(results[0][1][n], results[1][1][n]), n
