@@ -253,7 +253,7 @@ const char* bsr_static_last_error(void);
 /* Multi-head self-attention, Eq. 1, on packed projections.  qkv_dev [batch, t, 3, heads, d] in
  * `dtype`; out_dev [batch, t, heads*d]; cls_prob_dev_out optional [batch, heads, t-1] float32: the
  * classification token's row of the attention map without its own column. d must be 64 or less
- * and a multiple of 8.  use_tensor_cores != 0 selects the tcgen05 kernel (bf16, d = 64, t <= 256). */
+ * and a multiple of 8.  use_tensor_cores != 0 selects the tcgen05 kernels (bf16, d = 64). */
 int32_t bsr_attention_forward(const void* qkv_dev, int32_t dtype, int32_t batch, int32_t t, int32_t heads,
                               int32_t d, void* out_dev, float* cls_prob_dev_out, int32_t use_tensor_cores, void* stream);
 

@@ -202,6 +202,191 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict
 }
 
 // ------------------------------------------------------------------------------------------------
+// Forward for longer sequences (T > 256): the keys are walked in blocks of up to 256, twice.  The first walk
+// only computes S = Q K^T per block and keeps the running row maximum and row sum; the second walk recomputes S,
+// forms P = exp(S - max) with the final maximum (so the accumulator never needs rescaling) and adds P V into a
+// separate set of tensor-memory columns.  One CTA per (image, head, 128 queries), one block in flight.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+attn_fwd_tc_long_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict__ out, float* __restrict__ lse,
+                        float* __restrict__ cls_prob, int B, int T, int H, int* status) {
+  extern __shared__ unsigned char smem_dyn[];
+  uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+  constexpr int KB = AT_MAXKEYS;                         // keys per block
+  constexpr uint32_t KV_BYTES = KB * 128;                // 32 KB
+  uint32_t sQ = base, sK = sQ + 2 * AT_BOX_BYTES, sV = sK + KV_BYTES, sP = sV + KV_BYTES;
+  uint32_t bars = sP + 4 * (AT_QROWS * 128);
+  unsigned char* pP = base_ptr + (sP - base);
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  int tid = threadIdx.x, warp = tid >> 5;
+  int bh = blockIdx.y, b = bh / H, h = bh % H;
+  int q0 = blockIdx.x * AT_QROWS;
+  uint32_t tma_bar = bars, mma_bar = bars + 8;
+  if (tid == 0) {
+    abort_flag = 0;
+    mbar_init(tma_bar, 1);
+    mbar_init(mma_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    tmem_alloc(smem_u32(&tmem_slot), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  uint32_t tmem = tmem_slot;
+  constexpr uint32_t C_O = 256;
+  volatile int* abortp = &abort_flag;
+  const float c = 0.125f * 1.4426950408889634f;
+  uint32_t trow = tmem + ((uint32_t)(warp * 32) << 16);
+  int nblk = (T + KB - 1) / KB;
+  int row0 = b * T;
+  uint32_t tma_phase = 0, mma_phase = 0;
+  bool ok = true;
+  float mx = -INFINITY, sum = 0.f;
+  bool cls_row = (q0 == 0 && tid == 0 && cls_prob != nullptr);
+
+  for (int pass = 0; pass < 2 && ok; ++pass) {
+    for (int kb = 0; kb < nblk && ok; ++kb) {
+      int k0 = kb * KB;
+      int keys = min(KB, T - k0);
+      int kpad = (keys + 15) & ~15;
+      int nbox = (kpad + AT_BOX - 1) / AT_BOX;
+      if (tid == 0) {
+        bool first = (pass == 0 && kb == 0);
+        int boxes = nbox * (pass == 1 ? 2 : 1) + (first ? 2 : 0);
+        mbar_expect_tx(tma_bar, boxes * AT_BOX_BYTES);
+        if (first)
+          for (int j = 0; j < 2; ++j) tma_load_2d(sQ + j * AT_BOX_BYTES, &map_qkv, tma_bar, h * AT_D, row0 + q0 + j * AT_BOX);
+        for (int j = 0; j < nbox; ++j) {
+          tma_load_2d(sK + j * AT_BOX_BYTES, &map_qkv, tma_bar, (H + h) * AT_D, row0 + k0 + j * AT_BOX);
+          if (pass == 1) tma_load_2d(sV + j * AT_BOX_BYTES, &map_qkv, tma_bar, (2 * H + h) * AT_D, row0 + k0 + j * AT_BOX);
+        }
+        ok = mbar_wait(tma_bar, tma_phase, abortp);
+        if (ok) {
+          tc_fence_after();
+          uint32_t idesc = make_idesc_mn(AT_QROWS, kpad, false, false);
+#pragma unroll
+          for (int k = 0; k < AT_D / 16; ++k)
+            umma_bf16(tmem, make_desc(sQ + k * 32, 16, 1024), make_desc(sK + k * 32, 16, 1024), idesc, k > 0 ? 1u : 0u);
+          umma_commit(mma_bar);
+        }
+      }
+      tma_phase ^= 1u;
+      ok = mbar_wait(mma_bar, mma_phase, abortp);
+      mma_phase ^= 1u;
+      ok = __all_sync(0xffffffffu, ok);
+      tc_fence_after();
+      if (!ok) break;
+      int nchunk = (keys + 31) >> 5;
+      if (pass == 0) {
+        float bm = -INFINITY;
+        for (int ch = 0; ch < nchunk; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(trow + ch * 32, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (ch * 32 + j < keys) bm = fmaxf(bm, __uint_as_float(r[j]));
+        }
+        float nm = fmaxf(mx, bm);
+        float bs = 0.f;
+        for (int ch = 0; ch < nchunk; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(trow + ch * 32, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (ch * 32 + j < keys) bs += exp2f((__uint_as_float(r[j]) - nm) * c);
+        }
+        sum = sum * exp2f((mx - nm) * c) + bs;
+        mx = nm;
+        tc_fence_before();
+        __syncthreads();               // everyone has read S before the next block's MMA overwrites it
+        tc_fence_after();
+      } else {
+        float mc = mx * c, inv = 1.0f / sum;
+        for (int ch = 0; ch < nchunk; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(trow + ch * 32, r);
+          tmem_ld_wait();
+          float p[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            float e = exp2f(fmaf(__uint_as_float(r[j]), c, -mc));
+            p[j] = (ch * 32 + j < keys) ? e : 0.f;
+          }
+          if (cls_row) {
+            float* cp = cls_prob + ((size_t)b * H + h) * (T - 1);
+            for (int j = 0; j < 32; ++j) {
+              int key = k0 + ch * 32 + j;
+              if (key >= 1 && key < T) cp[key - 1] = p[j] * inv;
+            }
+          }
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            int key8 = ch * 4 + g;
+            if (key8 * 8 < nbox * AT_BOX) {
+              uint4 v;
+              __nv_bfloat162* hh = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) hh[i] = __floats2bfloat162_rn(p[g * 8 + 2 * i], p[g * 8 + 2 * i + 1]);
+              *reinterpret_cast<uint4*>(pP + p_offset(tid, key8)) = v;
+            }
+          }
+        }
+        fence_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        if (tid == 0) {
+          uint32_t idesc = make_idesc_mn(AT_QROWS, AT_D, false, true);
+          for (int k = 0; k < kpad / 16; ++k)
+            umma_bf16(tmem + C_O, make_desc(sP + (k >> 2) * (AT_QROWS * 128) + (k & 3) * 32, 16, 1024),
+                      make_desc(sV + k * (16 * 128), 8192, 1024), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          umma_commit(mma_bar);
+        }
+        ok = mbar_wait(mma_bar, mma_phase, abortp);      // P, K and V of this block are free again
+        mma_phase ^= 1u;
+        ok = __all_sync(0xffffffffu, ok);
+        tc_fence_after();
+      }
+    }
+  }
+  int q = q0 + tid;
+  if (ok) {
+    float inv = 1.0f / sum;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      uint32_t r[32];
+      tmem_ld32(trow + C_O + half * 32, r);
+      tmem_ld_wait();
+      if (q < T) {
+        bf16* orow = out + ((size_t)b * T + q) * H * AT_D + (size_t)h * AT_D + half * 32;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          float v[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[g * 8 + j]) * inv;
+          store16(orow + g * 8, v);
+        }
+      }
+    }
+    if (q < T && lse != nullptr) lse[((size_t)b * H + h) * T + q] = mx * 0.125f + logf(sum);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+  if (tid == 0 && abort_flag && status != nullptr) atomicOr(status, STATUS_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Backward (T <= 128): one CTA of 128 threads per (image, head).  With P = exp(S - lse):
 //   dP = dO V^T;  delta_i = sum_j P_ij dP_ij;  dS = P * (dP - delta) / sqrt(d)
 //   dQ = dS K;  dK = dS^T Q;  dV = P^T dO                      (chain rule through Eq. 1, cf. Eq. 3)
@@ -404,10 +589,22 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
 // Returns 0 when the tensor-core kernel took the problem, non-zero when the caller must use another kernel.
 int attention_fwd_tc(const Ctx& c, const void* qkv, void* out, float* lse, float* cls_prob, int B, int T, int H, int d) {
   using namespace tc;
-  if (c.dtype != 1 || d != AT_D || T > AT_MAXKEYS || T < 1) return -1;
+  if (c.dtype != 1 || d != AT_D || T < 1) return -1;
   if (((uintptr_t)qkv & 15) || ((uintptr_t)out & 15)) return -1;
   CUtensorMap map;
   if (!make_map(&map, qkv, (uint64_t)3 * H * d, (uint64_t)B * T, (uint64_t)3 * H * d, AT_BOX)) return -2;
+  if (T > AT_MAXKEYS) {
+    size_t smem_l = 1024 + 2 * (size_t)AT_BOX_BYTES + 2 * (size_t)AT_MAXKEYS * 128 + 4 * (size_t)(AT_QROWS * 128) + 64;
+    static bool attr_l = false;
+    if (!attr_l) {
+      if (cudaFuncSetAttribute(attn_fwd_tc_long_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_l) != cudaSuccess) return -3;
+      attr_l = true;
+    }
+    dim3 grid_l((T + AT_QROWS - 1) / AT_QROWS, B * H);
+    note_launch(1);
+    attn_fwd_tc_long_kernel<<<grid_l, 128, smem_l, c.stream>>>(map, (bf16*)out, lse, cls_prob, B, T, H, c.status);
+    return 0;
+  }
   int tpad = (T + 15) & ~15;
   int nbox = (tpad + AT_BOX - 1) / AT_BOX;
   size_t p_bytes = (size_t)nbox * (AT_QROWS * 128), qk_bytes = (size_t)(2 + nbox) * AT_BOX_BYTES;

@@ -1202,7 +1202,7 @@ int32_t bsr_attention_forward(const void* qkv, int32_t dtype, int32_t batch, int
   Ctx c = bare_ctx(dtype, stream);
   if (use_tensor_cores) {
     if (attention_fwd_tc(c, qkv, out, nullptr, cls_prob, batch, t, heads, d) != 0)
-      return set_err(g_error, BSR_ERR_UNSUPPORTED, "the tcgen05 attention kernel needs bf16, head dimension 64 and at most 256 tokens");
+      return set_err(g_error, BSR_ERR_UNSUPPORTED, "the tcgen05 attention kernels need bf16 and head dimension 64");
     return check_cuda(nullptr, "bsr_attention_forward");
   }
   if (attention_fwd(c, qkv, out, nullptr, cls_prob, batch, t, heads, d) != 0)
