@@ -64,7 +64,9 @@ typedef struct {
   float ln_eps;
 } bsr_dims;
 
-/* The BSR configuration (Section 4.1, Fig. 2): which blocks train, where and how many tokens drop. */
+/* The BSR configuration (Section 4.1, Fig. 2): which blocks train, where and how many tokens drop.  Any set of
+ * blocks may train (e.g. the paper's 4th, 8th and 12th): frozen blocks after the earliest trainable one pass the
+ * gradient on and get no parameter gradient (Eq. 2, Eq. 8); blocks before it run forward only and keep nothing. */
 typedef struct {
   bsr_dims dims;
   uint32_t trainable_mask;          /* bit l set: block l trains; head and final LayerNorm always train */
@@ -106,8 +108,8 @@ int32_t bsr_workspace_bytes(const bsr_config* cfg_host, size_t* bytes_host);
 
 /* Creates the step engine (Fig. 2).  `workspace_dev` must be 256-byte aligned device memory of at
  * least bsr_workspace_bytes() bytes and must outlive the handle.  Validates the configuration
- * (BSR_ERR_INVALID_ARG), rejects what is not built (BSR_ERR_UNSUPPORTED: a trainable set that is not
- * "the last k blocks"; MoE layers outside bf16 or with dim / mlp_hidden not multiples of 64), zeroes optimiser state and sets the step counter to 0.  Parameters are
+ * (BSR_ERR_INVALID_ARG), rejects what is not built (BSR_ERR_UNSUPPORTED: MoE layers outside bf16 or with
+ * dim / mlp_hidden not multiples of 64), zeroes optimiser state and sets the step counter to 0.  Parameters are
  * undefined until set with bsr_set_param.  On failure *out_host is NULL. */
 int32_t bsr_create(const bsr_config* cfg_host, void* workspace_dev, size_t bytes, bsr_handle** out_host);
 

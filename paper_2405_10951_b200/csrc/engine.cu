@@ -120,13 +120,6 @@ int validate(const bsr_config* cfg, char* err) {
     if (d.dtype != BSR_DTYPE_BF16) return set_err(err, BSR_ERR_UNSUPPORTED, "MoE layers run on the bf16 tensor-core kernels only");
     if (d.dim % 64 != 0 || d.mlp_hidden % 64 != 0) return set_err(err, BSR_ERR_UNSUPPORTED, "MoE layers need dim and mlp_hidden to be multiples of 64");
   }
-  // trainable set must be "the last k blocks"
-  uint32_t m = cfg->trainable_mask;
-  if (m != 0) {
-    int t0 = __builtin_ctz(m);
-    uint32_t suffix = (d.depth >= 32 ? 0xffffffffu : ((1u << d.depth) - 1u)) & ~((1u << t0) - 1u);
-    if (m != suffix) return set_err(err, BSR_ERR_UNSUPPORTED, "trainable blocks must be the last k blocks (frozen blocks inside the gradient path are not built yet)");
-  }
   return BSR_OK;
 }
 
@@ -552,6 +545,7 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
   bool shrinks = k >= 0 && Tf != Ta;
   bool bf = d.dtype == BSR_DTYPE_BF16;
   bool tail = cls_tail(h, l);
+  bool pg = (h->cfg.trainable_mask >> l) & 1u;     // a frozen block inside the gradient path only passes gradients on (Eq. 2)
   size_t es = dtype_size(d.dtype);
   int Mdense = Ma;
   if (tail) { Ma = B; Mf = B; }          // FFN and projection gradients live on the classification rows only
@@ -580,30 +574,39 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
     eg.act = 2;
     eg.aux_in = mb.zg;
     int r1 = gemm_tc_grouped_rows(c, dog, h->wb(l, "moe.fc2.weight"), 1, dzg, 0, cap, F, D, E, mb.tile_expert, eg);
-    int r2 = gemm_tc_grouped_wgrad(c, dog, mb.hg, h->gb(l, "moe.fc2.weight"), cap, D, F, E, mb.seg_start);
-    moe_seg_colsum(c, mb, dog, D, E, h->gb(l, "moe.fc2.bias"));
+    int r2 = 0, r4 = 0;
+    if (pg) {
+      r2 = gemm_tc_grouped_wgrad(c, dog, mb.hg, h->gb(l, "moe.fc2.weight"), cap, D, F, E, mb.seg_start);
+      moe_seg_colsum(c, mb, dog, D, E, h->gb(l, "moe.fc2.bias"));
+    }
     int r3 = gemm_tc_grouped_rows(c, dzg, h->wb(l, "moe.fc1.weight"), 1, dxg, 0, cap, D, F, E, mb.tile_expert, none);
-    int r4 = gemm_tc_grouped_wgrad(c, dzg, mb.xg, h->gb(l, "moe.fc1.weight"), cap, F, D, E, mb.seg_start);
-    moe_seg_colsum(c, mb, dzg, F, E, h->gb(l, "moe.fc1.bias"));
+    if (pg) {
+      r4 = gemm_tc_grouped_wgrad(c, dzg, mb.xg, h->gb(l, "moe.fc1.weight"), cap, F, D, E, mb.seg_start);
+      moe_seg_colsum(c, mb, dzg, F, E, h->gb(l, "moe.fc1.bias"));
+    }
     if (r1 || r2 || r3 || r4) return set_err(h->err, BSR_ERR_CUDA, "grouped GEMM set-up failed (%d, %d, %d, %d)", r1, r2, r3, r4);
     moe_gate_bwd(c, mb, dxg, dwsel, h->wb(l, "moe.gate.weight"), task_ids, tail ? 1 : Tf, d.num_tasks, Mf, D, E, K, dy,
-                 h->at<float>(h->off_m_dsel), h->gb(l, "moe.gate.weight"));
+                 h->at<float>(h->off_m_dsel), pg ? h->gb(l, "moe.gate.weight") : nullptr);
   } else {
   // FFN second layer: dz = (dxo W2) * GELU'(z); dW2 = dxo^T h; db2 = column sums of dxo
   GemmEpilogue eg;
   eg.act = 2;
   eg.aux_in = h->base + bb.z;
   gemm(c, op(dxo), D, 1, h->wb(l, "mlp.fc2.weight"), 1, F, dz, 0, Mf, F, D, eg);
-  gemm(c, op(dxo), 1, D, h->base + bb.hh, 1, F, h->gb(l, "mlp.fc2.weight"), 1, D, F, Mf, none);
-  colsum(cf, dxo.f, Mf, D, csp, h->gb(l, "mlp.fc2.bias"));
+  if (pg) {
+    gemm(c, op(dxo), 1, D, h->base + bb.hh, 1, F, h->gb(l, "mlp.fc2.weight"), 1, D, F, Mf, none);
+    colsum(cf, dxo.f, Mf, D, csp, h->gb(l, "mlp.fc2.bias"));
+  }
   // FFN first layer
   gemm(c, dz, F, 1, h->wb(l, "mlp.fc1.weight"), 1, D, dy, 0, Mf, D, F, none);
-  gemm(c, dz, 1, F, h->base + bb.y2, 1, D, h->gb(l, "mlp.fc1.weight"), 1, F, D, Mf, none);
-  colsum(c, dz, Mf, F, csp, h->gb(l, "mlp.fc1.bias"));
+  if (pg) {
+    gemm(c, dz, 1, F, h->base + bb.y2, 1, D, h->gb(l, "mlp.fc1.weight"), 1, F, D, Mf, none);
+    colsum(c, dz, Mf, F, csp, h->gb(l, "mlp.fc1.bias"));
+  }
   }
   layernorm_bwd(c, dy, 0, h->at<float>(bb.xp), D, h->at<float>(bb.mean2), h->at<float>(bb.rstd2),
                 (const float*)h->wb(l, "norm2.weight"), dxo.f, dxg.f, D, shrinks ? nullptr : dxg.c, lnp,
-                h->gb(l, "norm2.weight"), h->gb(l, "norm2.bias"), Mf, D);
+                pg ? h->gb(l, "norm2.weight") : nullptr, pg ? h->gb(l, "norm2.bias") : nullptr, Mf, D);
   const float* cls_extra = nullptr;
   if (shrinks) {
     gather_fuse_bwd(c, dxg.f, h->base + bb.xp_full, B, Ta - 1, D, k, h->at<int>(bb.kept), h->at<int>(bb.dropped),
@@ -614,14 +617,18 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
   const float* ln1_res = dxp.f;
   if (!tail) {
     gemm(c, op(dxp), D, 1, h->wb(l, "attn.proj.weight"), 1, D, d_o, 0, Ma, D, D, none);
-    gemm(c, op(dxp), 1, D, h->base + bb.o, 1, D, h->gb(l, "attn.proj.weight"), 1, D, D, Ma, none);
-    colsum(cf, dxp.f, Ma, D, csp, h->gb(l, "attn.proj.bias"));
+    if (pg) {
+      gemm(c, op(dxp), 1, D, h->base + bb.o, 1, D, h->gb(l, "attn.proj.weight"), 1, D, D, Ma, none);
+      colsum(cf, dxp.f, Ma, D, csp, h->gb(l, "attn.proj.bias"));
+    }
   } else {
     // B rows: dO_cls = dx'_cls Wo, dWo = dx'_cls^T o_cls; then both gradients go back into zeroed dense tensors
     void* do_cls = h->base + h->off_dy;                      // free at this point
     gemm(c, op(dxp), D, 1, h->wb(l, "attn.proj.weight"), 1, D, do_cls, 0, B, D, D, none);
-    gemm(c, op(dxp), 1, D, h->base + bb.o_cls, 1, D, h->gb(l, "attn.proj.weight"), 1, D, D, B, none);
-    colsum(cf, dxp.f, B, D, csp, h->gb(l, "attn.proj.bias"));
+    if (pg) {
+      gemm(c, op(dxp), 1, D, h->base + bb.o_cls, 1, D, h->gb(l, "attn.proj.weight"), 1, D, D, B, none);
+      colsum(cf, dxp.f, B, D, csp, h->gb(l, "attn.proj.bias"));
+    }
     cudaMemsetAsync(d_o, 0, (size_t)Mdense * D * es, c.stream);
     copy_rows(c.stream, do_cls, (long)D * es, d_o, (long)Ta * D * es, B, (int)(D * es));
     float* dense_res = h->at<float>(h->off_dxp);
@@ -635,11 +642,13 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
   if (rc != 0) return set_err(h->err, BSR_ERR_UNSUPPORTED, "attention backward: %d tokens do not fit this kernel", Ta);
   // QKV projection
   gemm(c, dqkv, 3 * D, 1, h->wb(l, "attn.qkv.weight"), 1, D, dy, 0, Ma, D, 3 * D, none);
-  gemm(c, dqkv, 1, 3 * D, h->base + bb.y1, 1, D, h->gb(l, "attn.qkv.weight"), 1, 3 * D, D, Ma, none);
-  colsum(c, dqkv, Ma, 3 * D, csp, h->gb(l, "attn.qkv.bias"));
+  if (pg) {
+    gemm(c, dqkv, 1, 3 * D, h->base + bb.y1, 1, D, h->gb(l, "attn.qkv.weight"), 1, 3 * D, D, Ma, none);
+    colsum(c, dqkv, Ma, 3 * D, csp, h->gb(l, "attn.qkv.bias"));
+  }
   layernorm_bwd(c, dy, 0, h->at<float>(bb.x_in), D, h->at<float>(bb.mean1), h->at<float>(bb.rstd1),
                 (const float*)h->wb(l, "norm1.weight"), ln1_res, need_dxi ? dxi.f : nullptr, D, need_dxi ? dxi.c : nullptr, lnp,
-                h->gb(l, "norm1.weight"), h->gb(l, "norm1.bias"), Ma, D);
+                pg ? h->gb(l, "norm1.weight") : nullptr, pg ? h->gb(l, "norm1.bias") : nullptr, Ma, D);
   return BSR_OK;
 }
 
@@ -1039,7 +1048,7 @@ int32_t bsr_get_footprint(const bsr_handle* h, bsr_footprint* out) {
     // Table 1 accounting in fp32: Q,K,V + softmax input + GELU input, plus the inputs of the six linear layers
     uint64_t ta = h->sched.ta[l], tf = h->sched.tf[l];
     uint64_t el = 3 * ta * d.dim + (uint64_t)d.heads * ta * ta + tf * d.mlp_hidden;
-    el += 3 * ta * d.dim + 2 * tf * d.dim + tf * d.mlp_hidden;
+    if ((h->cfg.trainable_mask >> l) & 1u) el += 3 * ta * d.dim + 2 * tf * d.dim + tf * d.mlp_hidden;   // inputs of the linear layers
     paper += el * 4 * (uint64_t)h->cfg.max_batch;
   }
   for (auto& t : h->tensors)

@@ -314,6 +314,7 @@ void layernorm_bwd(const Ctx& c, const void* dy, int dy_is_float, const float* x
     launch_ln_bwd<float, bf16>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, dx_copy, partials, rows, D);
   else
     launch_ln_bwd<bf16, bf16>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, dx_copy, partials, rows, D);
+  if (dgamma == nullptr) return;                          // a frozen block in the gradient path: only dx is wanted
   dim3 grid(ceil_div(D, 16), 2);
   reduce_partials_kernel<<<grid, 256, 0, c.stream>>>(partials, groups, D, dgamma, dbeta);
 }

@@ -348,10 +348,10 @@ void moe_gate_bwd(const Ctx& c, const MoeBufs& b, const void* dxg, const float* 
   int blocks = ceil_div((long)M * 32, 256);
   if (c.dtype == 0) {
     moe_gate_bwd_kernel<float><<<blocks, 256, 0, c.stream>>>((const float*)dxg, dw, b.pos, b.eidx, b.ew, (const float*)wg, task_ids, tokens_per_image, M, D, E, K, (float*)dy, dsel_row);
-    moe_gate_wgrad_kernel<float><<<dim3(ceil_div(D, 128), E, tasks), 256, 0, c.stream>>>((const float*)b.xg, dsel_row, b.row_token, b.seg_start, task_ids, tokens_per_image, D, E, dwg);
+    if (dwg != nullptr) moe_gate_wgrad_kernel<float><<<dim3(ceil_div(D, 128), E, tasks), 256, 0, c.stream>>>((const float*)b.xg, dsel_row, b.row_token, b.seg_start, task_ids, tokens_per_image, D, E, dwg);
   } else {
     moe_gate_bwd_kernel<bf16><<<blocks, 256, 0, c.stream>>>((const bf16*)dxg, dw, b.pos, b.eidx, b.ew, (const bf16*)wg, task_ids, tokens_per_image, M, D, E, K, (bf16*)dy, dsel_row);
-    moe_gate_wgrad_kernel<bf16><<<dim3(ceil_div(D, 256), E, tasks), 256, 0, c.stream>>>((const bf16*)b.xg, dsel_row, b.row_token, b.seg_start, task_ids, tokens_per_image, D, E, dwg);
+    if (dwg != nullptr) moe_gate_wgrad_kernel<bf16><<<dim3(ceil_div(D, 256), E, tasks), 256, 0, c.stream>>>((const bf16*)b.xg, dsel_row, b.row_token, b.seg_start, task_ids, tokens_per_image, D, E, dwg);
   }
 }
 

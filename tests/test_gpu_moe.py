@@ -16,6 +16,7 @@ CASES = {
     "moe_is_last_block": MINI_MOE.with_(depth=4, trainable=(2, 3)),
     "top1_single_task": MINI_MOE.with_(num_classes=(10,), moe_top_k=1, moe_experts=8),
     "moe_drop_block_trainable": MINI_MOE.with_(drop_blocks=(3,), trainable=(3, 4)),
+    "frozen_moe_in_gradient_path": MINI_MOE.with_(trainable=(2, 4)),
     "moe_vit_s_batch16": CONFIGS["moe_vit_s"].with_(batch=16),
 }
 

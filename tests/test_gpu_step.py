@@ -20,6 +20,7 @@ FP32_CASES = {
     "keep_one_all_trainable": TINY.with_(keep_num=1, keep_den=1, trainable=(0, 1, 2, 3, 4, 5)),
     "head_only": TINY.with_(trainable=()),
     "half_rate_three_locations": TINY.with_(drop_blocks=(1, 3, 5), keep_num=1, keep_den=2, trainable=(2, 3, 4, 5), batch=5),
+    "interleaved_trainable": TINY.with_(trainable=(1, 3, 5), drop_blocks=(1, 2, 4)),
     "odd_shapes": Config("odd", 20, 4, 96, 3, 3, 136, (7,), 3, (1, 2), (0, 1), 2, 3, dtype="fp32", seed=4),
 }
 
@@ -40,6 +41,7 @@ BF16_CASES = {
     "mini_no_fusion": MINI_BF16.with_(fuse_mode=0),
     "deit_s_batch4": CONFIGS["deit_s"].with_(batch=4),
     "vit_b_batch3": CONFIGS["vit_b"].with_(batch=3),
+    "deit_s_paper_setup": CONFIGS["deit_s"].with_(batch=4, trainable=(3, 7, 11), keep_num=1, keep_den=2),
     "vit_b_384_batch2": CONFIGS["vit_b_384"].with_(batch=2),
 }
 

@@ -67,7 +67,7 @@ def test_workspace_size_and_validation():
     assert status_of(tiny.with_(drop_blocks=(3, 2))) == -1           # not ascending
     assert status_of(tiny.with_(keep_num=11)) == -1                  # keep rate above one
     assert status_of(tiny.with_(trainable=(7,))) == -1               # beyond depth
-    assert status_of(tiny.with_(trainable=(1, 5))) == -2             # not the last k blocks
+    assert Bd.bsr_workspace_bytes(Bd.make_config(tiny.with_(trainable=(1, 5)))) > 0   # frozen blocks inside the gradient path
     assert Bd.bsr_workspace_bytes(Bd.make_config(synth.CONFIGS["moe_vit_s"])) > 0
     assert status_of(synth.CONFIGS["moe_vit_s"].with_(dtype="fp32")) == -2          # MoE runs on the bf16 kernels only
     assert status_of(synth.CONFIGS["moe_vit_s"].with_(moe_top_k=5)) == -1
