@@ -27,12 +27,24 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 
 // Byte offset of element (row, key) in a probability tile stored as 64-key chunks of [128 rows x 128 bytes],
 // 16-byte units XOR-swizzled with the row (the layout TMA produces for a 128-byte-swizzled operand tile).
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float ex2_fast(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t p_offset(int row, int key8) {   // key8: index of a group of 8 keys
   int chunk = key8 >> 3, unit = key8 & 7;
   return (uint32_t)(chunk * (AT_QROWS * 128) + row * 128 + ((unit ^ (row & 7)) << 4));
 }
 
-__global__ void __launch_bounds__(128)
+// 256 threads: warps w and w + 4 share the TMEM lane quarter w & 3 (query rows 32*(w&3) ..) and split the keys
+// (and later the output columns) between them; row maxima and sums are combined through shared memory.
+__global__ void __launch_bounds__(256)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict__ out, float* __restrict__ lse,
                    float* __restrict__ cls_prob, int B, int T, int H, int* status) {
   extern __shared__ unsigned char smem_dyn[];
@@ -46,12 +58,16 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict
   uint32_t sQ = base, sK = sQ + 2 * AT_BOX_BYTES, sP = base;
   uint32_t sV = base + (p_bytes > qk_bytes ? p_bytes : qk_bytes);
   uint32_t tail = sV + nbox * AT_BOX_BYTES;
-  float* cls_buf = reinterpret_cast<float*>(base_ptr + (tail - base));                   // [AT_MAXKEYS + 1]
-  uint32_t bars = tail + (AT_MAXKEYS + 8) * 4;                                           // tma, mma
+  float* cls_buf = reinterpret_cast<float*>(base_ptr + (tail - base));                   // [AT_MAXKEYS]
+  float* red_max = cls_buf + AT_MAXKEYS;                                                 // [2][128]
+  float* red_sum = red_max + 2 * AT_QROWS;                                               // [2][128]
+  uint32_t bars = tail + (AT_MAXKEYS + 4 * AT_QROWS) * 4;                                // tma, mma
   uint32_t tmem_cols = tpad <= 128 ? 128u : 256u;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  int tid = threadIdx.x, warp = tid >> 5;
+  int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int quarter = warp & 3, half = warp >> 2;
+  int row = quarter * 32 + lane;                 // query row inside the tile
   int bh = blockIdx.y, b = bh / H, h = bh % H;
   int q0 = blockIdx.x * AT_QROWS;
   uint32_t tma_bar = bars, mma_bar = bars + 8;
@@ -95,36 +111,52 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict
   ok = __all_sync(0xffffffffu, ok);               // tcgen05.ld below is warp-collective
   tc_fence_after();
 
-  // ---- softmax of this thread's row ------------------------------------------------------------
+  // ---- softmax: this thread's row, this half's chunks of 32 keys -----------------------------------
   const float c = 0.125f * 1.4426950408889634f;          // 1/sqrt(64) * log2(e)
-  uint32_t trow = tmem + ((uint32_t)(warp * 32) << 16);
+  uint32_t trow = tmem + ((uint32_t)(quarter * 32) << 16);
   int nchunk = (T + 31) >> 5;
-  float mx = -INFINITY;
-  if (ok) {
-    for (int ch = 0; ch < nchunk; ++ch) {
+  int split = (nchunk + 1) >> 1;
+  int ch0 = half == 0 ? 0 : split, ch1 = half == 0 ? split : nchunk;
+  bool live = ok && (q0 + quarter * 32 < T);     // warp-uniform: a quarter whose 32 rows all lie past T does no work
+  float pm = -INFINITY;
+  if (live) {
+    for (int ch = ch0; ch < ch1; ++ch) {
       uint32_t r[32];
       tmem_ld32(trow + ch * 32, r);
       tmem_ld_wait();
+      if (ch * 32 + 32 <= T) {
 #pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (ch * 32 + j < T) mx = fmaxf(mx, __uint_as_float(r[j]));
+        for (int j = 0; j < 32; j += 2) pm = fmax3(pm, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (ch * 32 + j < T) pm = fmaxf(pm, __uint_as_float(r[j]));
+      }
     }
   }
-  float sum = 0.f;
-  bool cls_row = (q0 == 0 && tid == 0 && cls_prob != nullptr);
-  if (ok) {
+  red_max[half * AT_QROWS + row] = pm;
+  __syncthreads();
+  float mx = fmaxf(red_max[row], red_max[AT_QROWS + row]);
+  float psum = 0.f;
+  bool cls_row = (q0 == 0 && row == 0 && cls_prob != nullptr);
+  if (live) {
     float mc = mx * c;
-    for (int ch = 0; ch < nchunk; ++ch) {
+    for (int ch = ch0; ch < ch1; ++ch) {
       uint32_t r[32];
       tmem_ld32(trow + ch * 32, r);
       tmem_ld_wait();
       float p[32];
+      if (ch * 32 + 32 <= T) {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        float e = exp2f(fmaf(__uint_as_float(r[j]), c, -mc));
-        p[j] = (ch * 32 + j < T) ? e : 0.f;
-        sum += p[j];
+        for (int j = 0; j < 32; ++j) p[j] = ex2_fast(fmaf(__uint_as_float(r[j]), c, -mc));
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) p[j] = (ch * 32 + j < T) ? ex2_fast(fmaf(__uint_as_float(r[j]), c, -mc)) : 0.f;
       }
+      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+      for (int j = 0; j < 32; j += 4) { s0 += p[j]; s1 += p[j + 1]; s2 += p[j + 2]; s3 += p[j + 3]; }
+      psum += (s0 + s1) + (s2 + s3);
       if (cls_row) {
 #pragma unroll
         for (int j = 0; j < 32; ++j) cls_buf[ch * 32 + j] = p[j];
@@ -137,21 +169,19 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict
           __nv_bfloat162* hh = reinterpret_cast<__nv_bfloat162*>(&v);
 #pragma unroll
           for (int i = 0; i < 4; ++i) hh[i] = __floats2bfloat162_rn(p[g * 8 + 2 * i], p[g * 8 + 2 * i + 1]);
-          *reinterpret_cast<uint4*>(base_ptr + (sP - base) + p_offset(tid, key8)) = v;
+          *reinterpret_cast<uint4*>(base_ptr + (sP - base) + p_offset(row, key8)) = v;
         }
       }
     }
-    // keys between the last 32-chunk and the padded MMA extent must read as zero
-    for (int key8 = nchunk * 4; key8 * 8 < tpad; ++key8)
-      *reinterpret_cast<uint4*>(base_ptr + (sP - base) + p_offset(tid, key8)) = make_uint4(0, 0, 0, 0);
   }
-  float inv = 1.0f / sum;
-  if (cls_row) cls_buf[AT_MAXKEYS] = inv;
+  red_sum[half * AT_QROWS + row] = psum;
   fence_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   ok = ok && !abort_flag;
+  float sum = red_sum[row] + red_sum[AT_QROWS + row];
+  float inv = 1.0f / sum;
 
   // ---- O = P V ----------------------------------------------------------------------------------
   if (tid == 0 && ok) {
@@ -167,29 +197,26 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict
   if (ok) ok = mbar_wait(mma_bar, 1, abortp);
   ok = __all_sync(0xffffffffu, ok);
   tc_fence_after();
-  int q = q0 + tid;
+  int q = q0 + row;
   if (ok) {
+    uint32_t r[32];
+    tmem_ld32(trow + half * 32, r);               // this half's 32 output columns
+    tmem_ld_wait();
+    if (q < T) {
+      bf16* orow = out + ((size_t)b * T + q) * H * AT_D + (size_t)h * AT_D + half * 32;
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      uint32_t r[32];
-      tmem_ld32(trow + half * 32, r);
-      tmem_ld_wait();
-      if (q < T) {
-        bf16* orow = out + ((size_t)b * T + q) * H * AT_D + (size_t)h * AT_D + half * 32;
+      for (int g = 0; g < 4; ++g) {
+        float v[8];
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          float v[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[g * 8 + j]) * inv;
-          store16(orow + g * 8, v);
-        }
+        for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[g * 8 + j]) * inv;
+        store16(orow + g * 8, v);
       }
     }
-    if (q < T && lse != nullptr) lse[((size_t)b * H + h) * T + q] = mx * 0.125f + logf(sum);
+    if (half == 0 && q < T && lse != nullptr) lse[((size_t)b * H + h) * T + q] = mx * 0.125f + logf(sum);
     if (q0 == 0 && cls_prob != nullptr) {
-      float s_inv = cls_buf[AT_MAXKEYS];
+      float s_inv = 1.0f / (red_sum[0] + red_sum[AT_QROWS]);
       float* cp = cls_prob + ((size_t)b * H + h) * (T - 1);
-      for (int j = 1 + tid; j < T; j += 128) cp[j - 1] = cls_buf[j] * s_inv;
+      for (int j = 1 + tid; j < T; j += 256) cp[j - 1] = cls_buf[j] * s_inv;
     }
   }
   tc_fence_before();
@@ -608,7 +635,7 @@ int attention_fwd_tc(const Ctx& c, const void* qkv, void* out, float* lse, float
   int tpad = (T + 15) & ~15;
   int nbox = (tpad + AT_BOX - 1) / AT_BOX;
   size_t p_bytes = (size_t)nbox * (AT_QROWS * 128), qk_bytes = (size_t)(2 + nbox) * AT_BOX_BYTES;
-  size_t smem = 1024 + (p_bytes > qk_bytes ? p_bytes : qk_bytes) + (size_t)nbox * AT_BOX_BYTES + (AT_MAXKEYS + 8) * 4 + 64;
+  size_t smem = 1024 + (p_bytes > qk_bytes ? p_bytes : qk_bytes) + (size_t)nbox * AT_BOX_BYTES + (AT_MAXKEYS + 4 * AT_QROWS) * 4 + 64;
   static size_t attr = 0;
   if (smem > attr) {
     if (cudaFuncSetAttribute(attn_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -3;
@@ -616,7 +643,7 @@ int attention_fwd_tc(const Ctx& c, const void* qkv, void* out, float* lse, float
   }
   dim3 grid((T + AT_QROWS - 1) / AT_QROWS, B * H);
   note_launch(1);
-  attn_fwd_tc_kernel<<<grid, 128, smem, c.stream>>>(map, (bf16*)out, lse, cls_prob, B, T, H, c.status);
+  attn_fwd_tc_kernel<<<grid, 256, smem, c.stream>>>(map, (bf16*)out, lse, cls_prob, B, T, H, c.status);
   return 0;
 }
 

@@ -473,12 +473,14 @@ __global__ void head_wgrad_kernel(HeadDev h, const float* __restrict__ xn, const
   int n = h.ncls[t];
   if (i >= n * (h.D + 1)) return;
   int cls = i / (h.D + 1), d = i % (h.D + 1);
+  // branch-free and unrolled: the loads of eight images are in flight together; the sum still runs in image order
   float s = 0.f;
+#pragma unroll 8
   for (int b = 0; b < B; ++b) {
     int tb = task_ids ? task_ids[b] : 0;
-    if (tb != t) continue;
-    float g = dlogits[(size_t)b * h.cmax + cls];
-    s += (d < h.D) ? g * xn[(size_t)b * h.D + d] : g;
+    float g = (tb == t) ? dlogits[(size_t)b * h.cmax + cls] : 0.f;
+    float x = (d < h.D) ? xn[(size_t)b * h.D + d] : 1.f;
+    s = fmaf(g, x, s);
   }
   if (d < h.D) h.dw[t][(size_t)cls * h.D + d] = s;
   else h.db[t][cls] = s;

@@ -16,37 +16,72 @@ struct Epi {
   int act;
 };
 
-// erf by the rational approximation 7.1.26 of Abramowitz and Stegun (|error| < 1.5e-7, about 1e-6 with the fast
-// reciprocal and exponential used here): far below the bf16 resolution of the values this epilogue produces.
-// Also returns e = exp(-x^2), which the derivative of GELU needs.
-__device__ __forceinline__ float erf_fast(float x, float& e) {
-  float ax = fabsf(x);
-  float t = __fdividef(1.0f, fmaf(0.3275911f, ax, 1.0f));
-  e = __expf(-ax * ax);
-  float poly = t * (0.254829592f + t * (-0.284496736f + t * (1.421413741f + t * (-1.453152027f + t * 1.061405429f))));
-  return copysignf(1.0f - poly * e, x);
+// Two fp32 lanes per instruction (fma.rn.f32x2 and friends): halves the issue slots of the polynomial below.
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
 }
-// GELU(z) = z * Phi(z) with Phi(z) - 1/2 as an odd polynomial of degree 17 on |z| <= 4 (clamped beyond), fitted
-// to erf in double precision: |error of Phi| < 3e-5 everywhere (4e-6 inside the interval), no special-function
-// unit involved.  Used where the result is rounded to bf16 (resolution 4e-3 relative).
-__device__ __forceinline__ float gelu_fast(float z) {
-  float zc = fminf(fmaxf(z, -4.0f), 4.0f);
-  float u = zc * zc;
-  float p = 8.065214468500059e-11f;
-  p = fmaf(p, u, -7.004623547857136e-09f);
-  p = fmaf(p, u, 2.716460869578441e-07f);
-  p = fmaf(p, u, -6.295422281255014e-06f);
-  p = fmaf(p, u, 9.891138324746862e-05f);
-  p = fmaf(p, u, -0.001133936457335949f);
-  p = fmaf(p, u, 0.009877507574856281f);
-  p = fmaf(p, u, -0.0664106160402298f);
-  p = fmaf(p, u, 0.3989226818084717f);
-  return z * fmaf(zc, p, 0.5f);
+__device__ __forceinline__ void unpack2(uint64_t r, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(r)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
 }
-__device__ __forceinline__ float gelu_grad_fast(float z) {
-  float e;
-  float er = erf_fast(z * 0.70710678118654752f, e);
-  return 0.5f * (1.0f + er) + z * 0.39894228040143268f * e;
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t dup2(float a) { return pack2(a, a); }
+
+// Phi(z) - 1/2 = z * q(z^2) with q a polynomial of degree 8 fitted to erf in double precision on |z| <= 4:
+// |error of Phi| < 3e-5 everywhere (4e-6 inside the interval), no special-function unit involved.  Returns
+// q(min(z^2, 16)) for two values: beyond |z| = 4 the product z * q(16) leaves [-1/2, 1/2], so that adding 1/2 with
+// saturation pins Phi to 0 or 1.  Used where the result is rounded to bf16 (resolution 4e-3 relative).
+__device__ __forceinline__ void phi_slope2(float u0, float u1, float& q0, float& q1) {
+  uint64_t u = pack2(fminf(u0, 16.0f), fminf(u1, 16.0f));
+  uint64_t q = dup2(8.065214468500059e-11f);
+  q = fma2(q, u, dup2(-7.004623547857136e-09f));
+  q = fma2(q, u, dup2(2.716460869578441e-07f));
+  q = fma2(q, u, dup2(-6.295422281255014e-06f));
+  q = fma2(q, u, dup2(9.891138324746862e-05f));
+  q = fma2(q, u, dup2(-0.001133936457335949f));
+  q = fma2(q, u, dup2(0.009877507574856281f));
+  q = fma2(q, u, dup2(-0.0664106160402298f));
+  q = fma2(q, u, dup2(0.3989226818084717f));
+  unpack2(q, q0, q1);
+}
+// z <- GELU(z) = z * Phi(z), two values.
+__device__ __forceinline__ void gelu_fast2(float& z0, float& z1) {
+  float u0, u1, q0, q1;
+  uint64_t z = pack2(z0, z1);
+  unpack2(mul2(z, z), u0, u1);
+  phi_slope2(u0, u1, q0, q1);
+  z0 *= __saturatef(fmaf(z0, q0, 0.5f));
+  z1 *= __saturatef(fmaf(z1, q1, 0.5f));
+}
+// g <- g * GELU'(z), two values: GELU'(z) = Phi(z) + z * phi(z), with the density phi(z) = exp(-z^2 / 2) / sqrt(2 pi)
+// from one exponential of the unclamped square.
+__device__ __forceinline__ void gelu_grad_mul2(float& g0, float& g1, float z0, float z1) {
+  float u0, u1, q0, q1, d0, d1, e0, e1;
+  uint64_t z = pack2(z0, z1);
+  unpack2(mul2(z, z), u0, u1);
+  phi_slope2(u0, u1, q0, q1);
+  const float kh = -0.5f * 1.4426950408889634f;          // exp(-u / 2) = 2^(kh u)
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(u0 * kh));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(u1 * kh));
+  unpack2(mul2(z, dup2(0.39894228040143268f)), d0, d1);
+  g0 *= fmaf(d0, e0, __saturatef(fmaf(z0, q0, 0.5f)));
+  g1 *= fmaf(d1, e1, __saturatef(fmaf(z1, q1, 0.5f)));
+}
+
+// 16-byte global load of data that is read once (residual stream, stored pre-activations).
+template <typename T>
+__device__ __forceinline__ uint4 ld_stream(const T* p) {
+  uint4 x;
+  asm volatile("ld.global.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(x.x), "=r"(x.y), "=r"(x.z), "=r"(x.w) : "l"(p));
+  return x;
 }
 
 // A warp moves a 32-row x 32-column chunk between registers (lane = row, v[32] = the row's columns) and global
@@ -59,20 +94,27 @@ struct ChunkIO {
   static constexpr int ROWS_PER_PASS = 32 / UNITS;
   __device__ static uint32_t slot(int r, int u) { return (uint32_t)(r * 128 + ((u ^ (r & 7)) << 4)); }
 
+  // All global loads are issued before the first shared-memory store: the staging pointer may alias anything as
+  // far as the compiler knows, so a load placed after a store could not be moved ahead of it.
   __device__ static void load(const T* g, int ld, int row0, int col0, int M, int N, unsigned char* st, int lane, float* v) {
+    uint4 x[UNITS];
 #pragma unroll
     for (int i = 0; i < UNITS; ++i) {
       int r = i * ROWS_PER_PASS + lane / UNITS, u = lane % UNITS;
       int col = col0 + u * E;
-      uint4 x = make_uint4(0, 0, 0, 0);
-      if (row0 + r < M && col < N) x = *reinterpret_cast<const uint4*>(g + (size_t)(row0 + r) * ld + col);
-      *reinterpret_cast<uint4*>(st + slot(r, u)) = x;
+      x[i] = make_uint4(0, 0, 0, 0);
+      if (row0 + r < M && col < N) x[i] = ld_stream(g + (size_t)(row0 + r) * ld + col);
+    }
+#pragma unroll
+    for (int i = 0; i < UNITS; ++i) {
+      int r = i * ROWS_PER_PASS + lane / UNITS, u = lane % UNITS;
+      *reinterpret_cast<uint4*>(st + slot(r, u)) = x[i];
     }
     __syncwarp();
 #pragma unroll
     for (int u = 0; u < UNITS; ++u) {
-      uint4 x = *reinterpret_cast<const uint4*>(st + slot(lane, u));
-      unpack(x, v + u * E);
+      uint4 y = *reinterpret_cast<const uint4*>(st + slot(lane, u));
+      unpack(y, v + u * E);
     }
     __syncwarp();
   }
@@ -80,12 +122,17 @@ struct ChunkIO {
 #pragma unroll
     for (int u = 0; u < UNITS; ++u) *reinterpret_cast<uint4*>(st + slot(lane, u)) = pack(v + u * E);
     __syncwarp();
+    uint4 x[UNITS];
+#pragma unroll
+    for (int i = 0; i < UNITS; ++i) {
+      int r = i * ROWS_PER_PASS + lane / UNITS, u = lane % UNITS;
+      x[i] = *reinterpret_cast<const uint4*>(st + slot(r, u));
+    }
 #pragma unroll
     for (int i = 0; i < UNITS; ++i) {
       int r = i * ROWS_PER_PASS + lane / UNITS, u = lane % UNITS;
       int col = col0 + u * E;
-      if (row0 + r < M && col < N)
-        *reinterpret_cast<uint4*>(g + (size_t)(row0 + r) * ld + col) = *reinterpret_cast<const uint4*>(st + slot(r, u));
+      if (row0 + r < M && col < N) *reinterpret_cast<uint4*>(g + (size_t)(row0 + r) * ld + col) = x[i];
     }
     __syncwarp();
   }
@@ -131,12 +178,12 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t* r, const Epi& ep,
     if (ep.act == 1) {
       if (ep.aux_out != nullptr) ChunkIO<TOut>::store((TOut*)ep.aux_out, N, row0, col0, M, N, st, lane, v);
 #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = gelu_fast(v[j]);
+      for (int j = 0; j < 32; j += 2) gelu_fast2(v[j], v[j + 1]);
     } else if (ep.act == 2) {
       float z[32];
       ChunkIO<bf16>::load((const bf16*)ep.aux_in, N, row0, col0, M, N, st, lane, z);
 #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] *= gelu_grad_fast(z[j]);
+      for (int j = 0; j < 32; j += 2) gelu_grad_mul2(v[j], v[j + 1], z[j], z[j + 1]);
     }
     if (ep.residual != nullptr) {
       float rr[32];
@@ -223,16 +270,16 @@ __device__ __forceinline__ void epilogue_warp_tile(LoadTmem load_tmem, const Epi
     if (ep.act == 1) {
       if (ep.aux_out != nullptr) ChunkIO<TOut>::store((TOut*)ep.aux_out, N, row0, col0, M, N, st_out, lane, v);
 #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = gelu_fast(v[j]);
+      for (int j = 0; j < 32; j += 2) gelu_fast2(v[j], v[j + 1]);
     } else if (ep.act == 2) {
       if (pre_aux) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] *= gelu_grad_fast(a[j]);
+        for (int j = 0; j < 32; j += 2) gelu_grad_mul2(v[j], v[j + 1], a[j], a[j + 1]);
       } else {
         float z[32];
         ChunkIO<bf16>::load((const bf16*)ep.aux_in, N, row0, col0, M, N, st_out, lane, z);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] *= gelu_grad_fast(z[j]);
+        for (int j = 0; j < 32; j += 2) gelu_grad_mul2(v[j], v[j + 1], z[j], z[j + 1]);
       }
     }
     if (pre_res) {
