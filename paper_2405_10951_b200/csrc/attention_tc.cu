@@ -1,11 +1,9 @@
 // Multi-head self-attention (paper Eq. 1) on the tcgen05 tensor cores for bf16, head dimension 64.
 //
-// Forward (T <= 256 keys): one CTA of 128 threads per (image, head, 128-query tile).
-//   TMA loads Q, K, V tiles of the packed projections [B*T, 3*H*64] into 128-byte-swizzled shared memory;
-//   S = Q K^T goes to tensor memory (one tcgen05.mma group, N = T rounded up to 16);
-//   each thread owns one query row: row maximum, exp2, row sum in float from tcgen05.ld; the probabilities
-//   are written as bf16 into shared memory in the same swizzled layout an operand tile has;
-//   O = P V accumulates over the S columns that are no longer needed; the epilogue scales by 1 / row sum.
+// Forward (T <= 256 keys): a persistent, warp-specialised kernel (see attn_fwd_ws_kernel): TMA loads Q, K, V tiles of
+//   the packed projections [B*T, 3*H*64] into 128-byte-swizzled shared memory; S = Q K^T goes to tensor memory; a
+//   thread owns (half of) a query row: row maximum, exp2, row sum in float from tcgen05.ld; the probabilities go back
+//   into tensor memory as bf16 and O = P V reads them from there; the epilogue scales by 1 / row sum.
 //   The classification token's row (query 0) is also written out as probabilities: these are the token
 //   importance scores of Eq. 6.
 // Rows and keys beyond T inside a tile belong to the next image (or are zero-filled past the tensor's end):
@@ -42,188 +40,301 @@ __device__ __forceinline__ uint32_t p_offset(int row, int key8) {   // key8: ind
   return (uint32_t)(chunk * (AT_QROWS * 128) + row * 128 + ((unit ^ (row & 7)) << 4));
 }
 
-// 256 threads: warps w and w + 4 share the TMEM lane quarter w & 3 (query rows 32*(w&3) ..) and split the keys
-// (and later the output columns) between them; row maxima and sums are combined through shared memory.
-__global__ void __launch_bounds__(256)
-attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict__ out, float* __restrict__ lse,
-                   float* __restrict__ cls_prob, int B, int T, int H, int* status) {
+// ------------------------------------------------------------------------------------------------
+// Forward for T <= 256, persistent and warp-specialised: one CTA per SM walks (image, head) pairs.
+//   loader warp : TMA (one lane): K and V of a pair into a ring of slots, each 128-query tile of Q into another
+//                 ring, running ahead of the tensor core as far as the slots allow;
+//   NBUF softmax groups, one per accumulator buffer in tensor memory, each working on every NBUF-th tile.  A group's
+//                 first thread also issues the group's MMAs: S = Q K^T for the group's next tile as soon as the
+//                 previous O has been read, and O = P V as soon as the group has written P.  A thread owns (half
+//                 of) a query row: row maximum and exp2 from tcgen05.ld, probabilities packed to bf16 and written
+//                 back with tcgen05.st over the S columns already consumed (P never goes through shared memory,
+//                 the second MMA reads it from tensor memory), then O scaled by the row sum and stored.
+// NBUF is 4, 3 or 2 for up to 128, 160 or 256 keys; with two groups a group has eight warps, two per lane quarter
+// splitting the keys (and the output columns).  Accumulator buffer layout (columns): S at 0 .. tpad-1 (fp32), P (bf16
+// pairs) over S columns its writer has already consumed, O in the last 64 columns of the buffer, beyond P.
+// ------------------------------------------------------------------------------------------------
+constexpr int WS_QSLOTS = 3;
+constexpr int WS_Q_BYTES = 2 * AT_BOX_BYTES;
+constexpr int WS_MAXBUF = 4, WS_MAXKV = 6;
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ void group_sync(int id, int threads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory"); }
+// mbar_wait that gives up at once when another role already has: after a failure the groups keep walking their
+// tiles (their named barriers need every thread) and every further wait must return quickly.
+__device__ __forceinline__ bool mbar_wait_q(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (*abort_flag) return false;
+  return mbar_wait(bar, parity, abort_flag);
+}
+
+template <int NBUF>
+__global__ void __launch_bounds__((NBUF == 2 ? 19 : 4 * NBUF + 3) * 32, 1)
+attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv, bf16* __restrict__ out,
+                   float* __restrict__ lse, float* __restrict__ cls_prob, int B, int T, int H, int kvslots, int* status) {
+  constexpr int GW = NBUF == 2 ? 8 : 4;                         // warps per softmax group
+  constexpr int GT = GW * 32;
+  constexpr uint32_t BUF_COLS = NBUF == 2 ? 256u : (NBUF == 3 ? 160u : 128u);
+  constexpr uint32_t O_COL = BUF_COLS - 64u;                                 // 192, 96, 64
   extern __shared__ unsigned char smem_dyn[];
   uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
-  int tpad = (T + 15) & ~15;                     // MMA N
-  int nbox = (tpad + AT_BOX - 1) / AT_BOX;       // 64-key boxes of K and V, 64-key chunks of P
-  // Q and K are dead once S = Q K^T has completed, so the probability tile P reuses their space (plus a tail).
-  uint32_t p_bytes = nbox * (AT_QROWS * 128);
-  uint32_t qk_bytes = (2 + nbox) * AT_BOX_BYTES;
-  uint32_t sQ = base, sK = sQ + 2 * AT_BOX_BYTES, sP = base;
-  uint32_t sV = base + (p_bytes > qk_bytes ? p_bytes : qk_bytes);
-  uint32_t tail = sV + nbox * AT_BOX_BYTES;
-  float* cls_buf = reinterpret_cast<float*>(base_ptr + (tail - base));                   // [AT_MAXKEYS]
-  float* red_max = cls_buf + AT_MAXKEYS;                                                 // [2][128]
-  float* red_sum = red_max + 2 * AT_QROWS;                                               // [2][128]
-  uint32_t bars = tail + (AT_MAXKEYS + 4 * AT_QROWS) * 4;                                // tma, mma
-  uint32_t tmem_cols = tpad <= 128 ? 128u : 256u;
+  const int tpad = (T + 15) & ~15;
+  const int nqt = (T + AT_QROWS - 1) / AT_QROWS;
+  const uint32_t kv_bytes = tpad * 128;                          // one of K, V: tpad rows of 64 bf16
+  const uint32_t sQ = base, sKV = sQ + WS_QSLOTS * WS_Q_BYTES;
+  const uint32_t tail = sKV + kvslots * 2 * kv_bytes;
+  float* cls_buf = reinterpret_cast<float*>(base_ptr + (tail - base));     // [NBUF][AT_MAXKEYS]
+  float* red = cls_buf + WS_MAXBUF * AT_MAXKEYS;                            // [NBUF][max, sum][2 halves][128 rows]
+  const uint32_t bars = tail + (WS_MAXBUF * AT_MAXKEYS + WS_MAXBUF * 4 * AT_QROWS) * 4;
+  auto q_full = [&](int s) { return bars + 8u * s; };
+  auto q_empty = [&](int s) { return bars + 8u * (4 + s); };
+  auto kv_full = [&](int s) { return bars + 8u * (8 + s); };
+  auto kv_empty = [&](int s) { return bars + 8u * (16 + s); };
+  auto s_full = [&](int b) { return bars + 8u * (24 + b); };
+  auto o_full = [&](int b) { return bars + 8u * (28 + b); };
+  auto p_full = [&](int b) { return bars + 8u * (32 + b); };
+  auto t_empty = [&](int b) { return bars + 8u * (36 + b); };
+  auto token = [&](int b) { return bars + 8u * (40 + b); };
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  int quarter = warp & 3, half = warp >> 2;
-  int row = quarter * 32 + lane;                 // query row inside the tile
-  int bh = blockIdx.y, b = bh / H, h = bh % H;
-  int q0 = blockIdx.x * AT_QROWS;
-  uint32_t tma_bar = bars, mma_bar = bars + 8;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int pairs = B * H;
+  constexpr int LOADER = NBUF * GW;                             // then the two MMA issuer warps
 
   if (tid == 0) {
     abort_flag = 0;
-    mbar_init(tma_bar, 1);
-    mbar_init(mma_bar, 1);
+    for (int s = 0; s < WS_QSLOTS; ++s) { mbar_init(q_full(s), 1); mbar_init(q_empty(s), 1); }
+    for (int s = 0; s < WS_MAXKV; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), nqt); }
+    for (int b = 0; b < WS_MAXBUF; ++b) {
+      mbar_init(s_full(b), 1); mbar_init(o_full(b), 1); mbar_init(p_full(b), GW); mbar_init(t_empty(b), GW); mbar_init(token(b), 1);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 0) {
-    tmem_alloc(smem_u32(&tmem_slot), tmem_cols);
+  if (warp == LOADER) {
+    tmem_alloc(smem_u32(&tmem_slot), 512);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  uint32_t tmem = tmem_slot;
+  const uint32_t tmem = tmem_slot;
   volatile int* abortp = &abort_flag;
-  bool ok = true;
 
-  if (tid == 0) {
-    mbar_expect_tx(tma_bar, (2 + 2 * nbox) * AT_BOX_BYTES);
-    int row0 = b * T;
-    for (int j = 0; j < 2; ++j) tma_load_2d(sQ + j * AT_BOX_BYTES, &map_qkv, tma_bar, h * AT_D, row0 + q0 + j * AT_BOX);
-    for (int j = 0; j < nbox; ++j) {
-      tma_load_2d(sK + j * AT_BOX_BYTES, &map_qkv, tma_bar, (H + h) * AT_D, row0 + j * AT_BOX);
-      tma_load_2d(sV + j * AT_BOX_BYTES, &map_qkv, tma_bar, (2 * H + h) * AT_D, row0 + j * AT_BOX);
-    }
-    ok = mbar_wait(tma_bar, 0, abortp);
-    if (ok) {
-      tc_fence_after();
-      uint32_t idesc = make_idesc_mn(AT_QROWS, tpad, false, false);
-#pragma unroll
-      for (int k = 0; k < AT_D / 16; ++k)
-        umma_bf16(tmem, make_desc(sQ + k * 32, 16, 1024), make_desc(sK + k * 32, 16, 1024), idesc, k > 0 ? 1u : 0u);
-      umma_commit(mma_bar);
-    }
-  }
-  ok = mbar_wait(mma_bar, 0, abortp);
-  ok = __all_sync(0xffffffffu, ok);               // tcgen05.ld below is warp-collective
-  tc_fence_after();
-
-  // ---- softmax: this thread's row, this half's chunks of 32 keys -----------------------------------
-  const float c = 0.125f * 1.4426950408889634f;          // 1/sqrt(64) * log2(e)
-  uint32_t trow = tmem + ((uint32_t)(quarter * 32) << 16);
-  int nchunk = (T + 31) >> 5;
-  int split = (nchunk + 1) >> 1;
-  int ch0 = half == 0 ? 0 : split, ch1 = half == 0 ? split : nchunk;
-  bool live = ok && (q0 + quarter * 32 < T);     // warp-uniform: a quarter whose 32 rows all lie past T does no work
-  float pm = -INFINITY;
-  if (live) {
-    for (int ch = ch0; ch < ch1; ++ch) {
-      uint32_t r[32];
-      tmem_ld32(trow + ch * 32, r);
-      tmem_ld_wait();
-      if (ch * 32 + 32 <= T) {
-#pragma unroll
-        for (int j = 0; j < 32; j += 2) pm = fmax3(pm, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
-      } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (ch * 32 + j < T) pm = fmaxf(pm, __uint_as_float(r[j]));
+  if (warp == LOADER) {
+    // ------------------------------- TMA loader ---------------------------------
+    if (lane == 0) {
+      int i = 0, n = 0;
+      bool ok = true;
+      for (int bh = blockIdx.x; bh < pairs && ok; bh += gridDim.x, ++n) {
+        int b = bh / H, h = bh % H, row0 = b * T;
+        int ks = n % kvslots;
+        if (!mbar_wait(kv_empty(ks), ((n / kvslots) & 1) ^ 1u, abortp)) { ok = false; break; }
+        mbar_expect_tx(kv_full(ks), 2 * kv_bytes);
+        uint32_t sK = sKV + ks * 2 * kv_bytes, sV = sK + kv_bytes;
+        tma_load_2d(sK, &map_kv, kv_full(ks), (H + h) * AT_D, row0);
+        tma_load_2d(sV, &map_kv, kv_full(ks), (2 * H + h) * AT_D, row0);
+        for (int qt = 0; qt < nqt; ++qt, ++i) {
+          int qs = i % WS_QSLOTS;
+          if (!mbar_wait(q_empty(qs), ((i / WS_QSLOTS) & 1) ^ 1u, abortp)) { ok = false; break; }
+          mbar_expect_tx(q_full(qs), WS_Q_BYTES);
+          tma_load_2d(sQ + qs * WS_Q_BYTES, &map_q, q_full(qs), h * AT_D, row0 + qt * AT_QROWS);
+        }
+      }
+      if (!ok) {                      // copies already issued still land: give them a bounded time before the CTA leaves
+        unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 1000000ull) {}
       }
     }
-  }
-  red_max[half * AT_QROWS + row] = pm;
-  __syncthreads();
-  float mx = fmaxf(red_max[row], red_max[AT_QROWS + row]);
-  float psum = 0.f;
-  bool cls_row = (q0 == 0 && row == 0 && cls_prob != nullptr);
-  if (live) {
-    float mc = mx * c;
-    for (int ch = ch0; ch < ch1; ++ch) {
-      uint32_t r[32];
-      tmem_ld32(trow + ch * 32, r);
-      tmem_ld_wait();
-      float p[32];
-      if (ch * 32 + 32 <= T) {
+  } else if (warp == LOADER + 1) {
+    // ------------------------------- S = Q K^T issuer ---------------------------
+    if (lane == 0) {
+      const uint32_t idesc_s = make_idesc_mn(AT_QROWS, tpad, false, false);
+      int i = 0, n = 0;
+      bool ok = true;
+      for (int bh = blockIdx.x; bh < pairs && ok; bh += gridDim.x, ++n) {
+        int ks = n % kvslots;
+        for (int qt = 0; qt < nqt; ++qt, ++i) {
+          int qs = i % WS_QSLOTS, buf = i % NBUF;
+          if (qt == 0 && !mbar_wait(kv_full(ks), (n / kvslots) & 1, abortp)) { ok = false; break; }
+          if (!mbar_wait(q_full(qs), (i / WS_QSLOTS) & 1, abortp)) { ok = false; break; }
+          if (!mbar_wait(t_empty(buf), ((i / NBUF) & 1) ^ 1u, abortp)) { ok = false; break; }
+          tc_fence_after();
+          uint32_t sq = sQ + qs * WS_Q_BYTES, sK = sKV + ks * 2 * kv_bytes;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) p[j] = ex2_fast(fmaf(__uint_as_float(r[j]), c, -mc));
-      } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) p[j] = (ch * 32 + j < T) ? ex2_fast(fmaf(__uint_as_float(r[j]), c, -mc)) : 0.f;
-      }
-      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-      for (int j = 0; j < 32; j += 4) { s0 += p[j]; s1 += p[j + 1]; s2 += p[j + 2]; s3 += p[j + 3]; }
-      psum += (s0 + s1) + (s2 + s3);
-      if (cls_row) {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) cls_buf[ch * 32 + j] = p[j];
-      }
-#pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        int key8 = ch * 4 + g;
-        if (key8 * 8 < nbox * AT_BOX) {
-          uint4 v;
-          __nv_bfloat162* hh = reinterpret_cast<__nv_bfloat162*>(&v);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) hh[i] = __floats2bfloat162_rn(p[g * 8 + 2 * i], p[g * 8 + 2 * i + 1]);
-          *reinterpret_cast<uint4*>(base_ptr + (sP - base) + p_offset(row, key8)) = v;
+          for (int k = 0; k < AT_D / 16; ++k)
+            umma_bf16(tmem + buf * BUF_COLS, make_desc(sq + k * 32, 16, 1024), make_desc(sK + k * 32, 16, 1024), idesc_s, k > 0 ? 1u : 0u);
+          umma_commit(s_full(buf));
+          umma_commit(q_empty(qs));
         }
       }
     }
-  }
-  red_sum[half * AT_QROWS + row] = psum;
-  fence_async_smem();
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  ok = ok && !abort_flag;
-  float sum = red_sum[row] + red_sum[AT_QROWS + row];
-  float inv = 1.0f / sum;
-
-  // ---- O = P V ----------------------------------------------------------------------------------
-  if (tid == 0 && ok) {
-    uint32_t idesc = make_idesc_mn(AT_QROWS, AT_D, false, true);
-    int ksteps = tpad / 16;
-    for (int k = 0; k < ksteps; ++k) {
-      uint64_t da = make_desc(sP + (k >> 2) * (AT_QROWS * 128) + (k & 3) * 32, 16, 1024);
-      uint64_t db = make_desc(sV + k * (16 * 128), 8192, 1024);
-      umma_bf16(tmem, da, db, idesc, k > 0 ? 1u : 0u);
-    }
-    umma_commit(mma_bar);
-  }
-  if (ok) ok = mbar_wait(mma_bar, 1, abortp);
-  ok = __all_sync(0xffffffffu, ok);
-  tc_fence_after();
-  int q = q0 + row;
-  if (ok) {
-    uint32_t r[32];
-    tmem_ld32(trow + half * 32, r);               // this half's 32 output columns
-    tmem_ld_wait();
-    if (q < T) {
-      bf16* orow = out + ((size_t)b * T + q) * H * AT_D + (size_t)h * AT_D + half * 32;
-#pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        float v[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[g * 8 + j]) * inv;
-        store16(orow + g * 8, v);
+  } else if (warp == LOADER + 2) {
+    // ------------------------------- O = P V issuer -----------------------------
+    if (lane == 0) {
+      const uint32_t idesc_o = make_idesc_mn(AT_QROWS, AT_D, false, true);
+      const int ksteps = tpad / 16;
+      const int chs2 = ((((T + 31) >> 5) + 1) >> 1) * 2;       // first 16-key step of the second half's probabilities
+      int i = 0, n = 0;
+      bool ok = true;
+      for (int bh = blockIdx.x; bh < pairs && ok; bh += gridDim.x, ++n) {
+        int ks = n % kvslots;
+        for (int qt = 0; qt < nqt; ++qt, ++i) {
+          int pb = i % NBUF;
+          if (!mbar_wait(p_full(pb), (i / NBUF) & 1, abortp)) { ok = false; break; }
+          tc_fence_after();
+          uint32_t tb = tmem + pb * BUF_COLS;
+          uint32_t sV = sKV + ks * 2 * kv_bytes + kv_bytes;
+          for (int k = 0; k < ksteps; ++k)
+            umma_bf16_ts(tb + O_COL, tb + 8 * k + ((GW == 8 && k >= chs2) ? 8 * chs2 : 0), make_desc(sV + k * (16 * 128), 8192, 1024),
+                         idesc_o, k > 0 ? 1u : 0u);
+          umma_commit(o_full(pb));
+          umma_commit(kv_empty(ks));
+        }
       }
     }
-    if (half == 0 && q < T && lse != nullptr) lse[((size_t)b * H + h) * T + q] = mx * 0.125f + logf(sum);
-    if (q0 == 0 && cls_prob != nullptr) {
-      float s_inv = 1.0f / (red_sum[0] + red_sum[AT_QROWS]);
-      float* cp = cls_prob + ((size_t)b * H + h) * (T - 1);
-      for (int j = 1 + tid; j < T; j += 256) cp[j - 1] = cls_buf[j] * s_inv;
+  } else {
+    // ------------------------------- softmax groups -----------------------------
+    const int g = warp / GW, gw = warp % GW;
+    const int quarter = gw & 3, half = gw >> 2;            // half: which part of the keys / output columns (eight-warp groups)
+    const bool leader = (gw == 0 && lane == 0);
+    const int row = quarter * 32 + lane;
+    const float c = 0.125f * 1.4426950408889634f;          // 1/sqrt(64) * log2(e)
+    const uint32_t tbuf = tmem + g * BUF_COLS;
+    const uint32_t trow = tbuf + ((uint32_t)(quarter * 32) << 16);
+    const int nchunk = (T + 31) >> 5;
+    const int ch0 = (GW == 8 && half == 1) ? (nchunk + 1) >> 1 : 0;
+    const int ch1 = (GW == 8 && half == 0) ? (nchunk + 1) >> 1 : nchunk;
+    // An eight-warp group writes the second half's probabilities over the S columns that half itself has consumed
+    // (the first half may still be reading its own): chunk ch >= chs lands 16 * chs columns further right.
+    const int chs = (nchunk + 1) >> 1;
+    const uint32_t p_shift = (GW == 8 && half == 1) ? 16u * chs : 0u;
+    float* cbuf = cls_buf + g * AT_MAXKEYS;
+    float* rmax = red + g * 4 * AT_QROWS;                  // [2][128]
+    float* rsum = rmax + 2 * AT_QROWS;                     // [2][128]
+    bool ok = true;
+    // tile i of this CTA: pair n = i / nqt (bh = blockIdx.x + n * gridDim.x), query tile qt = i % nqt
+    const int my_pairs = blockIdx.x < pairs ? (pairs - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const int items = my_pairs * nqt;
+    int use = 0;
+    for (int i = g; i < items; i += NBUF, ++use) {
+      const int n = i / nqt, qt = i - n * nqt;
+      const int bh = blockIdx.x + n * gridDim.x;
+      const int b = bh / H, h = bh - b * H;
+      const uint32_t par = use & 1;
+      const int q0 = qt * AT_QROWS;
+      const bool live = q0 + quarter * 32 < T;           // warp-uniform: a quarter whose rows all lie past T does no work
+      ok = mbar_wait_q(s_full(g), par, abortp) && ok;
+      ok = __all_sync(0xffffffffu, ok);
+      tc_fence_after();
+      float mx = -INFINITY, sum = 0.f;
+      const bool cls_row = (q0 == 0 && row == 0 && cls_prob != nullptr);
+      if (live) {
+        for (int ch = ch0; ch < ch1; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(trow + ch * 32, r);
+          tmem_ld_wait();
+          if (ch * 32 + 32 <= T) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) mx = fmax3(mx, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (ch * 32 + j < T) mx = fmaxf(mx, __uint_as_float(r[j]));
+          }
+        }
+      }
+      if (GW == 8) {
+        rmax[half * AT_QROWS + row] = mx;
+        group_sync(1 + g, GT);
+        mx = fmaxf(rmax[row], rmax[AT_QROWS + row]);
+      }
+      // With two groups the exponentials of successive tiles take turns (the special-function unit is shared), so
+      // that one group's exponentials overlap the other's tensor-core and load/store phases instead of colliding
+      // with its exponentials.  Three or four groups drift apart by themselves.
+      if (NBUF == 2 && i > 0) {
+        ok = mbar_wait_q(token(g), (g == 0 ? use - 1 : use) & 1, abortp) && ok;
+        ok = __all_sync(0xffffffffu, ok);
+      }
+      if (live) {
+        const float mc = mx * c;
+        for (int ch = ch0; ch < ch1; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(trow + ch * 32, r);
+          tmem_ld_wait();
+          float p[32];
+          if (ch * 32 + 32 <= T) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) p[j] = ex2_fast(fmaf(__uint_as_float(r[j]), c, -mc));
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) p[j] = (ch * 32 + j < T) ? ex2_fast(fmaf(__uint_as_float(r[j]), c, -mc)) : 0.f;
+          }
+          float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) { s0 += p[j]; s1 += p[j + 1]; s2 += p[j + 2]; s3 += p[j + 3]; }
+          sum += (s0 + s1) + (s2 + s3);
+          if (cls_row) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) cbuf[ch * 32 + j] = p[j];
+          }
+          uint32_t pk[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2(p[2 * j], p[2 * j + 1]);
+          tmem_st16(trow + ch * 16 + p_shift, pk);
+        }
+        tmem_st_wait();
+      }
+      if (GW == 8) rsum[half * AT_QROWS + row] = sum;
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(p_full(g));             // P of this warp's rows and keys is in tensor memory
+      if (GW == 8) group_sync(1 + g, GT);                // partial sums and the classification row are in shared memory
+      else __syncwarp();
+      if (NBUF == 2 && leader) mbar_arrive(token((g + 1) % NBUF));
+      if (GW == 8) sum = rsum[row] + rsum[AT_QROWS + row];
+      const float inv = 1.0f / sum;
+      const int q = q0 + row;
+      if (live && q < T && half == 0 && lse != nullptr) lse[((size_t)b * H + h) * T + q] = mx * 0.125f + logf(sum);
+      if (q0 == 0 && gw == 0 && cls_prob != nullptr) {        // this warp holds query 0 in lane 0
+        float s_inv = __shfl_sync(0xffffffffu, inv, 0);
+        float* cp = cls_prob + ((size_t)b * H + h) * (T - 1);
+        for (int j = 1 + lane; j < T; j += 32) cp[j - 1] = cbuf[j] * s_inv;
+      }
+      ok = mbar_wait_q(o_full(g), par, abortp) && ok;
+      ok = __all_sync(0xffffffffu, ok);
+      tc_fence_after();
+      constexpr int NH = GW == 8 ? 1 : 2;                // 32-column halves of O this thread reads
+      if (live) {
+#pragma unroll
+        for (int hh = 0; hh < NH; ++hh) {
+          uint32_t ro[32];
+          tmem_ld32(trow + O_COL + (half + hh) * 32, ro);
+          tmem_ld_wait();
+          if (q < T && ok) {
+            bf16* orow = out + ((size_t)b * T + q) * H * AT_D + (size_t)h * AT_D + (half + hh) * 32;
+#pragma unroll
+            for (int gq = 0; gq < 4; ++gq) {
+              float v[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(ro[gq * 8 + j]) * inv;
+              store16(orow + gq * 8, v);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(t_empty(g));            // O has been read: the buffer may take the next S
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) {
+  if (warp == LOADER) {
     tc_fence_after();
-    tmem_dealloc(tmem, tmem_cols);
+    tmem_dealloc(tmem, 512);
   }
   if (tid == 0 && abort_flag && status != nullptr) atomicOr(status, STATUS_TIMEOUT);
 }
@@ -633,18 +744,31 @@ int attention_fwd_tc(const Ctx& c, const void* qkv, void* out, float* lse, float
     return 0;
   }
   int tpad = (T + 15) & ~15;
-  int nbox = (tpad + AT_BOX - 1) / AT_BOX;
-  size_t p_bytes = (size_t)nbox * (AT_QROWS * 128), qk_bytes = (size_t)(2 + nbox) * AT_BOX_BYTES;
-  size_t smem = 1024 + (p_bytes > qk_bytes ? p_bytes : qk_bytes) + (size_t)nbox * AT_BOX_BYTES + (AT_MAXKEYS + 4 * AT_QROWS) * 4 + 64;
-  static size_t attr = 0;
-  if (smem > attr) {
-    if (cudaFuncSetAttribute(attn_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -3;
-    attr = smem;
-  }
-  dim3 grid((T + AT_QROWS - 1) / AT_QROWS, B * H);
-  note_launch(1);
-  attn_fwd_tc_kernel<<<grid, 256, smem, c.stream>>>(map, (bf16*)out, lse, cls_prob, B, T, H, c.status);
-  return 0;
+  CUtensorMap map_q, map_kv;
+  if (!make_map(&map_q, qkv, (uint64_t)3 * H * d, (uint64_t)B * T, (uint64_t)3 * H * d, AT_QROWS)) return -2;
+  if (!make_map(&map_kv, qkv, (uint64_t)3 * H * d, (uint64_t)B * T, (uint64_t)3 * H * d, tpad)) return -2;
+  int nbuf = tpad <= 128 ? 4 : (tpad <= 160 ? 3 : 2);
+  size_t fixed = 1024 + (size_t)WS_QSLOTS * WS_Q_BYTES + (WS_MAXBUF * AT_MAXKEYS + WS_MAXBUF * 4 * AT_QROWS) * 4 + 44 * 8 + 64;
+  size_t slot = (size_t)2 * tpad * 128;
+  int kvslots = (int)((227 * 1024 - fixed) / slot);
+  if (kvslots > WS_MAXKV) kvslots = WS_MAXKV;
+  if (kvslots < 2) return -1;
+  size_t smem = fixed + kvslots * slot;
+  int sms = c.sm_count > 0 ? c.sm_count : 148;
+  int grid = B * H < sms ? B * H : sms;
+  static size_t attr[5] = {0, 0, 0, 0, 0};
+  auto launch = [&](auto kern, int threads) -> int {
+    if (smem > attr[nbuf]) {
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -3;
+      attr[nbuf] = smem;
+    }
+    note_launch(1);
+    kern<<<grid, threads, smem, c.stream>>>(map_q, map_kv, (bf16*)out, lse, cls_prob, B, T, H, kvslots, c.status);
+    return 0;
+  };
+  if (nbuf == 4) return launch(attn_fwd_ws_kernel<4>, 19 * 32);
+  if (nbuf == 3) return launch(attn_fwd_ws_kernel<3>, 15 * 32);
+  return launch(attn_fwd_ws_kernel<2>, 19 * 32);
 }
 
 }  // namespace bsr

@@ -4,6 +4,7 @@
     python -m paper_2405_10951_b200.microbench backward --m 12800 --n 2304 --k 768
     python -m paper_2405_10951_b200.microbench select_gather --batch 4096 --heads 12 --tokens 197 --dim 768 --keep 0.7
     python -m paper_2405_10951_b200.microbench attention --batch 128 --heads 12 --tokens 197
+    python -m paper_2405_10951_b200.microbench step --workload vit_b --batch 32 --iters 4
 
 Each prints one JSON line with the time per launch (CUDA events on the current stream, after warm-up) and the
 achieved TFLOP/s or GB/s on the kernel's algorithmic work.  Inputs are seeded and synthetic.
@@ -38,7 +39,8 @@ def timed(fn, iters, flush=None):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["gemm", "backward", "select_gather", "attention"])
+    ap.add_argument("what", choices=["gemm", "backward", "select_gather", "attention", "step"])
+    ap.add_argument("--workload", default="vit_b")
     ap.add_argument("--m", type=int, default=25216)
     ap.add_argument("--n", type=int, default=2304)
     ap.add_argument("--k", type=int, default=768)
@@ -58,7 +60,21 @@ def main():
     dev = "cuda"
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev) if a.flush_l2 else None
     out = {"kernel": a.what}
-    if a.what == "gemm":
+    if a.what == "step":
+        # whole fine-tuning steps of a named workload at a chosen batch: the launch sequence a profiler is pointed at
+        from . import synth
+        cfg = synth.CONFIGS[a.workload]
+        cfg = cfg.with_(batch=min(a.batch, cfg.batch))
+        images, labels, task_ids, params = synth.make_workload(cfg)
+        eng = Bd.Engine(cfg)
+        eng.set_params(params)
+        img, lab = eng.images_to_device(images), torch.as_tensor(labels).cuda()
+        tid = torch.as_tensor(task_ids).cuda() if cfg.num_tasks > 1 else None
+        eng.set_graph_mode(False)
+        ms = timed(lambda: eng.train_step(img, lab, tid, want_kept=False), a.iters)
+        eng.sync_status()
+        out.update(workload=cfg.name, batch=cfg.batch, ms_per_step=ms, images_per_s=cfg.batch / ms * 1e3)
+    elif a.what == "gemm":
         x = torch.randn(a.m, a.k, device=dev).bfloat16()
         w = (torch.randn(a.n, a.k, device=dev) / math.sqrt(a.k)).bfloat16()
         b = torch.randn(a.n, device=dev)
@@ -96,7 +112,17 @@ def main():
     else:
         B, H, T = a.batch, a.heads, a.tokens
         qkv = torch.randn(B, T, 3, H, 64, device=dev).bfloat16()
-        ms = timed(lambda: Bd.bsr_attention_forward(qkv, H, use_tensor_cores=True), a.iters, flush)
+        import ctypes as C
+        o = torch.empty(B, T, H * 64, device=dev, dtype=torch.bfloat16)
+        cp = torch.empty(B, H, T - 1, device=dev, dtype=torch.float32)
+        L, st = Bd.lib(), C.c_void_p(torch.cuda.current_stream().cuda_stream)
+        ptr = lambda t: C.c_void_p(t.data_ptr())
+        reps = 10                                  # back-to-back launches per timing: the kernel is shorter than a host call
+
+        def run():
+            for _ in range(reps):
+                L.bsr_attention_forward(ptr(qkv), 1, B, T, H, 64, ptr(o), ptr(cp), 1, st)
+        ms = timed(run, a.iters, flush) / reps
         out.update(batch=B, heads=H, tokens=T, us=ms * 1e3, tflops=4.0 * B * H * T * T * 64 / ms / 1e9)
     print(json.dumps(out), flush=True)
 
