@@ -533,7 +533,7 @@ attn_fwd_tc_long_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __res
 // transposing descriptors (dK, dV), so nothing is transposed by hand.  A gradient arriving at the head-mean
 // score of token j (cls_extra[b, j-1], from the fused token) is added to dP of the classification row.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(256, 2)
 attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_constant__ CUtensorMap map_do,
                    const float* __restrict__ lse, const float* __restrict__ cls_extra, bf16* __restrict__ dqkv,
                    int B, int T, int H, int* status) {
@@ -546,12 +546,17 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
   uint32_t CH = (uint32_t)tpad * 128u;
   uint32_t sQ = base, sK = sQ + TILE, sG = sK + TILE, sV = sG + TILE, sS = sV;
   uint32_t sP = sV + (2 * CH > TILE ? 2 * CH : TILE);
-  uint32_t bars = sP + 2 * CH + (3 * CH < 16384u ? 16384u - 3 * CH : 0u);   // slack: MMA row extent past tpad stays in bounds
+  uint32_t red_off = sP + 2 * CH + (3 * CH < 16384u ? 16384u - 3 * CH : 0u);   // slack: MMA row extent past tpad stays in bounds
+  float* red = reinterpret_cast<float*>(base_ptr + (red_off - base));        // [2][128]: the halves' shares of delta
+  uint32_t bars = red_off + 2 * AT_QROWS * 4;
   unsigned char* pP = base_ptr + (sP - base);
   unsigned char* pS = base_ptr + (sS - base);
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
+  // 256 threads: warps w and w + 4 share the TMEM lane quarter w & 3 (query rows 32 * (w & 3) ..) and split the
+  // keys (chunks 0-1 and 2-3 of 32) and later the output columns between them.
   int tid = threadIdx.x, warp = tid >> 5;
+  int row = tid & 127, half = tid >> 7;
   int bh = blockIdx.x, b = bh / H, h = bh % H;
   uint32_t tma_bar = bars, mma_bar = bars + 8;
   if (tid == 0) {
@@ -599,17 +604,17 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
   tc_fence_after();
 
   const float c = 0.125f * 1.4426950408889634f;
-  uint32_t trow = tmem + ((uint32_t)(warp * 32) << 16);
-  bool valid_row = tid < T;
-  float l2 = valid_row ? lse[((size_t)b * H + h) * T + tid] * 1.4426950408889634f : 0.f;
-  bool extra_row = (tid == 0 && cls_extra != nullptr);
+  uint32_t trow = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+  bool valid_row = row < T;
+  float l2 = valid_row ? lse[((size_t)b * H + h) * T + row] * 1.4426950408889634f : 0.f;
+  bool extra_row = (row == 0 && cls_extra != nullptr);
   const float* ex = extra_row ? cls_extra + (size_t)b * (T - 1) : nullptr;
   float invH = 1.0f / (float)H;
   int nchunk = (T + 31) >> 5;
   float delta = 0.f;
   // tcgen05.ld is warp-collective: every lane issues it, rows past T only skip the arithmetic
   if (ok) {
-    for (int ch = 0; ch < nchunk; ++ch) {
+    for (int ch = 2 * half; ch < nchunk && ch < 2 * half + 2; ++ch) {
       uint32_t rs[32], rp[32];
       tmem_ld32(trow + C_S + ch * 32, rs);
       tmem_ld32(trow + C_DP + ch * 32, rp);
@@ -619,7 +624,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
         for (int j = 0; j < 32; ++j) {
           int key = ch * 32 + j;
           if (key < T) {
-            float p = exp2f(fmaf(__uint_as_float(rs[j]), c, -l2));
+            float p = ex2_fast(fmaf(__uint_as_float(rs[j]), c, -l2));
             float dp = __uint_as_float(rp[j]);
             if (extra_row && key > 0) dp += ex[key - 1] * invH;
             delta = fmaf(p, dp, delta);
@@ -627,7 +632,12 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
         }
       }
     }
-    for (int ch = 0; ch < 4; ++ch) {
+  }
+  red[half * AT_QROWS + row] = delta;          // every thread reaches this barrier, whatever the waits returned
+  __syncthreads();
+  delta = red[row] + red[AT_QROWS + row];
+  if (ok) {
+    for (int ch = 2 * half; ch < 2 * half + 2; ++ch) {
       float p[32], ds[32];
 #pragma unroll
       for (int j = 0; j < 32; ++j) { p[j] = 0.f; ds[j] = 0.f; }
@@ -641,7 +651,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
           for (int j = 0; j < 32; ++j) {
             int key = ch * 32 + j;
             if (key < T) {
-              float pv = exp2f(fmaf(__uint_as_float(rs[j]), c, -l2));
+              float pv = ex2_fast(fmaf(__uint_as_float(rs[j]), c, -l2));
               float dp = __uint_as_float(rp[j]);
               if (extra_row && key > 0) dp += ex[key - 1] * invH;
               p[j] = pv;
@@ -660,9 +670,9 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
           hp[i] = __floats2bfloat162_rn(p[g * 8 + 2 * i], p[g * 8 + 2 * i + 1]);
           hs[i] = __floats2bfloat162_rn(ds[g * 8 + 2 * i], ds[g * 8 + 2 * i + 1]);
         }
-        if (tid < tpad) {
+        if (row < tpad) {
           int key8 = ch * 4 + g;
-          uint32_t off = (uint32_t)(key8 >> 3) * CH + (uint32_t)tid * 128u + (uint32_t)(((key8 & 7) ^ (tid & 7)) << 4);
+          uint32_t off = (uint32_t)(key8 >> 3) * CH + (uint32_t)row * 128u + (uint32_t)(((key8 & 7) ^ (row & 7)) << 4);
           *reinterpret_cast<uint4*>(pP + off) = vp;
           *reinterpret_cast<uint4*>(pS + off) = vs;
         }
@@ -695,13 +705,12 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
     const uint32_t cols[3] = {C_DQ, C_DK, C_DV};
 #pragma unroll
     for (int which = 0; which < 3; ++which) {
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
+      {
         uint32_t r[32];
         tmem_ld32(trow + cols[which] + half * 32, r);
         tmem_ld_wait();
         if (valid_row) {
-          bf16* drow = dqkv + (((size_t)b * T + tid) * 3 + which) * H * AT_D + (size_t)h * AT_D + half * 32;
+          bf16* drow = dqkv + (((size_t)b * T + row) * 3 + which) * H * AT_D + (size_t)h * AT_D + half * 32;
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
             float v[8];
@@ -784,14 +793,14 @@ int attention_bwd_tc(const Ctx& c, const void* qkv, const void* dout, const floa
   if (!make_map(&mq, qkv, (uint64_t)3 * H * d, (uint64_t)B * T, (uint64_t)3 * H * d, AT_BOX)) return -2;
   if (!make_map(&mg, dout, (uint64_t)H * d, (uint64_t)B * T, (uint64_t)H * d, AT_BOX)) return -2;
   size_t tile = 2 * (size_t)AT_BOX_BYTES, ch = (size_t)((T + 15) & ~15) * 128;
-  size_t smem = 1024 + 3 * tile + (2 * ch > tile ? 2 * ch : tile) + 2 * ch + (3 * ch < 16384 ? 16384 - 3 * ch : 0) + 64;
+  size_t smem = 1024 + 3 * tile + (2 * ch > tile ? 2 * ch : tile) + 2 * ch + (3 * ch < 16384 ? 16384 - 3 * ch : 0) + 2 * AT_QROWS * 4 + 64;
   static size_t attr = 0;
   if (smem > attr) {
     if (cudaFuncSetAttribute(attn_bwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -3;
     attr = smem;
   }
   note_launch(1);
-  attn_bwd_tc_kernel<<<B * H, 128, smem, c.stream>>>(mq, mg, lse, cls_extra, (bf16*)dqkv, B, T, H, c.status);
+  attn_bwd_tc_kernel<<<B * H, 256, smem, c.stream>>>(mq, mg, lse, cls_extra, (bf16*)dqkv, B, T, H, c.status);
   return 0;
 }
 

@@ -184,36 +184,59 @@ __global__ void __launch_bounds__(256, 2) layernorm_bwd_kernel(const TDY* __rest
   extern __shared__ float sm[];   // [LNB_WARPS][2][D]
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int chunks = D / 4;
-  float ag[(NCH * 4)], ab[(NCH * 4)];
+  // The warp's partial sums for the scale and shift gradients live in its slice of shared memory (each lane owns
+  // its columns), which leaves the registers for a whole row of x, dy and the residual gradient in flight at once.
+  float* mine = sm + (size_t)warp * 2 * D;
 #pragma unroll
-  for (int i = 0; i < (NCH * 4); ++i) { ag[i] = 0.f; ab[i] = 0.f; }
+  for (int i = 0; i < NCH; ++i) {
+    int ch = lane + i * 32;
+    if (ch < chunks) {
+      *reinterpret_cast<float4*>(mine + ch * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+      *reinterpret_cast<float4*>(mine + D + ch * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
   for (int r = blockIdx.x * LNB_WARPS + warp; r < rows; r += gridDim.x * LNB_WARPS) {
     const float* xr = x + (long)r * x_stride;
     const TDY* dyr = dy + (long)r * D;
     float mu = mean[r], rs = rstd[r];
-    float xh[(NCH * 4)], dh[(NCH * 4)];
+    float xh[(NCH * 4)], dh[(NCH * 4)], o[(NCH * 4)];
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {                      // all loads of the row first
+      int ch = lane + i * 32;
+      if (ch < chunks) {
+        load16(xr + ch * 4, xh + i * 4);
+        load4(dyr + ch * 4, dh + i * 4);
+        if (dx != nullptr && dres != nullptr) load16(dres + (long)r * D + ch * 4, o + i * 4);
+        else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) o[i * 4 + j] = 0.f;
+        }
+      }
+    }
     float s1 = 0.f, s2 = 0.f;
 #pragma unroll
     for (int i = 0; i < NCH; ++i) {
       int ch = lane + i * 32;
       if (ch < chunks) {
-        float xv[4], dv[4];
-        load16(xr + ch * 4, xv);
-        load4(dyr + ch * 4, dv);
         float4 gg = *reinterpret_cast<const float4*>(g + ch * 4);
         float gv[4] = {gg.x, gg.y, gg.z, gg.w};
+        float4 pg = *reinterpret_cast<const float4*>(mine + ch * 4);
+        float4 pb = *reinterpret_cast<const float4*>(mine + D + ch * 4);
+        float pgv[4] = {pg.x, pg.y, pg.z, pg.w}, pbv[4] = {pb.x, pb.y, pb.z, pb.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          float d = dv[j];
-          float h = (xv[j] - mu) * rs;
+          float d = dh[i * 4 + j];
+          float h = (xh[i * 4 + j] - mu) * rs;
           xh[i * 4 + j] = h;
-          ag[i * 4 + j] += d * h;
-          ab[i * 4 + j] += d;
+          pgv[j] += d * h;
+          pbv[j] += d;
           float dxh = d * gv[j];
           dh[i * 4 + j] = dxh;
           s1 += dxh;
           s2 += dxh * h;
         }
+        *reinterpret_cast<float4*>(mine + ch * 4) = make_float4(pgv[0], pgv[1], pgv[2], pgv[3]);
+        *reinterpret_cast<float4*>(mine + D + ch * 4) = make_float4(pbv[0], pbv[1], pbv[2], pbv[3]);
       }
     }
     s1 = warp_sum(s1) / (float)D;
@@ -224,29 +247,11 @@ __global__ void __launch_bounds__(256, 2) layernorm_bwd_kernel(const TDY* __rest
       for (int i = 0; i < NCH; ++i) {
         int ch = lane + i * 32;
         if (ch < chunks) {
-          float o[4];
-          if (dres != nullptr) load16(dres + (long)r * D + ch * 4, o);
-          else {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) o[j] = 0.f;
-          }
-#pragma unroll
-          for (int j = 0; j < 4; ++j) o[j] += rs * (dh[i * 4 + j] - s1 - xh[i * 4 + j] * s2);
-          store16(dxr + ch * 4, o);
-          if (dx_copy != nullptr) store4(dx_copy + (long)r * dx_stride + ch * 4, o);
+          for (int j = 0; j < 4; ++j) o[i * 4 + j] += rs * (dh[i * 4 + j] - s1 - xh[i * 4 + j] * s2);
+          store16(dxr + ch * 4, o + i * 4);
+          if (dx_copy != nullptr) store4(dx_copy + (long)r * dx_stride + ch * 4, o + i * 4);
         }
-      }
-    }
-  }
-  float* mine = sm + (size_t)warp * 2 * D;
-#pragma unroll
-  for (int i = 0; i < NCH; ++i) {
-    int ch = lane + i * 32;
-    if (ch < chunks) {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        mine[ch * 4 + j] = ag[i * 4 + j];
-        mine[D + ch * 4 + j] = ab[i * 4 + j];
       }
     }
   }

@@ -79,8 +79,23 @@ token_select_reg_kernel(const float* __restrict__ p, int B, int H, int M, int k,
   // head sum in head order per token; the IPL loads of one head are independent, so many are in flight
 #pragma unroll
   for (int i = 0; i < IPL; ++i) acc[i] = (i * 32 + lane < M) ? pb[i * 32 + lane] : 0.f;
-#pragma unroll 2
-  for (int h = 1; h < H; ++h) {
+  // heads in groups of four: the loads of a group are all issued before its (ordered) additions
+  int h = 1;
+  for (; h + 4 <= H; h += 4) {
+    float v[4][IPL];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const float* ph = pb + (size_t)(h + u) * M;
+#pragma unroll
+      for (int i = 0; i < IPL; ++i) v[u][i] = (i * 32 + lane < M) ? ph[i * 32 + lane] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+#pragma unroll
+      for (int i = 0; i < IPL; ++i) acc[i] = acc[i] + v[u][i];
+    }
+  }
+  for (; h < H; ++h) {
     const float* ph = pb + (size_t)h * M;
 #pragma unroll
     for (int i = 0; i < IPL; ++i)
