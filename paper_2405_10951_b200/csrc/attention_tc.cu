@@ -548,7 +548,8 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
   uint32_t sP = sV + (2 * CH > TILE ? 2 * CH : TILE);
   uint32_t red_off = sP + 2 * CH + (3 * CH < 16384u ? 16384u - 3 * CH : 0u);   // slack: MMA row extent past tpad stays in bounds
   float* red = reinterpret_cast<float*>(base_ptr + (red_off - base));        // [2][128]: the halves' shares of delta
-  uint32_t bars = red_off + 2 * AT_QROWS * 4;
+  float* exs = red + 2 * AT_QROWS;                                             // [128]: classification-row score gradients / H
+  uint32_t bars = red_off + 3 * AT_QROWS * 4;
   unsigned char* pP = base_ptr + (sP - base);
   unsigned char* pS = base_ptr + (sS - base);
   __shared__ uint32_t tmem_slot;
@@ -558,11 +559,12 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
   int tid = threadIdx.x, warp = tid >> 5;
   int row = tid & 127, half = tid >> 7;
   int bh = blockIdx.x, b = bh / H, h = bh % H;
-  uint32_t tma_bar = bars, mma_bar = bars + 8;
+  uint32_t tma_bar = bars, mma_bar = bars + 8, mma2_bar = bars + 16;
   if (tid == 0) {
     abort_flag = 0;
     mbar_init(tma_bar, 1);
     mbar_init(mma_bar, 1);
+    mbar_init(mma2_bar, 3);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -586,6 +588,14 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
       tma_load_2d(sV + j * AT_BOX_BYTES, &map_qkv, tma_bar, (2 * H + h) * AT_D, row0 + j * AT_BOX);
       tma_load_2d(sG + j * AT_BOX_BYTES, &map_do, tma_bar, h * AT_D, row0 + j * AT_BOX);
     }
+  }
+  // inputs that do not come through TMA are fetched while the tiles are on their way
+  const bool valid_row = row < T;
+  const float l2 = valid_row ? lse[((size_t)b * H + h) * T + row] * 1.4426950408889634f : 0.f;
+  const bool has_extra = cls_extra != nullptr;
+  if (half == 0) exs[row] = (has_extra && row >= 1 && row < T) ? cls_extra[(size_t)b * (T - 1) + row - 1] * (1.0f / (float)H) : 0.f;
+  __syncthreads();
+  if (tid == 0) {
     ok = mbar_wait(tma_bar, 0, abortp);
     if (ok) {
       tc_fence_after();
@@ -605,11 +615,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
 
   const float c = 0.125f * 1.4426950408889634f;
   uint32_t trow = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-  bool valid_row = row < T;
-  float l2 = valid_row ? lse[((size_t)b * H + h) * T + row] * 1.4426950408889634f : 0.f;
-  bool extra_row = (row == 0 && cls_extra != nullptr);
-  const float* ex = extra_row ? cls_extra + (size_t)b * (T - 1) : nullptr;
-  float invH = 1.0f / (float)H;
+  const bool extra_row = (row == 0 && has_extra);
   int nchunk = (T + 31) >> 5;
   float delta = 0.f;
   // tcgen05.ld is warp-collective: every lane issues it, rows past T only skip the arithmetic
@@ -626,7 +632,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
           if (key < T) {
             float p = ex2_fast(fmaf(__uint_as_float(rs[j]), c, -l2));
             float dp = __uint_as_float(rp[j]);
-            if (extra_row && key > 0) dp += ex[key - 1] * invH;
+            if (extra_row) dp += exs[key];
             delta = fmaf(p, dp, delta);
           }
         }
@@ -653,7 +659,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
             if (key < T) {
               float pv = ex2_fast(fmaf(__uint_as_float(rs[j]), c, -l2));
               float dp = __uint_as_float(rp[j]);
-              if (extra_row && key > 0) dp += ex[key - 1] * invH;
+              if (extra_row) dp += exs[key];
               p[j] = pv;
               ds[j] = pv * (dp - delta) * 0.125f;
             }
@@ -684,21 +690,24 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
   __syncthreads();
   tc_fence_after();
   ok = ok && !abort_flag;
-  if (tid == 0 && ok) {
-    // dQ = dS K: A = dS (contiguous along keys), B = K read with keys as the reduction index
-    uint32_t id_q = make_idesc_mn(AT_QROWS, AT_D, false, true);
-    for (int k = 0; k < tpad / 16; ++k)
-      umma_bf16(tmem + C_DQ, make_desc(sS + (k >> 2) * CH + (k & 3) * 32, 16, 1024), make_desc(sK + k * 2048, 8192, 1024), id_q,
-                k > 0 ? 1u : 0u);
-    // dK = dS^T Q and dV = P^T dO: both operands read with queries as the reduction index
-    uint32_t id_t = make_idesc_mn(AT_QROWS, AT_D, true, true);
-    for (int k = 0; k < tpad / 16; ++k)
-      umma_bf16(tmem + C_DK, make_desc(sS + k * 2048, CH, 1024), make_desc(sQ + k * 2048, 8192, 1024), id_t, k > 0 ? 1u : 0u);
-    for (int k = 0; k < tpad / 16; ++k)
-      umma_bf16(tmem + C_DV, make_desc(sP + k * 2048, CH, 1024), make_desc(sG + k * 2048, 8192, 1024), id_t, k > 0 ? 1u : 0u);
-    umma_commit(mma_bar);
+  // dQ, dK and dV are issued by three different threads (lane 0 of warps 0, 1, 2), each committing to the same barrier
+  if (ok && (tid & 31) == 0 && warp < 3) {
+    if (warp == 0) {
+      // dQ = dS K: A = dS (contiguous along keys), B = K read with keys as the reduction index
+      uint32_t id_q = make_idesc_mn(AT_QROWS, AT_D, false, true);
+      for (int k = 0; k < tpad / 16; ++k)
+        umma_bf16(tmem + C_DQ, make_desc(sS + (k >> 2) * CH + (k & 3) * 32, 16, 1024), make_desc(sK + k * 2048, 8192, 1024), id_q,
+                  k > 0 ? 1u : 0u);
+    } else {
+      // dK = dS^T Q and dV = P^T dO: both operands read with queries as the reduction index
+      uint32_t id_t = make_idesc_mn(AT_QROWS, AT_D, true, true);
+      uint32_t sa = warp == 1 ? sS : sP, sb = warp == 1 ? sQ : sG, cd = warp == 1 ? C_DK : C_DV;
+      for (int k = 0; k < tpad / 16; ++k)
+        umma_bf16(tmem + cd, make_desc(sa + k * 2048, CH, 1024), make_desc(sb + k * 2048, 8192, 1024), id_t, k > 0 ? 1u : 0u);
+    }
+    umma_commit(mma2_bar);
   }
-  if (ok) ok = mbar_wait(mma_bar, 1, abortp);
+  if (ok) ok = mbar_wait(mma2_bar, 0, abortp);
   ok = __all_sync(0xffffffffu, ok);
   tc_fence_after();
   if (ok) {
@@ -793,7 +802,7 @@ int attention_bwd_tc(const Ctx& c, const void* qkv, const void* dout, const floa
   if (!make_map(&mq, qkv, (uint64_t)3 * H * d, (uint64_t)B * T, (uint64_t)3 * H * d, AT_BOX)) return -2;
   if (!make_map(&mg, dout, (uint64_t)H * d, (uint64_t)B * T, (uint64_t)H * d, AT_BOX)) return -2;
   size_t tile = 2 * (size_t)AT_BOX_BYTES, ch = (size_t)((T + 15) & ~15) * 128;
-  size_t smem = 1024 + 3 * tile + (2 * ch > tile ? 2 * ch : tile) + 2 * ch + (3 * ch < 16384 ? 16384 - 3 * ch : 0) + 2 * AT_QROWS * 4 + 64;
+  size_t smem = 1024 + 3 * tile + (2 * ch > tile ? 2 * ch : tile) + 2 * ch + (3 * ch < 16384 ? 16384 - 3 * ch : 0) + 3 * AT_QROWS * 4 + 64;
   static size_t attr = 0;
   if (smem > attr) {
     if (cudaFuncSetAttribute(attn_bwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -3;
