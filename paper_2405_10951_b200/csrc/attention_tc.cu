@@ -616,26 +616,28 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
   const float c = 0.125f * 1.4426950408889634f;
   uint32_t trow = tmem + ((uint32_t)((warp & 3) * 32) << 16);
   const bool extra_row = (row == 0 && has_extra);
-  int nchunk = (T + 31) >> 5;
   float delta = 0.f;
-  // tcgen05.ld is warp-collective: every lane issues it, rows past T only skip the arithmetic
+  // tcgen05.ld is warp-collective: every lane issues it, rows past T only skip the arithmetic.  Keys are taken 16 at
+  // a time (two loads of 16 columns) to keep the live registers of a step few.
   if (ok) {
-    for (int ch = 2 * half; ch < nchunk && ch < 2 * half + 2; ++ch) {
-      uint32_t rs[32], rp[32];
-      tmem_ld32(trow + C_S + ch * 32, rs);
-      tmem_ld32(trow + C_DP + ch * 32, rp);
+    for (int kk = 4 * half; kk < 4 * half + 4 && kk * 16 < T; ++kk) {
+      uint32_t rs[16], rp[16];
+      tmem_ld16(trow + C_S + kk * 16, rs);
+      tmem_ld16(trow + C_DP + kk * 16, rp);
       tmem_ld_wait();
       if (valid_row) {
+        float d0 = 0.f, d1 = 0.f;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          int key = ch * 32 + j;
-          if (key < T) {
-            float p = ex2_fast(fmaf(__uint_as_float(rs[j]), c, -l2));
-            float dp = __uint_as_float(rp[j]);
-            if (extra_row) dp += exs[key];
-            delta = fmaf(p, dp, delta);
-          }
+        for (int j = 0; j < 16; j += 2) {
+          int key = kk * 16 + j;
+          float p0 = key < T ? ex2_fast(fmaf(__uint_as_float(rs[j]), c, -l2)) : 0.f;
+          float p1 = key + 1 < T ? ex2_fast(fmaf(__uint_as_float(rs[j + 1]), c, -l2)) : 0.f;
+          float e0 = __uint_as_float(rp[j]), e1 = __uint_as_float(rp[j + 1]);
+          if (extra_row) { e0 += exs[key]; e1 += exs[key + 1]; }
+          d0 = fmaf(p0, e0, d0);
+          d1 = fmaf(p1, e1, d1);
         }
+        delta += d0 + d1;
       }
     }
   }
@@ -643,31 +645,29 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
   __syncthreads();
   delta = red[row] + red[AT_QROWS + row];
   if (ok) {
-    for (int ch = 2 * half; ch < 2 * half + 2; ++ch) {
-      float p[32], ds[32];
+    for (int kk = 4 * half; kk < 4 * half + 4; ++kk) {
+      float p[16], ds[16];
 #pragma unroll
-      for (int j = 0; j < 32; ++j) { p[j] = 0.f; ds[j] = 0.f; }
-      if (ch < nchunk) {
-        uint32_t rs[32], rp[32];
-        tmem_ld32(trow + C_S + ch * 32, rs);
-        tmem_ld32(trow + C_DP + ch * 32, rp);
+      for (int j = 0; j < 16; ++j) { p[j] = 0.f; ds[j] = 0.f; }
+      if (kk * 16 < T) {
+        uint32_t rs[16], rp[16];
+        tmem_ld16(trow + C_S + kk * 16, rs);
+        tmem_ld16(trow + C_DP + kk * 16, rp);
         tmem_ld_wait();
         if (valid_row) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            int key = ch * 32 + j;
-            if (key < T) {
-              float pv = ex2_fast(fmaf(__uint_as_float(rs[j]), c, -l2));
-              float dp = __uint_as_float(rp[j]);
-              if (extra_row) dp += exs[key];
-              p[j] = pv;
-              ds[j] = pv * (dp - delta) * 0.125f;
-            }
+          for (int j = 0; j < 16; ++j) {
+            int key = kk * 16 + j;
+            float pv = key < T ? ex2_fast(fmaf(__uint_as_float(rs[j]), c, -l2)) : 0.f;
+            float dp = __uint_as_float(rp[j]);
+            if (extra_row) dp += exs[key];
+            p[j] = pv;
+            ds[j] = pv * (dp - delta) * 0.125f;
           }
         }
       }
 #pragma unroll
-      for (int g = 0; g < 4; ++g) {
+      for (int g = 0; g < 2; ++g) {
         uint4 vp, vs;
         __nv_bfloat162* hp = reinterpret_cast<__nv_bfloat162*>(&vp);
         __nv_bfloat162* hs = reinterpret_cast<__nv_bfloat162*>(&vs);
@@ -677,7 +677,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
           hs[i] = __floats2bfloat162_rn(ds[g * 8 + 2 * i], ds[g * 8 + 2 * i + 1]);
         }
         if (row < tpad) {
-          int key8 = ch * 4 + g;
+          int key8 = kk * 2 + g;
           uint32_t off = (uint32_t)(key8 >> 3) * CH + (uint32_t)row * 128u + (uint32_t)(((key8 & 7) ^ (row & 7)) << 4);
           *reinterpret_cast<uint4*>(pP + off) = vp;
           *reinterpret_cast<uint4*>(pS + off) = vs;
