@@ -163,7 +163,7 @@ def run_reference(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="vit_b", choices=list(synth.CONFIGS))
@@ -265,6 +265,7 @@ def main():
 
     if rank == 0:
         pk = peaks()
+        fp = eng.footprint()
         flops = step_flops(cfg, cfg.batch)
         gemm_tflops = prof["gemm_flops"] / (prof["gemm_ms"] * 1e-3) / 1e12 if prof["gemm_ms"] > 0 else 0.0
         line = {
@@ -284,6 +285,8 @@ def main():
                          "frac": gemm_tflops / pk["tflops"], "traffic": None, "peak_source": pk["source"] + " (sustained)",
                          "gemm_ms_per_step": prof["gemm_ms"] / max(1, min(args.steps, 5)),
                          "gemm_launches_per_step": prof["gemm_launches"] / max(1, min(args.steps, 5))},
+            "footprint_bytes": {k: fp[k] for k in ("workspace_bytes", "weight_bytes", "master_bytes", "optimizer_bytes", "grad_bytes",
+                                                   "saved_activation_bytes", "scratch_bytes", "paper_activation_bytes")},
             "step_flops": flops,
             "step_tflops": flops / (ms_step * 1e-3) / 1e12,
             "step_roofline_frac": flops / (ms_step * 1e-3) / 1e12 / pk["tflops_burst"],
