@@ -238,13 +238,30 @@ def main():
     launches = eng.profile_read()["kernel_launches"]
 
     # ---- end to end: pinned host images in, loss out, every step ----------------------------------
+    # Two device staging buffers: the copy of the next step's images (its own stream) overlaps the current step, as an
+    # input pipeline would; every step still waits for its own copy and the host reads every step's loss.
+    stages = [torch.empty_like(dev_img), torch.empty_like(dev_img)]
+    copy_stream = torch.cuda.Stream()
+    copied = [torch.cuda.Event(), torch.cuda.Event()]
+    for sbuf in stages:                                   # untimed: lets the library capture its graph for each buffer
+        sbuf.copy_(dev_img)
+        eng.train_step(sbuf, lab, tid, want_kept=False, out=out)
+    eng.sync_status()
     barrier()
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    stage = torch.empty_like(dev_img)
     f0.record(stream)
-    for _ in range(args.steps):
-        stage.copy_(host_img, non_blocking=True)
-        loss, _ = eng.train_step(stage, lab, tid, want_kept=False, out=out)
+    copy_stream.wait_stream(stream)
+    with torch.cuda.stream(copy_stream):
+        stages[0].copy_(host_img, non_blocking=True)
+        copied[0].record(copy_stream)
+    for i in range(args.steps):
+        cur = i & 1
+        if i + 1 < args.steps:                            # the previous user of that buffer (step i-1) has been waited for
+            with torch.cuda.stream(copy_stream):
+                stages[cur ^ 1].copy_(host_img, non_blocking=True)
+                copied[cur ^ 1].record(copy_stream)
+        stream.wait_event(copied[cur])
+        loss, _ = eng.train_step(stages[cur], lab, tid, want_kept=False, out=out)
         host_loss.copy_(loss, non_blocking=True)
         stream.synchronize()
     f1.record(stream)

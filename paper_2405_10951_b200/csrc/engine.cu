@@ -404,7 +404,7 @@ size_t plan(bsr_handle* h) {
     h->off_m_dsel = b.take(cap * 4);
   }
   int maxn = 3 * D > F ? 3 * D : F;
-  h->off_ln_partials = b.take((size_t)2 * 512 * D * 4);
+  h->off_ln_partials = b.take((size_t)3 * 512 * D * 4);
   h->off_cs_partials = b.take((size_t)64 * maxn * 4);
   size_t biggest = 0;
   for (auto& t : h->tensors) biggest = t.numel > biggest ? t.numel : biggest;
@@ -595,7 +595,8 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
   gemm(c, op(dxo), D, 1, h->wb(l, "mlp.fc2.weight"), 1, F, dz, 0, Mf, F, D, eg);
   if (pg) {
     gemm(c, op(dxo), 1, D, h->base + bb.hh, 1, F, h->gb(l, "mlp.fc2.weight"), 1, D, F, Mf, none);
-    colsum(cf, dxo.f, Mf, D, csp, h->gb(l, "mlp.fc2.bias"));
+    // db2 = column sums of dxo: they came out of the following block's LayerNorm backward, which wrote dxo
+    if (l == d.depth - 1) colsum(cf, dxo.f, Mf, D, csp, h->gb(l, "mlp.fc2.bias"));
   }
   // FFN first layer
   gemm(c, dz, F, 1, h->wb(l, "mlp.fc1.weight"), 1, D, dy, 0, Mf, D, F, none);
@@ -606,7 +607,8 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
   }
   layernorm_bwd(c, dy, 0, h->at<float>(bb.xp), D, h->at<float>(bb.mean2), h->at<float>(bb.rstd2),
                 (const float*)h->wb(l, "norm2.weight"), dxo.f, dxg.f, D, shrinks ? nullptr : dxg.c, lnp,
-                pg ? h->gb(l, "norm2.weight") : nullptr, pg ? h->gb(l, "norm2.bias") : nullptr, Mf, D);
+                pg ? h->gb(l, "norm2.weight") : nullptr, pg ? h->gb(l, "norm2.bias") : nullptr, Mf, D,
+                (pg && !shrinks) ? h->gb(l, "attn.proj.bias") : nullptr);   // dx' = dxg here: its column sums are the projection's bias gradient
   const float* cls_extra = nullptr;
   if (shrinks) {
     gather_fuse_bwd(c, dxg.f, h->base + bb.xp_full, B, Ta - 1, D, k, h->at<int>(bb.kept), h->at<int>(bb.dropped),
@@ -619,7 +621,7 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
     gemm(c, op(dxp), D, 1, h->wb(l, "attn.proj.weight"), 1, D, d_o, 0, Ma, D, D, none);
     if (pg) {
       gemm(c, op(dxp), 1, D, h->base + bb.o, 1, D, h->gb(l, "attn.proj.weight"), 1, D, D, Ma, none);
-      colsum(cf, dxp.f, Ma, D, csp, h->gb(l, "attn.proj.bias"));
+      if (shrinks) colsum(cf, dxp.f, Ma, D, csp, h->gb(l, "attn.proj.bias"));
     }
   } else {
     // B rows: dO_cls = dx'_cls Wo, dWo = dx'_cls^T o_cls; then both gradients go back into zeroed dense tensors
@@ -627,7 +629,7 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
     gemm(c, op(dxp), D, 1, h->wb(l, "attn.proj.weight"), 1, D, do_cls, 0, B, D, D, none);
     if (pg) {
       gemm(c, op(dxp), 1, D, h->base + bb.o_cls, 1, D, h->gb(l, "attn.proj.weight"), 1, D, D, B, none);
-      colsum(cf, dxp.f, B, D, csp, h->gb(l, "attn.proj.bias"));
+      if (shrinks) colsum(cf, dxp.f, B, D, csp, h->gb(l, "attn.proj.bias"));
     }
     cudaMemsetAsync(d_o, 0, (size_t)Mdense * D * es, c.stream);
     copy_rows(c.stream, do_cls, (long)D * es, d_o, (long)Ta * D * es, B, (int)(D * es));
@@ -637,6 +639,9 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
     ln1_res = dense_res;
     Ma = Mdense;
   }
+  // the gradient this block hands to block l-1 is that block's output gradient: its column sums are the bias gradient
+  // of block l-1's second FFN layer (dense FFN, trainable)
+  float* prev_fc2_bias = (need_dxi && l > 0 && ((h->cfg.trainable_mask >> (l - 1)) & 1u) && !is_moe(h, l - 1)) ? h->gb(l - 1, "mlp.fc2.bias") : nullptr;
   int rc = attention_bwd(c, h->base + bb.qkv, h->base + bb.o, d_o, h->at<float>(bb.lse), h->at<float>(h->off_delta),
                          cls_extra, dqkv, B, Ta, H, hd);
   if (rc != 0) return set_err(h->err, BSR_ERR_UNSUPPORTED, "attention backward: %d tokens do not fit this kernel", Ta);
@@ -648,7 +653,7 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
   }
   layernorm_bwd(c, dy, 0, h->at<float>(bb.x_in), D, h->at<float>(bb.mean1), h->at<float>(bb.rstd1),
                 (const float*)h->wb(l, "norm1.weight"), ln1_res, need_dxi ? dxi.f : nullptr, D, need_dxi ? dxi.c : nullptr, lnp,
-                pg ? h->gb(l, "norm1.weight") : nullptr, pg ? h->gb(l, "norm1.bias") : nullptr, Ma, D);
+                pg ? h->gb(l, "norm1.weight") : nullptr, pg ? h->gb(l, "norm1.bias") : nullptr, Ma, D, prev_fc2_bias);
   return BSR_OK;
 }
 

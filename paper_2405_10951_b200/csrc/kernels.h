@@ -60,11 +60,12 @@ void layernorm_fwd(const Ctx& c, const float* x, long x_stride, const float* g, 
                    float* mean, float* rstd, int rows, int D, float eps);
 // dx[r] = dres[r] + LN'(dy[r]) (float; rows dx_stride apart); dx_copy (optional, bf16 configurations) receives
 // the same rows in the storage dtype.  Partial sums of dgamma/dbeta go to `partials` ([2][groups][D]) and are
-// reduced in a fixed order.  dx may be null (only parameter gradients wanted); dres may be null.
+// reduced in a fixed order; with dx_colsum the column sums of dx (a bias gradient of the layer that produced the
+// normalised input's predecessor) come out of the same pass ([3][groups][D] partials).  dx may be null (only parameter gradients wanted); dres may be null.
 // dy is in the storage dtype, or float [rows, D] when dy_is_float (head path).
 void layernorm_bwd(const Ctx& c, const void* dy, int dy_is_float, const float* x, long x_stride, const float* mean,
                    const float* rstd, const float* g, const float* dres, float* dx, long dx_stride, void* dx_copy,
-                   float* partials, float* dgamma, float* dbeta, int rows, int D);
+                   float* partials, float* dgamma, float* dbeta, int rows, int D, float* dx_colsum = nullptr);
 int layernorm_bwd_groups(const Ctx& c, int rows);
 
 // ---- column sums (bias gradients) -------------------------------------------------------------

@@ -180,19 +180,20 @@ template <typename TDY, typename TC, int NCH>
 __global__ void __launch_bounds__(256, 2) layernorm_bwd_kernel(const TDY* __restrict__ dy, const float* __restrict__ x, long x_stride,
                                      const float* __restrict__ mean, const float* __restrict__ rstd,
                                      const float* __restrict__ g, const float* __restrict__ dres, float* __restrict__ dx,
-                                     long dx_stride, TC* __restrict__ dx_copy, float* __restrict__ partials, int rows, int D) {
-  extern __shared__ float sm[];   // [LNB_WARPS][2][D]
+                                     long dx_stride, TC* __restrict__ dx_copy, float* __restrict__ partials, int rows, int D, int nsum) {
+  extern __shared__ float sm[];   // [LNB_WARPS][nsum][D]: dgamma, dbeta and (nsum == 3) the column sums of dx
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int chunks = D / 4;
   // The warp's partial sums for the scale and shift gradients live in its slice of shared memory (each lane owns
   // its columns), which leaves the registers for a whole row of x, dy and the residual gradient in flight at once.
-  float* mine = sm + (size_t)warp * 2 * D;
+  float* mine = sm + (size_t)warp * nsum * D;
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
     int ch = lane + i * 32;
     if (ch < chunks) {
       *reinterpret_cast<float4*>(mine + ch * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
       *reinterpret_cast<float4*>(mine + D + ch * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (nsum == 3) *reinterpret_cast<float4*>(mine + 2 * D + ch * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
     }
   }
   for (int r = blockIdx.x * LNB_WARPS + warp; r < rows; r += gridDim.x * LNB_WARPS) {
@@ -251,15 +252,20 @@ __global__ void __launch_bounds__(256, 2) layernorm_bwd_kernel(const TDY* __rest
           for (int j = 0; j < 4; ++j) o[i * 4 + j] += rs * (dh[i * 4 + j] - s1 - xh[i * 4 + j] * s2);
           store16(dxr + ch * 4, o + i * 4);
           if (dx_copy != nullptr) store4(dx_copy + (long)r * dx_stride + ch * 4, o + i * 4);
+          if (nsum == 3) {
+            float4 ps = *reinterpret_cast<const float4*>(mine + 2 * D + ch * 4);
+            ps.x += o[i * 4]; ps.y += o[i * 4 + 1]; ps.z += o[i * 4 + 2]; ps.w += o[i * 4 + 3];
+            *reinterpret_cast<float4*>(mine + 2 * D + ch * 4) = ps;
+          }
         }
       }
     }
   }
   __syncthreads();
-  for (int col = threadIdx.x; col < 2 * D; col += blockDim.x) {
+  for (int col = threadIdx.x; col < nsum * D; col += blockDim.x) {
     float s = 0.f;
 #pragma unroll
-    for (int w = 0; w < LNB_WARPS; ++w) s += sm[(size_t)w * 2 * D + col];
+    for (int w = 0; w < LNB_WARPS; ++w) s += sm[(size_t)w * nsum * D + col];
     int which = col / D, cc = col % D;
     partials[((size_t)which * gridDim.x + blockIdx.x) * D + cc] = s;
   }
@@ -268,7 +274,7 @@ __global__ void __launch_bounds__(256, 2) layernorm_bwd_kernel(const TDY* __rest
 // out_y[col] = sum over groups of partials[y][group][col] for y = blockIdx.y (one or two outputs per launch).
 // 16 lanes stride the groups and are combined through shared memory in lane order: the result is deterministic.
 __global__ void reduce_partials_kernel(const float* __restrict__ partials, int groups, int cols, float* __restrict__ out0,
-                                       float* __restrict__ out1) {
+                                       float* __restrict__ out1, float* __restrict__ out2 = nullptr) {
   __shared__ float sm[16][17];
   int cx = threadIdx.x & 15, gy = threadIdx.x >> 4;
   int col = blockIdx.x * 16 + cx;
@@ -282,7 +288,8 @@ __global__ void reduce_partials_kernel(const float* __restrict__ partials, int g
     float t = 0.f;
 #pragma unroll
     for (int i = 0; i < 16; ++i) t += sm[i][cx];
-    (blockIdx.y ? out1 : out0)[col] = t;
+    float* out = blockIdx.y == 0 ? out0 : (blockIdx.y == 1 ? out1 : out2);
+    if (out != nullptr) out[col] = t;
   }
 }
 
@@ -295,13 +302,13 @@ int layernorm_bwd_groups(const Ctx& c, int rows) {
 template <typename TDY, typename TC>
 static void launch_ln_bwd(const Ctx& c, int groups, size_t smem, const void* dy, const float* x, long x_stride, const float* mean,
                           const float* rstd, const float* g, const float* dres, float* dx, long dx_stride, void* dx_copy,
-                          float* partials, int rows, int D) {
+                          float* partials, int rows, int D, int nsum) {
   int nch = ceil_div(D, 128);
 #define BSR_LN_BWD(N)                                                                                                   \
   do {                                                                                                                  \
     cudaFuncSetAttribute(layernorm_bwd_kernel<TDY, TC, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);       \
     layernorm_bwd_kernel<TDY, TC, N><<<groups, LNB_WARPS * 32, smem, c.stream>>>((const TDY*)dy, x, x_stride, mean, rstd, g, dres, \
-                                                                                 dx, dx_stride, (TC*)dx_copy, partials, rows, D); \
+                                                                                 dx, dx_stride, (TC*)dx_copy, partials, rows, D, nsum); \
   } while (0)
   if (nch <= 2) BSR_LN_BWD(2); else if (nch == 3) BSR_LN_BWD(3); else if (nch == 4) BSR_LN_BWD(4); else if (nch <= 6) BSR_LN_BWD(6); else BSR_LN_BWD(8);
 #undef BSR_LN_BWD
@@ -309,19 +316,20 @@ static void launch_ln_bwd(const Ctx& c, int groups, size_t smem, const void* dy,
 
 void layernorm_bwd(const Ctx& c, const void* dy, int dy_is_float, const float* x, long x_stride, const float* mean,
                    const float* rstd, const float* g, const float* dres, float* dx, long dx_stride, void* dx_copy,
-                   float* partials, float* dgamma, float* dbeta, int rows, int D) {
+                   float* partials, float* dgamma, float* dbeta, int rows, int D, float* dx_colsum) {
   note_launch(2);
   int groups = layernorm_bwd_groups(c, rows);
-  size_t smem = (size_t)LNB_WARPS * 2 * D * sizeof(float);
+  int nsum = (dx_colsum != nullptr && dx != nullptr) ? 3 : 2;
+  size_t smem = (size_t)LNB_WARPS * nsum * D * sizeof(float);
   if (c.dtype == 0)
-    launch_ln_bwd<float, float>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, nullptr, partials, rows, D);
+    launch_ln_bwd<float, float>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, nullptr, partials, rows, D, nsum);
   else if (dy_is_float)
-    launch_ln_bwd<float, bf16>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, dx_copy, partials, rows, D);
+    launch_ln_bwd<float, bf16>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, dx_copy, partials, rows, D, nsum);
   else
-    launch_ln_bwd<bf16, bf16>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, dx_copy, partials, rows, D);
-  if (dgamma == nullptr) return;                          // a frozen block in the gradient path: only dx is wanted
-  dim3 grid(ceil_div(D, 16), 2);
-  reduce_partials_kernel<<<grid, 256, 0, c.stream>>>(partials, groups, D, dgamma, dbeta);
+    launch_ln_bwd<bf16, bf16>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, dx_copy, partials, rows, D, nsum);
+  if (dgamma == nullptr && nsum == 2) return;                          // a frozen block in the gradient path: only dx is wanted
+  dim3 grid(ceil_div(D, 16), nsum);
+  reduce_partials_kernel<<<grid, 256, 0, c.stream>>>(partials, groups, D, dgamma, dbeta, nsum == 3 ? dx_colsum : nullptr);
 }
 
 // ------------------------------------------------------------------------------------------------
