@@ -28,21 +28,21 @@ namespace bsr {
 
 namespace tc {
 
-constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int BM = 128, BN_MAX = 256, BK = 64;       // tile width BN is 256, or 192 where that wastes less of the last wave
 constexpr int STAGES = 4;
 constexpr int UMMA_K = 16;
-constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int STAGE_BYTES_MAX = A_BYTES + BN_MAX * BK * 2;
 constexpr int EPI_WARPS = 8;                     // two warps per TMEM lane quarter, each takes half of the columns
 constexpr int STAGING_BYTES = 32 * 128;          // per epilogue warp: 32 rows x 128 bytes, 16-byte units XOR-swizzled
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * STAGING_BYTES + 1024 /*alignment slack*/ + 128 /*barriers*/;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES_MAX + EPI_WARPS * STAGING_BYTES + 1024 /*alignment slack*/ + 128 /*barriers*/;
 constexpr int THREADS = 64 + EPI_WARPS * 32;
 constexpr uint32_t TMEM_COLS = 512;
 
-// Instruction descriptor: D = f32, A = B = bf16, M = 128, N = 256, operand majors as given.
-__host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn) {
+// Instruction descriptor: D = f32, A = B = bf16, M = 128, N = bn, operand majors as given.
+__host__ __device__ constexpr uint32_t make_idesc(bool a_mn, bool b_mn, int bn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+         ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
 
 // One unit of work of the persistent loop, decoded identically by the three roles.
@@ -77,10 +77,12 @@ __device__ __forceinline__ Work decode_work(int w, int tiles_m, int tiles_n, int
   return k;
 }
 
-template <bool A_MN, bool B_MN, typename TOut>
+template <bool A_MN, bool B_MN, typename TOut, int BN>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TOut* __restrict__ C,
                int M, int N, int K, Epi ep, int tiles_m, int tiles_n, int splits, int kb_per_split, GemmGroup grp, int* status) {
+  constexpr int B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr int HALF_CHUNKS = BN / 64;               // 32-column chunks per epilogue warp
   extern __shared__ unsigned char smem_dyn[];
   uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   uint32_t staging0 = base + STAGES * STAGE_BYTES;
@@ -151,7 +153,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else if (warp == 1) {
     // ------------------------------- MMA issuer ---------------------------------
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc(A_MN, B_MN);
+      constexpr uint32_t idesc = make_idesc(A_MN, B_MN, BN);
       int stage = 0;
       uint32_t phase = 0;
       int local = 0;
@@ -185,7 +187,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // ------------------------------- epilogue -----------------------------------
     int ew = warp - 2;                      // 0..7
     int quarter = warp & 3;                 // TMEM lanes 32*quarter .. 32*quarter+31 (fixed by the warp's rank)
-    int chalf = ew >> 2;                    // which 128 of the tile's 256 columns
+    int chalf = ew >> 2;                    // which half of the tile's columns
     unsigned char* st = smem_dyn + (staging0 - smem_u32(smem_dyn)) + ew * STAGING_BYTES;
     int local = 0;
     bool ok = true;
@@ -204,8 +206,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int row0 = mt * BM + quarter * 32;
       TOut* Cs = C + wk.c_off;
 #pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {
-        int cchunk = chalf * 4 + cc;
+      for (int cc = 0; cc < HALF_CHUNKS; ++cc) {
+        int cchunk = chalf * HALF_CHUNKS + cc;
         uint32_t r[32];
         uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cchunk * 32);
         tmem_ld32(taddr, r);
@@ -268,10 +270,10 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t outer,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool A_MN, bool B_MN, typename TOut>
+template <bool A_MN, bool B_MN, typename TOut, int BN = BN_MAX>
 static int launch(const Ctx& c, const CUtensorMap& ma, const CUtensorMap& mb, void* C, int m, int n, int k, const Epi& ep,
                   int tiles_m, int tiles_n, int splits, int kb_per_split, const GemmGroup& grp) {
-  auto kern = gemm_tc_kernel<A_MN, B_MN, TOut>;
+  auto kern = gemm_tc_kernel<A_MN, B_MN, TOut, BN>;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return -3;
@@ -308,13 +310,21 @@ int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const voi
   if (a_mn && !b_mn) return -1;                 // combination not instantiated
   CUtensorMap ma, mb;
   bool ok = a_mn ? make_map(&ma, A, (uint64_t)m, (uint64_t)k, (uint64_t)lda, BK) : make_map(&ma, A, (uint64_t)k, (uint64_t)m, (uint64_t)lda, BM);
-  ok = ok && (b_mn ? make_map(&mb, B, (uint64_t)n, (uint64_t)k, (uint64_t)ldb, BK) : make_map(&mb, B, (uint64_t)k, (uint64_t)n, (uint64_t)ldb, BN));
+  int sms = c.sm_count > 0 ? c.sm_count : 148;
+  // Tile width: 192 columns instead of 256 where the narrower tiles fill the SMs' last wave better (a persistent CTA
+  // per SM walks ceil(tiles / SMs) tiles; the time goes with that count times the tile width).  Not for operand A
+  // read along m (weight gradients: those are split along k instead).
+  int bn = BN_MAX;
+  if (!a_mn) {
+    long w256 = (long)ceil_div(ceil_div(m, BM) * ceil_div(n, 256), sms) * 256, w192 = (long)ceil_div(ceil_div(m, BM) * ceil_div(n, 192), sms) * 192;
+    if (w192 < w256) bn = 192;
+  }
+  ok = ok && (b_mn ? make_map(&mb, B, (uint64_t)n, (uint64_t)k, (uint64_t)ldb, BK) : make_map(&mb, B, (uint64_t)k, (uint64_t)n, (uint64_t)ldb, bn));
   if (!ok) return -2;
-  int tiles_m = ceil_div(m, BM), tiles_n = ceil_div(n, BN);
+  int tiles_m = ceil_div(m, BM), tiles_n = ceil_div(n, bn);
   int total_kb = ceil_div(k, BK);
   int splits = 1;
   bool plain = e.bias == nullptr && e.residual == nullptr && e.act == 0;
-  int sms = c.sm_count > 0 ? c.sm_count : 148;
   if (out_is_float && plain && split_ws != nullptr && tiles_m * tiles_n * 2 <= sms && total_kb >= 8) {
     splits = sms / (tiles_m * tiles_n);
     if (splits > total_kb / 4) splits = total_kb / 4;
@@ -329,14 +339,20 @@ int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const voi
   void* dst = (splits > 1) ? (void*)split_ws : C;
   if (c.prof != nullptr && c.prof->on) c.prof->begin(c.stream, 2.0 * m * n * (double)k);
   int rc;
-  if (out_is_float) {
-    if (a_mn) rc = launch<true, true, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, GemmGroup());
-    else if (b_mn) rc = launch<false, true, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, GemmGroup());
-    else rc = launch<false, false, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, GemmGroup());
+  GemmGroup gg;
+  if (bn == 192) {
+    if (out_is_float) rc = b_mn ? launch<false, true, float, 192>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, gg)
+                                : launch<false, false, float, 192>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, gg);
+    else rc = b_mn ? launch<false, true, bf16, 192>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, gg)
+                   : launch<false, false, bf16, 192>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, gg);
+  } else if (out_is_float) {
+    if (a_mn) rc = launch<true, true, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, gg);
+    else if (b_mn) rc = launch<false, true, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, gg);
+    else rc = launch<false, false, float>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, gg);
   } else {
-    if (a_mn) rc = launch<true, true, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, GemmGroup());
-    else if (b_mn) rc = launch<false, true, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, GemmGroup());
-    else rc = launch<false, false, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, GemmGroup());
+    if (a_mn) rc = launch<true, true, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, gg);
+    else if (b_mn) rc = launch<false, true, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, gg);
+    else rc = launch<false, false, bf16>(c, ma, mb, dst, m, n, k, ep, tiles_m, tiles_n, splits, kb_per_split, gg);
   }
   if (rc != 0) return rc;
   if (splits > 1) {
@@ -356,7 +372,7 @@ int gemm_tc_grouped_rows(const Ctx& c, const void* A, const void* Bst, int b_mn,
   CUtensorMap ma, mb;
   bool ok = make_map(&ma, A, (uint64_t)k, (uint64_t)rows_cap, (uint64_t)k, BM);
   ok = ok && (b_mn ? make_map(&mb, Bst, (uint64_t)n, (uint64_t)experts * k, (uint64_t)n, BK)
-                   : make_map(&mb, Bst, (uint64_t)k, (uint64_t)experts * n, (uint64_t)k, BN));
+                   : make_map(&mb, Bst, (uint64_t)k, (uint64_t)experts * n, (uint64_t)k, BN_MAX));
   if (!ok) return -2;
   GemmGroup g;
   g.mode = 1;
@@ -365,7 +381,7 @@ int gemm_tc_grouped_rows(const Ctx& c, const void* A, const void* Bst, int b_mn,
   g.bias_stride = n;
   Epi ep;
   ep.bias = e.bias; ep.residual = e.residual; ep.aux_out = e.aux_out; ep.aux_in = e.aux_in; ep.act = e.act;
-  int tiles_m = rows_cap / BM, tiles_n = ceil_div(n, BN);
+  int tiles_m = rows_cap / BM, tiles_n = ceil_div(n, BN_MAX);
   if (c.prof != nullptr && c.prof->on) c.prof->begin(c.stream, 2.0 * rows_cap * n * (double)k);
   int rc;
   if (out_is_float)
@@ -391,7 +407,7 @@ int gemm_tc_grouped_wgrad(const Ctx& c, const void* dY, const void* X, float* dW
   Epi ep;
   ep.bias = nullptr; ep.residual = nullptr; ep.aux_out = nullptr; ep.aux_in = nullptr; ep.act = 0;
   if (c.prof != nullptr && c.prof->on) c.prof->begin(c.stream, 2.0 * rows_cap * n * (double)m);
-  int rc = launch<true, true, float>(c, ma, mb, dW, m, n, rows_cap, ep, ceil_div(m, BM), ceil_div(n, BN), experts, 0, g);
+  int rc = launch<true, true, float>(c, ma, mb, dW, m, n, rows_cap, ep, ceil_div(m, BM), ceil_div(n, BN_MAX), experts, 0, g);
   if (c.prof != nullptr && c.prof->on) c.prof->end(c.stream);
   return rc;
 }
