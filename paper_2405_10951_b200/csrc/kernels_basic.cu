@@ -306,7 +306,11 @@ static void launch_ln_bwd(const Ctx& c, int groups, size_t smem, const void* dy,
   int nch = ceil_div(D, 128);
 #define BSR_LN_BWD(N)                                                                                                   \
   do {                                                                                                                  \
-    cudaFuncSetAttribute(layernorm_bwd_kernel<TDY, TC, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);       \
+    static size_t attr = 0;               /* the limit only grows: graph nodes captured earlier keep launching */ \
+    if (smem > attr) {                                                                                                  \
+      cudaFuncSetAttribute(layernorm_bwd_kernel<TDY, TC, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);     \
+      attr = smem;                                                                                                      \
+    }                                                                                                                   \
     layernorm_bwd_kernel<TDY, TC, N><<<groups, LNB_WARPS * 32, smem, c.stream>>>((const TDY*)dy, x, x_stride, mean, rstd, g, dres, \
                                                                                  dx, dx_stride, (TC*)dx_copy, partials, rows, D, nsum); \
   } while (0)
