@@ -199,12 +199,36 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       Epi epw = ep;
       if (epw.bias != nullptr) epw.bias += wk.bias_off;
       bool empty = wk.kb0 >= wk.kb1;          // an expert without tokens: its gradient tile is zero
+      int row0 = mt * BM + quarter * 32;
+      TOut* Cs = C + wk.c_off;
+      // float outputs without activation take the single-transposition path; their residual is fetched a chunk ahead
+      const bool f32_path = sizeof(TOut) == 4 && epw.act == 0 && epw.aux_out == nullptr;
+      const bool has_res = f32_path && epw.residual != nullptr;
+      uint4 xn[8];
+      if (has_res) chunk_issue((const float*)epw.residual, N, row0, nt * BN + chalf * HALF_CHUNKS * 32, M, N, lane, xn);
       ok = mbar_wait(tfull_bar(buf), (local >> 1) & 1, abortp);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      int row0 = mt * BM + quarter * 32;
-      TOut* Cs = C + wk.c_off;
+      if (f32_path) {
+#pragma unroll
+        for (int cc = 0; cc < HALF_CHUNKS; ++cc) {
+          int cchunk = chalf * HALF_CHUNKS + cc;
+          uint4 xc[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) xc[i] = xn[i];
+          if (has_res && cc + 1 < HALF_CHUNKS) chunk_issue((const float*)epw.residual, N, row0, nt * BN + (cchunk + 1) * 32, M, N, lane, xn);
+          uint32_t r[32];
+          uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cchunk * 32);
+          tmem_ld32(taddr, r);
+          tmem_ld_wait();
+          if (empty) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r[j] = 0u;
+          }
+          epilogue_chunk_f32(r, epw.bias, (float*)Cs, M, N, row0, nt * BN + cchunk * 32, st, lane, xc, has_res);
+        }
+      } else {
 #pragma unroll 1
       for (int cc = 0; cc < HALF_CHUNKS; ++cc) {
         int cchunk = chalf * HALF_CHUNKS + cc;
@@ -217,6 +241,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           for (int j = 0; j < 32; ++j) r[j] = 0u;
         }
         epilogue_chunk<TOut>(r, epw, Cs, M, N, row0, nt * BN + cchunk * 32, st, lane);
+      }
       }
       tc_fence_before();
       __syncwarp();

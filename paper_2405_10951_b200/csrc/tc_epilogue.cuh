@@ -196,6 +196,44 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t* r, const Epi& ep,
 }
 
 
+// ---- float outputs without activation (projection, second FFN layer, weight gradients) ----------------------------
+// The accumulators are transposed once, through the staging buffer, into the row-contiguous order in which global
+// memory is read and written; bias and residual are added in that order, so the residual needs no staging at all and
+// its loads (issued by chunk_issue a chunk ahead, the first of a tile before the tile's accumulator is complete) stay
+// in flight while the tensor-memory read and the transposition proceed.
+__device__ __forceinline__ void chunk_issue(const float* g, int ld, int row0, int col0, int M, int N, int lane, uint4* x) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    int r = i * 4 + lane / 8, col = col0 + (lane % 8) * 4;
+    x[i] = make_uint4(0, 0, 0, 0);
+    if (row0 + r < M && col < N) x[i] = ld_stream(g + (size_t)(row0 + r) * ld + col);
+  }
+}
+__device__ __forceinline__ void epilogue_chunk_f32(const uint32_t* r, const float* bias, float* Cs, int M, int N, int row0, int col0,
+                                                   unsigned char* st, int lane, const uint4* xres, bool has_res) {
+  if (row0 < M && col0 < N) {
+    using IO = ChunkIO<float>;
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      *reinterpret_cast<uint4*>(st + IO::slot(lane, u)) = make_uint4(r[4 * u], r[4 * u + 1], r[4 * u + 2], r[4 * u + 3]);
+    __syncwarp();
+    int u = lane % 8, col = col0 + u * 4;
+    float4 bb = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (bias != nullptr && col < N) bb = __ldg(reinterpret_cast<const float4*>(bias + col));
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      int rr = i * 4 + lane / 8;
+      uint4 a = *reinterpret_cast<const uint4*>(st + IO::slot(rr, u));
+      float4 v = make_float4(__uint_as_float(a.x) + bb.x, __uint_as_float(a.y) + bb.y, __uint_as_float(a.z) + bb.z, __uint_as_float(a.w) + bb.w);
+      if (has_res) {
+        v.x += __uint_as_float(xres[i].x); v.y += __uint_as_float(xres[i].y); v.z += __uint_as_float(xres[i].z); v.w += __uint_as_float(xres[i].w);
+      }
+      if (row0 + rr < M && col < N) *reinterpret_cast<float4*>(Cs + (size_t)(row0 + rr) * N + col) = v;
+    }
+    __syncwarp();
+  }
+}
+
 // ---- the same with the auxiliary input (residual, or the stored pre-activation) prefetched one chunk ahead ----
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
