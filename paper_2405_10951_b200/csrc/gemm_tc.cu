@@ -204,8 +204,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       // float outputs without activation take the single-transposition path; their residual is fetched a chunk ahead
       const bool f32_path = sizeof(TOut) == 4 && epw.act == 0 && epw.aux_out == nullptr;
       const bool has_res = f32_path && epw.residual != nullptr;
+      // the stored pre-activation of the GELU derivative is fetched a chunk ahead as well
+      const bool pre_z = sizeof(TOut) == 2 && epw.act == 2;       // (bf16 outputs: dz of the FFN backward)
       uint4 xn[8];
       if (has_res) chunk_issue((const float*)epw.residual, N, row0, nt * BN + chalf * HALF_CHUNKS * 32, M, N, lane, xn);
+      if (pre_z) chunk_issue((const bf16*)epw.aux_in, N, row0, nt * BN + chalf * HALF_CHUNKS * 32, M, N, lane, xn);
       ok = mbar_wait(tfull_bar(buf), (local >> 1) & 1, abortp);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -232,6 +235,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll 1
       for (int cc = 0; cc < HALF_CHUNKS; ++cc) {
         int cchunk = chalf * HALF_CHUNKS + cc;
+        float z[sizeof(TOut) == 2 ? 32 : 1];
+        if (sizeof(TOut) == 2 && pre_z) {
+          chunk_land_bf16(xn, st, lane, z);
+          if (cc + 1 < HALF_CHUNKS) chunk_issue((const bf16*)epw.aux_in, N, row0, nt * BN + (cchunk + 1) * 32, M, N, lane, xn);
+        }
         uint32_t r[32];
         uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cchunk * 32);
         tmem_ld32(taddr, r);
@@ -240,7 +248,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
           for (int j = 0; j < 32; ++j) r[j] = 0u;
         }
-        epilogue_chunk<TOut>(r, epw, Cs, M, N, row0, nt * BN + cchunk * 32, st, lane);
+        epilogue_chunk<TOut>(r, epw, Cs, M, N, row0, nt * BN + cchunk * 32, st, lane, pre_z ? z : nullptr);
       }
       }
       tc_fence_before();

@@ -159,9 +159,10 @@ template <> __device__ __forceinline__ uint4 ChunkIO<bf16>::pack(const float* f)
 }
 
 // v[j]: accumulator of (row0 + lane, col0 + j).  All lanes of the warp take part (row0, col0 are warp-uniform).
+// zpre: the chunk of the stored pre-activation for act == 2, already in this lane's row order (or null: loaded here).
 template <typename TOut>
 __device__ __forceinline__ void epilogue_chunk(const uint32_t* r, const Epi& ep, TOut* Cs, int M, int N, int row0, int col0,
-                                               unsigned char* st, int lane) {
+                                               unsigned char* st, int lane, const float* zpre = nullptr) {
   if (row0 < M && col0 < N) {
     float v[32];
 #pragma unroll
@@ -180,10 +181,15 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t* r, const Epi& ep,
 #pragma unroll
       for (int j = 0; j < 32; j += 2) gelu_fast2(v[j], v[j + 1]);
     } else if (ep.act == 2) {
-      float z[32];
-      ChunkIO<bf16>::load((const bf16*)ep.aux_in, N, row0, col0, M, N, st, lane, z);
+      if (zpre != nullptr) {
 #pragma unroll
-      for (int j = 0; j < 32; j += 2) gelu_grad_mul2(v[j], v[j + 1], z[j], z[j + 1]);
+        for (int j = 0; j < 32; j += 2) gelu_grad_mul2(v[j], v[j + 1], zpre[j], zpre[j + 1]);
+      } else {
+        float z[32];
+        ChunkIO<bf16>::load((const bf16*)ep.aux_in, N, row0, col0, M, N, st, lane, z);
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) gelu_grad_mul2(v[j], v[j + 1], z[j], z[j + 1]);
+      }
     }
     if (ep.residual != nullptr) {
       float rr[32];
@@ -232,6 +238,29 @@ __device__ __forceinline__ void epilogue_chunk_f32(const uint32_t* r, const floa
     }
     __syncwarp();
   }
+}
+
+// Stored pre-activation chunk (bf16) fetched ahead of use: four 16-byte units per lane in row-contiguous order, later
+// turned into this lane's row through the staging buffer.
+__device__ __forceinline__ void chunk_issue(const bf16* g, int ld, int row0, int col0, int M, int N, int lane, uint4* x) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    int r = i * 8 + lane / 4, col = col0 + (lane % 4) * 8;
+    x[i] = make_uint4(0, 0, 0, 0);
+    if (row0 + r < M && col < N) x[i] = ld_stream(g + (size_t)(row0 + r) * ld + col);
+  }
+}
+__device__ __forceinline__ void chunk_land_bf16(const uint4* x, unsigned char* st, int lane, float* v) {
+  using IO = ChunkIO<bf16>;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(st + IO::slot(i * 8 + lane / 4, lane % 4)) = x[i];
+  __syncwarp();
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    uint4 y = *reinterpret_cast<const uint4*>(st + IO::slot(lane, u));
+    IO::unpack(y, v + u * 8);
+  }
+  __syncwarp();
 }
 
 // ---- the same with the auxiliary input (residual, or the stored pre-activation) prefetched one chunk ahead ----
