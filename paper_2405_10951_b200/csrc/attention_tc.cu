@@ -20,6 +20,7 @@ constexpr int AT_BOX = 64;                       // rows per TMA box
 constexpr int AT_BOX_BYTES = AT_BOX * AT_D * 2;  // 8 KB
 constexpr int AT_QROWS = 128;
 constexpr int AT_MAXKEYS = 256;
+constexpr int AT_LONG_KB = 128;                  // keys per block of the two-walk kernel for longer sequences
 
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -340,7 +341,7 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 }
 
 // ------------------------------------------------------------------------------------------------
-// Forward for longer sequences (T > 256): the keys are walked in blocks of up to 256, twice.  The first walk
+// Forward for longer sequences (T > 256): the keys are walked in blocks of up to 128, twice.  The first walk
 // only computes S = Q K^T per block and keeps the running row maximum and row sum; the second walk recomputes S,
 // forms P = exp(S - max) with the final maximum (so the accumulator never needs rescaling) and adds P V into a
 // separate set of tensor-memory columns.  One CTA per (image, head, 128 queries), one block in flight.
@@ -351,10 +352,10 @@ attn_fwd_tc_long_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __res
   extern __shared__ unsigned char smem_dyn[];
   uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
-  constexpr int KB = AT_MAXKEYS;                         // keys per block
-  constexpr uint32_t KV_BYTES = KB * 128;                // 32 KB
+  constexpr int KB = AT_LONG_KB;                         // keys per block
+  constexpr uint32_t KV_BYTES = KB * 128;                // 16 KB
   uint32_t sQ = base, sK = sQ + 2 * AT_BOX_BYTES, sV = sK + KV_BYTES, sP = sV + KV_BYTES;
-  uint32_t bars = sP + 4 * (AT_QROWS * 128);
+  uint32_t bars = sP + (KB / 64) * (AT_QROWS * 128);
   unsigned char* pP = base_ptr + (sP - base);
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
@@ -369,14 +370,14 @@ attn_fwd_tc_long_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __res
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
-    tmem_alloc(smem_u32(&tmem_slot), 512);
+    tmem_alloc(smem_u32(&tmem_slot), 2 * KB);           // S in the first KB columns, O behind it: two CTAs share an SM
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   uint32_t tmem = tmem_slot;
-  constexpr uint32_t C_O = 256;
+  constexpr uint32_t C_O = KB;
   volatile int* abortp = &abort_flag;
   const float c = 0.125f * 1.4426950408889634f;
   uint32_t trow = tmem + ((uint32_t)(warp * 32) << 16);
@@ -519,7 +520,7 @@ attn_fwd_tc_long_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __res
   __syncthreads();
   if (warp == 0) {
     tc_fence_after();
-    tmem_dealloc(tmem, 512);
+    tmem_dealloc(tmem, 2 * AT_LONG_KB);
   }
   if (tid == 0 && abort_flag && status != nullptr) atomicOr(status, STATUS_TIMEOUT);
 }
@@ -750,7 +751,7 @@ int attention_fwd_tc(const Ctx& c, const void* qkv, void* out, float* lse, float
   CUtensorMap map;
   if (!make_map(&map, qkv, (uint64_t)3 * H * d, (uint64_t)B * T, (uint64_t)3 * H * d, AT_BOX)) return -2;
   if (T > AT_MAXKEYS) {
-    size_t smem_l = 1024 + 2 * (size_t)AT_BOX_BYTES + 2 * (size_t)AT_MAXKEYS * 128 + 4 * (size_t)(AT_QROWS * 128) + 64;
+    size_t smem_l = 1024 + 2 * (size_t)AT_BOX_BYTES + 2 * (size_t)AT_LONG_KB * 128 + (AT_LONG_KB / 64) * (size_t)(AT_QROWS * 128) + 64;
     static bool attr_l = false;
     if (!attr_l) {
       if (cudaFuncSetAttribute(attn_fwd_tc_long_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_l) != cudaSuccess) return -3;

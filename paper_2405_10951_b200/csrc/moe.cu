@@ -11,7 +11,7 @@
 
 namespace bsr {
 
-constexpr int MOE_BLOCK_TOKENS = 256;
+constexpr int MOE_BLOCK_TOKENS = 64;
 constexpr int MOE_MAX_E = 32;
 constexpr int MOE_MAX_K = 4;
 
@@ -31,13 +31,32 @@ moe_route_kernel(const T* __restrict__ y, const T* __restrict__ wg, const int* _
     int task = task_ids ? task_ids[tok / tokens_per_image] : 0;
     const T* yr = y + (size_t)tok * D;
     const T* wt = wg + (size_t)task * E * D;
+    // every lane multiplies its 16-byte pieces of the token by the same pieces of all gate rows (the gate matrix is
+    // small and stays in L1), then the per-expert partial sums are added over the warp
+    constexpr int N = Pack<T>::N;
+    float acc[MOE_MAX_E];
+#pragma unroll
+    for (int e = 0; e < MOE_MAX_E; ++e) acc[e] = 0.f;
+    for (int ch = lane; ch < D / N; ch += 32) {
+      float yv[N];
+      load16(yr + ch * N, yv);
+#pragma unroll
+      for (int e = 0; e < MOE_MAX_E; ++e) {
+        if (e < E) {
+          float wv[N];
+          load16(wt + (size_t)e * D + ch * N, wv);
+#pragma unroll
+          for (int j = 0; j < N; ++j) acc[e] = fmaf(yv[j], wv[j], acc[e]);
+        }
+      }
+    }
     float mine = -INFINITY;                       // lane e ends up with the logit of expert e
-    for (int e = 0; e < E; ++e) {
-      const T* we = wt + (size_t)e * D;
-      float s = 0.f;
-      for (int d = lane; d < D; d += 32) s = fmaf(to_f(yr[d]), to_f(we[d]), s);
-      s = warp_sum(s);
-      if (lane == e) mine = s;
+#pragma unroll
+    for (int e = 0; e < MOE_MAX_E; ++e) {
+      if (e < E) {
+        float s = warp_sum(acc[e]);
+        if (lane == e) mine = s;
+      }
     }
     float sel[MOE_MAX_K];
     int sid[MOE_MAX_K];
