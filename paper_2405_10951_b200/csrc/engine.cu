@@ -502,7 +502,7 @@ int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb
     // MoE layer in place of the FFN (Section 5.2): route, run the chosen experts as grouped GEMMs, combine
     int E = d.moe_experts, K = d.moe_top_k;
     MoeBufs mb = moe_bufs(h, bb);
-    moe_route(c, mb, h->base + bb.y2, h->wb(l, "moe.gate.weight"), task_ids, tail ? 1 : Tf, Mf, D, E, K);
+    moe_route(c, mb, h->base + bb.y2, h->wb(l, "moe.gate.weight"), task_ids, tail ? 1 : Tf, Mf, D, E, K, d.num_tasks);
     int cap = moe_rows_cap(Mf, E, K);
     GemmEpilogue m1;
     m1.bias = (const float*)h->wb(l, "moe.fc1.bias");

@@ -183,7 +183,7 @@ int moe_rows_cap(int M, int E, int K);
 int moe_blocks(int M);
 // y [M, D]: routes every token, builds the segment tables and gathers the expert inputs into b.xg.
 void moe_route(const Ctx& c, const MoeBufs& b, const void* y, const void* wg, const int* task_ids, int tokens_per_image, int M,
-               int D, int E, int K);
+               int D, int E, int K, int num_tasks);
 void moe_combine(const Ctx& c, const MoeBufs& b, const float* res, float* out, int M, int D, int K);
 void moe_combine_bwd(const Ctx& c, const MoeBufs& b, const float* dout, void* dog, float* dw, int M, int D, int E, int K);
 void moe_seg_colsum(const Ctx& c, const MoeBufs& b, const void* x, int cols, int E, float* out);

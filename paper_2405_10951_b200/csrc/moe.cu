@@ -11,73 +11,75 @@
 
 namespace bsr {
 
-constexpr int MOE_BLOCK_TOKENS = 64;
+constexpr int MOE_BLOCK_TOKENS = 128;
 constexpr int MOE_MAX_E = 32;
 constexpr int MOE_MAX_K = 4;
 
 // ---- routing: gate logits, top-k (ties -> lower expert id), softmax over the selected logits -------------------
 template <typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(MOE_BLOCK_TOKENS)
 moe_route_kernel(const T* __restrict__ y, const T* __restrict__ wg, const int* __restrict__ task_ids, int tokens_per_image,
-                 int M, int D, int E, int K, int* __restrict__ eidx, float* __restrict__ ew, int* __restrict__ blk_counts) {
+                 int M, int D, int E, int K, int gate_elems_in_smem, int* __restrict__ eidx, float* __restrict__ ew,
+                 int* __restrict__ blk_counts) {
+  // A thread per token: its row of y against every gate row, the gate matrices of all tasks staged in shared memory
+  // when they fit (all lanes read the same gate element: a broadcast), so no cross-lane reduction is needed and the
+  // top-k is a scan over the thread's own logits.
+  extern __shared__ __align__(16) unsigned char route_smem[];
   __shared__ int counts[MOE_MAX_E];
-  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int N = Pack<T>::N;
   if (threadIdx.x < MOE_MAX_E) counts[threadIdx.x] = 0;
+  const T* gates = wg;
+  if (gate_elems_in_smem > 0) {
+    T* sg = reinterpret_cast<T*>(route_smem);
+    for (int i = threadIdx.x * N; i < gate_elems_in_smem; i += blockDim.x * N)
+      *reinterpret_cast<uint4*>(sg + i) = *reinterpret_cast<const uint4*>(wg + i);
+    gates = sg;
+  }
   __syncthreads();
-  int t0 = blockIdx.x * MOE_BLOCK_TOKENS;
-  for (int tt = warp; tt < MOE_BLOCK_TOKENS; tt += 8) {
-    int tok = t0 + tt;
-    if (tok >= M) break;
+  int tok = blockIdx.x * MOE_BLOCK_TOKENS + threadIdx.x;
+  if (tok < M) {
     int task = task_ids ? task_ids[tok / tokens_per_image] : 0;
     const T* yr = y + (size_t)tok * D;
-    const T* wt = wg + (size_t)task * E * D;
-    // every lane multiplies its 16-byte pieces of the token by the same pieces of all gate rows (the gate matrix is
-    // small and stays in L1), then the per-expert partial sums are added over the warp
-    constexpr int N = Pack<T>::N;
+    const T* gt = gates + (size_t)task * E * D;
     float acc[MOE_MAX_E];
 #pragma unroll
     for (int e = 0; e < MOE_MAX_E; ++e) acc[e] = 0.f;
-    for (int ch = lane; ch < D / N; ch += 32) {
+    for (int ch = 0; ch < D / N; ++ch) {
       float yv[N];
       load16(yr + ch * N, yv);
 #pragma unroll
       for (int e = 0; e < MOE_MAX_E; ++e) {
         if (e < E) {
           float wv[N];
-          load16(wt + (size_t)e * D + ch * N, wv);
+          load16(gt + (size_t)e * D + ch * N, wv);
 #pragma unroll
           for (int j = 0; j < N; ++j) acc[e] = fmaf(yv[j], wv[j], acc[e]);
         }
       }
     }
-    float mine = -INFINITY;                       // lane e ends up with the logit of expert e
-#pragma unroll
-    for (int e = 0; e < MOE_MAX_E; ++e) {
-      if (e < E) {
-        float s = warp_sum(acc[e]);
-        if (lane == e) mine = s;
-      }
-    }
     float sel[MOE_MAX_K];
     int sid[MOE_MAX_K];
-    bool taken = false;
+    uint32_t taken = 0;
     for (int i = 0; i < K; ++i) {
-      float cand = taken ? -INFINITY : mine;
-      float mx = warp_max(cand);
-      uint32_t m = __ballot_sync(0xffffffffu, !taken && cand == mx && lane < E);
-      int win = __ffs(m) - 1;                     // lowest expert id among equals
-      sel[i] = mx;
-      sid[i] = win;
-      if (lane == win) taken = true;
+      float best = -INFINITY;
+      int bi = 0;
+      bool any = false;
+#pragma unroll
+      for (int e = 0; e < MOE_MAX_E; ++e) {
+        if (e < E && !((taken >> e) & 1u) && (!any || acc[e] > best)) {    // strictly greater: the lowest id wins among equals
+          best = acc[e]; bi = e; any = true;
+        }
+      }
+      taken |= 1u << bi;
+      sel[i] = best;
+      sid[i] = bi;
     }
     float den = 0.f;
     for (int i = 0; i < K; ++i) den += expf(sel[i] - sel[0]);
-    if (lane == 0) {
-      for (int i = 0; i < K; ++i) {
-        eidx[(size_t)tok * K + i] = sid[i];
-        ew[(size_t)tok * K + i] = expf(sel[i] - sel[0]) / den;
-        atomicAdd(&counts[sid[i]], 1);            // integer counts: order-independent
-      }
+    for (int i = 0; i < K; ++i) {
+      eidx[(size_t)tok * K + i] = sid[i];
+      ew[(size_t)tok * K + i] = expf(sel[i] - sel[0]) / den;
+      atomicAdd(&counts[sid[i]], 1);              // integer counts: order-independent
     }
   }
   __syncthreads();
@@ -323,14 +325,24 @@ int moe_rows_cap(int M, int E, int K) { return ((M * K + E * 127) + 127) & ~127;
 int moe_blocks(int M) { return ceil_div(M, MOE_BLOCK_TOKENS); }
 
 void moe_route(const Ctx& c, const MoeBufs& b, const void* y, const void* wg, const int* task_ids, int tokens_per_image, int M,
-               int D, int E, int K) {
+               int D, int E, int K, int num_tasks) {
   int nblk = moe_blocks(M);
   int rows_cap = moe_rows_cap(M, E, K);
   note_launch(4);
-  if (c.dtype == 0)
-    moe_route_kernel<float><<<nblk, 256, 0, c.stream>>>((const float*)y, (const float*)wg, task_ids, tokens_per_image, M, D, E, K, b.eidx, b.ew, b.blk_counts);
-  else
-    moe_route_kernel<bf16><<<nblk, 256, 0, c.stream>>>((const bf16*)y, (const bf16*)wg, task_ids, tokens_per_image, M, D, E, K, b.eidx, b.ew, b.blk_counts);
+  size_t es = c.dtype == 0 ? 4 : 2;
+  size_t gate_elems = (size_t)(num_tasks < 1 ? 1 : num_tasks) * E * D;
+  size_t smem = gate_elems * es;
+  if (smem > 96 * 1024) { smem = 0; gate_elems = 0; }       // too large to stage: the gates are read through L1 instead
+  static size_t attr[2] = {0, 0};
+  if (c.dtype == 0) {
+    if (smem > attr[0]) { cudaFuncSetAttribute(moe_route_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr[0] = smem; }
+    moe_route_kernel<float><<<nblk, MOE_BLOCK_TOKENS, smem, c.stream>>>((const float*)y, (const float*)wg, task_ids, tokens_per_image, M, D, E, K,
+                                                                        (int)gate_elems, b.eidx, b.ew, b.blk_counts);
+  } else {
+    if (smem > attr[1]) { cudaFuncSetAttribute(moe_route_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr[1] = smem; }
+    moe_route_kernel<bf16><<<nblk, MOE_BLOCK_TOKENS, smem, c.stream>>>((const bf16*)y, (const bf16*)wg, task_ids, tokens_per_image, M, D, E, K,
+                                                                       (int)gate_elems, b.eidx, b.ew, b.blk_counts);
+  }
   moe_scan_kernel<<<1, 128, 0, c.stream>>>(b.blk_counts, nblk, E, rows_cap / 128, b.blk_off, b.seg_start, b.tile_expert);
   cudaMemsetAsync(b.row_token, 0xFF, (size_t)rows_cap * sizeof(int), c.stream);
   moe_assign_kernel<<<nblk, 256, 0, c.stream>>>(b.eidx, b.ew, b.blk_off, b.seg_start, M, E, K, b.pos, b.row_token, b.row_w);
