@@ -121,34 +121,38 @@ def test_error_paths_leave_the_context_usable():
 
 def test_graph_replay_equals_launch_by_launch():
     """On a capturable stream the step is captured once and replayed; three steps give bit-identical results to the
-    same three steps enqueued kernel by kernel (AdamW's step-dependent scalars are read from device memory)."""
+    same three steps enqueued kernel by kernel on that stream and on the legacy default stream (AdamW's step-dependent
+    scalars are read from device memory)."""
+    import contextlib
     import torch
     from paper_2405_10951_b200 import binding as Bd
     cfg = MINI_BF16
     images, labels, task_ids, params = synth.make_workload(cfg, peaked=True)
     shapes = synth.param_shapes(cfg)
-    names = ("head.0.weight", "blocks.5.mlp.fc1.weight", "blocks.3.attn.qkv.weight")
+    names = ("head.0.weight", "blocks.5.mlp.fc1.weight", "blocks.3.attn.qkv.weight", "blocks.5.mlp.fc1.bias",
+             "blocks.4.attn.qkv.bias", "blocks.3.mlp.fc2.bias", "blocks.4.attn.proj.bias")
     results = []
-    for graph in (False, True):
+    for mode in ("default stream", "stream", "stream + graph"):
         eng = Bd.Engine(cfg)
         eng.set_params(params)
-        eng.set_graph_mode(graph)
+        eng.set_graph_mode(mode == "stream + graph")
         img = eng.images_to_device(images)
         lab = torch.as_tensor(labels).cuda()
         torch.cuda.synchronize()
         s = torch.cuda.Stream()
         losses, out = [], None
-        with torch.cuda.stream(s):
+        with (contextlib.nullcontext() if mode == "default stream" else torch.cuda.stream(s)):
             for _ in range(3):
                 loss, _ = eng.train_step(img, lab, out=out)      # same output buffers from the second step on
                 out = eng.last_out
-                s.synchronize()
+                torch.cuda.current_stream().synchronize()
                 losses.append(float(loss.cpu()[0]))
             eng.sync_status()
             w = {n: eng.get_tensor(n, shapes[n]).cpu().numpy() for n in names}
         results.append((losses, w))
         eng.close()
-    assert results[0][0] == results[1][0]
+    for other in results[1:]:
+        assert results[0][0] == other[0]
+        for n in names:
+            assert np.array_equal(results[0][1][n], other[1][n]), n
     assert results[0][0][2] < results[0][0][0]
-    for n in names:
-        assert np.array_equal(results[0][1][n], results[1][1][n]), n
