@@ -154,6 +154,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // ------------------------------- MMA issuer ---------------------------------
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc(A_MN, B_MN, BN);
+      // k step of 16 inside a stage: 32 bytes along a K-major row, 16 rows of 128 bytes for an MN-major operand
+      constexpr uint32_t A_KSTEP = (A_MN ? UMMA_K * 128 : UMMA_K * 2) >> 4, B_KSTEP = (B_MN ? UMMA_K * 128 : UMMA_K * 2) >> 4;
+      const uint64_t desc_a0 = A_MN ? make_desc(base, BK * 128, 1024) : make_desc(base, 16, 1024);
+      const uint64_t desc_b0 = B_MN ? make_desc(base + A_BYTES, BK * 128, 1024) : make_desc(base + A_BYTES, 16, 1024);
       int stage = 0;
       uint32_t phase = 0;
       int local = 0;
@@ -169,13 +173,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abortp)) { ok = false; break; }
           tc_fence_after();
-          uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
+          // descriptors of this stage: only the 16-byte-unit address field (low bits) moves with the stage and the k step
+          uint64_t da = desc_a0 + (uint64_t)((stage * STAGE_BYTES) >> 4), db = desc_b0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
+          umma_bf16(d_tmem, da, db, idesc, kb > kb0 ? 1u : 0u);
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
-            uint64_t da = A_MN ? make_desc(sa + k * (UMMA_K * 128), BK * 128, 1024) : make_desc(sa + k * (UMMA_K * 2), 16, 1024);
-            uint64_t db = B_MN ? make_desc(sb + k * (UMMA_K * 128), BK * 128, 1024) : make_desc(sb + k * (UMMA_K * 2), 16, 1024);
-            umma_bf16(d_tmem, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
-          }
+          for (int k = 1; k < BK / UMMA_K; ++k)
+            umma_bf16_acc(d_tmem, da + (uint64_t)(k * A_KSTEP), db + (uint64_t)(k * B_KSTEP), idesc);
           umma_commit(empty_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
