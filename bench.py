@@ -167,7 +167,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="vit_b", choices=list(synth.CONFIGS))
-    ap.add_argument("--ref-batch", type=int, default=8)
+    ap.add_argument("--ref-batch", type=int, default=48)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--gemm-mode", type=int, default=None, help="1: one CTA per tile, 2: CTA pairs (library default if omitted)")
     args = ap.parse_args()
@@ -239,10 +239,14 @@ def main():
 
     # ---- end to end: pinned host images in, loss out, every step ----------------------------------
     # Two device staging buffers: the copy of the next step's images (its own stream) overlaps the current step, as an
-    # input pipeline would; every step still waits for its own copy and the host reads every step's loss.
+    # input pipeline would; every step still waits for its own copy, and the host reads every step's loss, one step
+    # behind the launches (the read of step i-1 waits only for that step).
     stages = [torch.empty_like(dev_img), torch.empty_like(dev_img)]
     copy_stream = torch.cuda.Stream()
     copied = [torch.cuda.Event(), torch.cuda.Event()]
+    read_back = [torch.cuda.Event(), torch.cuda.Event()]
+    host_losses = [torch.empty(1, dtype=torch.float32).pin_memory(), torch.empty(1, dtype=torch.float32).pin_memory()]
+    e2e_losses = []
     for sbuf in stages:                                   # untimed: lets the library capture its graph for each buffer
         sbuf.copy_(dev_img)
         eng.train_step(sbuf, lab, tid, want_kept=False, out=out)
@@ -256,14 +260,21 @@ def main():
         copied[0].record(copy_stream)
     for i in range(args.steps):
         cur = i & 1
-        if i + 1 < args.steps:                            # the previous user of that buffer (step i-1) has been waited for
+        if i + 1 < args.steps:
             with torch.cuda.stream(copy_stream):
+                if i > 0:
+                    copy_stream.wait_event(read_back[cur ^ 1])       # step i-1, the last user of that buffer, is done
                 stages[cur ^ 1].copy_(host_img, non_blocking=True)
                 copied[cur ^ 1].record(copy_stream)
         stream.wait_event(copied[cur])
         loss, _ = eng.train_step(stages[cur], lab, tid, want_kept=False, out=out)
-        host_loss.copy_(loss, non_blocking=True)
-        stream.synchronize()
+        host_losses[cur].copy_(loss, non_blocking=True)
+        read_back[cur].record(stream)
+        if i > 0:                                         # the host reads every loss, one step behind the launches
+            read_back[cur ^ 1].synchronize()
+            e2e_losses.append(float(host_losses[cur ^ 1][0]))
+    read_back[(args.steps - 1) & 1].synchronize()
+    e2e_losses.append(float(host_losses[(args.steps - 1) & 1][0]))
     f1.record(stream)
     barrier()
     ms_e2e = f0.elapsed_time(f1)

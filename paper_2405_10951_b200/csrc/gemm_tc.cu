@@ -281,6 +281,43 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ partial, float* _
   *reinterpret_cast<float4*>(out + i) = acc;
 }
 
+// The same reduction followed by the epilogue the GEMM kernel would have applied (bias, GELU with optional copy of the
+// pre-activation, GELU derivative of a stored pre-activation, residual), for products whose few tiles are split along k.
+template <typename TOut>
+__global__ void splitk_reduce_epi_kernel(const float* __restrict__ partial, TOut* __restrict__ out, int m, int n, int splits, Epi ep) {
+  size_t total = (size_t)m * n;
+  size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i >= total) return;
+  float4 a4 = *reinterpret_cast<const float4*>(partial + i);
+  for (int s = 1; s < splits; ++s) {
+    float4 v = *reinterpret_cast<const float4*>(partial + (size_t)s * total + i);
+    a4.x += v.x; a4.y += v.y; a4.z += v.z; a4.w += v.w;
+  }
+  float v[4] = {a4.x, a4.y, a4.z, a4.w};
+  int col = (int)(i % (size_t)n);                    // n is a multiple of 4: the four values share a row
+  if (ep.bias != nullptr) {
+    float4 bb = *reinterpret_cast<const float4*>(ep.bias + col);
+    v[0] += bb.x; v[1] += bb.y; v[2] += bb.z; v[3] += bb.w;
+  }
+  if (ep.act == 1) {
+    if (ep.aux_out != nullptr) store4(reinterpret_cast<TOut*>(ep.aux_out) + i, v);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] = gelu_f(v[j]);
+  } else if (ep.act == 2) {
+    float z[4];
+    load4(reinterpret_cast<const bf16*>(ep.aux_in) + i, z);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] *= gelu_grad_f(z[j]);
+  }
+  if (ep.residual != nullptr) {
+    float r[4];
+    load4(reinterpret_cast<const TOut*>(ep.residual) + i, r);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] += r[j];
+  }
+  store4(out + i, v);
+}
+
 EncodeFn encode_fn() {
   static EncodeFn fn = nullptr;
   static bool tried = false;
@@ -361,7 +398,9 @@ int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const voi
   int total_kb = ceil_div(k, BK);
   int splits = 1;
   bool plain = e.bias == nullptr && e.residual == nullptr && e.act == 0;
-  if (out_is_float && plain && split_ws != nullptr && tiles_m * tiles_n * 2 <= sms && total_kb >= 8) {
+  // split along k: weight gradients (plain float outputs) and the few-row products of the classification-only tail,
+  // whose epilogue then runs in the reduction
+  if (split_ws != nullptr && tiles_m * tiles_n * 2 <= sms && total_kb >= 8 && ((out_is_float && plain) || (m <= 256 && (n % 4) == 0))) {
     splits = sms / (tiles_m * tiles_n);
     if (splits > total_kb / 4) splits = total_kb / 4;
     if (splits > 16) splits = 16;
@@ -370,8 +409,14 @@ int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const voi
   }
   int kb_per_split = ceil_div(total_kb, splits);
   splits = ceil_div(total_kb, kb_per_split);
-  Epi ep;
-  ep.bias = e.bias; ep.residual = e.residual; ep.aux_out = e.aux_out; ep.aux_in = e.aux_in; ep.act = e.act;
+  Epi ep_full;
+  ep_full.bias = e.bias; ep_full.residual = e.residual; ep_full.aux_out = e.aux_out; ep_full.aux_in = e.aux_in; ep_full.act = e.act;
+  // split products write plain float partials; their epilogue runs in the reduction
+  const bool deferred = splits > 1 && !(out_is_float && plain);
+  Epi ep = ep_full;
+  if (splits > 1) { ep.bias = nullptr; ep.residual = nullptr; ep.aux_out = nullptr; ep.aux_in = nullptr; ep.act = 0; }
+  const int final_is_float = out_is_float;
+  if (splits > 1) out_is_float = 1;
   void* dst = (splits > 1) ? (void*)split_ws : C;
   if (c.prof != nullptr && c.prof->on) c.prof->begin(c.stream, 2.0 * m * n * (double)k);
   int rc;
@@ -393,7 +438,14 @@ int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const voi
   if (rc != 0) return rc;
   if (splits > 1) {
     size_t total = (size_t)m * n;
-    splitk_reduce(c.stream, split_ws, (float*)C, total, splits);
+    if (!deferred) {
+      splitk_reduce(c.stream, split_ws, (float*)C, total, splits);
+    } else {
+      note_launch(1);
+      int blocks = ceil_div((long)(total / 4), 256);
+      if (final_is_float) splitk_reduce_epi_kernel<float><<<blocks, 256, 0, c.stream>>>(split_ws, (float*)C, m, n, splits, ep_full);
+      else splitk_reduce_epi_kernel<bf16><<<blocks, 256, 0, c.stream>>>(split_ws, (bf16*)C, m, n, splits, ep_full);
+    }
   }
   if (c.prof != nullptr && c.prof->on) c.prof->end(c.stream);
   return 0;
