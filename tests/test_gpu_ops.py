@@ -47,7 +47,9 @@ def test_linear_bf16_simt(m, n, k):
 @pytest.mark.parametrize("dtype,tol,tc", [("fp32", 2e-6, False), ("bf16", 4e-3, False), ("bf16", 6e-3, True)])
 @pytest.mark.parametrize("B,T,H,d", [(2, 65, 3, 64), (3, 47, 2, 32), (2, 197, 6, 64), (1, 5, 1, 16), (1, 290, 2, 64),
                                      (3, 140, 12, 64), (2, 100, 2, 64), (5, 72, 3, 64), (1, 256, 1, 64), (2, 129, 2, 64),
-                                     (1, 16, 1, 64), (4, 1, 2, 64), (2, 577, 3, 64), (1, 257, 2, 64), (1, 512, 1, 64)])
+                                     (1, 16, 1, 64), (4, 1, 2, 64), (2, 577, 3, 64), (1, 257, 2, 64), (1, 512, 1, 64),
+                                     # more (image, head) pairs than SMs: every persistent CTA walks several tiles
+                                     (40, 197, 12, 64), (31, 140, 12, 64), (64, 100, 12, 64), (50, 72, 7, 64), (13, 256, 12, 64)])
 def test_attention_forward(dtype, tol, tc, B, T, H, d):
     import torch
     from paper_2405_10951_b200 import binding as Bd
