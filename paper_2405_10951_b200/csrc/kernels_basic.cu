@@ -352,7 +352,20 @@ __global__ void colsum_kernel(const T* __restrict__ x, int rows, int cols, float
 #pragma unroll
   for (int j = 0; j < N; ++j) acc[j] = 0.f;
   if (col0 < cols) {
-    for (int r = blockIdx.y * CS_ROWLANES + ty; r < rows; r += gridDim.y * CS_ROWLANES) {
+    // four rows per trip: their loads are independent and issued together, the additions keep the row order
+    const int step = gridDim.y * CS_ROWLANES;
+    int r = blockIdx.y * CS_ROWLANES + ty;
+    for (; r + 3 * step < rows; r += 4 * step) {
+      float v[4][N];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) load16(x + (long)(r + u * step) * cols + col0, v[u]);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+#pragma unroll
+        for (int j = 0; j < N; ++j) acc[j] += v[u][j];
+      }
+    }
+    for (; r < rows; r += step) {
       float v[N];
       load16(x + (long)r * cols + col0, v);
 #pragma unroll
