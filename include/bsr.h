@@ -51,6 +51,7 @@ typedef enum {
 
 enum { BSR_DTYPE_FP32 = 0, BSR_DTYPE_BF16 = 1 };
 enum { BSR_FUSE_NONE = 0, BSR_FUSE_WEIGHTED_SUM = 1 };
+enum { BSR_OPT_ADAMW = 0, BSR_OPT_SGD = 1 };
 enum { BSR_MAX_DROPS = 8, BSR_MAX_TASKS = 4, BSR_MAX_DEPTH = 32 };
 
 /* Model dimensions (Section 3.1: N patches + 1 classification token, embedding length L, H heads). */
@@ -77,6 +78,11 @@ typedef struct {
   int32_t fuse_mode;                /* BSR_FUSE_* */
   float lr, beta1, beta2, eps, weight_decay;   /* AdamW (Section 5, training hyper-parameters) */
   int32_t max_batch;
+  /* Optimiser (Section 5: AdamW for the DeiT-S runs, SGD for the ViT-B and MoE runs).  BSR_OPT_SGD is SGD with
+   * momentum: d = g + weight_decay p (matrices only), buf <- momentum buf + d, p <- p - lr buf, buf starting at
+   * zero; the buffer is read under the name "adam_m/<param>" and "adam_v/<param>" stays zero. */
+  int32_t optimizer;                /* BSR_OPT_* */
+  float momentum;
 } bsr_config;
 
 /* HBM footprint of a created handle, in bytes. */

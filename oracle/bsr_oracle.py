@@ -451,6 +451,16 @@ def adamw(cfg, p, g, m, v, step, decay):
     return new, m, v
 
 
+def sgd_momentum(cfg, p, g, buf, decay):
+    """SGD with momentum (Section 5, training hyper-parameters: the ViT-B runs use SGD with cosine decay; the paper
+    gives neither momentum nor weight decay, so both are configuration values).  The weight decay is added to the
+    gradient, the buffer accumulates it with factor momentum and starts at zero: d = g + wd p; buf <- mu buf + d;
+    p <- p - lr buf."""
+    d = g + (cfg.weight_decay * p if decay else 0.0)
+    buf = cfg.momentum * buf + d
+    return p - cfg.lr * buf, buf
+
+
 def train_step(cfg, params, images, labels, task_ids=None, forced_keep=None, opt_state=None, step=1, forced_experts=None):
     """One BSR fine-tuning step.  Returns loss, logits, gradients, updated parameters and moments."""
     fw = forward(cfg, params, images, task_ids, forced_keep, keep_cache=True, forced_experts=forced_experts)
@@ -477,8 +487,12 @@ def train_step(cfg, params, images, labels, task_ids=None, forced_keep=None, opt
     new_params = dict(params)
     new_m, new_v = {}, {}
     for n in names:
-        new_params[n], new_m[n], new_v[n] = adamw(cfg, params[n], grads[n], opt_state["m"][n],
-                                                  opt_state["v"][n], step, is_decayed(n))
+        if getattr(cfg, "optimizer", "adamw") == "sgd":      # the momentum buffer takes the place of m, v stays zero
+            new_params[n], new_m[n] = sgd_momentum(cfg, params[n], grads[n], opt_state["m"][n], is_decayed(n))
+            new_v[n] = opt_state["v"][n]
+        else:
+            new_params[n], new_m[n], new_v[n] = adamw(cfg, params[n], grads[n], opt_state["m"][n],
+                                                      opt_state["v"][n], step, is_decayed(n))
     fw.pop("caches")
     return {"loss": loss, "logits": fw["logits"], "grads": grads, "params": new_params,
             "opt_state": {"m": new_m, "v": new_v}, "kept": fw["kept"], "margins": fw["margins"],

@@ -41,7 +41,7 @@ class bsr_config(C.Structure):
                 ("drop_block", C.c_int32 * MAX_DROPS), ("keep_num", C.c_int32 * MAX_DROPS),
                 ("keep_den", C.c_int32 * MAX_DROPS), ("fuse_mode", C.c_int32),
                 ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
-                ("weight_decay", C.c_float), ("max_batch", C.c_int32)]
+                ("weight_decay", C.c_float), ("max_batch", C.c_int32), ("optimizer", C.c_int32), ("momentum", C.c_float)]
 
 
 class bsr_footprint(C.Structure):
@@ -132,6 +132,8 @@ def make_config(cfg, max_batch: Optional[int] = None) -> bsr_config:
     c.fuse_mode = cfg.fuse_mode
     c.lr, c.beta1, c.beta2, c.eps, c.weight_decay = cfg.lr, cfg.beta1, cfg.beta2, cfg.eps, cfg.weight_decay
     c.max_batch = cfg.batch if max_batch is None else max_batch
+    c.optimizer = 1 if getattr(cfg, "optimizer", "adamw") == "sgd" else 0
+    c.momentum = float(getattr(cfg, "momentum", 0.9))
     return c
 
 

@@ -108,6 +108,8 @@ int validate(const bsr_config* cfg, char* err) {
     if (d.num_classes[t] < 1) return set_err(err, BSR_ERR_INVALID_ARG, "num_classes must be positive");
   if (cfg->max_batch < 1) return set_err(err, BSR_ERR_INVALID_ARG, "max_batch must be positive");
   if (cfg->fuse_mode != BSR_FUSE_NONE && cfg->fuse_mode != BSR_FUSE_WEIGHTED_SUM) return set_err(err, BSR_ERR_INVALID_ARG, "unknown fuse_mode");
+  if (cfg->optimizer != BSR_OPT_ADAMW && cfg->optimizer != BSR_OPT_SGD) return set_err(err, BSR_ERR_INVALID_ARG, "unknown optimizer");
+  if (cfg->optimizer == BSR_OPT_SGD && !(cfg->momentum >= 0.f && cfg->momentum < 1.f)) return set_err(err, BSR_ERR_INVALID_ARG, "momentum must lie in [0, 1)");
   if (!(d.ln_eps > 0.f)) return set_err(err, BSR_ERR_INVALID_ARG, "ln_eps must be positive");
   Schedule s;
   int rc = compute_schedule(cfg, &s, err);
@@ -946,9 +948,13 @@ static int enqueue_train_step(bsr_handle* h, const void* images, const int32_t* 
     layernorm_bwd(c, h->at<float>(h->off_dxn), 1, h->at<float>(x_last), (long)Tl * D, h->at<float>(h->off_meanf), h->at<float>(h->off_rstdf),
                   (const float*)h->w("norm.weight"), nullptr, nullptr, 0, nullptr, lnp, h->gradp("norm.weight"), h->gradp("norm.bias"), B, D);
   }
-  adamw(c, h->at<AdamChunk>(h->off_chunks), h->n_chunks, h->at<float>(h->off_master), h->at<float>(h->off_grad), h->at<float>(h->off_m),
-        h->at<float>(h->off_v), h->base + h->off_weights, h->at<float>(h->off_status + 128), h->cfg.beta1, h->cfg.beta2, h->cfg.eps,
-        h->cfg.weight_decay);
+  if (h->cfg.optimizer == BSR_OPT_SGD)
+    sgd_momentum(c, h->at<AdamChunk>(h->off_chunks), h->n_chunks, h->at<float>(h->off_master), h->at<float>(h->off_grad),
+                 h->at<float>(h->off_m), h->base + h->off_weights, h->at<float>(h->off_status + 128), h->cfg.momentum, h->cfg.weight_decay);
+  else
+    adamw(c, h->at<AdamChunk>(h->off_chunks), h->n_chunks, h->at<float>(h->off_master), h->at<float>(h->off_grad), h->at<float>(h->off_m),
+          h->at<float>(h->off_v), h->base + h->off_weights, h->at<float>(h->off_status + 128), h->cfg.beta1, h->cfg.beta2, h->cfg.eps,
+          h->cfg.weight_decay);
   return BSR_OK;
 }
 

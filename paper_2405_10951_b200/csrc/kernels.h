@@ -158,6 +158,9 @@ struct AdamChunk { uint32_t offset; uint32_t count; int64_t shadow; uint32_t dec
 // scalars (device): learning rate, 1 - beta1^t, 1 - beta2^t of the step being taken.
 void adamw(const Ctx& c, const AdamChunk* chunks, int nchunks, float* master, const float* grad, float* m, float* v,
            void* shadow_base, const float* scalars, float b1, float b2, float eps, float wd);
+// SGD with momentum (buf starts at zero): buf <- mu buf + (g + wd p on decayed tensors), p <- p - lr buf; lr from scalars[0].
+void sgd_momentum(const Ctx& c, const AdamChunk* chunks, int nchunks, float* master, const float* grad, float* buf,
+                  void* shadow_base, const float* scalars, float mu, float wd);
 void set_scalars(cudaStream_t s, float* dst, float a, float b, float c3);
 
 // dst row r = src row r (row_bytes a multiple of 16), independent pitches: gathers / scatters token rows.

@@ -569,6 +569,35 @@ __global__ void adamw_kernel(const AdamChunk* __restrict__ chunks, float* __rest
   }
 }
 
+// SGD with momentum on the same chunk table: buf <- mu buf + (g + wd p), p <- p - lr buf.
+template <typename T>
+__global__ void sgd_kernel(const AdamChunk* __restrict__ chunks, float* __restrict__ master, const float* __restrict__ grad,
+                           float* __restrict__ buf, T* __restrict__ shadow_base, const float* __restrict__ scalars, float mu,
+                           float wd) {
+  float lr = scalars[0];
+  AdamChunk ch = chunks[blockIdx.x];
+  float decay = ch.decay ? wd : 0.f;
+  for (uint32_t i = threadIdx.x; i < ch.count; i += blockDim.x) {
+    size_t idx = (size_t)ch.offset + i;
+    float p = master[idx];
+    float b = mu * buf[idx] + (grad[idx] + decay * p);
+    buf[idx] = b;
+    float np = p - lr * b;
+    master[idx] = np;
+    if (ch.shadow >= 0) shadow_base[ch.shadow + i] = from_f<T>(np);
+  }
+}
+
+void sgd_momentum(const Ctx& c, const AdamChunk* chunks, int nchunks, float* master, const float* grad, float* buf,
+                  void* shadow_base, const float* scalars, float mu, float wd) {
+  if (nchunks <= 0) return;
+  note_launch(1);
+  if (c.dtype == 0)
+    sgd_kernel<float><<<nchunks, 256, 0, c.stream>>>(chunks, master, grad, buf, (float*)shadow_base, scalars, mu, wd);
+  else
+    sgd_kernel<bf16><<<nchunks, 256, 0, c.stream>>>(chunks, master, grad, buf, (bf16*)shadow_base, scalars, mu, wd);
+}
+
 __global__ void set_scalars_kernel(float* dst, float a, float b, float c3) {
   dst[0] = a; dst[1] = b; dst[2] = c3;
 }

@@ -56,6 +56,8 @@ class Config:
     beta2: float = 0.999
     eps: float = 1e-8
     weight_decay: float = 0.05
+    optimizer: str = "adamw"              # "adamw" or "sgd" (with momentum)
+    momentum: float = 0.9
     seed: int = 0
 
     @property

@@ -93,6 +93,33 @@ def test_two_steps_follow_the_oracle_and_are_deterministic():
     assert o2["loss"] < o1["loss"]
 
 
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_sgd_momentum_follows_the_oracle(dtype):
+    """SGD with momentum (the paper's ViT-B recipe, Section 5): two steps; the update is linear in the gradient, so the
+    parameter change and the momentum buffer are compared with the oracle's directly, per tensor."""
+    base = TINY if dtype == "fp32" else MINI_BF16
+    cfg = base.with_(optimizer="sgd", momentum=0.9, lr=1e-2, weight_decay=0.01)
+    tol = P.FP32_TOL if dtype == "fp32" else P.BF16_TOL * 1.5
+    images, labels, task_ids, params = synth.make_workload(cfg, peaked=True)
+    gpu = P.run_gpu_step(cfg, images, labels, task_ids, params, steps=2)
+    names = O.trainable_names(cfg, params)
+    # the oracle takes the GPU's kept sets of the last step for both steps only if they agree; step 1 decides
+    first = P.run_gpu_step(cfg, images, labels, task_ids, params, steps=1)
+    o1 = O.train_step(cfg, params, images, labels, task_ids, forced_keep=first["kept"])
+    o2 = O.train_step(cfg, o1["params"], images, labels, task_ids, forced_keep=gpu["kept"], opt_state=o1["opt_state"], step=2)
+    for n in names:
+        want = o2["params"][n] - params[n]
+        got = gpu["params"][n] - params[n]
+        # the parameter itself is stored in float: half an ulp of it per step bounds what the difference can resolve
+        bound = 2 * tol * np.linalg.norm(want) + 2.4e-7 * np.linalg.norm(params[n])
+        assert np.linalg.norm(got - want) < bound, (n, np.linalg.norm(got - want), bound)
+        assert P.rel_err(gpu["m"][n], o2["opt_state"]["m"][n]) < 2 * tol, n
+        assert not gpu["v"][n].any(), n
+    for n in gpu["params"]:                       # frozen tensors are untouched (the synthetic values are exact in the storage type)
+        if n not in names:
+            assert np.array_equal(gpu["params"][n], params[n].astype(np.float32).astype(np.float64)), n
+
+
 def test_error_paths_leave_the_context_usable():
     import torch
     from paper_2405_10951_b200 import binding as Bd

@@ -119,6 +119,44 @@ def test_adamw_first_step_closed_form():
     assert np.allclose(new, p - cfg.lr * g / (np.abs(g) + cfg.eps) - cfg.lr * cfg.weight_decay * p, rtol=1e-12)
 
 
+def test_sgd_matches_library_optimiser():
+    """Three steps of the oracle's SGD-with-momentum update (Section 5: the ViT-B recipe) equal torch.optim.SGD, decay on
+    matrices only."""
+    cfg = CASES["drop_with_fusion"].with_(optimizer="sgd", momentum=0.9, lr=5e-2, weight_decay=0.01)
+    images, labels, task_ids, params = workload(cfg)
+    names = O.trainable_names(cfg, params)
+    tp = {n: torch.tensor(params[n], dtype=torch.float64, requires_grad=True) for n in names}
+    opt = torch.optim.SGD([
+        {"params": [tp[n] for n in names if O.is_decayed(n)], "weight_decay": cfg.weight_decay},
+        {"params": [tp[n] for n in names if not O.is_decayed(n)], "weight_decay": 0.0}],
+        lr=cfg.lr, momentum=cfg.momentum)
+    state, cur = None, params
+    for step in (1, 2, 3):
+        out = O.train_step(cfg, cur, images, labels, task_ids, opt_state=state, step=step)
+        for n in names:
+            tp[n].grad = torch.tensor(out["grads"][n])
+        opt.step()
+        cur, state = out["params"], out["opt_state"]
+        for n in names:
+            assert close(cur[n], tp[n].detach().numpy(), 1e-12), (step, n)
+
+
+def test_sgd_closed_forms():
+    """First step: p - lr (g + wd p).  Constant gradient without decay: after n steps the parameter has moved by
+    lr g sum_{k=1..n} (1 - mu^k) / (1 - mu)."""
+    cfg = TINY.with_(optimizer="sgd", momentum=0.8, lr=1e-2, weight_decay=0.05)
+    g = np.array([0.3, -2.0, 1e-3])
+    p = np.array([1.0, -1.0, 0.5])
+    new, buf = O.sgd_momentum(cfg, p, g, np.zeros(3), True)
+    assert np.allclose(new, p - cfg.lr * (g + cfg.weight_decay * p), rtol=1e-13)
+    assert np.allclose(buf, g + cfg.weight_decay * p, rtol=1e-13)
+    q, buf = p.copy(), np.zeros(3)
+    for _ in range(5):
+        q, buf = O.sgd_momentum(cfg, q, g, buf, False)
+    mu = cfg.momentum
+    assert np.allclose(p - q, cfg.lr * g * sum((1 - mu ** k) / (1 - mu) for k in range(1, 6)), rtol=1e-12)
+
+
 def test_order_of_kept_rows_is_immaterial():
     """No positional term is added after the embedding, so permuting the compacted rows leaves the CLS output alone."""
     cfg = TINY.with_(drop_blocks=(1,), depth=3, trainable=(2,))
