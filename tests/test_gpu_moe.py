@@ -18,6 +18,13 @@ CASES = {
     "moe_drop_block_trainable": MINI_MOE.with_(drop_blocks=(3,), trainable=(3, 4)),
     "frozen_moe_in_gradient_path": MINI_MOE.with_(trainable=(2, 4)),
     "moe_vit_s_batch16": CONFIGS["moe_vit_s"].with_(batch=16),
+    # the paper's own arrangement (Section 5.2): MoE layers only in the trainable blocks, 16 experts, the top four per
+    # token, a router per task, drops at frozen and trainable locations
+    "paper_style_top4_of_16": Config("mini_moe_paper", 64, 8, 128, 2, 6, 256, (10, 6), 6, (1, 3, 5), (1, 2, 4), 1, 2,
+                                     dtype="bf16", seed=3, moe_experts=16, moe_top_k=4, moe_blocks=(1, 3, 5)),
+    "paper_style_vit_b_batch4": CONFIGS["vit_b"].with_(name="vit_b_moe", batch=4, num_classes=(100, 10), trainable=(3, 7, 11),
+                                                       moe_experts=16, moe_top_k=4, moe_blocks=(3, 7, 11), mlp_hidden=768,
+                                                       keep_num=1, keep_den=2),
 }
 
 
