@@ -43,6 +43,9 @@ BF16_CASES = {
     "vit_b_batch3": CONFIGS["vit_b"].with_(batch=3),
     "deit_s_paper_setup": CONFIGS["deit_s"].with_(batch=4, trainable=(3, 7, 11), keep_num=1, keep_den=2),
     "vit_b_384_batch2": CONFIGS["vit_b_384"].with_(batch=2),
+    # the drop-rate ablation's other two schedules (Table 8): five locations at keep 0.7, three late ones at keep 0.3
+    "deit_s_five_drop_locations": CONFIGS["deit_s"].with_(batch=3, drop_blocks=(1, 3, 5, 7, 9), keep_num=7, keep_den=10),
+    "deit_s_keep_0p3_late": CONFIGS["deit_s"].with_(batch=3, drop_blocks=(5, 7, 9), keep_num=3, keep_den=10),
 }
 
 
