@@ -46,10 +46,21 @@ def test_vit_b_full_batch_sampled_outputs_and_properties():
         assert k.shape == (B, ks[loc])
         assert np.all(np.diff(k, axis=1) > 0) and k.min() >= 0
     # 4. gradient of the batch mean = mean of the gradients of the two halves (same parameters, two fresh handles)
-    names = ["head.0.weight", "blocks.11.attn.qkv.weight", "blocks.8.mlp.fc1.weight", "blocks.9.norm1.weight", "blocks.8.attn.proj.bias"]
+    names = ["head.0.weight", "blocks.11.attn.qkv.weight", "blocks.8.mlp.fc1.weight", "blocks.9.norm1.weight", "blocks.8.attn.proj.bias",
+             "blocks.9.mlp.fc2.bias", "blocks.10.mlp.fc1.bias", "blocks.9.attn.qkv.bias", "blocks.11.mlp.fc2.weight"]
     shapes = synth.param_shapes(cfg)
     full = {n: eng.get_tensor("grad/" + n, shapes[n]).cpu().numpy().astype(np.float64) for n in names}
     eng.close()
+    # 5. a second handle on the same inputs reproduces the step bit for bit (no atomics, fixed reduction orders)
+    e1 = Bd.Engine(cfg)
+    e1.set_params(params)
+    loss1, kept1 = e1.train_step(e1.images_to_device(images), torch.as_tensor(labels).cuda())
+    e1.sync_status()
+    assert float(loss1.cpu()[0]) == float(loss.cpu()[0])
+    assert all(np.array_equal(a.cpu().numpy(), b) for a, b in zip(kept1, kept))
+    for n in names:
+        assert np.array_equal(e1.get_tensor("grad/" + n, shapes[n]).cpu().numpy().astype(np.float64), full[n]), n
+    e1.close()
     halves = []
     for sl in (slice(0, 64), slice(64, 128)):
         e2 = Bd.Engine(cfg, max_batch=64)
