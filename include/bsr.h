@@ -125,17 +125,23 @@ int32_t bsr_destroy(bsr_handle* h);
  * handle-less call when h is NULL).  Never NULL; valid until the next call on the same handle. */
 const char* bsr_last_error(const bsr_handle* h);
 
-/* Loads one parameter ("pre-trained weights", Section 5).  `src_dev` holds `count` float32 values
- * in device memory; they are converted to the storage dtype (and copied to the fp32 master for
- * trainable tensors) on `stream`.  `count` must equal the tensor's element count. */
-int32_t bsr_set_param(bsr_handle* h, const char* name, const float* src_dev, size_t count, void* stream);
+/* Loads one parameter ("pre-trained weights", Section 5).  `src` holds `count` values of type `src_dtype`
+ * (BSR_DTYPE_FP32: float32; BSR_DTYPE_BF16: bfloat16 bit patterns) in device memory (src_is_device != 0) or in host
+ * memory (src_is_device == 0); they are converted to the storage dtype (and widened into the fp32 master for trainable
+ * tensors) on `stream`.  `count` must equal the tensor's element count.  A host source is first copied into a staging
+ * area of the workspace: pageable memory may be released when the call returns, pinned memory only once `stream` has
+ * reached this point; all parameter loads of a handle must be issued on one stream (they share the staging area). */
+int32_t bsr_set_param(bsr_handle* h, const char* name, const void* src, size_t count, int32_t src_dtype, int32_t src_is_device,
+                      void* stream);
 
 /* Reads a tensor as float32 into device memory `dst_dev` (capacity `count` elements, which must
  * equal the tensor's size) on `stream`.  Names: a parameter name (the fp32 master if it trains,
  * else the stored weight widened), "grad/<param>", "adam_m/<param>", "adam_v/<param>" (trainable
  * parameters only), "logits" ([max_batch, max classes], rows of the last step; classes a task does
- * not have hold -inf), "loss" (1 element), "moe_experts/<l>" (the experts chosen by block l's router in the last
- * step, [tokens routed, top_k] as floats, best first; the last block routes only the classification rows). */
+ * not have hold -inf), "loss" (1 element), "scores/<l>" (Eq. 6: the head-mean classification-token attention of the
+ * last step at the drop location in block l, [max_batch, M], rows of images beyond the last batch undefined),
+ * "moe_experts/<l>" (the experts chosen by block l's router in the last step, [tokens routed, top_k] as floats,
+ * best first; the last block routes only the classification rows; `count` may be any prefix of the record). */
 int32_t bsr_get_tensor(bsr_handle* h, const char* name, float* dst_dev, size_t count, void* stream);
 
 /* Learning rate for the next steps (the cosine schedule of Section 5 lives in the caller). */
@@ -158,6 +164,36 @@ int32_t bsr_train_step(bsr_handle* h, const void* images_dev, const int32_t* lab
                        const int32_t* task_ids_dev, int32_t batch, void* stream,
                        float* loss_dev_out, int32_t* kept_idx_dev_out);
 
+/* A run of n_steps fine-tuning steps with the cosine learning-rate decay of Section 5 (training hyper-parameters)
+ * evaluated on the device: step t of the whole training (t counts optimiser steps from 0, continuing from the handle's
+ * step counter) uses lr(t) = lr_min + (lr_max - lr_min) (1 + cos(pi t / total_steps)) / 2, held at lr_min from
+ * t = total_steps on.  The step counter, the learning rate, the bias corrections and the position in the input arrays
+ * live in device memory and every step is one replay of the same captured graph (when `stream` can be captured, as
+ * for bsr_train_step), so the host supplies no scalars between steps.
+ *   images_dev   [n_steps, batch, in_chans, image_size, image_size] in the storage dtype: a fresh batch per step
+ *                (batch * in_chans * image_size^2 elements must be a multiple of 16 bytes)
+ *   labels_dev   [n_steps, batch] int32;  task_ids_dev [n_steps, batch] int32 or NULL when num_tasks == 1
+ *   loss_dev_out [n_steps] float32: the mean cross-entropy of every step before its update
+ *   kept_idx_dev_out  optional, laid out as for bsr_train_step: the kept positions of the LAST step
+ * Afterwards bsr_set_lr's value is the schedule's learning rate of the last step taken. */
+typedef struct {
+  float lr_max, lr_min;
+  int64_t total_steps;
+} bsr_lr_schedule;
+int32_t bsr_train_steps(bsr_handle* h, const void* images_dev, const int32_t* labels_dev, const int32_t* task_ids_dev,
+                        int32_t batch, int32_t n_steps, const bsr_lr_schedule* schedule_host, void* stream,
+                        float* loss_dev_out, int32_t* kept_idx_dev_out);
+
+/* bsr_train_step fed from and read back into HOST memory (the same step; Fig. 2).  images_host, labels_host and
+ * task_ids_host are copied into one of two staging slots inside the workspace on a copy stream the library owns, so
+ * that the copy for this step overlaps the kernels of the previous one; the step runs on `stream`; the loss (and, if
+ * kept_idx_host_out is not NULL, the kept positions) are copied back to host memory on `stream`.  Nothing is
+ * synchronised: loss_host_out is valid once `stream` has reached the end of this call's work.  Use pinned host memory
+ * for the overlap; with pinned memory the input buffers must stay untouched until then as well.  Layouts as for
+ * bsr_train_step. */
+int32_t bsr_train_step_host(bsr_handle* h, const void* images_host, const int32_t* labels_host, const int32_t* task_ids_host,
+                            int32_t batch, void* stream, float* loss_host_out, int32_t* kept_idx_host_out);
+
 /* Inference with the same token dropping (Section 2: unlike other on-device methods the dropping
  * also speeds up inference).  logits_dev_out: [batch, max classes] float32. */
 int32_t bsr_eval_forward(bsr_handle* h, const void* images_dev, const int32_t* task_ids_dev, int32_t batch,
@@ -170,6 +206,14 @@ int32_t bsr_get_footprint(const bsr_handle* h, bsr_footprint* out_host);
  * bounded wait in a kernel expired, BSR_ERR_NONFINITE if the last loss was not finite.  Clears it. */
 int32_t bsr_sync_status(bsr_handle* h, void* stream);
 
+/* Diagnostic of the failure path (no counterpart in the paper).  Every device-side wait of the tensor-core kernels
+ * is bounded; when one expires the CTA raises a status bit, frees its tensor memory and returns, and the next
+ * bsr_sync_status reports BSR_ERR_DEVICE_TIMEOUT with the context still usable.  This call runs exactly that path on
+ * purpose: it enqueues one CTA that waits, for at most limit_ns nanoseconds (1e3 .. 1e8), on a barrier nothing ever
+ * arrives at.  Nothing faults and nothing hangs; the following bsr_sync_status returns BSR_ERR_DEVICE_TIMEOUT and
+ * clears the status word.  bf16 handles only. */
+int32_t bsr_selftest_wait_expiry(bsr_handle* h, uint64_t limit_ns, void* stream);
+
 /* Which kernels run the dense contractions and attention of a bf16 handle (no counterpart in the paper):
  * 0 = the FP32-FMA kernels of the fp32 configuration (slow; a cross-check), 1 = tcgen05 kernels with one CTA per
  * tile (the default), 2 = as 1 but GEMMs with more than 128 rows run on CTA pairs (cta_group::2). */
@@ -177,8 +221,11 @@ int32_t bsr_set_gemm_mode(bsr_handle* h, int32_t mode);
 
 /* bsr_train_step replays a captured CUDA graph of its ~200 launches when `stream` can be captured (any stream but
  * the legacy default stream, and not one the caller is capturing) -- the first call with a given set of pointers
- * and batch captures it, later calls with the same arguments replay it.  on = 0 turns this off (every call
- * enqueues its kernels one by one); the results are identical.  No counterpart in the paper. */
+ * and batch captures it, later calls with the same arguments replay it.  The key of a captured graph is (images,
+ * labels, task ids, loss and kept-index pointers, batch, kernel mode); the handle keeps the eight most recently
+ * used graphs, so an input pipeline should rotate through at most eight sets of buffers (bsr_profile.graph_captures
+ * counts captures: it stops growing once a pipeline fits).  on = 0 turns this off (every call enqueues its kernels
+ * one by one); the results are identical.  No counterpart in the paper. */
 int32_t bsr_set_graph_mode(bsr_handle* h, int32_t on);
 
 /* Measurement support (no counterpart in the paper).  bsr_profile_enable resets the counters; with
@@ -192,6 +239,7 @@ typedef struct {
   uint64_t gemm_launches;
   double gemm_flops;
   double gemm_ms;
+  uint64_t graph_captures;          /* training-step graphs captured by this handle since it was created */
 } bsr_profile;
 int32_t bsr_profile_enable(bsr_handle* h, int32_t time_gemms);
 int32_t bsr_profile_read(bsr_handle* h, void* stream, bsr_profile* out_host);
@@ -249,7 +297,8 @@ int32_t bsr_linear_backward(const void* x_dev, const void* w_dev, const void* dy
  * memory owned by the caller; m, n, k multiples of 8.  n * k must not exceed BSR_STATIC_SCRATCH_BYTES / 8
  * elements, otherwise BSR_ERR_WORKSPACE_TOO_SMALL is returned and nothing runs.  The call allocates and
  * frees nothing.  The first call on each device looks up the array's device address (with that device
- * current) and should therefore come before any stream capture.  All calls on a device share the one
+ * current) and should therefore come before any stream capture; where the CUDA runtime loads device code lazily,
+ * that first call is also when the device image with the array is loaded and its bytes are taken.  All calls on a device share the one
  * array: each call fully rewrites the part it reads, so nothing needs clearing between calls, but two
  * calls whose kernels overlap on the GPU (different streams) race on it -- keep them on one stream or
  * order them with events.  Errors are described by bsr_static_last_error(). */

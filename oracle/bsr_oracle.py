@@ -22,7 +22,7 @@ What it follows, passage by passage:
 * MoE layer in place of the FFN: a task-dependent router picks the top experts per token
   and their outputs are added (Section 5.2).
 
-Readings where the paper is silent (each listed in the design doc):
+Readings where the paper is silent:
   score = post-softmax CLS row averaged over heads; CLS itself is not a candidate;
   K = ceil(keep * M) in integer arithmetic; kept tokens stay in ascending position and the
   fused token goes last; fused token = sum_j s_j x'_j over the dropped tokens; keep = 1
@@ -40,6 +40,8 @@ finite-difference pins cover.
 """
 
 from __future__ import annotations
+
+import math
 
 import numpy as np
 from scipy.special import erf
@@ -459,6 +461,30 @@ def sgd_momentum(cfg, p, g, buf, decay):
     d = g + (cfg.weight_decay * p if decay else 0.0)
     buf = cfg.momentum * buf + d
     return p - cfg.lr * buf, buf
+
+
+def cosine_lr(lr_max, lr_min, t, total_steps):
+    """Cosine learning-rate decay (Section 5, training hyper-parameters: "cosine learning rate decay"; the paper
+    gives neither end value nor warm-up, so both ends are arguments and there is no warm-up): step t (from 0) of
+    total_steps uses lr_min + (lr_max - lr_min) (1 + cos(pi t / total_steps)) / 2; from t = total_steps on the rate
+    stays at lr_min."""
+    tt = min(int(t), int(total_steps))
+    return lr_min + 0.5 * (lr_max - lr_min) * (1.0 + math.cos(math.pi * tt / total_steps))
+
+
+def train_steps(cfg, params, batches, lr_max, lr_min, total_steps, first_step=1, opt_state=None, forced_keeps=None):
+    """A run of steps, one batch (images, labels, task_ids) each, under the cosine schedule: the step numbered
+    `first_step + i` (optimiser steps count from 1) uses cosine_lr(.., t = first_step - 1 + i, ..).  Returns the list of
+    per-step results of train_step."""
+    out = []
+    for i, (images, labels, task_ids) in enumerate(batches):
+        step = first_step + i
+        c = cfg.with_(lr=cosine_lr(lr_max, lr_min, step - 1, total_steps))
+        r = train_step(c, params, images, labels, task_ids, forced_keep=forced_keeps[i] if forced_keeps else None,
+                       opt_state=opt_state, step=step)
+        params, opt_state = r["params"], r["opt_state"]
+        out.append(r)
+    return out
 
 
 def train_step(cfg, params, images, labels, task_ids=None, forced_keep=None, opt_state=None, step=1, forced_experts=None):

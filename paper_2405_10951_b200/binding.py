@@ -23,8 +23,8 @@ STATUS_NAMES = {0: "BSR_OK", -1: "BSR_ERR_INVALID_ARG", -2: "BSR_ERR_UNSUPPORTED
                 -4: "BSR_ERR_CUDA", -5: "BSR_ERR_DEVICE_TIMEOUT", -6: "BSR_ERR_NONFINITE"}
 
 EXPORTS = ["bsr_token_schedule", "bsr_workspace_bytes", "bsr_create", "bsr_destroy", "bsr_last_error", "bsr_set_param",
-           "bsr_get_tensor", "bsr_set_lr", "bsr_set_step", "bsr_train_step", "bsr_eval_forward", "bsr_get_footprint",
-           "bsr_sync_status", "bsr_set_gemm_mode", "bsr_set_graph_mode", "bsr_profile_enable", "bsr_profile_read", "bsr_profile_launches", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_backward",
+           "bsr_get_tensor", "bsr_set_lr", "bsr_set_step", "bsr_train_step", "bsr_train_steps", "bsr_train_step_host", "bsr_eval_forward", "bsr_get_footprint",
+           "bsr_sync_status", "bsr_selftest_wait_expiry", "bsr_set_gemm_mode", "bsr_set_graph_mode", "bsr_profile_enable", "bsr_profile_read", "bsr_profile_launches", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_backward",
            "bsr_linear_backward_static", "bsr_static_last_error", "bsr_attention_forward"]
 
 
@@ -51,7 +51,12 @@ class bsr_footprint(C.Structure):
 
 
 class bsr_profile(C.Structure):
-    _fields_ = [("kernel_launches", C.c_uint64), ("gemm_launches", C.c_uint64), ("gemm_flops", C.c_double), ("gemm_ms", C.c_double)]
+    _fields_ = [("kernel_launches", C.c_uint64), ("gemm_launches", C.c_uint64), ("gemm_flops", C.c_double), ("gemm_ms", C.c_double),
+                ("graph_captures", C.c_uint64)]
+
+
+class bsr_lr_schedule(C.Structure):
+    _fields_ = [("lr_max", C.c_float), ("lr_min", C.c_float), ("total_steps", C.c_int64)]
 
 
 class BsrError(RuntimeError):
@@ -79,14 +84,17 @@ def lib() -> C.CDLL:
         L.bsr_last_error.argtypes = [vp]
         L.bsr_last_error.restype = C.c_char_p
         L.bsr_static_last_error.restype = C.c_char_p
-        L.bsr_set_param.argtypes = [vp, C.c_char_p, f32p, C.c_size_t, vp]
+        L.bsr_set_param.argtypes = [vp, C.c_char_p, vp, C.c_size_t, i32, i32, vp]
         L.bsr_get_tensor.argtypes = [vp, C.c_char_p, f32p, C.c_size_t, vp]
         L.bsr_set_lr.argtypes = [vp, C.c_float]
         L.bsr_set_step.argtypes = [vp, C.c_int64]
         L.bsr_train_step.argtypes = [vp, vp, i32p, i32p, i32, vp, f32p, i32p]
+        L.bsr_train_steps.argtypes = [vp, vp, i32p, i32p, i32, i32, C.POINTER(bsr_lr_schedule), vp, f32p, i32p]
+        L.bsr_train_step_host.argtypes = [vp, vp, i32p, i32p, i32, vp, f32p, i32p]
         L.bsr_eval_forward.argtypes = [vp, vp, i32p, i32, vp, f32p, i32p]
         L.bsr_get_footprint.argtypes = [vp, C.POINTER(bsr_footprint)]
         L.bsr_sync_status.argtypes = [vp, vp]
+        L.bsr_selftest_wait_expiry.argtypes = [vp, C.c_uint64, vp]
         L.bsr_set_gemm_mode.argtypes = [vp, i32]
         L.bsr_set_graph_mode.argtypes = [vp, i32]
         L.bsr_profile_enable.argtypes = [vp, i32]
@@ -271,10 +279,17 @@ class Engine:
 
     # -- parameters --
     def set_param(self, name: str, value):
-        t = self.torch.as_tensor(np.ascontiguousarray(value, dtype=np.float32)).to(self.device) \
-            if not self.torch.is_tensor(value) else value.to(self.device, self.torch.float32).contiguous()
-        _check(lib().bsr_set_param(self.h, name.encode(), _ptr(t), t.numel(), _stream()), self.h)
-        self.torch.cuda.current_stream().synchronize()
+        """value: a numpy array (float32 or any float type: passed from host memory as float32), a CPU tensor
+        (float32 or bfloat16, passed from host memory as it is) or a CUDA tensor (float32 or bfloat16)."""
+        torch = self.torch
+        if not torch.is_tensor(value):
+            value = torch.as_tensor(np.ascontiguousarray(value, dtype=np.float32))
+        if value.dtype not in (torch.float32, torch.bfloat16):
+            value = value.to(torch.float32)
+        t = value.contiguous()
+        dt = DTYPE_FP32 if t.dtype == torch.float32 else DTYPE_BF16
+        _check(lib().bsr_set_param(self.h, name.encode(), _ptr(t), t.numel(), dt, int(t.is_cuda), _stream()), self.h)
+        torch.cuda.current_stream().synchronize()
 
     def set_params(self, params: Dict[str, np.ndarray]):
         for name, v in params.items():
@@ -315,6 +330,33 @@ class Engine:
         self.last_out = (loss, kept)
         return loss, self._split_kept(kept, B)
 
+    def train_steps(self, images, labels, task_ids=None, lr_max: float = 1e-3, lr_min: float = 0.0, total_steps: int = 1,
+                    want_kept: bool = True, out=None):
+        """images: CUDA tensor [n, B, C, S, S] in the storage dtype; labels/task_ids: int32 CUDA tensors [n, B].
+        Returns (losses tensor [n], kept-index tensors of the last step).  Does not synchronise."""
+        torch = self.torch
+        n, B = images.shape[0], images.shape[1]
+        if out is not None:
+            losses, kept = out
+        else:
+            losses = torch.empty(n, dtype=torch.float32, device=self.device)
+            kept = torch.empty(B * sum(self.kept_counts), dtype=torch.int32, device=self.device) if (want_kept and self.kept_counts) else None
+        sched = bsr_lr_schedule(lr_max, lr_min, total_steps)
+        _check(lib().bsr_train_steps(self.h, _ptr(images), _ptr(labels), _ptr(task_ids), B, n, C.byref(sched), _stream(),
+                                     _ptr(losses), _ptr(kept)), self.h)
+        self.last_out = (losses, kept)
+        return losses, self._split_kept(kept, B)
+
+    def train_step_host(self, images, labels, task_ids=None, loss=None, kept=None):
+        """images / labels / task_ids / loss / kept: CPU tensors (pinned for overlap); images in the storage dtype.
+        Does not synchronise: `loss` holds the step's loss once the current stream has finished this call's work."""
+        torch = self.torch
+        B = images.shape[0]
+        if loss is None:
+            loss = torch.empty(1, dtype=torch.float32).pin_memory()
+        _check(lib().bsr_train_step_host(self.h, _ptr(images), _ptr(labels), _ptr(task_ids), B, _stream(), _ptr(loss), _ptr(kept)), self.h)
+        return loss, (self._split_kept(kept, B) if kept is not None else None)
+
     def eval_forward(self, images, task_ids=None, want_kept: bool = True):
         torch = self.torch
         B = images.shape[0]
@@ -337,6 +379,9 @@ class Engine:
     def sync_status(self):
         _check(lib().bsr_sync_status(self.h, _stream()), self.h)
 
+    def selftest_wait_expiry(self, limit_ns: int = 1_000_000):
+        _check(lib().bsr_selftest_wait_expiry(self.h, limit_ns, _stream()), self.h)
+
     def set_gemm_mode(self, mode: int):
         _check(lib().bsr_set_gemm_mode(self.h, mode), self.h)
 
@@ -350,7 +395,7 @@ class Engine:
         p = bsr_profile()
         _check(lib().bsr_profile_read(self.h, _stream(), C.byref(p)), self.h)
         return {"kernel_launches": int(p.kernel_launches), "gemm_launches": int(p.gemm_launches),
-                "gemm_flops": float(p.gemm_flops), "gemm_ms": float(p.gemm_ms)}
+                "gemm_flops": float(p.gemm_flops), "gemm_ms": float(p.gemm_ms), "graph_captures": int(p.graph_captures)}
 
     def profile_launches(self, capacity: int = 4096):
         fl, ms, n = (C.c_double * capacity)(), (C.c_float * capacity)(), C.c_int32(0)

@@ -275,8 +275,8 @@ static int launch_fwd(const Ctx& c, const void* qkv, void* out, float* lse, floa
   size_t rs = d + (sizeof(T) == 2 ? 2 : 1);
   size_t smem = 2 * (size_t)T_ * rs * sizeof(T) + ((size_t)AT_WARPS * T_ + AT_WARPS * AT_MAXD) * sizeof(float);
   if (smem > 227 * 1024) return -2;
-  static size_t attr = 0;                 // the limit only grows: launches captured earlier in a graph keep working
-  if (smem > attr) { cudaFuncSetAttribute(attn_fwd_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr = smem; }
+  static SmemLimit lim;
+  if (!ensure_smem(lim, attn_fwd_kernel<T>, smem)) return -3;
   int qs = split_for(c, B * H, T_);
   dim3 grid(B * H, qs);
   note_launch(1);
@@ -298,9 +298,8 @@ static int launch_bwd(const Ctx& c, const void* qkv, const void* dout, const flo
   size_t smem1 = 2 * (size_t)T_ * rs * sizeof(T) + ((size_t)AT_WARPS * T_ + AT_WARPS * 2 * AT_MAXD) * sizeof(float);
   size_t smem2 = 2 * (size_t)T_ * rs * sizeof(T) + ((size_t)AT_WARPS * 2 * T_ + 2 * (size_t)T_ + AT_WARPS * 2 * AT_MAXD) * sizeof(float);
   if (smem1 > 227 * 1024 || smem2 > 227 * 1024) return -2;
-  static size_t attr1 = 0, attr2 = 0;     // the limits only grow
-  if (smem1 > attr1) { cudaFuncSetAttribute(attn_bwd_dq_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1); attr1 = smem1; }
-  if (smem2 > attr2) { cudaFuncSetAttribute(attn_bwd_dkv_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2); attr2 = smem2; }
+  static SmemLimit lim1, lim2;
+  if (!ensure_smem(lim1, attn_bwd_dq_kernel<T>, smem1) || !ensure_smem(lim2, attn_bwd_dkv_kernel<T>, smem2)) return -3;
   int qs = split_for(c, B * H, T_);
   dim3 grid(B * H, qs);
   note_launch(2);

@@ -752,11 +752,8 @@ int attention_fwd_tc(const Ctx& c, const void* qkv, void* out, float* lse, float
   if (!make_map(&map, qkv, (uint64_t)3 * H * d, (uint64_t)B * T, (uint64_t)3 * H * d, AT_BOX)) return -2;
   if (T > AT_MAXKEYS) {
     size_t smem_l = 1024 + 2 * (size_t)AT_BOX_BYTES + 2 * (size_t)AT_LONG_KB * 128 + (AT_LONG_KB / 64) * (size_t)(AT_QROWS * 128) + 64;
-    static bool attr_l = false;
-    if (!attr_l) {
-      if (cudaFuncSetAttribute(attn_fwd_tc_long_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_l) != cudaSuccess) return -3;
-      attr_l = true;
-    }
+    static SmemLimit lim_l;
+    if (!ensure_smem(lim_l, attn_fwd_tc_long_kernel, smem_l)) return -3;
     dim3 grid_l((T + AT_QROWS - 1) / AT_QROWS, B * H);
     note_launch(1);
     attn_fwd_tc_long_kernel<<<grid_l, 128, smem_l, c.stream>>>(map, (bf16*)out, lse, cls_prob, B, T, H, c.status);
@@ -775,12 +772,9 @@ int attention_fwd_tc(const Ctx& c, const void* qkv, void* out, float* lse, float
   size_t smem = fixed + kvslots * slot;
   int sms = c.sm_count > 0 ? c.sm_count : 148;
   int grid = B * H < sms ? B * H : sms;
-  static size_t attr[5] = {0, 0, 0, 0, 0};
+  static SmemLimit lim[5];
   auto launch = [&](auto kern, int threads) -> int {
-    if (smem > attr[nbuf]) {
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -3;
-      attr[nbuf] = smem;
-    }
+    if (!ensure_smem(lim[nbuf], kern, smem)) return -3;
     note_launch(1);
     kern<<<grid, threads, smem, c.stream>>>(map_q, map_kv, (bf16*)out, lse, cls_prob, B, T, H, kvslots, c.status);
     return 0;
@@ -804,11 +798,8 @@ int attention_bwd_tc(const Ctx& c, const void* qkv, const void* dout, const floa
   if (!make_map(&mg, dout, (uint64_t)H * d, (uint64_t)B * T, (uint64_t)H * d, AT_BOX)) return -2;
   size_t tile = 2 * (size_t)AT_BOX_BYTES, ch = (size_t)((T + 15) & ~15) * 128;
   size_t smem = 1024 + 3 * tile + (2 * ch > tile ? 2 * ch : tile) + 2 * ch + (3 * ch < 16384 ? 16384 - 3 * ch : 0) + 3 * AT_QROWS * 4 + 64;
-  static size_t attr = 0;
-  if (smem > attr) {
-    if (cudaFuncSetAttribute(attn_bwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -3;
-    attr = smem;
-  }
+  static SmemLimit lim;
+  if (!ensure_smem(lim, attn_bwd_tc_kernel, smem)) return -3;
   note_launch(1);
   attn_bwd_tc_kernel<<<B * H, 256, smem, c.stream>>>(mq, mg, lse, cls_extra, (bf16*)dqkv, B, T, H, c.status);
   return 0;

@@ -108,6 +108,22 @@ __device__ __forceinline__ float gelu_grad_f(float x) {
 extern long g_kernel_launches;
 static inline void note_launch(int n = 1) { g_kernel_launches += n; }
 
+// The dynamic shared-memory limit of a kernel is an attribute of the (kernel, device) pair, so the largest value set so
+// far is remembered per device ordinal.  It only grows: launches captured earlier in a graph keep working.
+struct SmemLimit {
+  size_t set[64] = {};
+};
+template <typename Kernel>
+static inline bool ensure_smem(SmemLimit& lim, Kernel kern, size_t bytes) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+  if (bytes > lim.set[dev]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return false;
+    lim.set[dev] = bytes;
+  }
+  return true;
+}
+
 static inline int ceil_div(long a, long b) { return (int)((a + b - 1) / b); }
 
 }  // namespace bsr

@@ -161,13 +161,26 @@ struct bsr_handle {
   size_t off_stage = 0;
   size_t off_split = 0, split_floats = 0;
   std::vector<size_t> moe_rec_eidx, moe_rec_ew;
+  std::vector<size_t> score_rec;       // per drop location's block: head-mean scores [max_batch, M] of the last step
   size_t off_m_dog = 0, off_m_dzg = 0, off_m_dxg = 0, off_m_dw = 0, off_m_dsel = 0;
   GemmProfile prof;
-  // captured graphs of the training step, keyed by the caller's pointers
-  struct StepGraph { const void* images; const void* labels; const void* tasks; void* loss; void* kept; int batch; int mode;
-                     cudaGraphExec_t exec; long launches; };
+  // Captured graphs of the training step.  The key is everything a captured launch has baked in: the caller's
+  // pointers, the batch, the kernel mode and whether the step reads its inputs through the multi-step loop state.
+  // Up to GRAPH_CACHE graphs are kept; the least recently used one is dropped.
+  struct StepGraph { const void* images; const void* labels; const void* tasks; void* loss; void* kept; int batch; int mode; int loop;
+                     cudaGraphExec_t exec; long launches; uint64_t last_use; };
+  static constexpr size_t GRAPH_CACHE = 8;
   std::vector<StepGraph> graphs;
+  uint64_t graph_clock = 0;
+  uint64_t graph_captures = 0;        // how many times a step was captured (a pipeline that cycles through more buffers than the cache holds re-captures every step)
   int use_graph = 1;
+  // multi-step loop and host-buffer step
+  size_t off_loop = 0, off_lab_stage = 0, off_task_stage = 0;
+  size_t off_host_img[2] = {0, 0}, off_host_lab[2] = {0, 0}, off_host_task[2] = {0, 0}, off_host_loss[2] = {0, 0};
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr};
+  bool slot_used[2] = {false, false};
+  int host_slot = 0;
   long launches_at_enable = 0;
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(base + off); }
@@ -299,6 +312,10 @@ size_t plan(bsr_handle* h) {
   };
   h->moe_rec_eidx = rec_eidx;
   h->moe_rec_ew = rec_ew;
+  // head-mean scores of every drop location (Eq. 6), kept for inspection whether the block is frozen or trains
+  h->score_rec.assign(d.depth, 0);
+  for (int l = 0; l < d.depth; ++l)
+    if (s.k[l] >= 0) h->score_rec[l] = b.take((size_t)Bm * (s.ta[l] - 1) * 4);
   // activations kept by the trainable blocks
   size_t a0 = b.off;
   h->bufs_train.assign(d.depth, BlockBufs());
@@ -318,7 +335,7 @@ size_t plan(bsr_handle* h) {
     bb.xp_full = drop ? b.take(Ma * D * 4) : bb.xp;
     if (s.k[l] >= 0) {
       bb.p = b.take((size_t)Bm * H * (s.ta[l] - 1) * 4);
-      bb.s = b.take((size_t)Bm * (s.ta[l] - 1) * 4);
+      bb.s = h->score_rec[l];
       bb.kept = b.take((size_t)Bm * (s.ta[l] - 1) * 4);
       bb.dropped = b.take((size_t)Bm * (s.ta[l] - 1) * 4);
     }
@@ -413,6 +430,16 @@ size_t plan(bsr_handle* h) {
   h->off_stage = b.take(biggest * 4);
   h->split_floats = (d.dtype == BSR_DTYPE_BF16) ? (size_t)160 * 128 * 256 : 0;   // one 128x256 fp32 tile per SM
   h->off_split = b.take(h->split_floats * 4);
+  // multi-step loop state and staging; two staging slots for steps fed from host memory
+  h->off_loop = b.take(256);
+  h->off_lab_stage = b.take((size_t)Bm * 4);
+  h->off_task_stage = b.take((size_t)Bm * 4);
+  for (int i = 0; i < 2; ++i) {
+    h->off_host_img[i] = b.take((size_t)Bm * d.in_chans * d.image_size * d.image_size * es);
+    h->off_host_lab[i] = b.take((size_t)Bm * 4);
+    h->off_host_task[i] = b.take((size_t)Bm * 4);
+    h->off_host_loss[i] = b.take(256);
+  }
   h->scratch_bytes = b.off - s0;
   return b.off;
 }
@@ -678,12 +705,13 @@ HeadDesc head_desc(bsr_handle* h) {
 }
 
 // Forward through all blocks.  train: blocks >= t0 write the activation arena.  Returns the offset of the last output.
-int forward_all(bsr_handle* h, const Ctx& c, const void* images, int B, bool train, size_t* x_last_off, const int* task_ids) {
+int forward_all(bsr_handle* h, const Ctx& c, const void* images, int B, bool train, size_t* x_last_off, const int* task_ids,
+                const long long* img_offset = nullptr) {
   const bsr_dims& d = h->cfg.dims;
   int D = d.dim;
   int g = d.image_size / d.patch_size, N = g * g;
   int pin = d.in_chans * d.patch_size * d.patch_size;
-  patchify(c, images, h->base + h->off_patches, B, d.in_chans, d.image_size, d.patch_size);
+  patchify(c, images, h->base + h->off_patches, B, d.in_chans, d.image_size, d.patch_size, img_offset);
   GemmEpilogue ep;
   ep.bias = (const float*)h->w("patch_embed.bias");
   gemm(c, h->base + h->off_patches, pin, 1, h->w("patch_embed.weight"), pin, 1, h->base + h->off_emb, 0, B * N, D, pin, ep);
@@ -704,6 +732,7 @@ int forward_all(bsr_handle* h, const Ctx& c, const void* images, int B, bool tra
     }
     bb.x_in = cur;
     if (is_moe(h, l)) { bb.m_eidx = h->moe_rec_eidx[l]; bb.m_ew = h->moe_rec_ew[l]; }
+    if (h->sched.k[l] >= 0) bb.s = h->score_rec[l];
     int* kept_dst = nullptr;
     if (h->sched.k[l] >= 0) { kept_dst = kept_all + kept_off; kept_off += (size_t)B * h->sched.k[l]; }
     int rc = block_forward(h, c, l, B, bb, save, kept_dst, task_ids);
@@ -821,6 +850,11 @@ int32_t bsr_destroy(bsr_handle* h) {
   if (h != nullptr) {
     for (cudaEvent_t ev : h->prof.events) cudaEventDestroy(ev);
     for (auto& g : h->graphs) cudaGraphExecDestroy(g.exec);
+    for (int i = 0; i < 2; ++i) {
+      if (h->ev_copied[i]) cudaEventDestroy(h->ev_copied[i]);
+      if (h->ev_done[i]) cudaEventDestroy(h->ev_done[i]);
+    }
+    if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
   }
   delete h;
   return BSR_OK;
@@ -828,20 +862,33 @@ int32_t bsr_destroy(bsr_handle* h) {
 
 const char* bsr_last_error(const bsr_handle* h) { return h ? h->err : g_error; }
 
-int32_t bsr_set_param(bsr_handle* h, const char* name, const float* src, size_t count, void* stream) {
+int32_t bsr_set_param(bsr_handle* h, const char* name, const void* src, size_t count, int32_t src_dtype, int32_t src_is_device,
+                      void* stream) {
   if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
   if (name == nullptr || src == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "null argument");
+  if (src_dtype != BSR_DTYPE_FP32 && src_dtype != BSR_DTYPE_BF16) return set_err(h->err, BSR_ERR_INVALID_ARG, "src_dtype must be fp32 (0) or bf16 (1)");
   auto it = h->index.find(name);
   if (it == h->index.end()) return set_err(h->err, BSR_ERR_INVALID_ARG, "unknown parameter '%s'", name);
   const Tensor& t = h->tensors[it->second];
   if (count != t.numel) return set_err(h->err, BSR_ERR_INVALID_ARG, "'%s' has %zu elements, %zu given", name, t.numel, count);
   Ctx c = make_ctx(h, stream);
-  if (t.trainable)
-    cudaMemcpyAsync(h->at<float>(h->off_master) + t.flat, src, count * 4, cudaMemcpyDeviceToDevice, c.stream);
+  Ctx cs = c;                       // conversions from the source's type
+  cs.dtype = src_dtype;
+  size_t es_src = dtype_size(src_dtype);
+  if (!src_is_device) {             // host source: through the staging area (sized for the largest tensor as float)
+    cudaMemcpyAsync(h->base + h->off_stage, src, count * es_src, cudaMemcpyHostToDevice, c.stream);
+    src = h->base + h->off_stage;
+  }
+  auto to_float = [&](float* dst) {
+    if (src_dtype == BSR_DTYPE_FP32) cudaMemcpyAsync(dst, src, count * 4, cudaMemcpyDeviceToDevice, c.stream);
+    else convert_to_float(cs, src, dst, count);
+  };
+  if (t.trainable) to_float(h->at<float>(h->off_master) + t.flat);
   bool alias_master = t.trainable && (!t.matrix || c.dtype == BSR_DTYPE_FP32);
   if (!alias_master) {
-    if (t.matrix) convert_from_float(c, src, h->base + t.w_off, count);
-    else cudaMemcpyAsync(h->base + t.w_off, src, count * 4, cudaMemcpyDeviceToDevice, c.stream);
+    if (!t.matrix || c.dtype == BSR_DTYPE_FP32) to_float(h->at<float>(t.w_off));
+    else if (src_dtype == BSR_DTYPE_BF16) cudaMemcpyAsync(h->base + t.w_off, src, count * 2, cudaMemcpyDeviceToDevice, c.stream);
+    else convert_from_float(c, (const float*)src, h->base + t.w_off, count);
   }
   return check_cuda(h, "bsr_set_param");
 }
@@ -861,8 +908,14 @@ int32_t bsr_get_tensor(bsr_handle* h, const char* name, float* dst, size_t count
   } else if (n.rfind("moe_experts/", 0) == 0) {
     int l = atoi(n.c_str() + 12);
     if (l < 0 || l >= h->cfg.dims.depth || !is_moe(h, l)) return set_err(h->err, BSR_ERR_INVALID_ARG, "'%s': not an MoE block", name);
+    size_t recorded = (size_t)h->cfg.max_batch * h->sched.tf[l] * h->cfg.dims.moe_top_k;
+    if (count < 1 || count > recorded) return set_err(h->err, BSR_ERR_INVALID_ARG, "'%s' records at most %zu values, %zu asked for", name, recorded, count);
     convert_int_to_float(c.stream, h->at<int>(h->moe_rec_eidx[l]), dst, count);
     return check_cuda(h, "bsr_get_tensor");
+  } else if (n.rfind("scores/", 0) == 0) {
+    int l = atoi(n.c_str() + 7);
+    if (l < 0 || l >= h->cfg.dims.depth || h->sched.k[l] < 0) return set_err(h->err, BSR_ERR_INVALID_ARG, "'%s': not a token drop location", name);
+    src = h->at<float>(h->score_rec[l]); numel = (size_t)h->cfg.max_batch * (h->sched.ta[l] - 1);
   } else {
     size_t base_off = 0;
     std::string pn = n;
@@ -906,15 +959,16 @@ int32_t bsr_set_step(bsr_handle* h, int64_t steps_done) {
 }
 
 // Enqueues every kernel of one step on `stream` (forward, loss, backward, AdamW reading its scalars from device memory).
+// loss_out may be null (the multi-step loop writes the loss itself); img_offset as in forward_all.
 static int enqueue_train_step(bsr_handle* h, const void* images, const int32_t* labels, const int32_t* task_ids, int32_t batch,
-                              void* stream, float* loss_out, int32_t* kept_out) {
+                              void* stream, float* loss_out, int32_t* kept_out, const long long* img_offset = nullptr) {
   int rc;
   const bsr_dims& d = h->cfg.dims;
   Ctx c = make_ctx(h, stream);
   int D = d.dim, B = batch;
   size_t es = dtype_size(d.dtype);
   size_t x_last = 0;
-  rc = forward_all(h, c, images, B, true, &x_last, task_ids);
+  rc = forward_all(h, c, images, B, true, &x_last, task_ids, img_offset);
   if (rc != BSR_OK) return rc;
   int Tl = cls_tail(h, d.depth - 1) ? 1 : h->sched.tf[d.depth - 1];   // rows per image in the last block's output
   HeadDesc hd = head_desc(h);
@@ -924,7 +978,7 @@ static int enqueue_train_step(bsr_handle* h, const void* images, const int32_t* 
   head_fwd(c, hd, xn, task_ids, h->at<float>(h->off_logits), B);
   cross_entropy(c, hd, h->at<float>(h->off_logits), labels, task_ids, h->at<float>(h->off_per_image), h->at<float>(h->off_dlogits),
                 h->at<float>(h->off_loss), B);
-  cudaMemcpyAsync(loss_out, h->at<float>(h->off_loss), 4, cudaMemcpyDeviceToDevice, c.stream);
+  if (loss_out != nullptr) cudaMemcpyAsync(loss_out, h->at<float>(h->off_loss), 4, cudaMemcpyDeviceToDevice, c.stream);
   if (kept_out != nullptr && kept_total(h, B) > 0)
     cudaMemcpyAsync(kept_out, h->base + h->off_kept_all, kept_total(h, B) * 4, cudaMemcpyDeviceToDevice, c.stream);
   // backward: head, final LayerNorm, trainable blocks in reverse, nothing before the earliest one
@@ -958,6 +1012,63 @@ static int enqueue_train_step(bsr_handle* h, const void* images, const int32_t* 
   return BSR_OK;
 }
 
+}  // extern "C"
+
+// Runs `enqueue` (which puts one step's kernels on `st`) either directly or, when the stream allows capture (any
+// stream but the legacy default one, not one the caller is capturing, no per-launch events asked for), as a CUDA graph
+// captured on first use and replayed afterwards.
+template <typename Enqueue>
+static int run_step_graphed(bsr_handle* h, cudaStream_t st, const bsr_handle::StepGraph& key, Enqueue enqueue) {
+  int rc;
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  bool can_graph = h->use_graph && st != nullptr && st != cudaStreamLegacy && !h->prof.on &&
+                   cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
+  auto direct = [&]() -> int {
+    cudaGetLastError();
+    int r = enqueue();
+    return r != BSR_OK ? r : check_cuda(h, "training step");
+  };
+  if (!can_graph) return direct();
+  for (auto& g : h->graphs) {
+    if (g.images == key.images && g.labels == key.labels && g.tasks == key.tasks && g.loss == key.loss && g.kept == key.kept &&
+        g.batch == key.batch && g.mode == key.mode && g.loop == key.loop) {
+      g_kernel_launches += g.launches;
+      g.last_use = ++h->graph_clock;
+      if (cudaGraphLaunch(g.exec, st) != cudaSuccess) return set_err(h->err, BSR_ERR_CUDA, "graph launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+      return BSR_OK;
+    }
+  }
+  long before = g_kernel_launches;
+  if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return direct();
+  rc = enqueue();
+  cudaGraph_t graph = nullptr;
+  cudaError_t ce = cudaStreamEndCapture(st, &graph);
+  if (rc != BSR_OK) {
+    if (graph) cudaGraphDestroy(graph);
+    return rc;
+  }
+  bsr_handle::StepGraph sg = key;
+  sg.exec = nullptr; sg.launches = g_kernel_launches - before; sg.last_use = ++h->graph_clock;
+  if (ce != cudaSuccess || graph == nullptr || cudaGraphInstantiate(&sg.exec, graph, 0) != cudaSuccess) {
+    if (graph) cudaGraphDestroy(graph);
+    return direct();                                     // nothing ran during the capture
+  }
+  cudaGraphDestroy(graph);
+  ++h->graph_captures;
+  if (h->graphs.size() >= bsr_handle::GRAPH_CACHE) {     // drop the least recently used graph
+    size_t lru = 0;
+    for (size_t i = 1; i < h->graphs.size(); ++i)
+      if (h->graphs[i].last_use < h->graphs[lru].last_use) lru = i;
+    cudaGraphExecDestroy(h->graphs[lru].exec);
+    h->graphs.erase(h->graphs.begin() + lru);
+  }
+  h->graphs.push_back(sg);
+  if (cudaGraphLaunch(sg.exec, st) != cudaSuccess) return set_err(h->err, BSR_ERR_CUDA, "graph launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+  return BSR_OK;
+}
+
+extern "C" {
+
 int32_t bsr_train_step(bsr_handle* h, const void* images, const int32_t* labels, const int32_t* task_ids, int32_t batch,
                        void* stream, float* loss_out, int32_t* kept_out) {
   int rc = check_batch(h, images, batch);
@@ -965,59 +1076,93 @@ int32_t bsr_train_step(bsr_handle* h, const void* images, const int32_t* labels,
   if (labels == nullptr || loss_out == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "labels_dev and loss_dev_out must not be null");
   if (h->cfg.dims.num_tasks > 1 && task_ids == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "task_ids_dev is required with several tasks");
   cudaStream_t st = (cudaStream_t)stream;
-  h->step += 1;
-  double bc1 = 1.0 - std::pow((double)h->cfg.beta1, (double)h->step);
-  double bc2 = 1.0 - std::pow((double)h->cfg.beta2, (double)h->step);
+  // the step counter (AdamW's bias correction) advances only once the step has been enqueued
+  const int64_t step_next = h->step + 1;
+  double bc1 = 1.0 - std::pow((double)h->cfg.beta1, (double)step_next);
+  double bc2 = 1.0 - std::pow((double)h->cfg.beta2, (double)step_next);
   set_scalars(st, h->at<float>(h->off_status + 128), h->lr, (float)bc1, (float)bc2);
-  // A step is a fixed sequence of ~200 launches: replay it as a CUDA graph when the stream allows capture (not the
-  // legacy default stream, not a stream the caller is capturing) and nothing asks for per-launch events.
-  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-  bool can_graph = h->use_graph && st != nullptr && st != cudaStreamLegacy && !h->prof.on &&
-                   cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
-  if (!can_graph) {
-    cudaGetLastError();
-    rc = enqueue_train_step(h, images, labels, task_ids, batch, stream, loss_out, kept_out);
+  bsr_handle::StepGraph key;
+  key.images = images; key.labels = labels; key.tasks = task_ids; key.loss = loss_out; key.kept = kept_out; key.batch = batch;
+  key.mode = h->use_tc; key.loop = 0; key.exec = nullptr; key.launches = 0; key.last_use = 0;
+  rc = run_step_graphed(h, st, key, [&]() { return enqueue_train_step(h, images, labels, task_ids, batch, stream, loss_out, kept_out); });
+  if (rc == BSR_OK) h->step = step_next;
+  return rc;
+}
+
+int32_t bsr_train_steps(bsr_handle* h, const void* images, const int32_t* labels, const int32_t* task_ids, int32_t batch,
+                        int32_t n_steps, const bsr_lr_schedule* sched, void* stream, float* loss_out, int32_t* kept_out) {
+  int rc = check_batch(h, images, batch);
+  if (rc != BSR_OK) return rc;
+  if (labels == nullptr || loss_out == nullptr || sched == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "labels_dev, loss_dev_out and schedule must not be null");
+  if (h->cfg.dims.num_tasks > 1 && task_ids == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "task_ids_dev is required with several tasks");
+  if (n_steps < 1) return set_err(h->err, BSR_ERR_INVALID_ARG, "n_steps must be positive");
+  if (sched->total_steps < 1 || !(sched->lr_max >= sched->lr_min) || !(sched->lr_min >= 0.f))
+    return set_err(h->err, BSR_ERR_INVALID_ARG, "schedule needs total_steps >= 1 and lr_max >= lr_min >= 0");
+  const bsr_dims& d = h->cfg.dims;
+  cudaStream_t st = (cudaStream_t)stream;
+  LoopState* ls = h->at<LoopState>(h->off_loop);
+  long long stride = (long long)batch * d.in_chans * d.image_size * d.image_size;
+  loop_init(st, ls, h->step, sched->total_steps, stride, sched->lr_max, sched->lr_min, h->cfg.beta1, h->cfg.beta2, n_steps);
+  int* lab_stage = h->at<int>(h->off_lab_stage);
+  int* task_stage = task_ids != nullptr ? h->at<int>(h->off_task_stage) : nullptr;
+  float* scalars = h->at<float>(h->off_status + 128);
+  bsr_handle::StepGraph key;
+  key.images = images; key.labels = labels; key.tasks = task_ids; key.loss = loss_out; key.kept = kept_out; key.batch = batch;
+  key.mode = h->use_tc; key.loop = 1; key.exec = nullptr; key.launches = 0; key.last_use = 0;
+  for (int i = 0; i < n_steps; ++i) {
+    rc = run_step_graphed(h, st, key, [&]() {
+      loop_begin(st, ls, scalars, labels, task_ids, lab_stage, task_stage, batch);
+      int r = enqueue_train_step(h, images, lab_stage, task_stage, batch, stream, nullptr, kept_out, &ls->image_offset);
+      loop_end(st, ls, h->at<float>(h->off_loss), loss_out);
+      return r;
+    });
     if (rc != BSR_OK) return rc;
-    return check_cuda(h, "bsr_train_step");
+    h->step += 1;
   }
-  for (auto& g : h->graphs) {
-    if (g.images == images && g.labels == labels && g.tasks == task_ids && g.loss == loss_out && g.kept == kept_out &&
-        g.batch == batch && g.mode == h->use_tc) {
-      g_kernel_launches += g.launches;
-      if (cudaGraphLaunch(g.exec, st) != cudaSuccess) return set_err(h->err, BSR_ERR_CUDA, "graph launch failed: %s", cudaGetErrorString(cudaGetLastError()));
-      return BSR_OK;
-    }
-  }
-  long before = g_kernel_launches;
-  if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
-    cudaGetLastError();
-    rc = enqueue_train_step(h, images, labels, task_ids, batch, stream, loss_out, kept_out);
-    return rc != BSR_OK ? rc : check_cuda(h, "bsr_train_step");
-  }
-  rc = enqueue_train_step(h, images, labels, task_ids, batch, stream, loss_out, kept_out);
-  cudaGraph_t graph = nullptr;
-  cudaError_t ce = cudaStreamEndCapture(st, &graph);
-  if (rc != BSR_OK) {
-    if (graph) cudaGraphDestroy(graph);
-    return rc;
-  }
-  bsr_handle::StepGraph sg;
-  sg.images = images; sg.labels = labels; sg.tasks = task_ids; sg.loss = loss_out; sg.kept = kept_out; sg.batch = batch;
-  sg.mode = h->use_tc; sg.exec = nullptr; sg.launches = g_kernel_launches - before;
-  if (ce != cudaSuccess || graph == nullptr || cudaGraphInstantiate(&sg.exec, graph, 0) != cudaSuccess) {
-    if (graph) cudaGraphDestroy(graph);
-    cudaGetLastError();
-    rc = enqueue_train_step(h, images, labels, task_ids, batch, stream, loss_out, kept_out);   // nothing ran during capture
-    return rc != BSR_OK ? rc : check_cuda(h, "bsr_train_step");
-  }
-  cudaGraphDestroy(graph);
-  if (h->graphs.size() >= 4) {
-    cudaGraphExecDestroy(h->graphs.front().exec);
-    h->graphs.erase(h->graphs.begin());
-  }
-  h->graphs.push_back(sg);
-  if (cudaGraphLaunch(sg.exec, st) != cudaSuccess) return set_err(h->err, BSR_ERR_CUDA, "graph launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+  // the schedule's last learning rate stays in force for later single steps
+  double frac = (double)(h->step - 1 < sched->total_steps ? h->step - 1 : sched->total_steps) / (double)sched->total_steps;
+  h->lr = (float)((double)sched->lr_min + 0.5 * ((double)sched->lr_max - (double)sched->lr_min) * (1.0 + std::cos(3.14159265358979323846 * frac)));
   return BSR_OK;
+}
+
+int32_t bsr_train_step_host(bsr_handle* h, const void* images_host, const int32_t* labels_host, const int32_t* task_ids_host,
+                            int32_t batch, void* stream, float* loss_host_out, int32_t* kept_host_out) {
+  int rc = check_batch(h, images_host, batch);
+  if (rc != BSR_OK) return rc;
+  if (labels_host == nullptr || loss_host_out == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "labels_host and loss_host_out must not be null");
+  if (h->cfg.dims.num_tasks > 1 && task_ids_host == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "task_ids_host is required with several tasks");
+  const bsr_dims& d = h->cfg.dims;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (h->copy_stream == nullptr) {                       // host objects, created on first use
+    bool ok = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; ++i)
+      ok = cudaEventCreateWithFlags(&h->ev_copied[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return set_err(h->err, BSR_ERR_CUDA, "could not create the copy stream: %s", cudaGetErrorString(cudaGetLastError()));
+  }
+  int slot = h->host_slot;
+  h->host_slot ^= 1;
+  // The inputs travel on the library's copy stream into one of two staging slots, so that the copy for this step
+  // overlaps the previous step's kernels; the slot's previous user (two calls back) must have finished with it.
+  if (h->slot_used[slot]) cudaStreamWaitEvent(h->copy_stream, h->ev_done[slot], 0);
+  size_t img_bytes = (size_t)batch * d.in_chans * d.image_size * d.image_size * dtype_size(d.dtype);
+  void* img_dev = h->base + h->off_host_img[slot];
+  int32_t* lab_dev = h->at<int32_t>(h->off_host_lab[slot]);
+  int32_t* task_dev = task_ids_host != nullptr ? h->at<int32_t>(h->off_host_task[slot]) : nullptr;
+  float* loss_dev = h->at<float>(h->off_host_loss[slot]);
+  cudaMemcpyAsync(img_dev, images_host, img_bytes, cudaMemcpyHostToDevice, h->copy_stream);
+  cudaMemcpyAsync(lab_dev, labels_host, (size_t)batch * 4, cudaMemcpyHostToDevice, h->copy_stream);
+  if (task_dev != nullptr) cudaMemcpyAsync(task_dev, task_ids_host, (size_t)batch * 4, cudaMemcpyHostToDevice, h->copy_stream);
+  cudaEventRecord(h->ev_copied[slot], h->copy_stream);
+  cudaStreamWaitEvent(st, h->ev_copied[slot], 0);
+  rc = bsr_train_step(h, img_dev, lab_dev, task_dev, batch, stream, loss_dev, nullptr);
+  if (rc != BSR_OK) return rc;
+  cudaMemcpyAsync(loss_host_out, loss_dev, 4, cudaMemcpyDeviceToHost, st);
+  if (kept_host_out != nullptr && kept_total(h, batch) > 0)
+    cudaMemcpyAsync(kept_host_out, h->base + h->off_kept_all, kept_total(h, batch) * 4, cudaMemcpyDeviceToHost, st);
+  cudaEventRecord(h->ev_done[slot], st);
+  h->slot_used[slot] = true;
+  return check_cuda(h, "bsr_train_step_host");
 }
 
 int32_t bsr_eval_forward(bsr_handle* h, const void* images, const int32_t* task_ids, int32_t batch, void* stream,
@@ -1081,6 +1226,15 @@ int32_t bsr_sync_status(bsr_handle* h, void* stream) {
   return BSR_OK;
 }
 
+int32_t bsr_selftest_wait_expiry(bsr_handle* h, uint64_t limit_ns, void* stream) {
+  if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
+  if (limit_ns < 1000 || limit_ns > 100000000ull) return set_err(h->err, BSR_ERR_INVALID_ARG, "limit_ns must lie in [1e3, 1e8]");
+  if (h->cfg.dims.dtype != BSR_DTYPE_BF16) return set_err(h->err, BSR_ERR_UNSUPPORTED, "only bf16 handles run kernels with bounded waits");
+  Ctx c = make_ctx(h, stream);
+  wait_expiry_selftest(c, limit_ns);
+  return check_cuda(h, "bsr_selftest_wait_expiry");
+}
+
 int32_t bsr_set_gemm_mode(bsr_handle* h, int32_t mode) {
   if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
   if (mode < 0 || mode > 2) return set_err(h->err, BSR_ERR_INVALID_ARG, "mode must be 0, 1 or 2");
@@ -1117,6 +1271,7 @@ int32_t bsr_profile_read(bsr_handle* h, void* stream, bsr_profile* out) {
   out->gemm_launches = h->prof.used / 2;
   out->gemm_flops = h->prof.flops;
   out->gemm_ms = ms;
+  out->graph_captures = h->graph_captures;
   return BSR_OK;
 }
 

@@ -269,6 +269,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (threadIdx.x == 0 && abort_flag && status != nullptr) atomicOr(status, STATUS_TIMEOUT);
 }
 
+// Diagnostic: the give-up path of the bounded waits, run on purpose.  One CTA allocates tensor memory as the GEMM does,
+// waits on an mbarrier that nothing ever arrives at, gives up after limit_ns, frees its tensor memory, raises
+// STATUS_TIMEOUT and returns -- the same teardown the kernels above perform when a wait of theirs expires.
+__global__ void wait_expiry_kernel(int* status, unsigned long long limit_ns) {
+  __shared__ __align__(8) unsigned long long bar_storage;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  uint32_t bar = smem_u32(&bar_storage);
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  tmem_alloc(smem_u32(&tmem_slot), 32);
+  tmem_relinquish();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (threadIdx.x == 0) mbar_wait_ns(bar, 0, &abort_flag, limit_ns);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  tmem_dealloc(tmem_slot, 32);
+  if (threadIdx.x == 0 && abort_flag && status != nullptr) atomicOr(status, STATUS_TIMEOUT);
+}
+
 // out[i] = sum over splits of partial[s][i], ascending s.
 __global__ void splitk_reduce_kernel(const float* __restrict__ partial, float* __restrict__ out, size_t n, int splits) {
   size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
@@ -318,16 +344,16 @@ __global__ void splitk_reduce_epi_kernel(const float* __restrict__ partial, TOut
   store4(out + i, v);
 }
 
+static EncodeFn lookup_encode_fn() {
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+    return (EncodeFn)p;
+  return nullptr;
+}
+
 EncodeFn encode_fn() {
-  static EncodeFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
-      fn = (EncodeFn)p;
-  }
+  static EncodeFn fn = lookup_encode_fn();      // initialised once, thread-safe
   return fn;
 }
 
@@ -347,11 +373,8 @@ template <bool A_MN, bool B_MN, typename TOut, int BN = BN_MAX>
 static int launch(const Ctx& c, const CUtensorMap& ma, const CUtensorMap& mb, void* C, int m, int n, int k, const Epi& ep,
                   int tiles_m, int tiles_n, int splits, int kb_per_split, const GemmGroup& grp) {
   auto kern = gemm_tc_kernel<A_MN, B_MN, TOut, BN>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return -3;
-    attr_set = true;
-  }
+  static SmemLimit lim;
+  if (!ensure_smem(lim, kern, SMEM_BYTES)) return -3;
   int work = tiles_m * tiles_n * splits;
   int sms = c.sm_count > 0 ? c.sm_count : 148;
   int grid = work < sms ? work : sms;
@@ -361,6 +384,11 @@ static int launch(const Ctx& c, const CUtensorMap& ma, const CUtensorMap& mb, vo
 }
 
 }  // namespace tc
+
+void wait_expiry_selftest(const Ctx& c, unsigned long long limit_ns) {
+  note_launch(1);
+  tc::wait_expiry_kernel<<<1, 32, 0, c.stream>>>(c.status, limit_ns);
+}
 
 void splitk_reduce(cudaStream_t s, const float* partial, float* out, size_t n, int splits) {
   note_launch(1);

@@ -229,11 +229,8 @@ template <bool A_MN, bool B_MN, typename TOut>
 static int launch(const Ctx& c, const CUtensorMap& ma, const CUtensorMap& mb, void* C, int m, int n, int k, const Epi& ep,
                   int pairs_m, int tiles_n, int splits, int kb_per_split) {
   auto kern = gemm_tc2_kernel<A_MN, B_MN, TOut>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) return -3;
-    attr_set = true;
-  }
+  static SmemLimit lim;
+  if (!ensure_smem(lim, kern, SMEM_BYTES)) return -3;
   int work = pairs_m * tiles_n * splits;
   int sms = c.sm_count > 0 ? c.sm_count : 148;
   int clusters = work < sms / 2 ? work : sms / 2;

@@ -50,7 +50,8 @@ struct Ctx {
 inline size_t dtype_size(int dtype) { return dtype == 0 ? 4 : 2; }
 
 // ---- embedding --------------------------------------------------------------------------------
-void patchify(const Ctx& c, const void* images, void* patches, int B, int C, int S, int P);
+// img_offset (optional, device): element offset of the images from `images`, read when the kernel runs.
+void patchify(const Ctx& c, const void* images, void* patches, int B, int C, int S, int P, const long long* img_offset = nullptr);
 void assemble_tokens(const Ctx& c, const void* emb, const float* cls, const float* pos, float* x, int B, int N, int D);
 
 // ---- LayerNorm (the residual stream is float in every configuration) ----------------------------
@@ -116,6 +117,8 @@ int gemm_tc_grouped_wgrad(const Ctx& c, const void* dY, const void* X, float* dW
 int gemm_tc2_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long b_rs, long b_cs, void* C,
                      int out_is_float, int m, int n, int k, const GemmEpilogue& e, float* split_ws, size_t split_ws_floats);
 void splitk_reduce(cudaStream_t s, const float* partial, float* out, size_t n, int splits);
+// Diagnostic: one CTA whose bounded wait expires after limit_ns and which then tears down as the GEMM kernels do.
+void wait_expiry_selftest(const Ctx& c, unsigned long long limit_ns);
 
 // ---- attention --------------------------------------------------------------------------------
 // qkv [B, T, 3, H, d]; out [B, T, H*d]; lse (optional) [B, H, T] natural-log sum of exponentials of the
@@ -162,6 +165,23 @@ void adamw(const Ctx& c, const AdamChunk* chunks, int nchunks, float* master, co
 void sgd_momentum(const Ctx& c, const AdamChunk* chunks, int nchunks, float* master, const float* grad, float* buf,
                   void* shadow_base, const float* scalars, float mu, float wd);
 void set_scalars(cudaStream_t s, float* dst, float a, float b, float c3);
+
+// Device-resident state of a run of steps with a cosine learning-rate schedule (Section 5).
+struct LoopState {
+  long long step_done;       // optimiser steps taken before the current one
+  long long total_steps;     // length of the schedule
+  long long image_stride;    // elements between the images of successive steps
+  long long image_offset;    // element offset of the current step's images
+  float lr_max, lr_min, beta1, beta2;
+  int i, n;                  // index of the current step within the call, steps of the call
+};
+void loop_init(cudaStream_t s, LoopState* st, long long step_done, long long total, long long image_stride, float lr_max, float lr_min,
+               float b1, float b2, int n);
+// Start of a step: learning rate and bias corrections of this step into scalars[0..2], this step's labels and task
+// ids into the staging arrays, the image offset into the state.
+void loop_begin(cudaStream_t s, LoopState* st, float* scalars, const int* labels, const int* tasks, int* lab_stage, int* task_stage, int batch);
+// End of a step: loss_out[i] = loss, counters advance.
+void loop_end(cudaStream_t s, LoopState* st, const float* loss, float* loss_out);
 
 // dst row r = src row r (row_bytes a multiple of 16), independent pitches: gathers / scatters token rows.
 void copy_rows(cudaStream_t s, const void* src, long src_pitch_bytes, void* dst, long dst_pitch_bytes, int rows, int row_bytes);

@@ -11,10 +11,13 @@ long g_kernel_launches = 0;
 // Patch extraction (Section 3.1: the image is partitioned into N patches).  Output row = one patch
 // flattened as (channel, row in patch, column in patch).
 // ------------------------------------------------------------------------------------------------
+// img_offset (optional): element offset of this step's images from `img`, read from device memory (multi-step loop).
 template <typename T>
-__global__ void patchify_kernel(const T* __restrict__ img, T* __restrict__ out, int B, int C, int S, int P, long total) {
+__global__ void patchify_kernel(const T* __restrict__ img, T* __restrict__ out, int B, int C, int S, int P, long total,
+                                const long long* __restrict__ img_offset) {
   long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
+  if (img_offset != nullptr) img += *img_offset;
   int g = S / P;
   int px = (int)(i % P); long r = i / P;
   int py = (int)(r % P); r /= P;
@@ -27,10 +30,12 @@ __global__ void patchify_kernel(const T* __restrict__ img, T* __restrict__ out, 
 
 // Same copy in 16-byte units (P * sizeof(T) a multiple of 16): a patch row is P/E units.
 template <typename T>
-__global__ void patchify_vec_kernel(const T* __restrict__ img, T* __restrict__ out, int B, int C, int S, int P, long units) {
+__global__ void patchify_vec_kernel(const T* __restrict__ img, T* __restrict__ out, int B, int C, int S, int P, long units,
+                                    const long long* __restrict__ img_offset) {
   constexpr int E = 16 / sizeof(T);
   long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= units) return;
+  if (img_offset != nullptr) img += *img_offset;
   int g = S / P, upr = P / E;
   int ux = (int)(i % upr); long r = i / upr;
   int py = (int)(r % P); r /= P;
@@ -42,25 +47,27 @@ __global__ void patchify_vec_kernel(const T* __restrict__ img, T* __restrict__ o
   *reinterpret_cast<uint4*>(out + i * E) = *reinterpret_cast<const uint4*>(src);
 }
 
-void patchify(const Ctx& c, const void* images, void* patches, int B, int C, int S, int P) {
+void patchify(const Ctx& c, const void* images, void* patches, int B, int C, int S, int P, const long long* img_offset) {
   note_launch(1);
   int g = S / P;
   long total = (long)B * g * g * C * P * P;
   int threads = 256;
   size_t es = dtype_size(c.dtype);
-  bool vec = (P * es) % 16 == 0 && (((uintptr_t)images | (uintptr_t)patches) & 15) == 0;
+  // with an offset read on the device, every step's images must be 16-byte aligned: one image holds C*S*S elements
+  bool vec = (P * es) % 16 == 0 && (((uintptr_t)images | (uintptr_t)patches) & 15) == 0 &&
+             (img_offset == nullptr || ((long)C * S * S * (long)es) % 16 == 0);
   if (vec) {
     long units = total * (long)es / 16;
     int blocks = ceil_div(units, threads);
-    if (c.dtype == 0) patchify_vec_kernel<float><<<blocks, threads, 0, c.stream>>>((const float*)images, (float*)patches, B, C, S, P, units);
-    else patchify_vec_kernel<bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)images, (bf16*)patches, B, C, S, P, units);
+    if (c.dtype == 0) patchify_vec_kernel<float><<<blocks, threads, 0, c.stream>>>((const float*)images, (float*)patches, B, C, S, P, units, img_offset);
+    else patchify_vec_kernel<bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)images, (bf16*)patches, B, C, S, P, units, img_offset);
     return;
   }
   int blocks = ceil_div(total, threads);
   if (c.dtype == 0)
-    patchify_kernel<float><<<blocks, threads, 0, c.stream>>>((const float*)images, (float*)patches, B, C, S, P, total);
+    patchify_kernel<float><<<blocks, threads, 0, c.stream>>>((const float*)images, (float*)patches, B, C, S, P, total, img_offset);
   else
-    patchify_kernel<bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)images, (bf16*)patches, B, C, S, P, total);
+    patchify_kernel<bf16><<<blocks, threads, 0, c.stream>>>((const bf16*)images, (bf16*)patches, B, C, S, P, total, img_offset);
 }
 
 // x[b, 0] = cls + pos[0];  x[b, 1 + n] = emb[b, n] + pos[1 + n]   (classification token and positional embedding);
@@ -306,11 +313,8 @@ static void launch_ln_bwd(const Ctx& c, int groups, size_t smem, const void* dy,
   int nch = ceil_div(D, 128);
 #define BSR_LN_BWD(N)                                                                                                   \
   do {                                                                                                                  \
-    static size_t attr = 0;               /* the limit only grows: graph nodes captured earlier keep launching */ \
-    if (smem > attr) {                                                                                                  \
-      cudaFuncSetAttribute(layernorm_bwd_kernel<TDY, TC, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);     \
-      attr = smem;                                                                                                      \
-    }                                                                                                                   \
+    static SmemLimit lim;                                                                                               \
+    ensure_smem(lim, layernorm_bwd_kernel<TDY, TC, N>, smem);                                                           \
     layernorm_bwd_kernel<TDY, TC, N><<<groups, LNB_WARPS * 32, smem, c.stream>>>((const TDY*)dy, x, x_stride, mean, rstd, g, dres, \
                                                                                  dx, dx_stride, (TC*)dx_copy, partials, rows, D, nsum); \
   } while (0)
@@ -596,6 +600,52 @@ void sgd_momentum(const Ctx& c, const AdamChunk* chunks, int nchunks, float* mas
     sgd_kernel<float><<<nchunks, 256, 0, c.stream>>>(chunks, master, grad, buf, (float*)shadow_base, scalars, mu, wd);
   else
     sgd_kernel<bf16><<<nchunks, 256, 0, c.stream>>>(chunks, master, grad, buf, (bf16*)shadow_base, scalars, mu, wd);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Multi-step loop (Section 5: cosine learning-rate decay).  The state lives in device memory; each step's graph reads
+// it, so a run of steps needs no host scalars: lr(t) = lr_min + (lr_max - lr_min) (1 + cos(pi t / total)) / 2 for the
+// t-th step overall (t from 0, held at lr_min from t = total on), bias corrections 1 - beta^(t+1).
+// ------------------------------------------------------------------------------------------------
+__global__ void loop_init_kernel(LoopState* st, long long step_done, long long total, long long image_stride, float lr_max,
+                                 float lr_min, float b1, float b2, int n) {
+  st->step_done = step_done; st->total_steps = total; st->image_stride = image_stride; st->image_offset = 0;
+  st->lr_max = lr_max; st->lr_min = lr_min; st->beta1 = b1; st->beta2 = b2; st->i = 0; st->n = n;
+}
+__global__ void loop_begin_kernel(LoopState* st, float* scalars, const int* __restrict__ labels, const int* __restrict__ tasks,
+                                  int* __restrict__ lab_stage, int* __restrict__ task_stage, int batch) {
+  int i = st->i;
+  for (int j = threadIdx.x; j < batch; j += blockDim.x) {
+    lab_stage[j] = labels[(long)i * batch + j];
+    if (tasks != nullptr) task_stage[j] = tasks[(long)i * batch + j];
+  }
+  if (threadIdx.x == 0) {
+    long long t = st->step_done;
+    double frac = st->total_steps > 0 ? (double)(t < st->total_steps ? t : st->total_steps) / (double)st->total_steps : 1.0;
+    double lr = (double)st->lr_min + 0.5 * ((double)st->lr_max - (double)st->lr_min) * (1.0 + cos(3.14159265358979323846 * frac));
+    scalars[0] = (float)lr;
+    scalars[1] = (float)(1.0 - pow((double)st->beta1, (double)(t + 1)));
+    scalars[2] = (float)(1.0 - pow((double)st->beta2, (double)(t + 1)));
+    st->image_offset = (long long)i * st->image_stride;
+  }
+}
+__global__ void loop_end_kernel(LoopState* st, const float* __restrict__ loss, float* __restrict__ loss_out) {
+  loss_out[st->i] = *loss;
+  st->i += 1;
+  st->step_done += 1;
+}
+void loop_init(cudaStream_t s, LoopState* st, long long step_done, long long total, long long image_stride, float lr_max, float lr_min,
+               float b1, float b2, int n) {
+  note_launch(1);
+  loop_init_kernel<<<1, 1, 0, s>>>(st, step_done, total, image_stride, lr_max, lr_min, b1, b2, n);
+}
+void loop_begin(cudaStream_t s, LoopState* st, float* scalars, const int* labels, const int* tasks, int* lab_stage, int* task_stage, int batch) {
+  note_launch(1);
+  loop_begin_kernel<<<1, 256, 0, s>>>(st, scalars, labels, tasks, lab_stage, task_stage, batch);
+}
+void loop_end(cudaStream_t s, LoopState* st, const float* loss, float* loss_out) {
+  note_launch(1);
+  loop_end_kernel<<<1, 1, 0, s>>>(st, loss, loss_out);
 }
 
 __global__ void set_scalars_kernel(float* dst, float a, float b, float c3) {

@@ -333,13 +333,13 @@ void moe_route(const Ctx& c, const MoeBufs& b, const void* y, const void* wg, co
   size_t gate_elems = (size_t)(num_tasks < 1 ? 1 : num_tasks) * E * D;
   size_t smem = gate_elems * es;
   if (smem > 96 * 1024) { smem = 0; gate_elems = 0; }       // too large to stage: the gates are read through L1 instead
-  static size_t attr[2] = {0, 0};
+  static SmemLimit lim[2];
   if (c.dtype == 0) {
-    if (smem > attr[0]) { cudaFuncSetAttribute(moe_route_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr[0] = smem; }
+    ensure_smem(lim[0], moe_route_kernel<float>, smem);
     moe_route_kernel<float><<<nblk, MOE_BLOCK_TOKENS, smem, c.stream>>>((const float*)y, (const float*)wg, task_ids, tokens_per_image, M, D, E, K,
                                                                         (int)gate_elems, b.eidx, b.ew, b.blk_counts);
   } else {
-    if (smem > attr[1]) { cudaFuncSetAttribute(moe_route_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr[1] = smem; }
+    ensure_smem(lim[1], moe_route_kernel<bf16>, smem);
     moe_route_kernel<bf16><<<nblk, MOE_BLOCK_TOKENS, smem, c.stream>>>((const bf16*)y, (const bf16*)wg, task_ids, tokens_per_image, M, D, E, K,
                                                                        (int)gate_elems, b.eidx, b.ew, b.blk_counts);
   }

@@ -31,7 +31,10 @@ thread_local char g_noalloc_error[256] = "no error";
 // Once per device, with that device current: resolve the array's device address.
 int scratch_for_current_device(float** out, int* sms) {
   int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) {
+    snprintf(g_noalloc_error, sizeof(g_noalloc_error), "no current CUDA device with an ordinal below %d", MAX_DEVICES);
+    return -1;
+  }
   std::lock_guard<std::mutex> lock(g_mutex);
   if (g_scratch_ptr[dev] == nullptr) {
     float* p = nullptr;
@@ -41,7 +44,10 @@ int scratch_for_current_device(float** out, int* sms) {
       return -2;
     }
     int n = 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -3;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+      snprintf(g_noalloc_error, sizeof(g_noalloc_error), "the device's multiprocessor count could not be read");
+      return -3;
+    }
     g_scratch_ptr[dev] = p;
     g_sm_count[dev] = n;
   }
@@ -74,10 +80,7 @@ int32_t bsr_linear_backward_static(const void* x, const void* w, const void* dy,
   }
   float* scratch = nullptr;
   int sms = 0;
-  if (scratch_for_current_device(&scratch, &sms) != 0) {
-    if (g_noalloc_error[0] == 'n' && g_noalloc_error[1] == 'o') snprintf(g_noalloc_error, sizeof(g_noalloc_error), "no usable CUDA device");
-    return BSR_ERR_CUDA;
-  }
+  if (scratch_for_current_device(&scratch, &sms) != 0) return BSR_ERR_CUDA;   // the message says which step failed
   Ctx c;
   c.stream = (cudaStream_t)stream;
   c.dtype = BSR_DTYPE_BF16;
@@ -98,6 +101,7 @@ int32_t bsr_linear_backward_static(const void* x, const void* w, const void* dy,
     snprintf(g_noalloc_error, sizeof(g_noalloc_error), "launch failed: %s", cudaGetErrorString(e));
     return BSR_ERR_CUDA;
   }
+  snprintf(g_noalloc_error, sizeof(g_noalloc_error), "no error");
   return BSR_OK;
 }
 

@@ -7,15 +7,35 @@ from paper_2405_10951_b200 import synth
 FP32_TOL = 1e-4          # relative, ||gpu - ref||_2 / ||ref||_2 per tensor
 BF16_TOL = 2e-2
 EXACT_MARGIN = 1e-3      # kept sets must be identical where the oracle's boundary margin exceeds this (fp32)
-# bf16 storage perturbs every score by up to ~1e-2 relative (8 mantissa bits on q, k and on the block input),
-# so a bf16 run may legitimately swap tokens whose scores are closer than that.
-BF16_SCORE_TOL = 1e-1
+# In a bf16 step the scores at a drop location carry the rounding of everything upstream (weights, activations and
+# Q/K stored with 8 mantissa bits).  Measured on B200 against the oracle run on the same kept sets, as the largest
+# deviation of a score relative to itself (scores below the K-th: relative to the K-th): at most 2.0e-3 on the literal
+# configurations (std-0.02 weights, all five workloads at their full batch) and at most 5.6e-2 on the "peaked"
+# variants, whose 3-6x larger query/key weights amplify every rounding inside the attention logits.  The tolerances
+# are twice those figures; a kept set must be identical to the oracle's wherever the oracle's boundary margin exceeds
+# twice the tolerance (both sides of the boundary may move by one tolerance).  On identical bf16 Q/K/V the strict
+# rule (margin 1e-3) holds: tests/test_gpu_select_chain.py.
+BF16_SCORE_TOL = 5e-3
+BF16_SCORE_TOL_PEAKED = 1e-1
+BF16_EXACT_MARGIN = 2 * BF16_SCORE_TOL
+BF16_EXACT_MARGIN_PEAKED = 2 * BF16_SCORE_TOL_PEAKED
+# The largest single deviation of a tensor, max|gpu - ref| / max|ref|, may exceed the tensor's L2 figure by this factor
+# (measured: the two agree within 1.7x on every tensor of every case; a stale or mis-scaled tile shows as >> 1).
+MAX_FACTOR = 2.0
 
 
 def rel_err(a, b):
     a = np.asarray(a, dtype=np.float64).ravel()
     b = np.asarray(b, dtype=np.float64).ravel()
     return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def max_err(a, b):
+    """max |a - b| / max |b|: the largest single deviation against the tensor's own scale.  A stale or mis-scaled
+    tile that moves the L2 figure by little still shows here."""
+    a = np.asarray(a, dtype=np.float64).ravel()
+    b = np.asarray(b, dtype=np.float64).ravel()
+    return float(np.abs(a - b).max() / max(np.abs(b).max(), 1e-300))
 
 
 def param_shape(cfg, name):
@@ -50,26 +70,35 @@ def run_gpu_step(cfg, images, labels, task_ids, params, batch=None, steps=1):
         tokens = 1 if (l == cfg.depth - 1 and l not in cfg.drop_blocks) else eng.tf[l]     # last block: classification rows only
         e = eng.get_tensor(f"moe_experts/{l}", (B * tokens * cfg.moe_top_k,)).cpu().numpy()
         out["experts"][l] = e.astype(np.int64).reshape(B, tokens, cfg.moe_top_k)
+    # head-mean scores of every drop location (Eq. 6), as the select kernel saw them
+    out["scores"] = [eng.get_tensor(f"scores/{l}", (B, eng.ta[l] - 1)).cpu().numpy().astype(np.float64)
+                     for l in range(cfg.depth) if eng.k[l] >= 0]
     out["footprint"] = eng.footprint()
     out["engine"] = eng
     return out
 
 
-def check_selection(cfg, gpu_kept, forced_run, exact_margin, score_tol):
+def check_selection(cfg, gpu_kept, forced_run, exact_margin, score_tol, gpu_scores=None):
     """The rule for kept-index sets.
 
     `forced_run` is the oracle run with the GPU's kept sets forced, so its scores at every location are
     the oracle's scores for exactly the token sequence the GPU saw.  Per image and location:
-      * the GPU's set must be a valid top-K of those scores within score_tol
+      * with `gpu_scores` (the head-mean scores the select kernel itself read, float32): the GPU's set is bit for
+        bit the top-K of those scores under the oracle's rule (ties to the lower index), and every score agrees with
+        the oracle's within score_tol, relative to itself or, for scores below the K-th, to the K-th score;
+      * the GPU's set must be a valid top-K of the oracle's scores within score_tol
         (weakest kept score >= strongest dropped score - score_tol * s_(K));
       * where the oracle's own boundary margin exceeds exact_margin the set must be identical to the
         oracle's own choice.
-    Returns (number of sets compared, number identical to the oracle's own choice).
+    Returns a report: sets compared, sets identical to the oracle's own choice, sets whose margin demanded identity,
+    and per location the worst score deviation relative to the K-th score.
     """
-    total = same = 0
+    total = same = strict = 0
+    score_err = []
     for loc, (kept, scores) in enumerate(zip(gpu_kept, forced_run["scores"])):
         B, k = kept.shape
         m = scores.shape[1]
+        worst = 0.0
         for b in range(B):
             own, own_dropped = O.select_tokens(scores[b], k)
             mine = np.sort(kept[b])
@@ -79,13 +108,21 @@ def check_selection(cfg, gpu_kept, forced_run, exact_margin, score_tol):
             identical = np.array_equal(own, mine)
             total += 1
             same += int(identical)
+            sk = scores[b][own].min()
+            if gpu_scores is not None:
+                sg = gpu_scores[loc][b]
+                assert np.array_equal(O.select_tokens(sg.astype(np.float32), k)[0], mine), f"location {loc} image {b}: not the top-K of the GPU's own scores"
+                dev = float((np.abs(sg - scores[b]) / np.maximum(scores[b], sk)).max())   # relative; small scores against s_(K)
+                worst = max(worst, dev)
+                assert dev <= score_tol, f"location {loc} image {b}: scores off by {dev:.3e} of s_(K)"
             if len(rest):
-                sk = scores[b][own].min()
                 assert scores[b][mine].min() >= scores[b][rest].max() - score_tol * sk, (loc, b)
                 margin = O.boundary_margin(scores[b], own, own_dropped)
                 if margin > exact_margin:
+                    strict += 1
                     assert identical, f"location {loc} image {b}: margin {margin:.3e} but sets differ"
-    return total, same
+        score_err.append(worst)
+    return {"sets": total, "sets_identical": same, "sets_strict": strict, "score_err": score_err}
 
 
 def forced_experts_of(cfg, gpu, token_counts):
@@ -117,17 +154,50 @@ def check_routing(cfg, ref, gpu, logit_tol):
     return total, flips
 
 
-def compare_step(cfg, images, labels, task_ids, params, gpu, tol, exact_margin, score_tol):
+def oracle_reference(cfg, images, labels, task_ids, params, gpu, chunk=None):
+    """The oracle's step on the same inputs, with the GPU's kept sets (and expert choices) forced.  Images are
+    independent until the batch-mean loss, so a large batch is run in chunks: the loss and every gradient of the
+    full batch are the chunk results weighted by chunk size; logits, scores and routing records are concatenated."""
+    B = images.shape[0]
     forced = gpu["kept"] if gpu["kept"] else None
     fe = None
     if gpu.get("experts"):
         sched = O.token_schedule(cfg)
         fe = forced_experts_of(cfg, gpu, {l: sched[l][1] for l in cfg.moe_blocks})
-    ref = O.train_step(cfg, params, images, labels, task_ids, forced_keep=forced, forced_experts=fe)
+    if chunk is None or chunk >= B:
+        return O.train_step(cfg, params, images, labels, task_ids, forced_keep=forced, forced_experts=fe), fe
+    ref = None
+    for s0 in range(0, B, chunk):
+        sl = slice(s0, min(B, s0 + chunk))
+        part = O.train_step(cfg, params, images[sl], labels[sl], task_ids[sl], forced_keep=[k[sl] for k in forced] if forced else None,
+                            forced_experts={l: e[sl] for l, e in fe.items()} if fe else None)
+        wgt = (sl.stop - sl.start) / B
+        if ref is None:
+            ref = {"loss": 0.0, "grads": {n: np.zeros_like(g) for n, g in part["grads"].items()}, "logits": [], "scores": [[] for _ in part["scores"]],
+                   "routing": {l: {"glogits": [], "own_experts": []} for l in part["routing"]}}
+        ref["loss"] += wgt * part["loss"]
+        for n, g in part["grads"].items():
+            ref["grads"][n] += wgt * g
+        ref["logits"].append(part["logits"])
+        for i, sc in enumerate(part["scores"]):
+            ref["scores"][i].append(sc)
+        for l, r in part["routing"].items():
+            ref["routing"][l]["glogits"].append(r["glogits"])
+            ref["routing"][l]["own_experts"].append(r["own_experts"])
+    ref["logits"] = np.concatenate(ref["logits"], axis=0)
+    ref["scores"] = [np.concatenate(x, axis=0) for x in ref["scores"]]
+    ref["routing"] = {l: {k: np.concatenate(v, axis=0) for k, v in r.items()} for l, r in ref["routing"].items()}
+    return ref, fe
+
+
+def compare_step(cfg, images, labels, task_ids, params, gpu, tol, exact_margin, score_tol, chunk=None):
+    forced = gpu["kept"] if gpu["kept"] else None
+    ref, fe = oracle_reference(cfg, images, labels, task_ids, params, gpu, chunk)
     if fe:
         check_routing(cfg, ref, gpu, 2e-2)
-    total, same = check_selection(cfg, gpu["kept"], ref, exact_margin, score_tol) if forced else (0, 0)
-    report = {"sets": total, "sets_identical": same}
+    report = {"sets": 0, "sets_identical": 0, "sets_strict": 0, "score_err": []}
+    if forced:
+        report = check_selection(cfg, gpu["kept"], ref, exact_margin, score_tol, gpu.get("scores"))
     assert abs(gpu["loss"] - ref["loss"]) <= tol * abs(ref["loss"]), (gpu["loss"], ref["loss"])
     B = images.shape[0]
     fin = np.isfinite(ref["logits"])
@@ -135,13 +205,18 @@ def compare_step(cfg, images, labels, task_ids, params, gpu, tol, exact_margin, 
     e = rel_err(gpu["logits"][:B][fin], ref["logits"][fin])
     report["logits"] = e
     assert e <= tol, ("logits", e)
-    worst = 0.0
+    assert max_err(gpu["logits"][:B][fin], ref["logits"][fin]) <= MAX_FACTOR * tol, "logits (largest deviation)"
+    worst = worst_max = 0.0
     for n, g in ref["grads"].items():
         e = rel_err(gpu["grads"][n], g)
         worst = max(worst, e)
         assert e <= tol, (n, e)
+        em = max_err(gpu["grads"][n], g)
+        worst_max = max(worst_max, em)
+        assert em <= MAX_FACTOR * tol, (n, "largest deviation", em)
         assert rel_err(gpu["m"][n], (1 - cfg.beta1) * g) <= tol, n
     report["worst_grad"] = worst
+    report["worst_grad_max"] = worst_max
     # the update itself, from the GPU's own gradient (AdamW's first step is a sign function of g: comparing
     # updated weights across implementations would amplify rounding of near-zero gradients without bound)
     for n in ref["grads"]:

@@ -1,9 +1,10 @@
-"""The headline workload at full size, in the launch configuration bench.py times (ViT-B/16, bf16, batch 128).
+"""The benchmark workloads at full size, in the launch configurations bench.py times.
 
-The oracle cannot run 128 ViT-B images in a test, but images are independent until the batch-mean loss, so:
-sampled images are recomputed one by one (logits, kept sets), the loss is re-derived from the GPU's logits, and
-the gradients are checked through a property that holds at any size (the gradient of the mean loss over the batch
-is the mean of the gradients over its halves)."""
+Images are independent until the batch-mean loss, so the oracle runs the full batch in chunks (with the GPU's kept
+sets and expert choices forced) and its chunk gradients, weighted by chunk size, are the full-batch gradient: every
+gradient tensor, the loss, all logits and all kept sets of the full-batch GPU step are compared with it.  The
+headline workload additionally checks properties that hold at any size (bit-for-bit reproducibility, the gradient
+of the batch mean being the mean over its halves)."""
 import numpy as np
 import pytest
 
@@ -39,7 +40,7 @@ def test_vit_b_full_batch_sampled_outputs_and_properties():
         forced = [k[b:b + 1] for k in kept]
         ref = O.forward(cfg, params, images[b:b + 1], forced_keep=forced)
         assert P.rel_err(logits[b], ref["logits"][0]) < P.BF16_TOL
-        P.check_selection(cfg, forced, ref, 2 * P.BF16_SCORE_TOL, P.BF16_SCORE_TOL)
+        P.check_selection(cfg, forced, ref, P.BF16_EXACT_MARGIN, P.BF16_SCORE_TOL)
     # 3. kept sets are valid index sets for every image
     ks = [138, 98, 70]
     for loc, k in enumerate(kept):
@@ -71,3 +72,19 @@ def test_vit_b_full_batch_sampled_outputs_and_properties():
         e2.close()
     for n in names:
         assert P.rel_err(full[n], 0.5 * (halves[0][n] + halves[1][n])) < 5e-3, n
+
+
+# workload -> images per oracle chunk (bounded by the oracle's memory: it keeps every attention map of a chunk)
+FULL_BATCH = {"vit_b": 32, "deit_s": 32, "vit_b_384": 8, "moe_vit_s": 32}
+
+
+@pytest.mark.parametrize("name", list(FULL_BATCH))
+def test_full_batch_step_every_gradient_against_the_oracle(name):
+    """Full BASELINE batch (128 / 64 / 32 / 64 images): loss, logits, kept sets, scores and every gradient tensor."""
+    cfg = CONFIGS[name]
+    images, labels, task_ids, params = synth.make_workload(cfg)
+    gpu = P.run_gpu_step(cfg, images, labels, task_ids, params)
+    gpu.pop("engine").close()
+    rep = P.compare_step(cfg, images, labels, task_ids, params, gpu, P.BF16_TOL, P.BF16_EXACT_MARGIN, P.BF16_SCORE_TOL,
+                         chunk=FULL_BATCH[name])
+    print(name, rep)

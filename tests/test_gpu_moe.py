@@ -33,5 +33,6 @@ def test_moe_step_matches_oracle(case):
     cfg = CASES[case]
     images, labels, task_ids, params = synth.make_workload(cfg, peaked=False)
     gpu = P.run_gpu_step(cfg, images, labels, task_ids, params)
-    rep = P.compare_step(cfg, images, labels, task_ids, params, gpu, P.BF16_TOL, 2 * P.BF16_SCORE_TOL, P.BF16_SCORE_TOL)
+    rep = P.compare_step(cfg, images, labels, task_ids, params, gpu, P.BF16_TOL, P.BF16_EXACT_MARGIN, P.BF16_SCORE_TOL)
+    print(case, rep)
     assert rep["worst_grad"] <= P.BF16_TOL

@@ -49,18 +49,25 @@ BF16_CASES = {
 }
 
 
+# Peaked cases whose worst gradient tensor measures just above 2e-2 (2.01e-2 and 2.09e-2 on B200; every other case,
+# literal or peaked, stays below 1.9e-2): 4-6x larger query/key weights in a model of few, short rows leave little
+# averaging.  They alone get 1.5x the bf16 tolerance.
+PEAKED_WIDE = {"mini", "deit_s_keep_0p3_late"}
+
+
 @pytest.mark.parametrize("peaked", [False, True])
 @pytest.mark.parametrize("case", list(BF16_CASES))
 def test_bf16_step_matches_oracle(case, peaked):
-    """The literal configurations (std-0.02 weights) must hold the 2e-2 tolerance.  The peaked variant exists for
-    the selection check: its 4-6x larger query/key weights amplify every bf16 rounding inside the attention of
-    all blocks, so its numeric tolerance is 1.5x wider."""
+    """Every configuration holds the 2e-2 tolerance on loss, logits and every gradient (two named peaked cases:
+    3e-2); scores and kept sets follow the measured rule stated in parity.py."""
     cfg = BF16_CASES[case]
     images, labels, task_ids, params = synth.make_workload(cfg, peaked=peaked)
     gpu = P.run_gpu_step(cfg, images, labels, task_ids, params)
-    tol = P.BF16_TOL * (1.5 if peaked else 1.0)
-    rep = P.compare_step(cfg, images, labels, task_ids, params, gpu, tol, 2 * P.BF16_SCORE_TOL, P.BF16_SCORE_TOL)
-    assert rep["sets_identical"] >= 0.25 * rep["sets"], rep
+    tol = P.BF16_TOL * (1.5 if (peaked and case in PEAKED_WIDE) else 1.0)
+    margin, score_tol = (P.BF16_EXACT_MARGIN_PEAKED, P.BF16_SCORE_TOL_PEAKED) if peaked else (P.BF16_EXACT_MARGIN, P.BF16_SCORE_TOL)
+    rep = P.compare_step(cfg, images, labels, task_ids, params, gpu, tol, margin, score_tol)
+    print(case, "peaked" if peaked else "literal", rep)
+    assert rep["sets_identical"] >= 0.6 * rep["sets"], rep
 
 
 def test_eval_forward_matches_oracle_and_train_forward():
@@ -79,6 +86,35 @@ def test_eval_forward_matches_oracle_and_train_forward():
     # a smaller batch than max_batch
     logits3, kept3 = eng.eval_forward(eng.images_to_device(images[:3]))
     assert torch.equal(logits3, logits[:3])
+
+
+@pytest.mark.parametrize("peaked", [False, True])
+def test_eval_forward_bf16_matches_oracle(peaked):
+    """bsr_eval_forward on the tcgen05 path (ViT-B/16 shapes, three images): logits against the oracle run with the
+    same kept sets, the selection rule at every drop location, and bit-identical logits from the training step's
+    forward pass (same kernels, activations saved or not)."""
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    cfg = CONFIGS["vit_b"].with_(batch=3)
+    images, labels, task_ids, params = synth.make_workload(cfg, peaked=peaked)
+    eng = Bd.Engine(cfg)
+    eng.set_params(params)
+    img = eng.images_to_device(images)
+    logits, kept = eng.eval_forward(img)
+    torch.cuda.synchronize()
+    kept = [k.cpu().numpy().astype(np.int64) for k in kept]
+    scores = [eng.get_tensor(f"scores/{l}", (cfg.batch, eng.ta[l] - 1)).cpu().numpy().astype(np.float64) for l in cfg.drop_blocks]
+    ref = O.forward(cfg, params, images, forced_keep=kept)
+    assert P.rel_err(logits.cpu().numpy(), ref["logits"]) < P.BF16_TOL
+    assert P.max_err(logits.cpu().numpy(), ref["logits"]) < P.MAX_FACTOR * P.BF16_TOL
+    margin, score_tol = (P.BF16_EXACT_MARGIN_PEAKED, P.BF16_SCORE_TOL_PEAKED) if peaked else (P.BF16_EXACT_MARGIN, P.BF16_SCORE_TOL)
+    rep = P.check_selection(cfg, kept, ref, margin, score_tol, scores)
+    print("eval", "peaked" if peaked else "literal", rep)
+    loss, kept2 = eng.train_step(img, torch.as_tensor(labels).cuda())
+    eng.sync_status()
+    assert torch.equal(eng.get_tensor("logits", (cfg.batch, eng.cmax)), logits)
+    assert all(np.array_equal(a.cpu().numpy(), b) for a, b in zip(kept2, kept))
+    eng.close()
 
 
 def test_two_steps_follow_the_oracle_and_are_deterministic():
@@ -102,7 +138,7 @@ def test_sgd_momentum_follows_the_oracle(dtype):
     parameter change and the momentum buffer are compared with the oracle's directly, per tensor."""
     base = TINY if dtype == "fp32" else MINI_BF16
     cfg = base.with_(optimizer="sgd", momentum=0.9, lr=1e-2, weight_decay=0.01)
-    tol = P.FP32_TOL if dtype == "fp32" else P.BF16_TOL * 1.5
+    tol = P.FP32_TOL if dtype == "fp32" else P.BF16_TOL * 1.5      # mini, peaked: see PEAKED_WIDE
     images, labels, task_ids, params = synth.make_workload(cfg, peaked=True)
     gpu = P.run_gpu_step(cfg, images, labels, task_ids, params, steps=2)
     names = O.trainable_names(cfg, params)
@@ -147,6 +183,37 @@ def test_error_paths_leave_the_context_usable():
     fp = eng.footprint()
     assert fp["saved_activation_bytes"] > 0 and fp["trainable_params"] == sum(
         int(np.prod(synth.param_shapes(cfg)[n])) for n in O.trainable_names(cfg, params))
+
+
+def test_expired_device_wait_is_reported_and_the_context_stays_usable():
+    """The failure path of the tensor-core kernels without a fault: a CTA whose bounded wait runs out (a barrier that
+    nothing arrives at, limit 1 ms) frees its tensor memory and returns; bsr_sync_status reports
+    BSR_ERR_DEVICE_TIMEOUT once, and the next training step on the same handle gives the result of a fresh handle."""
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    cfg = MINI_BF16
+    images, labels, task_ids, params = synth.make_workload(cfg, peaked=True)
+    fresh = P.run_gpu_step(cfg, images, labels, task_ids, params)
+    eng = Bd.Engine(cfg)
+    eng.set_params(params)
+    eng.sync_status()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    eng.selftest_wait_expiry(1_000_000)
+    t1.record()
+    with pytest.raises(Bd.BsrError) as e:
+        eng.sync_status()
+    assert e.value.status == -5 and "wait expired" in str(e.value)
+    assert 0.9 < t0.elapsed_time(t1) < 50.0                 # it waited its millisecond and no longer
+    eng.sync_status()                                       # reported once, then clear
+    with pytest.raises(Bd.BsrError):
+        eng.selftest_wait_expiry(10)                        # limits outside [1e3, 1e8] ns are refused
+    loss, kept = eng.train_step(eng.images_to_device(images), torch.as_tensor(labels).cuda())
+    eng.sync_status()
+    assert float(loss.cpu()[0]) == fresh["loss"]
+    assert all(np.array_equal(a.cpu().numpy(), b) for a, b in zip(kept, fresh["kept"]))
+    eng.close()
 
 
 def test_graph_replay_equals_launch_by_launch():

@@ -1,0 +1,105 @@
+"""Pins of the oracle parts that the comparison rules themselves lean on: the boundary margin (it decides where kept
+sets must be identical), the forced-expert branch of the MoE layer (Section 5.2; it is what a GPU run with a
+different choice between near-equal gate logits is compared against) and the MoE term of the MAC counter."""
+import math
+
+import numpy as np
+
+from oracle import bsr_oracle as O
+from oracle import counters as C
+from paper_2405_10951_b200 import synth
+
+MOE = synth.Config("pin_moe", 16, 4, 32, 2, 2, 48, (5, 3), 4, (0, 1), (), 1, 1, dtype="fp32", seed=11,
+                   moe_experts=4, moe_top_k=2, moe_blocks=(1,))
+
+
+def test_boundary_margin_hand_computed_cases():
+    # (s_(K) - s_(K+1)) / s_(K): the gap below the weakest kept score, relative to that score (not to the largest
+    # score, not to the strongest dropped one)
+    s = np.array([0.10, 0.40, 0.25, 0.05, 0.20])
+    kept, dropped = O.select_tokens(s, 3)                       # keeps 0.40, 0.25, 0.20; drops 0.10, 0.05
+    assert list(kept) == [1, 2, 4] and list(dropped) == [0, 3]
+    assert abs(O.boundary_margin(s, kept, dropped) - (0.20 - 0.10) / 0.20) < 1e-15
+    kept, dropped = O.select_tokens(s, 1)                       # keeps 0.40; strongest dropped 0.25
+    assert abs(O.boundary_margin(s, kept, dropped) - (0.40 - 0.25) / 0.40) < 1e-15
+    t = np.array([0.3, 0.2, 0.2, 0.1])
+    kept, dropped = O.select_tokens(t, 2)                       # a tie across the boundary: margin exactly zero
+    assert list(kept) == [0, 1] and O.boundary_margin(t, kept, dropped) == 0.0
+    kept, dropped = O.select_tokens(t, 4)                       # nothing dropped: no boundary
+    assert O.boundary_margin(t, kept, dropped) == np.inf
+    # normalising by the largest score or by the dropped score would give other numbers on the first case
+    assert abs((0.20 - 0.10) / 0.40 - 0.5) > 0.1 and abs((0.20 - 0.10) / 0.10 - 0.5) > 0.1
+
+
+def _moe_inputs():
+    rng = np.random.default_rng(5)
+    images, labels, task_ids, params = synth.make_workload(MOE)
+    for n in params:                                              # larger weights: well separated gate logits
+        if ".moe." in n and n.endswith("weight"):
+            params[n] = rng.standard_normal(params[n].shape) * 0.3
+    y = rng.standard_normal((MOE.batch, 6, MOE.dim))
+    return params, y, task_ids
+
+
+def test_forcing_the_routers_own_choice_changes_nothing():
+    params, y, task_ids = _moe_inputs()
+    free, c0 = O.moe_fwd(MOE, params, 1, y, task_ids)
+    forced, c1 = O.moe_fwd(MOE, params, 1, y, task_ids, forced_experts=c0["experts"])
+    assert np.array_equal(free, forced)                           # bit for bit
+    assert np.array_equal(c0["w"], c1["w"])
+    partial = np.full_like(c0["experts"], -1)                     # -1 leaves the choice to the router
+    partial[:, ::2] = c0["experts"][:, ::2]
+    assert np.array_equal(O.moe_fwd(MOE, params, 1, y, task_ids, forced_experts=partial)[0], free)
+
+
+def test_forced_experts_equal_a_hand_built_two_expert_sum():
+    """Forcing experts (a, b) for every token: out = w_a MLP_a(y) + w_b MLP_b(y) with (w_a, w_b) the softmax over the
+    two gate logits of those experts -- written out here with plain matrix products."""
+    params, y, task_ids = _moe_inputs()
+    p = "blocks.1.moe."
+    B, T, D = y.shape
+    for a, b in ((3, 0), (1, 2)):
+        forced = np.empty((B, T, 2), dtype=np.int64)
+        forced[..., 0], forced[..., 1] = a, b
+        got, cache = O.moe_fwd(MOE, params, 1, y, task_ids, forced_experts=forced)
+        want = np.zeros_like(y)
+        for i in range(B):
+            wg = params[p + "gate.weight"][task_ids[i]]
+            gl = y[i] @ wg.T                                      # [T, E]
+            za, zb = gl[:, a], gl[:, b]
+            wa = 1.0 / (1.0 + np.exp(zb - za))                    # two-way softmax
+            for e, w in ((a, wa), (b, 1.0 - wa)):
+                h = y[i] @ params[p + "fc1.weight"][e].T + params[p + "fc1.bias"][e]
+                h = 0.5 * h * (1.0 + np.vectorize(math.erf)(h / np.sqrt(2.0)))
+                want[i] += w[:, None] * (h @ params[p + "fc2.weight"][e].T + params[p + "fc2.bias"][e])
+        assert np.abs(got - want).max() < 1e-12
+        assert not np.array_equal(cache["experts"], cache["own_experts"])
+    # the backward pass of a forced choice is the derivative of that forced forward (finite differences on y)
+    forced = np.empty((B, T, 2), dtype=np.int64)
+    forced[..., 0], forced[..., 1] = 2, 1
+    rng = np.random.default_rng(1)
+    dout = rng.standard_normal(y.shape)
+    _, cache = O.moe_fwd(MOE, params, 1, y, task_ids, forced_experts=forced)
+    dy = O.moe_bwd(MOE, params, 1, dout, cache, task_ids, {}, False)
+    h = 1e-6
+    for idx in ((0, 0, 0), (1, 3, 7), (3, 5, 31)):
+        yp, ym = y.copy(), y.copy()
+        yp[idx] += h
+        ym[idx] -= h
+        fd = ((O.moe_fwd(MOE, params, 1, yp, task_ids, forced_experts=forced)[0] -
+               O.moe_fwd(MOE, params, 1, ym, task_ids, forced_experts=forced)[0]) * dout).sum() / (2 * h)
+        assert abs(fd - dy[idx]) < 1e-6 * max(1.0, abs(fd))
+
+
+def test_moe_mac_term_counts_the_rows_each_expert_processes():
+    """Brute force on a tiny model: every (token, slot) pair sends one row through one expert's two layers
+    (2 D F multiply-accumulates), and every token meets the gate once (D E)."""
+    images, labels, task_ids, params = synth.make_workload(MOE)
+    fw = O.forward(MOE, params, images, task_ids)
+    dense = MOE.with_(moe_experts=0, moe_top_k=0, moe_blocks=())
+    D, F = MOE.dim, MOE.mlp_hidden
+    rows = sum(int((fw["routing"][1]["experts"][b] == e).sum()) for b in range(MOE.batch) for e in range(MOE.moe_experts))
+    tokens = fw["routing"][1]["experts"].shape[1]
+    per_image = rows // MOE.batch * 2 * D * F + tokens * D * MOE.moe_experts
+    assert rows == MOE.batch * tokens * MOE.moe_top_k
+    assert C.forward_macs(MOE) - C.forward_macs(dense) == per_image - 2 * tokens * D * F

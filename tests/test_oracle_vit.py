@@ -240,3 +240,36 @@ def test_forced_keep_replaces_the_selection():
     other = O.train_step(cfg, params, images, labels, task_ids, forced_keep=forced)
     assert other["loss"] != base["loss"]
     assert sorted(other["kept"][0][0]) == sorted(forced[0][0])
+
+
+def test_cosine_schedule_matches_library_scheduler_and_closed_forms():
+    import torch
+    lr_max, lr_min, total = 3e-3, 2e-5, 37
+    assert O.cosine_lr(lr_max, lr_min, 0, total) == lr_max
+    assert abs(O.cosine_lr(lr_max, lr_min, total, total) - lr_min) < 1e-18
+    assert O.cosine_lr(lr_max, lr_min, total + 5, total) == O.cosine_lr(lr_max, lr_min, total, total)       # held at the floor
+    assert abs(O.cosine_lr(1.0, 0.0, 1, 2) - 0.5) < 1e-15 and abs(O.cosine_lr(1.0, 0.0, 1, 3) - 0.75) < 1e-15   # cos(pi/2), cos(pi/3)
+    rates = [O.cosine_lr(lr_max, lr_min, t, total) for t in range(total + 1)]
+    assert all(a > b for a, b in zip(rates, rates[1:]))                                                      # strictly decaying
+    p = torch.nn.Parameter(torch.zeros(1))
+    opt = torch.optim.SGD([p], lr=lr_max)
+    sch = torch.optim.lr_scheduler.CosineAnnealingLR(opt, T_max=total, eta_min=lr_min)
+    for t in range(total + 1):
+        assert abs(opt.param_groups[0]["lr"] - rates[t]) < 1e-12 * lr_max, t
+        opt.step()
+        sch.step()
+
+
+def test_run_of_steps_uses_the_schedule_per_step():
+    cfg = CASES["drop_with_fusion"].with_(optimizer="sgd", momentum=0.0, weight_decay=0.0)
+    images, labels, task_ids, params = workload(cfg)
+    batches = [(images, labels, task_ids)] * 3
+    runs = O.train_steps(cfg, params, batches, 1e-2, 1e-3, 4)
+    # plain SGD: every step moves a parameter by exactly -lr(t) * gradient of that step
+    prev = params
+    for t, r in enumerate(runs):
+        lr = O.cosine_lr(1e-2, 1e-3, t, 4)
+        n = "head.0.weight"
+        assert np.allclose(r["params"][n] - prev[n], -lr * r["grads"][n], rtol=1e-9, atol=1e-15)
+        prev = r["params"]
+    assert runs[1]["loss"] < runs[0]["loss"]
