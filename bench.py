@@ -5,8 +5,9 @@
 Prints ONE JSON line (rank 0).  A step is one pass of the whole path (frozen-prefix forward, token
 selection and fusion, forward + backward of the trainable blocks and head, AdamW) over one synthetic
 batch.  `value` is images/s with inputs resident in HBM; `e2e` includes the pinned-host -> device copy of
-the images and the device -> host read of the loss in every step.  With N > 1 every rank runs an
-independent replica on its own batch (no data-path collective); the time is the maximum over ranks.
+the images and the device -> host read of the loss in every step, through bsr_train_step_host.  With N > 1 every rank runs an
+its share of the global batch (data parallel: images are independent up to the batch-mean loss, so the one exchange
+is an all-reduce of the trainable gradients between backward pass and update); the time is the maximum over ranks.
 """
 from __future__ import annotations
 
@@ -30,21 +31,42 @@ METRIC = "BSR fine-tune images/s"
 UNIT = "images/s"
 
 
-def step_flops(cfg, batch):
+def step_flops(cfg, batch, executed=False):
     """Algorithmic FLOPs of one step: forward of every block at its token counts, plus twice the forward
-    FLOPs of the trainable blocks for their backward pass, head x3.  Token counts from the library."""
+    FLOPs of the trainable blocks for their backward pass, head x3.  Token counts from the library.
+    executed=True counts what the engine runs: in the last block only the classification row goes through the
+    projection and the FFN (forward and backward), because nothing else of that block's output is ever read."""
     from paper_2405_10951_b200 import binding as Bd
-    ta, tf, _ = Bd.bsr_token_schedule(Bd.make_config(cfg))
+    ta, tf, keep = Bd.bsr_token_schedule(Bd.make_config(cfg))
     D, F = cfg.dim, cfg.mlp_hidden
+    ffn_mult = lambda l: (cfg.moe_top_k if l in cfg.moe_blocks else 1)
     fwd = 2 * cfg.num_patches * (cfg.in_chans * cfg.patch_size ** 2) * D
     bwd = 0
     for l in range(cfg.depth):
-        blk = 2 * (ta[l] * 4 * D * D + 2 * ta[l] * ta[l] * D + 2 * tf[l] * D * F)
+        t_proj, t_ffn = ta[l], tf[l]
+        if executed and l == cfg.depth - 1 and keep[l] < 0:
+            t_proj = t_ffn = 1
+        blk = 2 * (ta[l] * 3 * D * D + t_proj * D * D + 2 * ta[l] * ta[l] * D + 2 * t_ffn * D * F * ffn_mult(l))
         fwd += blk
         if l in cfg.trainable:
             bwd += 2 * blk
     head = 2 * D * max(cfg.num_classes)
     return float(batch) * (fwd + bwd + 3 * head)
+
+
+def step_bytes(cfg, batch, fp):
+    """HBM bytes a step must move even with perfect fusion: the images, every stored weight once, the saved
+    activations written and read back, and per trainable parameter its gradient, master copy, both moments (read and
+    written) and the bf16 shadow: about 30 bytes."""
+    es = 2 if cfg.dtype == "bf16" else 4
+    images = batch * cfg.in_chans * cfg.image_size ** 2 * es
+    return float(images + fp["weight_bytes"] + 2 * fp["saved_activation_bytes"] + 30 * fp["trainable_params"])
+
+
+# DRAM traffic of the dominant kernel (tcgen05 GEMM), bytes per launch averaged over the launches of one step, from the
+# ncu capture summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum).  None until the counters have
+# been taken on the kernel as it now stands.
+GEMM_DRAM_BYTES_PER_LAUNCH = {}
 
 
 def peaks():
@@ -118,6 +140,19 @@ def aggregate(dist, world, batch, steps, ms_local):
     return ms, [world * batch * steps / (m / 1e3) for m in ms]
 
 
+def dp_average(dist, world, grads):
+    """Data-parallel gradient exchange: in-place mean over the ranks of the flat gradient buffer (one all-reduce).
+    Every rank holds the gradient of its local batch mean; with equal shares their mean is the gradient of the
+    global batch mean."""
+    if dist is None:
+        return
+    if dist.get_backend() == "nccl":
+        dist.all_reduce(grads, op=dist.ReduceOp.AVG)
+    else:                                             # gloo has no AVG
+        dist.all_reduce(grads, op=dist.ReduceOp.SUM)
+        grads /= world
+
+
 def oracle_sample_step(cfg, images, labels, task_ids, params):
     from oracle import bsr_oracle as O
     t0 = time.perf_counter()
@@ -163,13 +198,16 @@ def run_reference(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200, help="timed steps (the default keeps the timed region above one second)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="vit_b", choices=list(synth.CONFIGS))
     ap.add_argument("--ref-batch", type=int, default=48)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--gemm-mode", type=int, default=None, help="1: one CTA per tile, 2: CTA pairs (library default if omitted)")
+    ap.add_argument("--parallel", default="auto", choices=["auto", "dp", "replicas"],
+                    help="several GPUs: dp = data parallel, one all-reduce of the trainable gradients per step (the default); "
+                         "replicas = independent copies with no exchange")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     cfg = synth.CONFIGS[args.workload]
@@ -186,12 +224,17 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dist = None
-    if world > 1:
+    dp = args.parallel == "dp" or (args.parallel == "auto" and world > 1)
+    if world > 1 or dp:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29577")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device("cuda", local))
     warm = max(args.warmup, 3)
 
-    images, labels, task_ids, params = synth.make_workload(cfg, seed=cfg.seed + rank)
+    images, labels, task_ids, params = synth.make_workload(cfg, seed=cfg.seed + rank)      # every rank its own batch ...
+    if rank > 0:
+        params = synth.make_workload(cfg, seed=cfg.seed)[3]                                # ... and the same parameters
     eng = Bd.Engine(cfg, device=f"cuda:{local}")
     eng.set_params(params)
     if args.gemm_mode is not None:
@@ -214,9 +257,21 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    grads = eng.grad_buffer() if dp else None
+
+    def step(img, out):
+        """One step on device-resident inputs: the whole step in one call, or, data parallel, its two halves with the
+        gradient all-reduce between them."""
+        if not dp:
+            return eng.train_step(img, lab, tid, want_kept=False, out=out)
+        r = eng.forward_backward(img, lab, tid, want_kept=False, out=out)
+        dp_average(dist, world, grads)
+        eng.optimizer_step()
+        return r
+
     out = None
     for _ in range(warm):
-        eng.train_step(dev_img, lab, tid, want_kept=False, out=out)
+        step(dev_img, out)
         out = eng.last_out
     eng.sync_status()
 
@@ -231,58 +286,58 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
-        loss, _ = eng.train_step(dev_img, lab, tid, want_kept=False, out=out)
+        loss, _ = step(dev_img, out)
     e1.record(stream)
     barrier()
     ms_total = e0.elapsed_time(e1)
     launches = eng.profile_read()["kernel_launches"]
 
     # ---- end to end: pinned host images in, loss out, every step ----------------------------------
-    # Two device staging buffers: the copy of the next step's images (its own stream) overlaps the current step, as an
-    # input pipeline would; every step still waits for its own copy, and the host reads every step's loss, one step
-    # behind the launches (the read of step i-1 waits only for that step).
-    stages = [torch.empty_like(dev_img), torch.empty_like(dev_img)]
-    copy_stream = torch.cuda.Stream()
-    copied = [torch.cuda.Event(), torch.cuda.Event()]
-    read_back = [torch.cuda.Event(), torch.cuda.Event()]
+    # bsr_train_step_host takes HOST buffers: it copies the images and labels into one of two staging slots of the
+    # workspace on its own copy stream (the copy of step i overlaps the kernels of step i-1, as an input pipeline
+    # would), runs the step and copies the loss back to pinned host memory; the host reads every loss, one step behind
+    # the launches.
+    host_lab = torch.as_tensor(labels.astype(np.int32)).pin_memory()
+    host_tid = torch.as_tensor(task_ids.astype(np.int32)).pin_memory() if cfg.num_tasks > 1 else None
     host_losses = [torch.empty(1, dtype=torch.float32).pin_memory(), torch.empty(1, dtype=torch.float32).pin_memory()]
+    done = [torch.cuda.Event(), torch.cuda.Event()]
     e2e_losses = []
-    for sbuf in stages:                                   # untimed: lets the library capture its graph for each buffer
-        sbuf.copy_(dev_img)
-        eng.train_step(sbuf, lab, tid, want_kept=False, out=out)
+    stage_img = torch.empty_like(dev_img) if dp else None
+
+    def host_step(slot):
+        """One step from host memory.  Data parallel, the two halves of the step have no host-buffer form: the images
+        are copied by torch into a device staging tensor on the step's stream (no overlap with the previous step)."""
+        if not dp:
+            eng.train_step_host(host_img, host_lab, host_tid, host_losses[slot])
+            return
+        stage_img.copy_(host_img, non_blocking=True)
+        loss_dev, _ = step(stage_img, out)
+        host_losses[slot].copy_(loss_dev, non_blocking=True)
+
+    for i in range(2):                                    # untimed: lets the library capture its graph for each slot
+        host_step(i)
     eng.sync_status()
     barrier()
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     f0.record(stream)
-    copy_stream.wait_stream(stream)
-    with torch.cuda.stream(copy_stream):
-        stages[0].copy_(host_img, non_blocking=True)
-        copied[0].record(copy_stream)
     for i in range(args.steps):
         cur = i & 1
-        if i + 1 < args.steps:
-            with torch.cuda.stream(copy_stream):
-                if i > 0:
-                    copy_stream.wait_event(read_back[cur ^ 1])       # step i-1, the last user of that buffer, is done
-                stages[cur ^ 1].copy_(host_img, non_blocking=True)
-                copied[cur ^ 1].record(copy_stream)
-        stream.wait_event(copied[cur])
-        loss, _ = eng.train_step(stages[cur], lab, tid, want_kept=False, out=out)
-        host_losses[cur].copy_(loss, non_blocking=True)
-        read_back[cur].record(stream)
-        if i > 0:                                         # the host reads every loss, one step behind the launches
-            read_back[cur ^ 1].synchronize()
+        host_step(cur)
+        done[cur].record(stream)
+        if i > 0:
+            done[cur ^ 1].synchronize()
             e2e_losses.append(float(host_losses[cur ^ 1][0]))
-    read_back[(args.steps - 1) & 1].synchronize()
+    done[(args.steps - 1) & 1].synchronize()
     e2e_losses.append(float(host_losses[(args.steps - 1) & 1][0]))
     f1.record(stream)
     barrier()
     ms_e2e = f0.elapsed_time(f1)
+    h2d_bytes = int(host_img.numel() * host_img.element_size() + host_lab.numel() * 4 + (host_tid.numel() * 4 if host_tid is not None else 0))
 
     # ---- dominant kernel (tcgen05 GEMM): every launch bracketed by CUDA events ---------------------
     eng.profile_enable(True)
     for _ in range(min(args.steps, 5)):
-        eng.train_step(dev_img, lab, tid, want_kept=False, out=out)
+        step(dev_img, out)
     prof = eng.profile_read()
     eng.profile_enable(False)
     eng.sync_status()
@@ -295,29 +350,52 @@ def main():
         pk = peaks()
         fp = eng.footprint()
         flops = step_flops(cfg, cfg.batch)
+        flops_exec = step_flops(cfg, cfg.batch, executed=True)
+        nbytes = step_bytes(cfg, cfg.batch, fp)
+        n_prof = max(1, min(args.steps, 5))
         gemm_tflops = prof["gemm_flops"] / (prof["gemm_ms"] * 1e-3) / 1e12 if prof["gemm_ms"] > 0 else 0.0
+        # The denominator is the measured burst peak (a cuBLAS GEMM timed alone), the stricter of the two measured
+        # figures, whatever the clocks did: under the 1 kW cap a long run of steps settles nearer the sustained figure,
+        # which is given beside it.
+        t_flops_ms = flops / (pk["tflops_burst"] * 1e12) * 1e3
+        t_bytes_ms = nbytes / (pk["hbm_gbs"] * 1e9) * 1e3
+        t_roof_ms = max(t_flops_ms, t_bytes_ms)
+        traffic = GEMM_DRAM_BYTES_PER_LAUNCH.get(cfg.name)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": cfg.name, "global_batch": world * cfg.batch, "tokens": cfg.num_patches + 1,
                        "trainable_blocks": list(cfg.trainable), "drop_blocks": list(cfg.drop_blocks),
-                       "keep_rate": cfg.keep_num / cfg.keep_den, "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                       "keep_rate": cfg.keep_num / cfg.keep_den,
+                       "parallelism": (f"data parallel x{world}: one NCCL all-reduce (mean) of the {fp['trainable_params']} trainable gradients per step"
+                                       if dp else (f"replicas x{world}" if world > 1 else "single GPU")),
                        "l2": "no flush: weights (172 MB) plus per-step activations (> 1 GB) exceed the 126 MB L2"},
             "clocks": {k: clocks.get(k) for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples")},
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(host_img.numel() * host_img.element_size()),
-                    "d2h_bytes_per_step": 4},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": 4,
+                    "api": ("bsr_forward_backward + all-reduce + bsr_optimizer_step around torch host copies" if dp
+                            else "bsr_train_step_host (host buffers in, loss to host memory)")},
             "gpu_launches": int(launches),
+            # the dominant kernel: all tcgen05 GEMM launches of a step, each bracketed by CUDA events on the launching stream
             "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel (tcgen05 bf16 GEMM, all launches of a step)",
-                         "achieved": gemm_tflops, "peak": pk["tflops"], "unit": "TFLOP/s",
-                         "frac": gemm_tflops / pk["tflops"], "traffic": None, "peak_source": pk["source"] + " (sustained)",
-                         "gemm_ms_per_step": prof["gemm_ms"] / max(1, min(args.steps, 5)),
-                         "gemm_launches_per_step": prof["gemm_launches"] / max(1, min(args.steps, 5))},
+                         "achieved": gemm_tflops, "peak": pk["tflops_burst"], "unit": "TFLOP/s",
+                         "frac": gemm_tflops / pk["tflops_burst"], "traffic": traffic,
+                         "peak_source": pk["source"] + " burst (cuBLAS bf16 GEMM timed alone); sustained " + f"{pk['tflops']:.0f}",
+                         "frac_of_sustained": gemm_tflops / pk["tflops"],
+                         "gemm_ms_per_step": prof["gemm_ms"] / n_prof, "gemm_launches_per_step": prof["gemm_launches"] / n_prof,
+                         "gemm_flops_per_step": prof["gemm_flops"] / n_prof},
+            # the whole step against the slower of its FLOPs at the tensor peak and its bytes at the HBM peak
+            "step_roofline": {"bound": "tensor" if t_flops_ms >= t_bytes_ms else "hbm", "step_flops": flops, "executed_flops": flops_exec,
+                              "step_bytes": nbytes, "t_flops_ms": t_flops_ms, "t_bytes_ms": t_bytes_ms, "peak_tflops": pk["tflops_burst"],
+                              "peak_hbm_gbs": pk["hbm_gbs"], "frac": t_roof_ms / ms_step,
+                              "frac_of_sustained": max(flops / (pk["tflops"] * 1e12) * 1e3, t_bytes_ms) / ms_step,
+                              "frac_executed": flops_exec / (pk["tflops_burst"] * 1e12) * 1e3 / ms_step},
             "footprint_bytes": {k: fp[k] for k in ("workspace_bytes", "weight_bytes", "master_bytes", "optimizer_bytes", "grad_bytes",
                                                    "saved_activation_bytes", "scratch_bytes", "paper_activation_bytes")},
             "step_flops": flops,
+            "executed_flops": flops_exec,
             "step_tflops": flops / (ms_step * 1e-3) / 1e12,
-            "step_roofline_frac": flops / (ms_step * 1e-3) / 1e12 / pk["tflops_burst"],
+            "step_roofline_frac": t_roof_ms / ms_step,
         }
         if world == 1 and not args.no_cpu_baseline:
             n_ref = min(cfg.batch, args.ref_batch)

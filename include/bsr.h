@@ -46,11 +46,15 @@ typedef enum {
   BSR_ERR_WORKSPACE_TOO_SMALL = -3,
   BSR_ERR_CUDA = -4,                /* a CUDA runtime/driver call failed; see bsr_last_error */
   BSR_ERR_DEVICE_TIMEOUT = -5,      /* a bounded device-side wait gave up (reported by bsr_sync_status) */
-  BSR_ERR_NONFINITE = -6            /* loss was not finite (reported by bsr_sync_status) */
+  BSR_ERR_NONFINITE = -6,           /* loss was not finite (reported by bsr_sync_status) */
+  BSR_ERR_MEMORY_GUARD = -7,        /* a guard word between two workspace slices was overwritten (bsr_sync_status) */
+  BSR_ERR_DEVICE_CHECK = -8         /* an index check of the checked build (-DBSR_DEBUG) failed (bsr_sync_status) */
 } bsr_status;
 
 enum { BSR_DTYPE_FP32 = 0, BSR_DTYPE_BF16 = 1 };
-enum { BSR_FUSE_NONE = 0, BSR_FUSE_WEIGHTED_SUM = 1 };
+/* What becomes of the dropped tokens (Section 4.1: "fused"): nothing, one extra token sum_j s_j x'_j weighted by the
+ * head-mean scores, or that sum divided by sum_j s_j (the weighted mean). */
+enum { BSR_FUSE_NONE = 0, BSR_FUSE_WEIGHTED_SUM = 1, BSR_FUSE_WEIGHTED_MEAN = 2 };
 enum { BSR_OPT_ADAMW = 0, BSR_OPT_SGD = 1 };
 enum { BSR_MAX_DROPS = 8, BSR_MAX_TASKS = 4, BSR_MAX_DEPTH = 32 };
 
@@ -96,6 +100,8 @@ typedef struct {
   uint64_t scratch_bytes;           /* forward/backward scratch shared by all blocks */
   uint64_t paper_activation_bytes;  /* the same blocks in the paper's fp32 accounting (Table 1), at max_batch */
   uint64_t trainable_params;
+  uint64_t block_saved_bytes[BSR_MAX_DEPTH]; /* per block, its share of saved_activation_bytes (0 before the earliest
+                                               trainable block); the earliest one also holds the fp32 input of the path */
 } bsr_footprint;
 
 typedef struct bsr_handle bsr_handle;
@@ -184,6 +190,23 @@ int32_t bsr_train_steps(bsr_handle* h, const void* images_dev, const int32_t* la
                         int32_t batch, int32_t n_steps, const bsr_lr_schedule* schedule_host, void* stream,
                         float* loss_dev_out, int32_t* kept_idx_dev_out);
 
+/* Data-parallel training over several GPUs (one process and one handle per GPU, each with its share of the batch):
+ * bsr_train_step in two halves with the caller's gradient exchange between them.  The images of a batch are independent
+ * up to the batch-mean loss, so the only coupling between the shares is the mean of their gradients:
+ *   bsr_forward_backward  forward, loss and backward of this GPU's share; the gradients of the local mean loss are
+ *                         left in the gradient buffer, nothing is updated (arguments as for bsr_train_step);
+ *   bsr_grad_buffer       the gradient buffer: `count` float32 values holding every trainable tensor (each padded to
+ *                         a multiple of 64 values, padding zero).  Average it over the GPUs in place on the same
+ *                         stream -- one all-reduce (NCCL over NVLink), equal shares assumed -- and every GPU holds
+ *                         the gradient of the global batch mean;
+ *   bsr_optimizer_step    AdamW / SGD on the buffer as it stands, with the bias corrections of the next step; advances
+ *                         the step counter.
+ * On one GPU the three calls equal bsr_train_step bit for bit.  The library itself never communicates. */
+int32_t bsr_forward_backward(bsr_handle* h, const void* images_dev, const int32_t* labels_dev, const int32_t* task_ids_dev,
+                             int32_t batch, void* stream, float* loss_dev_out, int32_t* kept_idx_dev_out);
+int32_t bsr_grad_buffer(bsr_handle* h, float** grads_dev_out_host, size_t* count_out_host);
+int32_t bsr_optimizer_step(bsr_handle* h, void* stream);
+
 /* bsr_train_step fed from and read back into HOST memory (the same step; Fig. 2).  images_host, labels_host and
  * task_ids_host are copied into one of two staging slots inside the workspace on a copy stream the library owns, so
  * that the copy for this step overlaps the kernels of the previous one; the step runs on `stream`; the loss (and, if
@@ -202,8 +225,11 @@ int32_t bsr_eval_forward(bsr_handle* h, const void* images_dev, const int32_t* t
 /* Memory report (Section 3.2, Table 1: activations dominate training memory). Host-only. */
 int32_t bsr_get_footprint(const bsr_handle* h, bsr_footprint* out_host);
 
-/* Synchronises `stream` and reads the device status word: BSR_OK, BSR_ERR_DEVICE_TIMEOUT if a
- * bounded wait in a kernel expired, BSR_ERR_NONFINITE if the last loss was not finite.  Clears it. */
+/* Checks the guard words that follow every slice of the workspace (weights, optimiser state, each saved activation,
+ * each scratch buffer), synchronises `stream` and reads the device status word: BSR_OK, BSR_ERR_DEVICE_TIMEOUT if a
+ * bounded wait in a kernel expired, BSR_ERR_MEMORY_GUARD if a kernel wrote past the end of its slice,
+ * BSR_ERR_DEVICE_CHECK if an index check of the checked build failed, BSR_ERR_NONFINITE if the last loss was not
+ * finite.  Clears the status word (an overwritten guard stays overwritten and is reported again). */
 int32_t bsr_sync_status(bsr_handle* h, void* stream);
 
 /* Diagnostic of the failure path (no counterpart in the paper).  Every device-side wait of the tensor-core kernels
@@ -262,9 +288,10 @@ int32_t bsr_token_select(const float* p_dev, int32_t batch, int32_t heads, int32
 
 /* Compaction between MHSA and FFN (Section 4.1: kept tokens preserved, the others fused).
  * x_dev [batch, 1+m, dim] in `dtype`; out_dev [batch, 1+k+f, dim] with f = 1 when
- * fuse_mode == BSR_FUSE_WEIGHTED_SUM and k < m, else 0.  Row 0 is copied, rows 1..k are the kept
+ * fuse_mode != BSR_FUSE_NONE and k < m, else 0.  Row 0 is copied, rows 1..k are the kept
  * rows in the order of kept_dev, the last row is sum_j scores[b, j] * x[b, 1+j] over dropped j
- * (float32 accumulation in a fixed order).  dim * sizeof(dtype) must be a multiple of 16. */
+ * (float32 accumulation in a fixed order), divided by sum_j scores[b, j] for BSR_FUSE_WEIGHTED_MEAN.
+ * dim * sizeof(dtype) must be a multiple of 16. */
 int32_t bsr_gather_fuse(const void* x_dev, int32_t dtype, int32_t batch, int32_t m, int32_t dim, int32_t k,
                         const int32_t* kept_dev, const int32_t* dropped_dev, const float* scores_dev,
                         int32_t fuse_mode, void* out_dev, void* stream);

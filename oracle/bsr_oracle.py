@@ -25,7 +25,8 @@ What it follows, passage by passage:
 Readings where the paper is silent:
   score = post-softmax CLS row averaged over heads; CLS itself is not a candidate;
   K = ceil(keep * M) in integer arithmetic; kept tokens stay in ascending position and the
-  fused token goes last; fused token = sum_j s_j x'_j over the dropped tokens; keep = 1
+  fused token goes last; fused token = sum_j s_j x'_j over the dropped tokens (fuse_mode 1), or that
+  sum divided by sum_j s_j (fuse_mode 2, the weighted mean: the other natural reading of "fused"); keep = 1
   appends nothing; ties go to the lower index; the index sets are constants for the
   backward pass while the fusion weights s_j are differentiated; final LayerNorm and head
   train with the chosen blocks; weight decay on matrices only.
@@ -70,7 +71,7 @@ def token_schedule(cfg):
             m = t - 1
             k = keep_count(m, cfg.keep_num, cfg.keep_den)
             if k < m:
-                t = 1 + k + (1 if cfg.fuse_mode == 1 else 0)
+                t = 1 + k + (1 if cfg.fuse_mode in (1, 2) else 0)
         out.append((ta, t, k))
     return out
 
@@ -307,10 +308,15 @@ def block_fwd(cfg, params, l, x, task_ids, k, forced_keep, forced_experts=None):
         info = {"kept": kept, "dropped": dropped, "scores": s, "margins": margins}
         if k < m:
             rows = [xp[:, :1], np.take_along_axis(xp[:, 1:], kept[:, :, None], axis=1)]
-            if cfg.fuse_mode == 1:
+            if cfg.fuse_mode in (1, 2):
                 xd = np.take_along_axis(xp[:, 1:], dropped[:, :, None], axis=1)
                 sd = np.take_along_axis(s, dropped, axis=1)
-                rows.append((sd[:, :, None] * xd).sum(axis=1, keepdims=True))
+                fused = (sd[:, :, None] * xd).sum(axis=1, keepdims=True)
+                if cfg.fuse_mode == 2:                          # weighted mean: the weights are normalised to sum to one
+                    c["ssum"] = sd.sum(axis=1)
+                    fused = fused / c["ssum"][:, None, None]
+                    c["fused"] = fused[:, 0]
+                rows.append(fused)
                 c["xd"], c["sd"] = xd, sd
             c["xp_full_shape"] = xp.shape
             xp = np.concatenate(rows, axis=1)
@@ -349,10 +355,15 @@ def block_bwd(cfg, params, l, dout, c, task_ids, grads, want_param_grads, need_d
         full[:, 0] = dxp[:, 0]
         bidx = np.arange(B)[:, None]
         full[bidx, 1 + kept] = dxp[:, 1 : 1 + kk]
-        if cfg.fuse_mode == 1:
+        if cfg.fuse_mode in (1, 2):
             gf = dxp[:, 1 + kk]                                        # gradient of the fused token
-            full[bidx, 1 + dropped] = c["sd"][:, :, None] * gf[:, None, :]
-            ds = (c["xd"] * gf[:, None, :]).sum(axis=-1)               # dL/ds_j for dropped j
+            ds = (c["xd"] * gf[:, None, :]).sum(axis=-1)               # dL/ds_j for dropped j (weighted sum)
+            wj = c["sd"]
+            if cfg.fuse_mode == 2:                                     # f = u / S, u = sum_j s_j x_j, S = sum_j s_j:
+                S = c["ssum"][:, None]                                 # df/dx_j = s_j / S, df/ds_j = (x_j - f) / S
+                ds = (ds - (c["fused"] * gf).sum(axis=-1)[:, None]) / S
+                wj = wj / S
+            full[bidx, 1 + dropped] = wj[:, :, None] * gf[:, None, :]
             dA_cls = np.zeros((B, T))
             dA_cls[bidx, 1 + dropped] = ds / cfg.heads                 # every head gets 1/H of it
         dxp = full
@@ -528,8 +539,9 @@ def train_step(cfg, params, images, labels, task_ids=None, forced_keep=None, opt
 def gather_fuse(xp, kept, dropped, s, fuse_mode=1):
     """Stand-alone compaction of one batch: xp [B, 1+M, D], index lists per image, scores s [B, M]."""
     rows = [xp[:, :1], np.take_along_axis(xp[:, 1:], kept[:, :, None], axis=1)]
-    if fuse_mode == 1 and dropped.shape[1] > 0:
+    if fuse_mode in (1, 2) and dropped.shape[1] > 0:
         xd = np.take_along_axis(xp[:, 1:], dropped[:, :, None], axis=1)
         sd = np.take_along_axis(s, dropped, axis=1)
-        rows.append((sd[:, :, None] * xd).sum(axis=1, keepdims=True))
+        fused = (sd[:, :, None] * xd).sum(axis=1, keepdims=True)
+        rows.append(fused / sd.sum(axis=1)[:, None, None] if fuse_mode == 2 else fused)
     return np.concatenate(rows, axis=1)

@@ -13,17 +13,19 @@ from typing import Dict, Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libbsr.so")
+# BSR_LIBRARY=checked selects the build with device-side index checks (python -m paper_2405_10951_b200.build --checked)
+LIB_PATH = os.path.join(_HERE, "libbsr_checked.so" if os.environ.get("BSR_LIBRARY") == "checked" else "libbsr.so")
 
 BSR_OK = 0
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 MAX_DROPS, MAX_TASKS, MAX_DEPTH = 8, 4, 32
 
 STATUS_NAMES = {0: "BSR_OK", -1: "BSR_ERR_INVALID_ARG", -2: "BSR_ERR_UNSUPPORTED", -3: "BSR_ERR_WORKSPACE_TOO_SMALL",
-                -4: "BSR_ERR_CUDA", -5: "BSR_ERR_DEVICE_TIMEOUT", -6: "BSR_ERR_NONFINITE"}
+                -4: "BSR_ERR_CUDA", -5: "BSR_ERR_DEVICE_TIMEOUT", -6: "BSR_ERR_NONFINITE", -7: "BSR_ERR_MEMORY_GUARD",
+                -8: "BSR_ERR_DEVICE_CHECK"}
 
 EXPORTS = ["bsr_token_schedule", "bsr_workspace_bytes", "bsr_create", "bsr_destroy", "bsr_last_error", "bsr_set_param",
-           "bsr_get_tensor", "bsr_set_lr", "bsr_set_step", "bsr_train_step", "bsr_train_steps", "bsr_train_step_host", "bsr_eval_forward", "bsr_get_footprint",
+           "bsr_get_tensor", "bsr_set_lr", "bsr_set_step", "bsr_train_step", "bsr_train_steps", "bsr_train_step_host", "bsr_forward_backward", "bsr_grad_buffer", "bsr_optimizer_step", "bsr_eval_forward", "bsr_get_footprint",
            "bsr_sync_status", "bsr_selftest_wait_expiry", "bsr_set_gemm_mode", "bsr_set_graph_mode", "bsr_profile_enable", "bsr_profile_read", "bsr_profile_launches", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_backward",
            "bsr_linear_backward_static", "bsr_static_last_error", "bsr_attention_forward"]
 
@@ -47,7 +49,7 @@ class bsr_config(C.Structure):
 class bsr_footprint(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in ("workspace_bytes", "weight_bytes", "master_bytes", "optimizer_bytes",
                                            "grad_bytes", "saved_activation_bytes", "scratch_bytes",
-                                           "paper_activation_bytes", "trainable_params")]
+                                           "paper_activation_bytes", "trainable_params")] + [("block_saved_bytes", C.c_uint64 * MAX_DEPTH)]
 
 
 class bsr_profile(C.Structure):
@@ -91,6 +93,9 @@ def lib() -> C.CDLL:
         L.bsr_train_step.argtypes = [vp, vp, i32p, i32p, i32, vp, f32p, i32p]
         L.bsr_train_steps.argtypes = [vp, vp, i32p, i32p, i32, i32, C.POINTER(bsr_lr_schedule), vp, f32p, i32p]
         L.bsr_train_step_host.argtypes = [vp, vp, i32p, i32p, i32, vp, f32p, i32p]
+        L.bsr_forward_backward.argtypes = [vp, vp, i32p, i32p, i32, vp, f32p, i32p]
+        L.bsr_grad_buffer.argtypes = [vp, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
+        L.bsr_optimizer_step.argtypes = [vp, vp]
         L.bsr_eval_forward.argtypes = [vp, vp, i32p, i32, vp, f32p, i32p]
         L.bsr_get_footprint.argtypes = [vp, C.POINTER(bsr_footprint)]
         L.bsr_sync_status.argtypes = [vp, vp]
@@ -184,7 +189,7 @@ def bsr_gather_fuse(x, kept, dropped, scores, fuse_mode: int = 1, out=None):
     import torch
     B, T, D = x.shape
     M, k = T - 1, kept.shape[1]
-    f = 1 if (fuse_mode == 1 and k < M) else 0
+    f = 1 if (fuse_mode in (1, 2) and k < M) else 0
     if out is None:
         out = torch.empty((B, 1 + k + f, D), dtype=x.dtype, device=x.device)
     dt = DTYPE_FP32 if x.dtype == torch.float32 else DTYPE_BF16
@@ -347,6 +352,29 @@ class Engine:
         self.last_out = (losses, kept)
         return losses, self._split_kept(kept, B)
 
+    def forward_backward(self, images, labels, task_ids=None, want_kept: bool = True, out=None):
+        """The step without its update: gradients of the local batch mean are left in the gradient buffer."""
+        torch = self.torch
+        B = images.shape[0]
+        if out is not None:
+            loss, kept = out
+        else:
+            loss = torch.empty(1, dtype=torch.float32, device=self.device)
+            kept = torch.empty(B * sum(self.kept_counts), dtype=torch.int32, device=self.device) if (want_kept and self.kept_counts) else None
+        _check(lib().bsr_forward_backward(self.h, _ptr(images), _ptr(labels), _ptr(task_ids), B, _stream(), _ptr(loss), _ptr(kept)), self.h)
+        self.last_out = (loss, kept)
+        return loss, self._split_kept(kept, B)
+
+    def grad_buffer(self):
+        """The flat float32 gradient buffer as a tensor view of the workspace (to be all-reduced in place)."""
+        p, n = C.c_void_p(), C.c_size_t()
+        _check(lib().bsr_grad_buffer(self.h, C.byref(p), C.byref(n)), self.h)
+        off = p.value - self.workspace.data_ptr()
+        return self.workspace[off: off + 4 * n.value].view(self.torch.float32)
+
+    def optimizer_step(self):
+        _check(lib().bsr_optimizer_step(self.h, _stream()), self.h)
+
     def train_step_host(self, images, labels, task_ids=None, loss=None, kept=None):
         """images / labels / task_ids / loss / kept: CPU tensors (pinned for overlap); images in the storage dtype.
         Does not synchronise: `loss` holds the step's loss once the current stream has finished this call's work."""
@@ -406,4 +434,6 @@ class Engine:
     def footprint(self) -> Dict[str, int]:
         fp = bsr_footprint()
         _check(lib().bsr_get_footprint(self.h, C.byref(fp)), self.h)
-        return {n: int(getattr(fp, n)) for n, _ in bsr_footprint._fields_}
+        out = {n: int(getattr(fp, n)) for n, _ in bsr_footprint._fields_ if n != "block_saved_bytes"}
+        out["block_saved_bytes"] = [int(x) for x in fp.block_saved_bytes[: self.cfg.depth]]
+        return out

@@ -317,4 +317,183 @@ int attention_bwd(const Ctx& c, const void* qkv, const void* out, const void* do
                       : launch_bwd<bf16>(c, qkv, dout, lse, delta, cls_extra, dqkv, B, T_, H, d);
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Classification row only.  In the last block nothing but the classification token's output is ever read (the head
+// takes row 0), so its attention reduces to one query per (image, head): o_0 = sum_j p_j v_j with p = softmax(q_0 K^T
+// / sqrt(d)) (Eq. 1, first row), and in the backward pass only that row carries a gradient: dV_j = p_j dO_0,
+// dS_j = p_j (dO_0 . v_j - sum_i p_i dO_0 . v_i), dK_j = dS_j q_0 / sqrt(d), dQ_0 = sum_j dS_j k_j / sqrt(d), every
+// other row of dQ is zero.  One warp per (image, head); the probabilities are recomputed in the backward kernel.
+// ---------------------------------------------------------------------------------------------
+constexpr int ATC_WARPS = 4;
+constexpr int ATC_MAXKEYS = 32 * 20;             // keys per lane held in registers: up to 640 tokens
+
+template <typename T> __device__ __forceinline__ float2 ld_pair(const T* p);
+template <> __device__ __forceinline__ float2 ld_pair<float>(const float* p) { return *reinterpret_cast<const float2*>(p); }
+template <> __device__ __forceinline__ float2 ld_pair<bf16>(const bf16* p) { return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p)); }
+template <typename T> __device__ __forceinline__ void st_pair(T* p, float a, float b);
+template <> __device__ __forceinline__ void st_pair<float>(float* p, float a, float b) { *reinterpret_cast<float2*>(p) = make_float2(a, b); }
+template <> __device__ __forceinline__ void st_pair<bf16>(bf16* p, float a, float b) { *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(a, b); }
+
+// Softmax row of the classification query of one (image, head), lanes striding the keys: p[i] belongs to key lane + 32 i.
+// vec: the query (d floats in shared memory).  Returns through p the probabilities.
+template <typename T, int KPL>
+__device__ __forceinline__ void cls_row_probs(const T* kbase, long row_stride, const float* vec, int T_, int d, float scale, int lane,
+                                              float* p) {
+  float mx = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < KPL; ++i) {
+    int j = lane + 32 * i;
+    p[i] = -INFINITY;
+    if (j < T_) {
+      const T* row = kbase + (long)j * row_stride;
+      float s = 0.f;
+      for (int e = 0; e < d; e += 2) {
+        float2 kv = ld_pair<T>(row + e);
+        s = fmaf(vec[e], kv.x, s);
+        s = fmaf(vec[e + 1], kv.y, s);
+      }
+      p[i] = s * scale;
+      mx = fmaxf(mx, p[i]);
+    }
+  }
+  mx = warp_max(mx);
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < KPL; ++i) {
+    p[i] = (lane + 32 * i < T_) ? expf(p[i] - mx) : 0.f;
+    sum += p[i];
+  }
+  sum = warp_sum(sum);
+  float inv = 1.0f / sum;
+#pragma unroll
+  for (int i = 0; i < KPL; ++i) p[i] *= inv;
+}
+
+template <typename T, int KPL>
+__global__ void __launch_bounds__(ATC_WARPS * 32)
+attn_cls_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ out_cls, int B, int T_, int H, int d) {
+  __shared__ float qs[ATC_WARPS][AT_MAXD];
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int pair = blockIdx.x * ATC_WARPS + warp;
+  if (pair >= B * H) return;
+  int b = pair / H, h = pair % H;
+  long row_stride = 3L * H * d;
+  const T* base = qkv + (long)b * T_ * row_stride + (long)h * d;
+  if (2 * lane < d) {
+    float2 q = ld_pair<T>(base + 2 * lane);
+    qs[warp][2 * lane] = q.x; qs[warp][2 * lane + 1] = q.y;
+  }
+  __syncwarp();
+  float p[KPL];
+  cls_row_probs<T, KPL>(base + (long)H * d, row_stride, qs[warp], T_, d, rsqrtf((float)d), lane, p);
+  // o_0 = sum_j p_j v_j: every lane owns two feature indices, the keys are walked in order
+  float o0 = 0.f, o1 = 0.f;
+  const T* vbase = base + 2L * H * d;
+#pragma unroll
+  for (int i = 0; i < KPL; ++i) {
+    for (int l = 0; l < 32; ++l) {
+      int j = l + 32 * i;
+      if (j >= T_) break;
+      float pj = __shfl_sync(0xffffffffu, p[i], l);
+      if (2 * lane < d) {
+        float2 v = ld_pair<T>(vbase + (long)j * row_stride + 2 * lane);
+        o0 = fmaf(pj, v.x, o0); o1 = fmaf(pj, v.y, o1);
+      }
+    }
+  }
+  if (2 * lane < d) st_pair<T>(out_cls + (long)b * H * d + (long)h * d + 2 * lane, o0, o1);
+}
+
+template <typename T, int KPL>
+__global__ void __launch_bounds__(ATC_WARPS * 32)
+attn_cls_bwd_kernel(const T* __restrict__ qkv, const T* __restrict__ dout_cls, T* __restrict__ dqkv, int B, int T_, int H, int d) {
+  __shared__ float qs[ATC_WARPS][AT_MAXD], gs[ATC_WARPS][AT_MAXD];
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int pair = blockIdx.x * ATC_WARPS + warp;
+  if (pair >= B * H) return;
+  int b = pair / H, h = pair % H;
+  long row_stride = 3L * H * d;
+  const T* base = qkv + (long)b * T_ * row_stride + (long)h * d;
+  T* dbase = dqkv + (long)b * T_ * row_stride + (long)h * d;
+  float q0 = 0.f, q1 = 0.f, g0 = 0.f, g1 = 0.f;
+  if (2 * lane < d) {
+    float2 q = ld_pair<T>(base + 2 * lane);
+    float2 g = ld_pair<T>(dout_cls + (long)b * H * d + (long)h * d + 2 * lane);
+    q0 = q.x; q1 = q.y; g0 = g.x; g1 = g.y;
+    qs[warp][2 * lane] = q0; qs[warp][2 * lane + 1] = q1;
+    gs[warp][2 * lane] = g0; gs[warp][2 * lane + 1] = g1;
+  }
+  __syncwarp();
+  float scale = rsqrtf((float)d);
+  float p[KPL], ds[KPL];
+  cls_row_probs<T, KPL>(base + (long)H * d, row_stride, qs[warp], T_, d, scale, lane, p);
+  // dP_j = dO_0 . v_j for the lane's keys, delta = sum_j p_j dP_j
+  const T* vbase = base + 2L * H * d;
+  float delta = 0.f;
+#pragma unroll
+  for (int i = 0; i < KPL; ++i) {
+    int j = lane + 32 * i;
+    ds[i] = 0.f;
+    if (j < T_) {
+      const T* row = vbase + (long)j * row_stride;
+      float s = 0.f;
+      for (int e = 0; e < d; e += 2) {
+        float2 v = ld_pair<T>(row + e);
+        s = fmaf(gs[warp][e], v.x, s);
+        s = fmaf(gs[warp][e + 1], v.y, s);
+      }
+      ds[i] = s;
+      delta += p[i] * s;
+    }
+  }
+  delta = warp_sum(delta);
+#pragma unroll
+  for (int i = 0; i < KPL; ++i) ds[i] = p[i] * (ds[i] - delta) * scale;      // dS_j / sqrt(d)
+  // rows: dV_j = p_j dO_0, dK_j = dS_j q_0 / sqrt(d), dQ_0 = sum_j dS_j k_j / sqrt(d), dQ_j = 0 for j > 0
+  float dq0 = 0.f, dq1 = 0.f;
+  const T* kbase = base + (long)H * d;
+#pragma unroll
+  for (int i = 0; i < KPL; ++i) {
+    for (int l = 0; l < 32; ++l) {
+      int j = l + 32 * i;
+      if (j >= T_) break;
+      float pj = __shfl_sync(0xffffffffu, p[i], l);
+      float dsj = __shfl_sync(0xffffffffu, ds[i], l);
+      if (2 * lane < d) {
+        float2 k = ld_pair<T>(kbase + (long)j * row_stride + 2 * lane);
+        dq0 = fmaf(dsj, k.x, dq0); dq1 = fmaf(dsj, k.y, dq1);
+        T* drow = dbase + (long)j * row_stride + 2 * lane;
+        st_pair<T>(drow + (long)H * d, dsj * q0, dsj * q1);
+        st_pair<T>(drow + 2L * H * d, pj * g0, pj * g1);
+        if (j > 0) st_pair<T>(drow, 0.f, 0.f);
+      }
+    }
+  }
+  if (2 * lane < d) st_pair<T>(dbase + 2 * lane, dq0, dq1);
+}
+
+template <typename T>
+static int launch_cls(const Ctx& c, bool bwd, const void* qkv, const void* io_cls, void* dqkv, int B, int T_, int H, int d) {
+  if (d > AT_MAXD || (d % 2) != 0 || T_ < 1 || T_ > ATC_MAXKEYS) return -2;
+  int blocks = ceil_div((long)B * H, ATC_WARPS);
+  note_launch(1);
+#define BSR_CLS(KPL)                                                                                                              \
+  do {                                                                                                                            \
+    if (bwd) attn_cls_bwd_kernel<T, KPL><<<blocks, ATC_WARPS * 32, 0, c.stream>>>((const T*)qkv, (const T*)io_cls, (T*)dqkv, B, T_, H, d); \
+    else attn_cls_fwd_kernel<T, KPL><<<blocks, ATC_WARPS * 32, 0, c.stream>>>((const T*)qkv, (T*)const_cast<void*>(io_cls), B, T_, H, d);  \
+  } while (0)
+  int kpl = ceil_div(T_, 32);
+  if (kpl <= 3) BSR_CLS(3); else if (kpl <= 5) BSR_CLS(5); else if (kpl <= 7) BSR_CLS(7); else if (kpl <= 10) BSR_CLS(10); else BSR_CLS(20);
+#undef BSR_CLS
+  return 0;
+}
+
+int attention_cls_fwd(const Ctx& c, const void* qkv, void* out_cls, int B, int T_, int H, int d) {
+  return c.dtype == 0 ? launch_cls<float>(c, false, qkv, out_cls, nullptr, B, T_, H, d) : launch_cls<bf16>(c, false, qkv, out_cls, nullptr, B, T_, H, d);
+}
+int attention_cls_bwd(const Ctx& c, const void* qkv, const void* dout_cls, void* dqkv, int B, int T_, int H, int d) {
+  return c.dtype == 0 ? launch_cls<float>(c, true, qkv, dout_cls, dqkv, B, T_, H, d) : launch_cls<bf16>(c, true, qkv, dout_cls, dqkv, B, T_, H, d);
+}
+
 }  // namespace bsr

@@ -10,7 +10,16 @@ namespace bsr {
 typedef __nv_bfloat16 bf16;
 
 // Device status word bits (read and cleared by bsr_sync_status).
-enum : int { STATUS_TIMEOUT = 1, STATUS_NONFINITE = 2 };
+enum : int { STATUS_TIMEOUT = 1, STATUS_NONFINITE = 2, STATUS_GUARD = 4, STATUS_CHECK = 8 };
+
+// Index checks of the checked build (-DBSR_DEBUG): a failed check raises STATUS_CHECK in the status word (never a trap:
+// the context stays usable) and the caller of the macro skips the access.  In the normal build the condition is not
+// evaluated.
+#ifdef BSR_DEBUG
+#define BSR_CHECK(cond, status) ((cond) ? true : (((status) != nullptr ? (void)atomicOr((status), bsr::STATUS_CHECK) : (void)0), false))
+#else
+#define BSR_CHECK(cond, status) (true)
+#endif
 
 template <typename T> struct Pack;          // 16-byte vector of storage elements
 template <> struct Pack<float> { static constexpr int N = 4; };

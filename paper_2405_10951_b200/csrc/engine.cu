@@ -44,11 +44,19 @@ struct BlockBufs {          // byte offsets into the workspace; filled for froze
   size_t m_eidx, m_ew, m_pos, m_row_token, m_row_w, m_seg, m_tile, m_cnt, m_off, m_xg, m_zg, m_hg, m_og;
 };
 
+// Carves the workspace.  Every slice is followed by a guard of GUARD_BYTES holding a fixed pattern; bsr_sync_status
+// checks the guards, so a kernel that writes past the end of its slice is reported instead of silently corrupting the
+// neighbour (the stand-in for a memory checker).
+constexpr size_t GUARD_BYTES = 256;
+constexpr uint32_t GUARD_WORD = 0xC5A3C5A3u;
 struct Bump {
   size_t off = 0;
+  std::vector<size_t>* guards = nullptr;
   size_t take(size_t bytes) {
     size_t o = off;
     off += (bytes + 255) & ~(size_t)255;
+    if (guards != nullptr) guards->push_back(off);
+    off += GUARD_BYTES;
     return o;
   }
 };
@@ -86,7 +94,7 @@ int compute_schedule(const bsr_config* cfg, Schedule* s, char* err) {
       if (k < 1) k = 1;
       if (k > m) k = m;
       s->k[l] = (int)k;
-      if (k < m) t = 1 + (int)k + (cfg->fuse_mode == BSR_FUSE_WEIGHTED_SUM ? 1 : 0);
+      if (k < m) t = 1 + (int)k + (cfg->fuse_mode != BSR_FUSE_NONE ? 1 : 0);
       ++di;
     }
     s->tf[l] = t;
@@ -107,7 +115,8 @@ int validate(const bsr_config* cfg, char* err) {
   for (int t = 0; t < d.num_tasks; ++t)
     if (d.num_classes[t] < 1) return set_err(err, BSR_ERR_INVALID_ARG, "num_classes must be positive");
   if (cfg->max_batch < 1) return set_err(err, BSR_ERR_INVALID_ARG, "max_batch must be positive");
-  if (cfg->fuse_mode != BSR_FUSE_NONE && cfg->fuse_mode != BSR_FUSE_WEIGHTED_SUM) return set_err(err, BSR_ERR_INVALID_ARG, "unknown fuse_mode");
+  if (cfg->fuse_mode != BSR_FUSE_NONE && cfg->fuse_mode != BSR_FUSE_WEIGHTED_SUM && cfg->fuse_mode != BSR_FUSE_WEIGHTED_MEAN)
+    return set_err(err, BSR_ERR_INVALID_ARG, "unknown fuse_mode");
   if (cfg->optimizer != BSR_OPT_ADAMW && cfg->optimizer != BSR_OPT_SGD) return set_err(err, BSR_ERR_INVALID_ARG, "unknown optimizer");
   if (cfg->optimizer == BSR_OPT_SGD && !(cfg->momentum >= 0.f && cfg->momentum < 1.f)) return set_err(err, BSR_ERR_INVALID_ARG, "momentum must lie in [0, 1)");
   if (!(d.ln_eps > 0.f)) return set_err(err, BSR_ERR_INVALID_ARG, "ln_eps must be positive");
@@ -151,6 +160,7 @@ struct bsr_handle {
   BlockBufs bufs_frozen[2];           // ping-pong by block parity
   size_t off_x_last = 0;
   size_t arena_bytes = 0, scratch_bytes = 0;
+  size_t block_saved_bytes[BSR_MAX_DEPTH] = {};
   // scratch
   size_t off_patches = 0, off_emb = 0;
   size_t off_xn = 0, off_meanf = 0, off_rstdf = 0, off_logits = 0, off_per_image = 0, off_dlogits = 0, off_dxn = 0;
@@ -175,6 +185,8 @@ struct bsr_handle {
   uint64_t graph_captures = 0;        // how many times a step was captured (a pipeline that cycles through more buffers than the cache holds re-captures every step)
   int use_graph = 1;
   // multi-step loop and host-buffer step
+  std::vector<size_t> guards;            // byte offsets of the guard words after every slice
+  size_t off_guard_table = 0;
   size_t off_loop = 0, off_lab_stage = 0, off_task_stage = 0;
   size_t off_host_img[2] = {0, 0}, off_host_lab[2] = {0, 0}, off_host_task[2] = {0, 0}, off_host_loss[2] = {0, 0};
   cudaStream_t copy_stream = nullptr;
@@ -259,6 +271,8 @@ size_t plan(bsr_handle* h) {
   int cmax = 0;
   for (int t = 0; t < d.num_tasks; ++t) cmax = d.num_classes[t] > cmax ? d.num_classes[t] : cmax;
   Bump b;
+  h->guards.clear();
+  b.guards = &h->guards;
   h->off_status = b.take(256);
   h->off_loss = h->off_status + 64;
   // flat trainable arrays
@@ -325,12 +339,19 @@ size_t plan(bsr_handle* h) {
     BlockBufs& bb = h->bufs_train[l];
     size_t Ma = (size_t)Bm * s.ta[l], Mf = (size_t)Bm * s.tf[l];
     bool drop = s.k[l] >= 0 && s.tf[l] != s.ta[l];
+    size_t block0 = b.off;
     bb.x_in = (l == h->t0) ? b.take(Ma * D * 4) : next_in;       // residual stream: float
+    // A trainable block keeps the input of every linear layer (Eq. 4: its weight gradient needs it); a frozen block
+    // inside the gradient path keeps only what passing the gradient on needs (Eq. 2; Section 3.2, Table 1): Q, K, V
+    // with the log-sum-exp, the FFN pre-activation, and the LayerNorm inputs with their statistics.  Its LayerNorm
+    // outputs and attention output live in the scratch the blocks before t0 use.  The GELU output is kept by no block:
+    // the backward pass recomputes it from the pre-activation where the second FFN layer's weight gradient needs it.
+    bool keeps_inputs = (cfg.trainable_mask >> l) & 1u;
     bb.mean1 = b.take(Ma * 4); bb.rstd1 = b.take(Ma * 4);
-    bb.y1 = b.take(Ma * D * es);
+    bb.y1 = keeps_inputs ? b.take(Ma * D * es) : 0;
     bb.qkv = b.take(Ma * 3 * D * es);
     bb.lse = b.take((size_t)Bm * H * s.ta[l] * 4);
-    bb.o = b.take(Ma * D * es);
+    bb.o = keeps_inputs ? b.take(Ma * D * es) : 0;
     bb.xp = b.take(Mf * D * 4);
     bb.xp_full = drop ? b.take(Ma * D * 4) : bb.xp;
     if (s.k[l] >= 0) {
@@ -340,14 +361,16 @@ size_t plan(bsr_handle* h) {
       bb.dropped = b.take((size_t)Bm * (s.ta[l] - 1) * 4);
     }
     bb.mean2 = b.take(Mf * 4); bb.rstd2 = b.take(Mf * 4);
-    bb.y2 = b.take(Mf * D * es);
-    bb.z = b.take(Mf * F * es);
-    bb.hh = b.take(Mf * F * es);
+    bb.y2 = keeps_inputs ? b.take(Mf * D * es) : 0;
+    bool moe = (d.moe_block_mask >> l) & 1u;
+    bb.z = moe ? 0 : b.take(Mf * F * es);
+    bb.hh = 0;
     bb.x_out = b.take(Mf * D * 4);
     bb.o_cls = b.take((size_t)Bm * D * es);
     bb.xin_cls = b.take((size_t)Bm * D * 4);
-    if ((d.moe_block_mask >> l) & 1u) take_moe(bb, l, s.tf[l]);
+    if (moe) take_moe(bb, l, s.tf[l]);
     next_in = bb.x_out;
+    h->block_saved_bytes[l] = b.off - block0;
   }
   h->arena_bytes = b.off - a0;
   // scratch
@@ -383,6 +406,12 @@ size_t plan(bsr_handle* h) {
     h->bufs_frozen[1] = bb;
     h->bufs_frozen[1].x_in = in1;
     h->bufs_frozen[1].x_out = out1;
+    // what the blocks from t0 on do not keep lives in the same scratch
+    for (int l = h->t0; l < d.depth; ++l) {
+      BlockBufs& tb = h->bufs_train[l];
+      tb.hh = bb.hh;
+      if (!((cfg.trainable_mask >> l) & 1u)) { tb.y1 = bb.y1; tb.o = bb.o; tb.y2 = bb.y2; }
+    }
   }
   h->off_xn = b.take((size_t)Bm * D * 4);
   h->off_meanf = b.take((size_t)Bm * 4);
@@ -441,6 +470,9 @@ size_t plan(bsr_handle* h) {
     h->off_host_loss[i] = b.take(256);
   }
   h->scratch_bytes = b.off - s0;
+  // table of the guard offsets, read by the kernels that write and check the guards (it has no guard of its own)
+  b.guards = nullptr;
+  h->off_guard_table = b.take(h->guards.size() * sizeof(unsigned long long));
   return b.off;
 }
 
@@ -621,6 +653,7 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
   GemmEpilogue eg;
   eg.act = 2;
   eg.aux_in = h->base + bb.z;
+  if (pg) eg.aux_out = h->base + bb.hh;       // GELU(z) again, into scratch, for the weight gradient below
   gemm(c, op(dxo), D, 1, h->wb(l, "mlp.fc2.weight"), 1, F, dz, 0, Mf, F, D, eg);
   if (pg) {
     gemm(c, op(dxo), 1, D, h->base + bb.hh, 1, F, h->gb(l, "mlp.fc2.weight"), 1, D, F, Mf, none);
@@ -641,10 +674,11 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
   const float* cls_extra = nullptr;
   if (shrinks) {
     gather_fuse_bwd(c, dxg.f, h->base + bb.xp_full, B, Ta - 1, D, k, h->at<int>(bb.kept), h->at<int>(bb.dropped),
-                    h->at<float>(bb.s), h->cfg.fuse_mode, dxp.f, dxp.c, h->at<float>(h->off_escore));
-    if (h->cfg.fuse_mode == BSR_FUSE_WEIGHTED_SUM) cls_extra = h->at<float>(h->off_escore);
+                    h->at<float>(bb.s), h->cfg.fuse_mode, dxp.f, dxp.c, h->at<float>(h->off_escore), h->base + bb.xp);
+    if (h->cfg.fuse_mode != BSR_FUSE_NONE) cls_extra = h->at<float>(h->off_escore);
   }
   // attention output projection
+  bool tail_cls_attn = false;
   const float* ln1_res = dxp.f;
   if (!tail) {
     gemm(c, op(dxp), D, 1, h->wb(l, "attn.proj.weight"), 1, D, d_o, 0, Ma, D, D, none);
@@ -660,8 +694,13 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
       gemm(c, op(dxp), 1, D, h->base + bb.o_cls, 1, D, h->gb(l, "attn.proj.weight"), 1, D, D, B, none);
       if (shrinks) colsum(cf, dxp.f, B, D, csp, h->gb(l, "attn.proj.bias"));
     }
-    cudaMemsetAsync(d_o, 0, (size_t)Mdense * D * es, c.stream);
-    copy_rows(c.stream, do_cls, (long)D * es, d_o, (long)Ta * D * es, B, (int)(D * es));
+    // with the classification-row attention, dqkv comes straight from do_cls; otherwise dO is scattered into a zeroed
+    // dense tensor for the general kernel
+    tail_cls_attn = attention_cls_bwd(c, h->base + bb.qkv, do_cls, dqkv, B, Ta, H, hd) == 0;
+    if (!tail_cls_attn) {
+      cudaMemsetAsync(d_o, 0, (size_t)Mdense * D * es, c.stream);
+      copy_rows(c.stream, do_cls, (long)D * es, d_o, (long)Ta * D * es, B, (int)(D * es));
+    }
     float* dense_res = h->at<float>(h->off_dxp);
     cudaMemsetAsync(dense_res, 0, (size_t)Mdense * D * 4, c.stream);
     copy_rows(c.stream, dxp.f, (long)D * 4, dense_res, (long)Ta * D * 4, B, D * 4);
@@ -671,9 +710,11 @@ int block_backward(bsr_handle* h, const Ctx& c, int l, int B, GradStream dxo, Gr
   // the gradient this block hands to block l-1 is that block's output gradient: its column sums are the bias gradient
   // of block l-1's second FFN layer (dense FFN, trainable)
   float* prev_fc2_bias = (need_dxi && l > 0 && ((h->cfg.trainable_mask >> (l - 1)) & 1u) && !is_moe(h, l - 1)) ? h->gb(l - 1, "mlp.fc2.bias") : nullptr;
-  int rc = attention_bwd(c, h->base + bb.qkv, h->base + bb.o, d_o, h->at<float>(bb.lse), h->at<float>(h->off_delta),
-                         cls_extra, dqkv, B, Ta, H, hd);
-  if (rc != 0) return set_err(h->err, BSR_ERR_UNSUPPORTED, "attention backward: %d tokens do not fit this kernel", Ta);
+  if (!tail_cls_attn) {
+    int rc = attention_bwd(c, h->base + bb.qkv, h->base + bb.o, d_o, h->at<float>(bb.lse), h->at<float>(h->off_delta),
+                           cls_extra, dqkv, B, Ta, H, hd);
+    if (rc != 0) return set_err(h->err, BSR_ERR_UNSUPPORTED, "attention backward: %d tokens do not fit this kernel", Ta);
+  }
   // QKV projection
   gemm(c, dqkv, 3 * D, 1, h->wb(l, "attn.qkv.weight"), 1, D, dy, 0, Ma, D, 3 * D, none);
   if (pg) {
@@ -837,6 +878,11 @@ int32_t bsr_create(const bsr_config* cfg, void* workspace, size_t bytes, bsr_han
   }
   if (!chunks.empty())
     cudaMemcpy(h->base + h->off_chunks, chunks.data(), chunks.size() * sizeof(AdamChunk), cudaMemcpyHostToDevice);
+  if (!h->guards.empty()) {
+    std::vector<unsigned long long> table(h->guards.begin(), h->guards.end());
+    cudaMemcpy(h->base + h->off_guard_table, table.data(), table.size() * sizeof(unsigned long long), cudaMemcpyHostToDevice);
+    guards_write(0, h->base, h->at<unsigned long long>(h->off_guard_table), (int)table.size(), (int)(GUARD_BYTES / 4), GUARD_WORD);
+  }
   cudaError_t e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     delete h;
@@ -960,8 +1006,10 @@ int32_t bsr_set_step(bsr_handle* h, int64_t steps_done) {
 
 // Enqueues every kernel of one step on `stream` (forward, loss, backward, AdamW reading its scalars from device memory).
 // loss_out may be null (the multi-step loop writes the loss itself); img_offset as in forward_all.
+static void enqueue_optimizer(bsr_handle* h, const Ctx& c);
 static int enqueue_train_step(bsr_handle* h, const void* images, const int32_t* labels, const int32_t* task_ids, int32_t batch,
-                              void* stream, float* loss_out, int32_t* kept_out, const long long* img_offset = nullptr) {
+                              void* stream, float* loss_out, int32_t* kept_out, const long long* img_offset = nullptr,
+                              bool with_update = true) {
   int rc;
   const bsr_dims& d = h->cfg.dims;
   Ctx c = make_ctx(h, stream);
@@ -1002,6 +1050,13 @@ static int enqueue_train_step(bsr_handle* h, const void* images, const int32_t* 
     layernorm_bwd(c, h->at<float>(h->off_dxn), 1, h->at<float>(x_last), (long)Tl * D, h->at<float>(h->off_meanf), h->at<float>(h->off_rstdf),
                   (const float*)h->w("norm.weight"), nullptr, nullptr, 0, nullptr, lnp, h->gradp("norm.weight"), h->gradp("norm.bias"), B, D);
   }
+  if (with_update) enqueue_optimizer(h, c);
+  return BSR_OK;
+}
+
+// The update of the trainable parameters from the flat gradient buffer; learning rate and bias corrections are read
+// from device memory (the three scalars at status + 128).
+static void enqueue_optimizer(bsr_handle* h, const Ctx& c) {
   if (h->cfg.optimizer == BSR_OPT_SGD)
     sgd_momentum(c, h->at<AdamChunk>(h->off_chunks), h->n_chunks, h->at<float>(h->off_master), h->at<float>(h->off_grad),
                  h->at<float>(h->off_m), h->base + h->off_weights, h->at<float>(h->off_status + 128), h->cfg.momentum, h->cfg.weight_decay);
@@ -1009,7 +1064,6 @@ static int enqueue_train_step(bsr_handle* h, const void* images, const int32_t* 
     adamw(c, h->at<AdamChunk>(h->off_chunks), h->n_chunks, h->at<float>(h->off_master), h->at<float>(h->off_grad), h->at<float>(h->off_m),
           h->at<float>(h->off_v), h->base + h->off_weights, h->at<float>(h->off_status + 128), h->cfg.beta1, h->cfg.beta2, h->cfg.eps,
           h->cfg.weight_decay);
-  return BSR_OK;
 }
 
 }  // extern "C"
@@ -1085,6 +1139,42 @@ int32_t bsr_train_step(bsr_handle* h, const void* images, const int32_t* labels,
   key.images = images; key.labels = labels; key.tasks = task_ids; key.loss = loss_out; key.kept = kept_out; key.batch = batch;
   key.mode = h->use_tc; key.loop = 0; key.exec = nullptr; key.launches = 0; key.last_use = 0;
   rc = run_step_graphed(h, st, key, [&]() { return enqueue_train_step(h, images, labels, task_ids, batch, stream, loss_out, kept_out); });
+  if (rc == BSR_OK) h->step = step_next;
+  return rc;
+}
+
+int32_t bsr_forward_backward(bsr_handle* h, const void* images, const int32_t* labels, const int32_t* task_ids, int32_t batch,
+                             void* stream, float* loss_out, int32_t* kept_out) {
+  int rc = check_batch(h, images, batch);
+  if (rc != BSR_OK) return rc;
+  if (labels == nullptr || loss_out == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "labels_dev and loss_dev_out must not be null");
+  if (h->cfg.dims.num_tasks > 1 && task_ids == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "task_ids_dev is required with several tasks");
+  bsr_handle::StepGraph key;
+  key.images = images; key.labels = labels; key.tasks = task_ids; key.loss = loss_out; key.kept = kept_out; key.batch = batch;
+  key.mode = h->use_tc; key.loop = 2; key.exec = nullptr; key.launches = 0; key.last_use = 0;
+  return run_step_graphed(h, (cudaStream_t)stream, key, [&]() {
+    return enqueue_train_step(h, images, labels, task_ids, batch, stream, loss_out, kept_out, nullptr, false);
+  });
+}
+
+int32_t bsr_grad_buffer(bsr_handle* h, float** grads_dev_out, size_t* count_out) {
+  if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
+  if (grads_dev_out == nullptr || count_out == nullptr) return set_err(h->err, BSR_ERR_INVALID_ARG, "null argument");
+  *grads_dev_out = h->at<float>(h->off_grad);
+  *count_out = h->n_flat;
+  return BSR_OK;
+}
+
+int32_t bsr_optimizer_step(bsr_handle* h, void* stream) {
+  if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
+  cudaStream_t st = (cudaStream_t)stream;
+  const int64_t step_next = h->step + 1;
+  double bc1 = 1.0 - std::pow((double)h->cfg.beta1, (double)step_next);
+  double bc2 = 1.0 - std::pow((double)h->cfg.beta2, (double)step_next);
+  set_scalars(st, h->at<float>(h->off_status + 128), h->lr, (float)bc1, (float)bc2);
+  Ctx c = make_ctx(h, stream);
+  enqueue_optimizer(h, c);
+  int rc = check_cuda(h, "bsr_optimizer_step");
   if (rc == BSR_OK) h->step = step_next;
   return rc;
 }
@@ -1211,17 +1301,23 @@ int32_t bsr_get_footprint(const bsr_handle* h, bsr_footprint* out) {
     if (t.trainable) params += t.numel;
   out->paper_activation_bytes = paper;
   out->trainable_params = params;
+  for (int l = 0; l < d.depth && l < BSR_MAX_DEPTH; ++l) out->block_saved_bytes[l] = h->block_saved_bytes[l];
   return BSR_OK;
 }
 
 int32_t bsr_sync_status(bsr_handle* h, void* stream) {
   if (h == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "handle is null");
   int st = 0;
+  if (!h->guards.empty())
+    guards_check((cudaStream_t)stream, h->base, h->at<unsigned long long>(h->off_guard_table), (int)h->guards.size(), (int)(GUARD_BYTES / 4),
+                 GUARD_WORD, h->at<int>(h->off_status));
   cudaError_t e = cudaMemcpyAsync(&st, h->base + h->off_status, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(h->base + h->off_status, 0, 4, (cudaStream_t)stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
   if (e != cudaSuccess) return set_err(h->err, BSR_ERR_CUDA, "bsr_sync_status: %s", cudaGetErrorString(e));
   if (st & STATUS_TIMEOUT) return set_err(h->err, BSR_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired");
+  if (st & STATUS_GUARD) return set_err(h->err, BSR_ERR_MEMORY_GUARD, "a guard word between two workspace slices was overwritten");
+  if (st & STATUS_CHECK) return set_err(h->err, BSR_ERR_DEVICE_CHECK, "a device-side index check failed (checked build)");
   if (st & STATUS_NONFINITE) return set_err(h->err, BSR_ERR_NONFINITE, "the loss was not finite");
   return BSR_OK;
 }
@@ -1317,7 +1413,7 @@ int32_t bsr_gather_fuse(const void* x, int32_t dtype, int32_t batch, int32_t m, 
   if (x == nullptr || kept == nullptr || out == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "null argument");
   if (dtype != BSR_DTYPE_FP32 && dtype != BSR_DTYPE_BF16) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad dtype");
   if (batch < 1 || m < 1 || k < 1 || k > m || dim < 1 || (dim * dtype_size(dtype)) % 16 != 0) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad shape: rows must be a multiple of 16 bytes, 1 <= k <= m");
-  bool fuse = fuse_mode == BSR_FUSE_WEIGHTED_SUM && k < m;
+  bool fuse = (fuse_mode == BSR_FUSE_WEIGHTED_SUM || fuse_mode == BSR_FUSE_WEIGHTED_MEAN) && k < m;
   if (fuse && (dropped == nullptr || scores == nullptr)) return set_err(g_error, BSR_ERR_INVALID_ARG, "fusion needs dropped_dev and scores_dev");
   Ctx c = bare_ctx(dtype, stream);
   gather_fuse(c, x, batch, m, dim, k, kept, dropped, scores, fuse_mode, out);

@@ -67,7 +67,9 @@ gemm_simt_kernel(const T* __restrict__ A, long a_rs, long a_cs, const T* __restr
         if (aux_out != nullptr) aux_out[o] = from_f<TC>(v);
         v = gelu_f(v);
       } else if (act == 2) {
-        v *= gelu_grad_f(to_f(aux_in[o]));
+        float z = to_f(aux_in[o]);
+        v *= gelu_grad_f(z);
+        if (aux_out != nullptr) reinterpret_cast<T*>(aux_out)[o] = from_f<T>(gelu_f(z));     // GELU(z), storage type
       }
       if (residual != nullptr) v += to_f(residual[o]);
       C[o] = from_f<TC>(v);

@@ -334,6 +334,11 @@ __global__ void splitk_reduce_epi_kernel(const float* __restrict__ partial, TOut
     load4(reinterpret_cast<const bf16*>(ep.aux_in) + i, z);
 #pragma unroll
     for (int j = 0; j < 4; ++j) v[j] *= gelu_grad_f(z[j]);
+    if (ep.aux_out != nullptr) {            // GELU(z), recomputed for the weight gradient that follows
+#pragma unroll
+      for (int j = 0; j < 4; ++j) z[j] = gelu_f(z[j]);
+      store4(reinterpret_cast<bf16*>(ep.aux_out) + i, z);
+    }
   }
   if (ep.residual != nullptr) {
     float r[4];

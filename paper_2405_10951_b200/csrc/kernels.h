@@ -92,7 +92,7 @@ struct GemmEpilogue {
   const float* bias = nullptr;      // [n]
   const void* residual = nullptr;   // [m, n] in the output type, added last
   int act = 0;                      // 0 none, 1 GELU (pre-activation optionally stored), 2 multiply by GELU'(aux_in)
-  void* aux_out = nullptr;          // act 1: pre-activation [m, n], output type
+  void* aux_out = nullptr;          // act 1: pre-activation [m, n], output type; act 2 (optional): GELU(aux_in) [m, n], storage type
   const void* aux_in = nullptr;     // act 2: pre-activation [m, n], storage type
 };
 void gemm(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long b_rs, long b_cs, void* C,
@@ -133,14 +133,22 @@ int attention_fwd(const Ctx& c, const void* qkv, void* out, float* lse, float* c
 int attention_bwd(const Ctx& c, const void* qkv, const void* out, const void* dout, const float* lse, float* delta,
                   const float* cls_extra, void* dqkv, int B, int T, int H, int d);
 
+// The classification row alone (last block: only that row of the block's output is ever read).  out_cls / dout_cls
+// [B, H*d]: attention output of query 0 and its gradient; dqkv [B, T, 3, H, d] is written in full (rows of dQ other
+// than the first are zero).  Return non-zero when the problem does not fit (more than 640 tokens, odd head dimension).
+int attention_cls_fwd(const Ctx& c, const void* qkv, void* out_cls, int B, int T, int H, int d);
+int attention_cls_bwd(const Ctx& c, const void* qkv, const void* dout_cls, void* dqkv, int B, int T, int H, int d);
+
 // ---- token selection --------------------------------------------------------------------------
 void token_select(cudaStream_t s, const float* p, int B, int H, int M, int k, float* scores, int* kept, int* dropped);
 void gather_fuse(const Ctx& c, const void* x, int B, int M, int D, int k, const int* kept, const int* dropped,
                  const float* scores, int fuse, void* out);
-// Backward of the compaction: dx [B, 1+M, D] from dout [B, 1+k+f, D]; escore [B, M] = <g_fused, x_j> for dropped j, else 0.
+// Backward of the compaction: dx [B, 1+M, D] from dout [B, 1+k+f, D]; escore [B, M] = gradient arriving at the fusion
+// weight of each dropped token (<g_fused, x_j> for the weighted sum), 0 for kept ones.  fuse: 0 none, 1 weighted sum,
+// 2 weighted mean (needs fwd_out, the forward pass's compacted tensor [B, 1+k+1, D] float, for the fused row).
 // dx_copy (optional): the same rows in bf16 for the GEMMs that consume them (float streams only).
 void gather_fuse_bwd(const Ctx& c, const void* dout, const void* x, int B, int M, int D, int k, const int* kept,
-                     const int* dropped, const float* scores, int fuse, void* dx, void* dx_copy, float* escore);
+                     const int* dropped, const float* scores, int fuse, void* dx, void* dx_copy, float* escore, const void* fwd_out);
 
 // ---- head, loss, optimiser --------------------------------------------------------------------
 // logits[b, c] = xn[b] . W_task(b)[c] + bias; classes beyond the task's count get -inf.
@@ -212,6 +220,12 @@ void moe_combine_bwd(const Ctx& c, const MoeBufs& b, const float* dout, void* do
 void moe_seg_colsum(const Ctx& c, const MoeBufs& b, const void* x, int cols, int E, float* out);
 void moe_gate_bwd(const Ctx& c, const MoeBufs& b, const void* dxg, const float* dw, const void* wg, const int* task_ids,
                   int tokens_per_image, int tasks, int M, int D, int E, int K, void* dy, float* dsel_row, float* dwg);
+
+// ---- guard words between workspace slices ------------------------------------------------------
+// table[i]: byte offset from base of guard i (words 32-bit values each).  guards_write fills them with `word`;
+// guards_check raises STATUS_GUARD in *status when any word differs.
+void guards_write(cudaStream_t s, char* base, const unsigned long long* table, int n, int words, uint32_t word);
+void guards_check(cudaStream_t s, const char* base, const unsigned long long* table, int n, int words, uint32_t word, int* status);
 
 // ---- conversions ------------------------------------------------------------------------------
 void convert_from_float(const Ctx& c, const float* src, void* dst, size_t n);   // float -> storage dtype

@@ -457,10 +457,16 @@ void head_fwd(const Ctx& c, const HeadDesc& h, const float* xn, const int* task_
 // One warp per image: loss_b = logsumexp(logits) - logits[label]; dlogits = (softmax - onehot) / B.
 __global__ void cross_entropy_kernel(HeadDev h, const float* __restrict__ logits, const int* __restrict__ labels,
                                      const int* __restrict__ task_ids, float* __restrict__ per_image,
-                                     float* __restrict__ dlogits, int B) {
+                                     float* __restrict__ dlogits, int B, int* status) {
   int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= B) return;
   int t = task_ids ? task_ids[warp] : 0;
+  // labels and task ids come from the caller: in every build a value outside its range raises STATUS_CHECK and is
+  // clamped, instead of indexing outside the logits
+  if (t < 0 || t >= h.num_tasks) {
+    if (lane == 0 && status != nullptr) atomicOr(status, STATUS_CHECK);
+    t = 0;
+  }
   int n = h.ncls[t];
   const float* lr = logits + (size_t)warp * h.cmax;
   float mx = -INFINITY;
@@ -470,6 +476,10 @@ __global__ void cross_entropy_kernel(HeadDev h, const float* __restrict__ logits
   for (int i = lane; i < n; i += 32) se += expf(lr[i] - mx);
   se = warp_sum(se);
   int label = labels[warp];
+  if (label < 0 || label >= n) {
+    if (lane == 0 && status != nullptr) atomicOr(status, STATUS_CHECK);
+    label = 0;
+  }
   float inv = 1.0f / se, invB = 1.0f / (float)B;
   for (int i = lane; i < h.cmax; i += 32) {
     float g = 0.f;
@@ -496,7 +506,7 @@ void cross_entropy(const Ctx& c, const HeadDesc& h, const float* logits, const i
                    float* per_image, float* dlogits, float* loss, int B) {
   note_launch(2);
   int threads = 128, blocks = ceil_div((long)B * 32, threads);
-  cross_entropy_kernel<<<blocks, threads, 0, c.stream>>>(to_dev(h), logits, labels, task_ids, per_image, dlogits, B);
+  cross_entropy_kernel<<<blocks, threads, 0, c.stream>>>(to_dev(h), logits, labels, task_ids, per_image, dlogits, B, c.status);
   loss_reduce_kernel<<<1, 32, 0, c.stream>>>(per_image, B, loss, c.status);
 }
 
@@ -646,6 +656,31 @@ void loop_begin(cudaStream_t s, LoopState* st, float* scalars, const int* labels
 void loop_end(cudaStream_t s, LoopState* st, const float* loss, float* loss_out) {
   note_launch(1);
   loop_end_kernel<<<1, 1, 0, s>>>(st, loss, loss_out);
+}
+
+// Guard words after every workspace slice: one warp per guard.
+__global__ void guards_write_kernel(char* base, const unsigned long long* __restrict__ table, int n, int words, uint32_t word) {
+  int g = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (g >= n) return;
+  uint32_t* p = reinterpret_cast<uint32_t*>(base + table[g]);
+  for (int i = lane; i < words; i += 32) p[i] = word;
+}
+__global__ void guards_check_kernel(const char* base, const unsigned long long* __restrict__ table, int n, int words, uint32_t word,
+                                    int* status) {
+  int g = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (g >= n) return;
+  const uint32_t* p = reinterpret_cast<const uint32_t*>(base + table[g]);
+  bool bad = false;
+  for (int i = lane; i < words; i += 32) bad |= p[i] != word;
+  if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(status, STATUS_GUARD);
+}
+void guards_write(cudaStream_t s, char* base, const unsigned long long* table, int n, int words, uint32_t word) {
+  note_launch(1);
+  guards_write_kernel<<<ceil_div((long)n * 32, 256), 256, 0, s>>>(base, table, n, words, word);
+}
+void guards_check(cudaStream_t s, const char* base, const unsigned long long* table, int n, int words, uint32_t word, int* status) {
+  note_launch(1);
+  guards_check_kernel<<<ceil_div((long)n * 32, 256), 256, 0, s>>>(base, table, n, words, word, status);
 }
 
 __global__ void set_scalars_kernel(float* dst, float a, float b, float c3) {

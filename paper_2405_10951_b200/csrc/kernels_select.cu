@@ -171,7 +171,7 @@ constexpr int GF_ROWLANES = GF_THREADS / GF_SLICE_CHUNKS;
 template <typename T>
 __global__ void gather_fuse_kernel(const T* __restrict__ x, int M, int D, int k, const int* __restrict__ kept,
                                    const int* __restrict__ dropped, const float* __restrict__ scores, int fuse,
-                                   T* __restrict__ out, int copy_splits) {
+                                   T* __restrict__ out, int copy_splits, int* status) {
   constexpr int N = Pack<T>::N;
   int b = blockIdx.x;
   int chunks = D / N;
@@ -186,12 +186,14 @@ __global__ void gather_fuse_kernel(const T* __restrict__ x, int M, int D, int k,
     for (int i = threadIdx.x; i < total; i += GF_THREADS) {
       int r = r0 + i / chunks, ch = i % chunks;
       int src = (r == 0) ? 0 : 1 + kept[(size_t)b * k + (r - 1)];
+      if (!BSR_CHECK(src >= 0 && src <= M, status)) continue;
       uint4 v = *reinterpret_cast<const uint4*>(xb + (size_t)src * D + ch * N);
       *reinterpret_cast<uint4*>(ob + (size_t)r * D + ch * N) = v;
     }
     return;
   }
   __shared__ float sm[GF_ROWLANES][GF_SLICE_CHUNKS * N];
+  __shared__ float weight_sum;
   int slice = blockIdx.y - copy_splits;
   int cs = threadIdx.x % GF_SLICE_CHUNKS, rl = threadIdx.x / GF_SLICE_CHUNKS;
   int ch = slice * GF_SLICE_CHUNKS + cs;
@@ -199,9 +201,16 @@ __global__ void gather_fuse_kernel(const T* __restrict__ x, int M, int D, int k,
 #pragma unroll
   for (int j = 0; j < N; ++j) acc[j] = 0.f;
   int nd = M - k;
+  if (fuse == 2 && threadIdx.x < 32) {        // weighted mean: the sum of the dropped tokens' weights, in a fixed order
+    float ws = 0.f;
+    for (int i = threadIdx.x; i < nd; i += 32) ws += scores[(size_t)b * M + dropped[(size_t)b * nd + i]];
+    ws = warp_sum(ws);
+    if (threadIdx.x == 0) weight_sum = ws;
+  }
   if (ch < chunks) {
     for (int i = rl; i < nd; i += GF_ROWLANES) {
       int j = dropped[(size_t)b * nd + i];
+      if (!BSR_CHECK(j >= 0 && j < M, status)) continue;
       float w = scores[(size_t)b * M + j];
       float v[N];
       load16(xb + (size_t)(1 + j) * D + ch * N, v);
@@ -219,7 +228,7 @@ __global__ void gather_fuse_kernel(const T* __restrict__ x, int M, int D, int k,
       float s = 0.f;
 #pragma unroll
       for (int r = 0; r < GF_ROWLANES; ++r) s += sm[r][cs * N + e];
-      o[e] = s;
+      o[e] = fuse == 2 ? s / weight_sum : s;
     }
     store16(ob + (size_t)(1 + k) * D + ch * N, o);
   }
@@ -230,7 +239,7 @@ void gather_fuse(const Ctx& c, const void* x, int B, int M, int D, int k, const 
   note_launch(1);
   int n = (c.dtype == 0) ? 4 : 8;
   int chunks = D / n;
-  int do_fuse = (fuse == 1 && k < M) ? 1 : 0;
+  int do_fuse = ((fuse == 1 || fuse == 2) && k < M) ? fuse : 0;          // 1: weighted sum, 2: weighted mean
   int fuse_slices = do_fuse ? ceil_div(chunks, GF_SLICE_CHUNKS) : 0;
   int sms = c.sm_count > 0 ? c.sm_count : 148;
   int copy_splits = ceil_div(4L * sms, B);            // about four blocks per SM in total
@@ -238,18 +247,21 @@ void gather_fuse(const Ctx& c, const void* x, int B, int M, int D, int k, const 
   if (copy_splits > 1 + k) copy_splits = 1 + k;
   dim3 grid(B, copy_splits + fuse_slices);
   if (c.dtype == 0)
-    gather_fuse_kernel<float><<<grid, GF_THREADS, 0, c.stream>>>((const float*)x, M, D, k, kept, dropped, scores, do_fuse, (float*)out, copy_splits);
+    gather_fuse_kernel<float><<<grid, GF_THREADS, 0, c.stream>>>((const float*)x, M, D, k, kept, dropped, scores, do_fuse, (float*)out, copy_splits, c.status);
   else
-    gather_fuse_kernel<bf16><<<grid, GF_THREADS, 0, c.stream>>>((const bf16*)x, M, D, k, kept, dropped, scores, do_fuse, (bf16*)out, copy_splits);
+    gather_fuse_kernel<bf16><<<grid, GF_THREADS, 0, c.stream>>>((const bf16*)x, M, D, k, kept, dropped, scores, do_fuse, (bf16*)out, copy_splits, c.status);
 }
 
 // Backward of the compaction, one warp per input row (the index sets are constants, the fusion weights are
 // differentiated):  dx_0 = g_0;  dx_{kept_i} = g_{1+i};  dx_j = s_j g_f and e_j = <g_f, x_j> for dropped j.
+// Weighted mean (fuse == 2, f = sum_j s_j x_j / S, S = sum_j s_j): dx_j = (s_j / S) g_f, e_j = (<g_f, x_j> - <g_f, f>) / S
+// with f read from the forward pass's compacted tensor `fwd_out`.
 // Rows are float (residual stream); dx_copy optionally receives the same rows in bf16.
 __global__ void gather_fuse_bwd_kernel(const float* __restrict__ dout, const float* __restrict__ x, int B, int M, int D, int k,
                                        const int* __restrict__ kept, const int* __restrict__ dropped,
                                        const float* __restrict__ scores, int fuse, float* __restrict__ dx,
-                                       bf16* __restrict__ dx_copy, float* __restrict__ escore) {
+                                       bf16* __restrict__ dx_copy, float* __restrict__ escore, const float* __restrict__ fwd_out,
+                                       int* status) {
   int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= B * (1 + M)) return;
   int b = warp / (1 + M), e = warp % (1 + M);
@@ -259,6 +271,7 @@ __global__ void gather_fuse_bwd_kernel(const float* __restrict__ dout, const flo
   size_t ob = (size_t)b * (1 + M) * D;
   if (e <= k) {                         // classification row or a kept row: plain copy
     int dst = (e == 0) ? 0 : 1 + kept[(size_t)b * k + (e - 1)];
+    if (!BSR_CHECK(dst >= 0 && dst <= M, status)) return;
     for (int ch = lane; ch < chunks; ch += 32) {
       float v[4];
       load16(gb + (size_t)e * D + ch * 4, v);
@@ -269,9 +282,27 @@ __global__ void gather_fuse_bwd_kernel(const float* __restrict__ dout, const flo
     return;
   }
   int j = dropped[(size_t)b * (M - k) + (e - 1 - k)];
+  if (!BSR_CHECK(j >= 0 && j < M, status)) return;
   float w = fuse ? scores[(size_t)b * M + j] : 0.f;
   const float* gf = gb + (size_t)(1 + k) * D;
   const float* xr = x + ob + (size_t)(1 + j) * D;
+  float inv_sum = 1.f, dot_f = 0.f;
+  if (fuse == 2) {
+    int nd = M - k;
+    float ws = 0.f;
+    for (int i = lane; i < nd; i += 32) ws += scores[(size_t)b * M + dropped[(size_t)b * nd + i]];
+    inv_sum = 1.0f / warp_sum(ws);
+    const float* fr = fwd_out + ((size_t)b * t_out + 1 + k) * D;
+    for (int ch = lane; ch < chunks; ch += 32) {
+      float g[4], fv[4];
+      load16(gf + ch * 4, g);
+      load16(fr + ch * 4, fv);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) dot_f += g[i] * fv[i];
+    }
+    dot_f = warp_sum(dot_f);
+    w *= inv_sum;
+  }
   float dot = 0.f;
   for (int ch = lane; ch < chunks; ch += 32) {
     float g[4], o[4];
@@ -289,16 +320,16 @@ __global__ void gather_fuse_bwd_kernel(const float* __restrict__ dout, const flo
     if (dx_copy != nullptr) store4(dx_copy + ob + (size_t)(1 + j) * D + ch * 4, o);
   }
   dot = warp_sum(dot);
-  if (lane == 0) escore[(size_t)b * M + j] = dot;
+  if (lane == 0) escore[(size_t)b * M + j] = fuse == 2 ? (dot - dot_f) * inv_sum : dot;
 }
 
 void gather_fuse_bwd(const Ctx& c, const void* dout, const void* x, int B, int M, int D, int k, const int* kept,
-                     const int* dropped, const float* scores, int fuse, void* dx, void* dx_copy, float* escore) {
+                     const int* dropped, const float* scores, int fuse, void* dx, void* dx_copy, float* escore, const void* fwd_out) {
   note_launch(1);
-  int do_fuse = (fuse == 1 && k < M) ? 1 : 0;
+  int do_fuse = ((fuse == 1 || fuse == 2) && k < M) ? fuse : 0;
   int threads = 256, blocks = ceil_div((long)B * (1 + M) * 32, threads);
   gather_fuse_bwd_kernel<<<blocks, threads, 0, c.stream>>>((const float*)dout, (const float*)x, B, M, D, k, kept, dropped, scores,
-                                                           do_fuse, (float*)dx, (bf16*)dx_copy, escore);
+                                                           do_fuse, (float*)dx, (bf16*)dx_copy, escore, (const float*)fwd_out, c.status);
 }
 
 }  // namespace bsr

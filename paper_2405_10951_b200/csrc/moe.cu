@@ -149,11 +149,12 @@ moe_assign_kernel(const int* __restrict__ eidx, const float* __restrict__ ew, co
 // ---- gather the expert inputs: xg[r] = y[row_token[r]], empty rows are zero ---------------------------------------
 template <typename T>
 __global__ void moe_gather_kernel(const T* __restrict__ y, const int* __restrict__ row_token, const int* __restrict__ seg_start,
-                                  int E, int D, T* __restrict__ xg, int rows_cap) {
+                                  int E, int D, T* __restrict__ xg, int rows_cap, int M, int* status) {
   constexpr int N = Pack<T>::N;
   int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= rows_cap || warp >= seg_start[E]) return;
   int tok = row_token[warp];
+  if (!BSR_CHECK(tok < M, status)) return;
   for (int ch = lane; ch < D / N; ch += 32) {
     uint4 v = make_uint4(0, 0, 0, 0);
     if (tok >= 0) v = *reinterpret_cast<const uint4*>(y + (size_t)tok * D + ch * N);
@@ -347,8 +348,8 @@ void moe_route(const Ctx& c, const MoeBufs& b, const void* y, const void* wg, co
   cudaMemsetAsync(b.row_token, 0xFF, (size_t)rows_cap * sizeof(int), c.stream);
   moe_assign_kernel<<<nblk, 256, 0, c.stream>>>(b.eidx, b.ew, b.blk_off, b.seg_start, M, E, K, b.pos, b.row_token, b.row_w);
   int blocks = ceil_div((long)rows_cap * 32, 256);
-  if (c.dtype == 0) moe_gather_kernel<float><<<blocks, 256, 0, c.stream>>>((const float*)y, b.row_token, b.seg_start, E, D, (float*)b.xg, rows_cap);
-  else moe_gather_kernel<bf16><<<blocks, 256, 0, c.stream>>>((const bf16*)y, b.row_token, b.seg_start, E, D, (bf16*)b.xg, rows_cap);
+  if (c.dtype == 0) moe_gather_kernel<float><<<blocks, 256, 0, c.stream>>>((const float*)y, b.row_token, b.seg_start, E, D, (float*)b.xg, rows_cap, M, c.status);
+  else moe_gather_kernel<bf16><<<blocks, 256, 0, c.stream>>>((const bf16*)y, b.row_token, b.seg_start, E, D, (bf16*)b.xg, rows_cap, M, c.status);
 }
 
 void moe_combine(const Ctx& c, const MoeBufs& b, const float* res, float* out, int M, int D, int K) {

@@ -76,6 +76,23 @@ __device__ __forceinline__ void gelu_grad_mul2(float& g0, float& g1, float z0, f
   g1 *= fmaf(d1, e1, __saturatef(fmaf(z1, q1, 0.5f)));
 }
 
+// The same, also returning h = GELU(z) = z * Phi(z) (the second FFN layer's input, recomputed in the backward pass
+// instead of being kept since the forward pass).
+__device__ __forceinline__ void gelu_grad_mul2h(float& g0, float& g1, float z0, float z1, float& h0, float& h1) {
+  float u0, u1, q0, q1, d0, d1, e0, e1;
+  uint64_t z = pack2(z0, z1);
+  unpack2(mul2(z, z), u0, u1);
+  phi_slope2(u0, u1, q0, q1);
+  const float kh = -0.5f * 1.4426950408889634f;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(u0 * kh));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(u1 * kh));
+  unpack2(mul2(z, dup2(0.39894228040143268f)), d0, d1);
+  float p0 = __saturatef(fmaf(z0, q0, 0.5f)), p1 = __saturatef(fmaf(z1, q1, 0.5f));
+  h0 = z0 * p0; h1 = z1 * p1;
+  g0 *= fmaf(d0, e0, p0);
+  g1 *= fmaf(d1, e1, p1);
+}
+
 // 16-byte global load of data that is read once (residual stream, stored pre-activations).
 template <typename T>
 __device__ __forceinline__ uint4 ld_stream(const T* p) {
@@ -181,12 +198,18 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t* r, const Epi& ep,
 #pragma unroll
       for (int j = 0; j < 32; j += 2) gelu_fast2(v[j], v[j + 1]);
     } else if (ep.act == 2) {
+      float z[32];
       if (zpre != nullptr) {
 #pragma unroll
-        for (int j = 0; j < 32; j += 2) gelu_grad_mul2(v[j], v[j + 1], zpre[j], zpre[j + 1]);
+        for (int j = 0; j < 32; ++j) z[j] = zpre[j];
       } else {
-        float z[32];
         ChunkIO<bf16>::load((const bf16*)ep.aux_in, N, row0, col0, M, N, st, lane, z);
+      }
+      if (ep.aux_out != nullptr) {          // GELU(z) recomputed for the weight gradient of the second FFN layer
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) gelu_grad_mul2h(v[j], v[j + 1], z[j], z[j + 1], z[j], z[j + 1]);
+        ChunkIO<bf16>::store((bf16*)ep.aux_out, N, row0, col0, M, N, st, lane, z);
+      } else {
 #pragma unroll
         for (int j = 0; j < 32; j += 2) gelu_grad_mul2(v[j], v[j + 1], z[j], z[j + 1]);
       }
@@ -339,14 +362,14 @@ __device__ __forceinline__ void epilogue_warp_tile(LoadTmem load_tmem, const Epi
 #pragma unroll
       for (int j = 0; j < 32; j += 2) gelu_fast2(v[j], v[j + 1]);
     } else if (ep.act == 2) {
-      if (pre_aux) {
+      if (!pre_aux) ChunkIO<bf16>::load((const bf16*)ep.aux_in, N, row0, col0, M, N, st_out, lane, a);
+      if (ep.aux_out != nullptr) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) gelu_grad_mul2h(v[j], v[j + 1], a[j], a[j + 1], a[j], a[j + 1]);
+        ChunkIO<bf16>::store((bf16*)ep.aux_out, N, row0, col0, M, N, st_out, lane, a);
+      } else {
 #pragma unroll
         for (int j = 0; j < 32; j += 2) gelu_grad_mul2(v[j], v[j + 1], a[j], a[j + 1]);
-      } else {
-        float z[32];
-        ChunkIO<bf16>::load((const bf16*)ep.aux_in, N, row0, col0, M, N, st_out, lane, z);
-#pragma unroll
-        for (int j = 0; j < 32; j += 2) gelu_grad_mul2(v[j], v[j + 1], z[j], z[j + 1]);
       }
     }
     if (pre_res) {

@@ -217,3 +217,60 @@ def test_graph_cache_keeps_eight_buffer_sets():
         eng.sync_status()
         assert eng.profile_read()["graph_captures"] == 8
     eng.close()
+
+
+def test_split_step_equals_whole_step_and_exposes_the_gradient_buffer():
+    """bsr_forward_backward + bsr_optimizer_step (the data-parallel halves) equal bsr_train_step bit for bit on one
+    GPU; the gradient buffer handed out for the all-reduce holds exactly the gradients bsr_get_tensor reports, and
+    scaling it before the update scales the SGD update (what an average over ranks does)."""
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    cfg = MINI_BF16
+    images, labels, task_ids, params = synth.make_workload(cfg, peaked=True)
+    shapes = synth.param_shapes(cfg)
+    names = ("head.0.weight", "blocks.5.mlp.fc1.weight", "blocks.3.attn.qkv.weight", "norm.bias", "blocks.4.mlp.fc2.bias")
+    whole = Bd.Engine(cfg)
+    whole.set_params(params)
+    split = Bd.Engine(cfg)
+    split.set_params(params)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        img = whole.images_to_device(images)
+        lab = torch.as_tensor(labels).cuda()
+        for _ in range(2):
+            l1, k1 = whole.train_step(img, lab)
+            l2, k2 = split.forward_backward(img, lab)
+            g = split.grad_buffer()
+            assert g.numel() >= sum(int(np.prod(shapes[n])) for n in O.trainable_names(cfg, params))
+            split.optimizer_step()
+            stream.synchronize()
+            assert float(l1.cpu()[0]) == float(l2.cpu()[0])
+            assert all(torch.equal(a, b) for a, b in zip(k1, k2))
+        whole.sync_status()
+        split.sync_status()
+        for n in names:
+            assert torch.equal(whole.get_tensor(n, shapes[n]), split.get_tensor(n, shapes[n])), n
+            assert torch.equal(whole.get_tensor("grad/" + n, shapes[n]), split.get_tensor("grad/" + n, shapes[n])), n
+        # the buffer is what the optimiser reads: the head's gradient sits in it verbatim
+        gh = split.get_tensor("grad/head.0.weight", shapes["head.0.weight"]).flatten()
+        flat = split.grad_buffer()
+        windows = flat.unfold(0, gh.numel(), 64)                     # tensors start at multiples of 64 values
+        assert bool((windows == gh).all(dim=1).any())
+    whole.close()
+    split.close()
+
+
+def test_bench_data_parallel_path_runs_on_one_rank():
+    """bench.py --parallel dp with a one-rank NCCL group: the split step, the all-reduce of the gradient buffer view and
+    the update run end to end and give the single-GPU throughput line."""
+    import json
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT="29631", RANK="0", WORLD_SIZE="1", LOCAL_RANK="0")
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--workload", "deit_s", "--steps", "5", "--warmup", "3",
+                        "--parallel", "dp", "--no-cpu-baseline"], capture_output=True, text=True, env=env, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    assert line["value"] > 0 and "data parallel" in line["config"]["parallelism"] and line["gpu_launches"] > 0

@@ -32,7 +32,9 @@ def test_select_bit_exact(B, H, M, k, ties):
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 @pytest.mark.parametrize("B,M,D,k,fuse", [(8, 64, 192, 45, 1), (16, 196, 768, 138, 1), (3, 139, 384, 98, 0), (2, 9, 8, 9, 1),
-                                           (4, 576, 768, 288, 1), (5, 33, 64, 1, 1)])
+                                           (4, 576, 768, 288, 1), (5, 33, 64, 1, 1),
+                                           # weighted mean of the dropped tokens (fuse mode 2)
+                                           (8, 64, 192, 45, 2), (16, 196, 768, 138, 2), (3, 33, 64, 32, 2)])
 def test_gather_fuse_matches_oracle(dtype, B, M, D, k, fuse):
     import torch
     from paper_2405_10951_b200 import binding as Bd

@@ -13,7 +13,7 @@ def loss_of(cfg, params, images, labels, task_ids, forced):
     return O.cross_entropy(fw["logits"], labels)[0]
 
 
-@pytest.mark.parametrize("case", ["drop_with_fusion", "suffix_trainable", "moe_multitask"])
+@pytest.mark.parametrize("case", ["drop_with_fusion", "drop_with_mean_fusion", "suffix_trainable", "moe_multitask"])
 def test_gradients_match_central_differences(case):
     """Directional derivatives along random directions, every trainable tensor, rel. error < 1e-6.
 
@@ -98,3 +98,13 @@ def test_gather_fuse_definition():
         fused = sum(s[b, j] * xp[b, 1 + j] for j in dropped[b])
         assert np.allclose(out[b, -1], fused, rtol=1e-13)
     assert O.gather_fuse(xp, kept, dropped, s, fuse_mode=0).shape == (B, k + 1, D)
+    # weighted mean (fuse_mode 2): the weighted sum over the sum of the weights; equal weights give the plain mean of
+    # the dropped tokens, a single dropped token comes back unchanged
+    mean = O.gather_fuse(xp, kept, dropped, s, fuse_mode=2)
+    for b in range(B):
+        assert np.allclose(mean[b, -1], out[b, -1] / s[b, dropped[b]].sum(), rtol=1e-13)
+    flat = O.gather_fuse(xp, kept, dropped, np.full_like(s, 0.125), fuse_mode=2)
+    for b in range(B):
+        assert np.allclose(flat[b, -1], xp[b, 1 + dropped[b]].mean(axis=0), rtol=1e-13)
+    one = O.gather_fuse(xp, np.stack([np.arange(M - 1)] * B), np.full((B, 1), M - 1), s, fuse_mode=2)
+    assert np.allclose(one[:, -1], xp[:, M], rtol=1e-15)

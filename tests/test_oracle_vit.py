@@ -37,6 +37,7 @@ CASES = {
     "keep_one_at_locations": TINY.with_(keep_num=1, keep_den=1),
     "drop_with_fusion": TINY,
     "drop_without_fusion": TINY.with_(fuse_mode=0),
+    "drop_with_mean_fusion": TINY.with_(fuse_mode=2),
     "suffix_trainable": TINY.with_(trainable=(2, 3), drop_blocks=(1, 3)),
     "interleaved_trainable": TINY.with_(trainable=(1, 3), drop_blocks=(1, 2)),
     "moe_multitask": TINY.with_(num_classes=(5, 3), batch=4, moe_experts=4, moe_top_k=2, moe_blocks=(1, 3)),

@@ -40,10 +40,13 @@ def run(cfg, params, images, labels, task_ids, keep_count_fn):
             if k < M:
                 body = x[:, 1:]
                 rows = [x[:, :1], torch.gather(body, 1, idx[:, :, None].expand(B, k, D))]
-                if cfg.fuse_mode == 1:
+                if cfg.fuse_mode in (1, 2):
                     mask = torch.ones(B, M, dtype=torch.float64)
                     mask.scatter_(1, idx, 0.0)
-                    rows.append(((s * mask)[:, :, None] * body).sum(dim=1, keepdim=True))
+                    w = s * mask
+                    if cfg.fuse_mode == 2:                           # weighted mean of the dropped tokens
+                        w = w / w.sum(dim=1, keepdim=True)
+                    rows.append((w[:, :, None] * body).sum(dim=1, keepdim=True))
                 x = torch.cat(rows, dim=1)
         y = F.layer_norm(x, (D,), P[p + "norm2.weight"], P[p + "norm2.bias"], cfg.ln_eps)
         if l in cfg.moe_blocks:
