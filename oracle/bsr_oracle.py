@@ -119,6 +119,44 @@ def linear_bwd(dy, x, w):
 
 
 # ----------------------------------------------------------------------------------------------
+# 8-bit floating point for the frozen prefix (Conclusions: activation / weight quantisation is orthogonal to BSR and
+# can be added on top; the paper fixes no format).  Reading taken: the frozen blocks before the earliest trainable
+# one carry no gradient, so their two LayerNorm-fed linear layers (QKV and the first FFN layer) may run on operands
+# rounded to E4M3 -- each LayerNorm output row and each weight row scaled so that its largest magnitude maps to 448,
+# the products accumulated exactly and rescaled.  Everything else stays as it is.
+# ----------------------------------------------------------------------------------------------
+E4M3_MAX = 448.0
+
+
+def e4m3_round(x):
+    """Nearest value of the 8-bit floating-point format E4M3 (1 sign bit, 4 exponent bits with bias 7, 3 mantissa bits,
+    no infinities: largest magnitude 448, normal numbers down to 2^-6, subnormals in steps of 2^-9), ties to the even
+    mantissa; magnitudes beyond 448 saturate to 448."""
+    x = np.asarray(x, dtype=np.float64)
+    a = np.minimum(np.abs(x), E4M3_MAX)
+    e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
+    e = np.maximum(e, -6.0)                        # below the smallest normal binade the spacing stays 2^-9
+    step = 2.0 ** (e - 3.0)                        # 3 mantissa bits: 8 steps per binade
+    q = np.minimum(np.round(a / step) * step, E4M3_MAX)      # a / step is exact (power of two); np.round ties to even
+    return np.sign(x) * q
+
+
+def quantize_rows_e4m3(a):
+    """Each row of a [..., K] rounded to E4M3 after scaling by scale = max|row| / 448 (1 for an all-zero row); scale and
+    quotient are formed in float32, as a kernel forms them.  Returns the dequantised values and the scales."""
+    a32 = np.asarray(a, dtype=np.float32)
+    amax = np.abs(a32).max(axis=-1, keepdims=True)
+    scale = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)
+    q = e4m3_round((a32 / scale).astype(np.float32))
+    return q * scale.astype(np.float64), scale
+
+
+def linear_e4m3(x, w, b):
+    """y = x W^T + b with the rows of x and of W rounded to E4M3 (quantize_rows_e4m3), exact accumulation."""
+    return quantize_rows_e4m3(x)[0] @ quantize_rows_e4m3(w)[0].T + b
+
+
+# ----------------------------------------------------------------------------------------------
 # token selection (Eq. 6; Section 4.1)
 # ----------------------------------------------------------------------------------------------
 def head_mean_scores(p, dtype=np.float64):
@@ -278,13 +316,15 @@ def moe_bwd(cfg, params, l, dout, cache, task_ids, grads, want_param_grads):
     return dy
 
 
-def block_fwd(cfg, params, l, x, task_ids, k, forced_keep, forced_experts=None):
-    """One encoder block; at a token drop location the compaction sits between MHSA and FFN."""
+def block_fwd(cfg, params, l, x, task_ids, k, forced_keep, forced_experts=None, fp8=False):
+    """One encoder block; at a token drop location the compaction sits between MHSA and FFN.  fp8: the two
+    LayerNorm-fed linear layers of this (frozen, gradient-free) block run on E4M3 operands."""
     p = f"blocks.{l}."
     c = {"x": x}
+    lin = linear_e4m3 if fp8 else linear
     y1, c["ln1"] = layer_norm(x, params[p + "norm1.weight"], params[p + "norm1.bias"], cfg.ln_eps)
     c["y1"] = y1
-    q, kk, v = split_heads(cfg, linear(y1, params[p + "attn.qkv.weight"], params[p + "attn.qkv.bias"]))
+    q, kk, v = split_heads(cfg, lin(y1, params[p + "attn.qkv.weight"], params[p + "attn.qkv.bias"]))
     o, A = attention_fwd(cfg, q, kk, v)
     c.update(q=q, k=kk, v=v, A=A)
     oc = merge_heads(o)
@@ -327,7 +367,7 @@ def block_fwd(cfg, params, l, x, task_ids, k, forced_keep, forced_experts=None):
     if l in cfg.moe_blocks:
         f, c["moe"] = moe_fwd(cfg, params, l, y2, task_ids, forced_experts)
     else:
-        z = linear(y2, params[p + "mlp.fc1.weight"], params[p + "mlp.fc1.bias"])
+        z = lin(y2, params[p + "mlp.fc1.weight"], params[p + "mlp.fc1.bias"])
         h = gelu(z)
         c.update(z=z, h=h)
         f = linear(h, params[p + "mlp.fc2.weight"], params[p + "mlp.fc2.bias"])
@@ -395,6 +435,8 @@ def forward(cfg, params, images, task_ids=None, forced_keep=None, keep_cache=Fal
         task_ids = np.zeros(B, dtype=np.int64)
     sched = token_schedule(cfg)
     x = embed(cfg, params, np.asarray(images, dtype=np.float64))
+    t0 = min(cfg.trainable) if len(cfg.trainable) else cfg.depth
+    fp8_upto = t0 if getattr(cfg, "frozen_fp8", 0) else 0          # dense blocks before the earliest trainable one
     caches, kept, margins, scores, tokens = [], [], [], [], []
     routing = {}
     di = 0
@@ -404,7 +446,7 @@ def forward(cfg, params, images, task_ids=None, forced_keep=None, keep_cache=Fal
         if k is not None and forced_keep is not None and forced_keep[di] is not None:
             fk = forced_keep[di]
         fe = forced_experts.get(l) if forced_experts else None
-        x, c, info = block_fwd(cfg, params, l, x, task_ids, k, fk, fe)
+        x, c, info = block_fwd(cfg, params, l, x, task_ids, k, fk, fe, fp8=(l < fp8_upto and l not in cfg.moe_blocks))
         if l in cfg.moe_blocks:
             routing[l] = {"experts": c["moe"]["experts"], "own_experts": c["moe"]["own_experts"], "glogits": c["moe"]["glogits"]}
         if k is not None:

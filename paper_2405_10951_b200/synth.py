@@ -58,6 +58,7 @@ class Config:
     weight_decay: float = 0.05
     optimizer: str = "adamw"              # "adamw" or "sgd" (with momentum)
     momentum: float = 0.9
+    frozen_fp8: int = 0                   # 1: the LayerNorm-fed linear layers of the blocks before the first trainable one run in E4M3
     seed: int = 0
 
     @property

@@ -103,3 +103,47 @@ def test_moe_mac_term_counts_the_rows_each_expert_processes():
     per_image = rows // MOE.batch * 2 * D * F + tokens * D * MOE.moe_experts
     assert rows == MOE.batch * tokens * MOE.moe_top_k
     assert C.forward_macs(MOE) - C.forward_macs(dense) == per_image - 2 * tokens * D * F
+
+
+def test_e4m3_rounding_matches_the_library_type_and_the_format_definition():
+    import torch
+    rng = np.random.default_rng(8)
+    x = np.concatenate([rng.standard_normal(20000) * s for s in (1e-3, 0.05, 1.0, 30.0, 150.0)])
+    x = np.clip(x, -448.0, 448.0).astype(np.float32)
+    want = torch.tensor(x).to(torch.float8_e4m3fn).float().numpy().astype(np.float64)
+    assert np.array_equal(O.e4m3_round(x), want)
+    # format facts: 3 mantissa bits, ties to the even mantissa, subnormal steps of 2^-9, top value 448, saturation
+    assert list(O.e4m3_round(np.array([17.0, 19.0, 21.0, 1.0625, 1.1875]))) == [16.0, 20.0, 20.0, 1.0, 1.25]
+    assert list(O.e4m3_round(np.array([2.0 ** -9, 2.0 ** -10, 1.5 * 2.0 ** -10, 3 * 2.0 ** -10]))) == [2.0 ** -9, 0.0, 2.0 ** -9, 2.0 ** -8]
+    assert list(O.e4m3_round(np.array([448.0, 449.0, 1e6, -1e6, 0.0]))) == [448.0, 448.0, 448.0, -448.0, 0.0]
+    grid = O.e4m3_round(np.linspace(-448, 448, 200001))
+    assert len(np.unique(np.abs(grid))) <= 127                   # 7 bits of magnitude, one code short of 128 (no NaN / inf here)
+
+
+def test_row_quantisation_scales_each_row_to_the_top_of_the_format():
+    rng = np.random.default_rng(9)
+    a = rng.standard_normal((7, 96)) * rng.random((7, 1)) * 10
+    a[3] = 0.0
+    deq, scale = O.quantize_rows_e4m3(a)
+    assert scale.shape == (7, 1) and scale[3, 0] == 1.0 and not deq[3].any()
+    for r in (0, 1, 2, 4, 5, 6):
+        assert abs(np.abs(deq[r]).max() - np.abs(a[r]).max()) <= 1e-6 * np.abs(a[r]).max()     # the largest entry maps to 448 exactly
+        assert np.abs(deq[r] - a[r]).max() <= np.abs(a[r]).max() / 448 * 16 + 1e-12             # half a step of the top binade
+        rel = np.abs(deq[r] - a[r]) / np.maximum(np.abs(a[r]), np.abs(a[r]).max() * 2.0 ** -6)
+        assert rel.max() <= 2.0 ** -4 + 1e-6                                                    # 3 mantissa bits: half an ulp
+    x, w, b = rng.standard_normal((5, 64)), rng.standard_normal((9, 64)), rng.standard_normal(9)
+    y = O.linear_e4m3(x, w, b)
+    assert np.linalg.norm(y - O.linear(x, w, b)) / np.linalg.norm(O.linear(x, w, b)) < 0.06    # a few percent, not exact
+    assert np.array_equal(y, O.quantize_rows_e4m3(x)[0] @ O.quantize_rows_e4m3(w)[0].T + b)
+
+
+def test_fp8_prefix_touches_only_the_blocks_before_the_first_trainable_one():
+    cfg = synth.CONFIGS["tiny_fp32"]
+    images, labels, task_ids, params = synth.make_workload(cfg, peaked=True)
+    plain = O.train_step(cfg, params, images, labels, task_ids)
+    q = O.train_step(cfg.with_(frozen_fp8=1), params, images, labels, task_ids, forced_keep=plain["kept"])
+    assert q["loss"] != plain["loss"] and abs(q["loss"] - plain["loss"]) < 0.05 * plain["loss"]
+    allb = cfg.with_(trainable=tuple(range(cfg.depth)), frozen_fp8=1)                # no frozen prefix: nothing to quantise
+    a = O.train_step(allb, params, images, labels, task_ids)
+    b = O.train_step(allb.with_(frozen_fp8=0), params, images, labels, task_ids)
+    assert a["loss"] == b["loss"]
