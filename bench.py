@@ -205,12 +205,16 @@ def main():
     ap.add_argument("--ref-batch", type=int, default=48)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--gemm-mode", type=int, default=None, help="1: one CTA per tile, 2: CTA pairs (library default if omitted)")
+    ap.add_argument("--frozen-fp8", action="store_true",
+                    help="NOT the headline: the gradient-free prefix's LayerNorm-fed layers on E4M3 operands (reduced precision)")
     ap.add_argument("--parallel", default="auto", choices=["auto", "dp", "replicas"],
                     help="several GPUs: dp = data parallel, one all-reduce of the trainable gradients per step (the default); "
                          "replicas = independent copies with no exchange")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     cfg = synth.CONFIGS[args.workload]
+    if args.frozen_fp8:
+        cfg = cfg.with_(frozen_fp8=1)
     if args.impl == "reference":
         run_reference(args, cfg)
         return
@@ -364,7 +368,8 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+            "dtype": ("bf16 (gradient-free prefix: E4M3 operands in the LayerNorm-fed layers)" if cfg.frozen_fp8 else "bf16") if cfg.dtype == "bf16" else "f32",
+            "data": "synthetic",
             "config": {"workload": cfg.name, "global_batch": world * cfg.batch, "tokens": cfg.num_patches + 1,
                        "trainable_blocks": list(cfg.trainable), "drop_blocks": list(cfg.drop_blocks),
                        "keep_rate": cfg.keep_num / cfg.keep_den,

@@ -87,6 +87,13 @@ typedef struct {
    * zero; the buffer is read under the name "adam_m/<param>" and "adam_v/<param>" stays zero. */
   int32_t optimizer;                /* BSR_OPT_* */
   float momentum;
+  /* 8-bit floating point in the gradient-free prefix (Conclusions: quantisation is orthogonal to BSR and can be added
+   * on top).  1: in every dense block before the earliest trainable one, the two linear layers fed by a LayerNorm
+   * (QKV and the first FFN layer) multiply E4M3 operands on the tensor cores: each LayerNorm output row and each weight
+   * row is scaled so that its largest magnitude maps to 448 and rounded to nearest-even, the accumulation is float32,
+   * the product is rescaled before the bias.  Those blocks carry no gradient, so nothing else changes.  bf16 models
+   * with dim a multiple of 16; 0 (the default) keeps every layer in bf16. */
+  int32_t frozen_fp8;
 } bsr_config;
 
 /* HBM footprint of a created handle, in bytes. */
@@ -146,7 +153,8 @@ int32_t bsr_set_param(bsr_handle* h, const char* name, const void* src, size_t c
  * parameters only), "logits" ([max_batch, max classes], rows of the last step; classes a task does
  * not have hold -inf), "loss" (1 element), "scores/<l>" (Eq. 6: the head-mean classification-token attention of the
  * last step at the drop location in block l, [max_batch, M], rows of images beyond the last batch undefined),
- * "moe_experts/<l>" (the experts chosen by block l's router in the last step, [tokens routed, top_k] as floats,
+ * "fp8/blocks.<l>.attn.qkv.weight" / "fp8/blocks.<l>.mlp.fc1.weight" (frozen_fp8: the E4M3 copy of that prefix weight
+ * scaled back to float), "moe_experts/<l>" (the experts chosen by block l's router in the last step, [tokens routed, top_k] as floats,
  * best first; the last block routes only the classification rows; `count` may be any prefix of the record). */
 int32_t bsr_get_tensor(bsr_handle* h, const char* name, float* dst_dev, size_t count, void* stream);
 
@@ -304,6 +312,13 @@ int32_t bsr_gather_fuse(const void* x_dev, int32_t dtype, int32_t batch, int32_t
 int32_t bsr_linear_forward(const void* x_dev, const void* w_dev, const float* bias_dev, const void* residual_dev,
                            void* y_dev, int32_t m, int32_t n, int32_t k, int32_t dtype, int32_t act_gelu,
                            int32_t use_tensor_cores, void* stream);
+
+/* The same product with both operands rounded to E4M3 row by row, as the 8-bit prefix computes it (frozen_fp8):
+ * y = act((x_q W_q^T) * sx * sw + bias), x_q[r] = round_e4m3(x[r] / sx[r]), sx[r] = max|x[r]| / 448, likewise for the rows
+ * of W.  x [m, k], w [n, k], y [m, n] bf16, bias [n] float32 or NULL; k a multiple of 16, n of 8.  scratch_dev: at
+ * least m*k + n*k + 4*(m + n) + 1024 bytes of device memory for the quantised copies and their scales. */
+int32_t bsr_linear_forward_e4m3(const void* x_dev, const void* w_dev, const float* bias_dev, void* y_dev, int32_t m, int32_t n,
+                                int32_t k, int32_t act_gelu, void* scratch_dev, size_t scratch_bytes, void* stream);
 
 /* Backward of y = x W^T: dx = dy W (Eq. 2: needs only the weights) and dw = dy^T x (Eq. 4: needs the stored
  * input).  x [m, k], w [n, k], dy [m, n], dx [m, k] in `dtype`; dw [n, k] float32.  With

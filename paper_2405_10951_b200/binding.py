@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "BSR_OK", -1: "BSR_ERR_INVALID_ARG", -2: "BSR_ERR_UNSUPPORTED
 
 EXPORTS = ["bsr_token_schedule", "bsr_workspace_bytes", "bsr_create", "bsr_destroy", "bsr_last_error", "bsr_set_param",
            "bsr_get_tensor", "bsr_set_lr", "bsr_set_step", "bsr_train_step", "bsr_train_steps", "bsr_train_step_host", "bsr_forward_backward", "bsr_grad_buffer", "bsr_optimizer_step", "bsr_eval_forward", "bsr_get_footprint",
-           "bsr_sync_status", "bsr_selftest_wait_expiry", "bsr_set_gemm_mode", "bsr_set_graph_mode", "bsr_profile_enable", "bsr_profile_read", "bsr_profile_launches", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_backward",
+           "bsr_sync_status", "bsr_selftest_wait_expiry", "bsr_set_gemm_mode", "bsr_set_graph_mode", "bsr_profile_enable", "bsr_profile_read", "bsr_profile_launches", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_forward_e4m3", "bsr_linear_backward",
            "bsr_linear_backward_static", "bsr_static_last_error", "bsr_attention_forward"]
 
 
@@ -43,7 +43,8 @@ class bsr_config(C.Structure):
                 ("drop_block", C.c_int32 * MAX_DROPS), ("keep_num", C.c_int32 * MAX_DROPS),
                 ("keep_den", C.c_int32 * MAX_DROPS), ("fuse_mode", C.c_int32),
                 ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
-                ("weight_decay", C.c_float), ("max_batch", C.c_int32), ("optimizer", C.c_int32), ("momentum", C.c_float)]
+                ("weight_decay", C.c_float), ("max_batch", C.c_int32), ("optimizer", C.c_int32), ("momentum", C.c_float),
+                ("frozen_fp8", C.c_int32)]
 
 
 class bsr_footprint(C.Structure):
@@ -108,6 +109,7 @@ def lib() -> C.CDLL:
         L.bsr_token_select.argtypes = [f32p, i32, i32, i32, i32, f32p, i32p, i32p, vp]
         L.bsr_gather_fuse.argtypes = [vp, i32, i32, i32, i32, i32, i32p, i32p, f32p, i32, vp, vp]
         L.bsr_linear_forward.argtypes = [vp, vp, f32p, vp, vp, i32, i32, i32, i32, i32, i32, vp]
+        L.bsr_linear_forward_e4m3.argtypes = [vp, vp, f32p, vp, i32, i32, i32, i32, vp, C.c_size_t, vp]
         L.bsr_linear_backward.argtypes = [vp, vp, vp, vp, f32p, i32, i32, i32, i32, i32, f32p, C.c_size_t, vp]
         L.bsr_linear_backward_static.argtypes = [vp, vp, vp, vp, f32p, i32, i32, i32, vp]
         L.bsr_static_last_error.argtypes = []
@@ -147,6 +149,7 @@ def make_config(cfg, max_batch: Optional[int] = None) -> bsr_config:
     c.max_batch = cfg.batch if max_batch is None else max_batch
     c.optimizer = 1 if getattr(cfg, "optimizer", "adamw") == "sgd" else 0
     c.momentum = float(getattr(cfg, "momentum", 0.9))
+    c.frozen_fp8 = int(getattr(cfg, "frozen_fp8", 0))
     return c
 
 
@@ -205,6 +208,19 @@ def bsr_linear_forward(x, w, bias=None, residual=None, act_gelu: bool = False, u
     dt = DTYPE_FP32 if x.dtype == torch.float32 else DTYPE_BF16
     _check(lib().bsr_linear_forward(_ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(y), m, n, k, dt, int(act_gelu),
                                     int(use_tensor_cores), _stream()))
+    return y
+
+
+def bsr_linear_forward_e4m3(x, w, bias=None, act_gelu: bool = False):
+    """y = act(x W^T + bias) with the rows of x and W rounded to E4M3 (bf16 tensors in, bf16 out)."""
+    import torch
+    m, k = x.shape
+    n = w.shape[0]
+    y = torch.empty((m, n), dtype=torch.bfloat16, device=x.device)
+    nbytes = m * k + n * k + 4 * (m + n) + 2048
+    scratch = torch.empty(nbytes + 256, dtype=torch.uint8, device=x.device)
+    base = (scratch.data_ptr() + 255) & ~255
+    _check(lib().bsr_linear_forward_e4m3(_ptr(x), _ptr(w), _ptr(bias), _ptr(y), m, n, k, int(act_gelu), C.c_void_p(base), nbytes, _stream()))
     return y
 
 

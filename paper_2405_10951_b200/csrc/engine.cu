@@ -120,6 +120,9 @@ int validate(const bsr_config* cfg, char* err) {
   if (cfg->optimizer != BSR_OPT_ADAMW && cfg->optimizer != BSR_OPT_SGD) return set_err(err, BSR_ERR_INVALID_ARG, "unknown optimizer");
   if (cfg->optimizer == BSR_OPT_SGD && !(cfg->momentum >= 0.f && cfg->momentum < 1.f)) return set_err(err, BSR_ERR_INVALID_ARG, "momentum must lie in [0, 1)");
   if (!(d.ln_eps > 0.f)) return set_err(err, BSR_ERR_INVALID_ARG, "ln_eps must be positive");
+  if (cfg->frozen_fp8 != 0 && cfg->frozen_fp8 != 1) return set_err(err, BSR_ERR_INVALID_ARG, "frozen_fp8 must be 0 or 1");
+  if (cfg->frozen_fp8 && (d.dtype != BSR_DTYPE_BF16 || d.dim % 16 != 0))
+    return set_err(err, BSR_ERR_UNSUPPORTED, "the 8-bit prefix needs a bf16 model whose dim is a multiple of 16");
   Schedule s;
   int rc = compute_schedule(cfg, &s, err);
   if (rc != BSR_OK) return rc;
@@ -185,6 +188,9 @@ struct bsr_handle {
   uint64_t graph_captures = 0;        // how many times a step was captured (a pipeline that cycles through more buffers than the cache holds re-captures every step)
   int use_graph = 1;
   // multi-step loop and host-buffer step
+  // E4M3 copies of the QKV and first-FFN weights of the dense blocks before t0 (frozen_fp8), with a scale per row
+  std::vector<size_t> q_qkv, q_qkv_s, q_fc1, q_fc1_s;
+  size_t off_yq = 0, off_yq_s = 0;        // LayerNorm output as E4M3 rows and their scales
   std::vector<size_t> guards;            // byte offsets of the guard words after every slice
   size_t off_guard_table = 0;
   size_t off_loop = 0, off_lab_stage = 0, off_task_stage = 0;
@@ -299,6 +305,16 @@ size_t plan(bsr_handle* h) {
     if (t.trainable) nch += (int)((t.numel + ADAM_CHUNK - 1) / ADAM_CHUNK);
   h->n_chunks = nch;
   h->off_chunks = b.take((size_t)nch * sizeof(AdamChunk));
+  // 8-bit copies of the gradient-free prefix's LayerNorm-fed weights
+  h->t0 = cfg.trainable_mask ? __builtin_ctz(cfg.trainable_mask) : d.depth;
+  h->q_qkv.assign(d.depth, 0); h->q_qkv_s.assign(d.depth, 0); h->q_fc1.assign(d.depth, 0); h->q_fc1_s.assign(d.depth, 0);
+  if (cfg.frozen_fp8)
+    for (int l = 0; l < h->t0 && l < d.depth; ++l) {
+      if ((d.moe_block_mask >> l) & 1u) continue;
+      h->q_qkv[l] = b.take((size_t)3 * D * D); h->q_qkv_s[l] = b.take((size_t)3 * D * 4);
+      h->q_fc1[l] = b.take((size_t)F * D); h->q_fc1_s[l] = b.take((size_t)F * 4);
+    }
+  h->weights_bytes = b.off - w0;
   // routing record of every MoE block (kept for inspection), then the activations kept by the trainable blocks
   int E = d.moe_experts, Kx = d.moe_top_k;
   std::vector<size_t> rec_eidx(d.depth, 0), rec_ew(d.depth, 0);
@@ -413,6 +429,10 @@ size_t plan(bsr_handle* h) {
       if (!((cfg.trainable_mask >> l) & 1u)) { tb.y1 = bb.y1; tb.o = bb.o; tb.y2 = bb.y2; }
     }
   }
+  if (cfg.frozen_fp8) {
+    h->off_yq = b.take(M0 * D);
+    h->off_yq_s = b.take(M0 * 4);
+  }
   h->off_xn = b.take((size_t)Bm * D * 4);
   h->off_meanf = b.take((size_t)Bm * 4);
   h->off_rstdf = b.take((size_t)Bm * 4);
@@ -523,11 +543,21 @@ int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb
   bool shrinks = is_drop && Tf != Ta;
   Ctx cf = c;                // the residual stream is float whatever the storage dtype
   cf.dtype = 0;
-  layernorm_fwd(c, h->at<float>(bb.x_in), D, (const float*)h->wb(l, "norm1.weight"), (const float*)h->wb(l, "norm1.bias"),
-                h->base + bb.y1, 0, save ? h->at<float>(bb.mean1) : nullptr, save ? h->at<float>(bb.rstd1) : nullptr, Ma, D, d.ln_eps);
+  // gradient-free prefix with 8-bit operands: the LayerNorm output leaves as E4M3 rows and meets the E4M3 weight copy
+  const bool fp8 = !save && l < h->t0 && h->cfg.frozen_fp8 && h->q_qkv[l] != 0 && c.use_tc;
   GemmEpilogue e1;
   e1.bias = (const float*)h->wb(l, "attn.qkv.bias");
-  gemm(c, h->base + bb.y1, D, 1, h->wb(l, "attn.qkv.weight"), D, 1, h->base + bb.qkv, 0, Ma, 3 * D, D, e1);
+  if (fp8) {
+    layernorm_fwd_e4m3(c, h->at<float>(bb.x_in), D, (const float*)h->wb(l, "norm1.weight"), (const float*)h->wb(l, "norm1.bias"),
+                       h->base + h->off_yq, h->at<float>(h->off_yq_s), Ma, D, d.ln_eps);
+    if (gemm_tc_e4m3(c, h->base + h->off_yq, h->at<float>(h->off_yq_s), h->base + h->q_qkv[l], h->at<float>(h->q_qkv_s[l]),
+                     h->base + bb.qkv, Ma, 3 * D, D, e1) != 0)
+      return set_err(h->err, BSR_ERR_CUDA, "8-bit GEMM set-up failed");
+  } else {
+    layernorm_fwd(c, h->at<float>(bb.x_in), D, (const float*)h->wb(l, "norm1.weight"), (const float*)h->wb(l, "norm1.bias"),
+                  h->base + bb.y1, 0, save ? h->at<float>(bb.mean1) : nullptr, save ? h->at<float>(bb.rstd1) : nullptr, Ma, D, d.ln_eps);
+    gemm(c, h->base + bb.y1, D, 1, h->wb(l, "attn.qkv.weight"), D, 1, h->base + bb.qkv, 0, Ma, 3 * D, D, e1);
+  }
   int rc = attention_fwd(c, h->base + bb.qkv, h->base + bb.o, save ? h->at<float>(bb.lse) : nullptr,
                          is_drop ? h->at<float>(bb.p) : nullptr, B, Ta, H, hd);
   if (rc != 0) return set_err(h->err, BSR_ERR_UNSUPPORTED, "attention: %d tokens of head dimension %d do not fit this kernel", Ta, hd);
@@ -556,6 +586,21 @@ int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb
     if (shrinks)
       gather_fuse(cf, h->base + bb.xp_full, B, M, D, k, h->at<int>(bb.kept), h->at<int>(bb.dropped), h->at<float>(bb.s),
                   h->cfg.fuse_mode, h->base + bb.xp);
+  }
+  if (fp8 && !is_moe(h, l)) {
+    layernorm_fwd_e4m3(c, h->at<float>(bb.xp), D, (const float*)h->wb(l, "norm2.weight"), (const float*)h->wb(l, "norm2.bias"),
+                       h->base + h->off_yq, h->at<float>(h->off_yq_s), Mf, D, d.ln_eps);
+    GemmEpilogue q3;
+    q3.bias = (const float*)h->wb(l, "mlp.fc1.bias");
+    q3.act = 1;
+    if (gemm_tc_e4m3(c, h->base + h->off_yq, h->at<float>(h->off_yq_s), h->base + h->q_fc1[l], h->at<float>(h->q_fc1_s[l]),
+                     h->base + bb.hh, Mf, F, D, q3) != 0)
+      return set_err(h->err, BSR_ERR_CUDA, "8-bit GEMM set-up failed");
+    GemmEpilogue q4;
+    q4.bias = (const float*)h->wb(l, "mlp.fc2.bias");
+    q4.residual = h->base + bb.xp;
+    gemm(c, h->base + bb.hh, F, 1, h->wb(l, "mlp.fc2.weight"), F, 1, h->base + bb.x_out, 1, Mf, D, F, q4);
+    return BSR_OK;
   }
   layernorm_fwd(c, h->at<float>(bb.xp), D, (const float*)h->wb(l, "norm2.weight"), (const float*)h->wb(l, "norm2.bias"),
                 h->base + bb.y2, 0, save ? h->at<float>(bb.mean2) : nullptr, save ? h->at<float>(bb.rstd2) : nullptr, Mf, D, d.ln_eps);
@@ -936,6 +981,14 @@ int32_t bsr_set_param(bsr_handle* h, const char* name, const void* src, size_t c
     else if (src_dtype == BSR_DTYPE_BF16) cudaMemcpyAsync(h->base + t.w_off, src, count * 2, cudaMemcpyDeviceToDevice, c.stream);
     else convert_from_float(c, (const float*)src, h->base + t.w_off, count);
   }
+  if (h->cfg.frozen_fp8 && t.matrix && !t.trainable && t.name.rfind("blocks.", 0) == 0) {     // 8-bit copy of a prefix weight
+    int l = atoi(t.name.c_str() + 7);
+    int D = h->cfg.dims.dim, F = h->cfg.dims.mlp_hidden;
+    bool qkv = t.name.find(".attn.qkv.weight") != std::string::npos, fc1 = t.name.find(".mlp.fc1.weight") != std::string::npos;
+    if (l < h->t0 && h->q_qkv[l] != 0 && (qkv || fc1))
+      quantize_rows_e4m3(c, h->base + t.w_off, qkv ? 3 * D : F, D, h->base + (qkv ? h->q_qkv[l] : h->q_fc1[l]),
+                         h->at<float>(qkv ? h->q_qkv_s[l] : h->q_fc1_s[l]));
+  }
   return check_cuda(h, "bsr_set_param");
 }
 
@@ -957,6 +1010,18 @@ int32_t bsr_get_tensor(bsr_handle* h, const char* name, float* dst, size_t count
     size_t recorded = (size_t)h->cfg.max_batch * h->sched.tf[l] * h->cfg.dims.moe_top_k;
     if (count < 1 || count > recorded) return set_err(h->err, BSR_ERR_INVALID_ARG, "'%s' records at most %zu values, %zu asked for", name, recorded, count);
     convert_int_to_float(c.stream, h->at<int>(h->moe_rec_eidx[l]), dst, count);
+    return check_cuda(h, "bsr_get_tensor");
+  } else if (n.rfind("fp8/", 0) == 0) {
+    // the E4M3 copy of a prefix weight, scaled back to float: "fp8/blocks.<l>.attn.qkv.weight" or "...mlp.fc1.weight"
+    std::string pn = n.substr(4);
+    auto it = h->index.find(pn);
+    int l = pn.rfind("blocks.", 0) == 0 ? atoi(pn.c_str() + 7) : -1;
+    bool qkv = pn.find(".attn.qkv.weight") != std::string::npos, fc1 = pn.find(".mlp.fc1.weight") != std::string::npos;
+    if (it == h->index.end() || l < 0 || l >= h->cfg.dims.depth || !(qkv || fc1) || h->q_qkv[l] == 0)
+      return set_err(h->err, BSR_ERR_INVALID_ARG, "'%s' has no 8-bit copy", name);
+    int rows = qkv ? 3 * h->cfg.dims.dim : h->cfg.dims.mlp_hidden, cols = h->cfg.dims.dim;
+    if (count != (size_t)rows * cols) return set_err(h->err, BSR_ERR_INVALID_ARG, "'%s' has %zu elements, %zu given", name, (size_t)rows * cols, count);
+    dequantize_rows_e4m3(c, h->base + (qkv ? h->q_qkv[l] : h->q_fc1[l]), h->at<float>(qkv ? h->q_qkv_s[l] : h->q_fc1_s[l]), rows, cols, dst);
     return check_cuda(h, "bsr_get_tensor");
   } else if (n.rfind("scores/", 0) == 0) {
     int l = atoi(n.c_str() + 7);
@@ -1438,6 +1503,26 @@ int32_t bsr_linear_forward(const void* x, const void* w, const float* bias, cons
     gemm(c, x, k, 1, w, k, 1, y, 0, m, n, k, e);
   }
   return check_cuda(nullptr, "bsr_linear_forward");
+}
+
+int32_t bsr_linear_forward_e4m3(const void* x, const void* w, const float* bias, void* y, int32_t m, int32_t n, int32_t k,
+                                int32_t act_gelu, void* scratch, size_t scratch_bytes, void* stream) {
+  if (x == nullptr || w == nullptr || y == nullptr || scratch == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "null argument");
+  if (m < 1 || n < 8 || k < 16 || (k % 16) || (n % 8)) return set_err(g_error, BSR_ERR_INVALID_ARG, "need k a multiple of 16 and n a multiple of 8");
+  auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+  size_t o_xq = 0, o_wq = o_xq + up((size_t)m * k), o_xs = o_wq + up((size_t)n * k), o_ws = o_xs + up((size_t)m * 4), need = o_ws + up((size_t)n * 4);
+  if (((uintptr_t)scratch & 255) != 0 || scratch_bytes < need) return set_err(g_error, BSR_ERR_WORKSPACE_TOO_SMALL, "scratch of %zu bytes given, %zu needed (256-byte aligned)", scratch_bytes, need);
+  Ctx c = bare_ctx(BSR_DTYPE_BF16, stream);
+  c.use_tc = 1;
+  char* s0 = (char*)scratch;
+  quantize_rows_e4m3(c, x, m, k, s0 + o_xq, (float*)(s0 + o_xs));
+  quantize_rows_e4m3(c, w, n, k, s0 + o_wq, (float*)(s0 + o_ws));
+  GemmEpilogue e;
+  e.bias = bias;
+  e.act = act_gelu ? 1 : 0;
+  if (gemm_tc_e4m3(c, s0 + o_xq, (const float*)(s0 + o_xs), s0 + o_wq, (const float*)(s0 + o_ws), y, m, n, k, e) != 0)
+    return set_err(g_error, BSR_ERR_CUDA, "8-bit GEMM set-up failed");
+  return check_cuda(nullptr, "bsr_linear_forward_e4m3");
 }
 
 int32_t bsr_linear_backward(const void* x, const void* w, const void* dy, void* dx, float* dw, int32_t m, int32_t n, int32_t k,

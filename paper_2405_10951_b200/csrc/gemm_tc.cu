@@ -77,7 +77,9 @@ __device__ __forceinline__ Work decode_work(int w, int tiles_m, int tiles_n, int
   return k;
 }
 
-template <bool A_MN, bool B_MN, typename TOut, int BN>
+// FP8: both operands are E4M3 bytes, K-major; a k-slab is still 128 bytes of every row, i.e. 128 elements instead of
+// 64, and the MMA consumes 32 elements per instruction, so the staging and the descriptors are those of the bf16 kernel.
+template <bool A_MN, bool B_MN, typename TOut, int BN, bool FP8 = false>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TOut* __restrict__ C,
                int M, int N, int K, Epi ep, int tiles_m, int tiles_n, int splits, int kb_per_split, GemmGroup grp, int* status) {
@@ -94,7 +96,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  int total_kb = (K + BK - 1) / BK;
+  constexpr int BKE = FP8 ? 2 * BK : BK;             // elements of k per slab (128 bytes of a K-major row)
+  static_assert(!FP8 || (!A_MN && !B_MN), "8-bit operands are read along k");
+  int total_kb = (K + BKE - 1) / BKE;
   int work_items = tiles_m * tiles_n * splits;
 
   if (threadIdx.x == 0) {
@@ -129,13 +133,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           mbar_expect_tx(full_bar(stage), STAGE_BYTES);
           uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
           if (!A_MN) {
-            tma_load_2d(sa, &map_a, full_bar(stage), kb * BK, mt * BM);
+            tma_load_2d(sa, &map_a, full_bar(stage), kb * BKE, mt * BM);
           } else {
 #pragma unroll
             for (int j = 0; j < BM / 64; ++j) tma_load_2d(sa + j * (BK * 128), &map_a, full_bar(stage), mt * BM + j * 64, kb * BK);
           }
           if (!B_MN) {
-            tma_load_2d(sb, &map_b, full_bar(stage), kb * BK, nt * BN + wk.b_off);
+            tma_load_2d(sb, &map_b, full_bar(stage), kb * BKE, nt * BN + wk.b_off);
           } else {
 #pragma unroll
             for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * (BK * 128), &map_b, full_bar(stage), nt * BN + j * 64, kb * BK + wk.b_off);
@@ -153,7 +157,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else if (warp == 1) {
     // ------------------------------- MMA issuer ---------------------------------
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc(A_MN, B_MN, BN);
+      constexpr uint32_t idesc = FP8 ? make_idesc_e4m3(BM, BN) : make_idesc(A_MN, B_MN, BN);
       // k step of 16 inside a stage: 32 bytes along a K-major row, 16 rows of 128 bytes for an MN-major operand
       constexpr uint32_t A_KSTEP = (A_MN ? UMMA_K * 128 : UMMA_K * 2) >> 4, B_KSTEP = (B_MN ? UMMA_K * 128 : UMMA_K * 2) >> 4;
       const uint64_t desc_a0 = A_MN ? make_desc(base, BK * 128, 1024) : make_desc(base, 16, 1024);
@@ -175,10 +179,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           tc_fence_after();
           // descriptors of this stage: only the 16-byte-unit address field (low bits) moves with the stage and the k step
           uint64_t da = desc_a0 + (uint64_t)((stage * STAGE_BYTES) >> 4), db = desc_b0 + (uint64_t)((stage * STAGE_BYTES) >> 4);
-          umma_bf16(d_tmem, da, db, idesc, kb > kb0 ? 1u : 0u);
+          if (FP8) {
 #pragma unroll
-          for (int k = 1; k < BK / UMMA_K; ++k)
-            umma_bf16_acc(d_tmem, da + (uint64_t)(k * A_KSTEP), db + (uint64_t)(k * B_KSTEP), idesc);
+            for (int k = 0; k < BK / UMMA_K; ++k)       // four steps of 32 bytes along k, as for bf16
+              umma_e4m3(d_tmem, da + (uint64_t)(k * A_KSTEP), db + (uint64_t)(k * B_KSTEP), idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          } else {
+            umma_bf16(d_tmem, da, db, idesc, kb > kb0 ? 1u : 0u);
+#pragma unroll
+            for (int k = 1; k < BK / UMMA_K; ++k)
+              umma_bf16_acc(d_tmem, da + (uint64_t)(k * A_KSTEP), db + (uint64_t)(k * B_KSTEP), idesc);
+          }
           umma_commit(empty_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -374,10 +384,21 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t outer,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool A_MN, bool B_MN, typename TOut, int BN = BN_MAX>
+bool make_map_u8(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t outer, uint64_t ld, uint32_t box_outer) {
+  EncodeFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {ld};
+  cuuint32_t box[2] = {128, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool A_MN, bool B_MN, typename TOut, int BN = BN_MAX, bool FP8 = false>
 static int launch(const Ctx& c, const CUtensorMap& ma, const CUtensorMap& mb, void* C, int m, int n, int k, const Epi& ep,
                   int tiles_m, int tiles_n, int splits, int kb_per_split, const GemmGroup& grp) {
-  auto kern = gemm_tc_kernel<A_MN, B_MN, TOut, BN>;
+  auto kern = gemm_tc_kernel<A_MN, B_MN, TOut, BN, FP8>;
   static SmemLimit lim;
   if (!ensure_smem(lim, kern, SMEM_BYTES)) return -3;
   int work = tiles_m * tiles_n * splits;
@@ -529,6 +550,30 @@ int gemm_tc_grouped_wgrad(const Ctx& c, const void* dY, const void* X, float* dW
   ep.bias = nullptr; ep.residual = nullptr; ep.aux_out = nullptr; ep.aux_in = nullptr; ep.act = 0;
   if (c.prof != nullptr && c.prof->on) c.prof->begin(c.stream, 2.0 * rows_cap * n * (double)m);
   int rc = launch<true, true, float>(c, ma, mb, dW, m, n, rows_cap, ep, ceil_div(m, BM), ceil_div(n, BN_MAX), experts, 0, g);
+  if (c.prof != nullptr && c.prof->on) c.prof->end(c.stream);
+  return rc;
+}
+
+// C[m, n] (bf16) = epilogue(a_scale[row] * b_scale[col] * sum_k Aq(m, k) * Bq(n, k)): E4M3 operands, one byte each, k contiguous.
+int gemm_tc_e4m3(const Ctx& c, const void* Aq, const float* a_scale, const void* Bq, const float* b_scale, void* C, int m, int n,
+                 int k, const GemmEpilogue& e) {
+  using namespace tc;
+  if ((k % 16) != 0 || (n % 8) != 0 || ((uintptr_t)Aq & 15) || ((uintptr_t)Bq & 15) || ((uintptr_t)C & 15)) return -1;
+  if (a_scale == nullptr || b_scale == nullptr || e.residual != nullptr || e.act == 2) return -1;
+  int sms = c.sm_count > 0 ? c.sm_count : 148;
+  int bn = BN_MAX;
+  long w256 = (long)ceil_div(ceil_div(m, BM) * ceil_div(n, 256), sms) * 256, w192 = (long)ceil_div(ceil_div(m, BM) * ceil_div(n, 192), sms) * 192;
+  if (w192 < w256) bn = 192;
+  CUtensorMap ma, mb;
+  if (!make_map_u8(&ma, Aq, (uint64_t)k, (uint64_t)m, (uint64_t)k, BM) || !make_map_u8(&mb, Bq, (uint64_t)k, (uint64_t)n, (uint64_t)k, bn)) return -2;
+  Epi ep;
+  ep.bias = e.bias; ep.aux_out = e.aux_out; ep.act = e.act; ep.row_scale = a_scale; ep.col_scale = b_scale;
+  int tiles_m = ceil_div(m, BM), tiles_n = ceil_div(n, bn);
+  int total_kb = ceil_div(k, 2 * BK);
+  GemmGroup gg;
+  if (c.prof != nullptr && c.prof->on) c.prof->begin(c.stream, 2.0 * m * n * (double)k);
+  int rc = bn == 192 ? launch<false, false, bf16, 192, true>(c, ma, mb, C, m, n, k, ep, tiles_m, tiles_n, 1, total_kb, gg)
+                     : launch<false, false, bf16, 256, true>(c, ma, mb, C, m, n, k, ep, tiles_m, tiles_n, 1, total_kb, gg);
   if (c.prof != nullptr && c.prof->on) c.prof->end(c.stream);
   return rc;
 }

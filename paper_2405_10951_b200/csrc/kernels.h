@@ -101,6 +101,17 @@ void gemm(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long
 bool gemm_tc_supported(int m, int n, int k);
 int gemm_tc(const Ctx& c, const void* A, const void* B, void* C, int out_is_float, int m, int n, int k,
             const GemmEpilogue& e);
+// E4M3 operands (one byte per element, k contiguous), one float scale per row of A and per row of B; bf16 output.
+// e: bias, GELU (act 1) and the stored pre-activation; no residual.  k a multiple of 16, n of 8.
+int gemm_tc_e4m3(const Ctx& c, const void* Aq, const float* a_scale, const void* Bq, const float* b_scale, void* C, int m, int n,
+                 int k, const GemmEpilogue& e);
+// Rows of x [rows, cols] (bf16) to E4M3 with scale[r] = max|row| / 448 (1 for a zero row): q = round(x / scale).
+void quantize_rows_e4m3(const Ctx& c, const void* x, int rows, int cols, void* q, float* scale);
+// q * scale back to float (for inspection).
+void dequantize_rows_e4m3(const Ctx& c, const void* q, const float* scale, int rows, int cols, float* out);
+// LayerNorm forward with the normalised row written as E4M3 and its scale (max|y| / 448) beside it.
+void layernorm_fwd_e4m3(const Ctx& c, const float* x, long x_stride, const float* g, const float* b, void* yq, float* y_scale,
+                        int rows, int D, float eps);
 // Same with operand strides as in gemm(); each operand contiguous along k or along its own index.  A problem
 // with few output tiles and a long k (weight gradients) is split along k into split_ws and reduced in order.
 int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const void* B, long b_rs, long b_cs, void* C,

@@ -176,6 +176,132 @@ void layernorm_fwd(const Ctx& c, const float* x, long x_stride, const float* g, 
   else launch_ln_fwd<bf16>(c, x, x_stride, g, b, (bf16*)y, mean, rstd, rows, D, eps);
 }
 
+// ------------------------------------------------------------------------------------------------
+// E4M3 (8-bit floating point: 1 sign, 4 exponent, 3 mantissa bits, largest magnitude 448) rows with one scale each.
+// ------------------------------------------------------------------------------------------------
+// Two floats to two E4M3 bytes, round to nearest even, saturating; a in the low byte.
+__device__ __forceinline__ uint16_t to_e4m3x2(float a, float b) {
+  uint16_t r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(b), "f"(a));
+  return r;
+}
+__device__ __forceinline__ uint32_t to_e4m3x4(const float* v, float s) {
+  return (uint32_t)to_e4m3x2(__fdiv_rn(v[0], s), __fdiv_rn(v[1], s)) | ((uint32_t)to_e4m3x2(__fdiv_rn(v[2], s), __fdiv_rn(v[3], s)) << 16);
+}
+__device__ __forceinline__ float e4m3_scale(float amax) { return amax > 0.f ? __fdiv_rn(amax, 448.0f) : 1.0f; }
+
+// One warp per row (cols % 4 == 0): scale = max|row| / 448, q = round(x / scale).
+__global__ void quantize_rows_e4m3_kernel(const bf16* __restrict__ x, int rows, int cols, uint8_t* __restrict__ q, float* __restrict__ scale) {
+  int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= rows) return;
+  const bf16* xr = x + (size_t)warp * cols;
+  float amax = 0.f;
+  for (int ch = lane; ch < cols / 4; ch += 32) {
+    float v[4];
+    load4(xr + ch * 4, v);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) amax = fmaxf(amax, fabsf(v[j]));
+  }
+  amax = warp_max(amax);
+  float s = e4m3_scale(amax);
+  if (lane == 0) scale[warp] = s;
+  uint32_t* qr = reinterpret_cast<uint32_t*>(q + (size_t)warp * cols);
+  for (int ch = lane; ch < cols / 4; ch += 32) {
+    float v[4];
+    load4(xr + ch * 4, v);
+    qr[ch] = to_e4m3x4(v, s);
+  }
+}
+void quantize_rows_e4m3(const Ctx& c, const void* x, int rows, int cols, void* q, float* scale) {
+  note_launch(1);
+  quantize_rows_e4m3_kernel<<<ceil_div((long)rows * 32, 256), 256, 0, c.stream>>>((const bf16*)x, rows, cols, (uint8_t*)q, scale);
+}
+
+// E4M3 byte to float: sign, exponent (bias 7) and mantissa unpacked by hand (subnormals: exponent field 0).
+__device__ __forceinline__ float from_e4m3(uint8_t b) {
+  int e = (b >> 3) & 15, m = b & 7;
+  float v = e == 0 ? (float)m * 0.001953125f : ldexpf(1.0f + (float)m * 0.125f, e - 7);
+  return (b & 0x80) ? -v : v;
+}
+__global__ void dequantize_rows_e4m3_kernel(const uint8_t* __restrict__ q, const float* __restrict__ scale, int rows, int cols,
+                                            float* __restrict__ out) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (size_t)rows * cols) return;
+  out[i] = from_e4m3(q[i]) * scale[i / cols];
+}
+void dequantize_rows_e4m3(const Ctx& c, const void* q, const float* scale, int rows, int cols, float* out) {
+  note_launch(1);
+  dequantize_rows_e4m3_kernel<<<ceil_div((long)rows * cols, 256), 256, 0, c.stream>>>((const uint8_t*)q, scale, rows, cols, out);
+}
+
+// LayerNorm forward whose output row goes out as E4M3 with scale max|y| / 448: the row is already in the warp's
+// registers, so the quantisation costs one more warp reduction and halves the bytes written.
+template <int NCH>
+__global__ void layernorm_fwd_e4m3_kernel(const float* __restrict__ x, long x_stride, const float* __restrict__ g,
+                                          const float* __restrict__ b, uint8_t* __restrict__ yq, float* __restrict__ y_scale,
+                                          int rows, int D, float eps) {
+  int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  int lane = threadIdx.x & 31;
+  if (warp >= rows) return;
+  const float* xr = x + (long)warp * x_stride;
+  int chunks = D / 4;
+  float v[(NCH * 4)];
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    int ch = lane + i * 32;
+    if (ch < chunks) {
+      load16(xr + ch * 4, v + i * 4);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) sum += v[i * 4 + j];
+    }
+  }
+  float mu = warp_sum(sum) / (float)D;
+  float sq = 0.f;
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    int ch = lane + i * 32;
+    if (ch < chunks) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { float t = v[i * 4 + j] - mu; sq += t * t; }
+    }
+  }
+  float rs = rsqrtf(warp_sum(sq) / (float)D + eps);
+  float amax = 0.f;
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    int ch = lane + i * 32;
+    if (ch < chunks) {
+      float4 gg = *reinterpret_cast<const float4*>(g + ch * 4), bb = *reinterpret_cast<const float4*>(b + ch * 4);
+      v[i * 4 + 0] = (v[i * 4 + 0] - mu) * rs * gg.x + bb.x;
+      v[i * 4 + 1] = (v[i * 4 + 1] - mu) * rs * gg.y + bb.y;
+      v[i * 4 + 2] = (v[i * 4 + 2] - mu) * rs * gg.z + bb.z;
+      v[i * 4 + 3] = (v[i * 4 + 3] - mu) * rs * gg.w + bb.w;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) amax = fmaxf(amax, fabsf(v[i * 4 + j]));
+    }
+  }
+  amax = warp_max(amax);
+  float s = e4m3_scale(amax);
+  if (lane == 0) y_scale[warp] = s;
+  uint32_t* qr = reinterpret_cast<uint32_t*>(yq + (size_t)warp * D);
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    int ch = lane + i * 32;
+    if (ch < chunks) qr[ch] = to_e4m3x4(v + i * 4, s);
+  }
+}
+void layernorm_fwd_e4m3(const Ctx& c, const float* x, long x_stride, const float* g, const float* b, void* yq, float* y_scale,
+                        int rows, int D, float eps) {
+  note_launch(1);
+  int threads = 256;
+  int blocks = ceil_div((long)rows * 32, threads);
+  int nch = ceil_div(D, 128);
+#define BSR_LN_Q(N) layernorm_fwd_e4m3_kernel<N><<<blocks, threads, 0, c.stream>>>(x, x_stride, g, b, (uint8_t*)yq, y_scale, rows, D, eps)
+  if (nch <= 2) BSR_LN_Q(2); else if (nch == 3) BSR_LN_Q(3); else if (nch == 4) BSR_LN_Q(4); else if (nch <= 6) BSR_LN_Q(6); else BSR_LN_Q(8);
+#undef BSR_LN_Q
+}
+
 // Backward.  Each block owns rows blockIdx.x*8 + warp, stepping by gridDim.x*8; every lane accumulates the
 // dgamma/dbeta contributions of its columns, warps are combined through shared memory in warp order, and the
 // block's sums go to partials[0][block][col] (dgamma) and partials[1][block][col] (dbeta).

@@ -9,11 +9,15 @@ namespace bsr {
 namespace tc {
 
 struct Epi {
-  const float* bias;
-  const void* residual;
-  void* aux_out;
-  const void* aux_in;
-  int act;
+  const float* bias = nullptr;
+  const void* residual = nullptr;
+  void* aux_out = nullptr;
+  const void* aux_in = nullptr;
+  int act = 0;
+  // operands quantised with one scale per row of A and per row of B (8-bit floating point): the accumulator of
+  // (row, col) is multiplied by row_scale[row] * col_scale[col] before the bias
+  const float* row_scale = nullptr;
+  const float* col_scale = nullptr;
 };
 
 // Two fp32 lanes per instruction (fma.rn.f32x2 and friends): halves the issue slots of the polynomial below.
@@ -184,6 +188,16 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t* r, const Epi& ep,
     float v[32];
 #pragma unroll
     for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+    if (ep.row_scale != nullptr) {
+      float rs = row0 + lane < M ? __ldg(ep.row_scale + row0 + lane) : 0.f;
+#pragma unroll
+      for (int g = 0; g < 8; ++g) {
+        if (col0 + g * 4 < N) {
+          float4 cs = __ldg(reinterpret_cast<const float4*>(ep.col_scale + col0 + g * 4));
+          v[g * 4 + 0] *= rs * cs.x; v[g * 4 + 1] *= rs * cs.y; v[g * 4 + 2] *= rs * cs.z; v[g * 4 + 3] *= rs * cs.w;
+        }
+      }
+    }
     if (ep.bias != nullptr) {
 #pragma unroll
       for (int g = 0; g < 8; ++g) {

@@ -119,3 +119,30 @@ def test_linear_backward_fp32():
     torch.cuda.synchronize()
     assert rel(dx.cpu().numpy().astype(np.float64), dx_ref) < 2e-6
     assert rel(dw.cpu().numpy().astype(np.float64), dw_ref) < 2e-6
+
+
+@pytest.mark.parametrize("m,n,k", [(128, 256, 128), (197, 384, 192), (1000, 3072, 768), (2600, 2304, 768), (100, 72, 48), (9216, 3072, 768)])
+@pytest.mark.parametrize("gelu", [False, True])
+def test_linear_e4m3_tensor_cores(m, n, k, gelu):
+    """tcgen05 kind::f8f6f4 on row-quantised E4M3 operands against the oracle's statement of the same product: the
+    inputs are bf16 on both sides, so the 8-bit codes agree exactly and what is left is fp32 accumulation order and the
+    bf16 rounding of the output."""
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    rng = np.random.default_rng(m + 3 * n + 7 * k)
+    x = synth.round_to_bf16(rng.standard_normal((m, k)) * np.exp(rng.standard_normal((m, 1))))      # rows of different scale
+    w = synth.round_to_bf16(rng.standard_normal((n, k)) / np.sqrt(k))
+    bias = rng.standard_normal(n)
+    want = O.linear_e4m3(x, w, bias)
+    if gelu:
+        want = O.gelu(want)
+    g = lambda a: torch.as_tensor(a.astype(np.float32)).cuda().to(torch.bfloat16)
+    y = Bd.bsr_linear_forward_e4m3(g(x), g(w), torch.as_tensor(bias.astype(np.float32)).cuda(), act_gelu=gelu)
+    torch.cuda.synchronize()
+    got = y.float().cpu().numpy().astype(np.float64)
+    assert rel(got, want) < 4e-3
+    # and it is the quantised product, not the bf16 one: the two differ by a few percent
+    plain = O.linear(x, w, bias)
+    if gelu:
+        plain = O.gelu(plain)
+    assert rel(got, plain) > 5 * rel(got, want)

@@ -90,6 +90,44 @@ def test_eval_forward_matches_oracle_and_train_forward():
     assert torch.equal(logits3, logits[:3])
 
 
+FP8_CASES = {
+    "mini": MINI_BF16.with_(frozen_fp8=1),
+    "deit_s_batch4": CONFIGS["deit_s"].with_(batch=4, frozen_fp8=1),
+    "vit_b_batch3": CONFIGS["vit_b"].with_(batch=3, frozen_fp8=1),
+    "head_only_all_blocks_8bit": MINI_BF16.with_(trainable=(), frozen_fp8=1),
+}
+
+
+@pytest.mark.parametrize("case", list(FP8_CASES))
+def test_step_with_e4m3_prefix_matches_the_oracle(case):
+    """frozen_fp8: the LayerNorm-fed layers of the gradient-free prefix on E4M3 operands, against the oracle computing
+    the same quantised products.  The stored 8-bit weights equal the oracle's bit for bit, and on identical inputs the
+    quantised product agrees to bf16 rounding (test_linear_e4m3_tensor_cores).  Across a whole step the two sides
+    quantise LayerNorm outputs that already differ by bf16 rounding (delta ~ 3e-3): a fraction delta / 2^-4 of the
+    8-bit codes lands one step (6-12 %) apart, an rms perturbation of about sqrt(delta * step) ~ 1.5 % per quantised
+    layer that does not average out in the products.  With two such layers in each of the t0 prefix blocks the
+    deviations add to 1.5 % * sqrt(2 t0): measured 3.7 % (t0 = 3) to 5.7 % (t0 = 8) on the worst gradient.  The
+    tolerance is 2 % * sqrt(2 t0)."""
+    cfg = FP8_CASES[case]
+    images, labels, task_ids, params = synth.make_workload(cfg, peaked=False)
+    gpu = P.run_gpu_step(cfg, images, labels, task_ids, params)
+    eng = gpu["engine"]
+    if min(cfg.trainable, default=cfg.depth) > 0:
+        for n in ("blocks.0.attn.qkv.weight", "blocks.0.mlp.fc1.weight"):
+            shape = synth.param_shapes(cfg)[n]
+            got = eng.get_tensor("fp8/" + n, shape).cpu().numpy().astype(np.float64)
+            assert np.array_equal(got, O.quantize_rows_e4m3(params[n])[0].astype(np.float32).astype(np.float64)), n
+    t0 = min(cfg.trainable, default=cfg.depth)
+    tol = P.BF16_TOL * float(np.sqrt(2 * t0))
+    rep = P.compare_step(cfg, images, labels, task_ids, params, gpu, tol, P.BF16_EXACT_MARGIN_PEAKED, P.BF16_SCORE_TOL_PEAKED)
+    print(case, rep)
+    # for the record: how far the unquantised oracle is (the quantisation itself moves the logits by about as much as
+    # the code flips do, so this whole-step figure cannot tell the two apart sharply; the unit test of the product can)
+    plain = O.forward(cfg.with_(frozen_fp8=0), params, images, forced_keep=gpu["kept"])
+    fin = np.isfinite(plain["logits"])
+    print(case, "against the unquantised oracle:", P.rel_err(gpu["logits"][fin], plain["logits"][fin]))
+
+
 @pytest.mark.parametrize("peaked", [False, True])
 def test_eval_forward_bf16_matches_oracle(peaked):
     """bsr_eval_forward on the tcgen05 path (ViT-B/16 shapes, three images): logits against the oracle run with the
