@@ -1,10 +1,10 @@
 """Stand-alone timing of single kernels of the BSR step through the C ABI.
 
-    python -m paper_2405_10951_b200.microbench gemm --m 25216 --n 2304 --k 768 [--gelu] [--mode 1|2] [--iters 20]
-    python -m paper_2405_10951_b200.microbench backward --m 12800 --n 2304 --k 768
-    python -m paper_2405_10951_b200.microbench select_gather --batch 4096 --heads 12 --tokens 197 --dim 768 --keep 0.7
-    python -m paper_2405_10951_b200.microbench attention --batch 128 --heads 12 --tokens 197
-    python -m paper_2405_10951_b200.microbench step --workload vit_b --batch 32 --iters 4
+    python microbench.py gemm --m 25216 --n 2304 --k 768 [--gelu] [--e4m3] [--mode 1|2] [--iters 20]
+    python microbench.py backward --m 12800 --n 2304 --k 768
+    python microbench.py select_gather --batch 4096 --heads 12 --tokens 197 --dim 768 --keep 0.7
+    python microbench.py attention --batch 128 --heads 12 --tokens 197
+    python microbench.py step --workload vit_b --batch 32 --iters 4
 
 Each prints one JSON line with the time per launch (CUDA events on the current stream, after warm-up) and the
 achieved TFLOP/s or GB/s on the kernel's algorithmic work.  Inputs are seeded and synthetic.
@@ -15,9 +15,13 @@ import argparse
 import json
 import math
 
+import os
+import sys
+
 import torch
 
-from . import binding as Bd
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+from paper_2405_10951_b200 import binding as Bd  # noqa: E402
 
 
 def timed(fn, iters, flush=None):
@@ -46,6 +50,7 @@ def main():
     ap.add_argument("--k", type=int, default=768)
     ap.add_argument("--gelu", action="store_true")
     ap.add_argument("--residual", action="store_true")
+    ap.add_argument("--e4m3", action="store_true", help="gemm: operands rounded to E4M3 row by row (the 8-bit prefix's product)")
     ap.add_argument("--mode", type=int, default=1)
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--batch", type=int, default=4096)
@@ -62,7 +67,7 @@ def main():
     out = {"kernel": a.what}
     if a.what == "step":
         # whole fine-tuning steps of a named workload at a chosen batch: the launch sequence a profiler is pointed at
-        from . import synth
+        from paper_2405_10951_b200 import synth
         cfg = synth.CONFIGS[a.workload]
         cfg = cfg.with_(batch=min(a.batch, cfg.batch))
         images, labels, task_ids, params = synth.make_workload(cfg)
@@ -79,8 +84,11 @@ def main():
         w = (torch.randn(a.n, a.k, device=dev) / math.sqrt(a.k)).bfloat16()
         b = torch.randn(a.n, device=dev)
         r = torch.randn(a.m, a.n, device=dev).bfloat16() if a.residual else None
-        ms = timed(lambda: Bd.bsr_linear_forward(x, w, b, r, act_gelu=a.gelu, use_tensor_cores=a.mode), a.iters, flush)
-        out.update(m=a.m, n=a.n, k=a.k, gelu=a.gelu, mode=a.mode, us=ms * 1e3, tflops=2.0 * a.m * a.n * a.k / ms / 1e9)
+        if a.e4m3:
+            ms = timed(lambda: Bd.bsr_linear_forward_e4m3(x, w, b, act_gelu=a.gelu), a.iters, flush)     # includes the two row-quantisation passes
+        else:
+            ms = timed(lambda: Bd.bsr_linear_forward(x, w, b, r, act_gelu=a.gelu, use_tensor_cores=a.mode), a.iters, flush)
+        out.update(m=a.m, n=a.n, k=a.k, gelu=a.gelu, mode=a.mode, e4m3=a.e4m3, us=ms * 1e3, tflops=2.0 * a.m * a.n * a.k / ms / 1e9)
     elif a.what == "backward":
         x = torch.randn(a.m, a.k, device=dev).bfloat16()
         w = (torch.randn(a.n, a.k, device=dev) / math.sqrt(a.k)).bfloat16()

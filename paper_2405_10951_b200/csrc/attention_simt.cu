@@ -323,7 +323,7 @@ int attention_bwd(const Ctx& c, const void* qkv, const void* out, const void* do
 // takes row 0), so its attention reduces to one query per (image, head): o_0 = sum_j p_j v_j with p = softmax(q_0 K^T
 // / sqrt(d)) (Eq. 1, first row), and in the backward pass only that row carries a gradient: dV_j = p_j dO_0,
 // dS_j = p_j (dO_0 . v_j - sum_i p_i dO_0 . v_i), dK_j = dS_j q_0 / sqrt(d), dQ_0 = sum_j dS_j k_j / sqrt(d), every
-// other row of dQ is zero.  One warp per (image, head); the probabilities are recomputed in the backward kernel.
+// other row of dQ is zero.  One block per (image, head); the probabilities are recomputed in the backward kernel.
 // ---------------------------------------------------------------------------------------------
 constexpr int ATC_WARPS = 4;
 constexpr int ATC_MAXKEYS = 32 * 20;             // keys per lane held in registers: up to 640 tokens
@@ -370,48 +370,58 @@ __device__ __forceinline__ void cls_row_probs(const T* kbase, long row_stride, c
   for (int i = 0; i < KPL; ++i) p[i] *= inv;
 }
 
+// One block of ATC_WARPS warps per (image, head): every warp forms the softmax row (cheap, and it spares a block-wide
+// exchange), then the warps share the keys of the second phase (warp w takes keys w, w + ATC_WARPS, ...) and their
+// partial sums are combined through shared memory in warp order.
 template <typename T, int KPL>
 __global__ void __launch_bounds__(ATC_WARPS * 32)
 attn_cls_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ out_cls, int B, int T_, int H, int d) {
-  __shared__ float qs[ATC_WARPS][AT_MAXD];
+  __shared__ float qs[AT_MAXD];
+  __shared__ float part[ATC_WARPS][AT_MAXD];
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  int pair = blockIdx.x * ATC_WARPS + warp;
-  if (pair >= B * H) return;
+  int pair = blockIdx.x;
   int b = pair / H, h = pair % H;
   long row_stride = 3L * H * d;
   const T* base = qkv + (long)b * T_ * row_stride + (long)h * d;
-  if (2 * lane < d) {
+  if (warp == 0 && 2 * lane < d) {
     float2 q = ld_pair<T>(base + 2 * lane);
-    qs[warp][2 * lane] = q.x; qs[warp][2 * lane + 1] = q.y;
+    qs[2 * lane] = q.x; qs[2 * lane + 1] = q.y;
   }
-  __syncwarp();
+  __syncthreads();
   float p[KPL];
-  cls_row_probs<T, KPL>(base + (long)H * d, row_stride, qs[warp], T_, d, rsqrtf((float)d), lane, p);
-  // o_0 = sum_j p_j v_j: every lane owns two feature indices, the keys are walked in order
+  cls_row_probs<T, KPL>(base + (long)H * d, row_stride, qs, T_, d, rsqrtf((float)d), lane, p);
+  // o_0 = sum_j p_j v_j: every lane owns two feature indices; this warp's keys in order
   float o0 = 0.f, o1 = 0.f;
   const T* vbase = base + 2L * H * d;
 #pragma unroll
   for (int i = 0; i < KPL; ++i) {
-    for (int l = 0; l < 32; ++l) {
+#pragma unroll 4
+    for (int l = warp; l < 32; l += ATC_WARPS) {
       int j = l + 32 * i;
-      if (j >= T_) break;
       float pj = __shfl_sync(0xffffffffu, p[i], l);
-      if (2 * lane < d) {
+      if (j < T_ && 2 * lane < d) {
         float2 v = ld_pair<T>(vbase + (long)j * row_stride + 2 * lane);
         o0 = fmaf(pj, v.x, o0); o1 = fmaf(pj, v.y, o1);
       }
     }
   }
-  if (2 * lane < d) st_pair<T>(out_cls + (long)b * H * d + (long)h * d + 2 * lane, o0, o1);
+  if (2 * lane < d) { part[warp][2 * lane] = o0; part[warp][2 * lane + 1] = o1; }
+  __syncthreads();
+  if (warp == 0 && 2 * lane < d) {
+    float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+    for (int w = 0; w < ATC_WARPS; ++w) { a0 += part[w][2 * lane]; a1 += part[w][2 * lane + 1]; }
+    st_pair<T>(out_cls + (long)b * H * d + (long)h * d + 2 * lane, a0, a1);
+  }
 }
 
 template <typename T, int KPL>
 __global__ void __launch_bounds__(ATC_WARPS * 32)
 attn_cls_bwd_kernel(const T* __restrict__ qkv, const T* __restrict__ dout_cls, T* __restrict__ dqkv, int B, int T_, int H, int d) {
-  __shared__ float qs[ATC_WARPS][AT_MAXD], gs[ATC_WARPS][AT_MAXD];
+  __shared__ float qs[AT_MAXD], gs[AT_MAXD];
+  __shared__ float part[ATC_WARPS][AT_MAXD];
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  int pair = blockIdx.x * ATC_WARPS + warp;
-  if (pair >= B * H) return;
+  int pair = blockIdx.x;
   int b = pair / H, h = pair % H;
   long row_stride = 3L * H * d;
   const T* base = qkv + (long)b * T_ * row_stride + (long)h * d;
@@ -421,13 +431,15 @@ attn_cls_bwd_kernel(const T* __restrict__ qkv, const T* __restrict__ dout_cls, T
     float2 q = ld_pair<T>(base + 2 * lane);
     float2 g = ld_pair<T>(dout_cls + (long)b * H * d + (long)h * d + 2 * lane);
     q0 = q.x; q1 = q.y; g0 = g.x; g1 = g.y;
-    qs[warp][2 * lane] = q0; qs[warp][2 * lane + 1] = q1;
-    gs[warp][2 * lane] = g0; gs[warp][2 * lane + 1] = g1;
+    if (warp == 0) {
+      qs[2 * lane] = q0; qs[2 * lane + 1] = q1;
+      gs[2 * lane] = g0; gs[2 * lane + 1] = g1;
+    }
   }
-  __syncwarp();
+  __syncthreads();
   float scale = rsqrtf((float)d);
   float p[KPL], ds[KPL];
-  cls_row_probs<T, KPL>(base + (long)H * d, row_stride, qs[warp], T_, d, scale, lane, p);
+  cls_row_probs<T, KPL>(base + (long)H * d, row_stride, qs, T_, d, scale, lane, p);
   // dP_j = dO_0 . v_j for the lane's keys, delta = sum_j p_j dP_j
   const T* vbase = base + 2L * H * d;
   float delta = 0.f;
@@ -440,8 +452,8 @@ attn_cls_bwd_kernel(const T* __restrict__ qkv, const T* __restrict__ dout_cls, T
       float s = 0.f;
       for (int e = 0; e < d; e += 2) {
         float2 v = ld_pair<T>(row + e);
-        s = fmaf(gs[warp][e], v.x, s);
-        s = fmaf(gs[warp][e + 1], v.y, s);
+        s = fmaf(gs[e], v.x, s);
+        s = fmaf(gs[e + 1], v.y, s);
       }
       ds[i] = s;
       delta += p[i] * s;
@@ -450,17 +462,17 @@ attn_cls_bwd_kernel(const T* __restrict__ qkv, const T* __restrict__ dout_cls, T
   delta = warp_sum(delta);
 #pragma unroll
   for (int i = 0; i < KPL; ++i) ds[i] = p[i] * (ds[i] - delta) * scale;      // dS_j / sqrt(d)
-  // rows: dV_j = p_j dO_0, dK_j = dS_j q_0 / sqrt(d), dQ_0 = sum_j dS_j k_j / sqrt(d), dQ_j = 0 for j > 0
+  // rows of this warp's keys: dV_j = p_j dO_0, dK_j = dS_j q_0 / sqrt(d), dQ_j = 0 for j > 0; dQ_0 = sum_j dS_j k_j / sqrt(d)
   float dq0 = 0.f, dq1 = 0.f;
   const T* kbase = base + (long)H * d;
 #pragma unroll
   for (int i = 0; i < KPL; ++i) {
-    for (int l = 0; l < 32; ++l) {
+#pragma unroll 4
+    for (int l = warp; l < 32; l += ATC_WARPS) {
       int j = l + 32 * i;
-      if (j >= T_) break;
       float pj = __shfl_sync(0xffffffffu, p[i], l);
       float dsj = __shfl_sync(0xffffffffu, ds[i], l);
-      if (2 * lane < d) {
+      if (j < T_ && 2 * lane < d) {
         float2 k = ld_pair<T>(kbase + (long)j * row_stride + 2 * lane);
         dq0 = fmaf(dsj, k.x, dq0); dq1 = fmaf(dsj, k.y, dq1);
         T* drow = dbase + (long)j * row_stride + 2 * lane;
@@ -470,13 +482,20 @@ attn_cls_bwd_kernel(const T* __restrict__ qkv, const T* __restrict__ dout_cls, T
       }
     }
   }
-  if (2 * lane < d) st_pair<T>(dbase + 2 * lane, dq0, dq1);
+  if (2 * lane < d) { part[warp][2 * lane] = dq0; part[warp][2 * lane + 1] = dq1; }
+  __syncthreads();
+  if (warp == 0 && 2 * lane < d) {
+    float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+    for (int w = 0; w < ATC_WARPS; ++w) { a0 += part[w][2 * lane]; a1 += part[w][2 * lane + 1]; }
+    st_pair<T>(dbase + 2 * lane, a0, a1);
+  }
 }
 
 template <typename T>
 static int launch_cls(const Ctx& c, bool bwd, const void* qkv, const void* io_cls, void* dqkv, int B, int T_, int H, int d) {
   if (d > AT_MAXD || (d % 2) != 0 || T_ < 1 || T_ > ATC_MAXKEYS) return -2;
-  int blocks = ceil_div((long)B * H, ATC_WARPS);
+  int blocks = B * H;
   note_launch(1);
 #define BSR_CLS(KPL)                                                                                                              \
   do {                                                                                                                            \

@@ -20,7 +20,7 @@ constexpr int AT_BOX = 64;                       // rows per TMA box
 constexpr int AT_BOX_BYTES = AT_BOX * AT_D * 2;  // 8 KB
 constexpr int AT_QROWS = 128;
 constexpr int AT_MAXKEYS = 256;
-constexpr int AT_LONG_KB = 128;                  // keys per block of the two-walk kernel for longer sequences
+constexpr int AT_LONG_KB = 64;                   // keys per block of the two-walk kernel for longer sequences (four CTAs per SM)
 
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -370,7 +370,7 @@ attn_fwd_tc_long_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __res
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
-    tmem_alloc(smem_u32(&tmem_slot), 2 * KB);           // S in the first KB columns, O behind it: two CTAs share an SM
+    tmem_alloc(smem_u32(&tmem_slot), 2 * KB);           // S in the first KB columns, O behind it: several CTAs share an SM
     tmem_relinquish();
   }
   tc_fence_before();

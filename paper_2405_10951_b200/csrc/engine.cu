@@ -558,15 +558,19 @@ int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb
                   h->base + bb.y1, 0, save ? h->at<float>(bb.mean1) : nullptr, save ? h->at<float>(bb.rstd1) : nullptr, Ma, D, d.ln_eps);
     gemm(c, h->base + bb.y1, D, 1, h->wb(l, "attn.qkv.weight"), D, 1, h->base + bb.qkv, 0, Ma, 3 * D, D, e1);
   }
-  int rc = attention_fwd(c, h->base + bb.qkv, h->base + bb.o, save ? h->at<float>(bb.lse) : nullptr,
-                         is_drop ? h->at<float>(bb.p) : nullptr, B, Ta, H, hd);
-  if (rc != 0) return set_err(h->err, BSR_ERR_UNSUPPORTED, "attention: %d tokens of head dimension %d do not fit this kernel", Ta, hd);
   size_t es = dtype_size(d.dtype);
   bool tail = cls_tail(h, l);
+  // the last block needs the classification query only (its other outputs feed nothing)
+  bool cls_attn = tail && attention_cls_fwd(c, h->base + bb.qkv, h->base + bb.o_cls, B, Ta, H, hd) == 0;
+  if (!cls_attn) {
+    int rc = attention_fwd(c, h->base + bb.qkv, h->base + bb.o, save ? h->at<float>(bb.lse) : nullptr,
+                           is_drop ? h->at<float>(bb.p) : nullptr, B, Ta, H, hd);
+    if (rc != 0) return set_err(h->err, BSR_ERR_UNSUPPORTED, "attention: %d tokens of head dimension %d do not fit this kernel", Ta, hd);
+  }
   const void* proj_in = h->base + bb.o;
   const void* proj_res = h->base + bb.x_in;
   if (tail) {                  // from here on: B rows
-    copy_rows(c.stream, h->base + bb.o, (long)Ta * D * es, h->base + bb.o_cls, (long)D * es, B, (int)(D * es));
+    if (!cls_attn) copy_rows(c.stream, h->base + bb.o, (long)Ta * D * es, h->base + bb.o_cls, (long)D * es, B, (int)(D * es));
     copy_rows(c.stream, h->base + bb.x_in, (long)Ta * D * 4, h->base + bb.xin_cls, (long)D * 4, B, D * 4);
     proj_in = h->base + bb.o_cls;
     proj_res = h->base + bb.xin_cls;

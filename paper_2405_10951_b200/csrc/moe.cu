@@ -16,14 +16,16 @@ constexpr int MOE_MAX_E = 32;
 constexpr int MOE_MAX_K = 4;
 
 // ---- routing: gate logits, top-k (ties -> lower expert id), softmax over the selected logits -------------------
+constexpr int MOE_ROUTE_WARPS = 8;
 template <typename T>
-__global__ void __launch_bounds__(MOE_BLOCK_TOKENS)
+__global__ void __launch_bounds__(MOE_ROUTE_WARPS * 32)
 moe_route_kernel(const T* __restrict__ y, const T* __restrict__ wg, const int* __restrict__ task_ids, int tokens_per_image,
                  int M, int D, int E, int K, int gate_elems_in_smem, int* __restrict__ eidx, float* __restrict__ ew,
                  int* __restrict__ blk_counts) {
-  // A thread per token: its row of y against every gate row, the gate matrices of all tasks staged in shared memory
-  // when they fit (all lanes read the same gate element: a broadcast), so no cross-lane reduction is needed and the
-  // top-k is a scan over the thread's own logits.
+  // A block owns MOE_BLOCK_TOKENS consecutive tokens, a warp one token at a time: the lanes read the token's row of y
+  // in 16-byte pieces (coalesced), multiply it with the same pieces of every gate row -- the gate matrices of all tasks
+  // are staged in shared memory when they fit -- and the E partial dot products are summed over the lanes in a fixed
+  // (butterfly) order.  Lane 0 then scans the logits for the top k.
   extern __shared__ __align__(16) unsigned char route_smem[];
   __shared__ int counts[MOE_MAX_E];
   constexpr int N = Pack<T>::N;
@@ -36,15 +38,18 @@ moe_route_kernel(const T* __restrict__ y, const T* __restrict__ wg, const int* _
     gates = sg;
   }
   __syncthreads();
-  int tok = blockIdx.x * MOE_BLOCK_TOKENS + threadIdx.x;
-  if (tok < M) {
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int chunks = D / N;
+  for (int t = warp; t < MOE_BLOCK_TOKENS; t += MOE_ROUTE_WARPS) {
+    int tok = blockIdx.x * MOE_BLOCK_TOKENS + t;
+    if (tok >= M) break;
     int task = task_ids ? task_ids[tok / tokens_per_image] : 0;
     const T* yr = y + (size_t)tok * D;
     const T* gt = gates + (size_t)task * E * D;
     float acc[MOE_MAX_E];
 #pragma unroll
     for (int e = 0; e < MOE_MAX_E; ++e) acc[e] = 0.f;
-    for (int ch = 0; ch < D / N; ++ch) {
+    for (int ch = lane; ch < chunks; ch += 32) {
       float yv[N];
       load16(yr + ch * N, yv);
 #pragma unroll
@@ -57,29 +62,34 @@ moe_route_kernel(const T* __restrict__ y, const T* __restrict__ wg, const int* _
         }
       }
     }
-    float sel[MOE_MAX_K];
-    int sid[MOE_MAX_K];
-    uint32_t taken = 0;
-    for (int i = 0; i < K; ++i) {
-      float best = -INFINITY;
-      int bi = 0;
-      bool any = false;
 #pragma unroll
-      for (int e = 0; e < MOE_MAX_E; ++e) {
-        if (e < E && !((taken >> e) & 1u) && (!any || acc[e] > best)) {    // strictly greater: the lowest id wins among equals
-          best = acc[e]; bi = e; any = true;
+    for (int e = 0; e < MOE_MAX_E; ++e)
+      if (e < E) acc[e] = warp_sum(acc[e]);
+    if (lane == 0) {
+      float sel[MOE_MAX_K];
+      int sid[MOE_MAX_K];
+      uint32_t taken = 0;
+      for (int i = 0; i < K; ++i) {
+        float best = -INFINITY;
+        int bi = 0;
+        bool any = false;
+#pragma unroll
+        for (int e = 0; e < MOE_MAX_E; ++e) {
+          if (e < E && !((taken >> e) & 1u) && (!any || acc[e] > best)) {    // strictly greater: the lowest id wins among equals
+            best = acc[e]; bi = e; any = true;
+          }
         }
+        taken |= 1u << bi;
+        sel[i] = best;
+        sid[i] = bi;
       }
-      taken |= 1u << bi;
-      sel[i] = best;
-      sid[i] = bi;
-    }
-    float den = 0.f;
-    for (int i = 0; i < K; ++i) den += expf(sel[i] - sel[0]);
-    for (int i = 0; i < K; ++i) {
-      eidx[(size_t)tok * K + i] = sid[i];
-      ew[(size_t)tok * K + i] = expf(sel[i] - sel[0]) / den;
-      atomicAdd(&counts[sid[i]], 1);              // integer counts: order-independent
+      float den = 0.f;
+      for (int i = 0; i < K; ++i) den += expf(sel[i] - sel[0]);
+      for (int i = 0; i < K; ++i) {
+        eidx[(size_t)tok * K + i] = sid[i];
+        ew[(size_t)tok * K + i] = expf(sel[i] - sel[0]) / den;
+        atomicAdd(&counts[sid[i]], 1);              // integer counts: order-independent
+      }
     }
   }
   __syncthreads();
@@ -337,11 +347,11 @@ void moe_route(const Ctx& c, const MoeBufs& b, const void* y, const void* wg, co
   static SmemLimit lim[2];
   if (c.dtype == 0) {
     ensure_smem(lim[0], moe_route_kernel<float>, smem);
-    moe_route_kernel<float><<<nblk, MOE_BLOCK_TOKENS, smem, c.stream>>>((const float*)y, (const float*)wg, task_ids, tokens_per_image, M, D, E, K,
+    moe_route_kernel<float><<<nblk, MOE_ROUTE_WARPS * 32, smem, c.stream>>>((const float*)y, (const float*)wg, task_ids, tokens_per_image, M, D, E, K,
                                                                         (int)gate_elems, b.eidx, b.ew, b.blk_counts);
   } else {
     ensure_smem(lim[1], moe_route_kernel<bf16>, smem);
-    moe_route_kernel<bf16><<<nblk, MOE_BLOCK_TOKENS, smem, c.stream>>>((const bf16*)y, (const bf16*)wg, task_ids, tokens_per_image, M, D, E, K,
+    moe_route_kernel<bf16><<<nblk, MOE_ROUTE_WARPS * 32, smem, c.stream>>>((const bf16*)y, (const bf16*)wg, task_ids, tokens_per_image, M, D, E, K,
                                                                        (int)gate_elems, b.eidx, b.ew, b.blk_counts);
   }
   moe_scan_kernel<<<1, 128, 0, c.stream>>>(b.blk_counts, nblk, E, rows_cap / 128, b.blk_off, b.seg_start, b.tile_expert);
