@@ -326,7 +326,8 @@ int attention_bwd(const Ctx& c, const void* qkv, const void* out, const void* do
 // other row of dQ is zero.  One block per (image, head); the probabilities are recomputed in the backward kernel.
 // ---------------------------------------------------------------------------------------------
 constexpr int ATC_WARPS = 4;
-constexpr int ATC_MAXKEYS = 32 * 20;             // keys per lane held in registers: up to 640 tokens
+constexpr int ATC_THREADS = ATC_WARPS * 32;
+constexpr int ATC_MAXKEYS = 1024;                // scores of one row in shared memory
 
 template <typename T> __device__ __forceinline__ float2 ld_pair(const T* p);
 template <> __device__ __forceinline__ float2 ld_pair<float>(const float* p) { return *reinterpret_cast<const float2*>(p); }
@@ -335,49 +336,77 @@ template <typename T> __device__ __forceinline__ void st_pair(T* p, float a, flo
 template <> __device__ __forceinline__ void st_pair<float>(float* p, float a, float b) { *reinterpret_cast<float2*>(p) = make_float2(a, b); }
 template <> __device__ __forceinline__ void st_pair<bf16>(bf16* p, float a, float b) { *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(a, b); }
 
-// Softmax row of the classification query of one (image, head), lanes striding the keys: p[i] belongs to key lane + 32 i.
-// vec: the query (d floats in shared memory).  Returns through p the probabilities.
-template <typename T, int KPL>
-__device__ __forceinline__ void cls_row_probs(const T* kbase, long row_stride, const float* vec, int T_, int d, float scale, int lane,
-                                              float* p) {
-  float mx = -INFINITY;
+// One thread, one key: dot product of the key's (or value's) d entries with a vector in shared memory, 16 bytes a load.
+template <typename T>
+__device__ __forceinline__ float row_dot(const T* row, const float* vec, int d) {
+  constexpr int N = Pack<T>::N;
+  float s = 0.f;
+  for (int e = 0; e < d; e += N) {
+    float kv[N];
+    load16(row + e, kv);
 #pragma unroll
-  for (int i = 0; i < KPL; ++i) {
-    int j = lane + 32 * i;
-    p[i] = -INFINITY;
-    if (j < T_) {
-      const T* row = kbase + (long)j * row_stride;
-      float s = 0.f;
-      for (int e = 0; e < d; e += 2) {
-        float2 kv = ld_pair<T>(row + e);
-        s = fmaf(vec[e], kv.x, s);
-        s = fmaf(vec[e + 1], kv.y, s);
-      }
-      p[i] = s * scale;
-      mx = fmaxf(mx, p[i]);
+    for (int i = 0; i < N; i += 4) {
+      float4 v = *reinterpret_cast<const float4*>(vec + e + i);
+      s = fmaf(v.x, kv[i], s); s = fmaf(v.y, kv[i + 1], s); s = fmaf(v.z, kv[i + 2], s); s = fmaf(v.w, kv[i + 3], s);
     }
   }
-  mx = warp_max(mx);
-  float sum = 0.f;
-#pragma unroll
-  for (int i = 0; i < KPL; ++i) {
-    p[i] = (lane + 32 * i < T_) ? expf(p[i] - mx) : 0.f;
-    sum += p[i];
-  }
-  sum = warp_sum(sum);
-  float inv = 1.0f / sum;
-#pragma unroll
-  for (int i = 0; i < KPL; ++i) p[i] *= inv;
+  return s;
 }
 
-// One block of ATC_WARPS warps per (image, head): every warp forms the softmax row (cheap, and it spares a block-wide
-// exchange), then the warps share the keys of the second phase (warp w takes keys w, w + ATC_WARPS, ...) and their
-// partial sums are combined through shared memory in warp order.
-template <typename T, int KPL>
-__global__ void __launch_bounds__(ATC_WARPS * 32)
+// Block-wide maximum / sum over ATC_WARPS warps, combined in warp order; red holds ATC_WARPS floats.
+__device__ __forceinline__ float cls_block_max(float v, float* red) {
+  v = warp_max(v);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float r = red[0];
+#pragma unroll
+  for (int w = 1; w < ATC_WARPS; ++w) r = fmaxf(r, red[w]);
+  __syncthreads();
+  return r;
+}
+__device__ __forceinline__ float cls_block_sum(float v, float* red) {
+  v = warp_sum(v);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float r = red[0];
+#pragma unroll
+  for (int w = 1; w < ATC_WARPS; ++w) r += red[w];
+  __syncthreads();
+  return r;
+}
+
+// Softmax row of the classification query of one (image, head) into sp[0..T): the block's threads stride the keys.
+template <typename T>
+__device__ __forceinline__ void cls_row_probs(const T* kbase, long row_stride, const float* qs, int T_, int d, float scale,
+                                              float* sp, float* red) {
+  float mx = -INFINITY;
+  for (int j = threadIdx.x; j < T_; j += ATC_THREADS) {
+    float s = row_dot<T>(kbase + (long)j * row_stride, qs, d) * scale;
+    sp[j] = s;
+    mx = fmaxf(mx, s);
+  }
+  mx = cls_block_max(mx, red);
+  float sum = 0.f;
+  for (int j = threadIdx.x; j < T_; j += ATC_THREADS) {
+    float e = expf(sp[j] - mx);
+    sp[j] = e;
+    sum += e;
+  }
+  float inv = 1.0f / cls_block_sum(sum, red);
+  for (int j = threadIdx.x; j < T_; j += ATC_THREADS) sp[j] *= inv;
+  __syncthreads();
+}
+
+// One block of ATC_WARPS warps per (image, head).  Scores: a thread per key.  Weighted sums over the keys: warp w takes
+// keys w, w + ATC_WARPS, ... with the lanes across the features (whole rows, coalesced), and the warps' partial sums are
+// combined through shared memory in warp order.
+template <typename T>
+__global__ void __launch_bounds__(ATC_THREADS)
 attn_cls_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ out_cls, int B, int T_, int H, int d) {
-  __shared__ float qs[AT_MAXD];
+  __shared__ __align__(16) float qs[AT_MAXD];
   __shared__ float part[ATC_WARPS][AT_MAXD];
+  __shared__ float red[ATC_WARPS];
+  __shared__ float sp[ATC_MAXKEYS];
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int pair = blockIdx.x;
   int b = pair / H, h = pair % H;
@@ -388,24 +417,19 @@ attn_cls_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ out_cls, int B, i
     qs[2 * lane] = q.x; qs[2 * lane + 1] = q.y;
   }
   __syncthreads();
-  float p[KPL];
-  cls_row_probs<T, KPL>(base + (long)H * d, row_stride, qs, T_, d, rsqrtf((float)d), lane, p);
+  cls_row_probs<T>(base + (long)H * d, row_stride, qs, T_, d, rsqrtf((float)d), sp, red);
   // o_0 = sum_j p_j v_j: every lane owns two feature indices; this warp's keys in order
   float o0 = 0.f, o1 = 0.f;
   const T* vbase = base + 2L * H * d;
-#pragma unroll
-  for (int i = 0; i < KPL; ++i) {
+  if (2 * lane < d) {
 #pragma unroll 4
-    for (int l = warp; l < 32; l += ATC_WARPS) {
-      int j = l + 32 * i;
-      float pj = __shfl_sync(0xffffffffu, p[i], l);
-      if (j < T_ && 2 * lane < d) {
-        float2 v = ld_pair<T>(vbase + (long)j * row_stride + 2 * lane);
-        o0 = fmaf(pj, v.x, o0); o1 = fmaf(pj, v.y, o1);
-      }
+    for (int j = warp; j < T_; j += ATC_WARPS) {
+      float2 v = ld_pair<T>(vbase + (long)j * row_stride + 2 * lane);
+      float pj = sp[j];
+      o0 = fmaf(pj, v.x, o0); o1 = fmaf(pj, v.y, o1);
     }
+    part[warp][2 * lane] = o0; part[warp][2 * lane + 1] = o1;
   }
-  if (2 * lane < d) { part[warp][2 * lane] = o0; part[warp][2 * lane + 1] = o1; }
   __syncthreads();
   if (warp == 0 && 2 * lane < d) {
     float a0 = 0.f, a1 = 0.f;
@@ -415,11 +439,14 @@ attn_cls_fwd_kernel(const T* __restrict__ qkv, T* __restrict__ out_cls, int B, i
   }
 }
 
-template <typename T, int KPL>
-__global__ void __launch_bounds__(ATC_WARPS * 32)
+template <typename T>
+__global__ void __launch_bounds__(ATC_THREADS)
 attn_cls_bwd_kernel(const T* __restrict__ qkv, const T* __restrict__ dout_cls, T* __restrict__ dqkv, int B, int T_, int H, int d) {
-  __shared__ float qs[AT_MAXD], gs[AT_MAXD];
+  __shared__ __align__(16) float qs[AT_MAXD];
+  __shared__ __align__(16) float gs[AT_MAXD];
   __shared__ float part[ATC_WARPS][AT_MAXD];
+  __shared__ float red[ATC_WARPS];
+  __shared__ float sp[ATC_MAXKEYS], sd[ATC_MAXKEYS];
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int pair = blockIdx.x;
   int b = pair / H, h = pair % H;
@@ -438,51 +465,34 @@ attn_cls_bwd_kernel(const T* __restrict__ qkv, const T* __restrict__ dout_cls, T
   }
   __syncthreads();
   float scale = rsqrtf((float)d);
-  float p[KPL], ds[KPL];
-  cls_row_probs<T, KPL>(base + (long)H * d, row_stride, qs, T_, d, scale, lane, p);
-  // dP_j = dO_0 . v_j for the lane's keys, delta = sum_j p_j dP_j
+  cls_row_probs<T>(base + (long)H * d, row_stride, qs, T_, d, scale, sp, red);
+  // dP_j = dO_0 . v_j (a thread per key), delta = sum_j p_j dP_j
   const T* vbase = base + 2L * H * d;
   float delta = 0.f;
-#pragma unroll
-  for (int i = 0; i < KPL; ++i) {
-    int j = lane + 32 * i;
-    ds[i] = 0.f;
-    if (j < T_) {
-      const T* row = vbase + (long)j * row_stride;
-      float s = 0.f;
-      for (int e = 0; e < d; e += 2) {
-        float2 v = ld_pair<T>(row + e);
-        s = fmaf(gs[e], v.x, s);
-        s = fmaf(gs[e + 1], v.y, s);
-      }
-      ds[i] = s;
-      delta += p[i] * s;
-    }
+  for (int j = threadIdx.x; j < T_; j += ATC_THREADS) {
+    float dp = row_dot<T>(vbase + (long)j * row_stride, gs, d);
+    sd[j] = dp;
+    delta = fmaf(sp[j], dp, delta);
   }
-  delta = warp_sum(delta);
-#pragma unroll
-  for (int i = 0; i < KPL; ++i) ds[i] = p[i] * (ds[i] - delta) * scale;      // dS_j / sqrt(d)
+  delta = cls_block_sum(delta, red);
+  for (int j = threadIdx.x; j < T_; j += ATC_THREADS) sd[j] = sp[j] * (sd[j] - delta) * scale;      // dS_j / sqrt(d)
+  __syncthreads();
   // rows of this warp's keys: dV_j = p_j dO_0, dK_j = dS_j q_0 / sqrt(d), dQ_j = 0 for j > 0; dQ_0 = sum_j dS_j k_j / sqrt(d)
   float dq0 = 0.f, dq1 = 0.f;
   const T* kbase = base + (long)H * d;
-#pragma unroll
-  for (int i = 0; i < KPL; ++i) {
+  if (2 * lane < d) {
 #pragma unroll 4
-    for (int l = warp; l < 32; l += ATC_WARPS) {
-      int j = l + 32 * i;
-      float pj = __shfl_sync(0xffffffffu, p[i], l);
-      float dsj = __shfl_sync(0xffffffffu, ds[i], l);
-      if (j < T_ && 2 * lane < d) {
-        float2 k = ld_pair<T>(kbase + (long)j * row_stride + 2 * lane);
-        dq0 = fmaf(dsj, k.x, dq0); dq1 = fmaf(dsj, k.y, dq1);
-        T* drow = dbase + (long)j * row_stride + 2 * lane;
-        st_pair<T>(drow + (long)H * d, dsj * q0, dsj * q1);
-        st_pair<T>(drow + 2L * H * d, pj * g0, pj * g1);
-        if (j > 0) st_pair<T>(drow, 0.f, 0.f);
-      }
+    for (int j = warp; j < T_; j += ATC_WARPS) {
+      float pj = sp[j], dsj = sd[j];
+      float2 k = ld_pair<T>(kbase + (long)j * row_stride + 2 * lane);
+      dq0 = fmaf(dsj, k.x, dq0); dq1 = fmaf(dsj, k.y, dq1);
+      T* drow = dbase + (long)j * row_stride + 2 * lane;
+      st_pair<T>(drow + (long)H * d, dsj * q0, dsj * q1);
+      st_pair<T>(drow + 2L * H * d, pj * g0, pj * g1);
+      if (j > 0) st_pair<T>(drow, 0.f, 0.f);
     }
+    part[warp][2 * lane] = dq0; part[warp][2 * lane + 1] = dq1;
   }
-  if (2 * lane < d) { part[warp][2 * lane] = dq0; part[warp][2 * lane + 1] = dq1; }
   __syncthreads();
   if (warp == 0 && 2 * lane < d) {
     float a0 = 0.f, a1 = 0.f;
@@ -494,17 +504,11 @@ attn_cls_bwd_kernel(const T* __restrict__ qkv, const T* __restrict__ dout_cls, T
 
 template <typename T>
 static int launch_cls(const Ctx& c, bool bwd, const void* qkv, const void* io_cls, void* dqkv, int B, int T_, int H, int d) {
-  if (d > AT_MAXD || (d % 2) != 0 || T_ < 1 || T_ > ATC_MAXKEYS) return -2;
+  if (d > AT_MAXD || (d % 8) != 0 || T_ < 1 || T_ > ATC_MAXKEYS) return -2;
   int blocks = B * H;
   note_launch(1);
-#define BSR_CLS(KPL)                                                                                                              \
-  do {                                                                                                                            \
-    if (bwd) attn_cls_bwd_kernel<T, KPL><<<blocks, ATC_WARPS * 32, 0, c.stream>>>((const T*)qkv, (const T*)io_cls, (T*)dqkv, B, T_, H, d); \
-    else attn_cls_fwd_kernel<T, KPL><<<blocks, ATC_WARPS * 32, 0, c.stream>>>((const T*)qkv, (T*)const_cast<void*>(io_cls), B, T_, H, d);  \
-  } while (0)
-  int kpl = ceil_div(T_, 32);
-  if (kpl <= 3) BSR_CLS(3); else if (kpl <= 5) BSR_CLS(5); else if (kpl <= 7) BSR_CLS(7); else if (kpl <= 10) BSR_CLS(10); else BSR_CLS(20);
-#undef BSR_CLS
+  if (bwd) attn_cls_bwd_kernel<T><<<blocks, ATC_THREADS, 0, c.stream>>>((const T*)qkv, (const T*)io_cls, (T*)dqkv, B, T_, H, d);
+  else attn_cls_fwd_kernel<T><<<blocks, ATC_THREADS, 0, c.stream>>>((const T*)qkv, (T*)const_cast<void*>(io_cls), B, T_, H, d);
   return 0;
 }
 

@@ -199,6 +199,8 @@ struct bsr_handle {
   cudaEvent_t ev_copied[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr};
   bool slot_used[2] = {false, false};
   int host_slot = 0;
+  SideLane side;                        // second lane for the reductions only the optimiser reads
+  int use_side = 1;
   long launches_at_enable = 0;
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(base + off); }
@@ -506,6 +508,7 @@ Ctx make_ctx(const bsr_handle* h, void* stream) {
   c.split_ws = h->split_floats ? h->at<float>(h->off_split) : nullptr;
   c.split_ws_floats = h->split_floats;
   c.prof = const_cast<GemmProfile*>(&h->prof);
+  c.side = (h->use_side && h->side.stream != nullptr && !h->prof.on) ? const_cast<SideLane*>(&h->side) : nullptr;
   return c;
 }
 
@@ -937,6 +940,11 @@ int32_t bsr_create(const bsr_config* cfg, void* workspace, size_t bytes, bsr_han
     delete h;
     return set_err(g_error, BSR_ERR_CUDA, "workspace initialisation failed: %s", cudaGetErrorString(e));
   }
+  // host objects of the side lane (no device memory); without them the reductions simply stay on the main stream
+  bool lane = cudaStreamCreateWithFlags(&h->side.stream, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&h->side.fork, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; i < 3 && lane; ++i) lane = cudaEventCreateWithFlags(&h->side.done[i], cudaEventDisableTiming) == cudaSuccess;
+  if (!lane) { cudaGetLastError(); h->side.stream = nullptr; }
   *out = h;
   return BSR_OK;
 }
@@ -950,6 +958,10 @@ int32_t bsr_destroy(bsr_handle* h) {
       if (h->ev_done[i]) cudaEventDestroy(h->ev_done[i]);
     }
     if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
+    if (h->side.fork) cudaEventDestroy(h->side.fork);
+    for (int i = 0; i < 3; ++i)
+      if (h->side.done[i]) cudaEventDestroy(h->side.done[i]);
+    if (h->side.stream) cudaStreamDestroy(h->side.stream);
   }
   delete h;
   return BSR_OK;
@@ -1119,6 +1131,7 @@ static int enqueue_train_step(bsr_handle* h, const void* images, const int32_t* 
     layernorm_bwd(c, h->at<float>(h->off_dxn), 1, h->at<float>(x_last), (long)Tl * D, h->at<float>(h->off_meanf), h->at<float>(h->off_rstdf),
                   (const float*)h->w("norm.weight"), nullptr, nullptr, 0, nullptr, lnp, h->gradp("norm.weight"), h->gradp("norm.bias"), B, D);
   }
+  side_join_all(c);                      // every gradient is complete on the main stream from here on
   if (with_update) enqueue_optimizer(h, c);
   return BSR_OK;
 }

@@ -472,6 +472,7 @@ int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const voi
   const int final_is_float = out_is_float;
   if (splits > 1) out_is_float = 1;
   void* dst = (splits > 1) ? (void*)split_ws : C;
+  if (splits > 1) side_join(c, 2);         // the previous split sum has read the workspace
   if (c.prof != nullptr && c.prof->on) c.prof->begin(c.stream, 2.0 * m * n * (double)k);
   int rc;
   GemmGroup gg;
@@ -492,8 +493,9 @@ int gemm_tc_strided(const Ctx& c, const void* A, long a_rs, long a_cs, const voi
   if (rc != 0) return rc;
   if (splits > 1) {
     size_t total = (size_t)m * n;
-    if (!deferred) {
-      splitk_reduce(c.stream, split_ws, (float*)C, total, splits);
+    if (!deferred) {                       // a weight gradient: only the optimiser reads the sum
+      splitk_reduce(side_begin(c), split_ws, (float*)C, total, splits);
+      side_end(c, 2);
     } else {
       note_launch(1);
       int blocks = ceil_div((long)(total / 4), 256);

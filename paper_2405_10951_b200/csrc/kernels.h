@@ -36,6 +36,17 @@ struct GemmProfile {
   }
 };
 
+// Reductions whose results only the optimiser reads (split sums of weight gradients, partial sums of LayerNorm
+// parameter gradients and of bias gradients) need not sit on the chain of the backward pass: they are enqueued on a
+// second stream that forks from the main one and is joined before the buffer they read is written again, and before
+// the update.  Inside a stream capture the fork and the joins become edges of the graph.
+struct SideLane {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr;
+  cudaEvent_t done[3] = {nullptr, nullptr, nullptr};   // 0: LayerNorm partials, 1: column-sum partials, 2: split-k workspace
+  bool pending[3] = {false, false, false};
+};
+
 struct Ctx {
   cudaStream_t stream;
   int dtype;        // 0 fp32, 1 bf16
@@ -45,7 +56,32 @@ struct Ctx {
   float* split_ws = nullptr;       // scratch for split-k partial sums (optional)
   size_t split_ws_floats = 0;
   GemmProfile* prof = nullptr;
+  SideLane* side = nullptr;        // optional second lane for optimiser-only reductions
 };
+
+// The main stream is about to rewrite buffer `which`: wait for the side reduction that may still read it.
+inline void side_join(const Ctx& c, int which) {
+  if (c.side != nullptr && c.side->pending[which]) {
+    cudaStreamWaitEvent(c.stream, c.side->done[which], 0);
+    c.side->pending[which] = false;
+  }
+}
+inline void side_join_all(const Ctx& c) {
+  for (int w = 0; w < 3; ++w) side_join(c, w);
+}
+// Stream for a reduction of buffer `which`: the side lane, made to wait for everything enqueued on the main stream so far
+// (the main stream itself when there is no side lane).  side_end marks the reduction as in flight.
+inline cudaStream_t side_begin(const Ctx& c) {
+  if (c.side == nullptr) return c.stream;
+  cudaEventRecord(c.side->fork, c.stream);
+  cudaStreamWaitEvent(c.side->stream, c.side->fork, 0);
+  return c.side->stream;
+}
+inline void side_end(const Ctx& c, int which) {
+  if (c.side == nullptr) return;
+  cudaEventRecord(c.side->done[which], c.side->stream);
+  c.side->pending[which] = true;
+}
 
 inline size_t dtype_size(int dtype) { return dtype == 0 ? 4 : 2; }
 
@@ -146,7 +182,7 @@ int attention_bwd(const Ctx& c, const void* qkv, const void* out, const void* do
 
 // The classification row alone (last block: only that row of the block's output is ever read).  out_cls / dout_cls
 // [B, H*d]: attention output of query 0 and its gradient; dqkv [B, T, 3, H, d] is written in full (rows of dQ other
-// than the first are zero).  Return non-zero when the problem does not fit (more than 640 tokens, odd head dimension).
+// than the first are zero).  Return non-zero when the problem does not fit (more than 1024 tokens, a head dimension above 64 or not a multiple of 8).
 int attention_cls_fwd(const Ctx& c, const void* qkv, void* out_cls, int B, int T, int H, int d);
 int attention_cls_bwd(const Ctx& c, const void* qkv, const void* dout_cls, void* dqkv, int B, int T, int H, int d);
 

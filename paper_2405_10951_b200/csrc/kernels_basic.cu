@@ -455,6 +455,7 @@ void layernorm_bwd(const Ctx& c, const void* dy, int dy_is_float, const float* x
   int groups = layernorm_bwd_groups(c, rows);
   int nsum = (dx_colsum != nullptr && dx != nullptr) ? 3 : 2;
   size_t smem = (size_t)LNB_WARPS * nsum * D * sizeof(float);
+  side_join(c, 0);                                                     // the previous reduction has read the partials
   if (c.dtype == 0)
     launch_ln_bwd<float, float>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, nullptr, partials, rows, D, nsum);
   else if (dy_is_float)
@@ -463,7 +464,9 @@ void layernorm_bwd(const Ctx& c, const void* dy, int dy_is_float, const float* x
     launch_ln_bwd<bf16, bf16>(c, groups, smem, dy, x, x_stride, mean, rstd, g, dres, dx, dx_stride, dx_copy, partials, rows, D, nsum);
   if (dgamma == nullptr && nsum == 2) return;                          // a frozen block in the gradient path: only dx is wanted
   dim3 grid(ceil_div(D, 16), nsum);
-  reduce_partials_kernel<<<grid, 256, 0, c.stream>>>(partials, groups, D, dgamma, dbeta, nsum == 3 ? dx_colsum : nullptr);
+  cudaStream_t rs = side_begin(c);                                     // only the optimiser reads these sums
+  reduce_partials_kernel<<<grid, 256, 0, rs>>>(partials, groups, D, dgamma, dbeta, nsum == 3 ? dx_colsum : nullptr);
+  side_end(c, 0);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -525,6 +528,7 @@ void colsum(const Ctx& c, const void* x, int rows, int cols, float* partials, fl
   note_launch(2);
   int groups = colsum_groups(rows);
   int threads = CS_ROWLANES * 32;
+  side_join(c, 1);
   if (c.dtype == 0) {
     dim3 grid(ceil_div(cols, 32 * 4), groups);
     colsum_kernel<float><<<grid, threads, 0, c.stream>>>((const float*)x, rows, cols, partials);
@@ -532,7 +536,9 @@ void colsum(const Ctx& c, const void* x, int rows, int cols, float* partials, fl
     dim3 grid(ceil_div(cols, 32 * 8), groups);
     colsum_kernel<bf16><<<grid, threads, 0, c.stream>>>((const bf16*)x, rows, cols, partials);
   }
-  reduce_partials_kernel<<<dim3(ceil_div(cols, 16), 1), 256, 0, c.stream>>>(partials, groups, cols, out, out);
+  cudaStream_t rs = side_begin(c);
+  reduce_partials_kernel<<<dim3(ceil_div(cols, 16), 1), 256, 0, rs>>>(partials, groups, cols, out, out);
+  side_end(c, 1);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -17,15 +17,20 @@ constexpr int MOE_MAX_K = 4;
 
 // ---- routing: gate logits, top-k (ties -> lower expert id), softmax over the selected logits -------------------
 constexpr int MOE_ROUTE_WARPS = 8;
+constexpr int MOE_ROUTE_TOKENS = 16;
+static_assert(MOE_BLOCK_TOKENS % MOE_ROUTE_TOKENS == 0, "a routing block must not straddle two counting groups");
 template <typename T>
 __global__ void __launch_bounds__(MOE_ROUTE_WARPS * 32)
 moe_route_kernel(const T* __restrict__ y, const T* __restrict__ wg, const int* __restrict__ task_ids, int tokens_per_image,
                  int M, int D, int E, int K, int gate_elems_in_smem, int* __restrict__ eidx, float* __restrict__ ew,
                  int* __restrict__ blk_counts) {
-  // A block owns MOE_BLOCK_TOKENS consecutive tokens, a warp one token at a time: the lanes read the token's row of y
-  // in 16-byte pieces (coalesced), multiply it with the same pieces of every gate row -- the gate matrices of all tasks
-  // are staged in shared memory when they fit -- and the E partial dot products are summed over the lanes in a fixed
-  // (butterfly) order.  Lane 0 then scans the logits for the top k.
+  // A block takes MOE_ROUTE_TOKENS consecutive tokens (a divisor of MOE_BLOCK_TOKENS, so all of them fall into one
+  // counting group), a warp one token at a time.  Expert by expert the lanes multiply 16-byte pieces of the token's row
+  // of y (coalesced; from L1 after the first expert) with the same pieces of the gate row -- the gate matrices of all
+  // tasks are staged in shared memory when they are small -- and the partial dot products are summed over the lanes
+  // in a fixed (butterfly) order; lane e keeps logit e.  The top k then come from k warp-wide maxima (among equal
+  // logits the lowest expert id, found with a ballot).  Few registers, so many tokens are in flight per SM: the work
+  // per token is a chain of dependent loads.  The per-group expert counts (zeroed before the launch) are integer sums.
   extern __shared__ __align__(16) unsigned char route_smem[];
   __shared__ int counts[MOE_MAX_E];
   constexpr int N = Pack<T>::N;
@@ -40,60 +45,61 @@ moe_route_kernel(const T* __restrict__ y, const T* __restrict__ wg, const int* _
   __syncthreads();
   int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int chunks = D / N;
-  for (int t = warp; t < MOE_BLOCK_TOKENS; t += MOE_ROUTE_WARPS) {
-    int tok = blockIdx.x * MOE_BLOCK_TOKENS + t;
+  const uint32_t all = (E >= 32) ? 0xffffffffu : ((1u << E) - 1u);
+  for (int t = warp; t < MOE_ROUTE_TOKENS; t += MOE_ROUTE_WARPS) {
+    int tok = blockIdx.x * MOE_ROUTE_TOKENS + t;
     if (tok >= M) break;
     int task = task_ids ? task_ids[tok / tokens_per_image] : 0;
     const T* yr = y + (size_t)tok * D;
     const T* gt = gates + (size_t)task * E * D;
-    float acc[MOE_MAX_E];
+    float logit = -INFINITY;                      // lane e: logit of expert e
+#pragma unroll 4
+    for (int e = 0; e < E; ++e) {
+      float acc = 0.f;
+      for (int ch = lane; ch < chunks; ch += 32) {
+        float yv[N], wv[N];
+        load16(yr + ch * N, yv);
+        load16(gt + (size_t)e * D + ch * N, wv);
 #pragma unroll
-    for (int e = 0; e < MOE_MAX_E; ++e) acc[e] = 0.f;
-    for (int ch = lane; ch < chunks; ch += 32) {
-      float yv[N];
-      load16(yr + ch * N, yv);
+        for (int j = 0; j < N; ++j) acc = fmaf(yv[j], wv[j], acc);
+      }
+      acc = warp_sum(acc);
+      if (lane == e) logit = acc;
+    }
+    float sel[MOE_MAX_K];
+    int sid[MOE_MAX_K];
+    uint32_t taken = 0;
 #pragma unroll
-      for (int e = 0; e < MOE_MAX_E; ++e) {
-        if (e < E) {
-          float wv[N];
-          load16(gt + (size_t)e * D + ch * N, wv);
-#pragma unroll
-          for (int j = 0; j < N; ++j) acc[e] = fmaf(yv[j], wv[j], acc[e]);
-        }
+    for (int i = 0; i < MOE_MAX_K; ++i) {
+      if (i < K) {
+        bool open = lane < E && !((taken >> lane) & 1u);
+        float best = warp_max(open ? logit : -INFINITY);
+        uint32_t at = __ballot_sync(0xffffffffu, open && logit == best);
+        if (at == 0) at = all & ~taken;             // nothing compares equal (a NaN among the logits): lowest open id
+        int bi = __ffs(at) - 1;                     // the lowest id wins among equals
+        sel[i] = __shfl_sync(0xffffffffu, logit, bi);
+        sid[i] = bi;
+        taken |= 1u << bi;
       }
     }
-#pragma unroll
-    for (int e = 0; e < MOE_MAX_E; ++e)
-      if (e < E) acc[e] = warp_sum(acc[e]);
     if (lane == 0) {
-      float sel[MOE_MAX_K];
-      int sid[MOE_MAX_K];
-      uint32_t taken = 0;
-      for (int i = 0; i < K; ++i) {
-        float best = -INFINITY;
-        int bi = 0;
-        bool any = false;
-#pragma unroll
-        for (int e = 0; e < MOE_MAX_E; ++e) {
-          if (e < E && !((taken >> e) & 1u) && (!any || acc[e] > best)) {    // strictly greater: the lowest id wins among equals
-            best = acc[e]; bi = e; any = true;
-          }
-        }
-        taken |= 1u << bi;
-        sel[i] = best;
-        sid[i] = bi;
-      }
       float den = 0.f;
-      for (int i = 0; i < K; ++i) den += expf(sel[i] - sel[0]);
-      for (int i = 0; i < K; ++i) {
-        eidx[(size_t)tok * K + i] = sid[i];
-        ew[(size_t)tok * K + i] = expf(sel[i] - sel[0]) / den;
-        atomicAdd(&counts[sid[i]], 1);              // integer counts: order-independent
+#pragma unroll
+      for (int i = 0; i < MOE_MAX_K; ++i)
+        if (i < K) den += expf(sel[i] - sel[0]);
+#pragma unroll
+      for (int i = 0; i < MOE_MAX_K; ++i) {
+        if (i < K) {
+          eidx[(size_t)tok * K + i] = sid[i];
+          ew[(size_t)tok * K + i] = expf(sel[i] - sel[0]) / den;
+          atomicAdd(&counts[sid[i]], 1);            // integer counts: order-independent
+        }
       }
     }
   }
   __syncthreads();
-  if (threadIdx.x < E) blk_counts[(size_t)blockIdx.x * E + threadIdx.x] = counts[threadIdx.x];
+  if (threadIdx.x < E && counts[threadIdx.x] != 0)
+    atomicAdd(&blk_counts[(size_t)(blockIdx.x * MOE_ROUTE_TOKENS / MOE_BLOCK_TOKENS) * E + threadIdx.x], counts[threadIdx.x]);
 }
 
 // ---- segment table: one warp per expert walks the token blocks in order ------------------------------------------
@@ -343,15 +349,17 @@ void moe_route(const Ctx& c, const MoeBufs& b, const void* y, const void* wg, co
   size_t es = c.dtype == 0 ? 4 : 2;
   size_t gate_elems = (size_t)(num_tasks < 1 ? 1 : num_tasks) * E * D;
   size_t smem = gate_elems * es;
-  if (smem > 96 * 1024) { smem = 0; gate_elems = 0; }       // too large to stage: the gates are read through L1 instead
+  if (smem > 16 * 1024) { smem = 0; gate_elems = 0; }       // not worth staging for 16 tokens: the gates are read through L1 instead
   static SmemLimit lim[2];
+  int rblk = ceil_div(M, MOE_ROUTE_TOKENS);
+  cudaMemsetAsync(b.blk_counts, 0, (size_t)nblk * E * sizeof(int), c.stream);
   if (c.dtype == 0) {
     ensure_smem(lim[0], moe_route_kernel<float>, smem);
-    moe_route_kernel<float><<<nblk, MOE_ROUTE_WARPS * 32, smem, c.stream>>>((const float*)y, (const float*)wg, task_ids, tokens_per_image, M, D, E, K,
+    moe_route_kernel<float><<<rblk, MOE_ROUTE_WARPS * 32, smem, c.stream>>>((const float*)y, (const float*)wg, task_ids, tokens_per_image, M, D, E, K,
                                                                         (int)gate_elems, b.eidx, b.ew, b.blk_counts);
   } else {
     ensure_smem(lim[1], moe_route_kernel<bf16>, smem);
-    moe_route_kernel<bf16><<<nblk, MOE_ROUTE_WARPS * 32, smem, c.stream>>>((const bf16*)y, (const bf16*)wg, task_ids, tokens_per_image, M, D, E, K,
+    moe_route_kernel<bf16><<<rblk, MOE_ROUTE_WARPS * 32, smem, c.stream>>>((const bf16*)y, (const bf16*)wg, task_ids, tokens_per_image, M, D, E, K,
                                                                        (int)gate_elems, b.eidx, b.ew, b.blk_counts);
   }
   moe_scan_kernel<<<1, 128, 0, c.stream>>>(b.blk_counts, nblk, E, rows_cap / 128, b.blk_off, b.seg_start, b.tile_expert);

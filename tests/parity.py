@@ -89,11 +89,15 @@ def check_selection(cfg, gpu_kept, forced_run, exact_margin, score_tol, gpu_scor
       * the GPU's set must be a valid top-K of the oracle's scores within score_tol
         (weakest kept score >= strongest dropped score - score_tol * s_(K));
       * where the oracle's own boundary margin exceeds exact_margin the set must be identical to the
-        oracle's own choice.
-    Returns a report: sets compared, sets identical to the oracle's own choice, sets whose margin demanded identity,
-    and per location the worst score deviation relative to the K-th score.
+        oracle's own choice; so it must where the margin exceeds twice the score deviation measured for that image
+        (a kept score can fall by at most that deviation times itself, a dropped one rise by at most that deviation
+        times s_(K), so the order across the boundary cannot change) -- the sets counted as "determined".
+    Returns a report: sets compared, sets identical to the oracle's own choice, sets whose margin demanded identity
+    (by the fixed margin, and by the measured deviation), and per location the worst score deviation relative to
+    the K-th score.  How many of the remaining sets coincide is chance (a 576-token row has several scores within a
+    few percent of the K-th) and is reported, not asserted.
     """
-    total = same = strict = 0
+    total = same = strict = determined = 0
     score_err = []
     for loc, (kept, scores) in enumerate(zip(gpu_kept, forced_run["scores"])):
         B, k = kept.shape
@@ -109,6 +113,7 @@ def check_selection(cfg, gpu_kept, forced_run, exact_margin, score_tol, gpu_scor
             total += 1
             same += int(identical)
             sk = scores[b][own].min()
+            dev = None
             if gpu_scores is not None:
                 sg = gpu_scores[loc][b]
                 assert np.array_equal(O.select_tokens(sg.astype(np.float32), k)[0], mine), f"location {loc} image {b}: not the top-K of the GPU's own scores"
@@ -121,8 +126,13 @@ def check_selection(cfg, gpu_kept, forced_run, exact_margin, score_tol, gpu_scor
                 if margin > exact_margin:
                     strict += 1
                     assert identical, f"location {loc} image {b}: margin {margin:.3e} but sets differ"
+                if margin > exact_margin or (dev is not None and margin > 2.0 * dev):
+                    determined += 1
+                    assert identical, f"location {loc} image {b}: margin {margin:.3e}, score deviation {dev}, but sets differ"
+            else:
+                determined += 1
         score_err.append(worst)
-    return {"sets": total, "sets_identical": same, "sets_strict": strict, "score_err": score_err}
+    return {"sets": total, "sets_identical": same, "sets_strict": strict, "sets_determined": determined, "score_err": score_err}
 
 
 def forced_experts_of(cfg, gpu, token_counts):
@@ -195,7 +205,7 @@ def compare_step(cfg, images, labels, task_ids, params, gpu, tol, exact_margin, 
     ref, fe = oracle_reference(cfg, images, labels, task_ids, params, gpu, chunk)
     if fe:
         check_routing(cfg, ref, gpu, 2e-2)
-    report = {"sets": 0, "sets_identical": 0, "sets_strict": 0, "score_err": []}
+    report = {"sets": 0, "sets_identical": 0, "sets_strict": 0, "sets_determined": 0, "score_err": []}
     if forced:
         report = check_selection(cfg, gpu["kept"], ref, exact_margin, score_tol, gpu.get("scores"))
     assert abs(gpu["loss"] - ref["loss"]) <= tol * abs(ref["loss"]), (gpu["loss"], ref["loss"])

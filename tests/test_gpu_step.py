@@ -61,7 +61,9 @@ PEAKED_WIDE = {"mini", "mini_mean_fusion", "deit_s_keep_0p3_late"}
 @pytest.mark.parametrize("case", list(BF16_CASES))
 def test_bf16_step_matches_oracle(case, peaked):
     """Every configuration holds the 2e-2 tolerance on loss, logits and every gradient (two named peaked cases:
-    3e-2); scores and kept sets follow the measured rule stated in parity.py."""
+    3e-2); scores and kept sets follow the rule stated in parity.py (every set is the top-K of the scores the kernel
+    read, those scores agree with the oracle's within the score tolerance, and a set whose boundary margin exceeds
+    twice the measured deviation is identical to the oracle's)."""
     cfg = BF16_CASES[case]
     images, labels, task_ids, params = synth.make_workload(cfg, peaked=peaked)
     gpu = P.run_gpu_step(cfg, images, labels, task_ids, params)
@@ -69,7 +71,7 @@ def test_bf16_step_matches_oracle(case, peaked):
     margin, score_tol = (P.BF16_EXACT_MARGIN_PEAKED, P.BF16_SCORE_TOL_PEAKED) if peaked else (P.BF16_EXACT_MARGIN, P.BF16_SCORE_TOL)
     rep = P.compare_step(cfg, images, labels, task_ids, params, gpu, tol, margin, score_tol)
     print(case, "peaked" if peaked else "literal", rep)
-    assert rep["sets_identical"] >= 0.6 * rep["sets"], rep
+    assert rep["sets_identical"] >= rep["sets_determined"], rep
 
 
 def test_eval_forward_matches_oracle_and_train_forward():
