@@ -20,7 +20,9 @@ constexpr int AT_BOX = 64;                       // rows per TMA box
 constexpr int AT_BOX_BYTES = AT_BOX * AT_D * 2;  // 8 KB
 constexpr int AT_QROWS = 128;
 constexpr int AT_MAXKEYS = 256;
-constexpr int AT_LONG_KB = 64;                   // keys per block of the two-walk kernel for longer sequences (four CTAs per SM)
+constexpr float AT_LONG_SLACK = 8.0f;             // binary orders the row maximum may exceed the reference before a rescale
+constexpr int AT_LONG_MAXBLK = 64;                // key blocks of the longest sequence the kernel takes
+constexpr int AT_LONG_KB = 64;                   // keys per block of the kernel for longer sequences (four CTAs per SM)
 
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -341,10 +343,14 @@ attn_fwd_ws_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 }
 
 // ------------------------------------------------------------------------------------------------
-// Forward for longer sequences (T > 256): the keys are walked in blocks of up to 128, twice.  The first walk
-// only computes S = Q K^T per block and keeps the running row maximum and row sum; the second walk recomputes S,
-// forms P = exp(S - max) with the final maximum (so the accumulator never needs rescaling) and adds P V into a
-// separate set of tensor-memory columns.  One CTA per (image, head, 128 queries), one block in flight.
+// Forward for longer sequences (T > 256): the keys are walked once in blocks of AT_LONG_KB.  Per block S = Q K^T
+// goes into tensor memory, each thread reads its row, forms P = exp(S - m) against the row's reference maximum m,
+// sums P as it goes and hands P (bf16, through shared memory) to the second product, which adds P V into a separate
+// set of tensor-memory columns; the output is divided by the sum at the end.  m follows the running maximum only in
+// jumps of more than AT_LONG_SLACK binary orders, at which the accumulator is rescaled in place (rare after the first
+// block), so that almost every block costs one product, one exponential per score and one more product.  The
+// classification row's probabilities are written out block by block against the m of the moment and brought onto the
+// final scale by its warp at the end.  One CTA per (image, head, 128 queries), one block in flight, several CTAs per SM.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(128)
 attn_fwd_tc_long_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restrict__ out, float* __restrict__ lse,
@@ -387,113 +393,133 @@ attn_fwd_tc_long_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __res
   bool ok = true;
   float mx = -INFINITY, sum = 0.f;
   bool cls_row = (q0 == 0 && tid == 0 && cls_prob != nullptr);
+  bool cls_warp = (q0 == 0 && warp == 0 && cls_prob != nullptr);
+  __shared__ float cls_m[AT_LONG_MAXBLK];               // reference maximum of the classification row, block by block
 
-  for (int pass = 0; pass < 2 && ok; ++pass) {
-    for (int kb = 0; kb < nblk && ok; ++kb) {
-      int k0 = kb * KB;
-      int keys = min(KB, T - k0);
-      int kpad = (keys + 15) & ~15;
-      int nbox = (kpad + AT_BOX - 1) / AT_BOX;
-      if (tid == 0) {
-        bool first = (pass == 0 && kb == 0);
-        int boxes = nbox * (pass == 1 ? 2 : 1) + (first ? 2 : 0);
-        mbar_expect_tx(tma_bar, boxes * AT_BOX_BYTES);
-        if (first)
-          for (int j = 0; j < 2; ++j) tma_load_2d(sQ + j * AT_BOX_BYTES, &map_qkv, tma_bar, h * AT_D, row0 + q0 + j * AT_BOX);
-        for (int j = 0; j < nbox; ++j) {
-          tma_load_2d(sK + j * AT_BOX_BYTES, &map_qkv, tma_bar, (H + h) * AT_D, row0 + k0 + j * AT_BOX);
-          if (pass == 1) tma_load_2d(sV + j * AT_BOX_BYTES, &map_qkv, tma_bar, (2 * H + h) * AT_D, row0 + k0 + j * AT_BOX);
-        }
-        ok = mbar_wait(tma_bar, tma_phase, abortp);
-        if (ok) {
-          tc_fence_after();
-          uint32_t idesc = make_idesc_mn(AT_QROWS, kpad, false, false);
-#pragma unroll
-          for (int k = 0; k < AT_D / 16; ++k)
-            umma_bf16(tmem, make_desc(sQ + k * 32, 16, 1024), make_desc(sK + k * 32, 16, 1024), idesc, k > 0 ? 1u : 0u);
-          umma_commit(mma_bar);
-        }
+  for (int kb = 0; kb < nblk && ok; ++kb) {
+    int k0 = kb * KB;
+    int keys = min(KB, T - k0);
+    int kpad = (keys + 15) & ~15;
+    int nbox = (kpad + AT_BOX - 1) / AT_BOX;
+    if (tid == 0) {
+      int boxes = 2 * nbox + (kb == 0 ? 2 : 0);
+      mbar_expect_tx(tma_bar, boxes * AT_BOX_BYTES);
+      if (kb == 0)
+        for (int j = 0; j < 2; ++j) tma_load_2d(sQ + j * AT_BOX_BYTES, &map_qkv, tma_bar, h * AT_D, row0 + q0 + j * AT_BOX);
+      for (int j = 0; j < nbox; ++j) {
+        tma_load_2d(sK + j * AT_BOX_BYTES, &map_qkv, tma_bar, (H + h) * AT_D, row0 + k0 + j * AT_BOX);
+        tma_load_2d(sV + j * AT_BOX_BYTES, &map_qkv, tma_bar, (2 * H + h) * AT_D, row0 + k0 + j * AT_BOX);
       }
-      tma_phase ^= 1u;
-      ok = mbar_wait(mma_bar, mma_phase, abortp);
-      mma_phase ^= 1u;
-      ok = __all_sync(0xffffffffu, ok);
-      tc_fence_after();
-      if (!ok) break;
-      int nchunk = (keys + 31) >> 5;
-      if (pass == 0) {
-        float bm = -INFINITY;
-        for (int ch = 0; ch < nchunk; ++ch) {
-          uint32_t r[32];
-          tmem_ld32(trow + ch * 32, r);
-          tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (ch * 32 + j < keys) bm = fmaxf(bm, __uint_as_float(r[j]));
-        }
-        float nm = fmaxf(mx, bm);
-        float bs = 0.f;
-        for (int ch = 0; ch < nchunk; ++ch) {
-          uint32_t r[32];
-          tmem_ld32(trow + ch * 32, r);
-          tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (ch * 32 + j < keys) bs += exp2f((__uint_as_float(r[j]) - nm) * c);
-        }
-        sum = sum * exp2f((mx - nm) * c) + bs;
-        mx = nm;
-        tc_fence_before();
-        __syncthreads();               // everyone has read S before the next block's MMA overwrites it
+      ok = mbar_wait(tma_bar, tma_phase, abortp);
+      if (ok) {
         tc_fence_after();
-      } else {
-        float mc = mx * c, inv = 1.0f / sum;
-        for (int ch = 0; ch < nchunk; ++ch) {
-          uint32_t r[32];
-          tmem_ld32(trow + ch * 32, r);
-          tmem_ld_wait();
-          float p[32];
+        uint32_t idesc = make_idesc_mn(AT_QROWS, kpad, false, false);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            float e = exp2f(fmaf(__uint_as_float(r[j]), c, -mc));
-            p[j] = (ch * 32 + j < keys) ? e : 0.f;
-          }
-          if (cls_row) {
-            float* cp = cls_prob + ((size_t)b * H + h) * (T - 1);
-            for (int j = 0; j < 32; ++j) {
-              int key = k0 + ch * 32 + j;
-              if (key >= 1 && key < T) cp[key - 1] = p[j] * inv;
-            }
-          }
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            int key8 = ch * 4 + g;
-            if (key8 * 8 < nbox * AT_BOX) {
-              uint4 v;
-              __nv_bfloat162* hh = reinterpret_cast<__nv_bfloat162*>(&v);
-#pragma unroll
-              for (int i = 0; i < 4; ++i) hh[i] = __floats2bfloat162_rn(p[g * 8 + 2 * i], p[g * 8 + 2 * i + 1]);
-              *reinterpret_cast<uint4*>(pP + p_offset(tid, key8)) = v;
-            }
-          }
-        }
-        fence_async_smem();
-        tc_fence_before();
-        __syncthreads();
-        tc_fence_after();
-        if (tid == 0) {
-          uint32_t idesc = make_idesc_mn(AT_QROWS, AT_D, false, true);
-          for (int k = 0; k < kpad / 16; ++k)
-            umma_bf16(tmem + C_O, make_desc(sP + (k >> 2) * (AT_QROWS * 128) + (k & 3) * 32, 16, 1024),
-                      make_desc(sV + k * (16 * 128), 8192, 1024), idesc, (kb > 0 || k > 0) ? 1u : 0u);
-          umma_commit(mma_bar);
-        }
-        ok = mbar_wait(mma_bar, mma_phase, abortp);      // P, K and V of this block are free again
-        mma_phase ^= 1u;
-        ok = __all_sync(0xffffffffu, ok);
-        tc_fence_after();
+        for (int k = 0; k < AT_D / 16; ++k)
+          umma_bf16(tmem, make_desc(sQ + k * 32, 16, 1024), make_desc(sK + k * 32, 16, 1024), idesc, k > 0 ? 1u : 0u);
+        umma_commit(mma_bar);
       }
     }
+    tma_phase ^= 1u;
+    ok = mbar_wait(mma_bar, mma_phase, abortp);
+    mma_phase ^= 1u;
+    ok = __all_sync(0xffffffffu, ok);
+    tc_fence_after();
+    if (!ok) break;
+    // the block's maximum of this thread's query row (the scores are read again below: cheaper than holding them)
+    float bm = -INFINITY;
+#pragma unroll
+    for (int ch = 0; ch < KB / 32; ++ch) {
+      uint32_t r[32];
+      tmem_ld32(trow + ch * 32, r);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (ch * 32 + j < keys) bm = fmaxf(bm, __uint_as_float(r[j]));
+    }
+    // The reference maximum of a row moves only when the block's maximum exceeds it by more than AT_LONG_SLACK in the
+    // exponent (the probabilities then stay below 2^AT_LONG_SLACK, harmless in bf16 and in the fp32 sum); when it
+    // moves, the accumulated output and sum of that row are scaled down.  The decision is taken per warp, because the
+    // accumulator is read and written with warp-wide instructions; rows that do not move scale by one.
+    if (kb == 0) {
+      mx = bm;
+    } else {
+      bool grow = (bm - mx) * c > AT_LONG_SLACK;
+      if (__any_sync(0xffffffffu, grow)) {
+        float nm = grow ? bm : mx;
+        float f = ex2_fast((mx - nm) * c);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t r[32];
+          tmem_ld32(trow + C_O + half * 32, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * f);
+          tmem_st16(trow + C_O + half * 32, r);
+          tmem_st16(trow + C_O + half * 32 + 16, r + 16);
+        }
+        tmem_st_wait();
+        sum *= f;
+        mx = nm;
+      }
+    }
+    if (cls_row) cls_m[kb] = mx;
+    float mc = mx * c;
+#pragma unroll
+    for (int ch = 0; ch < KB / 32; ++ch) {
+      uint32_t r[32];
+      tmem_ld32(trow + ch * 32, r);
+      tmem_ld_wait();
+      float p[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        float e = ex2_fast(fmaf(__uint_as_float(r[j]), c, -mc));
+        p[j] = (ch * 32 + j < keys) ? e : 0.f;
+        sum += p[j];
+      }
+      if (cls_row) {                  // relative to this block's reference maximum; put on the final scale below
+        float* cp = cls_prob + ((size_t)b * H + h) * (T - 1);
+        for (int j = 0; j < 32; ++j) {
+          int key = k0 + ch * 32 + j;
+          if (key >= 1 && key < T) cp[key - 1] = p[j];
+        }
+      }
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        int key8 = ch * 4 + g;
+        if (key8 * 8 < nbox * AT_BOX) {
+          uint4 v;
+          __nv_bfloat162* hh = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) hh[i] = __floats2bfloat162_rn(p[g * 8 + 2 * i], p[g * 8 + 2 * i + 1]);
+          *reinterpret_cast<uint4*>(pP + p_offset(tid, key8)) = v;
+        }
+      }
+    }
+    fence_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (tid == 0) {
+      uint32_t idesc = make_idesc_mn(AT_QROWS, AT_D, false, true);
+      for (int k = 0; k < kpad / 16; ++k)
+        umma_bf16(tmem + C_O, make_desc(sP + (k >> 2) * (AT_QROWS * 128) + (k & 3) * 32, 16, 1024),
+                  make_desc(sV + k * (16 * 128), 8192, 1024), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+      umma_commit(mma_bar);
+    }
+    ok = mbar_wait(mma_bar, mma_phase, abortp);      // P, K and V of this block are free again; O is complete
+    mma_phase ^= 1u;
+    ok = __all_sync(0xffffffffu, ok);
+    tc_fence_after();
+  }
+  if (ok && cls_warp) {
+    // the classification row's probabilities: from each block's reference maximum to the final one, over the row sum
+    float fm = __shfl_sync(0xffffffffu, mx, 0), fs = __shfl_sync(0xffffffffu, sum, 0);
+    float inv0 = 1.0f / fs;
+    __syncwarp();
+    float* cp = cls_prob + ((size_t)b * H + h) * (T - 1);
+    for (int key = 1 + (tid & 31); key < T; key += 32)
+      cp[key - 1] *= ex2_fast((cls_m[key / KB] - fm) * c) * inv0;
   }
   int q = q0 + tid;
   if (ok) {
@@ -746,7 +772,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
 // Returns 0 when the tensor-core kernel took the problem, non-zero when the caller must use another kernel.
 int attention_fwd_tc(const Ctx& c, const void* qkv, void* out, float* lse, float* cls_prob, int B, int T, int H, int d) {
   using namespace tc;
-  if (c.dtype != 1 || d != AT_D || T < 1) return -1;
+  if (c.dtype != 1 || d != AT_D || T < 1 || T > AT_LONG_KB * AT_LONG_MAXBLK) return -1;
   if (((uintptr_t)qkv & 15) || ((uintptr_t)out & 15)) return -1;
   CUtensorMap map;
   if (!make_map(&map, qkv, (uint64_t)3 * H * d, (uint64_t)B * T, (uint64_t)3 * H * d, AT_BOX)) return -2;

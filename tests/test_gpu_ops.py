@@ -76,6 +76,41 @@ def test_attention_forward(dtype, tol, tc, B, T, H, d):
         assert rel(cp.cpu().numpy().astype(np.float64), A[:, :, 0, 1:]) < (2e-6 if dtype == "fp32" else 2e-5)
 
 
+@pytest.mark.parametrize("B,T,H", [(2, 577, 3), (1, 290, 2), (1, 512, 1), (3, 1000, 2)])
+@pytest.mark.parametrize("pattern", ["rising", "steps", "falling"])
+def test_long_attention_when_the_row_maximum_jumps_between_key_blocks(B, T, H, pattern):
+    """The kernel for more than 256 tokens walks the keys once and rescales its accumulator when a block's row maximum
+    exceeds the reference by more than eight binary orders.  Standard normal inputs never do that after the first
+    block, so here the key rows grow (or shrink) from one 64-key block to the next: 'rising' makes every block jump,
+    'steps' makes some rows jump late and leaves others alone, 'falling' must never rescale."""
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    d = 64
+    rng = np.random.default_rng(T + len(pattern))
+    qkv = rng.standard_normal((B, T, 3, H, d))
+    blk = np.arange(T) // 64
+    if pattern == "rising":
+        f = 1.0 + 1.5 * blk
+    elif pattern == "falling":
+        f = 1.0 + 1.5 * (blk.max() - blk)
+    else:
+        f = np.where(blk % 3 == 2, 6.0, 1.0)
+    qkv[:, :, 1] *= f[None, :, None, None]
+    if pattern == "steps":                                     # half of the queries barely see the large keys
+        qkv[:, ::2, 0] *= 0.05
+    qkv = synth.round_to_bf16(qkv)
+    q, k, v = (qkv[:, :, i].transpose(0, 2, 1, 3) for i in range(3))
+
+    class Cfg:
+        heads = H
+        dim = H * d
+    o, A = O.attention_fwd(Cfg, q, k, v)
+    out, cp = Bd.bsr_attention_forward(torch.as_tensor(qkv.astype(np.float32)).cuda().bfloat16(), H, use_tensor_cores=True)
+    torch.cuda.synchronize()
+    assert rel(out.float().cpu().numpy().astype(np.float64), O.merge_heads(o)) < 6e-3
+    assert rel(cp.cpu().numpy().astype(np.float64), A[:, :, 0, 1:]) < 2e-5
+
+
 TC_SHAPES = [(128, 256, 64), (197, 384, 192), (1000, 3072, 768), (2600, 768, 3072), (100, 72, 40), (9216, 2304, 768)]
 
 
