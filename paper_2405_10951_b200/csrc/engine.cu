@@ -615,8 +615,18 @@ int block_forward(bsr_handle* h, const Ctx& c, int l, int B, const BlockBufs& bb
     // MoE layer in place of the FFN (Section 5.2): route, run the chosen experts as grouped GEMMs, combine
     int E = d.moe_experts, K = d.moe_top_k;
     MoeBufs mb = moe_bufs(h, bb);
-    moe_route(c, mb, h->base + bb.y2, h->wb(l, "moe.gate.weight"), task_ids, tail ? 1 : Tf, Mf, D, E, K, d.num_tasks);
     int cap = moe_rows_cap(Mf, E, K);
+    // Gate logits of every task at once as one product y Wg^T ([Mf, D] x [D, tasks E]) on the tensor cores; they land in
+    // the expert-output buffer, which is not written before the routing has consumed them.  (Small or odd gate shapes:
+    // the routing kernel forms the logits itself.)
+    int NG = d.num_tasks * E;
+    const float* logits = nullptr;
+    if (c.use_tc && d.dtype == BSR_DTYPE_BF16 && Mf >= 256 && NG % 8 == 0 && (size_t)Mf * NG <= (size_t)cap * D) {
+      GemmEpilogue none;
+      gemm(c, h->base + bb.y2, D, 1, h->wb(l, "moe.gate.weight"), D, 1, mb.og, 1, Mf, NG, D, none);
+      logits = mb.og;
+    }
+    moe_route(c, mb, h->base + bb.y2, h->wb(l, "moe.gate.weight"), task_ids, tail ? 1 : Tf, Mf, D, E, K, d.num_tasks, logits, NG);
     GemmEpilogue m1;
     m1.bias = (const float*)h->wb(l, "moe.fc1.bias");
     m1.act = 1;

@@ -259,9 +259,11 @@ struct MoeBufs {
 };
 int moe_rows_cap(int M, int E, int K);
 int moe_blocks(int M);
-// y [M, D]: routes every token, builds the segment tables and gathers the expert inputs into b.xg.
+// y [M, D]: routes every token, builds the segment tables and gathers the expert inputs into b.xg.  logits (optional):
+// the gate logits of all tasks, [M, logit_stride] with task t's experts at columns t E .. t E + E - 1, formed beforehand
+// (y times the transposed gate matrices); without them the kernel forms each token's own task's logits itself.
 void moe_route(const Ctx& c, const MoeBufs& b, const void* y, const void* wg, const int* task_ids, int tokens_per_image, int M,
-               int D, int E, int K, int num_tasks);
+               int D, int E, int K, int num_tasks, const float* logits = nullptr, int logit_stride = 0);
 void moe_combine(const Ctx& c, const MoeBufs& b, const float* res, float* out, int M, int D, int K);
 void moe_combine_bwd(const Ctx& c, const MoeBufs& b, const float* dout, void* dog, float* dw, int M, int D, int E, int K);
 void moe_seg_colsum(const Ctx& c, const MoeBufs& b, const void* x, int cols, int E, float* out);

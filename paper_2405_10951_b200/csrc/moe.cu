@@ -21,9 +21,9 @@ constexpr int MOE_ROUTE_TOKENS = 16;
 static_assert(MOE_BLOCK_TOKENS % MOE_ROUTE_TOKENS == 0, "a routing block must not straddle two counting groups");
 template <typename T>
 __global__ void __launch_bounds__(MOE_ROUTE_WARPS * 32)
-moe_route_kernel(const T* __restrict__ y, const T* __restrict__ wg, const int* __restrict__ task_ids, int tokens_per_image,
-                 int M, int D, int E, int K, int gate_elems_in_smem, int* __restrict__ eidx, float* __restrict__ ew,
-                 int* __restrict__ blk_counts) {
+moe_route_kernel(const T* __restrict__ y, const T* __restrict__ wg, const float* __restrict__ logits, int logit_stride,
+                 const int* __restrict__ task_ids, int tokens_per_image, int M, int D, int E, int K, int gate_elems_in_smem,
+                 int* __restrict__ eidx, float* __restrict__ ew, int* __restrict__ blk_counts) {
   // A block takes MOE_ROUTE_TOKENS consecutive tokens (a divisor of MOE_BLOCK_TOKENS, so all of them fall into one
   // counting group), a warp one token at a time.  Expert by expert the lanes multiply 16-byte pieces of the token's row
   // of y (coalesced; from L1 after the first expert) with the same pieces of the gate row -- the gate matrices of all
@@ -31,12 +31,14 @@ moe_route_kernel(const T* __restrict__ y, const T* __restrict__ wg, const int* _
   // in a fixed (butterfly) order; lane e keeps logit e.  The top k then come from k warp-wide maxima (among equal
   // logits the lowest expert id, found with a ballot).  Few registers, so many tokens are in flight per SM: the work
   // per token is a chain of dependent loads.  The per-group expert counts (zeroed before the launch) are integer sums.
+  // When `logits` is given (row stride logit_stride, the E logits of task t at column t E), the products were formed
+  // by a GEMM over all tasks' gates beforehand and lane e just reads its logit.
   extern __shared__ __align__(16) unsigned char route_smem[];
   __shared__ int counts[MOE_MAX_E];
   constexpr int N = Pack<T>::N;
   if (threadIdx.x < MOE_MAX_E) counts[threadIdx.x] = 0;
   const T* gates = wg;
-  if (gate_elems_in_smem > 0) {
+  if (logits == nullptr && gate_elems_in_smem > 0) {
     T* sg = reinterpret_cast<T*>(route_smem);
     for (int i = threadIdx.x * N; i < gate_elems_in_smem; i += blockDim.x * N)
       *reinterpret_cast<uint4*>(sg + i) = *reinterpret_cast<const uint4*>(wg + i);
@@ -53,6 +55,9 @@ moe_route_kernel(const T* __restrict__ y, const T* __restrict__ wg, const int* _
     const T* yr = y + (size_t)tok * D;
     const T* gt = gates + (size_t)task * E * D;
     float logit = -INFINITY;                      // lane e: logit of expert e
+    if (logits != nullptr) {
+      if (lane < E) logit = logits[(size_t)tok * logit_stride + task * E + lane];
+    } else
 #pragma unroll 4
     for (int e = 0; e < E; ++e) {
       float acc = 0.f;
@@ -342,24 +347,24 @@ int moe_rows_cap(int M, int E, int K) { return ((M * K + E * 127) + 127) & ~127;
 int moe_blocks(int M) { return ceil_div(M, MOE_BLOCK_TOKENS); }
 
 void moe_route(const Ctx& c, const MoeBufs& b, const void* y, const void* wg, const int* task_ids, int tokens_per_image, int M,
-               int D, int E, int K, int num_tasks) {
+               int D, int E, int K, int num_tasks, const float* logits, int logit_stride) {
   int nblk = moe_blocks(M);
   int rows_cap = moe_rows_cap(M, E, K);
   note_launch(4);
   size_t es = c.dtype == 0 ? 4 : 2;
   size_t gate_elems = (size_t)(num_tasks < 1 ? 1 : num_tasks) * E * D;
   size_t smem = gate_elems * es;
-  if (smem > 16 * 1024) { smem = 0; gate_elems = 0; }       // not worth staging for 16 tokens: the gates are read through L1 instead
+  if (smem > 16 * 1024 || logits != nullptr) { smem = 0; gate_elems = 0; }       // not worth staging for 16 tokens: the gates are read through L1 instead
   static SmemLimit lim[2];
   int rblk = ceil_div(M, MOE_ROUTE_TOKENS);
   cudaMemsetAsync(b.blk_counts, 0, (size_t)nblk * E * sizeof(int), c.stream);
   if (c.dtype == 0) {
     ensure_smem(lim[0], moe_route_kernel<float>, smem);
-    moe_route_kernel<float><<<rblk, MOE_ROUTE_WARPS * 32, smem, c.stream>>>((const float*)y, (const float*)wg, task_ids, tokens_per_image, M, D, E, K,
+    moe_route_kernel<float><<<rblk, MOE_ROUTE_WARPS * 32, smem, c.stream>>>((const float*)y, (const float*)wg, logits, logit_stride, task_ids, tokens_per_image, M, D, E, K,
                                                                         (int)gate_elems, b.eidx, b.ew, b.blk_counts);
   } else {
     ensure_smem(lim[1], moe_route_kernel<bf16>, smem);
-    moe_route_kernel<bf16><<<rblk, MOE_ROUTE_WARPS * 32, smem, c.stream>>>((const bf16*)y, (const bf16*)wg, task_ids, tokens_per_image, M, D, E, K,
+    moe_route_kernel<bf16><<<rblk, MOE_ROUTE_WARPS * 32, smem, c.stream>>>((const bf16*)y, (const bf16*)wg, logits, logit_stride, task_ids, tokens_per_image, M, D, E, K,
                                                                        (int)gate_elems, b.eidx, b.ew, b.blk_counts);
   }
   moe_scan_kernel<<<1, 128, 0, c.stream>>>(b.blk_counts, nblk, E, rows_cap / 128, b.blk_off, b.seg_start, b.tile_expert);
