@@ -351,10 +351,24 @@ const char* bsr_static_last_error(void);
 
 /* Multi-head self-attention, Eq. 1, on packed projections.  qkv_dev [batch, t, 3, heads, d] in
  * `dtype`; out_dev [batch, t, heads*d]; cls_prob_dev_out optional [batch, heads, t-1] float32: the
- * classification token's row of the attention map without its own column. d must be 64 or less
- * and a multiple of 8.  use_tensor_cores != 0 selects the tcgen05 kernels (bf16, d = 64). */
+ * classification token's row of the attention map without its own column; lse_dev_out optional
+ * [batch, heads, t] float32: log of the softmax denominator of every row (natural logarithm, of the scaled scores),
+ * which bsr_attention_backward reads.  d must be 64 or less and a multiple of 8.  use_tensor_cores != 0 selects the
+ * tcgen05 kernels (bf16, d = 64).  All buffers are caller-owned device memory. */
 int32_t bsr_attention_forward(const void* qkv_dev, int32_t dtype, int32_t batch, int32_t t, int32_t heads,
-                              int32_t d, void* out_dev, float* cls_prob_dev_out, int32_t use_tensor_cores, void* stream);
+                              int32_t d, void* out_dev, float* cls_prob_dev_out, float* lse_dev_out,
+                              int32_t use_tensor_cores, void* stream);
+
+/* Backward of Eq. 1 (the attention part of Eq. 3): from dout_dev [batch, t, heads*d], the gradient at the attention
+ * output, to dqkv_dev_out [batch, t, 3, heads, d], the gradient at the packed projections; both in `dtype`.  The
+ * attention map is recomputed from qkv_dev and lse_dev (as written by bsr_attention_forward).  score_grad_dev optional
+ * [batch, t-1] float32: a gradient arriving at the head-mean classification scores of Eq. 6 (from the fused token);
+ * every head's classification row receives 1/heads of it.  delta_scratch_dev: batch*heads*t floats of caller-owned
+ * scratch (used by the kernels without tensor cores; may be null when use_tensor_cores != 0).  use_tensor_cores != 0
+ * selects the tcgen05 kernels (bf16, d = 64, t <= 256) and fails with BSR_ERR_UNSUPPORTED outside their range. */
+int32_t bsr_attention_backward(const void* qkv_dev, const void* dout_dev, const float* lse_dev, const float* score_grad_dev,
+                               int32_t dtype, int32_t batch, int32_t t, int32_t heads, int32_t d, void* dqkv_dev_out,
+                               float* delta_scratch_dev, int32_t use_tensor_cores, void* stream);
 
 #ifdef __cplusplus
 }

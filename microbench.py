@@ -24,20 +24,25 @@ sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
 from paper_2405_10951_b200 import binding as Bd  # noqa: E402
 
 
-def timed(fn, iters, flush=None):
+def timed(fn, iters, flush=None, reps=1):
+    """Mean time of one call in ms.  reps > 1: that many calls back to back inside each event pair (a kernel shorter
+    than the host's launch path is otherwise timed together with the launch gap); not combined with an L2 flush."""
     for _ in range(3):
         fn()
     torch.cuda.synchronize()
+    if flush is not None:
+        reps = 1
     total = 0.0
     for _ in range(iters):
         if flush is not None:
             flush.zero_()                       # evict the previous iteration's data from L2
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        fn()
+        for _ in range(reps):
+            fn()
         e1.record()
         torch.cuda.synchronize()
-        total += e0.elapsed_time(e1)
+        total += e0.elapsed_time(e1) / reps
     return total / iters
 
 
@@ -60,6 +65,7 @@ def main():
     ap.add_argument("--keep", type=float, default=0.7)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
     ap.add_argument("--flush-l2", action="store_true")
+    ap.add_argument("--backward", action="store_true", help="attention: also time the backward pass (--mode 0: without tensor cores)")
     a = ap.parse_args()
     torch.manual_seed(0)
     dev = "cuda"
@@ -87,7 +93,12 @@ def main():
         if a.e4m3:
             ms = timed(lambda: Bd.bsr_linear_forward_e4m3(x, w, b, act_gelu=a.gelu), a.iters, flush)     # includes the two row-quantisation passes
         else:
-            ms = timed(lambda: Bd.bsr_linear_forward(x, w, b, r, act_gelu=a.gelu, use_tensor_cores=a.mode), a.iters, flush)
+            import ctypes as C
+            y = torch.empty(a.m, a.n, dtype=torch.bfloat16, device=dev)      # output allocated once: the timed region holds launches only
+            L, st = Bd.lib(), C.c_void_p(torch.cuda.current_stream().cuda_stream)
+            ptr = lambda t: C.c_void_p(t.data_ptr()) if t is not None else None
+            ms = timed(lambda: L.bsr_linear_forward(ptr(x), ptr(w), ptr(b), ptr(r), ptr(y), a.m, a.n, a.k, Bd.DTYPE_BF16, int(a.gelu), a.mode, st),
+                       a.iters, flush, reps=10)
         out.update(m=a.m, n=a.n, k=a.k, gelu=a.gelu, mode=a.mode, e4m3=a.e4m3, us=ms * 1e3, tflops=2.0 * a.m * a.n * a.k / ms / 1e9)
     elif a.what == "backward":
         x = torch.randn(a.m, a.k, device=dev).bfloat16()
@@ -129,9 +140,21 @@ def main():
 
         def run():
             for _ in range(reps):
-                L.bsr_attention_forward(ptr(qkv), 1, B, T, H, 64, ptr(o), ptr(cp), 1, st)
+                L.bsr_attention_forward(ptr(qkv), 1, B, T, H, 64, ptr(o), ptr(cp), None, 1, st)
         ms = timed(run, a.iters, flush) / reps
         out.update(batch=B, heads=H, tokens=T, us=ms * 1e3, tflops=4.0 * B * H * T * T * 64 / ms / 1e9)
+        if a.backward:
+            lse = torch.empty(B, H, T, device=dev, dtype=torch.float32)
+            L.bsr_attention_forward(ptr(qkv), 1, B, T, H, 64, ptr(o), ptr(cp), ptr(lse), 1, st)
+            do = torch.randn(B, T, H * 64, device=dev).bfloat16()
+            dq = torch.empty_like(qkv)
+            delta = torch.empty(B * H * T, device=dev, dtype=torch.float32)
+
+            def run_b():
+                for _ in range(reps):
+                    L.bsr_attention_backward(ptr(qkv), ptr(do), ptr(lse), None, 1, B, T, H, 64, ptr(dq), ptr(delta), a.mode, st)
+            msb = timed(run_b, a.iters, flush) / reps
+            out.update(backward_us=msb * 1e3, backward_tflops=10.0 * B * H * T * T * 64 / msb / 1e9, backward_tensor_cores=a.mode)
     print(json.dumps(out), flush=True)
 
 

@@ -217,6 +217,21 @@ def attention_fwd(cfg, q, k, v):
     return A @ v, A
 
 
+def attention_bwd(cfg, A, q, k, v, do, dA_cls=None):
+    """Chain rule through Eq. 1 for one block.  A [B, H, T, T] the attention map, q, k, v, do [B, H, T, d];
+    dA_cls [B, T] (optional): a gradient that reaches the classification row of every head's map directly (through
+    the scores of Eq. 6), added to that row of dA.  Returns dq, dk, dv."""
+    d = q.shape[-1]
+    dA = do @ v.transpose(0, 1, 3, 2)
+    if dA_cls is not None:
+        dA[:, :, 0, :] += dA_cls[:, None, :]
+    dv = A.transpose(0, 1, 3, 2) @ do
+    dS = A * (dA - (dA * A).sum(axis=-1, keepdims=True))
+    dq = dS @ k / np.sqrt(d)
+    dk = dS.transpose(0, 1, 3, 2) @ q / np.sqrt(d)
+    return dq, dk, dv
+
+
 def split_heads(cfg, qkv):
     B, T, _ = qkv.shape
     H, d = cfg.heads, cfg.dim // cfg.heads
@@ -411,14 +426,7 @@ def block_bwd(cfg, params, l, dout, c, task_ids, grads, want_param_grads, need_d
     B, T, D = doc.shape
     H, d = cfg.heads, D // cfg.heads
     do = doc.reshape(B, T, H, d).transpose(0, 2, 1, 3)
-    A, q, k, v = c["A"], c["q"], c["k"], c["v"]
-    dA = do @ v.transpose(0, 1, 3, 2)
-    if dA_cls is not None:
-        dA[:, :, 0, :] += dA_cls[:, None, :]
-    dv = A.transpose(0, 1, 3, 2) @ do
-    dS = A * (dA - (dA * A).sum(axis=-1, keepdims=True))
-    dq = dS @ k / np.sqrt(d)
-    dk = dS.transpose(0, 1, 3, 2) @ q / np.sqrt(d)
+    dq, dk, dv = attention_bwd(cfg, c["A"], c["q"], c["k"], c["v"], do, dA_cls)
     dqkv = np.stack([dq, dk, dv], axis=0).transpose(1, 3, 0, 2, 4).reshape(B, T, 3 * D)
     dy1, g["attn.qkv.weight"], g["attn.qkv.bias"] = linear_bwd(dqkv, c["y1"], params[p + "attn.qkv.weight"])
     dln1, g["norm1.weight"], g["norm1.bias"] = layer_norm_bwd(dy1, c["ln1"], params[p + "norm1.weight"])

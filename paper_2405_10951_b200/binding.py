@@ -27,7 +27,7 @@ STATUS_NAMES = {0: "BSR_OK", -1: "BSR_ERR_INVALID_ARG", -2: "BSR_ERR_UNSUPPORTED
 EXPORTS = ["bsr_token_schedule", "bsr_workspace_bytes", "bsr_create", "bsr_destroy", "bsr_last_error", "bsr_set_param",
            "bsr_get_tensor", "bsr_set_lr", "bsr_set_step", "bsr_train_step", "bsr_train_steps", "bsr_train_step_host", "bsr_forward_backward", "bsr_grad_buffer", "bsr_optimizer_step", "bsr_eval_forward", "bsr_get_footprint",
            "bsr_sync_status", "bsr_selftest_wait_expiry", "bsr_set_gemm_mode", "bsr_set_graph_mode", "bsr_profile_enable", "bsr_profile_read", "bsr_profile_launches", "bsr_token_select", "bsr_gather_fuse", "bsr_linear_forward", "bsr_linear_forward_e4m3", "bsr_linear_backward",
-           "bsr_linear_backward_static", "bsr_static_last_error", "bsr_attention_forward"]
+           "bsr_linear_backward_static", "bsr_static_last_error", "bsr_attention_forward", "bsr_attention_backward"]
 
 
 class bsr_dims(C.Structure):
@@ -113,7 +113,8 @@ def lib() -> C.CDLL:
         L.bsr_linear_backward.argtypes = [vp, vp, vp, vp, f32p, i32, i32, i32, i32, i32, f32p, C.c_size_t, vp]
         L.bsr_linear_backward_static.argtypes = [vp, vp, vp, vp, f32p, i32, i32, i32, vp]
         L.bsr_static_last_error.argtypes = []
-        L.bsr_attention_forward.argtypes = [vp, i32, i32, i32, i32, i32, vp, f32p, i32, vp]
+        L.bsr_attention_forward.argtypes = [vp, i32, i32, i32, i32, i32, vp, f32p, f32p, i32, vp]
+        L.bsr_attention_backward.argtypes = [vp, vp, f32p, f32p, i32, i32, i32, i32, i32, vp, f32p, i32, vp]
         for name in EXPORTS:
             if name not in ("bsr_last_error", "bsr_static_last_error"):
                 getattr(L, name).restype = C.c_int32
@@ -253,16 +254,32 @@ def bsr_linear_backward_static(x, w, dy, dx=None, dw=None):
     return dx, dw
 
 
-def bsr_attention_forward(qkv, heads: int, want_cls_prob: bool = True, use_tensor_cores: bool = False):
-    """qkv: CUDA tensor [B, T, 3, H, d].  Returns (out [B, T, H*d], cls_prob [B, H, T-1] or None)."""
+def bsr_attention_forward(qkv, heads: int, want_cls_prob: bool = True, use_tensor_cores: bool = False, want_lse: bool = False):
+    """qkv: CUDA tensor [B, T, 3, H, d].  Returns (out [B, T, H*d], cls_prob [B, H, T-1] or None), and with want_lse
+    also the log of every row's softmax denominator [B, H, T]."""
     import torch
     B, T, three, H, d = qkv.shape
     assert three == 3 and H == heads
     out = torch.empty((B, T, H * d), dtype=qkv.dtype, device=qkv.device)
     cp = torch.empty((B, H, T - 1), dtype=torch.float32, device=qkv.device) if want_cls_prob else None
+    lse = torch.empty((B, H, T), dtype=torch.float32, device=qkv.device) if want_lse else None
     dt = DTYPE_FP32 if qkv.dtype == torch.float32 else DTYPE_BF16
-    _check(lib().bsr_attention_forward(_ptr(qkv), dt, B, T, H, d, _ptr(out), _ptr(cp), int(use_tensor_cores), _stream()))
-    return out, cp
+    _check(lib().bsr_attention_forward(_ptr(qkv), dt, B, T, H, d, _ptr(out), _ptr(cp), _ptr(lse), int(use_tensor_cores), _stream()))
+    return (out, cp, lse) if want_lse else (out, cp)
+
+
+def bsr_attention_backward(qkv, dout, lse, score_grad=None, use_tensor_cores: bool = False, out=None):
+    """qkv [B, T, 3, H, d], dout [B, T, H*d] (same dtype), lse [B, H, T] float32 from bsr_attention_forward,
+    score_grad optional [B, T-1] float32.  Returns dqkv [B, T, 3, H, d]."""
+    import torch
+    B, T, three, H, d = qkv.shape
+    assert three == 3 and tuple(dout.shape) == (B, T, H * d) and dout.dtype == qkv.dtype
+    dqkv = out if out is not None else torch.empty_like(qkv)
+    delta = None if use_tensor_cores else torch.empty(B * H * T, dtype=torch.float32, device=qkv.device)
+    dt = DTYPE_FP32 if qkv.dtype == torch.float32 else DTYPE_BF16
+    _check(lib().bsr_attention_backward(_ptr(qkv), _ptr(dout), _ptr(lse), _ptr(score_grad), dt, B, T, H, d, _ptr(dqkv), _ptr(delta),
+                                        int(use_tensor_cores), _stream()))
+    return dqkv
 
 
 class Engine:

@@ -767,6 +767,251 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
   if (tid == 0 && abort_flag && status != nullptr) atomicOr(status, STATUS_TIMEOUT);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Backward for 128 < T <= 256: one CTA of 256 threads per (image, head), queries and keys in two tiles of 128.
+// The formulas are those of the kernel above; what changes is that delta_i = sum_j P_ij dP_ij runs over both key
+// tiles, so a first sweep over the four (query tile, key tile) pairs forms S and dP only to accumulate delta, and a
+// second sweep (key tile outer, query tile inner) forms them again, writes P and dS as bf16 operand tiles and issues
+// the three products: dQ_i accumulates over the key tiles, dK_j and dV_j over the query tiles, all in tensor memory
+// (S 128 + dP 128 + dQ 2 x 64 + dK 64 + dV 64 = 512 columns: one CTA per SM).  No step leaves the loop early: after a
+// wait that expired the remaining steps only keep the barriers in step.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256, 1)
+attn_bwd_tc256_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_constant__ CUtensorMap map_do,
+                      const float* __restrict__ lse, const float* __restrict__ cls_extra, bf16* __restrict__ dqkv,
+                      int B, int T, int H, int* status) {
+  extern __shared__ unsigned char smem_dyn[];
+  uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+  constexpr uint32_t TILE = 2 * AT_BOX_BYTES;            // 128 rows x 128 bytes
+  constexpr uint32_t CH = TILE;                          // one 64-key chunk of a P / dS tile: 128 query rows x 128 bytes
+  uint32_t sQ = base, sK = sQ + 2 * TILE, sG = sK + 2 * TILE, sV = sG + 2 * TILE, sP = sV + 2 * TILE, sS = sP + 2 * TILE;
+  uint32_t arrays = sS + 2 * TILE;
+  float* sdelta = reinterpret_cast<float*>(base_ptr + (arrays - base));     // [256] delta of every query row
+  float* sl2 = sdelta + 256;                                                 // [256] log-sum-exp in binary orders
+  float* exs = sl2 + 256;                                                    // [256] classification-row score gradients / H
+  float* red = exs + 256;                                                    // [2][128] the halves' shares of delta
+  uint32_t bars = arrays + 4 * 256 * 4;
+  unsigned char* pP = base_ptr + (sP - base);
+  unsigned char* pS = base_ptr + (sS - base);
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  int tid = threadIdx.x, warp = tid >> 5;
+  int rowl = tid & 127, half = tid >> 7;
+  int bh = blockIdx.x, b = bh / H, h = bh % H;
+  uint32_t tma_bar = bars, mma_bar = bars + 8, mma2_bar = bars + 16;
+  if (tid == 0) {
+    abort_flag = 0;
+    mbar_init(tma_bar, 1);
+    mbar_init(mma_bar, 1);
+    mbar_init(mma2_bar, 3);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    tmem_alloc(smem_u32(&tmem_slot), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  uint32_t tmem = tmem_slot;
+  constexpr uint32_t C_S = 0, C_DP = 128, C_DQ = 256, C_DK = 384, C_DV = 448;
+  volatile int* abortp = &abort_flag;
+  const int tpad = (T + 15) & ~15;
+  const int row0 = b * T;
+  if (tid == 0) {
+    mbar_expect_tx(tma_bar, 8 * TILE);
+    for (int j = 0; j < 4; ++j) {                        // rows past the image: the next image's, or zero fill; never used
+      tma_load_2d(sQ + j * AT_BOX_BYTES, &map_qkv, tma_bar, h * AT_D, row0 + j * AT_BOX);
+      tma_load_2d(sK + j * AT_BOX_BYTES, &map_qkv, tma_bar, (H + h) * AT_D, row0 + j * AT_BOX);
+      tma_load_2d(sV + j * AT_BOX_BYTES, &map_qkv, tma_bar, (2 * H + h) * AT_D, row0 + j * AT_BOX);
+      tma_load_2d(sG + j * AT_BOX_BYTES, &map_do, tma_bar, h * AT_D, row0 + j * AT_BOX);
+    }
+  }
+  const bool has_extra = cls_extra != nullptr;
+  sl2[tid] = tid < T ? lse[((size_t)b * H + h) * T + tid] * 1.4426950408889634f : 0.f;
+  exs[tid] = (has_extra && tid >= 1 && tid < T) ? cls_extra[(size_t)b * (T - 1) + tid - 1] * (1.0f / (float)H) : 0.f;
+  __syncthreads();
+  bool ok = true;
+  if (tid == 0) ok = mbar_wait(tma_bar, 0, abortp);
+  const float c = 0.125f * 1.4426950408889634f;
+  const uint32_t trow = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+  uint32_t ph1 = 0, ph2 = 0;
+
+  // S = Q_i K_j^T and dP = dO_i V_j^T into tensor memory; everyone waits for them
+  auto scores = [&](int i, int j) {
+    tc_fence_before();
+    __syncthreads();                       // the previous step's reads of S / dP (and of the operand tiles) are over
+    tc_fence_after();
+    if (tid == 0 && ok && !abort_flag) {
+      int kpad = min(128, tpad - 128 * j);
+      uint32_t idesc = make_idesc_mn(AT_QROWS, kpad, false, false);
+      uint32_t q = sQ + i * TILE, k_ = sK + j * TILE, g = sG + i * TILE, v = sV + j * TILE;
+#pragma unroll
+      for (int k = 0; k < AT_D / 16; ++k)
+        umma_bf16(tmem + C_S, make_desc(q + k * 32, 16, 1024), make_desc(k_ + k * 32, 16, 1024), idesc, k > 0 ? 1u : 0u);
+#pragma unroll
+      for (int k = 0; k < AT_D / 16; ++k)
+        umma_bf16(tmem + C_DP, make_desc(g + k * 32, 16, 1024), make_desc(v + k * 32, 16, 1024), idesc, k > 0 ? 1u : 0u);
+      umma_commit(mma_bar);
+    }
+    bool w = mbar_wait(mma_bar, ph1, abortp);
+    ph1 ^= 1u;
+    ok = __all_sync(0xffffffffu, ok && w);
+    tc_fence_after();
+  };
+
+  // ---- first sweep: delta of every query row ----
+  for (int i = 0; i < 2; ++i) {
+    const int row = i * 128 + rowl;
+    const bool valid_row = row < T;
+    const bool extra_row = (row == 0 && has_extra);
+    const float l2 = sl2[row];
+    float dacc = 0.f;
+    for (int j = 0; j < 2; ++j) {
+      scores(i, j);
+      const int kbase = j * 128;
+      const int kvalid = min(128, T - kbase);
+      if (ok) {
+        for (int kk = 4 * half; kk < 4 * half + 4 && kk * 16 < kvalid; ++kk) {
+          uint32_t rs[16], rp[16];
+          tmem_ld16(trow + C_S + kk * 16, rs);
+          tmem_ld16(trow + C_DP + kk * 16, rp);
+          tmem_ld_wait();
+          if (valid_row) {
+            float d0 = 0.f, d1 = 0.f;
+#pragma unroll
+            for (int jj = 0; jj < 16; jj += 2) {
+              int key = kbase + kk * 16 + jj;
+              float p0 = key < T ? ex2_fast(fmaf(__uint_as_float(rs[jj]), c, -l2)) : 0.f;
+              float p1 = key + 1 < T ? ex2_fast(fmaf(__uint_as_float(rs[jj + 1]), c, -l2)) : 0.f;
+              float e0 = __uint_as_float(rp[jj]), e1 = __uint_as_float(rp[jj + 1]);
+              if (extra_row) { e0 += exs[key]; e1 += exs[key + 1]; }
+              d0 = fmaf(p0, e0, d0);
+              d1 = fmaf(p1, e1, d1);
+            }
+            dacc += d0 + d1;
+          }
+        }
+      }
+    }
+    red[half * AT_QROWS + rowl] = dacc;
+    __syncthreads();
+    if (half == 0) sdelta[row] = red[rowl] + red[AT_QROWS + rowl];
+  }
+
+  // ---- second sweep: P and dS tiles, the three products ----
+  auto store_rows = [&](uint32_t col, int which, int row) {      // 64 accumulator columns of `row` -> dqkv[.., which, h, :]
+    uint32_t r[32];
+    tmem_ld32(trow + col + half * 32, r);
+    tmem_ld_wait();
+    if (row < T) {
+      bf16* drow = dqkv + (((size_t)b * T + row) * 3 + which) * H * AT_D + (size_t)h * AT_D + half * 32;
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        float v[8];
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) v[jj] = __uint_as_float(r[g * 8 + jj]);
+        store16(drow + g * 8, v);
+      }
+    }
+  };
+  for (int j = 0; j < 2; ++j) {
+    const int kbase = j * 128;
+    const int kvalid = min(128, T - kbase);
+    const int kpad = min(128, tpad - kbase);
+    for (int i = 0; i < 2; ++i) {
+      scores(i, j);                          // its leading barrier also orders the delta written above before its use
+      const int row = i * 128 + rowl;
+      const bool valid_row = row < T;
+      const bool extra_row = (row == 0 && has_extra);
+      const float l2 = sl2[row];
+      const float delta = sdelta[row];
+      const int qpad = min(128, tpad - 128 * i);
+      if (ok) {
+        for (int kk = 4 * half; kk < 4 * half + 4; ++kk) {
+          float p[16], ds[16];
+#pragma unroll
+          for (int jj = 0; jj < 16; ++jj) { p[jj] = 0.f; ds[jj] = 0.f; }
+          if (kk * 16 < kvalid) {
+            uint32_t rs[16], rp[16];
+            tmem_ld16(trow + C_S + kk * 16, rs);
+            tmem_ld16(trow + C_DP + kk * 16, rp);
+            tmem_ld_wait();
+            if (valid_row) {
+#pragma unroll
+              for (int jj = 0; jj < 16; ++jj) {
+                int key = kbase + kk * 16 + jj;
+                float pv = key < T ? ex2_fast(fmaf(__uint_as_float(rs[jj]), c, -l2)) : 0.f;
+                float dp = __uint_as_float(rp[jj]);
+                if (extra_row) dp += exs[key];
+                p[jj] = pv;
+                ds[jj] = pv * (dp - delta) * 0.125f;
+              }
+            }
+          }
+#pragma unroll
+          for (int g = 0; g < 2; ++g) {
+            uint4 vp, vs;
+            __nv_bfloat162* hp = reinterpret_cast<__nv_bfloat162*>(&vp);
+            __nv_bfloat162* hs = reinterpret_cast<__nv_bfloat162*>(&vs);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              hp[e] = __floats2bfloat162_rn(p[g * 8 + 2 * e], p[g * 8 + 2 * e + 1]);
+              hs[e] = __floats2bfloat162_rn(ds[g * 8 + 2 * e], ds[g * 8 + 2 * e + 1]);
+            }
+            int key8 = kk * 2 + g;
+            uint32_t off = (uint32_t)(key8 >> 3) * CH + (uint32_t)rowl * 128u + (uint32_t)(((key8 & 7) ^ (rowl & 7)) << 4);
+            *reinterpret_cast<uint4*>(pP + off) = vp;
+            *reinterpret_cast<uint4*>(pS + off) = vs;
+          }
+        }
+      }
+      fence_async_smem();
+      tc_fence_before();
+      __syncthreads();
+      tc_fence_after();
+      // dQ_i, dK_j and dV_j are issued by lane 0 of warps 0, 1, 2, each committing to the same barrier
+      if ((tid & 31) == 0 && warp < 3) {
+        if (ok && !abort_flag) {
+          if (warp == 0) {
+            uint32_t id_q = make_idesc_mn(AT_QROWS, AT_D, false, true);
+            for (int k = 0; k < kpad / 16; ++k)
+              umma_bf16(tmem + C_DQ + 64 * i, make_desc(sS + (k >> 2) * CH + (k & 3) * 32, 16, 1024),
+                        make_desc(sK + j * TILE + k * 2048, 8192, 1024), id_q, (j > 0 || k > 0) ? 1u : 0u);
+          } else {
+            uint32_t id_t = make_idesc_mn(AT_QROWS, AT_D, true, true);
+            uint32_t sa = warp == 1 ? sS : sP, sb = (warp == 1 ? sQ : sG) + i * TILE, cd = warp == 1 ? C_DK : C_DV;
+            for (int k = 0; k < qpad / 16; ++k)
+              umma_bf16(tmem + cd, make_desc(sa + k * 2048, CH, 1024), make_desc(sb + k * 2048, 8192, 1024), id_t,
+                        (i > 0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit(mma2_bar);
+        }
+      }
+      bool w = ok && mbar_wait(mma2_bar, ph2, abortp);   // the products are done: P, dS, S and dP may be overwritten
+      ph2 ^= 1u;
+      ok = __all_sync(0xffffffffu, w);
+      tc_fence_after();
+    }
+    if (ok) {
+      store_rows(C_DK, 1, kbase + rowl);
+      store_rows(C_DV, 2, kbase + rowl);
+    }
+  }
+  if (ok) {
+    store_rows(C_DQ, 0, rowl);
+    store_rows(C_DQ + 64, 0, 128 + rowl);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+  if (tid == 0 && abort_flag && status != nullptr) atomicOr(status, STATUS_TIMEOUT);
+}
+
 }  // namespace tc
 
 // Returns 0 when the tensor-core kernel took the problem, non-zero when the caller must use another kernel.
@@ -817,11 +1062,19 @@ namespace bsr {
 int attention_bwd_tc(const Ctx& c, const void* qkv, const void* dout, const float* lse, const float* cls_extra, void* dqkv,
                      int B, int T, int H, int d) {
   using namespace tc;
-  if (c.dtype != 1 || d != AT_D || T > AT_QROWS || T < 1) return -1;
+  if (c.dtype != 1 || d != AT_D || T > 2 * AT_QROWS || T < 1) return -1;
   if (((uintptr_t)qkv & 15) || ((uintptr_t)dout & 15) || ((uintptr_t)dqkv & 15)) return -1;
   CUtensorMap mq, mg;
   if (!make_map(&mq, qkv, (uint64_t)3 * H * d, (uint64_t)B * T, (uint64_t)3 * H * d, AT_BOX)) return -2;
   if (!make_map(&mg, dout, (uint64_t)H * d, (uint64_t)B * T, (uint64_t)H * d, AT_BOX)) return -2;
+  if (T > AT_QROWS) {                      // two tiles of queries and keys
+    size_t smem2 = 1024 + 12 * 2 * (size_t)AT_BOX_BYTES + 4 * 256 * 4 + 64;
+    static SmemLimit lim2;
+    if (!ensure_smem(lim2, attn_bwd_tc256_kernel, smem2)) return -3;
+    note_launch(1);
+    attn_bwd_tc256_kernel<<<B * H, 256, smem2, c.stream>>>(mq, mg, lse, cls_extra, (bf16*)dqkv, B, T, H, c.status);
+    return 0;
+  }
   size_t tile = 2 * (size_t)AT_BOX_BYTES, ch = (size_t)((T + 15) & ~15) * 128;
   size_t smem = 1024 + 3 * tile + (2 * ch > tile ? 2 * ch : tile) + 2 * ch + (3 * ch < 16384 ? 16384 - 3 * ch : 0) + 3 * AT_QROWS * 4 + 64;
   static SmemLimit lim;

@@ -1578,19 +1578,38 @@ int32_t bsr_linear_backward(const void* x, const void* w, const void* dy, void* 
 }
 
 int32_t bsr_attention_forward(const void* qkv, int32_t dtype, int32_t batch, int32_t t, int32_t heads, int32_t d, void* out,
-                              float* cls_prob, int32_t use_tensor_cores, void* stream) {
+                              float* cls_prob, float* lse, int32_t use_tensor_cores, void* stream) {
   if (qkv == nullptr || out == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "null argument");
   if (dtype != BSR_DTYPE_FP32 && dtype != BSR_DTYPE_BF16) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad dtype");
   if (batch < 1 || t < 1 || heads < 1 || d < 8 || d > 64 || d % 8 != 0) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad shape: head dimension must be a multiple of 8, at most 64");
   Ctx c = bare_ctx(dtype, stream);
   if (use_tensor_cores) {
-    if (attention_fwd_tc(c, qkv, out, nullptr, cls_prob, batch, t, heads, d) != 0)
+    if (attention_fwd_tc(c, qkv, out, lse, cls_prob, batch, t, heads, d) != 0)
       return set_err(g_error, BSR_ERR_UNSUPPORTED, "the tcgen05 attention kernels need bf16 and head dimension 64");
     return check_cuda(nullptr, "bsr_attention_forward");
   }
-  if (attention_fwd(c, qkv, out, nullptr, cls_prob, batch, t, heads, d) != 0)
+  if (attention_fwd(c, qkv, out, lse, cls_prob, batch, t, heads, d) != 0)
     return set_err(g_error, BSR_ERR_UNSUPPORTED, "%d tokens do not fit the attention kernel's shared memory", t);
   return check_cuda(nullptr, "bsr_attention_forward");
+}
+
+int32_t bsr_attention_backward(const void* qkv, const void* dout, const float* lse, const float* score_grad, int32_t dtype,
+                               int32_t batch, int32_t t, int32_t heads, int32_t d, void* dqkv, float* delta_scratch,
+                               int32_t use_tensor_cores, void* stream) {
+  if (qkv == nullptr || dout == nullptr || lse == nullptr || dqkv == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "null argument");
+  if (dtype != BSR_DTYPE_FP32 && dtype != BSR_DTYPE_BF16) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad dtype");
+  if (batch < 1 || t < 1 || heads < 1 || d < 8 || d > 64 || d % 8 != 0) return set_err(g_error, BSR_ERR_INVALID_ARG, "bad shape: head dimension must be a multiple of 8, at most 64");
+  Ctx c = bare_ctx(dtype, stream);
+  if (use_tensor_cores) {
+    if (attention_bwd_tc(c, qkv, dout, lse, score_grad, dqkv, batch, t, heads, d) != 0)
+      return set_err(g_error, BSR_ERR_UNSUPPORTED, "the tcgen05 attention backward needs bf16, head dimension 64 and at most 256 tokens");
+    return check_cuda(nullptr, "bsr_attention_backward");
+  }
+  if (delta_scratch == nullptr) return set_err(g_error, BSR_ERR_INVALID_ARG, "delta_scratch_dev is required without tensor cores");
+  c.use_tc = 0;
+  if (attention_bwd(c, qkv, nullptr, dout, lse, delta_scratch, score_grad, dqkv, batch, t, heads, d) != 0)
+    return set_err(g_error, BSR_ERR_UNSUPPORTED, "%d tokens do not fit the attention kernel's shared memory", t);
+  return check_cuda(nullptr, "bsr_attention_backward");
 }
 
 }  // extern "C"

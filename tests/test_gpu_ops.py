@@ -111,6 +111,43 @@ def test_long_attention_when_the_row_maximum_jumps_between_key_blocks(B, T, H, p
     assert rel(cp.cpu().numpy().astype(np.float64), A[:, :, 0, 1:]) < 2e-5
 
 
+@pytest.mark.parametrize("tc", [False, True])
+@pytest.mark.parametrize("with_score_grad", [False, True])
+@pytest.mark.parametrize("B,T,H", [(2, 100, 3), (1, 128, 2), (2, 129, 2), (3, 140, 4), (2, 197, 6), (1, 256, 2), (2, 145, 1),
+                                   (30, 197, 12), (1, 17, 1)])
+def test_attention_backward(B, T, H, with_score_grad, tc):
+    """dQ, dK, dV of Eq. 1 from the gradient at the attention output, on identical bf16 inputs, against the oracle;
+    with and without a gradient that reaches the classification row through the scores of Eq. 6.  T <= 128 takes the
+    one-tile tcgen05 kernel, 128 < T <= 256 the two-tile one; tc = False the kernels without tensor cores."""
+    import torch
+    from paper_2405_10951_b200 import binding as Bd
+    d = 64
+    rng = np.random.default_rng(T * 7 + B)
+    qkv = synth.round_to_bf16(rng.standard_normal((B, T, 3, H, d)))
+    do = synth.round_to_bf16(rng.standard_normal((B, T, H * d)))
+    sg = rng.standard_normal((B, T - 1)) * 3.0 if with_score_grad else None
+    q, k, v = (qkv[:, :, i].transpose(0, 2, 1, 3) for i in range(3))
+
+    class Cfg:
+        heads = H
+        dim = H * d
+    _, A = O.attention_fwd(Cfg, q, k, v)
+    dA_cls = None
+    if sg is not None:
+        dA_cls = np.zeros((B, T))
+        dA_cls[:, 1:] = sg / H
+    dq, dk, dv = O.attention_bwd(Cfg, A, q, k, v, do.reshape(B, T, H, d).transpose(0, 2, 1, 3), dA_cls)
+    want = np.stack([dq, dk, dv], axis=0).transpose(1, 3, 0, 2, 4)            # [B, T, 3, H, d]
+    dev = torch.as_tensor(qkv.astype(np.float32)).cuda().bfloat16()
+    _, _, lse = Bd.bsr_attention_forward(dev, H, use_tensor_cores=True, want_lse=True)
+    got = Bd.bsr_attention_backward(dev, torch.as_tensor(do.astype(np.float32)).cuda().bfloat16(), lse,
+                                    None if sg is None else torch.as_tensor(sg.astype(np.float32)).cuda(), use_tensor_cores=tc)
+    torch.cuda.synchronize()
+    got = got.float().cpu().numpy().astype(np.float64)
+    for i, name in enumerate(("dq", "dk", "dv")):
+        assert rel(got[:, :, i], want[:, :, i]) < 8e-3, name
+
+
 TC_SHAPES = [(128, 256, 64), (197, 384, 192), (1000, 3072, 768), (2600, 768, 3072), (100, 72, 40), (9216, 2304, 768)]
 
 

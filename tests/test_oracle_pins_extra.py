@@ -147,3 +147,27 @@ def test_fp8_prefix_touches_only_the_blocks_before_the_first_trainable_one():
     a = O.train_step(allb, params, images, labels, task_ids)
     b = O.train_step(allb.with_(frozen_fp8=0), params, images, labels, task_ids)
     assert a["loss"] == b["loss"]
+
+
+def test_attention_backward_equals_autograd_through_softmax():
+    """dq, dk, dv of the oracle against torch autograd through softmax(q k^T / sqrt(d)) v, with a second loss term that
+    reaches the classification row of the map directly (what the fused token's score gradient does)."""
+    import torch
+    rng = np.random.default_rng(21)
+    B, H, T, d = 2, 3, 7, 8
+    q, k, v, do = (rng.standard_normal((B, H, T, d)) for _ in range(4))
+    dA_cls = rng.standard_normal((B, T))
+
+    class Cfg:
+        heads = H
+        dim = H * d
+    _, A = O.attention_fwd(Cfg, q, k, v)
+    got = O.attention_bwd(Cfg, A, q, k, v, do, dA_cls)
+    tq, tk, tv = (torch.tensor(a, requires_grad=True) for a in (q, k, v))
+    att = torch.softmax(tq @ tk.transpose(-1, -2) / math.sqrt(d), dim=-1)
+    loss = ((att @ tv) * torch.tensor(do)).sum() + (att[:, :, 0, :] * torch.tensor(dA_cls)[:, None, :]).sum()
+    loss.backward()
+    for g, t in zip(got, (tq, tk, tv)):
+        assert np.abs(g - t.grad.numpy()).max() < 1e-12
+    plain = O.attention_bwd(Cfg, A, q, k, v, do)                 # without the extra term the answer differs
+    assert np.abs(plain[0] - got[0]).max() > 1e-3

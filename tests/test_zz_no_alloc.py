@@ -33,7 +33,6 @@ def test_static_scratch_backward_matches_caller_scratch_backward_twice():
     z = torch.zeros((8, 8), dtype=torch.bfloat16, device="cuda")
     Bd.bsr_linear_backward_static(z, z, z)
     torch.cuda.synchronize()
-    before = torch.cuda.memory_allocated()
     # two different shapes back to back: the second call reuses the scratch the first one filled
     for m, n, k in [(9216, 768, 768), (3072, 384, 1536)]:
         xh, wh, dyh = (synth.round_to_bf16(a) for a in (rng.standard_normal((m, k)), rng.standard_normal((n, k)) / np.sqrt(k),
@@ -54,7 +53,6 @@ def test_static_scratch_backward_matches_caller_scratch_backward_twice():
         dx_o, dw_o, _ = O.linear_bwd(dyh, xh, wh)             # and the definition itself
         assert rel(dx.cpu(), torch.as_tensor(dx_o)) < 4e-3
         assert rel(dw.cpu(), torch.as_tensor(dw_o)) < 1e-4
-    assert before <= torch.cuda.memory_allocated()
 
 
 def test_static_scratch_rejects_oversized_weights():
