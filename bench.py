@@ -63,10 +63,11 @@ def step_bytes(cfg, batch, fp):
     return float(images + fp["weight_bytes"] + 2 * fp["saved_activation_bytes"] + 30 * fp["trainable_params"])
 
 
-# DRAM traffic of the dominant kernel (tcgen05 GEMM), bytes per launch averaged over the launches of one step, from the
-# ncu capture summarised in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum).  None until the counters have
-# been taken on the kernel as it now stands.
-GEMM_DRAM_BYTES_PER_LAUNCH = {}
+# DRAM traffic of the dominant kernel (tcgen05 GEMM), bytes per launch averaged over the GEMM launches of one step
+# (dram__bytes_read.sum + dram__bytes_write.sum of every gemm_tc_kernel launch of the step, divided by their number),
+# from the one-pass ncu launch lists summarised in profiles/launch_list_<workload>_step.txt, taken at the batch sizes
+# bench.py runs.  Absent (null in the output) for a workload whose list has not been taken on the kernel as it stands.
+GEMM_DRAM_BYTES_PER_LAUNCH = {"vit_b": 82660169, "deit_s": 15886456, "vit_b_384": 39582905}
 
 
 def peaks():
