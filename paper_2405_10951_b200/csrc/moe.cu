@@ -107,19 +107,29 @@ moe_route_kernel(const T* __restrict__ y, const T* __restrict__ wg, const float*
     atomicAdd(&blk_counts[(size_t)(blockIdx.x * MOE_ROUTE_TOKENS / MOE_BLOCK_TOKENS) * E + threadIdx.x], counts[threadIdx.x]);
 }
 
-// ---- segment table: one warp per expert walks the token blocks in order ------------------------------------------
-__global__ void moe_scan_kernel(const int* __restrict__ blk_counts, int nblk, int E, int tiles_cap, int* __restrict__ blk_off,
-                                int* __restrict__ seg_start, int* __restrict__ tile_expert) {
+// ---- segment table and row assignment in one kernel ---------------------------------------------------------------
+// A block per group of MOE_BLOCK_TOKENS tokens.  Every block sums the per-group expert counts itself (a few KB): the
+// totals give the start of every expert's segment (padded to 128 rows), the counts of the groups before its own give
+// its place inside each segment.  Then the position of every (token, slot) inside its expert's segment, in token order.
+// Block 0 also publishes the segment starts and the expert of every 128-row tile for the grouped GEMMs.
+__global__ void __launch_bounds__(256)
+moe_assign_kernel(const int* __restrict__ eidx, const float* __restrict__ ew, const int* __restrict__ blk_counts, int nblk,
+                  int tiles_cap, int M, int E, int K, int* __restrict__ seg_start, int* __restrict__ tile_expert,
+                  int* __restrict__ pos, int* __restrict__ row_token, float* __restrict__ row_w) {
   __shared__ int total[MOE_MAX_E];
+  __shared__ int before[MOE_MAX_E];
   __shared__ int start[MOE_MAX_E + 1];
-  int e = threadIdx.x;
-  if (e < E) {
-    int run = 0;
-    for (int b = 0; b < nblk; ++b) {
-      blk_off[(size_t)b * E + e] = run;
-      run += blk_counts[(size_t)b * E + e];
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int e = warp; e < E; e += 8) {
+    int all = 0, pre = 0;
+    for (int g = lane; g < nblk; g += 32) {
+      int cnt = blk_counts[(size_t)g * E + e];
+      all += cnt;
+      if (g < (int)blockIdx.x) pre += cnt;
     }
-    total[e] = run;
+    all = warp_sum_int(all);
+    pre = warp_sum_int(pre);
+    if (lane == 0) { total[e] = all; before[e] = pre; }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -129,28 +139,22 @@ __global__ void moe_scan_kernel(const int* __restrict__ blk_counts, int nblk, in
       s += (total[i] + 127) & ~127;
     }
     start[E] = s;
-    for (int i = 0; i <= E; ++i) seg_start[i] = start[i];
   }
   __syncthreads();
-  for (int t = threadIdx.x; t < tiles_cap; t += blockDim.x) {
-    int row = t * 128, ex = -1;
-    for (int i = 0; i < E; ++i)
-      if (row >= start[i] && row < start[i + 1]) ex = i;
-    tile_expert[t] = ex;
+  if (blockIdx.x == 0) {
+    for (int i = threadIdx.x; i <= E; i += blockDim.x) seg_start[i] = start[i];
+    for (int t = threadIdx.x; t < tiles_cap; t += blockDim.x) {
+      int row = t * 128, ex = -1;
+      for (int i = 0; i < E; ++i)
+        if (row >= start[i] && row < start[i + 1]) ex = i;
+      tile_expert[t] = ex;
+    }
   }
-}
-
-// ---- row assignment: position of every (token, slot) inside its expert's segment, in token order ---------------
-__global__ void __launch_bounds__(256)
-moe_assign_kernel(const int* __restrict__ eidx, const float* __restrict__ ew, const int* __restrict__ blk_off,
-                  const int* __restrict__ seg_start, int M, int E, int K, int* __restrict__ pos, int* __restrict__ row_token,
-                  float* __restrict__ row_w) {
-  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int t0 = blockIdx.x * MOE_BLOCK_TOKENS;
   int n_entries = min(MOE_BLOCK_TOKENS, M - t0) * K;
   uint32_t lt = (1u << lane) - 1u;
   for (int e = warp; e < E; e += 8) {
-    int base = seg_start[e] + blk_off[(size_t)blockIdx.x * E + e];
+    int base = start[e] + before[e];
     int run = 0;
     for (int i0 = 0; i0 < n_entries; i0 += 32) {
       int i = i0 + lane;
@@ -350,7 +354,7 @@ void moe_route(const Ctx& c, const MoeBufs& b, const void* y, const void* wg, co
                int D, int E, int K, int num_tasks, const float* logits, int logit_stride) {
   int nblk = moe_blocks(M);
   int rows_cap = moe_rows_cap(M, E, K);
-  note_launch(4);
+  note_launch(3);
   size_t es = c.dtype == 0 ? 4 : 2;
   size_t gate_elems = (size_t)(num_tasks < 1 ? 1 : num_tasks) * E * D;
   size_t smem = gate_elems * es;
@@ -367,9 +371,9 @@ void moe_route(const Ctx& c, const MoeBufs& b, const void* y, const void* wg, co
     moe_route_kernel<bf16><<<rblk, MOE_ROUTE_WARPS * 32, smem, c.stream>>>((const bf16*)y, (const bf16*)wg, logits, logit_stride, task_ids, tokens_per_image, M, D, E, K,
                                                                        (int)gate_elems, b.eidx, b.ew, b.blk_counts);
   }
-  moe_scan_kernel<<<1, 128, 0, c.stream>>>(b.blk_counts, nblk, E, rows_cap / 128, b.blk_off, b.seg_start, b.tile_expert);
   cudaMemsetAsync(b.row_token, 0xFF, (size_t)rows_cap * sizeof(int), c.stream);
-  moe_assign_kernel<<<nblk, 256, 0, c.stream>>>(b.eidx, b.ew, b.blk_off, b.seg_start, M, E, K, b.pos, b.row_token, b.row_w);
+  moe_assign_kernel<<<nblk, 256, 0, c.stream>>>(b.eidx, b.ew, b.blk_counts, nblk, rows_cap / 128, M, E, K, b.seg_start, b.tile_expert,
+                                                b.pos, b.row_token, b.row_w);
   int blocks = ceil_div((long)rows_cap * 32, 256);
   if (c.dtype == 0) moe_gather_kernel<float><<<blocks, 256, 0, c.stream>>>((const float*)y, b.row_token, b.seg_start, E, D, (float*)b.xg, rows_cap, M, c.status);
   else moe_gather_kernel<bf16><<<blocks, 256, 0, c.stream>>>((const bf16*)y, b.row_token, b.seg_start, E, D, (bf16*)b.xg, rows_cap, M, c.status);
