@@ -770,7 +770,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_con
 // ------------------------------------------------------------------------------------------------
 // Backward for 128 < T <= 256: one CTA of 256 threads per (image, head), queries and keys in two tiles of 128.
 // The formulas are those of the kernel above; what changes is that delta_i = sum_j P_ij dP_ij runs over both key
-// tiles, so a first sweep over the four (query tile, key tile) pairs forms S and dP only to accumulate delta, and a
+// tiles, so a first sweep (one step per query tile, both key tiles at once) forms S and dP only to accumulate delta, and a
 // second sweep (key tile outer, query tile inner) forms them again, writes P and dS as bf16 operand tiles and issues
 // the three products: dQ_i accumulates over the key tiles, dK_j and dV_j over the query tiles, all in tensor memory
 // (S 128 + dP 128 + dQ 2 x 64 + dK 64 + dV 64 = 512 columns: one CTA per SM).  No step leaves the loop early: after a
@@ -861,6 +861,34 @@ attn_bwd_tc256_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_
     tc_fence_after();
   };
 
+  // S and dP of query tile i against BOTH key tiles at once: the second pair lands in the columns that hold dQ, dK, dV
+  // later (free during the first sweep), so the sweep takes one product group and one wait per query tile
+  auto scores_both = [&](int i) {
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (tid == 0 && ok && !abort_flag) {
+      uint32_t q = sQ + i * TILE, g = sG + i * TILE;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        int kpad = min(128, tpad - 128 * j);
+        uint32_t idesc = make_idesc_mn(AT_QROWS, kpad, false, false);
+        uint32_t k_ = sK + j * TILE, v = sV + j * TILE;
+#pragma unroll
+        for (int k = 0; k < AT_D / 16; ++k)
+          umma_bf16(tmem + 256 * j + C_S, make_desc(q + k * 32, 16, 1024), make_desc(k_ + k * 32, 16, 1024), idesc, k > 0 ? 1u : 0u);
+#pragma unroll
+        for (int k = 0; k < AT_D / 16; ++k)
+          umma_bf16(tmem + 256 * j + C_DP, make_desc(g + k * 32, 16, 1024), make_desc(v + k * 32, 16, 1024), idesc, k > 0 ? 1u : 0u);
+      }
+      umma_commit(mma_bar);
+    }
+    bool w = mbar_wait(mma_bar, ph1, abortp);
+    ph1 ^= 1u;
+    ok = __all_sync(0xffffffffu, ok && w);
+    tc_fence_after();
+  };
+
   // ---- first sweep: delta of every query row ----
   for (int i = 0; i < 2; ++i) {
     const int row = i * 128 + rowl;
@@ -868,15 +896,15 @@ attn_bwd_tc256_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_
     const bool extra_row = (row == 0 && has_extra);
     const float l2 = sl2[row];
     float dacc = 0.f;
+    scores_both(i);
     for (int j = 0; j < 2; ++j) {
-      scores(i, j);
       const int kbase = j * 128;
       const int kvalid = min(128, T - kbase);
       if (ok) {
         for (int kk = 4 * half; kk < 4 * half + 4 && kk * 16 < kvalid; ++kk) {
           uint32_t rs[16], rp[16];
-          tmem_ld16(trow + C_S + kk * 16, rs);
-          tmem_ld16(trow + C_DP + kk * 16, rp);
+          tmem_ld16(trow + 256 * j + C_S + kk * 16, rs);
+          tmem_ld16(trow + 256 * j + C_DP + kk * 16, rp);
           tmem_ld_wait();
           if (valid_row) {
             float d0 = 0.f, d1 = 0.f;
